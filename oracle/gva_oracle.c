@@ -1,0 +1,243 @@
+/*
+ * fp64 CPU oracle for one decode step of Grouped Value Attention with decoupled RoPE.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the plain definition the CUDA library is checked
+ * against.  It is deliberately slow and unblocked: two-pass softmax, no tiling, no split-KV, pages
+ * resolved by direct indexing.  It shares no code, header, table or constant with the CUDA path and
+ * must never be called from it.  Only tests, the smoke check and the benchmark's CPU-baseline leg
+ * may load it.
+ *
+ * Notation follows the paper (row vectors).  d_v = value width (paper d_h), d_c = content-key
+ * width (paper d_n), d_r = RoPE width, g(h) = h / (H/G).
+ *
+ *   rope      : x R_p^T with R_p block-diagonal 2x2 rotations, angle p * base^(-2i/d_r)
+ *               (Section 3.3, Eq. krope; the pairing/frequency convention is this build's reading)
+ *   absorb    : q~_h = q_h^nope M_h^T                     (Section 3.2, Eq. absorb; Algorithm 1)
+ *   append    : V_{1:t,g} <- [V_{1:t-1,g}; v_{t,g}],  k^rope_t = (.)R_t^T appended   (Algorithm 1)
+ *   decode    : s_j = q~_h v_{j,g(h)}^T + q^rope_h (k^rope_j)^T ;  o_h = softmax(s/sqrt(d_qk)) V_{g(h)}
+ *               with d_qk = d_c + d_r                     (Section 3.3 score equation; Algorithm 1)
+ *   gqa       : matched GQA decode over cached K and V    (Section 2, GQA; Section 3.4)
+ *
+ * All arithmetic is double precision.  Cache pools are read in their storage type (bf16 bit
+ * patterns or float32) and widened exactly.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_F32 0
+#define ORACLE_BF16 1
+
+/* ---- storage <-> double ---------------------------------------------------------------------- */
+static double load_elem(const void *pool, int dtype, int64_t idx) {
+    if (dtype == ORACLE_BF16) {
+        uint32_t u = ((uint32_t)((const uint16_t *)pool)[idx]) << 16;
+        float f;
+        memcpy(&f, &u, 4);
+        return (double)f;
+    }
+    return (double)((const float *)pool)[idx];
+}
+
+/* Round a double to bfloat16, nearest with ties to even, straight from the fp64 value (no
+ * intermediate float rounding).  Works on the value, not on bit tricks shared with anyone:
+ * scale into [2^7, 2^8) so that the 8 significant bits of bf16 are the integer part, round the
+ * integer with nearbyint (default rounding mode = ties-to-even), scale back (exact). */
+uint16_t oracle_bf16_from_double(double x) {
+    if (x != x) return 0x7FC0;
+    uint16_t sign = signbit(x) ? 0x8000 : 0;
+    double a = fabs(x);
+    if (a == 0.0) return sign;
+    if (isinf(a)) return (uint16_t)(sign | 0x7F80);
+    int e;
+    (void)frexp(a, &e);        /* a = m * 2^e, m in [0.5, 1)  => a in [2^(e-1), 2^e) */
+    int exp_unb = e - 1;        /* floor(log2 a) */
+    if (exp_unb < -126) exp_unb = -126;   /* subnormal bf16: fixed quantum 2^-133 */
+    double q = ldexp(a, 7 - exp_unb);     /* in [128, 256) for normals */
+    double r = nearbyint(q);              /* ties-to-even */
+    double y = ldexp(r, exp_unb - 7);     /* exact */
+    if (y >= ldexp(1.0, 128)) return (uint16_t)(sign | 0x7F80); /* rounded past the largest finite bf16 */
+    float f = (float)y;                   /* exact: y has at most 8 significant bits */
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    return (uint16_t)(sign | (uint16_t)(u >> 16));
+}
+
+static void store_elem(void *pool, int dtype, int64_t idx, double x) {
+    if (dtype == ORACLE_BF16)
+        ((uint16_t *)pool)[idx] = oracle_bf16_from_double(x);
+    else
+        ((float *)pool)[idx] = (float)x;  /* IEEE nearest-even conversion */
+}
+
+/* ---- RoPE: y = x R_p^T, pairs (2i, 2i+1), theta_i = base^(-2i/d_r) ---------------------------- */
+void oracle_rope(const double *x, int d_r, double pos, double base, double *y) {
+    for (int i = 0; i < d_r / 2; ++i) {
+        double theta = pow(base, -2.0 * (double)i / (double)d_r);
+        double a = pos * theta;
+        double c = cos(a), s = sin(a);
+        double x0 = x[2 * i], x1 = x[2 * i + 1];
+        y[2 * i] = x0 * c - x1 * s;
+        y[2 * i + 1] = x0 * s + x1 * c;
+    }
+}
+
+/* ---- absorb: q_abs[b,h,0:d_v] = q_c[b,h,:] M_h^T ; q_abs[b,h,d_v:] = rope(q_r[b,h,:], q_pos[b]) --
+ * M is [H][d_v][d_c] row-major (M_h in R^{d_h x d_n}), so (q M_h^T)[i] = sum_j q[j] M_h[i][j].   */
+void oracle_absorb(const double *q_c, const double *q_r, const double *M, const int32_t *q_pos,
+                   int B, int H, int d_v, int d_c, int d_r, double base, double *q_abs) {
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            double *dst = q_abs + ((int64_t)b * H + h) * (d_v + d_r);
+            const double *q = q_c + ((int64_t)b * H + h) * d_c;
+            const double *Mh = M + (int64_t)h * d_v * d_c;
+            for (int i = 0; i < d_v; ++i) {
+                double acc = 0.0;
+                for (int j = 0; j < d_c; ++j) acc += q[j] * Mh[(int64_t)i * d_c + j];
+                dst[i] = acc;
+            }
+            oracle_rope(q_r + ((int64_t)b * H + h) * d_r, d_r, (double)q_pos[b], base, dst + d_v);
+        }
+}
+
+/* physical page of logical page j of sequence b; block_table == NULL means contiguous */
+static int64_t page_of(const int32_t *block_table, int max_pages, int b, int j) {
+    return block_table ? (int64_t)block_table[(int64_t)b * max_pages + j] : (int64_t)b * max_pages + j;
+}
+
+/* ---- append: write the new token's G value rows and its rotated positional key -----------------
+ * v_pool [num_pages][G][P][d_v], kr_pool [num_pages][P][d_r].  v_new [B][G][d_v], kr_new [B][d_r]
+ * (unrotated), pos [B].  Returns 0, or 1+b for the first sequence whose page id is out of range. */
+int oracle_append(void *v_pool, void *kr_pool, int dtype, const int32_t *block_table, int num_pages,
+                  int max_pages, int P, int G, int d_v, int d_r, double base, const double *v_new,
+                  const double *kr_new, const int32_t *pos, int B) {
+    double *rot = (double *)malloc(sizeof(double) * (size_t)d_r);
+    int rc = 0;
+    for (int b = 0; b < B && !rc; ++b) {
+        int t = pos[b];
+        int64_t page = page_of(block_table, max_pages, b, t / P);
+        int slot = t % P;
+        if (t < 0 || t / P >= max_pages || page < 0 || page >= num_pages) { rc = 1 + b; break; }
+        for (int g = 0; g < G; ++g)
+            for (int i = 0; i < d_v; ++i)
+                store_elem(v_pool, dtype, ((page * G + g) * P + slot) * d_v + i,
+                           v_new[((int64_t)b * G + g) * d_v + i]);
+        oracle_rope(kr_new + (int64_t)b * d_r, d_r, (double)t, base, rot);
+        for (int k = 0; k < d_r; ++k) store_elem(kr_pool, dtype, (page * P + slot) * d_r + k, rot[k]);
+    }
+    free(rot);
+    return rc;
+}
+
+/* ---- decode: plain two-pass softmax attention over the paged GVA cache ---------------------------
+ * q_abs [B][H][d_v+d_r] (absorbed content query, then rotated positional query), out [B][H][d_v],
+ * lse [B][H] = log sum_j exp(scale * s_j).  seq_len == 0 gives out = 0, lse = -inf.            */
+void oracle_decode(const void *v_pool, const void *kr_pool, int dtype, const int32_t *block_table,
+                   int max_pages, int P, const int32_t *seq_lens, const double *q_abs, double scale,
+                   int B, int H, int G, int d_v, int d_r, double *out, double *lse) {
+    int hpg = H / G;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            int g = h / hpg;
+            int T = seq_lens[b];
+            const double *q = q_abs + ((int64_t)b * H + h) * (d_v + d_r);
+            double *o = out + ((int64_t)b * H + h) * d_v;
+            for (int i = 0; i < d_v; ++i) o[i] = 0.0;
+            if (T <= 0) { if (lse) lse[(int64_t)b * H + h] = -INFINITY; continue; }
+            double *s = (double *)malloc(sizeof(double) * (size_t)T);
+            double m = -INFINITY;
+            for (int t = 0; t < T; ++t) {
+                int64_t page = page_of(block_table, max_pages, b, t / P);
+                int slot = t % P;
+                int64_t vrow = ((page * G + g) * P + slot) * d_v;
+                int64_t krow = (page * P + slot) * d_r;
+                double acc = 0.0;
+                for (int i = 0; i < d_v; ++i) acc += q[i] * load_elem(v_pool, dtype, vrow + i);
+                for (int k = 0; k < d_r; ++k) acc += q[d_v + k] * load_elem(kr_pool, dtype, krow + k);
+                s[t] = acc * scale;
+                if (s[t] > m) m = s[t];
+            }
+            double L = 0.0;
+            for (int t = 0; t < T; ++t) { s[t] = exp(s[t] - m); L += s[t]; }
+            for (int t = 0; t < T; ++t) {
+                int64_t page = page_of(block_table, max_pages, b, t / P);
+                int slot = t % P;
+                int64_t vrow = ((page * G + g) * P + slot) * d_v;
+                double p = s[t] / L;
+                for (int i = 0; i < d_v; ++i) o[i] += p * load_elem(v_pool, dtype, vrow + i);
+            }
+            if (lse) lse[(int64_t)b * H + h] = m + log(L);
+            free(s);
+        }
+}
+
+/* ---- softmax weights of one (b, h) row, for invariant checks (sum to one, flat case) ------------- */
+void oracle_decode_weights(const void *v_pool, const void *kr_pool, int dtype, const int32_t *block_table,
+                           int max_pages, int P, const int32_t *seq_lens, const double *q_abs, double scale,
+                           int H, int G, int d_v, int d_r, int b, int h, double *p) {
+    int g = h / (H / G);
+    int T = seq_lens[b];
+    const double *q = q_abs + ((int64_t)b * H + h) * (d_v + d_r);
+    double m = -INFINITY;
+    for (int t = 0; t < T; ++t) {
+        int64_t page = page_of(block_table, max_pages, b, t / P);
+        int slot = t % P;
+        double acc = 0.0;
+        for (int i = 0; i < d_v; ++i) acc += q[i] * load_elem(v_pool, dtype, ((page * G + g) * P + slot) * d_v + i);
+        for (int k = 0; k < d_r; ++k) acc += q[d_v + k] * load_elem(kr_pool, dtype, (page * P + slot) * d_r + k);
+        p[t] = acc * scale;
+        if (p[t] > m) m = p[t];
+    }
+    double L = 0.0;
+    for (int t = 0; t < T; ++t) { p[t] = exp(p[t] - m); L += p[t]; }
+    for (int t = 0; t < T; ++t) p[t] /= L;
+}
+
+/* ---- matched GQA decode: s_j = q_h K_{j,g(h)}^T / sqrt(d_h), o_h = softmax(s) V_{g(h)} -----------
+ * k_pool, v_pool [num_pages][G][P][d_h]; q [B][H][d_h] already rotated; K cached already rotated. */
+void oracle_gqa_decode(const void *k_pool, const void *v_pool, int dtype, const int32_t *block_table,
+                       int max_pages, int P, const int32_t *seq_lens, const double *q, double scale,
+                       int B, int H, int G, int d_h, double *out, double *lse) {
+    int hpg = H / G;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            int g = h / hpg;
+            int T = seq_lens[b];
+            const double *qq = q + ((int64_t)b * H + h) * d_h;
+            double *o = out + ((int64_t)b * H + h) * d_h;
+            for (int i = 0; i < d_h; ++i) o[i] = 0.0;
+            if (T <= 0) { if (lse) lse[(int64_t)b * H + h] = -INFINITY; continue; }
+            double *s = (double *)malloc(sizeof(double) * (size_t)T);
+            double m = -INFINITY;
+            for (int t = 0; t < T; ++t) {
+                int64_t page = page_of(block_table, max_pages, b, t / P);
+                int64_t row = ((page * G + g) * P + (t % P)) * d_h;
+                double acc = 0.0;
+                for (int i = 0; i < d_h; ++i) acc += qq[i] * load_elem(k_pool, dtype, row + i);
+                s[t] = acc * scale;
+                if (s[t] > m) m = s[t];
+            }
+            double L = 0.0;
+            for (int t = 0; t < T; ++t) { s[t] = exp(s[t] - m); L += s[t]; }
+            for (int t = 0; t < T; ++t) {
+                int64_t page = page_of(block_table, max_pages, b, t / P);
+                int64_t row = ((page * G + g) * P + (t % P)) * d_h;
+                double p = s[t] / L;
+                for (int i = 0; i < d_h; ++i) o[i] += p * load_elem(v_pool, dtype, row + i);
+            }
+            if (lse) lse[(int64_t)b * H + h] = m + log(L);
+            free(s);
+        }
+}
+
+#ifdef _OPENMP
+#include <omp.h>
+int oracle_num_threads(void) { return omp_get_max_threads(); }
+void oracle_set_threads(int n) { omp_set_num_threads(n); }
+#else
+int oracle_num_threads(void) { return 1; }
+void oracle_set_threads(int n) { (void)n; }
+#endif

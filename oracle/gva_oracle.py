@@ -1,0 +1,191 @@
+"""ctypes front end of the fp64 CPU oracle (oracle/gva_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: imported by tests, the smoke check and the benchmark's CPU-baseline
+leg.  The CUDA library never imports or links it, and it never imports the CUDA package.
+
+All functions take and return numpy arrays.  Cache pools are passed in storage dtype
+(uint16 = bfloat16 bit patterns, or float32); everything else is float64.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gva_oracle.c")
+_LIB = os.path.join(_HERE, "libgva_oracle.so")
+_lib = None
+
+F32, BF16 = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP over (batch, head)); returns the .so path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared", _SRC, "-o", _LIB, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_bf16_from_double.restype = ctypes.c_uint16
+        _lib.oracle_bf16_from_double.argtypes = [ctypes.c_double]
+        _lib.oracle_num_threads.restype = ctypes.c_int
+        _lib.oracle_append.restype = ctypes.c_int
+    return _lib
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _dt(pool: np.ndarray) -> int:
+    if pool.dtype == np.uint16:
+        return BF16
+    if pool.dtype == np.float32:
+        return F32
+    raise TypeError("cache pools must be uint16 (bf16 bits) or float32")
+
+
+def _f64(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def set_threads(n: int) -> None:
+    lib().oracle_set_threads(ctypes.c_int(int(n)))
+
+
+def bf16_from_double(x: float) -> int:
+    return int(lib().oracle_bf16_from_double(ctypes.c_double(float(x))))
+
+
+def rope(x, pos: float, base: float = 10000.0) -> np.ndarray:
+    """y = x R_pos^T on the last axis (pairs (2i, 2i+1))."""
+    x = _f64(x)
+    y = np.empty_like(x)
+    d_r = x.shape[-1]
+    xf, yf = x.reshape(-1, d_r), y.reshape(-1, d_r)
+    for r in range(xf.shape[0]):
+        lib().oracle_rope(_p(xf[r]), ctypes.c_int(d_r), ctypes.c_double(float(pos)), ctypes.c_double(base), _p(yf[r]))
+    return y
+
+
+def absorb(q_c, q_r, M, q_pos, base: float = 10000.0) -> np.ndarray:
+    """q_abs [B,H,d_v+d_r]: absorbed content query q_c M_h^T, then q_r rotated at q_pos[b]."""
+    q_c, q_r, M, q_pos = _f64(q_c), _f64(q_r), _f64(M), _i32(q_pos)
+    B, H, d_c = q_c.shape
+    d_r = q_r.shape[-1]
+    d_v = M.shape[1]
+    assert M.shape == (H, d_v, d_c)
+    out = np.empty((B, H, d_v + d_r), dtype=np.float64)
+    lib().oracle_absorb(_p(q_c), _p(q_r), _p(M), _p(q_pos), *map(ctypes.c_int, (B, H, d_v, d_c, d_r)),
+                        ctypes.c_double(base), _p(out))
+    return out
+
+
+def append(v_pool, kr_pool, block_table, v_new, kr_new, pos, base: float = 10000.0,
+           max_pages_per_seq: Optional[int] = None) -> int:
+    """In-place cache append (Algorithm 1's append lines).  Returns 0 or 1+b of the first bad page."""
+    dt = _dt(v_pool)
+    assert v_pool.flags.c_contiguous and kr_pool.flags.c_contiguous and _dt(kr_pool) == dt
+    num_pages, G, P, d_v = v_pool.shape
+    d_r = kr_pool.shape[-1]
+    v_new, kr_new, pos = _f64(v_new), _f64(kr_new), _i32(pos)
+    B = pos.shape[0]
+    bt = None if block_table is None else _i32(block_table)
+    max_pages = bt.shape[1] if bt is not None else int(max_pages_per_seq)
+    return int(lib().oracle_append(_p(v_pool), _p(kr_pool), ctypes.c_int(dt), _p(bt), ctypes.c_int(num_pages),
+                                   ctypes.c_int(max_pages), ctypes.c_int(P), ctypes.c_int(G), ctypes.c_int(d_v),
+                                   ctypes.c_int(d_r), ctypes.c_double(base), _p(v_new), _p(kr_new), _p(pos),
+                                   ctypes.c_int(B)))
+
+
+def decode(v_pool, kr_pool, block_table, seq_lens, q_abs, H: int, scale: Optional[float] = None,
+           d_c: Optional[int] = None, max_pages_per_seq: Optional[int] = None):
+    """(out [B,H,d_v], lse [B,H]) by the plain definition.  scale defaults to 1/sqrt(d_c+d_r)."""
+    dt = _dt(v_pool)
+    assert v_pool.flags.c_contiguous and kr_pool.flags.c_contiguous and _dt(kr_pool) == dt
+    _, G, P, d_v = v_pool.shape
+    d_r = kr_pool.shape[-1]
+    q_abs, seq_lens = _f64(q_abs), _i32(seq_lens)
+    B = seq_lens.shape[0]
+    assert q_abs.shape == (B, H, d_v + d_r)
+    if scale is None:
+        scale = 1.0 / np.sqrt(float((d_v if d_c is None else d_c) + d_r))
+    bt = None if block_table is None else _i32(block_table)
+    max_pages = bt.shape[1] if bt is not None else int(max_pages_per_seq)
+    out = np.empty((B, H, d_v), dtype=np.float64)
+    lse = np.empty((B, H), dtype=np.float64)
+    lib().oracle_decode(_p(v_pool), _p(kr_pool), ctypes.c_int(dt), _p(bt), ctypes.c_int(max_pages), ctypes.c_int(P),
+                        _p(seq_lens), _p(q_abs), ctypes.c_double(scale), *map(ctypes.c_int, (B, H, G, d_v, d_r)),
+                        _p(out), _p(lse))
+    return out, lse
+
+
+def decode_weights(v_pool, kr_pool, block_table, seq_lens, q_abs, H: int, b: int, h: int, scale: float,
+                   max_pages_per_seq: Optional[int] = None) -> np.ndarray:
+    """Softmax weights p_t of one (b, h) row."""
+    dt = _dt(v_pool)
+    _, G, P, d_v = v_pool.shape
+    d_r = kr_pool.shape[-1]
+    q_abs, seq_lens = _f64(q_abs), _i32(seq_lens)
+    bt = None if block_table is None else _i32(block_table)
+    max_pages = bt.shape[1] if bt is not None else int(max_pages_per_seq)
+    p = np.empty(int(seq_lens[b]), dtype=np.float64)
+    lib().oracle_decode_weights(_p(v_pool), _p(kr_pool), ctypes.c_int(dt), _p(bt), ctypes.c_int(max_pages),
+                                ctypes.c_int(P), _p(seq_lens), _p(q_abs), ctypes.c_double(scale),
+                                *map(ctypes.c_int, (H, G, d_v, d_r, b, h)), _p(p))
+    return p
+
+
+def gqa_decode(k_pool, v_pool, block_table, seq_lens, q, scale: Optional[float] = None,
+               max_pages_per_seq: Optional[int] = None):
+    """Matched GQA decode: (out [B,H,d_h], lse [B,H]); scale defaults to 1/sqrt(d_h)."""
+    dt = _dt(v_pool)
+    assert _dt(k_pool) == dt and k_pool.shape == v_pool.shape
+    _, G, P, d_h = v_pool.shape
+    q, seq_lens = _f64(q), _i32(seq_lens)
+    B, H, _ = q.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d_h))
+    bt = None if block_table is None else _i32(block_table)
+    max_pages = bt.shape[1] if bt is not None else int(max_pages_per_seq)
+    out = np.empty((B, H, d_h), dtype=np.float64)
+    lse = np.empty((B, H), dtype=np.float64)
+    lib().oracle_gqa_decode(_p(k_pool), _p(v_pool), ctypes.c_int(dt), _p(bt), ctypes.c_int(max_pages), ctypes.c_int(P),
+                            _p(seq_lens), _p(q), ctypes.c_double(scale), *map(ctypes.c_int, (B, H, G, d_h)),
+                            _p(out), _p(lse))
+    return out, lse
+
+
+# ---- convenience over a workloads.DecodeCase-like object (duck-typed; no import of the generator) ----
+def absorb_case(case) -> np.ndarray:
+    return absorb(case.q_c, case.q_r, case.M, case.q_pos, case.rope_base)
+
+
+def decode_case(case, q_abs=None, seq_lens=None):
+    if q_abs is None:
+        q_abs = absorb_case(case)
+    s = case.shape
+    return decode(case.v_pool, case.kr_pool, case.block_table, case.seq_lens if seq_lens is None else seq_lens,
+                  q_abs, s.H, scale=1.0 / np.sqrt(float(s.d_c + s.d_r)), max_pages_per_seq=case.max_pages_per_seq)
+
+
+def append_case(case) -> int:
+    return append(case.v_pool, case.kr_pool, case.block_table, case.v_new, case.kr_new, case.append_pos,
+                  case.rope_base, max_pages_per_seq=case.max_pages_per_seq)
