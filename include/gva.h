@@ -1,0 +1,185 @@
+/*
+ * gva.h -- C ABI of the B200 (sm_100a) Grouped Value Attention decode library.
+ *
+ * One decode step of GVA with decoupled RoPE (Algorithm 1 of the paper) is three calls:
+ *
+ *   gva_absorb_query   q~_h = q^nope_h M_h^T  and  q^rope_h <- q^rope_h R_t^T      (Eq. absorb; Alg. 1)
+ *   gva_append_cache   V_{1:t,g} <- [V_{1:t-1,g}; v_{t,g}],  k^rope_t = (.) R_t^T  (Eq. krope;  Alg. 1)
+ *   gva_decode         s_j = q~_h v_{j,g(h)}^T + q^rope_h (k^rope_j)^T,
+ *                      o_h = softmax(s / sqrt(d_qk)) V_{1:t,g(h)},  d_qk = d_c + d_r   (Section 3.3; Alg. 1)
+ *
+ * plus gqa_decode, a matched GQA decode over cached K and V (Section 2 / Section 3.4), built the
+ * same way, as the reference point for the cache-bytes comparison N_GVA/N_GQA = 1/2 + d_r/(2 G d_h).
+ *
+ * Names: d_v = value width (paper d_h), d_c = content-key width (paper d_n), d_r = RoPE width,
+ * H query heads, G value groups, head h reads group g(h) = h / (H/G).
+ *
+ * Conventions
+ *   - All pointers are DEVICE pointers unless a parameter is marked [host].  The library allocates
+ *     no device memory, keeps no caller pointer after a call returns, and never synchronises: every
+ *     call enqueues work on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *   - Return value: a gva_status detected on the host before/at launch.  Conditions only the device
+ *     can see (a page id outside [0, num_pages), a sequence longer than its block table) are
+ *     recorded once in *dev_status (caller-zeroed int32 on the device; may be NULL) as
+ *     code | (sequence_index << 8); the offending work is skipped and the kernel ends normally.
+ *   - RoPE: pairs (2i, 2i+1) of the d_r-wide slice are rotated by the angle pos * base^(-2i/d_r)
+ *     (y[2i] = x[2i] cos a - x[2i+1] sin a, y[2i+1] = x[2i] sin a + x[2i+1] cos a), evaluated in fp64.
+ *   - Cache layout ("pools"): v_pool [num_pages][G][page_size][d_v], kr_pool [num_pages][page_size][d_r],
+ *     element type = cfg.cache_dtype.  Logical page j of sequence b is block_table[b*max_pages_per_seq + j];
+ *     block_table == NULL means contiguous: page j of sequence b is b*max_pages_per_seq + j.
+ *     Slots at or beyond seq_lens[b] and block-table entries beyond ceil(seq_lens[b]/page_size) are never
+ *     read by gva_decode (they may hold NaN / -1).
+ */
+#ifndef GVA_H_
+#define GVA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GVA_OK = 0,
+    GVA_ERR_INVALID_ARG = 1,  /* null pointer, negative size, misaligned pointer                         */
+    GVA_ERR_UNSUPPORTED = 2,  /* shape / dtype / page size outside the instantiated kernels              */
+    GVA_ERR_WORKSPACE = 3,    /* workspace smaller than gva_decode_workspace_bytes()                     */
+    GVA_ERR_CUDA = 4,         /* a CUDA runtime/driver call failed (launch error, no sm_100 device, ...) */
+    GVA_ERR_BAD_PAGE = 5,     /* [device] block-table entry outside [0, num_pages) in the live range     */
+    GVA_ERR_SEQ_LEN = 6,      /* [device] seq_len < 0 or beyond max_pages_per_seq * page_size            */
+    GVA_ERR_TIMEOUT = 7       /* [device] a bounded wait on an asynchronous copy expired                 */
+} gva_status;
+
+typedef enum { GVA_F32 = 0, GVA_BF16 = 1 } gva_dtype;
+
+/* Which decode kernel gva_decode launches.  AUTO = tensor-core kernel when the cache is bf16,
+ * CUDA-core (FMA) kernel for an f32 cache.  FMA / MMA force one (MMA with an f32 cache is
+ * GVA_ERR_UNSUPPORTED). */
+typedef enum { GVA_KERNEL_AUTO = 0, GVA_KERNEL_FMA = 1, GVA_KERNEL_MMA = 2 } gva_kernel;
+
+typedef struct {
+    int32_t H, G;          /* query heads, value groups; H % G == 0 and H/G == 4                          */
+    int32_t d_v;           /* value width: 64 or 128                                                      */
+    int32_t d_c;           /* content-key width (only gva_absorb_query uses it): 1..256                   */
+    int32_t d_r;           /* RoPE width: 16 with d_v = 64, 32 with d_v = 128                             */
+    int32_t page_size;     /* tokens per page, a multiple of 32                                           */
+    int32_t cache_dtype;   /* gva_dtype                                                                   */
+    int32_t kernel;        /* gva_kernel                                                                  */
+    double rope_base;      /* 10000.0                                                                     */
+    float softmax_scale;   /* 0 => 1/sqrt(d_c + d_r)                                                      */
+    int32_t reserved;      /* set to 0                                                                    */
+} gva_config;
+
+typedef struct {
+    void *v_pool;               /* [num_pages][G][page_size][d_v]   16-byte aligned                        */
+    void *kr_pool;              /* [num_pages][page_size][d_r]      16-byte aligned                        */
+    const int32_t *block_table; /* [B][max_pages_per_seq] or NULL (contiguous)                             */
+    int32_t num_pages;
+    int32_t max_pages_per_seq;
+} gva_cache;
+
+typedef struct {
+    void *k_pool;               /* [num_pages][G][page_size][d_h]  keys, already rotated                    */
+    void *v_pool;               /* [num_pages][G][page_size][d_h]                                           */
+    const int32_t *block_table;
+    int32_t num_pages;
+    int32_t max_pages_per_seq;
+} gqa_cache;
+
+typedef struct gva_handle gva_handle; /* opaque host-side state: config, device properties, last launch geometry */
+
+/* Create / destroy a handle for one head configuration on one device.  Validates cfg
+ * (GVA_ERR_UNSUPPORTED / GVA_ERR_INVALID_ARG), checks that `device` is compute capability 10.x
+ * (GVA_ERR_CUDA otherwise) and raises the kernels' shared-memory limits.  Makes `device` current. */
+int gva_create(gva_handle **out, const gva_config *cfg, int device);
+int gva_destroy(gva_handle *h);
+
+/* Bytes of scratch gva_decode / gqa_decode need for B sequences of at most max_seq_len tokens with
+ * the given num_splits (same meaning as in gva_decode).  Holds the split-KV partial results
+ * (unnormalised output, running max and sum per partition and head).  0 on invalid arguments. */
+size_t gva_decode_workspace_bytes(const gva_handle *h, int B, int max_seq_len, int num_splits);
+
+/* Eq. absorb and the query-side rotation of Algorithm 1.
+ *   q_c   [B][H][d_c] f32   content ("nope") query slices
+ *   q_r   [B][H][d_r] f32   positional query slices, unrotated
+ *   M     [H][d_v][d_c] f32 reconstruction maps, row-major (M_h in R^{d_h x d_n}; K_h = V_g(h) M_h)
+ *   q_pos [B] i32           query positions t (0-based)
+ *   q_abs [B][H][d_v+d_r] f32 out:  [:d_v] = q_c M_h^T  (q~[i] = sum_j q_c[j] M_h[i][j]),
+ *                                   [d_v:] = q_r R_t^T */
+int gva_absorb_query(gva_handle *h, const float *q_c, const float *q_r, const float *M,
+                     const int32_t *q_pos, float *q_abs, int B, void *stream);
+
+/* Algorithm 1's cache append for one new token per sequence.
+ *   v_new  [B][G][d_v] f32   new value rows;  kr_new [B][d_r] f32 unrotated positional key (x_t W_r)
+ *   pos    [B] i32           0-based position t of the new token
+ * Writes, for each b, rows (page = block_table[b][t/page_size], slot = t % page_size):
+ *   v_pool[page][g][slot][:] = cast(v_new[b][g][:]),  kr_pool[page][slot][:] = cast(kr_new[b] R_t^T)
+ * cast = round-to-nearest-even to the cache dtype (from the fp64 rotation for k^rope); no other byte
+ * of the pools changes.  pos < 0 or beyond the block table -> GVA_ERR_SEQ_LEN in *dev_status, bad
+ * page id -> GVA_ERR_BAD_PAGE; that sequence is skipped. */
+int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, const float *kr_new,
+                     const int32_t *pos, int B, int32_t *dev_status, void *stream);
+
+/* Decode attention over the cache (the score and softmax-value lines of Algorithm 1) for B
+ * sequences, query heads sharing each value group's stream.
+ *   q_abs    [B][H][d_v+d_r] f32  from gva_absorb_query
+ *   seq_lens [B] i32              number of cached tokens attended (positions 0..seq_len-1)
+ *   out      [B][H][d_v] f32      o_h;  seq_len == 0 gives 0
+ *   lse      [B][H] f32 or NULL   natural log of sum_j exp(scale * s_j); -inf for seq_len == 0
+ *   workspace / workspace_bytes   scratch of at least gva_decode_workspace_bytes(h, B, max_seq_len, num_splits),
+ *                                 256-byte aligned; contents are overwritten; calls sharing it must be
+ *                                 stream-ordered
+ *   max_seq_len                   upper bound on seq_lens[] (sizes the launch; a longer sequence is
+ *                                 still computed correctly as long as it fits its block table)
+ *   num_splits                    0: the cache stream is cut into equal contiguous ranges of tiles, one
+ *                                 per resident thread block (ranges may cross sequence boundaries);
+ *                                 n >= 1: every sequence is cut into exactly n ranges.
+ * Partial results are merged by log-sum-exp weights in a second kernel.  For fixed arguments the
+ * result is bitwise reproducible from run to run. */
+int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens,
+               float *out, float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len,
+               int num_splits, int32_t *dev_status, void *stream);
+
+/* Matched GQA decode (two cached streams): s_j = q_h K_{j,g(h)}^T / sqrt(d_h), o_h = softmax(s) V_{g(h)},
+ * with d_h = cfg.d_v, q [B][H][d_h] f32 already rotated, K cached already rotated.  Same paging,
+ * splitting, workspace and error rules as gva_decode.  cfg.d_c, cfg.d_r and cfg.softmax_scale are
+ * ignored (scale = 1/sqrt(d_h)). */
+int gqa_decode(gva_handle *h, const gqa_cache *cache, const float *q, const int32_t *seq_lens, float *out,
+               float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
+               int32_t *dev_status, void *stream);
+
+/* One whole decode step (Algorithm 1 from the split queries to the per-head outputs) for callers whose
+ * per-step tensors live in HOST memory: copies the step's inputs to the device, runs
+ * gva_absorb_query -> gva_append_cache -> gva_decode, and copies the outputs back, all enqueued on
+ * `stream`; the caller synchronises the stream before reading out_host.  The cache and the maps M stay
+ * resident on the device (they are state, not per-step input).
+ *   [host] q_c_host [B][H][d_c], q_r_host [B][H][d_r], v_new_host [B][G][d_v], kr_new_host [B][d_r] f32,
+ *          pos_host [B] i32 (position t of the new token = query position), seq_lens_host [B] i32
+ *          (tokens attended, normally t + 1).  Use pinned memory for truly asynchronous copies.
+ *   [host] out_host [B][H][d_v] f32
+ *   M                device, as in gva_absorb_query
+ *   scratch          device, at least gva_step_scratch_bytes(h, B, max_seq_len, num_splits) bytes, 256-byte aligned;
+ *                    holds the staged inputs, q_abs, out and the decode workspace.
+ * Bytes moved per call: host->device B*(H*(d_c+d_r) + G*d_v + d_r)*4 + 8*B, device->host B*H*d_v*4. */
+size_t gva_step_scratch_bytes(const gva_handle *h, int B, int max_seq_len, int num_splits);
+int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, const float *q_c_host,
+                         const float *q_r_host, const float *v_new_host, const float *kr_new_host,
+                         const int32_t *pos_host, const int32_t *seq_lens_host, float *out_host, void *scratch,
+                         size_t scratch_bytes, int B, int max_seq_len, int num_splits, int32_t *dev_status,
+                         void *stream);
+
+/* Geometry of the most recent gva_decode / gqa_decode launch on this handle (reporting only):
+ * number of split-KV partitions launched (thread blocks of the decode kernel). */
+int gva_last_num_splits(const gva_handle *h);
+/* 1 = CUDA-core (FMA) kernel, 2 = tensor-core (MMA) kernel, 0 = none yet. */
+int gva_last_kernel(const gva_handle *h);
+/* Tokens per tile of the kernel chosen by the last launch (the unit in which ranges are cut). */
+int gva_last_tile_tokens(const gva_handle *h);
+
+const char *gva_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GVA_H_ */

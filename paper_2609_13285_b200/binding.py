@@ -1,0 +1,194 @@
+"""Thin ctypes binding of the C ABI in include/gva.h: argument marshalling only.
+
+Every function mirrors the C entry point of the same name.  Device buffers are torch CUDA
+tensors (torch is used for device memory and streams, nothing else); each call enqueues on the
+current torch stream.  There is no CPU fallback: if libgva.so is missing or fails to load, the
+first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgva.so")
+
+GVA_OK = 0
+GVA_ERR_INVALID_ARG, GVA_ERR_UNSUPPORTED, GVA_ERR_WORKSPACE, GVA_ERR_CUDA = 1, 2, 3, 4
+GVA_ERR_BAD_PAGE, GVA_ERR_SEQ_LEN, GVA_ERR_TIMEOUT = 5, 6, 7
+GVA_F32, GVA_BF16 = 0, 1
+GVA_KERNEL_AUTO, GVA_KERNEL_FMA, GVA_KERNEL_MMA = 0, 1, 2
+
+EXPORTS = ["gva_create", "gva_destroy", "gva_decode_workspace_bytes", "gva_absorb_query", "gva_append_cache",
+           "gva_decode", "gqa_decode", "gva_step_scratch_bytes", "gva_decode_step_host", "gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens",
+           "gva_status_string"]
+
+
+class GvaConfig(ctypes.Structure):
+    _fields_ = [("H", ctypes.c_int32), ("G", ctypes.c_int32), ("d_v", ctypes.c_int32), ("d_c", ctypes.c_int32),
+                ("d_r", ctypes.c_int32), ("page_size", ctypes.c_int32), ("cache_dtype", ctypes.c_int32),
+                ("kernel", ctypes.c_int32), ("rope_base", ctypes.c_double), ("softmax_scale", ctypes.c_float),
+                ("reserved", ctypes.c_int32)]
+
+
+class GvaCache(ctypes.Structure):
+    _fields_ = [("v_pool", ctypes.c_void_p), ("kr_pool", ctypes.c_void_p), ("block_table", ctypes.c_void_p),
+                ("num_pages", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32)]
+
+
+class GqaCache(ctypes.Structure):
+    _fields_ = [("k_pool", ctypes.c_void_p), ("v_pool", ctypes.c_void_p), ("block_table", ctypes.c_void_p),
+                ("num_pages", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32)]
+
+
+class GvaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (gva_status {status})")
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load() -> ctypes.CDLL:
+    """dlopen libgva.so and declare the prototypes.  Raises if the library has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2609_13285_b200.build` "
+                           "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ip, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.gva_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(GvaConfig), ip]
+    lib.gva_destroy.argtypes = [vp]
+    lib.gva_decode_workspace_bytes.argtypes = [vp, ip, ip, ip]
+    lib.gva_decode_workspace_bytes.restype = sz
+    lib.gva_step_scratch_bytes.argtypes = [vp, ip, ip, ip]
+    lib.gva_step_scratch_bytes.restype = sz
+    lib.gva_decode_step_host.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, ip, ip,
+                                         ip, vp, vp]
+    lib.gva_absorb_query.argtypes = [vp, vp, vp, vp, vp, vp, ip, vp]
+    lib.gva_append_cache.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, ip, vp, vp]
+    lib.gva_decode.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, vp, sz, ip, ip, ip, vp, vp]
+    lib.gqa_decode.argtypes = [vp, ctypes.POINTER(GqaCache), vp, vp, vp, vp, vp, sz, ip, ip, ip, vp, vp]
+    for name in ("gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens"):
+        getattr(lib, name).argtypes = [vp]
+    lib.gva_status_string.argtypes = [ip]
+    lib.gva_status_string.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name not in ("gva_decode_workspace_bytes", "gva_step_scratch_bytes", "gva_status_string"):
+            getattr(lib, name).restype = ip
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().gva_status_string(int(status)).decode()
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+def _stream() -> int:
+    import torch
+    return int(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != GVA_OK:
+        raise GvaError(rc, where)
+
+
+def gva_create(*, H: int, G: int, d_v: int, d_c: int, d_r: int, page_size: int, cache_dtype: int = GVA_BF16,
+               kernel: int = GVA_KERNEL_AUTO, rope_base: float = 10000.0, softmax_scale: float = 0.0,
+               device: int = 0) -> int:
+    cfg = GvaConfig(H, G, d_v, d_c, d_r, page_size, cache_dtype, kernel, rope_base, softmax_scale, 0)
+    h = ctypes.c_void_p()
+    _check(load().gva_create(ctypes.byref(h), ctypes.byref(cfg), int(device)), "gva_create")
+    return h.value
+
+
+def gva_destroy(handle: int) -> None:
+    _check(load().gva_destroy(handle), "gva_destroy")
+
+
+def gva_decode_workspace_bytes(handle: int, B: int, max_seq_len: int, num_splits: int = 0) -> int:
+    return int(load().gva_decode_workspace_bytes(handle, int(B), int(max_seq_len), int(num_splits)))
+
+
+def gva_absorb_query(handle: int, q_c, q_r, M, q_pos, q_abs, B: int, check: bool = True) -> int:
+    rc = load().gva_absorb_query(handle, _ptr(q_c), _ptr(q_r), _ptr(M), _ptr(q_pos), _ptr(q_abs), int(B), _stream())
+    if check:
+        _check(rc, "gva_absorb_query")
+    return rc
+
+
+def make_cache(v_pool, kr_pool, block_table, num_pages: int, max_pages_per_seq: int) -> GvaCache:
+    return GvaCache(_ptr(v_pool), _ptr(kr_pool), _ptr(block_table), int(num_pages), int(max_pages_per_seq))
+
+
+def make_gqa_cache(k_pool, v_pool, block_table, num_pages: int, max_pages_per_seq: int) -> GqaCache:
+    return GqaCache(_ptr(k_pool), _ptr(v_pool), _ptr(block_table), int(num_pages), int(max_pages_per_seq))
+
+
+def gva_append_cache(handle: int, cache: GvaCache, v_new, kr_new, pos, B: int, dev_status=None,
+                     check: bool = True) -> int:
+    rc = load().gva_append_cache(handle, ctypes.byref(cache), _ptr(v_new), _ptr(kr_new), _ptr(pos), int(B),
+                                 _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gva_append_cache")
+    return rc
+
+
+def gva_decode(handle: int, cache: GvaCache, q_abs, seq_lens, out, lse, workspace, B: int, max_seq_len: int,
+               num_splits: int = 0, dev_status=None, workspace_bytes: Optional[int] = None, check: bool = True) -> int:
+    wb = (workspace.numel() * workspace.element_size() if workspace is not None else 0) \
+        if workspace_bytes is None else int(workspace_bytes)
+    rc = load().gva_decode(handle, ctypes.byref(cache), _ptr(q_abs), _ptr(seq_lens), _ptr(out), _ptr(lse),
+                           _ptr(workspace), wb, int(B), int(max_seq_len), int(num_splits), _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gva_decode")
+    return rc
+
+
+def gqa_decode(handle: int, cache: GqaCache, q, seq_lens, out, lse, workspace, B: int, max_seq_len: int,
+               num_splits: int = 0, dev_status=None, workspace_bytes: Optional[int] = None, check: bool = True) -> int:
+    wb = (workspace.numel() * workspace.element_size() if workspace is not None else 0) \
+        if workspace_bytes is None else int(workspace_bytes)
+    rc = load().gqa_decode(handle, ctypes.byref(cache), _ptr(q), _ptr(seq_lens), _ptr(out), _ptr(lse),
+                           _ptr(workspace), wb, int(B), int(max_seq_len), int(num_splits), _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gqa_decode")
+    return rc
+
+
+def gva_step_scratch_bytes(handle: int, B: int, max_seq_len: int, num_splits: int = 0) -> int:
+    return int(load().gva_step_scratch_bytes(handle, int(B), int(max_seq_len), int(num_splits)))
+
+
+def gva_decode_step_host(handle: int, cache: GvaCache, M, q_c_host, q_r_host, v_new_host, kr_new_host, pos_host,
+                         seq_lens_host, out_host, scratch, B: int, max_seq_len: int, num_splits: int = 0,
+                         dev_status=None, check: bool = True) -> int:
+    """Host tensors are CPU torch tensors (pinned for asynchronous copies); M, scratch, dev_status are CUDA tensors."""
+    rc = load().gva_decode_step_host(handle, ctypes.byref(cache), _ptr(M), _ptr(q_c_host), _ptr(q_r_host),
+                                     _ptr(v_new_host), _ptr(kr_new_host), _ptr(pos_host), _ptr(seq_lens_host),
+                                     _ptr(out_host), _ptr(scratch), scratch.numel() * scratch.element_size(), int(B),
+                                     int(max_seq_len), int(num_splits), _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gva_decode_step_host")
+    return rc
+
+
+def gva_last_num_splits(handle: int) -> int:
+    return int(load().gva_last_num_splits(handle))
+
+
+def gva_last_kernel(handle: int) -> int:
+    return int(load().gva_last_kernel(handle))
+
+
+def gva_last_tile_tokens(handle: int) -> int:
+    return int(load().gva_last_tile_tokens(handle))

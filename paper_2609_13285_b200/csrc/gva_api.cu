@@ -1,0 +1,429 @@
+// Host side of the C ABI declared in include/gva.h: argument validation, launch geometry, kernel
+// dispatch.  No device memory is allocated here and no call synchronises.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "gva_common.cuh"
+#include "gva_decode_fma.cuh"
+#include "gva_small_kernels.cuh"
+#ifdef GVA_WITH_MMA
+#include "gva_decode_mma.cuh"
+#endif
+
+using namespace gva;
+
+struct gva_handle {
+    gva_config cfg;
+    int device;
+    int sm_count;
+    int smem_optin;          // max dynamic shared memory per block
+    float scale;             // softmax scale of gva_decode
+    RopeTable rope;
+    int last_num_splits;
+    int last_kernel;
+    int last_tile;
+#ifdef GVA_WITH_MMA
+    MmaHostState mma;
+#endif
+};
+
+namespace {
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- FMA kernel dispatch ---------------------------------------------------------------------
+using KernelFn = void (*)(DecodeParams);
+
+template <typename CT, int DV, int DR, bool GQA>
+KernelFn fma_kernel_for(int nstage) {
+    switch (nstage) {
+        case 1: return decode_fma_kernel<CT, DV, DR, GQA, 1>;
+        case 2: return decode_fma_kernel<CT, DV, DR, GQA, 2>;
+        default: return decode_fma_kernel<CT, DV, DR, GQA, 3>;
+    }
+}
+
+struct FmaPlan {
+    KernelFn fn;
+    int nstage;
+    size_t smem;
+    int threads;
+};
+
+template <typename CT, int DV, int DR, bool GQA>
+bool plan_fma_t(const gva_handle *h, int B, FmaPlan *out) {
+    using T = FmaTraits<CT, DV, DR, GQA>;
+    const int G = h->cfg.G, H = h->cfg.H;
+    const size_t fixed = T::fixed_bytes(B, H, G);
+    const size_t stage = T::stage_bytes(G);
+    int nstage = 3;
+    // three stages when that still leaves room for three blocks per SM, else two, else one
+    if (fixed + 3 * stage > (size_t)h->smem_optin / 3) nstage = 2;
+    if (fixed + (size_t)nstage * stage > (size_t)h->smem_optin) nstage = 1;
+    if (fixed + (size_t)nstage * stage > (size_t)h->smem_optin) return false;
+    out->fn = fma_kernel_for<CT, DV, DR, GQA>(nstage);
+    out->nstage = nstage;
+    out->smem = fixed + (size_t)nstage * stage;
+    out->threads = 32 * G;
+    return true;
+}
+
+template <bool GQA>
+bool plan_fma(const gva_handle *h, int B, FmaPlan *out) {
+    const bool bf = h->cfg.cache_dtype == GVA_BF16;
+    if (h->cfg.d_v == 64)
+        return bf ? plan_fma_t<__nv_bfloat16, 64, 16, GQA>(h, B, out) : plan_fma_t<float, 64, 16, GQA>(h, B, out);
+    return bf ? plan_fma_t<__nv_bfloat16, 128, 32, GQA>(h, B, out) : plan_fma_t<float, 128, 32, GQA>(h, B, out);
+}
+
+// Workspace: header ints, then partial outputs, then (max, sum) pairs.
+struct WorkspaceLayout {
+    size_t hdr_bytes, rec_o_bytes, rec_ml_bytes, total;
+    int n_rec;
+};
+
+int max_blocks_balanced(const gva_handle *h) {
+    // an upper bound on resident decode blocks that any kernel variant launches: 4 per SM
+    return 4 * h->sm_count;
+}
+
+WorkspaceLayout workspace_layout(const gva_handle *h, int B, int num_splits) {
+    WorkspaceLayout w;
+    w.n_rec = num_splits > 0 ? B * num_splits : max_blocks_balanced(h) + B;
+    w.hdr_bytes = align_up((size_t)(kHdrInts + B + 1) * 4, 256);
+    w.rec_o_bytes = align_up((size_t)w.n_rec * h->cfg.H * h->cfg.d_v * 4, 256);
+    w.rec_ml_bytes = align_up((size_t)w.n_rec * h->cfg.H * 2 * 4, 256);
+    w.total = w.hdr_bytes + w.rec_o_bytes + w.rec_ml_bytes;
+    return w;
+}
+
+int check_common(const gva_handle *h, int B, int max_seq_len, int num_splits) {
+    if (!h) return GVA_ERR_INVALID_ARG;
+    if (B < 0 || max_seq_len < 0 || num_splits < 0) return GVA_ERR_INVALID_ARG;
+    if (B > 8192 || num_splits > 4096) return GVA_ERR_UNSUPPORTED;
+    // total tiles must fit an int with headroom
+    if ((long long)B * ((max_seq_len + 31) / 32 + 1) >= (1ll << 30)) return GVA_ERR_UNSUPPORTED;
+    return GVA_OK;
+}
+
+template <bool GQA>
+int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspace_bytes, int B, int max_seq_len,
+                  int num_splits, cudaStream_t stream) {
+    const WorkspaceLayout w = workspace_layout(h, B, num_splits);
+    if (!workspace || workspace_bytes < w.total) return GVA_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return GVA_ERR_INVALID_ARG;
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    p.hdr = reinterpret_cast<int32_t *>(ws);
+    p.rec_o = reinterpret_cast<float *>(ws + w.hdr_bytes);
+    p.rec_ml = reinterpret_cast<float *>(ws + w.hdr_bytes + w.rec_o_bytes);
+    p.num_splits = num_splits;
+    if (B == 0) return GVA_OK;
+
+    int kernel = h->cfg.kernel;
+    if (kernel == GVA_KERNEL_AUTO) {
+#ifdef GVA_WITH_MMA
+        kernel = (h->cfg.cache_dtype == GVA_BF16 && mma_supported(h->cfg, GQA)) ? GVA_KERNEL_MMA : GVA_KERNEL_FMA;
+#else
+        kernel = GVA_KERNEL_FMA;
+#endif
+    }
+    if (kernel == GVA_KERNEL_MMA) {
+#ifdef GVA_WITH_MMA
+        int rc = launch_decode_mma<GQA>(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, max_seq_len, num_splits,
+                                        max_blocks_balanced(h), stream, &h->last_num_splits, &h->last_tile);
+        if (rc != GVA_OK) return rc;
+        h->last_kernel = GVA_KERNEL_MMA;
+#else
+        return GVA_ERR_UNSUPPORTED;
+#endif
+    } else {
+        FmaPlan plan;
+        if (!plan_fma<GQA>(h, B, &plan)) return GVA_ERR_UNSUPPORTED;
+        if (cudaFuncSetAttribute(plan.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem) != cudaSuccess)
+            return GVA_ERR_CUDA;
+        int grid;
+        if (num_splits > 0) {
+            grid = B * num_splits;
+        } else {
+            int per_sm = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, plan.fn, plan.threads, plan.smem) != cudaSuccess)
+                return GVA_ERR_CUDA;
+            if (per_sm < 1) per_sm = 1;
+            if (per_sm > 4) per_sm = 4;
+            const long long tiles_ub = (long long)B * ((max_seq_len + 31) / 32);
+            grid = (int)std::min<long long>((long long)per_sm * h->sm_count, std::max<long long>(tiles_ub, 1));
+        }
+        plan.fn<<<grid, plan.threads, plan.smem, stream>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return GVA_ERR_CUDA;
+        h->last_num_splits = grid;
+        h->last_kernel = GVA_KERNEL_FMA;
+        h->last_tile = 32;
+    }
+    dim3 cgrid(B, (h->cfg.H + 3) / 4);
+    if (h->cfg.d_v == 64) combine_kernel<64><<<cgrid, 128, 0, stream>>>(p);
+    else combine_kernel<128><<<cgrid, 128, 0, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return GVA_ERR_CUDA;
+    return GVA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gva_create(gva_handle **out, const gva_config *cfg, int device) {
+    if (!out || !cfg) return GVA_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->H <= 0 || cfg->G <= 0 || cfg->d_v <= 0 || cfg->d_c <= 0 || cfg->d_r <= 0 || cfg->page_size <= 0 ||
+        !(cfg->rope_base > 1.0) || !(cfg->softmax_scale >= 0.f) || device < 0)
+        return GVA_ERR_INVALID_ARG;
+    if (cfg->cache_dtype != GVA_F32 && cfg->cache_dtype != GVA_BF16) return GVA_ERR_INVALID_ARG;
+    if (cfg->kernel < GVA_KERNEL_AUTO || cfg->kernel > GVA_KERNEL_MMA) return GVA_ERR_INVALID_ARG;
+    if (cfg->H % cfg->G != 0 || cfg->H / cfg->G != kHeadsPerGroup) return GVA_ERR_UNSUPPORTED;
+    if (!((cfg->d_v == 64 && cfg->d_r == 16) || (cfg->d_v == 128 && cfg->d_r == 32))) return GVA_ERR_UNSUPPORTED;
+    if (cfg->G > 8 || cfg->d_c > 256 || cfg->page_size % 32 != 0) return GVA_ERR_UNSUPPORTED;
+    if (cfg->kernel == GVA_KERNEL_MMA && cfg->cache_dtype != GVA_BF16) return GVA_ERR_UNSUPPORTED;
+#ifndef GVA_WITH_MMA
+    if (cfg->kernel == GVA_KERNEL_MMA) return GVA_ERR_UNSUPPORTED;
+#endif
+
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device >= n_dev) return GVA_ERR_CUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return GVA_ERR_CUDA;
+    int major = 0, sms = 0, optin = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
+        return GVA_ERR_CUDA;
+    if (major != 10) return GVA_ERR_CUDA;   // the kernels are built for sm_100a only
+
+    gva_handle *h = new (std::nothrow) gva_handle();
+    if (!h) return GVA_ERR_INVALID_ARG;
+    h->cfg = *cfg;
+    h->device = device;
+    h->sm_count = sms;
+    h->smem_optin = optin;
+    h->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : (float)(1.0 / std::sqrt((double)(cfg->d_c + cfg->d_r)));
+    for (int i = 0; i < kMaxRopePairs; ++i)
+        h->rope.inv_freq[i] = (2 * i < cfg->d_r) ? std::pow(cfg->rope_base, -2.0 * (double)i / (double)cfg->d_r) : 0.0;
+    h->last_num_splits = 0;
+    h->last_kernel = 0;
+    h->last_tile = 0;
+#ifdef GVA_WITH_MMA
+    int rc = mma_host_init(&h->mma);
+    if (rc != GVA_OK) {
+        delete h;
+        return rc;
+    }
+#endif
+    // the absorb kernel may need more than 48 KB for a 128 x 128 map
+    const size_t absorb_smem = ((size_t)cfg->d_v * (cfg->d_c + 1) + (size_t)kAbsorbBatch * cfg->d_c) * 4;
+    if (absorb_smem > (size_t)optin ||
+        cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)absorb_smem) != cudaSuccess) {
+        delete h;
+        return GVA_ERR_CUDA;
+    }
+    *out = h;
+    return GVA_OK;
+}
+
+int gva_destroy(gva_handle *h) {
+    if (!h) return GVA_ERR_INVALID_ARG;
+    delete h;
+    return GVA_OK;
+}
+
+size_t gva_decode_workspace_bytes(const gva_handle *h, int B, int max_seq_len, int num_splits) {
+    if (check_common(h, B, max_seq_len, num_splits) != GVA_OK) return 0;
+    return workspace_layout(h, B, num_splits).total;
+}
+
+int gva_absorb_query(gva_handle *h, const float *q_c, const float *q_r, const float *M, const int32_t *q_pos,
+                     float *q_abs, int B, void *stream) {
+    if (!h || B < 0) return GVA_ERR_INVALID_ARG;
+    if (B == 0) return GVA_OK;
+    if (!q_c || !q_r || !M || !q_pos || !q_abs) return GVA_ERR_INVALID_ARG;
+    if (!aligned(q_c, 4) || !aligned(q_r, 4) || !aligned(M, 4) || !aligned(q_pos, 4) || !aligned(q_abs, 16))
+        return GVA_ERR_INVALID_ARG;
+    const gva_config &c = h->cfg;
+    const size_t smem = ((size_t)c.d_v * (c.d_c + 1) + (size_t)kAbsorbBatch * c.d_c) * 4;
+    dim3 grid(c.H, (B + kAbsorbBatch - 1) / kAbsorbBatch);
+    absorb_kernel<<<grid, 128, smem, static_cast<cudaStream_t>(stream)>>>(q_c, q_r, M, q_pos, q_abs, B, c.H, c.d_v,
+                                                                          c.d_c, c.d_r, h->rope);
+    return cudaGetLastError() == cudaSuccess ? GVA_OK : GVA_ERR_CUDA;
+}
+
+int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, const float *kr_new,
+                     const int32_t *pos, int B, int32_t *dev_status, void *stream) {
+    if (!h || !cache || B < 0) return GVA_ERR_INVALID_ARG;
+    if (B == 0) return GVA_OK;
+    if (!cache->v_pool || !cache->kr_pool || !v_new || !kr_new || !pos) return GVA_ERR_INVALID_ARG;
+    if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
+    if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16)) return GVA_ERR_INVALID_ARG;
+    const gva_config &c = h->cfg;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (c.cache_dtype == GVA_BF16)
+        append_kernel<__nv_bfloat16><<<B, 128, 0, s>>>(static_cast<__nv_bfloat16 *>(cache->v_pool),
+                                                       static_cast<__nv_bfloat16 *>(cache->kr_pool), cache->block_table,
+                                                       v_new, kr_new, pos, c.G, c.d_v, c.d_r, c.page_size,
+                                                       cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+    else
+        append_kernel<float><<<B, 128, 0, s>>>(static_cast<float *>(cache->v_pool), static_cast<float *>(cache->kr_pool),
+                                               cache->block_table, v_new, kr_new, pos, c.G, c.d_v, c.d_r, c.page_size,
+                                               cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+    return cudaGetLastError() == cudaSuccess ? GVA_OK : GVA_ERR_CUDA;
+}
+
+int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
+               float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
+               int32_t *dev_status, void *stream) {
+    int rc = check_common(h, B, max_seq_len, num_splits);
+    if (rc != GVA_OK) return rc;
+    if (!cache) return GVA_ERR_INVALID_ARG;
+    if (B > 0) {
+        if (!cache->v_pool || !cache->kr_pool || !q_abs || !seq_lens || !out) return GVA_ERR_INVALID_ARG;
+        if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
+        if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16) || !aligned(q_abs, 16) || !aligned(out, 16))
+            return GVA_ERR_INVALID_ARG;
+    }
+    const gva_config &c = h->cfg;
+    DecodeParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.v_pool = cache->v_pool;
+    p.kr_pool = cache->kr_pool;
+    p.block_table = cache->block_table;
+    p.seq_lens = seq_lens;
+    p.q = q_abs;
+    p.out = out;
+    p.lse = lse;
+    p.dev_status = dev_status;
+    p.B = B; p.H = c.H; p.G = c.G; p.P = c.page_size;
+    p.num_pages = cache->num_pages;
+    p.max_pages = cache->max_pages_per_seq;
+    p.scale_log2 = h->scale * kLog2e;
+    return launch_decode<false>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
+                                static_cast<cudaStream_t>(stream));
+}
+
+int gqa_decode(gva_handle *h, const gqa_cache *cache, const float *q, const int32_t *seq_lens, float *out, float *lse,
+               void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits, int32_t *dev_status,
+               void *stream) {
+    int rc = check_common(h, B, max_seq_len, num_splits);
+    if (rc != GVA_OK) return rc;
+    if (!cache) return GVA_ERR_INVALID_ARG;
+    if (B > 0) {
+        if (!cache->k_pool || !cache->v_pool || !q || !seq_lens || !out) return GVA_ERR_INVALID_ARG;
+        if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
+        if (!aligned(cache->k_pool, 16) || !aligned(cache->v_pool, 16) || !aligned(q, 16) || !aligned(out, 16))
+            return GVA_ERR_INVALID_ARG;
+    }
+    const gva_config &c = h->cfg;
+    DecodeParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.v_pool = cache->v_pool;
+    p.k_pool = cache->k_pool;
+    p.block_table = cache->block_table;
+    p.seq_lens = seq_lens;
+    p.q = q;
+    p.out = out;
+    p.lse = lse;
+    p.dev_status = dev_status;
+    p.B = B; p.H = c.H; p.G = c.G; p.P = c.page_size;
+    p.num_pages = cache->num_pages;
+    p.max_pages = cache->max_pages_per_seq;
+    p.scale_log2 = (float)(1.0 / std::sqrt((double)c.d_v)) * kLog2e;
+    return launch_decode<true>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
+                               static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+struct StepLayout {
+    size_t q_c, q_r, v_new, kr_new, pos, lens, q_abs, out, ws, total, ws_bytes;
+};
+StepLayout step_layout(const gva_handle *h, int B, int num_splits) {
+    const gva_config &c = h->cfg;
+    StepLayout L;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
+    L.q_c = take((size_t)B * c.H * c.d_c * 4);
+    L.q_r = take((size_t)B * c.H * c.d_r * 4);
+    L.v_new = take((size_t)B * c.G * c.d_v * 4);
+    L.kr_new = take((size_t)B * c.d_r * 4);
+    L.pos = take((size_t)B * 4);
+    L.lens = take((size_t)B * 4);
+    L.q_abs = take((size_t)B * c.H * (c.d_v + c.d_r) * 4);
+    L.out = take((size_t)B * c.H * c.d_v * 4);
+    L.ws_bytes = workspace_layout(h, B, num_splits).total;
+    L.ws = take(L.ws_bytes);
+    L.total = off;
+    return L;
+}
+}  // namespace
+
+size_t gva_step_scratch_bytes(const gva_handle *h, int B, int max_seq_len, int num_splits) {
+    if (check_common(h, B, max_seq_len, num_splits) != GVA_OK) return 0;
+    return step_layout(h, B, num_splits).total;
+}
+
+int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, const float *q_c_host,
+                         const float *q_r_host, const float *v_new_host, const float *kr_new_host,
+                         const int32_t *pos_host, const int32_t *seq_lens_host, float *out_host, void *scratch,
+                         size_t scratch_bytes, int B, int max_seq_len, int num_splits, int32_t *dev_status,
+                         void *stream) {
+    int rc = check_common(h, B, max_seq_len, num_splits);
+    if (rc != GVA_OK) return rc;
+    if (B == 0) return GVA_OK;
+    if (!cache || !M || !q_c_host || !q_r_host || !v_new_host || !kr_new_host || !pos_host || !seq_lens_host || !out_host)
+        return GVA_ERR_INVALID_ARG;
+    const StepLayout L = step_layout(h, B, num_splits);
+    if (!scratch || scratch_bytes < L.total) return GVA_ERR_WORKSPACE;
+    if (!aligned(scratch, 256)) return GVA_ERR_INVALID_ARG;
+    const gva_config &c = h->cfg;
+    unsigned char *s = static_cast<unsigned char *>(scratch);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    auto h2d = [&](size_t off, const void *src, size_t bytes) {
+        return cudaMemcpyAsync(s + off, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    };
+    if (!h2d(L.q_c, q_c_host, (size_t)B * c.H * c.d_c * 4) || !h2d(L.q_r, q_r_host, (size_t)B * c.H * c.d_r * 4) ||
+        !h2d(L.v_new, v_new_host, (size_t)B * c.G * c.d_v * 4) || !h2d(L.kr_new, kr_new_host, (size_t)B * c.d_r * 4) ||
+        !h2d(L.pos, pos_host, (size_t)B * 4) || !h2d(L.lens, seq_lens_host, (size_t)B * 4))
+        return GVA_ERR_CUDA;
+    const int32_t *pos = reinterpret_cast<const int32_t *>(s + L.pos);
+    float *q_abs = reinterpret_cast<float *>(s + L.q_abs);
+    float *out = reinterpret_cast<float *>(s + L.out);
+    rc = gva_absorb_query(h, reinterpret_cast<const float *>(s + L.q_c), reinterpret_cast<const float *>(s + L.q_r), M,
+                          pos, q_abs, B, stream);
+    if (rc != GVA_OK) return rc;
+    rc = gva_append_cache(h, cache, reinterpret_cast<const float *>(s + L.v_new),
+                          reinterpret_cast<const float *>(s + L.kr_new), pos, B, dev_status, stream);
+    if (rc != GVA_OK) return rc;
+    rc = gva_decode(h, cache, q_abs, reinterpret_cast<const int32_t *>(s + L.lens), out, nullptr, s + L.ws, L.ws_bytes,
+                    B, max_seq_len, num_splits, dev_status, stream);
+    if (rc != GVA_OK) return rc;
+    if (cudaMemcpyAsync(out_host, out, (size_t)B * c.H * c.d_v * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return GVA_ERR_CUDA;
+    return GVA_OK;
+}
+
+int gva_last_num_splits(const gva_handle *h) { return h ? h->last_num_splits : 0; }
+int gva_last_kernel(const gva_handle *h) { return h ? h->last_kernel : 0; }
+int gva_last_tile_tokens(const gva_handle *h) { return h ? h->last_tile : 0; }
+
+const char *gva_status_string(int status) {
+    switch (status) {
+        case GVA_OK: return "ok";
+        case GVA_ERR_INVALID_ARG: return "invalid argument";
+        case GVA_ERR_UNSUPPORTED: return "unsupported shape, dtype or page size";
+        case GVA_ERR_WORKSPACE: return "workspace missing or too small";
+        case GVA_ERR_CUDA: return "CUDA call failed";
+        case GVA_ERR_BAD_PAGE: return "block-table entry outside the page pool";
+        case GVA_ERR_SEQ_LEN: return "sequence length or position outside the block table";
+        case GVA_ERR_TIMEOUT: return "bounded wait on an asynchronous copy expired";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

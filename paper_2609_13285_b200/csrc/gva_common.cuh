@@ -1,0 +1,171 @@
+// Shared device-side pieces of the GVA decode library: launch parameters, the split-KV work
+// partition, the workspace layout, and small PTX wrappers.  sm_100a only.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/gva.h"
+
+namespace gva {
+
+constexpr int kHeadsPerGroup = 4;   // H / G of every instantiated kernel
+constexpr int kHdrInts = 8;         // workspace header: [0]=total tiles, [1]=partitions in use, [2]=num_splits, [3]=tile tokens
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Everything a decode / combine launch needs, passed by value.
+struct DecodeParams {
+    const void *v_pool;          // GVA: values.  GQA: values.
+    const void *kr_pool;         // GVA: shared rotated positional keys.  GQA: unused.
+    const void *k_pool;          // GQA only: keys.
+    const int32_t *block_table;  // nullable
+    const int32_t *seq_lens;
+    const float *q;              // [B][H][d_q]
+    int32_t *hdr;                // workspace header (kHdrInts + B + 1 ints)
+    float *rec_o;                // [n_rec][H][d_v] unnormalised partial outputs
+    float *rec_ml;               // [n_rec][H][2]   running max (log2 domain) and sum
+    float *out;                  // [B][H][d_v]
+    float *lse;                  // nullable
+    int32_t *dev_status;         // nullable
+    int B, H, G, P, num_pages, max_pages;
+    int num_splits;              // 0 = balanced flat partition
+    float scale_log2;            // softmax scale * log2(e)
+};
+
+__device__ __forceinline__ void report_error(int32_t *dev_status, int code, int b) {
+    if (dev_status) atomicCAS(dev_status, 0, code | (b << 8));
+}
+
+// ---- work partition --------------------------------------------------------------------------
+// The cache stream of a batch is the concatenation of every sequence's tiles (TILE tokens each).
+// s_off[b] = number of tiles before sequence b; s_off[B] = total.
+//   balanced mode (num_splits == 0): the n_eff = ceil(total / ceil(total / gridDim.x)) leading thread
+//     blocks take equal contiguous ranges of the flat tile list; block c, sequence b -> record c + b
+//     (unique because c and b never decrease along the list and one of them grows at each cut).
+//   uniform mode (num_splits == S): block c handles split c % S of sequence c / S -> record c.
+// Must be called by every thread of the block; ends with a barrier.
+template <int TILE>
+__device__ __forceinline__ void compute_tile_offsets(const DecodeParams &p, int *s_off) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const long long cap = (long long)p.max_pages * p.P;
+    for (int b = tid; b < p.B; b += nt) {
+        int len = p.seq_lens[b];
+        if (len < 0 || (long long)len > cap) {
+            report_error(p.dev_status, GVA_ERR_SEQ_LEN, b);
+            len = 0;
+        }
+        s_off[b + 1] = (len + TILE - 1) / TILE;
+    }
+    if (tid == 0) s_off[0] = 0;
+    __syncthreads();
+    if (tid < 32) {
+        const int per = (p.B + 31) / 32;
+        const int start = 1 + tid * per;
+        const int end = min(start + per, p.B + 1);
+        int sum = 0;
+        for (int i = start; i < end; ++i) sum += s_off[i];
+        int x = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int y = __shfl_up_sync(0xffffffffu, x, o);
+            if (tid >= o) x += y;
+        }
+        int base = x - sum;
+        for (int i = start; i < end; ++i) {
+            base += s_off[i];
+            s_off[i] = base;
+        }
+    }
+    __syncthreads();
+}
+
+__host__ __device__ __forceinline__ int partitions_in_use(int total_tiles, int n_blocks) {
+    if (total_tiles <= 0) return 0;
+    int per = (total_tiles + n_blocks - 1) / n_blocks;
+    return (total_tiles + per - 1) / per;
+}
+__host__ __device__ __forceinline__ int range_begin(int c, int total_tiles, int n_eff) {
+    return (int)(((long long)c * total_tiles) / n_eff);
+}
+// block that owns flat tile x under range_begin(): the smallest c with range_begin(c+1) > x
+__host__ __device__ __forceinline__ int range_owner(int x, int total_tiles, int n_eff) {
+    return (int)((((long long)x + 1) * n_eff + total_tiles - 1) / total_tiles) - 1;
+}
+
+// This block's flat tile range and, in uniform mode, its fixed record.
+struct BlockRange {
+    int lo, hi;      // flat tiles [lo, hi)
+    int rec_fixed;   // uniform mode: record index; balanced: -1
+    int b_first;     // sequence containing tile lo (valid when lo < hi)
+};
+
+__device__ __forceinline__ int seq_of_tile(const int *s_off, int B, int x) {
+    int lo = 0, hi = B - 1;   // largest b with s_off[b] <= x  (and s_off[b+1] > x because x < total)
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (s_off[mid] <= x) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ BlockRange block_range(const DecodeParams &p, const int *s_off) {
+    BlockRange r;
+    const int total = s_off[p.B];
+    if (p.num_splits > 0) {
+        const int b = blockIdx.x / p.num_splits, s = blockIdx.x % p.num_splits;
+        const int tiles = s_off[b + 1] - s_off[b];
+        r.lo = s_off[b] + (int)(((long long)s * tiles) / p.num_splits);
+        r.hi = s_off[b] + (int)(((long long)(s + 1) * tiles) / p.num_splits);
+        r.rec_fixed = blockIdx.x;
+        r.b_first = b;
+    } else {
+        const int n_eff = partitions_in_use(total, gridDim.x);
+        r.rec_fixed = -1;
+        if ((int)blockIdx.x >= n_eff) {
+            r.lo = r.hi = 0;
+            r.b_first = 0;
+        } else {
+            r.lo = range_begin(blockIdx.x, total, n_eff);
+            r.hi = range_begin(blockIdx.x + 1, total, n_eff);
+            r.b_first = (r.lo < r.hi) ? seq_of_tile(s_off, p.B, r.lo) : 0;
+        }
+    }
+    return r;
+}
+
+// Block 0 publishes the tile offsets for the combine kernel.
+__device__ __forceinline__ void publish_header(const DecodeParams &p, const int *s_off, int tile_tokens) {
+    if (blockIdx.x != 0) return;
+    const int total = s_off[p.B];
+    if (threadIdx.x == 0) {
+        p.hdr[0] = total;
+        p.hdr[1] = (p.num_splits > 0) ? p.B * p.num_splits : partitions_in_use(total, gridDim.x);
+        p.hdr[2] = p.num_splits;
+        p.hdr[3] = tile_tokens;
+    }
+    for (int i = threadIdx.x; i <= p.B; i += blockDim.x) p.hdr[kHdrInts + i] = s_off[i];
+}
+
+// ---- small PTX wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *ptr) {
+    return (uint32_t)__cvta_generic_to_shared(ptr);
+}
+// 16-byte asynchronous global->shared copy; src_bytes == 0 writes 16 zero bytes instead.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+
+}  // namespace gva

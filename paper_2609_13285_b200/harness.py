@@ -1,0 +1,107 @@
+"""Moves a generated decode case into device memory and wraps the three library calls.
+
+No arithmetic happens here: tensors are uploaded as generated (bf16 pools as raw 16-bit patterns)
+and handed to the C ABI through `binding`.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import binding as gb
+from .workloads import DecodeCase
+
+
+def _dev(a: Optional[np.ndarray], device) -> Optional[torch.Tensor]:
+    if a is None:
+        return None
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).to(device)   # raw bf16 bit patterns
+    return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+
+
+@dataclass
+class DeviceCase:
+    case: DecodeCase
+    handle: int
+    v_pool: torch.Tensor
+    kr_pool: torch.Tensor
+    block_table: Optional[torch.Tensor]
+    seq_lens: torch.Tensor
+    q_c: torch.Tensor
+    q_r: torch.Tensor
+    M: torch.Tensor
+    q_pos: torch.Tensor
+    v_new: torch.Tensor
+    kr_new: torch.Tensor
+    append_pos: torch.Tensor
+    q_abs: torch.Tensor
+    out: torch.Tensor
+    lse: torch.Tensor
+    status: torch.Tensor
+    workspace: Optional[torch.Tensor] = None
+    workspace_splits: int = -1
+
+    @property
+    def cache(self) -> gb.GvaCache:
+        c = self.case
+        return gb.make_cache(self.v_pool, self.kr_pool, self.block_table, c.num_pages, c.max_pages_per_seq)
+
+    def ensure_workspace(self, num_splits: int) -> torch.Tensor:
+        need = gb.gva_decode_workspace_bytes(self.handle, self.case.B, self.max_seq_len, num_splits)
+        if self.workspace is None or self.workspace.numel() < need:
+            self.workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=self.v_pool.device)
+        return self.workspace
+
+    @property
+    def max_seq_len(self) -> int:
+        return int(self.case.seq_lens.max()) if self.case.B else 0
+
+    def absorb(self) -> torch.Tensor:
+        gb.gva_absorb_query(self.handle, self.q_c, self.q_r, self.M, self.q_pos, self.q_abs, self.case.B)
+        return self.q_abs
+
+    def append(self) -> None:
+        gb.gva_append_cache(self.handle, self.cache, self.v_new, self.kr_new, self.append_pos, self.case.B,
+                            self.status)
+
+    def decode(self, num_splits: int = 0, q_abs: Optional[torch.Tensor] = None, seq_lens=None,
+               max_seq_len: Optional[int] = None):
+        ws = self.ensure_workspace(num_splits)
+        gb.gva_decode(self.handle, self.cache, self.q_abs if q_abs is None else q_abs,
+                      self.seq_lens if seq_lens is None else seq_lens, self.out, self.lse, ws, self.case.B,
+                      self.max_seq_len if max_seq_len is None else max_seq_len, num_splits, self.status)
+        return self.out, self.lse
+
+    def pools_to_host(self):
+        v = self.v_pool.cpu().numpy()
+        k = self.kr_pool.cpu().numpy()
+        if self.case.cache_dtype == "bf16":
+            v, k = v.view(np.uint16), k.view(np.uint16)
+        return v, k
+
+    def close(self) -> None:
+        if self.handle:
+            gb.gva_destroy(self.handle)
+            self.handle = 0
+
+
+def upload(case: DecodeCase, device="cuda:0", kernel: int = gb.GVA_KERNEL_AUTO) -> DeviceCase:
+    dev = torch.device(device)
+    s = case.shape
+    handle = gb.gva_create(H=s.H, G=s.G, d_v=s.d_v, d_c=s.d_c, d_r=s.d_r, page_size=case.page_size,
+                           cache_dtype=gb.GVA_BF16 if case.cache_dtype == "bf16" else gb.GVA_F32, kernel=kernel,
+                           rope_base=case.rope_base, device=dev.index or 0)
+    B = case.B
+    return DeviceCase(
+        case=case, handle=handle, v_pool=_dev(case.v_pool, dev), kr_pool=_dev(case.kr_pool, dev),
+        block_table=_dev(case.block_table, dev), seq_lens=_dev(case.seq_lens, dev), q_c=_dev(case.q_c, dev),
+        q_r=_dev(case.q_r, dev), M=_dev(case.M, dev), q_pos=_dev(case.q_pos, dev), v_new=_dev(case.v_new, dev),
+        kr_new=_dev(case.kr_new, dev), append_pos=_dev(case.append_pos, dev),
+        q_abs=torch.empty((B, s.H, s.d_v + s.d_r), dtype=torch.float32, device=dev),
+        out=torch.full((B, s.H, s.d_v), float("nan"), dtype=torch.float32, device=dev),
+        lse=torch.full((B, s.H), float("nan"), dtype=torch.float32, device=dev),
+        status=torch.zeros(1, dtype=torch.int32, device=dev))

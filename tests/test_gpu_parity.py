@@ -1,0 +1,274 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gva_oracle as orc
+from paper_2609_13285_b200 import binding as gb
+from paper_2609_13285_b200 import harness
+from paper_2609_13285_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from tests import gpu_util
+    gpu_util.ensure_built()
+
+
+def U():
+    from tests import gpu_util
+    return gpu_util
+
+
+KERNELS_BF16 = [gb.GVA_KERNEL_FMA, gb.GVA_KERNEL_MMA]
+
+
+def _mma_or_skip(kernel):
+    if kernel == gb.GVA_KERNEL_MMA:
+        try:
+            h = gb.gva_create(H=16, G=4, d_v=64, d_c=64, d_r=16, page_size=64, kernel=gb.GVA_KERNEL_MMA)
+            gb.gva_destroy(h)
+        except gb.GvaError as e:
+            if e.status == gb.GVA_ERR_UNSUPPORTED:
+                pytest.skip("tensor-core kernel not built")
+            raise
+
+
+# ------------------------------------------------------------------ absorb
+@pytest.mark.parametrize("shape,B", [(wl.SHAPE_A, 1), (wl.SHAPE_A, 19), (wl.SHAPE_B, 9)])
+def test_absorb_matches_oracle(shape, B):
+    lens = np.arange(B) * 37 + 5
+    case = wl.make_case("absorb", shape, lens, page_size=64, cache_dtype="bf16", seed=101,
+                        q_pos=(np.arange(B) * 911 + 3) % 20000)
+    dc = harness.upload(case)
+    try:
+        q = dc.absorb().cpu().numpy().astype(np.float64)
+        ref = orc.absorb_case(case)
+        assert np.max(np.abs(q - ref)) <= U().TOL_QABS
+        # rotated slice: fp64 rotation rounded once to f32
+        assert np.array_equal(q[..., shape.d_v:].astype(np.float32), ref[..., shape.d_v:].astype(np.float32))
+    finally:
+        dc.close()
+
+
+# ------------------------------------------------------------------ append (bit exact)
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+def test_append_is_bit_exact_and_touches_nothing_else(dtype, shape):
+    lens = [1, 64, 65, 300, 129, 4000, 8193]
+    case = wl.make_case("append", shape, lens, page_size=64, cache_dtype=dtype, seed=102, extra_pages=3)
+    dc = harness.upload(case)
+    try:
+        dc.append()
+        torch.cuda.synchronize()
+        assert int(dc.status.item()) == 0
+        v_gpu, k_gpu = dc.pools_to_host()
+        assert orc.append_case(case) == 0                  # oracle applies the same append to the host copy
+        assert np.array_equal(v_gpu, case.v_pool)
+        assert np.array_equal(k_gpu, case.kr_pool)
+    finally:
+        dc.close()
+
+
+def test_append_contiguous_and_bad_positions():
+    case = wl.make_case("append_c", wl.SHAPE_A, [100, 128, 7], page_size=64, cache_dtype="bf16", paged=False, seed=103)
+    dc = harness.upload(case)
+    try:
+        dc.append()
+        torch.cuda.synchronize()
+        v_gpu, k_gpu = dc.pools_to_host()
+        orc.append_case(case)
+        assert np.array_equal(v_gpu, case.v_pool) and np.array_equal(k_gpu, case.kr_pool)
+        # position beyond the block table: reported, nothing written
+        before_v = dc.v_pool.clone()
+        dc.append_pos.copy_(torch.tensor([5, 64 * case.max_pages_per_seq, 3], dtype=torch.int32))
+        dc.append()
+        torch.cuda.synchronize()
+        st = int(dc.status.item())
+        assert st & 0xFF == gb.GVA_ERR_SEQ_LEN and st >> 8 == 1
+        changed = (before_v != dc.v_pool).view(case.num_pages, 4, 64, 64).any(dim=(1, 3)).nonzero().tolist()
+        assert sorted(map(tuple, changed)) == [(0, 5), (2 * case.max_pages_per_seq, 3)]
+    finally:
+        dc.close()
+
+
+def test_append_reports_bad_page():
+    case = wl.make_case("append_bad", wl.SHAPE_A, [10, 10], page_size=64, cache_dtype="bf16", seed=104)
+    case.block_table[1, 0] = case.num_pages + 5
+    dc = harness.upload(case)
+    try:
+        before = dc.v_pool.clone()
+        dc.append()
+        torch.cuda.synchronize()
+        st = int(dc.status.item())
+        assert st & 0xFF == gb.GVA_ERR_BAD_PAGE and st >> 8 == 1
+        p0 = int(case.block_table[0, 0])
+        diff = (before != dc.v_pool).view(case.num_pages, -1).any(dim=1).nonzero().flatten().tolist()
+        assert diff == [p0]
+    finally:
+        dc.close()
+
+
+# ------------------------------------------------------------------ decode: the named small configs
+def test_config0_f32_contiguous():
+    err = U().check_decode(wl.config0(), gb.GVA_KERNEL_FMA)
+    assert err <= 1e-5
+
+
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+@pytest.mark.parametrize("num_splits", [0, 1, 2, 7, 16])
+def test_config1_bf16_all_split_counts(kernel, num_splits):
+    _mma_or_skip(kernel)
+    case = wl.config1()
+    dc = harness.upload(case, kernel=kernel)
+    try:
+        U().check_decode(case, kernel, num_splits=num_splits, dc=dc)
+        n = gb.gva_last_num_splits(dc.handle)
+        assert n == (case.B * num_splits if num_splits else n) and n >= 1
+        assert gb.gva_last_kernel(dc.handle) == kernel
+    finally:
+        dc.close()
+
+
+# ------------------------------------------------------------------ decode: edge cases
+EDGE_LENS = [0, 1, 31, 32, 33, 63, 64, 65, 127, 128, 129, 640, 641, 1000]
+
+
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+@pytest.mark.parametrize("num_splits", [0, 1, 5, 40])
+def test_ragged_edge_lengths_poisoned(kernel, shape, num_splits):
+    # lengths around tile and page boundaries, an empty sequence, more splits than tiles;
+    # every slot no live token occupies holds NaN and unused block-table entries are -1
+    _mma_or_skip(kernel)
+    case = wl.make_case("edge", shape, EDGE_LENS, page_size=64, cache_dtype="bf16", seed=201, poison_unused=True,
+                        extra_pages=2)
+    U().check_decode(case, kernel, num_splits=num_splits)
+
+
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+@pytest.mark.parametrize("num_splits", [0, 3])
+def test_ragged_edge_lengths_f32(shape, num_splits):
+    case = wl.make_case("edge32", shape, EDGE_LENS, page_size=64, cache_dtype="f32", seed=202, poison_unused=True)
+    U().check_decode(case, gb.GVA_KERNEL_FMA, num_splits=num_splits)
+
+
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+def test_single_sequence_and_page_sizes(kernel):
+    _mma_or_skip(kernel)
+    for P, paged in ((32, True), (128, True), (256, False), (64, False)):
+        case = wl.make_case("ps", wl.SHAPE_A, [777], page_size=P, cache_dtype="bf16", paged=paged, seed=203 + P,
+                            poison_unused=True)
+        U().check_decode(case, kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+def test_peaked_and_flat_scores(kernel):
+    _mma_or_skip(kernel)
+    # queries x30: near one-hot rows (max subtraction); zero queries: all scores equal
+    case = wl.make_case("peak", wl.SHAPE_A, [500, 2049, 64], page_size=64, cache_dtype="bf16", seed=204, q_gain=30.0)
+    U().check_decode(case, kernel, tight=False)
+    case = wl.make_case("flat", wl.SHAPE_A, [500, 2049, 64], page_size=64, cache_dtype="bf16", seed=205, q_gain=0.0)
+    U().check_decode(case, kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+def test_shared_prefix_pages(kernel):
+    _mma_or_skip(kernel)
+    case = wl.make_case("prefix", wl.SHAPE_A, [300, 300, 200], page_size=64, cache_dtype="bf16", seed=206)
+    case.block_table[1, :2] = case.block_table[0, :2]        # two sequences read the same physical prefix
+    U().check_decode(case, kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+def test_bitwise_reproducible(kernel):
+    _mma_or_skip(kernel)
+    case = wl.make_case("repro", wl.SHAPE_A, [3000, 1234, 64, 5000], page_size=64, cache_dtype="bf16", seed=207)
+    dc = harness.upload(case, kernel=kernel)
+    try:
+        dc.absorb()
+        for ns in (0, 6):
+            a = dc.decode(num_splits=ns)[0].clone()
+            b = dc.decode(num_splits=ns)[0].clone()
+            torch.cuda.synchronize()
+            assert torch.equal(a, b)
+    finally:
+        dc.close()
+
+
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+def test_bad_page_and_bad_length_are_reported_not_read(kernel):
+    _mma_or_skip(kernel)
+    case = wl.make_case("bad", wl.SHAPE_A, [200, 200, 200], page_size=64, cache_dtype="bf16", seed=208)
+    good = U().oracle_for_gpu_q
+    dc = harness.upload(case, kernel=kernel)
+    try:
+        dc.absorb()
+        bt = dc.block_table.clone()
+        dc.block_table[1, 1] = -7
+        dc.decode()
+        torch.cuda.synchronize()
+        st = int(dc.status.item())
+        assert st & 0xFF == gb.GVA_ERR_BAD_PAGE and st >> 8 == 1
+        ref, _ = good(case, dc.q_abs)
+        o = dc.out.cpu().numpy()
+        assert np.max(np.abs(o[[0, 2]] - ref[[0, 2]])) <= U().TOL_TIGHT_MAXABS      # other sequences unaffected
+        assert np.isfinite(o).all()
+        dc.block_table.copy_(bt)
+        dc.status.zero_()
+        lens = dc.seq_lens.clone()
+        lens[2] = case.max_pages_per_seq * 64 + 1
+        dc.decode(seq_lens=lens)
+        torch.cuda.synchronize()
+        st = int(dc.status.item())
+        assert st & 0xFF == gb.GVA_ERR_SEQ_LEN and st >> 8 == 2
+        o = dc.out.cpu().numpy()
+        assert np.all(o[2] == 0) and np.max(np.abs(o[:2] - ref[:2])) <= U().TOL_TIGHT_MAXABS
+    finally:
+        dc.close()
+
+
+def test_host_side_argument_errors():
+    case = wl.make_case("args", wl.SHAPE_A, [100], page_size=64, cache_dtype="bf16", seed=209)
+    dc = harness.upload(case)
+    try:
+        dc.absorb()
+        ws = dc.ensure_workspace(0)
+        rc = gb.gva_decode(dc.handle, dc.cache, dc.q_abs, dc.seq_lens, dc.out, dc.lse, ws, 1, 100, 0, dc.status,
+                           workspace_bytes=128, check=False)
+        assert rc == gb.GVA_ERR_WORKSPACE
+        rc = gb.gva_decode(dc.handle, dc.cache, None, dc.seq_lens, dc.out, dc.lse, ws, 1, 100, 0, dc.status, check=False)
+        assert rc == gb.GVA_ERR_INVALID_ARG
+        rc = gb.gva_decode(dc.handle, dc.cache, dc.q_abs, dc.seq_lens, dc.out, dc.lse, ws, 1, 100, -1, dc.status, check=False)
+        assert rc == gb.GVA_ERR_INVALID_ARG
+        assert gb.gva_decode_workspace_bytes(dc.handle, 1, 100, 0) > 0
+        assert gb.gva_decode_workspace_bytes(dc.handle, 4, 100, 8) >= 4 * 8 * 16 * 66 * 4
+        # lse is optional
+        gb.gva_decode(dc.handle, dc.cache, dc.q_abs, dc.seq_lens, dc.out, None, ws, 1, 100, 0, dc.status)
+        torch.cuda.synchronize()
+    finally:
+        dc.close()
+
+
+# ------------------------------------------------------------------ end to end: absorb -> append -> decode
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+def test_full_step_follows_algorithm_order(kernel):
+    _mma_or_skip(kernel)
+    T = 1000
+    lens = np.full(6, T + 1, dtype=np.int32)
+    case = wl.make_case("step", wl.SHAPE_A, lens, page_size=64, cache_dtype="bf16", seed=210,
+                        q_pos=np.full(6, T), append_pos=np.full(6, T))
+    dc = harness.upload(case, kernel=kernel)
+    try:
+        dc.absorb()
+        dc.append()
+        out, lse = dc.decode()
+        torch.cuda.synchronize()
+        assert orc.append_case(case) == 0                      # oracle: append, then attend over T+1 tokens
+        ref_out, ref_lse = orc.decode_case(case)               # with its own fp64 absorbed query
+        o = out.cpu().numpy().astype(np.float64)
+        assert np.max(np.abs(o - ref_out)) <= 5e-5
+    finally:
+        dc.close()
