@@ -48,7 +48,8 @@ typedef enum {
     GVA_ERR_CUDA = 4,         /* a CUDA runtime/driver call failed (launch error, no sm_100 device, ...) */
     GVA_ERR_BAD_PAGE = 5,     /* [device] block-table entry outside [0, num_pages) in the live range     */
     GVA_ERR_SEQ_LEN = 6,      /* [device] seq_len < 0 or beyond max_pages_per_seq * page_size            */
-    GVA_ERR_TIMEOUT = 7       /* [device] a bounded wait on an asynchronous copy expired                 */
+    GVA_ERR_TIMEOUT = 7,      /* [device] a bounded wait on an asynchronous copy expired                 */
+    GVA_ERR_STATIC_LIMIT = 8  /* gva_decode_static: the request needs more than GVA_STATIC_SCRATCH_BYTES  */
 } gva_status;
 
 typedef enum { GVA_F32 = 0, GVA_BF16 = 1 } gva_dtype;
@@ -140,6 +141,32 @@ int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, 
 int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens,
                float *out, float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len,
                int num_splits, int32_t *dev_status, void *stream);
+
+/* gva_decode for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * entry point exists for the library's users, not for the method.)
+ *
+ * Who this is for: code that runs where cudaMalloc is off limits -- inside a serving loop whose memory
+ * pool was sized and frozen at start-up, under a framework allocator that forbids side allocations, or
+ * in a plug-in that is handed tensors but no allocator.  Such callers cannot provide the split-KV
+ * workspace gva_decode asks for, so here the partial results live in a fixed array compiled into the
+ * library (GVA_STATIC_SCRATCH_BYTES of device memory, held by every GPU that loads the library until
+ * the process exits).  Inputs and outputs are still the caller's, with the same meaning, layout and
+ * error rules as gva_decode; neither this call nor anything it uses calls cudaMalloc, cudaFree or an
+ * allocating library routine.
+ *
+ *  - Limit: if gva_decode_workspace_bytes(h, B, max_seq_len, num_splits) exceeds
+ *    GVA_STATIC_SCRATCH_BYTES the call launches nothing and returns GVA_ERR_STATIC_LIMIT.
+ *  - Set-up: the first call on each device looks up the array's device address (once per device; the
+ *    handle's device must be the current device, otherwise GVA_ERR_INVALID_ARG).  Make that first
+ *    call outside any stream capture.
+ *  - Sharing: every call on a device uses the same array, and it keeps whatever the previous call left.
+ *    Nothing needs clearing -- each call writes every word it later reads -- but two calls that may run
+ *    at the same time on one GPU (different streams, different handles, different threads) race on it:
+ *    keep calls to this entry point stream-ordered per device. */
+#define GVA_STATIC_SCRATCH_BYTES (16u << 20)
+int gva_decode_static(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens,
+                      float *out, float *lse, int B, int max_seq_len, int num_splits, int32_t *dev_status,
+                      void *stream);
 
 /* Matched GQA decode (two cached streams): s_j = q_h K_{j,g(h)}^T / sqrt(d_h), o_h = softmax(s) V_{g(h)},
  * with d_h = cfg.d_v, q [B][H][d_h] f32 already rotated, K cached already rotated.  Same paging,

@@ -16,12 +16,13 @@ LIB_PATH = os.path.join(_HERE, "libgva.so")
 
 GVA_OK = 0
 GVA_ERR_INVALID_ARG, GVA_ERR_UNSUPPORTED, GVA_ERR_WORKSPACE, GVA_ERR_CUDA = 1, 2, 3, 4
-GVA_ERR_BAD_PAGE, GVA_ERR_SEQ_LEN, GVA_ERR_TIMEOUT = 5, 6, 7
+GVA_ERR_BAD_PAGE, GVA_ERR_SEQ_LEN, GVA_ERR_TIMEOUT, GVA_ERR_STATIC_LIMIT = 5, 6, 7, 8
+GVA_STATIC_SCRATCH_BYTES = 16 << 20
 GVA_F32, GVA_BF16 = 0, 1
 GVA_KERNEL_AUTO, GVA_KERNEL_FMA, GVA_KERNEL_MMA = 0, 1, 2
 
 EXPORTS = ["gva_create", "gva_destroy", "gva_decode_workspace_bytes", "gva_absorb_query", "gva_append_cache",
-           "gva_decode", "gqa_decode", "gva_step_scratch_bytes", "gva_decode_step_host", "gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens",
+           "gva_decode", "gva_decode_static", "gqa_decode", "gva_step_scratch_bytes", "gva_decode_step_host", "gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens",
            "gva_status_string"]
 
 
@@ -72,6 +73,7 @@ def load() -> ctypes.CDLL:
     lib.gva_absorb_query.argtypes = [vp, vp, vp, vp, vp, vp, ip, vp]
     lib.gva_append_cache.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, ip, vp, vp]
     lib.gva_decode.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, vp, sz, ip, ip, ip, vp, vp]
+    lib.gva_decode_static.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, ip, ip, ip, vp, vp]
     lib.gqa_decode.argtypes = [vp, ctypes.POINTER(GqaCache), vp, vp, vp, vp, vp, sz, ip, ip, ip, vp, vp]
     for name in ("gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens"):
         getattr(lib, name).argtypes = [vp]
@@ -151,6 +153,18 @@ def gva_decode(handle: int, cache: GvaCache, q_abs, seq_lens, out, lse, workspac
                            _ptr(workspace), wb, int(B), int(max_seq_len), int(num_splits), _ptr(dev_status), _stream())
     if check:
         _check(rc, "gva_decode")
+    return rc
+
+
+def gva_decode_static(handle: int, cache: GvaCache, q_abs, seq_lens, out, lse, B: int, max_seq_len: int,
+                      num_splits: int = 0, dev_status=None, check: bool = True) -> int:
+    """gva_decode without a caller workspace: the partial results use the library's built-in scratch
+    (GVA_STATIC_SCRATCH_BYTES per GPU).  For callers that must not allocate device memory; calls on
+    one GPU must be stream-ordered, and the first call on a device should come before any stream capture."""
+    rc = load().gva_decode_static(handle, ctypes.byref(cache), _ptr(q_abs), _ptr(seq_lens), _ptr(out), _ptr(lse),
+                                  int(B), int(max_seq_len), int(num_splits), _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gva_decode_static")
     return rc
 
 

@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "gva_common.cuh"
@@ -308,6 +309,46 @@ int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const 
                                 static_cast<cudaStream_t>(stream));
 }
 
+// ---- gva_decode without caller scratch ---------------------------------------------------------
+// The split-KV partial results of gva_decode_static live in this array.  In host code the name is
+// only a stand-in for the symbol; the device address is looked up once per device below.
+static __device__ __align__(256) unsigned char g_static_scratch[GVA_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_ptr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on `device` (which must be current); nullptr on failure.
+void *static_scratch_for(int device) {
+    if (device < 0 || device >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        g_static_ptr[device] = ptr;
+    }
+    return g_static_ptr[device];
+}
+}  // namespace
+
+int gva_decode_static(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
+                      float *lse, int B, int max_seq_len, int num_splits, int32_t *dev_status, void *stream) {
+    int rc = check_common(h, B, max_seq_len, num_splits);
+    if (rc != GVA_OK) return rc;
+    if (workspace_layout(h, B, num_splits).total > (size_t)GVA_STATIC_SCRATCH_BYTES) return GVA_ERR_STATIC_LIMIT;
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess) return GVA_ERR_CUDA;
+    if (current != h->device) return GVA_ERR_INVALID_ARG;
+    void *scratch = static_scratch_for(current);
+    if (!scratch) return GVA_ERR_CUDA;
+    return gva_decode(h, cache, q_abs, seq_lens, out, lse, scratch, (size_t)GVA_STATIC_SCRATCH_BYTES, B, max_seq_len,
+                      num_splits, dev_status, stream);
+}
+
 int gqa_decode(gva_handle *h, const gqa_cache *cache, const float *q, const int32_t *seq_lens, float *out, float *lse,
                void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits, int32_t *dev_status,
                void *stream) {
@@ -422,6 +463,7 @@ const char *gva_status_string(int status) {
         case GVA_ERR_BAD_PAGE: return "block-table entry outside the page pool";
         case GVA_ERR_SEQ_LEN: return "sequence length or position outside the block table";
         case GVA_ERR_TIMEOUT: return "bounded wait on an asynchronous copy expired";
+        case GVA_ERR_STATIC_LIMIT: return "request exceeds the built-in scratch of gva_decode_static";
         default: return "unknown status";
     }
 }
