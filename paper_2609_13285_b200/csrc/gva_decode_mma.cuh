@@ -1,0 +1,487 @@
+// Tensor-core split-KV decode kernel over the paged bf16 GVA cache (sm_100a).
+//
+// Why tensor cores at all: per cached token the path needs 4 heads x (d_v + d_r + d_v) multiply-adds
+// per group on 2-byte elements, about 8.5 flop per byte.  On CUDA cores that is more issue slots than
+// an SM has at the HBM rate; on the tensor pipe it is a few percent.
+//
+// Layout of the work
+//   thread block = contiguous range of TILE-token tiles of the batch's cache stream (see gva_common.cuh)
+//   warp g < G   = consumer of value group g (its 4 query heads);  warp G = producer (one elected lane)
+//   producer     : TMA (cp.async.bulk.tensor.2d) loads of the G value tiles and the shared positional-key
+//                  tile of each cache tile into an NSTAGE ring, completion on mbarriers; 128-byte
+//                  swizzle so that ldmatrix is bank-conflict free
+//   consumer     : S^T[token, col] = V_tile . Q^T  with mma.sync.m16n8k16 (bf16 in, f32 accumulate):
+//                  M = 16 tokens, K = value dims then RoPE dims, N = 8 columns = 4 heads x {hi, lo};
+//                  the absorbed f32 query is split q = hi + lo into two bf16 numbers, so the otherwise
+//                  idle half of the N dimension carries the low-order bits and the score keeps ~16
+//                  mantissa bits of q.  Online softmax (base 2) down the token rows with warp shuffles.
+//                  P is split the same way, transposed in registers with movmatrix, and
+//                  O^T[dim, col] += V_tile^T . P^T uses the same shared-memory tile through
+//                  ldmatrix.trans.  Each value byte is read from HBM once and serves all 4 heads.
+//   all waits are bounded: on expiry the block records GVA_ERR_TIMEOUT, drains its copies and exits.
+#pragma once
+
+#include <cuda.h>
+
+#include "gva_common.cuh"
+
+namespace gva {
+
+// ---- host-side state: the driver entry point for tensor-map encoding ---------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+struct MmaHostState {
+    EncodeTiledFn encode;
+};
+
+inline int mma_host_init(MmaHostState *st) {
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn)
+        return GVA_ERR_CUDA;
+    st->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    return GVA_OK;
+}
+
+// ---- PTX wrappers ----------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after about kWaitLimitNs of wall time or when another thread of the block
+// has aborted; never spins without limit.
+constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
+constexpr int kDrainPolls = 1 << 16;
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    unsigned long long t0 = 0;
+    for (unsigned it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 127u) == 127u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(y) : "r"(x));
+    return y;
+}
+// x = hi + lo with hi, lo bf16; returns hi in the low half-word, lo in the high half-word.
+__device__ __forceinline__ uint32_t split_hi_lo(float x) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+    return (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16);
+}
+
+// ---- compile-time geometry -------------------------------------------------------------------------
+template <int DV, int DR, int TILE, bool GQA>
+struct MmaTraits {
+    static constexpr int BOXES = DV / 64;                       // 64-dim (128-byte) boxes per value row
+    static constexpr int VBOX_BYTES = TILE * 128;               // one box of one group
+    static constexpr int VTILE_BYTES = BOXES * VBOX_BYTES;      // one group's tile
+    static constexpr int KR_ROW = DR * 2;                       // 32 or 64 bytes
+    static constexpr int KR_BYTES = TILE * KR_ROW;
+    static constexpr int KSTEPS_V = DV / 16;
+    static constexpr int KSTEPS_R = GQA ? 0 : DR / 16;
+    static constexpr int KSTEPS = KSTEPS_V + KSTEPS_R;
+    static constexpr int MT = DV / 16;                          // output m-tiles
+    static constexpr int CHUNKS = TILE / 16;
+    static constexpr int DQ = GQA ? DV : DV + DR;
+    __host__ __device__ static constexpr int stage_bytes(int G) {
+        return GQA ? 2 * G * VTILE_BYTES : G * VTILE_BYTES + ((KR_BYTES + 1023) & ~1023);
+    }
+    __host__ __device__ static constexpr int tail_bytes(int B, int nstage) {
+        return nstage * 16 /* barriers */ + nstage * 8 /* per-stage meta */ + 16 /* abort */ + (B + 1) * 4;
+    }
+};
+
+// Byte offset of 16-byte chunk `chunk` of row `row` inside a 128-byte-swizzled box (rows of 128 bytes).
+__device__ __forceinline__ uint32_t swz128(int row, int chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
+// Positional-key tile: 32-byte rows use the 32-byte swizzle, 64-byte rows the 64-byte swizzle.
+template <int KR_ROW>
+__device__ __forceinline__ uint32_t swz_kr(int row, int chunk) {
+    if constexpr (KR_ROW == 32) return row * 32 + ((chunk ^ ((row >> 2) & 1)) << 4);
+    else return row * 64 + ((chunk ^ ((row >> 1) & 3)) << 4);
+}
+
+template <int DV, int DR, int TILE, int NSTAGE, bool GQA>
+__global__ void __launch_bounds__(288)
+decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
+    using T = MmaTraits<DV, DR, TILE, GQA>;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    // dynamic shared memory is only guaranteed 16-byte aligned: round up to the swizzle atom
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int G = p.G, H = p.H;
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int stage_bytes = T::stage_bytes(G);
+
+    unsigned char *tail = smem + (size_t)NSTAGE * stage_bytes;
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(tail);
+    uint64_t *empty_bar = full_bar + NSTAGE;
+    int *s_meta = reinterpret_cast<int *>(empty_bar + NSTAGE);   // [NSTAGE][2]: n_valid, sequence
+    volatile int *s_abort = reinterpret_cast<volatile int *>(s_meta + 2 * NSTAGE);
+    int *s_off = s_meta + 2 * NSTAGE + 4;
+
+    if (tid == 0) {
+        for (int s = 0; s < NSTAGE; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), 1);
+            mbar_init(smem_u32(&empty_bar[s]), G);
+        }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    compute_tile_offsets<TILE>(p, s_off);   // ends with __syncthreads(): barriers are initialised for everyone
+    publish_header(p, s_off, TILE);
+    const BlockRange rg = block_range(p, s_off);
+    const int n_tiles = rg.hi - rg.lo;
+
+    if (n_tiles <= 0) {
+        if (rg.rec_fixed >= 0) {
+            for (int i = tid; i < H; i += blockDim.x) {
+                p.rec_ml[((size_t)rg.rec_fixed * H + i) * 2] = -INFINITY;
+                p.rec_ml[((size_t)rg.rec_fixed * H + i) * 2 + 1] = 0.f;
+            }
+        }
+        return;
+    }
+
+    if (warp == G) {
+        // ================================ producer ================================
+        if (lane == 0) {
+            int b = rg.b_first;
+            int issued = 0;
+            bool ok = true;
+            for (int i = 0; i < n_tiles && ok; ++i) {
+                const int st = i % NSTAGE;
+                const uint32_t par = ((i / NSTAGE) & 1) ^ 1;
+                if (!mbar_wait_bounded(smem_u32(&empty_bar[st]), par, s_abort)) {
+                    if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+                    *s_abort = 1;
+                    ok = false;
+                    break;
+                }
+                const int f = rg.lo + i;
+                while (f >= s_off[b + 1]) ++b;
+                const int t0 = (f - s_off[b]) * TILE;
+                int n_valid = min(TILE, p.seq_lens[b] - t0);
+                const int pj = t0 / p.P, slot0 = t0 % p.P;
+                long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
+                                               : (long long)b * p.max_pages + pj;
+                if (page < 0 || page >= p.num_pages) {
+                    report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
+                    page = 0;
+                    n_valid = 0;
+                }
+                s_meta[2 * st] = n_valid;
+                s_meta[2 * st + 1] = b;
+                const uint32_t bar = smem_u32(&full_bar[st]);
+                const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
+                mbar_expect_tx(bar, GQA ? 2 * G * T::VTILE_BYTES : G * T::VTILE_BYTES + T::KR_BYTES);
+                for (int g = 0; g < G; ++g) {
+                    const int row = (int)((page * G + g) * p.P + slot0);
+#pragma unroll
+                    for (int bx = 0; bx < T::BOXES; ++bx)
+                        tma_load_2d(base + g * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, bar);
+                    if constexpr (GQA) {
+#pragma unroll
+                        for (int bx = 0; bx < T::BOXES; ++bx)
+                            tma_load_2d(base + (G + g) * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_k, bx * 64, row, bar);
+                    }
+                }
+                if constexpr (!GQA) tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
+                ++issued;
+            }
+            if (!ok) {
+                // drain: every copy this block started must land before its shared memory is released
+                const int first = max(0, issued - NSTAGE);
+                for (int i = first; i < issued; ++i) {
+                    const int st = i % NSTAGE;
+                    for (int it = 0; it < kDrainPolls; ++it)
+                        if (mbar_try_wait(smem_u32(&full_bar[st]), (i / NSTAGE) & 1)) break;
+                }
+            }
+        }
+    } else {
+        // ================================ consumer: value group `warp` ================================
+        const int g = warp;
+        const int jh = lane & 3;          // head within the group this lane's score/output columns belong to
+        const int r8 = lane >> 2;         // row within an 8-row block
+        uint32_t qf[T::KSTEPS][2];        // B fragments of Q^T: column n = lane/4 = 2*head + {hi, lo}
+        float oacc[T::MT][4];
+        float m_run = -INFINITY, l_run = 0.f;
+        int cur_b = -1;
+        int b = rg.b_first;
+        bool ok = true;
+
+#pragma unroll 1
+        for (int i = 0; i < n_tiles; ++i) {
+            const int st = i % NSTAGE;
+            if (!mbar_wait_bounded(smem_u32(&full_bar[st]), (i / NSTAGE) & 1, s_abort)) {
+                if (!*s_abort && lane == 0) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+                *s_abort = 1;
+                ok = false;
+                break;
+            }
+            const int f = rg.lo + i;
+            while (f >= s_off[b + 1]) ++b;
+            const int n_valid = s_meta[2 * st];
+            if (b != cur_b) {
+                cur_b = b;
+                // absorbed query of head (lane/4)/2, hi or lo part by (lane/4)&1, as mma B fragments
+                const float *q = p.q + ((size_t)b * H + g * kHeadsPerGroup + (r8 >> 1)) * T::DQ;
+                const int part = r8 & 1;
+#pragma unroll
+                for (int kk = 0; kk < T::KSTEPS; ++kk) {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const float2 v = *reinterpret_cast<const float2 *>(q + kk * 16 + half * 8 + 2 * jh);
+                        const uint32_t sx = split_hi_lo(v.x), sy = split_hi_lo(v.y);
+                        qf[kk][half] = part ? ((sx >> 16) | (sy & 0xffff0000u)) : ((sx & 0xffffu) | (sy << 16));
+                    }
+                }
+                m_run = -INFINITY;
+                l_run = 0.f;
+#pragma unroll
+                for (int mt = 0; mt < T::MT; ++mt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) oacc[mt][e] = 0.f;
+            }
+            unsigned char *stage = smem + (size_t)st * stage_bytes;
+            unsigned char *vt = stage + (size_t)g * T::VTILE_BYTES;
+            if (n_valid < TILE) {
+                // rows past the sequence end may hold anything (NaN included): zero them so that 0 * row == 0
+                const int n_zero_chunks = (TILE - n_valid) * 8;
+                for (int c = lane; c < n_zero_chunks * T::BOXES; c += 32) {
+                    const int bx = c / n_zero_chunks, cc = c % n_zero_chunks;
+                    *reinterpret_cast<uint4 *>(vt + bx * T::VBOX_BYTES + (n_valid + cc / 8) * 128 + (cc % 8) * 16) =
+                        make_uint4(0, 0, 0, 0);
+                }
+                // these generic-proxy writes must be ordered before the TMA write that later refills the stage
+                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                __syncwarp();
+            }
+            const uint32_t vt_u32 = smem_u32(vt);
+            const uint32_t ks_u32 = GQA ? smem_u32(stage + (size_t)(G + g) * T::VTILE_BYTES) : vt_u32;
+            const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES);
+
+            // ---- S^T = (score source tile) . Q^T, 16 tokens per m-tile ----
+            float sacc[T::CHUNKS][4];
+#pragma unroll
+            for (int c = 0; c < T::CHUNKS; ++c) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) sacc[c][e] = 0.f;
+                const int row = c * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;   // matrices 0,2: rows 0-7; 1,3: rows 8-15
+#pragma unroll
+                for (int kk = 0; kk < T::KSTEPS_V; ++kk) {
+                    const int chunk = kk * 2 + (lane >> 4);                    // matrices 2,3: second 8 dims
+                    uint32_t a[4];
+                    ldsm_x4(ks_u32 + (chunk >> 3) * T::VBOX_BYTES + swz128(row, chunk & 7), a);
+                    mma_bf16(sacc[c], a, qf[kk][0], qf[kk][1]);
+                }
+                if constexpr (!GQA) {
+#pragma unroll
+                    for (int kk = 0; kk < T::KSTEPS_R; ++kk) {
+                        const int chunk = kk * 2 + (lane >> 4);
+                        uint32_t a[4];
+                        ldsm_x4(kr_u32 + swz_kr<T::KR_ROW>(row, chunk), a);
+                        mma_bf16(sacc[c], a, qf[T::KSTEPS_V + kk][0], qf[T::KSTEPS_V + kk][1]);
+                    }
+                }
+            }
+            // ---- online softmax for head jh over this tile's tokens (rows r8, r8+8 of every m-tile) ----
+            float sc[T::CHUNKS][2];
+            float tmax = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < T::CHUNKS; ++c) {
+                const int t_lo = c * 16 + r8;
+                sc[c][0] = (t_lo < n_valid) ? (sacc[c][0] + sacc[c][1]) * p.scale_log2 : -INFINITY;
+                sc[c][1] = (t_lo + 8 < n_valid) ? (sacc[c][2] + sacc[c][3]) * p.scale_log2 : -INFINITY;
+                tmax = fmaxf(tmax, fmaxf(sc[c][0], sc[c][1]));
+            }
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 4));
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 8));
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
+            const float m_new = fmaxf(m_run, tmax);
+            const bool live = m_new != -INFINITY;
+            const float corr = live ? exp2f(m_run - m_new) : 1.f;
+            m_run = m_new;
+            l_run *= corr;
+#pragma unroll
+            for (int mt = 0; mt < T::MT; ++mt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) oacc[mt][e] *= corr;
+
+            // ---- O^T += V_tile^T . P^T ----
+#pragma unroll
+            for (int c = 0; c < T::CHUNKS; ++c) {
+                const float p0 = live ? exp2f(sc[c][0] - m_new) : 0.f;
+                const float p1 = live ? exp2f(sc[c][1] - m_new) : 0.f;
+                l_run += p0 + p1;
+                // (hi, lo) of p for token row r8 / r8+8 and columns 2*jh, 2*jh+1 -> transpose to B fragments
+                const uint32_t pb0 = movmatrix_trans(split_hi_lo(p0));
+                const uint32_t pb1 = movmatrix_trans(split_hi_lo(p1));
+                const int row = c * 16 + (lane & 7) + (lane >> 4) * 8;          // matrices 0,1: tokens 0-7; 2,3: 8-15
+#pragma unroll
+                for (int mt = 0; mt < T::MT; ++mt) {
+                    const int chunk = mt * 2 + ((lane >> 3) & 1);               // matrices 1,3: second 8 dims
+                    uint32_t a[4];
+                    ldsm_x4_trans(vt_u32 + (chunk >> 3) * T::VBOX_BYTES + swz128(row, chunk & 7), a);
+                    mma_bf16(oacc[mt], a, pb0, pb1);
+                }
+            }
+            // release the stage to the producer
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&empty_bar[st]));
+
+            // ---- segment end: write this (block, sequence) partial ----
+            if (i + 1 == n_tiles || f + 1 >= s_off[b + 1]) {
+                const int rec = (rg.rec_fixed >= 0) ? rg.rec_fixed : (int)blockIdx.x + b;
+                float l = l_run;
+                l += __shfl_xor_sync(0xffffffffu, l, 4);
+                l += __shfl_xor_sync(0xffffffffu, l, 8);
+                l += __shfl_xor_sync(0xffffffffu, l, 16);
+                const size_t rh = (size_t)rec * H + g * kHeadsPerGroup + jh;
+                float *o_dst = p.rec_o + rh * DV;
+#pragma unroll
+                for (int mt = 0; mt < T::MT; ++mt) {
+                    o_dst[mt * 16 + r8] = oacc[mt][0] + oacc[mt][1];
+                    o_dst[mt * 16 + r8 + 8] = oacc[mt][2] + oacc[mt][3];
+                }
+                if (r8 == 0) {
+                    p.rec_ml[rh * 2] = m_run;
+                    p.rec_ml[rh * 2 + 1] = l;
+                }
+            }
+        }
+        (void)ok;
+    }
+    // keep shared memory alive until every warp (and every copy in flight) is done
+    __syncthreads();
+}
+
+// ---- host: support check, tensor maps, launch ------------------------------------------------------
+// Tokens per tile: sized so that three stages of (G value tiles + the score-source tile(s)) fit in shared memory.
+inline int mma_tile_for(const gva_config &cfg, bool gqa) {
+    if (cfg.d_v == 64) return cfg.page_size % 64 == 0 ? 64 : 32;
+    return gqa ? 16 : 32;
+}
+
+inline bool mma_supported(const gva_config &cfg, bool gqa) {
+    return cfg.cache_dtype == GVA_BF16 && cfg.page_size % mma_tile_for(cfg, gqa) == 0;
+}
+
+inline bool encode_map(const MmaHostState &st, CUtensorMap *map, const void *base, uint64_t inner, uint64_t rows,
+                       uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz) {
+    cuuint64_t dims[2] = {inner, rows};
+    cuuint64_t strides[1] = {inner * 2};
+    cuuint32_t box[2] = {box_inner, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return st.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int DV, int DR, int TILE, int NSTAGE, bool GQA>
+int launch_mma_t(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
+                 int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream, int *n_blocks_out) {
+    using T = MmaTraits<DV, DR, TILE, GQA>;
+    const int G = cfg.G;
+    const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
+    if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
+    auto fn = decode_mma_kernel<DV, DR, TILE, NSTAGE, GQA>;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
+    CUtensorMap tm_v, tm_k;
+    const uint64_t vrows = (uint64_t)p.num_pages * G * p.P;
+    if (!encode_map(st, &tm_v, p.v_pool, DV, vrows, 64, TILE, CU_TENSOR_MAP_SWIZZLE_128B)) return GVA_ERR_CUDA;
+    if (GQA) {
+        if (!encode_map(st, &tm_k, p.k_pool, DV, vrows, 64, TILE, CU_TENSOR_MAP_SWIZZLE_128B)) return GVA_ERR_CUDA;
+    } else {
+        if (!encode_map(st, &tm_k, p.kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, TILE,
+                        DR == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B))
+            return GVA_ERR_CUDA;
+    }
+    const int threads = 32 * (G + 1);
+    int grid;
+    if (num_splits > 0) {
+        grid = B * num_splits;
+    } else {
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, smem) != cudaSuccess) return GVA_ERR_CUDA;
+        per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);
+        const long long tiles_ub = (long long)B * ((max_seq_len + TILE - 1) / TILE);
+        long long want = (long long)per_sm * sm_count;
+        if (want > max_blocks) want = max_blocks;
+        grid = (int)(tiles_ub < want ? (tiles_ub < 1 ? 1 : tiles_ub) : want);
+    }
+    fn<<<grid, threads, smem, stream>>>(p, tm_v, tm_k);
+    if (cudaGetLastError() != cudaSuccess) return GVA_ERR_CUDA;
+    *n_blocks_out = grid;
+    return GVA_OK;
+}
+
+template <bool GQA>
+int launch_decode_mma(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p,
+                      int B, int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream, int *n_blocks_out,
+                      int *tile_out) {
+    if (!mma_supported(cfg, GQA)) return GVA_ERR_UNSUPPORTED;
+    // the tensor maps address rows with 32-bit coordinates
+    if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
+    *tile_out = mma_tile_for(cfg, GQA);
+    if (cfg.d_v == 64 && *tile_out == 64)
+        return launch_mma_t<64, 16, 64, 3, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks,
+                                                stream, n_blocks_out);
+    if (cfg.d_v == 64)
+        return launch_mma_t<64, 16, 32, 3, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks,
+                                                stream, n_blocks_out);
+    return launch_mma_t<128, 32, GQA ? 16 : 32, 3, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits,
+                                                        max_blocks, stream, n_blocks_out);
+}
+
+}  // namespace gva

@@ -105,3 +105,53 @@ def upload(case: DecodeCase, device="cuda:0", kernel: int = gb.GVA_KERNEL_AUTO) 
         out=torch.full((B, s.H, s.d_v), float("nan"), dtype=torch.float32, device=dev),
         lse=torch.full((B, s.H), float("nan"), dtype=torch.float32, device=dev),
         status=torch.zeros(1, dtype=torch.int32, device=dev))
+
+
+@dataclass
+class GqaDeviceCase:
+    """Matched GQA decode inputs on the device (from workloads.gqa_case)."""
+    g: dict
+    handle: int
+    k_pool: torch.Tensor
+    v_pool: torch.Tensor
+    block_table: Optional[torch.Tensor]
+    seq_lens: torch.Tensor
+    q: torch.Tensor
+    out: torch.Tensor
+    lse: torch.Tensor
+    status: torch.Tensor
+    workspace: Optional[torch.Tensor] = None
+
+    @property
+    def cache(self) -> gb.GqaCache:
+        return gb.make_gqa_cache(self.k_pool, self.v_pool, self.block_table, self.g["num_pages"],
+                                 self.g["max_pages_per_seq"])
+
+    def decode(self, num_splits: int = 0):
+        B = self.g["B"]
+        max_len = int(self.g["seq_lens"].max()) if B else 0
+        need = gb.gva_decode_workspace_bytes(self.handle, B, max_len, num_splits)
+        if self.workspace is None or self.workspace.numel() < need:
+            self.workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=self.q.device)
+        gb.gqa_decode(self.handle, self.cache, self.q, self.seq_lens, self.out, self.lse, self.workspace, B, max_len,
+                      num_splits, self.status)
+        return self.out, self.lse
+
+    def close(self) -> None:
+        if self.handle:
+            gb.gva_destroy(self.handle)
+            self.handle = 0
+
+
+def upload_gqa(g: dict, device="cuda:0", kernel: int = gb.GVA_KERNEL_AUTO) -> GqaDeviceCase:
+    dev = torch.device(device)
+    d_h = g["d_h"]
+    handle = gb.gva_create(H=g["H"], G=g["G"], d_v=d_h, d_c=d_h, d_r=16 if d_h == 64 else 32, page_size=g["page_size"],
+                           cache_dtype=gb.GVA_BF16 if g["cache_dtype"] == "bf16" else gb.GVA_F32, kernel=kernel,
+                           device=dev.index or 0)
+    B = g["B"]
+    return GqaDeviceCase(g=g, handle=handle, k_pool=_dev(g["k_pool"], dev), v_pool=_dev(g["v_pool"], dev),
+                         block_table=_dev(g["block_table"], dev), seq_lens=_dev(g["seq_lens"], dev), q=_dev(g["q"], dev),
+                         out=torch.full((B, g["H"], d_h), float("nan"), dtype=torch.float32, device=dev),
+                         lse=torch.full((B, g["H"]), float("nan"), dtype=torch.float32, device=dev),
+                         status=torch.zeros(1, dtype=torch.int32, device=dev))
