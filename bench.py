@@ -48,6 +48,8 @@ def make_workload(name: str, rank: int):
         return wl.config2(seed=wl.MASTER_SEED + 2000 + seed_shift)
     if name == "cfg3":
         return wl.config3(seed=wl.MASTER_SEED + 3000 + seed_shift)
+    if name == "cfg2-ncu":   # profiler-sized: 143 MB of cache (> L2), same shapes and paging as cfg2
+        return wl.config2(seed=wl.MASTER_SEED + 2000 + seed_shift, B=16, T=16384)
     if name == "cfg2-small":
         return wl.config2(seed=wl.MASTER_SEED + 2000 + seed_shift, B=8, T=8192)
     raise SystemExit(f"unknown workload {name}")

@@ -32,6 +32,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
              "-Xcompiler", "-fPIC"]
     if os.path.exists(os.path.join(CSRC, "gva_decode_mma.cuh")):
         flags.append("-DGVA_WITH_MMA")
+    flags += os.environ.get("GVA_EXTRA_NVCC_FLAGS", "").split()   # e.g. tuning macros such as -DGVA_MMA_WPG64=1
     if verbose:
         flags += ["-Xptxas", "-v"]
     cmd = [nvcc] + flags + [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]

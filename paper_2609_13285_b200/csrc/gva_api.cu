@@ -94,7 +94,8 @@ int max_blocks_balanced(const gva_handle *h) {
 
 WorkspaceLayout workspace_layout(const gva_handle *h, int B, int num_splits) {
     WorkspaceLayout w;
-    w.n_rec = num_splits > 0 ? B * num_splits : max_blocks_balanced(h) + B;
+    // up to two partial records per (block, sequence): the tensor-core kernel may run two warps per group
+    w.n_rec = 2 * (num_splits > 0 ? B * num_splits : max_blocks_balanced(h) + B);
     w.hdr_bytes = align_up((size_t)(kHdrInts + B + 1) * 4, 256);
     w.rec_o_bytes = align_up((size_t)w.n_rec * h->cfg.H * h->cfg.d_v * 4, 256);
     w.rec_ml_bytes = align_up((size_t)w.n_rec * h->cfg.H * 2 * 4, 256);
@@ -122,6 +123,7 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     p.rec_o = reinterpret_cast<float *>(ws + w.hdr_bytes);
     p.rec_ml = reinterpret_cast<float *>(ws + w.hdr_bytes + w.rec_o_bytes);
     p.num_splits = num_splits;
+    p.rec_mult = 1;
     if (B == 0) return GVA_OK;
 
     int kernel = h->cfg.kernel;
@@ -135,7 +137,7 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     if (kernel == GVA_KERNEL_MMA) {
 #ifdef GVA_WITH_MMA
         int rc = launch_decode_mma<GQA>(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, max_seq_len, num_splits,
-                                        max_blocks_balanced(h), stream, &h->last_num_splits, &h->last_tile);
+                                        max_blocks_balanced(h), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult);
         if (rc != GVA_OK) return rc;
         h->last_kernel = GVA_KERNEL_MMA;
 #else
@@ -158,16 +160,21 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
             const long long tiles_ub = (long long)B * ((max_seq_len + 31) / 32);
             grid = (int)std::min<long long>((long long)per_sm * h->sm_count, std::max<long long>(tiles_ub, 1));
         }
-        plan.fn<<<grid, plan.threads, plan.smem, stream>>>(p);
-        if (cudaGetLastError() != cudaSuccess) return GVA_ERR_CUDA;
+        if (launch_pdl(plan.fn, dim3(grid), dim3(plan.threads), plan.smem, stream, p) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return GVA_ERR_CUDA;
+        }
         h->last_num_splits = grid;
         h->last_kernel = GVA_KERNEL_FMA;
         h->last_tile = 32;
     }
     dim3 cgrid(B, (h->cfg.H + 3) / 4);
-    if (h->cfg.d_v == 64) combine_kernel<64><<<cgrid, 128, 0, stream>>>(p);
-    else combine_kernel<128><<<cgrid, 128, 0, stream>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return GVA_ERR_CUDA;
+    const cudaError_t ce = (h->cfg.d_v == 64) ? launch_pdl(combine_kernel<64>, cgrid, dim3(128), 0, stream, p)
+                                              : launch_pdl(combine_kernel<128>, cgrid, dim3(128), 0, stream, p);
+    if (ce != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GVA_ERR_CUDA;
+    }
     return GVA_OK;
 }
 
@@ -252,9 +259,12 @@ int gva_absorb_query(gva_handle *h, const float *q_c, const float *q_r, const fl
     const gva_config &c = h->cfg;
     const size_t smem = ((size_t)c.d_v * (c.d_c + 1) + (size_t)kAbsorbBatch * c.d_c) * 4;
     dim3 grid(c.H, (B + kAbsorbBatch - 1) / kAbsorbBatch);
-    absorb_kernel<<<grid, 128, smem, static_cast<cudaStream_t>(stream)>>>(q_c, q_r, M, q_pos, q_abs, B, c.H, c.d_v,
-                                                                          c.d_c, c.d_r, h->rope);
-    return cudaGetLastError() == cudaSuccess ? GVA_OK : GVA_ERR_CUDA;
+    if (launch_pdl(absorb_kernel, grid, dim3(kAbsorbThreads), smem, static_cast<cudaStream_t>(stream), q_c, q_r, M, q_pos,
+                   q_abs, B, c.H, c.d_v, c.d_c, c.d_r, h->rope) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GVA_ERR_CUDA;
+    }
+    return GVA_OK;
 }
 
 int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, const float *kr_new,
@@ -266,16 +276,21 @@ int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, 
     if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16)) return GVA_ERR_INVALID_ARG;
     const gva_config &c = h->cfg;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (c.G * c.d_v > kAppendMaxPerThread * 128) return GVA_ERR_UNSUPPORTED;
+    cudaError_t ce;
     if (c.cache_dtype == GVA_BF16)
-        append_kernel<__nv_bfloat16><<<B, 128, 0, s>>>(static_cast<__nv_bfloat16 *>(cache->v_pool),
-                                                       static_cast<__nv_bfloat16 *>(cache->kr_pool), cache->block_table,
-                                                       v_new, kr_new, pos, c.G, c.d_v, c.d_r, c.page_size,
-                                                       cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+        ce = launch_pdl(append_kernel<__nv_bfloat16>, dim3(B), dim3(128), 0, s, static_cast<__nv_bfloat16 *>(cache->v_pool),
+                        static_cast<__nv_bfloat16 *>(cache->kr_pool), cache->block_table, v_new, kr_new, pos, c.G, c.d_v,
+                        c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
     else
-        append_kernel<float><<<B, 128, 0, s>>>(static_cast<float *>(cache->v_pool), static_cast<float *>(cache->kr_pool),
-                                               cache->block_table, v_new, kr_new, pos, c.G, c.d_v, c.d_r, c.page_size,
-                                               cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
-    return cudaGetLastError() == cudaSuccess ? GVA_OK : GVA_ERR_CUDA;
+        ce = launch_pdl(append_kernel<float>, dim3(B), dim3(128), 0, s, static_cast<float *>(cache->v_pool),
+                        static_cast<float *>(cache->kr_pool), cache->block_table, v_new, kr_new, pos, c.G, c.d_v, c.d_r,
+                        c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+    if (ce != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GVA_ERR_CUDA;
+    }
+    return GVA_OK;
 }
 
 int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,

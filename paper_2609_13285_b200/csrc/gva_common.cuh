@@ -31,6 +31,7 @@ struct DecodeParams {
     int32_t *dev_status;         // nullable
     int B, H, G, P, num_pages, max_pages;
     int num_splits;              // 0 = balanced flat partition
+    int rec_mult;                // partial records per (block, sequence): consumer warps per value group
     float scale_log2;            // softmax scale * log2(e)
 };
 
@@ -162,10 +163,38 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 
+// Programmatic dependent launch.  Every kernel of the library is launched with the
+// "programmatic stream serialization" attribute and
+//   - calls grid_dependency_launch() first, so the next kernel in the stream may be scheduled and run
+//     its own set-up while this one works, and
+//   - calls grid_dependency_wait() before its first global-memory access, which blocks until every
+//     earlier kernel in the stream has completed and its writes are visible.
+// Because each kernel waits before it touches memory (and so cannot finish before its predecessor),
+// stream order is preserved for data; only launch latency and set-up overlap.  Kernels of other
+// libraries never trigger early, so they are fully serialised as usual.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
     return y;
+}
+
+// Host: launch with the programmatic-stream-serialization attribute (see above).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*fn)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, static_cast<KArgs>(args)...);
 }
 
 }  // namespace gva

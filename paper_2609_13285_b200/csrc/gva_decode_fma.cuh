@@ -58,6 +58,7 @@ __global__ void __launch_bounds__(256)
 decode_fma_kernel(DecodeParams p) {
     using T = FmaTraits<CT, DV, DR, GQA>;
     constexpr int TILE = T::TILE;
+    grid_dependency_launch();
     extern __shared__ __align__(16) unsigned char smem[];
     const int G = p.G, H = p.H;
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -70,6 +71,7 @@ decode_fma_kernel(DecodeParams p) {
     unsigned char *stages = reinterpret_cast<unsigned char *>(s_nvalid) + 64;
     const int stage_bytes = T::stage_bytes(G);
 
+    grid_dependency_wait();
     compute_tile_offsets<TILE>(p, s_off);
     publish_header(p, s_off, TILE);
     const BlockRange rg = block_range(p, s_off);

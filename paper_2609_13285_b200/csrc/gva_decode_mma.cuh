@@ -150,16 +150,30 @@ __device__ __forceinline__ uint32_t swz_kr(int row, int chunk) {
     else return row * 64 + ((chunk ^ ((row >> 1) & 3)) << 4);
 }
 
-template <int DV, int DR, int TILE, int NSTAGE, bool GQA>
-__global__ void __launch_bounds__(288)
+// {hi, lo} of x as two bf16 numbers with x ~= hi + lo: hi in the low half-word, lo in the high one.
+// Four instructions: round, widen, subtract, round both.
+__device__ __forceinline__ uint32_t split_hi_lo_fast(float x) {
+    uint32_t t, d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(t) : "f"(0.f), "f"(x));          // low half = bf16(x)
+    const float lo = x - __uint_as_float(t << 16);
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(d) : "f"(lo), "f"(x));           // {bf16(lo), bf16(x)}
+    return d;
+}
+
+template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA>
+__global__ void __launch_bounds__(32 * 9)
 decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = MmaTraits<DV, DR, TILE, GQA>;
+    constexpr int CPW = T::CHUNKS / WPG;          // 16-token chunks per consumer warp and tile
+    static_assert(CPW >= 1 && CPW * WPG == T::CHUNKS, "tile must split evenly over the group's warps");
+    grid_dependency_launch();
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     // dynamic shared memory is only guaranteed 16-byte aligned: round up to the swizzle atom
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int G = p.G, H = p.H;
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
+    const int n_consumers = G * WPG;
     const int stage_bytes = T::stage_bytes(G);
 
     unsigned char *tail = smem + (size_t)NSTAGE * stage_bytes;
@@ -172,27 +186,28 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     if (tid == 0) {
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(smem_u32(&full_bar[s]), 1);
-            mbar_init(smem_u32(&empty_bar[s]), G);
+            mbar_init(smem_u32(&empty_bar[s]), n_consumers);
         }
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
+    grid_dependency_wait();
     compute_tile_offsets<TILE>(p, s_off);   // ends with __syncthreads(): barriers are initialised for everyone
     publish_header(p, s_off, TILE);
     const BlockRange rg = block_range(p, s_off);
     const int n_tiles = rg.hi - rg.lo;
 
     if (n_tiles <= 0) {
-        if (rg.rec_fixed >= 0) {
-            for (int i = tid; i < H; i += blockDim.x) {
-                p.rec_ml[((size_t)rg.rec_fixed * H + i) * 2] = -INFINITY;
-                p.rec_ml[((size_t)rg.rec_fixed * H + i) * 2 + 1] = 0.f;
+        if (rg.rec_fixed >= 0) {   // uniform mode: an empty split still owns its records (weight 0 in the merge)
+            for (int i = tid; i < H * WPG; i += blockDim.x) {
+                p.rec_ml[((size_t)rg.rec_fixed * WPG * H + i) * 2] = -INFINITY;
+                p.rec_ml[((size_t)rg.rec_fixed * WPG * H + i) * 2 + 1] = 0.f;
             }
         }
         return;
     }
 
-    if (warp == G) {
+    if (warp == n_consumers) {
         // ================================ producer ================================
         if (lane == 0) {
             int b = rg.b_first;
@@ -224,18 +239,18 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 const uint32_t bar = smem_u32(&full_bar[st]);
                 const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
                 mbar_expect_tx(bar, GQA ? 2 * G * T::VTILE_BYTES : G * T::VTILE_BYTES + T::KR_BYTES);
+                if constexpr (!GQA) tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
                 for (int g = 0; g < G; ++g) {
                     const int row = (int)((page * G + g) * p.P + slot0);
-#pragma unroll
-                    for (int bx = 0; bx < T::BOXES; ++bx)
-                        tma_load_2d(base + g * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, bar);
                     if constexpr (GQA) {
 #pragma unroll
                         for (int bx = 0; bx < T::BOXES; ++bx)
                             tma_load_2d(base + (G + g) * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_k, bx * 64, row, bar);
                     }
+#pragma unroll
+                    for (int bx = 0; bx < T::BOXES; ++bx)
+                        tma_load_2d(base + g * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, bar);
                 }
-                if constexpr (!GQA) tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
                 ++issued;
             }
             if (!ok) {
@@ -249,16 +264,26 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             }
         }
     } else {
-        // ================================ consumer: value group `warp` ================================
-        const int g = warp;
+        // ============ consumer: value group g, token chunks [part*CPW, part*CPW + CPW) of every tile ============
+        const int g = warp / WPG;
+        const int part = warp % WPG;
         const int jh = lane & 3;          // head within the group this lane's score/output columns belong to
         const int r8 = lane >> 2;         // row within an 8-row block
+        // ldmatrix lane addressing inside a 16-token chunk of a 128-byte-swizzled box.  The 16-byte chunk index
+        // is (k-step or m-tile) * 2 + hi, XOR row % 8; the compile-time part is applied as "^ (idx << 5)" below.
+        const int r7 = lane & 7;
+        const int row_qk = r7 + ((lane >> 3) & 1) * 8, hi_qk = lane >> 4;          // matrices: (r0-7,k0-7) (r8-15,k0-7) (r0-7,k8-15) (r8-15,k8-15)
+        const int row_pv = r7 + (lane >> 4) * 8, hi_pv = (lane >> 3) & 1;          // transposed: (t0-7,d0-7) (t0-7,d8-15) (t8-15,d0-7) (t8-15,d8-15)
+        const uint32_t off_qk = row_qk * 128 + ((hi_qk ^ r7) << 4);
+        const uint32_t off_pv = row_pv * 128 + ((hi_pv ^ r7) << 4);
+        const uint32_t off_kr = (T::KR_ROW == 32) ? row_qk * 32 + ((hi_qk ^ ((row_qk >> 2) & 1)) << 4)
+                                                  : row_qk * 64 + ((hi_qk ^ ((row_qk >> 1) & 3)) << 4);
         uint32_t qf[T::KSTEPS][2];        // B fragments of Q^T: column n = lane/4 = 2*head + {hi, lo}
         float oacc[T::MT][4];
         float m_run = -INFINITY, l_run = 0.f;
         int cur_b = -1;
         int b = rg.b_first;
-        bool ok = true;
+        const float scale = p.scale_log2;
 
 #pragma unroll 1
         for (int i = 0; i < n_tiles; ++i) {
@@ -266,7 +291,6 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             if (!mbar_wait_bounded(smem_u32(&full_bar[st]), (i / NSTAGE) & 1, s_abort)) {
                 if (!*s_abort && lane == 0) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
                 *s_abort = 1;
-                ok = false;
                 break;
             }
             const int f = rg.lo + i;
@@ -276,14 +300,14 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 cur_b = b;
                 // absorbed query of head (lane/4)/2, hi or lo part by (lane/4)&1, as mma B fragments
                 const float *q = p.q + ((size_t)b * H + g * kHeadsPerGroup + (r8 >> 1)) * T::DQ;
-                const int part = r8 & 1;
+                const int lo_part = r8 & 1;
 #pragma unroll
                 for (int kk = 0; kk < T::KSTEPS; ++kk) {
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
                         const float2 v = *reinterpret_cast<const float2 *>(q + kk * 16 + half * 8 + 2 * jh);
                         const uint32_t sx = split_hi_lo(v.x), sy = split_hi_lo(v.y);
-                        qf[kk][half] = part ? ((sx >> 16) | (sy & 0xffff0000u)) : ((sx & 0xffffu) | (sy << 16));
+                        qf[kk][half] = lo_part ? ((sx >> 16) | (sy & 0xffff0000u)) : ((sx & 0xffffu) | (sy << 16));
                     }
                 }
                 m_run = -INFINITY;
@@ -295,62 +319,68 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             }
             unsigned char *stage = smem + (size_t)st * stage_bytes;
             unsigned char *vt = stage + (size_t)g * T::VTILE_BYTES;
-            if (n_valid < TILE) {
-                // rows past the sequence end may hold anything (NaN included): zero them so that 0 * row == 0
-                const int n_zero_chunks = (TILE - n_valid) * 8;
+            const int row0 = part * CPW * 16;                 // first token row of this warp's share of the tile
+            const bool ragged = n_valid < row0 + CPW * 16;
+            if (ragged) {
+                // rows past the sequence end may hold anything (NaN included): zero this warp's share of them
+                // so that a zero weight times such a row stays zero
+                const int z0 = max(n_valid, row0);
+                const int n_zero_chunks = (row0 + CPW * 16 - z0) * 8;
                 for (int c = lane; c < n_zero_chunks * T::BOXES; c += 32) {
                     const int bx = c / n_zero_chunks, cc = c % n_zero_chunks;
-                    *reinterpret_cast<uint4 *>(vt + bx * T::VBOX_BYTES + (n_valid + cc / 8) * 128 + (cc % 8) * 16) =
+                    *reinterpret_cast<uint4 *>(vt + bx * T::VBOX_BYTES + (z0 + cc / 8) * 128 + (cc % 8) * 16) =
                         make_uint4(0, 0, 0, 0);
                 }
-                // these generic-proxy writes must be ordered before the TMA write that later refills the stage
+                // generic-proxy writes must be ordered before the TMA write that later refills the stage
                 asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                 __syncwarp();
             }
-            const uint32_t vt_u32 = smem_u32(vt);
-            const uint32_t ks_u32 = GQA ? smem_u32(stage + (size_t)(G + g) * T::VTILE_BYTES) : vt_u32;
-            const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES);
+            const uint32_t vt_u32 = smem_u32(vt) + row0 * 128;
+            const uint32_t ks_u32 = GQA ? smem_u32(stage + (size_t)(G + g) * T::VTILE_BYTES) + row0 * 128 : vt_u32;
+            const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES) + row0 * T::KR_ROW;
 
             // ---- S^T = (score source tile) . Q^T, 16 tokens per m-tile ----
-            float sacc[T::CHUNKS][4];
+            float sacc[CPW][4];
 #pragma unroll
-            for (int c = 0; c < T::CHUNKS; ++c) {
+            for (int c = 0; c < CPW; ++c) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) sacc[c][e] = 0.f;
-                const int row = c * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;   // matrices 0,2: rows 0-7; 1,3: rows 8-15
 #pragma unroll
                 for (int kk = 0; kk < T::KSTEPS_V; ++kk) {
-                    const int chunk = kk * 2 + (lane >> 4);                    // matrices 2,3: second 8 dims
                     uint32_t a[4];
-                    ldsm_x4(ks_u32 + (chunk >> 3) * T::VBOX_BYTES + swz128(row, chunk & 7), a);
+                    ldsm_x4(ks_u32 + (kk >> 2) * T::VBOX_BYTES + c * 2048 + (off_qk ^ ((kk & 3) << 5)), a);
                     mma_bf16(sacc[c], a, qf[kk][0], qf[kk][1]);
                 }
                 if constexpr (!GQA) {
 #pragma unroll
                     for (int kk = 0; kk < T::KSTEPS_R; ++kk) {
-                        const int chunk = kk * 2 + (lane >> 4);
                         uint32_t a[4];
-                        ldsm_x4(kr_u32 + swz_kr<T::KR_ROW>(row, chunk), a);
+                        ldsm_x4(kr_u32 + c * 16 * T::KR_ROW + (off_kr ^ (kk << 5)), a);
                         mma_bf16(sacc[c], a, qf[T::KSTEPS_V + kk][0], qf[T::KSTEPS_V + kk][1]);
                     }
                 }
             }
-            // ---- online softmax for head jh over this tile's tokens (rows r8, r8+8 of every m-tile) ----
-            float sc[T::CHUNKS][2];
+            // ---- online softmax for head jh over this warp's tokens (rows r8, r8+8 of every m-tile) ----
+            float sr[CPW][2];              // raw scores (hi + lo columns summed)
             float tmax = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < T::CHUNKS; ++c) {
-                const int t_lo = c * 16 + r8;
-                sc[c][0] = (t_lo < n_valid) ? (sacc[c][0] + sacc[c][1]) * p.scale_log2 : -INFINITY;
-                sc[c][1] = (t_lo + 8 < n_valid) ? (sacc[c][2] + sacc[c][3]) * p.scale_log2 : -INFINITY;
-                tmax = fmaxf(tmax, fmaxf(sc[c][0], sc[c][1]));
+            for (int c = 0; c < CPW; ++c) {
+                sr[c][0] = sacc[c][0] + sacc[c][1];
+                sr[c][1] = sacc[c][2] + sacc[c][3];
+                if (ragged) {
+                    const int t_lo = row0 + c * 16 + r8;
+                    if (t_lo >= n_valid) sr[c][0] = -INFINITY;
+                    if (t_lo + 8 >= n_valid) sr[c][1] = -INFINITY;
+                }
+                tmax = fmaxf(tmax, fmaxf(sr[c][0], sr[c][1]));
             }
             tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 4));
             tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 8));
             tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
-            const float m_new = fmaxf(m_run, tmax);
+            const float m_new = fmaxf(m_run, tmax * scale);          // scale > 0: max commutes with it
             const bool live = m_new != -INFINITY;
-            const float corr = live ? exp2f(m_run - m_new) : 1.f;
+            const float m_use = live ? m_new : 0.f;                  // keeps (-inf) - (-inf) out of the exponent
+            const float corr = fast_exp2(m_run - m_use);             // 2^(-inf) = 0 for the first live tile
             m_run = m_new;
             l_run *= corr;
 #pragma unroll
@@ -360,19 +390,17 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 
             // ---- O^T += V_tile^T . P^T ----
 #pragma unroll
-            for (int c = 0; c < T::CHUNKS; ++c) {
-                const float p0 = live ? exp2f(sc[c][0] - m_new) : 0.f;
-                const float p1 = live ? exp2f(sc[c][1] - m_new) : 0.f;
+            for (int c = 0; c < CPW; ++c) {
+                const float p0 = fast_exp2(fmaf(sr[c][0], scale, -m_use));
+                const float p1 = fast_exp2(fmaf(sr[c][1], scale, -m_use));
                 l_run += p0 + p1;
                 // (hi, lo) of p for token row r8 / r8+8 and columns 2*jh, 2*jh+1 -> transpose to B fragments
-                const uint32_t pb0 = movmatrix_trans(split_hi_lo(p0));
-                const uint32_t pb1 = movmatrix_trans(split_hi_lo(p1));
-                const int row = c * 16 + (lane & 7) + (lane >> 4) * 8;          // matrices 0,1: tokens 0-7; 2,3: 8-15
+                const uint32_t pb0 = movmatrix_trans(split_hi_lo_fast(p0));
+                const uint32_t pb1 = movmatrix_trans(split_hi_lo_fast(p1));
 #pragma unroll
                 for (int mt = 0; mt < T::MT; ++mt) {
-                    const int chunk = mt * 2 + ((lane >> 3) & 1);               // matrices 1,3: second 8 dims
                     uint32_t a[4];
-                    ldsm_x4_trans(vt_u32 + (chunk >> 3) * T::VBOX_BYTES + swz128(row, chunk & 7), a);
+                    ldsm_x4_trans(vt_u32 + (mt >> 2) * T::VBOX_BYTES + c * 2048 + (off_pv ^ ((mt & 3) << 5)), a);
                     mma_bf16(oacc[mt], a, pb0, pb1);
                 }
             }
@@ -380,9 +408,9 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&empty_bar[st]));
 
-            // ---- segment end: write this (block, sequence) partial ----
+            // ---- segment end: write this (block, sequence, part) partial ----
             if (i + 1 == n_tiles || f + 1 >= s_off[b + 1]) {
-                const int rec = (rg.rec_fixed >= 0) ? rg.rec_fixed : (int)blockIdx.x + b;
+                const int rec = ((rg.rec_fixed >= 0) ? rg.rec_fixed : (int)blockIdx.x + b) * WPG + part;
                 float l = l_run;
                 l += __shfl_xor_sync(0xffffffffu, l, 4);
                 l += __shfl_xor_sync(0xffffffffu, l, 8);
@@ -400,7 +428,6 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 }
             }
         }
-        (void)ok;
     }
     // keep shared memory alive until every warp (and every copy in flight) is done
     __syncthreads();
@@ -412,6 +439,11 @@ inline int mma_tile_for(const gva_config &cfg, bool gqa) {
     if (cfg.d_v == 64) return cfg.page_size % 64 == 0 ? 64 : 32;
     return gqa ? 16 : 32;
 }
+// Consumer warps per value group (each takes an equal share of a tile's 16-token chunks and writes its own partial).
+#ifndef GVA_MMA_WPG64
+#define GVA_MMA_WPG64 2   // build-time tuning knob for the d_v = 64 kernels: 1 or 2
+#endif
+inline int mma_warps_per_group(const gva_config &cfg, bool /*gqa*/) { return cfg.d_v == 64 ? GVA_MMA_WPG64 : 1; }
 
 inline bool mma_supported(const gva_config &cfg, bool gqa) {
     return cfg.cache_dtype == GVA_BF16 && cfg.page_size % mma_tile_for(cfg, gqa) == 0;
@@ -428,14 +460,14 @@ inline bool encode_map(const MmaHostState &st, CUtensorMap *map, const void *bas
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int DV, int DR, int TILE, int NSTAGE, bool GQA>
+template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA>
 int launch_mma_t(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
                  int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream, int *n_blocks_out) {
     using T = MmaTraits<DV, DR, TILE, GQA>;
     const int G = cfg.G;
     const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
-    auto fn = decode_mma_kernel<DV, DR, TILE, NSTAGE, GQA>;
+    auto fn = decode_mma_kernel<DV, DR, TILE, NSTAGE, WPG, GQA>;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
     CUtensorMap tm_v, tm_k;
     const uint64_t vrows = (uint64_t)p.num_pages * G * p.P;
@@ -447,7 +479,7 @@ int launch_mma_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
                         DR == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B))
             return GVA_ERR_CUDA;
     }
-    const int threads = 32 * (G + 1);
+    const int threads = 32 * (G * WPG + 1);
     int grid;
     if (num_splits > 0) {
         grid = B * num_splits;
@@ -460,8 +492,12 @@ int launch_mma_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
         if (want > max_blocks) want = max_blocks;
         grid = (int)(tiles_ub < want ? (tiles_ub < 1 ? 1 : tiles_ub) : want);
     }
-    fn<<<grid, threads, smem, stream>>>(p, tm_v, tm_k);
-    if (cudaGetLastError() != cudaSuccess) return GVA_ERR_CUDA;
+    DecodeParams pp = p;
+    pp.rec_mult = WPG;
+    if (launch_pdl(fn, dim3(grid), dim3(threads), smem, stream, pp, tm_v, tm_k) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GVA_ERR_CUDA;
+    }
     *n_blocks_out = grid;
     return GVA_OK;
 }
@@ -469,19 +505,20 @@ int launch_mma_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
 template <bool GQA>
 int launch_decode_mma(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p,
                       int B, int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream, int *n_blocks_out,
-                      int *tile_out) {
+                      int *tile_out, int *rec_mult_out) {
     if (!mma_supported(cfg, GQA)) return GVA_ERR_UNSUPPORTED;
     // the tensor maps address rows with 32-bit coordinates
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
     *tile_out = mma_tile_for(cfg, GQA);
+    *rec_mult_out = mma_warps_per_group(cfg, GQA);
     if (cfg.d_v == 64 && *tile_out == 64)
-        return launch_mma_t<64, 16, 64, 3, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks,
-                                                stream, n_blocks_out);
+        return launch_mma_t<64, 16, 64, 3, GVA_MMA_WPG64, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks,
+                                                   stream, n_blocks_out);
     if (cfg.d_v == 64)
-        return launch_mma_t<64, 16, 32, 3, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks,
-                                                stream, n_blocks_out);
-    return launch_mma_t<128, 32, GQA ? 16 : 32, 3, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits,
-                                                        max_blocks, stream, n_blocks_out);
+        return launch_mma_t<64, 16, 32, 3, GVA_MMA_WPG64, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks,
+                                                   stream, n_blocks_out);
+    return launch_mma_t<128, 32, GQA ? 16 : 32, 3, 1, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits,
+                                                           max_blocks, stream, n_blocks_out);
 }
 
 }  // namespace gva

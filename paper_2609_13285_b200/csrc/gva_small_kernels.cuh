@@ -2,6 +2,8 @@
 // append (Algorithm 1's append lines) and the log-sum-exp merge of split-KV partial results.
 #pragma once
 
+#include <type_traits>
+
 #include "gva_common.cuh"
 
 namespace gva {
@@ -37,14 +39,17 @@ __device__ __forceinline__ void rope_pair(double x0, double x1, int pos, double 
 }
 
 // ---- absorb --------------------------------------------------------------------------------------
-// grid (H, ceil(B / kAbsorbBatch)), block 128.  M_h is staged once per block in shared memory
-// (row stride d_c + 1 floats) and reused for kAbsorbBatch sequences.
+// grid (H, ceil(B / kAbsorbBatch)), block 256.  M_h is staged once per block in shared memory
+// (row stride d_c + 1 floats, conflict-free for the row-per-thread dot products) with all of a
+// thread's 16-byte loads in flight at once, and reused for kAbsorbBatch sequences.
 constexpr int kAbsorbBatch = 8;
+constexpr int kAbsorbThreads = 256;
 
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kAbsorbThreads)
 absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, const float *__restrict__ M,
               const int32_t *__restrict__ q_pos, float *__restrict__ q_abs, int B, int H, int d_v, int d_c,
               int d_r, RopeTable rope) {
+    grid_dependency_launch();
     extern __shared__ float smem_f[];
     float *sM = smem_f;                            // [d_v][d_c + 1]
     float *sq = smem_f + d_v * (d_c + 1);          // [kAbsorbBatch][d_c]
@@ -53,11 +58,36 @@ absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, cons
     const int nb = min(kAbsorbBatch, B - b0);
     const int tid = threadIdx.x;
     const float *Mh = M + (size_t)h * d_v * d_c;
-    for (int i = tid; i < d_v * d_c; i += 128) sM[(i / d_c) * (d_c + 1) + (i % d_c)] = Mh[i];
-    for (int i = tid; i < nb * d_c; i += 128) sq[i] = q_c[((size_t)(b0 + i / d_c) * H + h) * d_c + (i % d_c)];
+    grid_dependency_wait();
+    const int n_elem = d_v * d_c;
+    if ((d_c & 3) == 0) {
+        const float4 *M4 = reinterpret_cast<const float4 *>(Mh);    // M is 16-byte aligned per head: d_v*d_c*4 % 16 == 0
+        const int n4 = n_elem >> 2;
+        for (int base = 0; base < n4; base += kAbsorbThreads * 4) {
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = base + u * kAbsorbThreads + tid;
+                if (i < n4) v[u] = M4[i];
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = base + u * kAbsorbThreads + tid;
+                if (i < n4) {
+                    const int e = i << 2;
+                    float *dst = sM + (e / d_c) * (d_c + 1) + (e % d_c);
+                    dst[0] = v[u].x; dst[1] = v[u].y; dst[2] = v[u].z; dst[3] = v[u].w;
+                }
+            }
+        }
+    } else {
+        for (int i = tid; i < n_elem; i += kAbsorbThreads) sM[(i / d_c) * (d_c + 1) + (i % d_c)] = Mh[i];
+    }
+    for (int i = tid; i < nb * d_c; i += kAbsorbThreads)
+        sq[i] = q_c[((size_t)(b0 + i / d_c) * H + h) * d_c + (i % d_c)];
     __syncthreads();
     const int dq = d_v + d_r;
-    for (int o = tid; o < nb * d_v; o += 128) {
+    for (int o = tid; o < nb * d_v; o += kAbsorbThreads) {
         const int bb = o / d_v, i = o % d_v;
         const float *mrow = sM + i * (d_c + 1);
         const float *qrow = sq + bb * d_c;
@@ -66,7 +96,7 @@ absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, cons
         q_abs[((size_t)(b0 + bb) * H + h) * dq + i] = acc;
     }
     const int half = d_r / 2;
-    for (int o = tid; o < nb * half; o += 128) {
+    for (int o = tid; o < nb * half; o += kAbsorbThreads) {
         const int bb = o / half, i = o % half;
         const size_t src = ((size_t)(b0 + bb) * H + h) * d_r + 2 * i;
         double y0, y1;
@@ -79,13 +109,31 @@ absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, cons
 
 // ---- append --------------------------------------------------------------------------------------
 // grid B, block 128.  Integer page arithmetic, round-to-nearest-even stores, nothing else touched.
+// The new rows are loaded before the page lookup so that the two dependent lookups (position, then
+// block-table entry) overlap with them.
+constexpr int kAppendMaxPerThread = 8;    // G * d_v <= 8 * 128 elements
+
 template <typename CT>
 __global__ void __launch_bounds__(128)
 append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *__restrict__ block_table,
               const float *__restrict__ v_new, const float *__restrict__ kr_new, const int32_t *__restrict__ pos,
               int G, int d_v, int d_r, int P, int num_pages, int max_pages, int32_t *dev_status, RopeTable rope) {
+    grid_dependency_launch();
     const int b = blockIdx.x;
+    const int n_v = G * d_v;
+    grid_dependency_wait();
     const int t = pos[b];
+    float x[kAppendMaxPerThread];
+#pragma unroll
+    for (int u = 0; u < kAppendMaxPerThread; ++u) {
+        const int i = u * 128 + threadIdx.x;
+        x[u] = (i < n_v) ? v_new[(size_t)b * n_v + i] : 0.f;
+    }
+    float k0 = 0.f, k1 = 0.f;
+    if (threadIdx.x < d_r / 2) {
+        k0 = kr_new[(size_t)b * d_r + 2 * threadIdx.x];
+        k1 = kr_new[(size_t)b * d_r + 2 * threadIdx.x + 1];
+    }
     if (t < 0 || t / P >= max_pages) {
         if (threadIdx.x == 0) report_error(dev_status, GVA_ERR_SEQ_LEN, b);
         return;
@@ -97,17 +145,20 @@ append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *
         return;
     }
     const int slot = t % P;
-    for (int i = threadIdx.x; i < G * d_v; i += 128) {
-        const int g = i / d_v, d = i % d_v;
-        const float x = v_new[(size_t)b * G * d_v + i];
-        const size_t dst = (((size_t)page * G + g) * P + slot) * d_v + d;
-        if constexpr (sizeof(CT) == 2) reinterpret_cast<uint16_t *>(v_pool)[dst] = float_to_bf16_bits(x);
-        else reinterpret_cast<float *>(v_pool)[dst] = x;
+#pragma unroll
+    for (int u = 0; u < kAppendMaxPerThread; ++u) {
+        const int i = u * 128 + threadIdx.x;
+        if (i < n_v) {
+            const int g = i / d_v, d = i % d_v;
+            const size_t dst = (((size_t)page * G + g) * P + slot) * d_v + d;
+            if constexpr (sizeof(CT) == 2) reinterpret_cast<uint16_t *>(v_pool)[dst] = float_to_bf16_bits(x[u]);
+            else reinterpret_cast<float *>(v_pool)[dst] = x[u];
+        }
     }
-    for (int i = threadIdx.x; i < d_r / 2; i += 128) {
+    if (threadIdx.x < d_r / 2) {
+        const int i = threadIdx.x;
         double y0, y1;
-        rope_pair((double)kr_new[(size_t)b * d_r + 2 * i], (double)kr_new[(size_t)b * d_r + 2 * i + 1], t,
-                  rope.inv_freq[i], y0, y1);
+        rope_pair((double)k0, (double)k1, t, rope.inv_freq[i], y0, y1);
         const size_t dst = ((size_t)page * P + slot) * d_r + 2 * i;
         if constexpr (sizeof(CT) == 2) {
             reinterpret_cast<uint16_t *>(kr_pool)[dst] = double_to_bf16_bits(y0);
@@ -123,17 +174,21 @@ append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *
 // grid (B, H / 4), block 128: one warp per (sequence, head).  Records are merged in index order, so
 // the result is reproducible for fixed launch geometry.
 //   m* = max_r m_r ;  L = sum_r l_r 2^(m_r - m*) ;  out = sum_r 2^(m_r - m*) o_r / L ;  lse = (m* + log2 L) ln 2
+// Lanes first fetch one record's (m, l) each, so the weights of 32 records cost one memory round
+// trip; the partial outputs are then read four records at a time.
 template <int DV>
 __global__ void __launch_bounds__(128)
 combine_kernel(DecodeParams p) {
+    grid_dependency_launch();
     const int b = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = blockIdx.y * 4 + warp;
     if (h >= p.H) return;
+    grid_dependency_wait();
     int first, n;
     if (p.num_splits > 0) {
-        first = b * p.num_splits;
-        n = p.num_splits;
+        first = b * p.num_splits * p.rec_mult;
+        n = p.num_splits * p.rec_mult;
     } else {
         const int total = p.hdr[0], n_eff = p.hdr[1];
         const int off0 = p.hdr[kHdrInts + b], off1 = p.hdr[kHdrInts + b + 1];
@@ -142,11 +197,12 @@ combine_kernel(DecodeParams p) {
             first = 0;
         } else {
             const int c0 = range_owner(off0, total, n_eff), c1 = range_owner(off1 - 1, total, n_eff);
-            first = c0 + b;
-            n = c1 - c0 + 1;
+            first = (c0 + b) * p.rec_mult;
+            n = (c1 - c0 + 1) * p.rec_mult;
         }
     }
     constexpr int DPL = DV / 32;
+    using VecT = typename std::conditional<DPL == 2, float2, float4>::type;
     float *o_dst = p.out + ((size_t)b * p.H + h) * DV + lane * DPL;
     float mstar = -INFINITY;
     for (int r = lane; r < n; r += 32) mstar = fmaxf(mstar, p.rec_ml[((size_t)(first + r) * p.H + h) * 2]);
@@ -161,23 +217,41 @@ combine_kernel(DecodeParams p) {
     float L = 0.f, acc[DPL];
 #pragma unroll
     for (int d = 0; d < DPL; ++d) acc[d] = 0.f;
-    for (int r = 0; r < n; ++r) {
-        const size_t rh = (size_t)(first + r) * p.H + h;
-        const float2 ml = *reinterpret_cast<const float2 *>(p.rec_ml + rh * 2);
-        if (ml.x == -INFINITY) continue;   // empty partition: weight 0
-        const float w = exp2f(ml.x - mstar);
-        L = fmaf(ml.y, w, L);
-        const float *o = p.rec_o + rh * DV + lane * DPL;
-        if constexpr (DPL == 2) {
-            const float2 v = *reinterpret_cast<const float2 *>(o);
-            acc[0] = fmaf(w, v.x, acc[0]);
-            acc[1] = fmaf(w, v.y, acc[1]);
-        } else {
-            const float4 v = *reinterpret_cast<const float4 *>(o);
-            acc[0] = fmaf(w, v.x, acc[0]);
-            acc[1] = fmaf(w, v.y, acc[1]);
-            acc[2] = fmaf(w, v.z, acc[2]);
-            acc[3] = fmaf(w, v.w, acc[3]);
+    for (int r0 = 0; r0 < n; r0 += 32) {
+        // lane r: weight of record r0 + r (0 for an empty partition or past the end)
+        float w_lane = 0.f, l_lane = 0.f;
+        if (r0 + lane < n) {
+            const float2 ml = *reinterpret_cast<const float2 *>(p.rec_ml + ((size_t)(first + r0 + lane) * p.H + h) * 2);
+            if (ml.x != -INFINITY) {
+                w_lane = exp2f(ml.x - mstar);
+                l_lane = ml.y;
+            }
+        }
+        const int cnt = min(32, n - r0);
+        for (int r = 0; r < cnt; r += 4) {
+            VecT v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int rr = min(r + u, cnt - 1);      // clamped: duplicates get weight 0 below
+                v[u] = *reinterpret_cast<const VecT *>(p.rec_o + ((size_t)(first + r0 + rr) * p.H + h) * DV + lane * DPL);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int rr = r + u;
+                float w = __shfl_sync(0xffffffffu, w_lane, rr & 31);
+                const float l = __shfl_sync(0xffffffffu, l_lane, rr & 31);
+                if (rr >= cnt || w == 0.f) continue;     // an empty partition's output was never written: skip, do not multiply
+                L = fmaf(l, w, L);
+                if constexpr (DPL == 2) {
+                    acc[0] = fmaf(w, v[u].x, acc[0]);
+                    acc[1] = fmaf(w, v[u].y, acc[1]);
+                } else {
+                    acc[0] = fmaf(w, v[u].x, acc[0]);
+                    acc[1] = fmaf(w, v[u].y, acc[1]);
+                    acc[2] = fmaf(w, v[u].z, acc[2]);
+                    acc[3] = fmaf(w, v[u].w, acc[3]);
+                }
+            }
         }
     }
     const float inv = 1.f / L;
