@@ -176,9 +176,25 @@ int gqa_decode(gva_handle *h, const gqa_cache *cache, const float *q, const int3
                float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
                int32_t *dev_status, void *stream);
 
+/* One whole decode step on device buffers: the same results, bit for bit, as gva_absorb_query ->
+ * gva_append_cache -> gva_decode called in that order (Algorithm 1 from the split queries to the
+ * per-head outputs), in two launches instead of four: absorb and append run in one kernel, and the
+ * decode kernel starts its bookkeeping and its first cache loads while that kernel computes.
+ *   pos      [B] i32  position t of the new token: the append slot and the query position
+ *   seq_lens [B] i32  tokens attended (normally t + 1, so the query sees its own token)
+ *   q_abs    [B][H][d_v+d_r] f32  written by the call (the absorbed queries), then read by the decode
+ *   other arguments as in the three separate calls.
+ * Because the decode kernel reads seq_lens, pos, the block table and cache tiles other than the one
+ * receiving the new token before the fused front kernel has finished, those must not be outputs of
+ * that same call; everything enqueued on the stream before the call is complete before any of it is read. */
+int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const float *q_c, const float *q_r,
+                    const float *v_new, const float *kr_new, const int32_t *pos, const int32_t *seq_lens,
+                    float *q_abs, float *out, float *lse, void *workspace, size_t workspace_bytes, int B,
+                    int max_seq_len, int num_splits, int32_t *dev_status, void *stream);
+
 /* One whole decode step (Algorithm 1 from the split queries to the per-head outputs) for callers whose
  * per-step tensors live in HOST memory: copies the step's inputs to the device, runs
- * gva_absorb_query -> gva_append_cache -> gva_decode, and copies the outputs back, all enqueued on
+ * gva_decode_step, and copies the outputs back, all enqueued on
  * `stream`; the caller synchronises the stream before reading out_host.  The cache and the maps M stay
  * resident on the device (they are state, not per-step input).
  *   [host] q_c_host [B][H][d_c], q_r_host [B][H][d_r], v_new_host [B][G][d_v], kr_new_host [B][d_r] f32,

@@ -22,7 +22,7 @@ GVA_F32, GVA_BF16 = 0, 1
 GVA_KERNEL_AUTO, GVA_KERNEL_FMA, GVA_KERNEL_MMA = 0, 1, 2
 
 EXPORTS = ["gva_create", "gva_destroy", "gva_decode_workspace_bytes", "gva_absorb_query", "gva_append_cache",
-           "gva_decode", "gva_decode_static", "gqa_decode", "gva_step_scratch_bytes", "gva_decode_step_host", "gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens",
+           "gva_decode", "gva_decode_static", "gqa_decode", "gva_decode_step", "gva_step_scratch_bytes", "gva_decode_step_host", "gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens",
            "gva_status_string"]
 
 
@@ -66,6 +66,7 @@ def load() -> ctypes.CDLL:
     lib.gva_destroy.argtypes = [vp]
     lib.gva_decode_workspace_bytes.argtypes = [vp, ip, ip, ip]
     lib.gva_decode_workspace_bytes.restype = sz
+    lib.gva_decode_step.argtypes = [vp, ctypes.POINTER(GvaCache)] + [vp] * 11 + [sz, ip, ip, ip, vp, vp]
     lib.gva_step_scratch_bytes.argtypes = [vp, ip, ip, ip]
     lib.gva_step_scratch_bytes.restype = sz
     lib.gva_decode_step_host.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, ip, ip,
@@ -176,6 +177,17 @@ def gqa_decode(handle: int, cache: GqaCache, q, seq_lens, out, lse, workspace, B
                            _ptr(workspace), wb, int(B), int(max_seq_len), int(num_splits), _ptr(dev_status), _stream())
     if check:
         _check(rc, "gqa_decode")
+    return rc
+
+
+def gva_decode_step(handle: int, cache: GvaCache, M, q_c, q_r, v_new, kr_new, pos, seq_lens, q_abs, out, lse, workspace,
+                    B: int, max_seq_len: int, num_splits: int = 0, dev_status=None, check: bool = True) -> int:
+    rc = load().gva_decode_step(handle, ctypes.byref(cache), _ptr(M), _ptr(q_c), _ptr(q_r), _ptr(v_new), _ptr(kr_new),
+                                _ptr(pos), _ptr(seq_lens), _ptr(q_abs), _ptr(out), _ptr(lse), _ptr(workspace),
+                                workspace.numel() * workspace.element_size(), int(B), int(max_seq_len), int(num_splits),
+                                _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gva_decode_step")
     return rc
 
 

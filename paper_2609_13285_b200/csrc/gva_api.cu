@@ -230,7 +230,11 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
     // the absorb kernel may need more than 48 KB for a 128 x 128 map
     const size_t absorb_smem = ((size_t)cfg->d_v * (cfg->d_c + 1) + (size_t)kAbsorbBatch * cfg->d_c) * 4;
     if (absorb_smem > (size_t)optin ||
-        cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)absorb_smem) != cudaSuccess) {
+        cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)absorb_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(step_front_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)absorb_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(step_front_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)absorb_smem) !=
+            cudaSuccess) {
         delete h;
         return GVA_ERR_CUDA;
     }
@@ -293,9 +297,9 @@ int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, 
     return GVA_OK;
 }
 
-int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
-               float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
-               int32_t *dev_status, void *stream) {
+static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
+                       float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
+                       int32_t *dev_status, void *stream, int early_start, const int32_t *append_pos) {
     int rc = check_common(h, B, max_seq_len, num_splits);
     if (rc != GVA_OK) return rc;
     if (!cache) return GVA_ERR_INVALID_ARG;
@@ -320,8 +324,54 @@ int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const 
     p.num_pages = cache->num_pages;
     p.max_pages = cache->max_pages_per_seq;
     p.scale_log2 = h->scale * kLog2e;
+    p.early_start = early_start;
+    p.append_pos = append_pos;
     return launch_decode<false>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
                                 static_cast<cudaStream_t>(stream));
+}
+
+int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
+               float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
+               int32_t *dev_status, void *stream) {
+    return decode_impl(h, cache, q_abs, seq_lens, out, lse, workspace, workspace_bytes, B, max_seq_len, num_splits,
+                       dev_status, stream, 0, nullptr);
+}
+
+int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const float *q_c, const float *q_r,
+                    const float *v_new, const float *kr_new, const int32_t *pos, const int32_t *seq_lens, float *q_abs,
+                    float *out, float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len,
+                    int num_splits, int32_t *dev_status, void *stream) {
+    int rc = check_common(h, B, max_seq_len, num_splits);
+    if (rc != GVA_OK) return rc;
+    if (B == 0) return GVA_OK;
+    if (!cache || !M || !q_c || !q_r || !v_new || !kr_new || !pos || !seq_lens || !q_abs || !out)
+        return GVA_ERR_INVALID_ARG;
+    if (!cache->v_pool || !cache->kr_pool || cache->num_pages <= 0 || cache->max_pages_per_seq <= 0)
+        return GVA_ERR_INVALID_ARG;
+    if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16) || !aligned(q_abs, 16) || !aligned(out, 16) ||
+        !aligned(M, 16))
+        return GVA_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < workspace_layout(h, B, num_splits).total) return GVA_ERR_WORKSPACE;
+    const gva_config &c = h->cfg;
+    if (c.G * c.d_v > kAppendMaxPerThread * 128) return GVA_ERR_UNSUPPORTED;
+    StepFrontParams a;
+    a.q_c = q_c; a.q_r = q_r; a.M = M; a.v_new = v_new; a.kr_new = kr_new;
+    a.pos = pos; a.block_table = cache->block_table; a.q_abs = q_abs;
+    a.v_pool = cache->v_pool; a.kr_pool = cache->kr_pool; a.dev_status = dev_status;
+    a.B = B; a.H = c.H; a.G = c.G; a.d_v = c.d_v; a.d_c = c.d_c; a.d_r = c.d_r; a.P = c.page_size;
+    a.num_pages = cache->num_pages; a.max_pages = cache->max_pages_per_seq;
+    a.n_absorb = c.H * ((B + kAbsorbBatch - 1) / kAbsorbBatch);
+    const size_t smem = ((size_t)c.d_v * (c.d_c + 1) + (size_t)kAbsorbBatch * c.d_c) * 4;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const cudaError_t ce = (c.cache_dtype == GVA_BF16)
+        ? launch_pdl(step_front_kernel<__nv_bfloat16>, dim3(a.n_absorb + B), dim3(kAbsorbThreads), smem, st, a, h->rope)
+        : launch_pdl(step_front_kernel<float>, dim3(a.n_absorb + B), dim3(kAbsorbThreads), smem, st, a, h->rope);
+    if (ce != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GVA_ERR_CUDA;
+    }
+    return decode_impl(h, cache, q_abs, seq_lens, out, lse, workspace, workspace_bytes, B, max_seq_len, num_splits,
+                       dev_status, stream, 1, pos);
 }
 
 // ---- gva_decode without caller scratch ---------------------------------------------------------
@@ -450,14 +500,10 @@ int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, 
     const int32_t *pos = reinterpret_cast<const int32_t *>(s + L.pos);
     float *q_abs = reinterpret_cast<float *>(s + L.q_abs);
     float *out = reinterpret_cast<float *>(s + L.out);
-    rc = gva_absorb_query(h, reinterpret_cast<const float *>(s + L.q_c), reinterpret_cast<const float *>(s + L.q_r), M,
-                          pos, q_abs, B, stream);
-    if (rc != GVA_OK) return rc;
-    rc = gva_append_cache(h, cache, reinterpret_cast<const float *>(s + L.v_new),
-                          reinterpret_cast<const float *>(s + L.kr_new), pos, B, dev_status, stream);
-    if (rc != GVA_OK) return rc;
-    rc = gva_decode(h, cache, q_abs, reinterpret_cast<const int32_t *>(s + L.lens), out, nullptr, s + L.ws, L.ws_bytes,
-                    B, max_seq_len, num_splits, dev_status, stream);
+    rc = gva_decode_step(h, cache, M, reinterpret_cast<const float *>(s + L.q_c), reinterpret_cast<const float *>(s + L.q_r),
+                         reinterpret_cast<const float *>(s + L.v_new), reinterpret_cast<const float *>(s + L.kr_new), pos,
+                         reinterpret_cast<const int32_t *>(s + L.lens), q_abs, out, nullptr, s + L.ws, L.ws_bytes, B,
+                         max_seq_len, num_splits, dev_status, stream);
     if (rc != GVA_OK) return rc;
     if (cudaMemcpyAsync(out_host, out, (size_t)B * c.H * c.d_v * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return GVA_ERR_CUDA;

@@ -32,6 +32,8 @@ struct DecodeParams {
     int B, H, G, P, num_pages, max_pages;
     int num_splits;              // 0 = balanced flat partition
     int rec_mult;                // partial records per (block, sequence): consumer warps per value group
+    int early_start;             // 1: launched right behind step_front_kernel (see gva_decode_mma.cuh)
+    const int32_t *append_pos;   // early_start: position being appended per sequence (its tile must not be read early)
     float scale_log2;            // softmax scale * log2(e)
 };
 
@@ -137,16 +139,17 @@ __device__ __forceinline__ BlockRange block_range(const DecodeParams &p, const i
 }
 
 // Block 0 publishes the tile offsets for the combine kernel.
-__device__ __forceinline__ void publish_header(const DecodeParams &p, const int *s_off, int tile_tokens) {
+__device__ __forceinline__ void publish_header(const DecodeParams &p, const int *s_off, int tile_tokens,
+                                               int tid = threadIdx.x, int nt = blockDim.x) {
     if (blockIdx.x != 0) return;
     const int total = s_off[p.B];
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
         p.hdr[0] = total;
         p.hdr[1] = (p.num_splits > 0) ? p.B * p.num_splits : partitions_in_use(total, gridDim.x);
         p.hdr[2] = p.num_splits;
         p.hdr[3] = tile_tokens;
     }
-    for (int i = threadIdx.x; i <= p.B; i += blockDim.x) p.hdr[kHdrInts + i] = s_off[i];
+    for (int i = tid; i <= p.B; i += nt) p.hdr[kHdrInts + i] = s_off[i];
 }
 
 // ---- small PTX wrappers ------------------------------------------------------------------------

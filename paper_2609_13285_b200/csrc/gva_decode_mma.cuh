@@ -191,13 +191,20 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    grid_dependency_wait();
+    // Early start (only behind step_front_kernel, which has already waited for everything before it): the
+    // tile bookkeeping and the producer's first loads run while the front kernel computes.  Nothing the front
+    // kernel writes is touched before grid_dependency_wait(): consumers wait before reading the absorbed
+    // query, the producer waits before loading the tile that holds the token being appended, and the
+    // workspace is written only after the wait.
+    const bool early = p.early_start != 0;
+    if (!early) grid_dependency_wait();
     compute_tile_offsets<TILE>(p, s_off);   // ends with __syncthreads(): barriers are initialised for everyone
-    publish_header(p, s_off, TILE);
     const BlockRange rg = block_range(p, s_off);
     const int n_tiles = rg.hi - rg.lo;
 
     if (n_tiles <= 0) {
+        if (early) grid_dependency_wait();
+        publish_header(p, s_off, TILE);
         if (rg.rec_fixed >= 0) {   // uniform mode: an empty split still owns its records (weight 0 in the merge)
             for (int i = tid; i < H * WPG; i += blockDim.x) {
                 p.rec_ml[((size_t)rg.rec_fixed * WPG * H + i) * 2] = -INFINITY;
@@ -206,6 +213,10 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         }
         return;
     }
+    if (warp < n_consumers) {
+        if (early) grid_dependency_wait();
+        publish_header(p, s_off, TILE, tid, n_consumers * 32);
+    }
 
     if (warp == n_consumers) {
         // ================================ producer ================================
@@ -213,8 +224,13 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             int b = rg.b_first;
             int issued = 0;
             bool ok = true;
+            bool waited = !early;
             for (int i = 0; i < n_tiles && ok; ++i) {
                 const int st = i % NSTAGE;
+                if (!waited && i >= NSTAGE) {   // the ring is full: nothing more to gain from running ahead
+                    grid_dependency_wait();
+                    waited = true;
+                }
                 const uint32_t par = ((i / NSTAGE) & 1) ^ 1;
                 if (!mbar_wait_bounded(smem_u32(&empty_bar[st]), par, s_abort)) {
                     if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
@@ -225,11 +241,22 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 const int f = rg.lo + i;
                 while (f >= s_off[b + 1]) ++b;
                 const int t0 = (f - s_off[b]) * TILE;
+                if (!waited) {
+                    const int ap = p.append_pos[b];
+                    if (ap >= t0 && ap < t0 + TILE) {   // this tile receives the new token: it must be complete first
+                        grid_dependency_wait();
+                        waited = true;
+                    }
+                }
                 int n_valid = min(TILE, p.seq_lens[b] - t0);
                 const int pj = t0 / p.P, slot0 = t0 % p.P;
                 long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
                                                : (long long)b * p.max_pages + pj;
                 if (page < 0 || page >= p.num_pages) {
+                    if (!waited) {               // dev_status belongs to the stream-ordered part of the call
+                        grid_dependency_wait();
+                        waited = true;
+                    }
                     report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
                     page = 0;
                     n_valid = 0;

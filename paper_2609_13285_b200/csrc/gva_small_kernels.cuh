@@ -45,20 +45,16 @@ __device__ __forceinline__ void rope_pair(double x0, double x1, int pos, double 
 constexpr int kAbsorbBatch = 8;
 constexpr int kAbsorbThreads = 256;
 
-__global__ void __launch_bounds__(kAbsorbThreads)
-absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, const float *__restrict__ M,
-              const int32_t *__restrict__ q_pos, float *__restrict__ q_abs, int B, int H, int d_v, int d_c,
-              int d_r, RopeTable rope) {
-    grid_dependency_launch();
-    extern __shared__ float smem_f[];
+// One block's share: head h, sequences [b0, b0 + kAbsorbBatch).  All kAbsorbThreads threads must call it.
+__device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, const float *__restrict__ q_r,
+                                             const float *__restrict__ M, const int32_t *__restrict__ q_pos,
+                                             float *__restrict__ q_abs, int B, int H, int d_v, int d_c, int d_r,
+                                             const RopeTable &rope, int h, int b0, float *smem_f) {
     float *sM = smem_f;                            // [d_v][d_c + 1]
     float *sq = smem_f + d_v * (d_c + 1);          // [kAbsorbBatch][d_c]
-    const int h = blockIdx.x;
-    const int b0 = blockIdx.y * kAbsorbBatch;
     const int nb = min(kAbsorbBatch, B - b0);
     const int tid = threadIdx.x;
     const float *Mh = M + (size_t)h * d_v * d_c;
-    grid_dependency_wait();
     const int n_elem = d_v * d_c;
     if ((d_c & 3) == 0) {
         const float4 *M4 = reinterpret_cast<const float4 *>(Mh);    // M is 16-byte aligned per head: d_v*d_c*4 % 16 == 0
@@ -107,26 +103,36 @@ absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, cons
     }
 }
 
+__global__ void __launch_bounds__(kAbsorbThreads)
+absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, const float *__restrict__ M,
+              const int32_t *__restrict__ q_pos, float *__restrict__ q_abs, int B, int H, int d_v, int d_c,
+              int d_r, RopeTable rope) {
+    grid_dependency_launch();
+    extern __shared__ float smem_f[];
+    grid_dependency_wait();
+    absorb_block(q_c, q_r, M, q_pos, q_abs, B, H, d_v, d_c, d_r, rope, blockIdx.x, blockIdx.y * kAbsorbBatch, smem_f);
+}
+
 // ---- append --------------------------------------------------------------------------------------
 // grid B, block 128.  Integer page arithmetic, round-to-nearest-even stores, nothing else touched.
 // The new rows are loaded before the page lookup so that the two dependent lookups (position, then
 // block-table entry) overlap with them.
-constexpr int kAppendMaxPerThread = 8;    // G * d_v <= 8 * 128 elements
+constexpr int kAppendMaxPerThread = 8;    // G * d_v <= 8 * 128 elements (blocks have at least 128 threads)
 
+// One sequence's append.  Every thread of the block must call it (blockDim.x >= 128).
 template <typename CT>
-__global__ void __launch_bounds__(128)
-append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *__restrict__ block_table,
-              const float *__restrict__ v_new, const float *__restrict__ kr_new, const int32_t *__restrict__ pos,
-              int G, int d_v, int d_r, int P, int num_pages, int max_pages, int32_t *dev_status, RopeTable rope) {
-    grid_dependency_launch();
-    const int b = blockIdx.x;
+__device__ __forceinline__ void append_block(CT *__restrict__ v_pool, CT *__restrict__ kr_pool,
+                                             const int32_t *__restrict__ block_table, const float *__restrict__ v_new,
+                                             const float *__restrict__ kr_new, const int32_t *__restrict__ pos, int G,
+                                             int d_v, int d_r, int P, int num_pages, int max_pages, int32_t *dev_status,
+                                             const RopeTable &rope, int b) {
     const int n_v = G * d_v;
-    grid_dependency_wait();
+    const int nt = blockDim.x;
     const int t = pos[b];
     float x[kAppendMaxPerThread];
 #pragma unroll
     for (int u = 0; u < kAppendMaxPerThread; ++u) {
-        const int i = u * 128 + threadIdx.x;
+        const int i = u * nt + threadIdx.x;
         x[u] = (i < n_v) ? v_new[(size_t)b * n_v + i] : 0.f;
     }
     float k0 = 0.f, k1 = 0.f;
@@ -147,7 +153,7 @@ append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *
     const int slot = t % P;
 #pragma unroll
     for (int u = 0; u < kAppendMaxPerThread; ++u) {
-        const int i = u * 128 + threadIdx.x;
+        const int i = u * nt + threadIdx.x;
         if (i < n_v) {
             const int g = i / d_v, d = i % d_v;
             const size_t dst = (((size_t)page * G + g) * P + slot) * d_v + d;
@@ -167,6 +173,47 @@ append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *
             reinterpret_cast<float *>(kr_pool)[dst] = __double2float_rn(y0);
             reinterpret_cast<float *>(kr_pool)[dst + 1] = __double2float_rn(y1);
         }
+    }
+}
+
+template <typename CT>
+__global__ void __launch_bounds__(128)
+append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *__restrict__ block_table,
+              const float *__restrict__ v_new, const float *__restrict__ kr_new, const int32_t *__restrict__ pos,
+              int G, int d_v, int d_r, int P, int num_pages, int max_pages, int32_t *dev_status, RopeTable rope) {
+    grid_dependency_launch();
+    grid_dependency_wait();
+    append_block<CT>(v_pool, kr_pool, block_table, v_new, kr_new, pos, G, d_v, d_r, P, num_pages, max_pages, dev_status,
+                     rope, blockIdx.x);
+}
+
+// ---- fused front of a decode step: absorb and append in one launch ------------------------------------
+// Blocks [0, n_absorb) run absorb_block (head = block % H, batch tile = block / H); blocks
+// [n_absorb, n_absorb + B) run append_block.  The two are independent of each other.  This kernel
+// waits for everything earlier in the stream BEFORE it lets its dependent (the decode kernel) start, so
+// whatever the decode kernel does ahead of its own wait overlaps with this kernel only.
+struct StepFrontParams {
+    const float *q_c, *q_r, *M, *v_new, *kr_new;
+    const int32_t *pos, *block_table;
+    float *q_abs;
+    void *v_pool, *kr_pool;
+    int32_t *dev_status;
+    int B, H, G, d_v, d_c, d_r, P, num_pages, max_pages, n_absorb;
+};
+
+template <typename CT>
+__global__ void __launch_bounds__(kAbsorbThreads)
+step_front_kernel(StepFrontParams a, RopeTable rope) {
+    extern __shared__ float smem_f[];
+    grid_dependency_wait();
+    grid_dependency_launch();
+    if ((int)blockIdx.x < a.n_absorb) {
+        absorb_block(a.q_c, a.q_r, a.M, a.pos, a.q_abs, a.B, a.H, a.d_v, a.d_c, a.d_r, rope, blockIdx.x % a.H,
+                     (blockIdx.x / a.H) * kAbsorbBatch, smem_f);
+    } else {
+        append_block<CT>(static_cast<CT *>(a.v_pool), static_cast<CT *>(a.kr_pool), a.block_table, a.v_new, a.kr_new,
+                         a.pos, a.G, a.d_v, a.d_r, a.P, a.num_pages, a.max_pages, a.dev_status, rope,
+                         blockIdx.x - a.n_absorb);
     }
 }
 

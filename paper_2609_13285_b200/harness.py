@@ -76,6 +76,14 @@ class DeviceCase:
                       self.max_seq_len if max_seq_len is None else max_seq_len, num_splits, self.status)
         return self.out, self.lse
 
+    def step(self, num_splits: int = 0):
+        """absorb + append + decode through the fused entry point (append position = query position)."""
+        ws = self.ensure_workspace(num_splits)
+        gb.gva_decode_step(self.handle, self.cache, self.M, self.q_c, self.q_r, self.v_new, self.kr_new, self.append_pos,
+                           self.seq_lens, self.q_abs, self.out, self.lse, ws, self.case.B, self.max_seq_len, num_splits,
+                           self.status)
+        return self.out, self.lse
+
     def pools_to_host(self):
         v = self.v_pool.cpu().numpy()
         k = self.kr_pool.cpu().numpy()

@@ -272,3 +272,64 @@ def test_full_step_follows_algorithm_order(kernel):
         assert np.max(np.abs(o - ref_out)) <= 5e-5
     finally:
         dc.close()
+
+
+# ------------------------------------------------------------------ fused step entry point
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+def test_fused_step_is_bitwise_the_three_calls(kernel, shape):
+    _mma_or_skip(kernel)
+    lens = np.array([1, 64, 65, 1001, 4096, 130], dtype=np.int32)
+    mk = lambda: wl.make_case("fstep", shape, lens, page_size=64, cache_dtype="bf16", seed=211,
+                              q_pos=lens - 1, append_pos=lens - 1)
+    a, b = harness.upload(mk(), kernel=kernel), harness.upload(mk(), kernel=kernel)
+    try:
+        a.absorb(); a.append(); a.decode()
+        b.step()
+        torch.cuda.synchronize()
+        assert int(a.status.item()) == 0 and int(b.status.item()) == 0
+        assert torch.equal(a.q_abs, b.q_abs)
+        assert torch.equal(a.v_pool, b.v_pool) and torch.equal(a.kr_pool, b.kr_pool)
+        assert torch.equal(a.out, b.out) and torch.equal(a.lse, b.lse)
+    finally:
+        a.close(); b.close()
+
+
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+def test_fused_steps_back_to_back_generate_tokens(kernel):
+    # 24 decode steps in a row with no host synchronisation in between: every step appends one token that the
+    # same step's query must already see (the decode kernel starts early, behind the fused front kernel)
+    _mma_or_skip(kernel)
+    T0, n_steps, B = 120, 24, 5
+    lens0 = np.array([T0, T0 + 7, 63, 64, 1], dtype=np.int32)
+    case = wl.make_case("gen", wl.SHAPE_A, lens0 + n_steps, page_size=64, cache_dtype="bf16", seed=212)
+    rng = np.random.default_rng(5)
+    v_steps = rng.standard_normal((n_steps, B, 4, 64)).astype(np.float32) * 3.0
+    k_steps = rng.standard_normal((n_steps, B, 16)).astype(np.float32)
+    qc_steps = rng.standard_normal((n_steps, B, 16, 64)).astype(np.float32)
+    dc = harness.upload(case, kernel=kernel)
+    try:
+        dv, dk, dq = (torch.from_numpy(x).cuda() for x in (v_steps, k_steps, qc_steps))
+        outs = []
+        for s in range(n_steps):
+            pos = torch.from_numpy(lens0 + s).cuda()
+            dc.append_pos.copy_(pos); dc.q_pos.copy_(pos); dc.seq_lens.copy_(pos + 1)
+            dc.v_new.copy_(dv[s]); dc.kr_new.copy_(dk[s]); dc.q_c.copy_(dq[s])
+            ws = dc.ensure_workspace(0)
+            gb.gva_decode_step(dc.handle, dc.cache, dc.M, dc.q_c, dc.q_r, dc.v_new, dc.kr_new, dc.append_pos, dc.seq_lens,
+                               dc.q_abs, dc.out, dc.lse, ws, B, int(lens0.max()) + n_steps, 0, dc.status)
+            outs.append(dc.out.clone())
+        torch.cuda.synchronize()
+        assert int(dc.status.item()) == 0
+        for s in range(n_steps):                                   # oracle replays the same generation
+            pos = (lens0 + s).astype(np.int32)
+            case.append_pos[:] = pos; case.q_pos[:] = pos
+            case.v_new[:] = v_steps[s]; case.kr_new[:] = k_steps[s]; case.q_c[:] = qc_steps[s]
+            assert orc.append_case(case) == 0
+            ref, _ = orc.decode_case(case, seq_lens=pos + 1)
+            # end to end against the oracle's own fp64 absorbed query; rows here reach |v| ~ 10
+            assert np.max(np.abs(outs[s].cpu().numpy() - ref)) <= 2e-5 * max(1.0, float(np.max(np.abs(ref)))), s
+        v_gpu, k_gpu = dc.pools_to_host()
+        assert np.array_equal(v_gpu, case.v_pool) and np.array_equal(k_gpu, case.kr_pool)
+    finally:
+        dc.close()
