@@ -12,7 +12,7 @@ import os
 from typing import Optional
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libgva.so")
+LIB_PATH = os.environ.get("GVA_LIBRARY", os.path.join(_HERE, "libgva.so"))   # override: load another build of the library
 
 GVA_OK = 0
 GVA_ERR_INVALID_ARG, GVA_ERR_UNSUPPORTED, GVA_ERR_WORKSPACE, GVA_ERR_CUDA = 1, 2, 3, 4

@@ -25,6 +25,8 @@ def _stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
+    if os.environ.get("GVA_LIBRARY"):      # a prebuilt library was named explicitly: nothing to do
+        return os.environ["GVA_LIBRARY"]
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")

@@ -26,10 +26,47 @@ struct gva_handle {
     int last_num_splits;
     int last_kernel;
     int last_tile;
+    int32_t *ticket;         // this handle's dynamic-unit ticket (device, inside the library image)
+    int ticket_slot;
 #ifdef GVA_WITH_MMA
     MmaHostState mma;
 #endif
 };
+
+// ---- dynamic-unit tickets --------------------------------------------------------------------------
+// The tensor-core kernel hands out the tail of the tile list through an atomic counter that must be zero
+// when a decode kernel starts.  The counters live inside the library image (zero at load, reset by the
+// combine kernel after every call), one per handle, so no caller buffer has to be initialised and no
+// caller can overwrite them.  Calls on one handle are stream-ordered by contract, so a counter has one user at a time.
+constexpr int kMaxHandles = 4096;
+static __device__ int32_t g_tickets[kMaxHandles];
+
+namespace {
+std::mutex g_slot_mutex;
+bool g_slot_used[kMaxHandles] = {};
+
+// Reserves a slot and resolves its device address (the device must be current).  -1 on failure.
+int acquire_ticket_slot(int /*device*/, int32_t **addr) {
+    void *base = nullptr;
+    if (cudaGetSymbolAddress(&base, g_tickets) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -1;
+    }
+    std::lock_guard<std::mutex> lock(g_slot_mutex);
+    for (int i = 0; i < kMaxHandles; ++i)
+        if (!g_slot_used[i]) {
+            g_slot_used[i] = true;
+            *addr = static_cast<int32_t *>(base) + i;
+            return i;
+        }
+    return -1;
+}
+void release_ticket_slot(int slot) {
+    if (slot < 0 || slot >= kMaxHandles) return;
+    std::lock_guard<std::mutex> lock(g_slot_mutex);
+    g_slot_used[slot] = false;
+}
+}  // namespace
 
 namespace {
 
@@ -92,10 +129,18 @@ int max_blocks_balanced(const gva_handle *h) {
     return 4 * h->sm_count;
 }
 
+// Upper bound on units (records per sequence come on top): the CUDA-core kernel uses one unit per block; the
+// tensor-core kernel runs at most 2 blocks per SM (d_v = 64) or 1 (d_v = 128), each range with up to 4 tail units.
+int max_units_balanced(const gva_handle *h) {
+    const int mma_blocks = (h->cfg.d_v == 64 ? 2 : 1) * h->sm_count;
+    const int a = max_blocks_balanced(h), b = unit_bound(mma_blocks);
+    return a > b ? a : b;
+}
+
 WorkspaceLayout workspace_layout(const gva_handle *h, int B, int num_splits) {
     WorkspaceLayout w;
     // up to two partial records per (block, sequence): the tensor-core kernel may run two warps per group
-    w.n_rec = 2 * (num_splits > 0 ? B * num_splits : max_blocks_balanced(h) + B);
+    w.n_rec = 2 * (num_splits > 0 ? B * num_splits : max_units_balanced(h) + B);
     w.hdr_bytes = align_up((size_t)(kHdrInts + B + 1) * 4, 256);
     w.rec_o_bytes = align_up((size_t)w.n_rec * h->cfg.H * h->cfg.d_v * 4, 256);
     w.rec_ml_bytes = align_up((size_t)w.n_rec * h->cfg.H * 2 * 4, 256);
@@ -125,6 +170,7 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     p.num_splits = num_splits;
     p.rec_mult = 1;
     if (B == 0) return GVA_OK;
+
 
     int kernel = h->cfg.kernel;
     if (kernel == GVA_KERNEL_AUTO) {
@@ -168,11 +214,12 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
         h->last_kernel = GVA_KERNEL_FMA;
         h->last_tile = 32;
     }
-    dim3 cgrid(B, (h->cfg.H + 3) / 4);
-    const cudaError_t ce = (h->cfg.d_v == 64) ? launch_pdl(combine_kernel<64>, cgrid, dim3(128), 0, stream, p)
-                                              : launch_pdl(combine_kernel<128>, cgrid, dim3(128), 0, stream, p);
+    const cudaError_t ce = (h->cfg.d_v == 64)
+        ? launch_pdl(combine_kernel<64, 4>, dim3(B, h->cfg.H), dim3(128), 0, stream, p)
+        : launch_pdl(combine_kernel<128, 1>, dim3(B, (h->cfg.H + 3) / 4), dim3(128), 0, stream, p);
     if (ce != cudaSuccess) {
         (void)cudaGetLastError();
+        (void)cudaMemsetAsync(h->ticket, 0, sizeof(int32_t), stream);   // the merge that would have reset it never ran
         return GVA_ERR_CUDA;
     }
     return GVA_OK;
@@ -220,6 +267,11 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
     h->last_num_splits = 0;
     h->last_kernel = 0;
     h->last_tile = 0;
+    h->ticket_slot = acquire_ticket_slot(device, &h->ticket);
+    if (h->ticket_slot < 0) {
+        delete h;
+        return GVA_ERR_CUDA;
+    }
 #ifdef GVA_WITH_MMA
     int rc = mma_host_init(&h->mma);
     if (rc != GVA_OK) {
@@ -244,6 +296,7 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
 
 int gva_destroy(gva_handle *h) {
     if (!h) return GVA_ERR_INVALID_ARG;
+    release_ticket_slot(h->ticket_slot);
     delete h;
     return GVA_OK;
 }
@@ -326,6 +379,7 @@ static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs
     p.scale_log2 = h->scale * kLog2e;
     p.early_start = early_start;
     p.append_pos = append_pos;
+    p.ticket = h->ticket;
     return launch_decode<false>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
                                 static_cast<cudaStream_t>(stream));
 }
@@ -441,6 +495,7 @@ int gqa_decode(gva_handle *h, const gqa_cache *cache, const float *q, const int3
     p.num_pages = cache->num_pages;
     p.max_pages = cache->max_pages_per_seq;
     p.scale_log2 = (float)(1.0 / std::sqrt((double)c.d_v)) * kLog2e;
+    p.ticket = h->ticket;
     return launch_decode<true>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
                                static_cast<cudaStream_t>(stream));
 }

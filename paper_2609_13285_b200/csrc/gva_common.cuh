@@ -11,7 +11,13 @@
 namespace gva {
 
 constexpr int kHeadsPerGroup = 4;   // H / G of every instantiated kernel
-constexpr int kHdrInts = 8;         // workspace header: [0]=total tiles, [1]=partitions in use, [2]=num_splits, [3]=tile tokens
+// Workspace header (ints): the partition of the flat tile list into units, published by block 0 of
+// the decode kernel for the combine kernel.
+constexpr int kHdrInts = 8;
+constexpr int kHdrTotal = 0;        // total tiles
+constexpr int kHdrRanges = 1;       // equal contiguous ranges the tile list is cut into
+constexpr int kHdrU = 2;            // tail units per range
+constexpr int kHdrK = 3;            // tiles per tail unit
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -29,6 +35,7 @@ struct DecodeParams {
     float *out;                  // [B][H][d_v]
     float *lse;                  // nullable
     int32_t *dev_status;         // nullable
+    int32_t *ticket;             // next dynamic unit to hand out; zero between calls
     int B, H, G, P, num_pages, max_pages;
     int num_splits;              // 0 = balanced flat partition
     int rec_mult;                // partial records per (block, sequence): consumer warps per value group
@@ -97,6 +104,84 @@ __host__ __device__ __forceinline__ int range_owner(int x, int total_tiles, int 
     return (int)((((long long)x + 1) * n_eff + total_tiles - 1) / total_tiles) - 1;
 }
 
+// ---- units ---------------------------------------------------------------------------------------
+// Balanced mode cuts the flat tile list into n_ranges equal contiguous ranges (one per thread block), and
+// each range into 1 + U units: a static head that its block always processes, and U tail units of K tiles
+// each that are handed out through an atomic ticket to whichever block gets there first.  Blocks that stream
+// slower than the rest therefore lose their tails to faster ones instead of setting the kernel time.
+//   unit id  u = range * (U + 1) + j   (j = 0 head, j >= 1 tails): ordered by tile position, so the units that
+//   intersect a sequence are one contiguous run, and (unit u, sequence b) -> record u + b is collision-free
+//   (u and b never decrease along the tile list and one of them grows at every cut).
+struct UnitPlan {
+    int total, n_ranges, U, K;
+};
+
+// size of tail j (1-based): K, K/2, K/4, ... (at least 1), so the last pieces handed out are the smallest
+__host__ __device__ __forceinline__ int tail_size(const UnitPlan &u, int j) {
+    const int k = u.K >> (j - 1);
+    return k > 0 ? k : 1;
+}
+__host__ __device__ __forceinline__ int tail_total(const UnitPlan &u) {
+    int d = 0;
+    for (int j = 1; j <= u.U; ++j) d += tail_size(u, j);
+    return d;
+}
+
+__host__ __device__ __forceinline__ UnitPlan make_unit_plan(int total, int n_blocks, bool allow_dynamic) {
+    UnitPlan u;
+    u.total = total;
+    u.n_ranges = partitions_in_use(total, n_blocks);
+    u.U = 0;
+    u.K = 1;
+    const int per_block = total / (n_blocks > 0 ? n_blocks : 1);
+#ifndef GVA_TAIL_DEN
+#define GVA_TAIL_DEN 16     // build-time knobs: the first tail is 1/GVA_TAIL_DEN of a range, each next one half of that
+#define GVA_TAIL_UNITS 3
+#endif
+    if (allow_dynamic && per_block >= 8) {
+        u.U = GVA_TAIL_UNITS;
+        u.K = per_block / GVA_TAIL_DEN;
+        if (u.K < 1) u.K = 1;
+    }
+    return u;
+}
+__host__ __device__ __forceinline__ int plan_units(const UnitPlan &u) { return u.n_ranges * (u.U + 1); }
+// tiles [lo, hi) of unit (range c, part j)
+__host__ __device__ __forceinline__ void unit_range(const UnitPlan &u, int c, int j, int &lo, int &hi) {
+    const int r0 = range_begin(c, u.total, u.n_ranges), r1 = range_begin(c + 1, u.total, u.n_ranges);
+    const int len = r1 - r0;
+    const int dt = tail_total(u);
+    const int d = len < dt ? len : dt;
+    const int head = len - d;
+    if (j == 0) {
+        lo = r0;
+        hi = r0 + head;
+    } else {
+        lo = r0 + head;
+        for (int k = 1; k < j; ++k) lo += tail_size(u, k);
+        hi = lo + tail_size(u, j);
+        if (lo > r1) lo = r1;
+        if (hi > r1) hi = r1;
+    }
+}
+__host__ __device__ __forceinline__ int unit_of_tile(const UnitPlan &u, int x) {
+    const int c = range_owner(x, u.total, u.n_ranges);
+    const int r0 = range_begin(c, u.total, u.n_ranges), r1 = range_begin(c + 1, u.total, u.n_ranges);
+    const int len = r1 - r0;
+    const int dt = tail_total(u);
+    const int d = len < dt ? len : dt;
+    int rel = x - r0 - (len - d);
+    if (rel < 0) return c * (u.U + 1);
+    int j = 1;
+    while (j < u.U && rel >= tail_size(u, j)) {
+        rel -= tail_size(u, j);
+        ++j;
+    }
+    return c * (u.U + 1) + j;
+}
+// upper bound on units for any total (for sizing the workspace)
+__host__ __device__ __forceinline__ int unit_bound(int n_blocks) { return 5 * n_blocks; }
+
 // This block's flat tile range and, in uniform mode, its fixed record.
 struct BlockRange {
     int lo, hi;      // flat tiles [lo, hi)
@@ -113,6 +198,7 @@ __device__ __forceinline__ int seq_of_tile(const int *s_off, int B, int x) {
     return lo;
 }
 
+// Static-only partition (CUDA-core kernel, and uniform mode of both kernels).
 __device__ __forceinline__ BlockRange block_range(const DecodeParams &p, const int *s_off) {
     BlockRange r;
     const int total = s_off[p.B];
@@ -138,16 +224,15 @@ __device__ __forceinline__ BlockRange block_range(const DecodeParams &p, const i
     return r;
 }
 
-// Block 0 publishes the tile offsets for the combine kernel.
-__device__ __forceinline__ void publish_header(const DecodeParams &p, const int *s_off, int tile_tokens,
+// Block 0 publishes the tile offsets and the unit plan for the combine kernel.
+__device__ __forceinline__ void publish_header(const DecodeParams &p, const int *s_off, const UnitPlan &plan,
                                                int tid = threadIdx.x, int nt = blockDim.x) {
     if (blockIdx.x != 0) return;
-    const int total = s_off[p.B];
     if (tid == 0) {
-        p.hdr[0] = total;
-        p.hdr[1] = (p.num_splits > 0) ? p.B * p.num_splits : partitions_in_use(total, gridDim.x);
-        p.hdr[2] = p.num_splits;
-        p.hdr[3] = tile_tokens;
+        p.hdr[kHdrTotal] = plan.total;
+        p.hdr[kHdrRanges] = plan.n_ranges;
+        p.hdr[kHdrU] = plan.U;
+        p.hdr[kHdrK] = plan.K;
     }
     for (int i = tid; i <= p.B; i += nt) p.hdr[kHdrInts + i] = s_off[i];
 }

@@ -137,7 +137,7 @@ struct MmaTraits {
         return GQA ? 2 * G * VTILE_BYTES : G * VTILE_BYTES + ((KR_BYTES + 1023) & ~1023);
     }
     __host__ __device__ static constexpr int tail_bytes(int B, int nstage) {
-        return nstage * 16 /* barriers */ + nstage * 8 /* per-stage meta */ + 16 /* abort */ + (B + 1) * 4;
+        return nstage * 16 /* barriers */ + nstage * 16 /* per-stage meta */ + 16 /* abort */ + (B + 1) * 4;
     }
 };
 
@@ -160,6 +160,14 @@ __device__ __forceinline__ uint32_t split_hi_lo_fast(float x) {
     return d;
 }
 
+// Per-stage message from the producer to the consumers.
+struct StageMeta {
+    int n_valid;   // live tokens in the tile; -1 = no more tiles for this block
+    int b;         // sequence
+    int rec;       // partial record this tile's segment belongs to (before the per-warp multiplier)
+    int flags;     // bit 0: first tile of its segment, bit 1: last tile of its segment
+};
+
 template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA>
 __global__ void __launch_bounds__(32 * 9)
 decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
@@ -179,9 +187,9 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     unsigned char *tail = smem + (size_t)NSTAGE * stage_bytes;
     uint64_t *full_bar = reinterpret_cast<uint64_t *>(tail);
     uint64_t *empty_bar = full_bar + NSTAGE;
-    int *s_meta = reinterpret_cast<int *>(empty_bar + NSTAGE);   // [NSTAGE][2]: n_valid, sequence
-    volatile int *s_abort = reinterpret_cast<volatile int *>(s_meta + 2 * NSTAGE);
-    int *s_off = s_meta + 2 * NSTAGE + 4;
+    StageMeta *s_meta = reinterpret_cast<StageMeta *>(empty_bar + NSTAGE);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(s_meta + NSTAGE);
+    int *s_off = reinterpret_cast<int *>(s_meta + NSTAGE) + 4;
 
     if (tid == 0) {
         for (int s = 0; s < NSTAGE; ++s) {
@@ -190,6 +198,9 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         }
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        // fetch the two tensor-map descriptors now, not at the first copy
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
     }
     // Early start (only behind step_front_kernel, which has already waited for everything before it): the
     // tile bookkeeping and the producer's first loads run while the front kernel computes.  Nothing the front
@@ -199,86 +210,140 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     const bool early = p.early_start != 0;
     if (!early) grid_dependency_wait();
     compute_tile_offsets<TILE>(p, s_off);   // ends with __syncthreads(): barriers are initialised for everyone
-    const BlockRange rg = block_range(p, s_off);
-    const int n_tiles = rg.hi - rg.lo;
-
-    if (n_tiles <= 0) {
-        if (early) grid_dependency_wait();
-        publish_header(p, s_off, TILE);
-        if (rg.rec_fixed >= 0) {   // uniform mode: an empty split still owns its records (weight 0 in the merge)
+    const bool uniform = p.num_splits > 0;
+    // Tail stealing pays where two blocks share an SM and their speeds differ by +-20 % (d_v = 64: measured -2.7 us
+    // of 100 on the long-context workload); with one block per SM (d_v = 128) speeds differ by +-4 % and the extra
+    // partial records cost more than the balance gains (measured +3.9 us of 180), so there the ranges stay static.
+#ifndef GVA_MMA_DYNAMIC_TAIL
+#define GVA_MMA_DYNAMIC_TAIL 1   // build-time knob: 0 = equal static ranges only
+#endif
+    const UnitPlan plan = make_unit_plan(s_off[p.B], gridDim.x, GVA_MMA_DYNAMIC_TAIL != 0 && DV == 64);
+    BlockRange rg;
+    rg.lo = rg.hi = 0;
+    rg.rec_fixed = -1;
+    rg.b_first = 0;
+    int first_unit = -1;
+    if (uniform) {
+        rg = block_range(p, s_off);
+        if (rg.hi <= rg.lo) {   // an empty split still owns its records (weight 0 in the merge)
+            if (early) grid_dependency_wait();
             for (int i = tid; i < H * WPG; i += blockDim.x) {
                 p.rec_ml[((size_t)rg.rec_fixed * WPG * H + i) * 2] = -INFINITY;
                 p.rec_ml[((size_t)rg.rec_fixed * WPG * H + i) * 2 + 1] = 0.f;
             }
+            return;
+        }
+    } else if ((int)blockIdx.x < plan.n_ranges) {
+        first_unit = blockIdx.x * (plan.U + 1);          // the head of this block's own range
+        unit_range(plan, blockIdx.x, 0, rg.lo, rg.hi);
+        rg.b_first = (rg.lo < rg.hi) ? seq_of_tile(s_off, p.B, rg.lo) : 0;
+    }
+    const int n_tickets = uniform ? 0 : plan.n_ranges * plan.U;    // tail units on offer
+    if (!uniform && first_unit < 0 && n_tickets == 0) {   // more blocks than ranges and no tails to share
+        if (blockIdx.x == 0) {                            // (total == 0): the header is still needed by the merge
+            if (early) grid_dependency_wait();
+            publish_header(p, s_off, plan);
         }
         return;
     }
-    if (warp < n_consumers) {
-        if (early) grid_dependency_wait();
-        publish_header(p, s_off, TILE, tid, n_consumers * 32);
-    }
 
     if (warp == n_consumers) {
-        // ================================ producer ================================
+        // ================================ producer (one elected lane) ================================
         if (lane == 0) {
-            int b = rg.b_first;
-            int issued = 0;
-            bool ok = true;
             bool waited = !early;
-            for (int i = 0; i < n_tiles && ok; ++i) {
-                const int st = i % NSTAGE;
-                if (!waited && i >= NSTAGE) {   // the ring is full: nothing more to gain from running ahead
-                    grid_dependency_wait();
-                    waited = true;
+            bool ok = true;
+            int issued = 0;       // tiles issued by this block: ring position
+            int lo = rg.lo, hi = rg.hi, unit = first_unit;
+            int b = rg.b_first;
+            for (;;) {
+                // the next tail unit is requested while this one is being issued (the ticket is reset
+                // by the previous call's combine kernel: never touch it before grid_dependency_wait())
+                int ticket = -1;
+                bool asked = n_tickets == 0;
+                for (int f = lo; f < hi && ok; ++f) {
+                    const int st = issued % NSTAGE;
+                    if (!waited && issued >= NSTAGE) {   // the ring is full: nothing more to gain from running ahead
+                        grid_dependency_wait();
+                        waited = true;
+                    }
+                    if (!asked && waited && hi - f <= 2) {   // late, so that tails go to whoever really is ahead
+                        ticket = atomicAdd(p.ticket, 1);
+                        asked = true;
+                    }
+                    while (f >= s_off[b + 1]) ++b;
+                    const int t0 = (f - s_off[b]) * TILE;
+                    if (!waited) {
+                        const int ap = p.append_pos[b];
+                        if (ap >= t0 && ap < t0 + TILE) {   // this tile receives the new token: it must be complete first
+                            grid_dependency_wait();
+                            waited = true;
+                        }
+                    }
+                    int n_valid = min(TILE, p.seq_lens[b] - t0);
+                    const int pj = t0 / p.P, slot0 = t0 % p.P;
+                    long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
+                                                   : (long long)b * p.max_pages + pj;
+                    if (page < 0 || page >= p.num_pages) {
+                        report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
+                        page = 0;
+                        n_valid = 0;
+                    }
+                    // the bookkeeping above overlaps with the wait for the stage to be released
+                    if (!mbar_wait_bounded(smem_u32(&empty_bar[st]), ((issued / NSTAGE) & 1) ^ 1, s_abort)) {
+                        if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+                        *s_abort = 1;
+                        ok = false;
+                        break;
+                    }
+                    StageMeta m;
+                    m.n_valid = n_valid;
+                    m.b = b;
+                    m.rec = uniform ? rg.rec_fixed : unit + b;
+                    m.flags = ((f == lo || f == s_off[b]) ? 1 : 0) | ((f + 1 == hi || f + 1 >= s_off[b + 1]) ? 2 : 0);
+                    s_meta[st] = m;
+                    const uint32_t bar = smem_u32(&full_bar[st]);
+                    const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
+                    mbar_expect_tx(bar, GQA ? 2 * G * T::VTILE_BYTES : G * T::VTILE_BYTES + T::KR_BYTES);
+                    if constexpr (!GQA) tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
+                    for (int g = 0; g < G; ++g) {
+                        const int row = (int)((page * G + g) * p.P + slot0);
+                        if constexpr (GQA) {
+#pragma unroll
+                            for (int bx = 0; bx < T::BOXES; ++bx)
+                                tma_load_2d(base + (G + g) * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_k, bx * 64, row, bar);
+                        }
+#pragma unroll
+                        for (int bx = 0; bx < T::BOXES; ++bx)
+                            tma_load_2d(base + g * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, bar);
+                    }
+                    ++issued;
                 }
-                const uint32_t par = ((i / NSTAGE) & 1) ^ 1;
-                if (!mbar_wait_bounded(smem_u32(&empty_bar[st]), par, s_abort)) {
+                if (!ok) break;
+                if (!asked) {
+                    if (!waited) {
+                        grid_dependency_wait();
+                        waited = true;
+                    }
+                    ticket = atomicAdd(p.ticket, 1);
+                }
+                if (ticket < 0 || ticket >= n_tickets) break;
+                // ticket t -> tail j = 1 + t / n_ranges of range t % n_ranges: first every range's first tail, then the second, ...
+                const int c = ticket % plan.n_ranges, j = 1 + ticket / plan.n_ranges;
+                unit = c * (plan.U + 1) + j;
+                unit_range(plan, c, j, lo, hi);
+                if (lo < hi) b = seq_of_tile(s_off, p.B, lo);
+            }
+            if (ok) {
+                // tell the consumers that nothing more is coming
+                const int st = issued % NSTAGE;
+                if (mbar_wait_bounded(smem_u32(&empty_bar[st]), ((issued / NSTAGE) & 1) ^ 1, s_abort)) {
+                    s_meta[st].n_valid = -1;
+                    mbar_arrive(smem_u32(&full_bar[st]));
+                } else {
                     if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
                     *s_abort = 1;
                     ok = false;
-                    break;
                 }
-                const int f = rg.lo + i;
-                while (f >= s_off[b + 1]) ++b;
-                const int t0 = (f - s_off[b]) * TILE;
-                if (!waited) {
-                    const int ap = p.append_pos[b];
-                    if (ap >= t0 && ap < t0 + TILE) {   // this tile receives the new token: it must be complete first
-                        grid_dependency_wait();
-                        waited = true;
-                    }
-                }
-                int n_valid = min(TILE, p.seq_lens[b] - t0);
-                const int pj = t0 / p.P, slot0 = t0 % p.P;
-                long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
-                                               : (long long)b * p.max_pages + pj;
-                if (page < 0 || page >= p.num_pages) {
-                    if (!waited) {               // dev_status belongs to the stream-ordered part of the call
-                        grid_dependency_wait();
-                        waited = true;
-                    }
-                    report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
-                    page = 0;
-                    n_valid = 0;
-                }
-                s_meta[2 * st] = n_valid;
-                s_meta[2 * st + 1] = b;
-                const uint32_t bar = smem_u32(&full_bar[st]);
-                const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
-                mbar_expect_tx(bar, GQA ? 2 * G * T::VTILE_BYTES : G * T::VTILE_BYTES + T::KR_BYTES);
-                if constexpr (!GQA) tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
-                for (int g = 0; g < G; ++g) {
-                    const int row = (int)((page * G + g) * p.P + slot0);
-                    if constexpr (GQA) {
-#pragma unroll
-                        for (int bx = 0; bx < T::BOXES; ++bx)
-                            tma_load_2d(base + (G + g) * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_k, bx * 64, row, bar);
-                    }
-#pragma unroll
-                    for (int bx = 0; bx < T::BOXES; ++bx)
-                        tma_load_2d(base + g * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, bar);
-                }
-                ++issued;
             }
             if (!ok) {
                 // drain: every copy this block started must land before its shared memory is released
@@ -308,34 +373,47 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         uint32_t qf[T::KSTEPS][2];        // B fragments of Q^T: column n = lane/4 = 2*head + {hi, lo}
         float oacc[T::MT][4];
         float m_run = -INFINITY, l_run = 0.f;
-        int cur_b = -1;
-        int b = rg.b_first;
         const float scale = p.scale_log2;
+        const int lo_part = r8 & 1;
+
+        // absorbed query of head (lane/4)/2, hi or lo part by (lane/4)&1, as mma B fragments
+        auto load_query = [&](int b) {
+            const float *q = p.q + ((size_t)b * H + g * kHeadsPerGroup + (r8 >> 1)) * T::DQ;
+#pragma unroll
+            for (int kk = 0; kk < T::KSTEPS; ++kk) {
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const float2 v = *reinterpret_cast<const float2 *>(q + kk * 16 + half * 8 + 2 * jh);
+                    const uint32_t sx = split_hi_lo(v.x), sy = split_hi_lo(v.y);
+                    qf[kk][half] = lo_part ? ((sx >> 16) | (sy & 0xffff0000u)) : ((sx & 0xffffu) | (sy << 16));
+                }
+            }
+        };
+        if (early) grid_dependency_wait();
+        publish_header(p, s_off, plan, tid, n_consumers * 32);
+        // the first sequence is known before any tile arrives: fetch its query while the first copies fly
+        int cur_b = -1;
+        if (rg.lo < rg.hi) {
+            cur_b = rg.b_first;
+            load_query(cur_b);
+        }
 
 #pragma unroll 1
-        for (int i = 0; i < n_tiles; ++i) {
+        for (int i = 0;; ++i) {
             const int st = i % NSTAGE;
             if (!mbar_wait_bounded(smem_u32(&full_bar[st]), (i / NSTAGE) & 1, s_abort)) {
-                if (!*s_abort && lane == 0) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+                if (!*s_abort && lane == 0) report_error(p.dev_status, GVA_ERR_TIMEOUT, cur_b < 0 ? 0 : cur_b);
                 *s_abort = 1;
                 break;
             }
-            const int f = rg.lo + i;
-            while (f >= s_off[b + 1]) ++b;
-            const int n_valid = s_meta[2 * st];
-            if (b != cur_b) {
-                cur_b = b;
-                // absorbed query of head (lane/4)/2, hi or lo part by (lane/4)&1, as mma B fragments
-                const float *q = p.q + ((size_t)b * H + g * kHeadsPerGroup + (r8 >> 1)) * T::DQ;
-                const int lo_part = r8 & 1;
-#pragma unroll
-                for (int kk = 0; kk < T::KSTEPS; ++kk) {
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        const float2 v = *reinterpret_cast<const float2 *>(q + kk * 16 + half * 8 + 2 * jh);
-                        const uint32_t sx = split_hi_lo(v.x), sy = split_hi_lo(v.y);
-                        qf[kk][half] = lo_part ? ((sx >> 16) | (sy & 0xffff0000u)) : ((sx & 0xffffu) | (sy << 16));
-                    }
+            const StageMeta meta = s_meta[st];
+            const int n_valid = meta.n_valid;
+            if (n_valid < 0) break;       // producer is done
+            const int b = meta.b;
+            if (meta.flags & 1) {         // a new segment: its own softmax state (and query, if the sequence changed)
+                if (b != cur_b) {
+                    cur_b = b;
+                    load_query(b);
                 }
                 m_run = -INFINITY;
                 l_run = 0.f;
@@ -435,9 +513,9 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&empty_bar[st]));
 
-            // ---- segment end: write this (block, sequence, part) partial ----
-            if (i + 1 == n_tiles || f + 1 >= s_off[b + 1]) {
-                const int rec = ((rg.rec_fixed >= 0) ? rg.rec_fixed : (int)blockIdx.x + b) * WPG + part;
+            // ---- segment end: write this (unit, sequence, part) partial ----
+            if (meta.flags & 2) {
+                const int rec = meta.rec * WPG + part;
                 float l = l_run;
                 l += __shfl_xor_sync(0xffffffffu, l, 4);
                 l += __shfl_xor_sync(0xffffffffu, l, 8);
@@ -468,7 +546,7 @@ inline int mma_tile_for(const gva_config &cfg, bool gqa) {
 }
 // Consumer warps per value group (each takes an equal share of a tile's 16-token chunks and writes its own partial).
 #ifndef GVA_MMA_WPG64
-#define GVA_MMA_WPG64 2   // build-time tuning knob for the d_v = 64 kernels: 1 or 2
+#define GVA_MMA_WPG64 1   // build-time tuning knob for the d_v = 64 kernels: 1 or 2 (measured equal; 1 halves the partial records)
 #endif
 inline int mma_warps_per_group(const gva_config &cfg, bool /*gqa*/) { return cfg.d_v == 64 ? GVA_MMA_WPG64 : 1; }
 

@@ -218,77 +218,88 @@ step_front_kernel(StepFrontParams a, RopeTable rope) {
 }
 
 // ---- LSE combine ---------------------------------------------------------------------------------
-// grid (B, H / 4), block 128: one warp per (sequence, head).  Records are merged in index order, so
-// the result is reproducible for fixed launch geometry.
+// block 128 = 4 warps; WPH warps share one (sequence, head), so a block covers 4 / WPH heads:
+//   WPH = 4 (d_v = 64):  grid (B, H).     Warp w takes records w, w+4, ... -- 32 records per memory round trip
+//                        per block -- and the four warp states are merged through shared memory.
+//   WPH = 1 (d_v = 128): grid (B, H / 4). One warp per head, no shared memory, so that every block fits beside
+//                        the decode kernel's blocks and is already resident when that kernel ends.
+// Each warp requests kCombineUnroll records' (max, sum) pairs and partial outputs before using any, and keeps
+// a running (m, L, acc) by the usual rescaling; everything is merged in a fixed order, so the result is
+// reproducible for fixed launch geometry.
 //   m* = max_r m_r ;  L = sum_r l_r 2^(m_r - m*) ;  out = sum_r 2^(m_r - m*) o_r / L ;  lse = (m* + log2 L) ln 2
-// Lanes first fetch one record's (m, l) each, so the weights of 32 records cost one memory round
-// trip; the partial outputs are then read four records at a time.
-template <int DV>
+template <int DV, int WPH>
 __global__ void __launch_bounds__(128)
 combine_kernel(DecodeParams p) {
     grid_dependency_launch();
-    const int b = blockIdx.x;
+    constexpr int DPL = DV / 32;
+    constexpr int UNROLL = 8;
+    using VecT = typename std::conditional<DPL == 2, float2, float4>::type;
+    __shared__ float s_acc[WPH > 1 ? 4 : 1][WPH > 1 ? DV : 1];
+    __shared__ float s_ml[4][2];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int h = blockIdx.y * 4 + warp;
-    if (h >= p.H) return;
-    grid_dependency_wait();
-    int first, n;
-    if (p.num_splits > 0) {
-        first = b * p.num_splits * p.rec_mult;
-        n = p.num_splits * p.rec_mult;
-    } else {
-        const int total = p.hdr[0], n_eff = p.hdr[1];
-        const int off0 = p.hdr[kHdrInts + b], off1 = p.hdr[kHdrInts + b + 1];
+    const int b = blockIdx.x;
+    const int h = blockIdx.y * (4 / WPH) + warp / WPH;
+    const int part = warp % WPH;
+    const bool active = h < p.H;
+
+    auto read_plan = [&](int &first, int &n) {
+        UnitPlan plan;
+        plan.total = __ldcg(p.hdr + kHdrTotal);
+        plan.n_ranges = __ldcg(p.hdr + kHdrRanges);
+        plan.U = __ldcg(p.hdr + kHdrU);
+        plan.K = __ldcg(p.hdr + kHdrK);
+        const int off0 = __ldcg(p.hdr + kHdrInts + b), off1 = __ldcg(p.hdr + kHdrInts + b + 1);
         if (off1 == off0) {
             n = 0;
             first = 0;
         } else {
-            const int c0 = range_owner(off0, total, n_eff), c1 = range_owner(off1 - 1, total, n_eff);
-            first = (c0 + b) * p.rec_mult;
-            n = (c1 - c0 + 1) * p.rec_mult;
+            const int u0 = unit_of_tile(plan, off0), u1 = unit_of_tile(plan, off1 - 1);
+            first = (u0 + b) * p.rec_mult;
+            n = (u1 - u0 + 1) * p.rec_mult;
         }
+    };
+    grid_dependency_wait();
+    int first = 0, n = 0;
+    if (p.num_splits > 0) {
+        first = b * p.num_splits * p.rec_mult;
+        n = p.num_splits * p.rec_mult;
+    } else {
+        read_plan(first, n);
     }
-    constexpr int DPL = DV / 32;
-    using VecT = typename std::conditional<DPL == 2, float2, float4>::type;
-    float *o_dst = p.out + ((size_t)b * p.H + h) * DV + lane * DPL;
-    float mstar = -INFINITY;
-    for (int r = lane; r < n; r += 32) mstar = fmaxf(mstar, p.rec_ml[((size_t)(first + r) * p.H + h) * 2]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, o));
-    if (n == 0 || mstar == -INFINITY) {
-#pragma unroll
-        for (int d = 0; d < DPL; ++d) o_dst[d] = 0.f;
-        if (p.lse && lane == 0) p.lse[(size_t)b * p.H + h] = -INFINITY;
-        return;
-    }
-    float L = 0.f, acc[DPL];
+    // the decode kernel is complete: hand the tail-unit ticket back at zero for the next call
+    if (b == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.ticket = 0;
+
+    float m_w = -INFINITY, L_w = 0.f, acc[DPL];
 #pragma unroll
     for (int d = 0; d < DPL; ++d) acc[d] = 0.f;
-    for (int r0 = 0; r0 < n; r0 += 32) {
-        // lane r: weight of record r0 + r (0 for an empty partition or past the end)
-        float w_lane = 0.f, l_lane = 0.f;
-        if (r0 + lane < n) {
-            const float2 ml = *reinterpret_cast<const float2 *>(p.rec_ml + ((size_t)(first + r0 + lane) * p.H + h) * 2);
-            if (ml.x != -INFINITY) {
-                w_lane = exp2f(ml.x - mstar);
-                l_lane = ml.y;
-            }
-        }
-        const int cnt = min(32, n - r0);
-        for (int r = 0; r < cnt; r += 4) {
-            VecT v[4];
+    if (active) {
+        for (int r0 = part; r0 < n; r0 += WPH * UNROLL) {
+            float2 ml[UNROLL];
+            VecT v[UNROLL];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int rr = min(r + u, cnt - 1);      // clamped: duplicates get weight 0 below
-                v[u] = *reinterpret_cast<const VecT *>(p.rec_o + ((size_t)(first + r0 + rr) * p.H + h) * DV + lane * DPL);
+            for (int u = 0; u < UNROLL; ++u) {
+                const int r = r0 + WPH * u;
+                ml[u] = make_float2(-INFINITY, 0.f);
+                if (r < n) {
+                    const size_t rh = (size_t)(first + r) * p.H + h;
+                    ml[u] = __ldcg(reinterpret_cast<const float2 *>(p.rec_ml + rh * 2));
+                    v[u] = __ldcg(reinterpret_cast<const VecT *>(p.rec_o + rh * DV + lane * DPL));
+                }
             }
+            float m_new = m_w;
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int rr = r + u;
-                float w = __shfl_sync(0xffffffffu, w_lane, rr & 31);
-                const float l = __shfl_sync(0xffffffffu, l_lane, rr & 31);
-                if (rr >= cnt || w == 0.f) continue;     // an empty partition's output was never written: skip, do not multiply
-                L = fmaf(l, w, L);
+            for (int u = 0; u < UNROLL; ++u) m_new = fmaxf(m_new, ml[u].x);
+            if (m_new == -INFINITY) continue;            // nothing live yet
+            const float corr = exp2f(m_w - m_new);       // 0 when m_w = -inf
+            L_w *= corr;
+#pragma unroll
+            for (int d = 0; d < DPL; ++d) acc[d] *= corr;
+            m_w = m_new;
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                if (ml[u].x == -INFINITY) continue;      // empty partition or past the end: its output was never written
+                const float w = exp2f(ml[u].x - m_new);
+                L_w = fmaf(ml[u].y, w, L_w);
                 if constexpr (DPL == 2) {
                     acc[0] = fmaf(w, v[u].x, acc[0]);
                     acc[1] = fmaf(w, v[u].y, acc[1]);
@@ -301,9 +312,44 @@ combine_kernel(DecodeParams p) {
             }
         }
     }
+    float mstar = m_w, L = L_w, o[DPL];
+#pragma unroll
+    for (int d = 0; d < DPL; ++d) o[d] = acc[d];
+    if constexpr (WPH > 1) {
+#pragma unroll
+        for (int d = 0; d < DPL; ++d) s_acc[warp][lane * DPL + d] = acc[d];
+        if (lane == 0) {
+            s_ml[warp][0] = m_w;
+            s_ml[warp][1] = L_w;
+        }
+        __syncthreads();
+        if (part != 0) return;
+        mstar = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < WPH; ++w) mstar = fmaxf(mstar, s_ml[warp + w][0]);
+        L = 0.f;
+#pragma unroll
+        for (int d = 0; d < DPL; ++d) o[d] = 0.f;
+#pragma unroll
+        for (int w = 0; w < WPH; ++w) {
+            if (s_ml[warp + w][0] == -INFINITY) continue;
+            const float sc = exp2f(s_ml[warp + w][0] - mstar);
+            L = fmaf(s_ml[warp + w][1], sc, L);
+#pragma unroll
+            for (int d = 0; d < DPL; ++d) o[d] = fmaf(sc, s_acc[warp + w][lane * DPL + d], o[d]);
+        }
+    }
+    if (!active) return;
+    float *o_dst = p.out + ((size_t)b * p.H + h) * DV + lane * DPL;
+    if (mstar == -INFINITY) {
+#pragma unroll
+        for (int d = 0; d < DPL; ++d) o_dst[d] = 0.f;
+        if (p.lse && lane == 0) p.lse[(size_t)b * p.H + h] = -INFINITY;
+        return;
+    }
     const float inv = 1.f / L;
 #pragma unroll
-    for (int d = 0; d < DPL; ++d) o_dst[d] = acc[d] * inv;
+    for (int d = 0; d < DPL; ++d) o_dst[d] = o[d] * inv;
     if (p.lse && lane == 0) p.lse[(size_t)b * p.H + h] = (mstar + log2f(L)) * kLn2;
 }
 
