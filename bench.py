@@ -1,15 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the GVA decode hot path on B200.
 
-A step = one pass of the whole path over one batch: gva_absorb_query -> gva_append_cache ->
-gva_decode (split-KV kernel + LSE combine), on the long-context paged workload (cfg2: B=32, H=16,
-G=4, d_v=64, d_c=64, d_r=16, T=32768, bf16 cache in 64-token pages behind a permuted block table).
-The metric is cache-read GB/s: the live cache bytes one step must stream, divided by the step time.
+A step = one pass of the whole path over one batch: absorbed queries, cache append, split-KV decode
+and the LSE merge, i.e. one gva_decode_step call (fused absorb + append kernel, decode kernel, combine
+kernel).  The headline workload is the long-context paged one (cfg2: B=32, H=16, G=4, d_v=64, d_c=64,
+d_r=16, T=32768, bf16 cache in 64-token pages behind a permuted block table).  The metric is cache-read
+GB/s: the live cache bytes one step must stream, divided by the step time.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg1|cfg2|cfg3|cfg4]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+                    [--workload cfg1|cfg2|cfg3|cfg4] [--kernel auto|fma|mma] [--headline-only]
 
-N > 1 runs N independent replicas (one process per GPU under torch.distributed.run): the path
-has no exchange step, so there is no collective on the data path; only the timing barrier and the
+N > 1 runs N independent replicas (one process per GPU under torch.distributed.run): the path has no
+exchange step, so there is no collective on the data path; only the timing barrier and the
 max-over-ranks reduction use NCCL.
 """
 from __future__ import annotations
@@ -30,6 +32,10 @@ if ROOT not in sys.path:
 METRIC = "gva_decode_cache_read_bandwidth"
 UNIT = "GB/s"
 
+# DRAM traffic of one decode-kernel launch on cfg2 at full size, from ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum, mean of two launches; profiles/decode_mma_kernel_cfg2.md).
+NCU_TRAFFIC_BYTES = {"cfg2": 0.5 * ((571_091_200 + 3_437_056) + (571_084_544 + 409_856))}
+
 
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -41,28 +47,46 @@ def load_peaks():
 
 def make_workload(name: str, rank: int):
     from paper_2609_13285_b200 import workloads as wl
-    seed_shift = 7919 * rank
+    shift = 7919 * rank
     if name == "cfg1":
-        return wl.config1(seed=wl.MASTER_SEED + 1000 + seed_shift)
+        return wl.config1(seed=wl.MASTER_SEED + 1000 + shift)
     if name == "cfg2":
-        return wl.config2(seed=wl.MASTER_SEED + 2000 + seed_shift)
+        return wl.config2(seed=wl.MASTER_SEED + 2000 + shift)
     if name == "cfg3":
-        return wl.config3(seed=wl.MASTER_SEED + 3000 + seed_shift)
+        return wl.config3(seed=wl.MASTER_SEED + 3000 + shift)
+    if name == "cfg4":
+        return wl.config4_layer(0, seed=wl.MASTER_SEED + 4000 + shift)
     if name == "cfg2-ncu":   # profiler-sized: 143 MB of cache (> L2), same shapes and paging as cfg2
-        return wl.config2(seed=wl.MASTER_SEED + 2000 + seed_shift, B=16, T=16384)
+        return wl.config2(seed=wl.MASTER_SEED + 2000 + shift, B=16, T=16384)
     if name == "cfg2-small":
-        return wl.config2(seed=wl.MASTER_SEED + 2000 + seed_shift, B=8, T=8192)
+        return wl.config2(seed=wl.MASTER_SEED + 2000 + shift, B=8, T=8192)
     raise SystemExit(f"unknown workload {name}")
 
 
-def workload_description(case) -> dict:
+WORKLOAD_TEXT = {
+    "cfg1": "batched decode step, contiguous bf16 cache (B=8, T=4096)",
+    "cfg2": "long-context paged decode step (B=32, T=32768, 64-token pages, permuted block table)",
+    "cfg3": "wider-head ragged serving batch (B=64, H=32, G=8, d_v=128, seq_lens ~ U[1024,16384], paged)",
+    "cfg4": "24-layer decode step (B=128, T=8192 cached + 1 appended per layer, paged, one pool per layer)",
+}
+
+
+def workload_description(name: str, case, layers: int = 1) -> dict:
     s = case.shape
-    return {"workload": f"{case.name}: long-context paged GVA decode step (absorb + append + decode)",
-            "B": case.B, "H": s.H, "G": s.G, "d_v": s.d_v, "d_c": s.d_c, "d_r": s.d_r,
+    cache_bytes = case.cache_bytes() * layers
+    if layers > 1:
+        l2 = "each step walks 24 distinct per-layer pools (13.7 GB), far beyond L2"
+    elif cache_bytes > 2.5e8:
+        l2 = "cache stream is several times the 126 MB L2 and alternates between two pool copies"
+    else:
+        l2 = "cache smaller than L2: enough pool copies (>= 300 MB together) are rotated that every step streams from HBM"
+    return {"workload": f"{name}: {WORKLOAD_TEXT.get(name.split('-')[0], name)}; step = absorb + append + "
+                        "split-KV decode + LSE combine" + (f", {layers} layers" if layers > 1 else ""),
+            "B": case.B, "H": s.H, "G": s.G, "d_v": s.d_v, "d_c": s.d_c, "d_r": s.d_r, "layers": layers,
             "total_tokens": int(case.seq_lens.astype(np.int64).sum()), "max_seq_len": int(case.seq_lens.max()),
-            "page_size": case.page_size, "cache": case.cache_dtype + (" paged" if case.block_table is not None else " contiguous"),
-            "cache_bytes_per_step": case.cache_bytes(),
-            "l2": "cache stream (>= 4x the 126 MB L2) alternates between two pool copies; no flush needed"}
+            "page_size": case.page_size,
+            "cache": case.cache_dtype + (" paged" if case.block_table is not None else " contiguous"),
+            "cache_bytes_per_step": cache_bytes, "l2": l2}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -143,7 +167,7 @@ def oracle_sample(case, n_seq: int):
 
 def cpu_baseline(case, budget_s: float = 12.0) -> dict:
     """The oracle as it stands, timed on this host's cores on a bounded sample of the workload."""
-    dt1, bytes1, threads = oracle_sample(case, 1)
+    dt1, _, threads = oracle_sample(case, 1)
     n = int(max(1, min(case.B, budget_s / max(dt1, 1e-3))))
     dt, nbytes, threads = oracle_sample(case, n)
     return {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
@@ -152,99 +176,116 @@ def cpu_baseline(case, budget_s: float = 12.0) -> dict:
 
 
 def run_reference(args) -> None:
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    """The reference arm: the CPU oracle, as it stands, on the same workload (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
         return
-    case = make_workload(args.workload, 0)
-    from oracle import gva_oracle as orc
+    name = args.workload
+    case = make_workload(name, 0)
     dt1, _, threads = oracle_sample(case, 1)
-    n = int(max(1, min(case.B, 8.0 / max(dt1, 1e-3))))      # each step: a sample worth ~8 s of CPU work at most
-    for _ in range(min(args.warmup, 1)):
+    n = int(max(1, min(case.B, 8.0 / max(dt1, 1e-3))))      # each step: at most ~8 s of CPU work
+    warm = min(args.warmup, 1)
+    for _ in range(warm):
         oracle_sample(case, n)
-    times, nbytes = [], 0
     steps = max(1, min(args.steps, 5))
+    times, nbytes = [], 0
     for _ in range(steps):
         dt, nbytes, threads = oracle_sample(case, n)
         times.append(dt)
     ms = 1e3 * float(np.mean(times))
     value = nbytes / (ms * 1e-3) / 1e9
-    cfg = workload_description(case)
-    sample = f"each step = fp64 oracle on the first {n} of {case.B} sequences ({nbytes} cache bytes)"
+    sample = f"each step = fp64 oracle (absorb + decode) on the first {n} of {case.B} sequences ({nbytes} cache bytes)"
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-            "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
+            "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": workload_description(name, case),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
 # ----------------------------------------------------------------------------------------------
-def main() -> None:
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2")
-    ap.add_argument("--kernel", default="auto", choices=["auto", "fma", "mma"])
-    ap.add_argument("--num-splits", type=int, default=0)
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    args = ap.parse_args()
+class Layer:
+    """Device tensors of one decode layer: its cache handles and, for the multi-layer workload, its own inputs."""
 
-    if args.impl == "reference":
-        run_reference(args)
-        return
+    def __init__(self, caches):
+        self.caches = caches
 
-    import torch
-    from paper_2609_13285_b200 import binding as gb, build as gbuild, harness
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
-    if rank == 0:
-        gbuild.build()
-    if dist is not None:
-        dist.barrier()
-    gb.load()
-
-    warmup = max(3, args.warmup)
-    steps = max(1, args.steps)
-    kernel = {"auto": gb.GVA_KERNEL_AUTO, "fma": gb.GVA_KERNEL_FMA, "mma": gb.GVA_KERNEL_MMA}[args.kernel]
-    case = make_workload(args.workload, rank)
-    s = case.shape
-    B = case.B
-    # Algorithm 1's order: the step's new token takes the last position of each sequence
-    # (append at t = seq_len - 1), then its query attends over all seq_len tokens.
-    pos_np = (case.seq_lens - 1).astype(np.int32)
-    case.q_pos[:] = pos_np
-    case.append_pos[:] = pos_np
+def build_layers(case, dev, kernel, n_layers, torch, gb, harness):
+    """Layer 0 comes from the seeded host generator.  For the multi-layer workload the other layers' pools,
+    maps and inputs are drawn on the device from a seeded torch generator (13.7 GB would take minutes on the
+    host), each layer with its own seeded block-table permutation."""
     dc = harness.upload(case, device=dev, kernel=kernel)
-    # second copy of the pools at other addresses: consecutive steps never re-read what L2 may still hold
-    pools = [(dc.v_pool, dc.kr_pool), (dc.v_pool.clone(), dc.kr_pool.clone())]
-    caches = [gb.make_cache(v, k, dc.block_table, case.num_pages, case.max_pages_per_seq) for v, k in pools]
+    s = case.shape
+    if n_layers == 1:
+        cache_mb = case.cache_bytes() / 1e6
+        n_copies = 2 if cache_mb > 250 else max(2, int(np.ceil(300.0 / max(cache_mb, 1e-3))))
+        pools = [(dc.v_pool, dc.kr_pool)] + [(dc.v_pool.clone(), dc.kr_pool.clone()) for _ in range(n_copies - 1)]
+        caches = [gb.make_cache(v, k, dc.block_table, case.num_pages, case.max_pages_per_seq) for v, k in pools]
+        return dc, [Layer(caches)], pools
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(int(case.meta["seed"]) + 77)
+    rng = np.random.Generator(np.random.Philox(int(case.meta["seed"]) + 78))
+    keep, layers = [], []
+    for layer in range(n_layers):
+        if layer == 0:
+            v, k, bt, M = dc.v_pool, dc.kr_pool, dc.block_table, dc.M
+        else:
+            v = torch.randn(dc.v_pool.shape, generator=gen, device=dev, dtype=torch.bfloat16).view(torch.int16)
+            k = torch.randn(dc.kr_pool.shape, generator=gen, device=dev, dtype=torch.bfloat16).view(torch.int16)
+            bt = torch.from_numpy(rng.permutation(case.num_pages).astype(np.int32).reshape(case.B, -1)).to(dev)
+            M = torch.randn(dc.M.shape, generator=gen, device=dev) * float(1.0 / np.sqrt(s.d_v))
+        lay = Layer([gb.make_cache(v, k, bt, case.num_pages, case.max_pages_per_seq)])
+        lay.M = M
+        lay.q_c = torch.randn(dc.q_c.shape, generator=gen, device=dev)
+        lay.q_r = torch.randn(dc.q_r.shape, generator=gen, device=dev)
+        lay.v_new = torch.randn(dc.v_new.shape, generator=gen, device=dev)
+        lay.kr_new = torch.randn(dc.kr_new.shape, generator=gen, device=dev)
+        keep.append((v, k, bt))
+        layers.append(lay)
+    return dc, layers, keep
+
+
+def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with_e2e, with_clocks):
+    """Times one workload on this rank; returns per-rank numbers (the caller reduces them over ranks)."""
+    from paper_2609_13285_b200 import multirank
+    dev = torch.device("cuda", local_rank)
+    case = make_workload(name, rank)
+    n_layers = 24 if name == "cfg4" else 1
+    s, B = case.shape, case.B
+    if n_layers == 1:
+        # Algorithm 1's order: the step's new token takes the last position of each sequence (append at
+        # t = seq_len - 1), then its query attends over all seq_len tokens.
+        pos_np = (case.seq_lens - 1).astype(np.int32)
+        case.q_pos[:] = pos_np
+        case.append_pos[:] = pos_np
+    else:
+        pos_np = case.append_pos.copy()          # append at T, attend T + 1 tokens
+    dc, layers, keep = build_layers(case, dev, kernel, n_layers, torch, gb, harness)
     max_len = int(case.seq_lens.max())
     ns = args.num_splits
     ws = dc.ensure_workspace(ns)
     stream = torch.cuda.current_stream()
+    warmup, steps = max(3, args.warmup), max(1, args.steps)
+    if n_layers > 1:
+        warmup, steps = max(3, warmup // 5), max(3, steps // 10)
 
     def step(i: int):
-        # the whole path in one call: fused absorb + append kernel, split-KV decode kernel, LSE combine kernel
-        gb.gva_decode_step(dc.handle, caches[i & 1], dc.M, dc.q_c, dc.q_r, dc.v_new, dc.kr_new, dc.append_pos,
-                           dc.seq_lens, dc.q_abs, dc.out, dc.lse, ws, B, max_len, ns, dc.status)
+        for lay in layers:
+            c = lay.caches[i % len(lay.caches)]
+            if n_layers == 1:
+                gb.gva_decode_step(dc.handle, c, dc.M, dc.q_c, dc.q_r, dc.v_new, dc.kr_new, dc.append_pos,
+                                   dc.seq_lens, dc.q_abs, dc.out, dc.lse, ws, B, max_len, ns, dc.status)
+            else:
+                gb.gva_decode_step(dc.handle, c, lay.M, lay.q_c, lay.q_r, lay.v_new, lay.kr_new, dc.append_pos,
+                                   dc.seq_lens, dc.q_abs, dc.out, dc.lse, ws, B, max_len, ns, dc.status)
 
     def decode_only(i: int):
-        gb.gva_decode(dc.handle, caches[i & 1], dc.q_abs, dc.seq_lens, dc.out, dc.lse, ws, B, max_len, ns, dc.status)
+        for lay in layers:
+            gb.gva_decode(dc.handle, lay.caches[i % len(lay.caches)], dc.q_abs, dc.seq_lens, dc.out, dc.lse, ws, B,
+                          max_len, ns, dc.status)
 
     def sync_all():
-        if dist is not None:
-            dist.barrier()
+        multirank.barrier(dist)
         torch.cuda.synchronize()
 
     def timed(fn, n):
@@ -255,97 +296,152 @@ def main() -> None:
         b.record(stream)
         return a, b
 
-    # ---- device-resident timing: K whole steps between two events --------------------------------
     for i in range(warmup):
         step(i)
     sync_all()
-    sampler = ClockSampler(physical_gpu_index(local_rank))
-    sampler.start()
-    ev0, ev1 = timed(step, steps)
+    sampler = ClockSampler(physical_gpu_index(local_rank)) if with_clocks else None
+    if sampler:
+        sampler.start()
+    ev0, ev1 = timed(step, steps)                     # K whole steps between two events
     sync_all()
-    total_ms = ev0.elapsed_time(ev1)
-    # ---- the dominant kernel by itself: K gva_decode calls (split-KV kernel + combine) back to back ----
+    step_ms = ev0.elapsed_time(ev1) / steps
     for i in range(warmup):
         decode_only(i)
     sync_all()
-    d0, d1 = timed(decode_only, steps)
+    d0, d1 = timed(decode_only, steps)                # the dominant kernel: K gva_decode calls back to back
     sync_all()
-    clocks = sampler.finish()
-    decode_ms = d0.elapsed_time(d1) / steps
-    status = int(dc.status.item())
-    n_part = gb.gva_last_num_splits(dc.handle)
-    kernel_used = {1: "fma", 2: "mma"}.get(gb.gva_last_kernel(dc.handle), "?")
+    clocks = sampler.finish() if sampler else None
+    res = {"case": case, "layers": n_layers, "step_ms": step_ms, "decode_ms": d0.elapsed_time(d1) / steps / n_layers,
+           "steps": steps, "warmup": warmup, "clocks": clocks, "status": int(dc.status.item()),
+           "partitions": gb.gva_last_num_splits(dc.handle),
+           "kernel": {1: "fma", 2: "mma"}.get(gb.gva_last_kernel(dc.handle), "?"),
+           "cache_bytes": case.cache_bytes() * n_layers}
 
-    # ---- end to end: host buffers in, host buffer out, through the C ABI -----------------------
-    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
-    h_qc, h_qr, h_vn, h_kn = pin(case.q_c), pin(case.q_r), pin(case.v_new), pin(case.kr_new)
-    h_pos, h_len = pin(pos_np), pin(case.seq_lens)
-    h_out = torch.empty((B, s.H, s.d_v), dtype=torch.float32).pin_memory()
-    scratch = torch.empty(gb.gva_step_scratch_bytes(dc.handle, B, max_len, ns), dtype=torch.uint8, device=dev)
-    h2d = sum(t.numel() * t.element_size() for t in (h_qc, h_qr, h_vn, h_kn, h_pos, h_len))
-    d2h = h_out.numel() * 4
+    if with_e2e:
+        # end to end: host buffers in, host buffer out, through the C ABI (one call per step, then a sync)
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        h_qc, h_qr, h_vn, h_kn = pin(case.q_c), pin(case.q_r), pin(case.v_new), pin(case.kr_new)
+        h_pos, h_len = pin(pos_np), pin(case.seq_lens)
+        h_out = torch.empty((B, s.H, s.d_v), dtype=torch.float32).pin_memory()
+        scratch = torch.empty(gb.gva_step_scratch_bytes(dc.handle, B, max_len, ns), dtype=torch.uint8, device=dev)
+        caches = layers[0].caches
 
-    def e2e_step(i: int):
-        gb.gva_decode_step_host(dc.handle, caches[i & 1], dc.M, h_qc, h_qr, h_vn, h_kn, h_pos, h_len, h_out, scratch,
-                                B, max_len, ns, dc.status)
-        stream.synchronize()           # the caller reads the result every step
+        def e2e_step(i: int):
+            gb.gva_decode_step_host(dc.handle, caches[i % len(caches)], dc.M, h_qc, h_qr, h_vn, h_kn, h_pos, h_len,
+                                    h_out, scratch, B, max_len, ns, dc.status)
+            stream.synchronize()           # the caller reads the result every step
 
-    for i in range(warmup):
-        e2e_step(i)
-    sync_all()
-    t0 = time.perf_counter()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(steps):
-        e2e_step(i)
-    e1.record(stream)
-    sync_all()
-    e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0))
-    out_e2e = h_out.clone()
+        for i in range(warmup):
+            e2e_step(i)
+        sync_all()
+        t0 = time.perf_counter()
+        e0, e1 = timed(e2e_step, steps)
+        sync_all()
+        res["e2e_ms"] = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / steps
+        res["h2d"] = sum(t.numel() * t.element_size() for t in (h_qc, h_qr, h_vn, h_kn, h_pos, h_len))
+        res["d2h"] = h_out.numel() * 4
+        step(steps - 1)
+        torch.cuda.synchronize()
+        res["e2e_matches"] = bool(torch.allclose(h_out, dc.out.cpu(), atol=1e-5, rtol=1e-5))
+    dc.close()
+    del keep, layers
+    torch.cuda.empty_cache()
+    return res
 
-    # ---- reduce over ranks: slowest rank sets the time, bytes add up -----------------------------
-    cache_bytes = case.cache_bytes()
-    vals = torch.tensor([total_ms, e2e_ms, decode_ms], dtype=torch.float64, device=dev)
-    tot_bytes = torch.tensor([float(cache_bytes)], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tot_bytes, op=dist.ReduceOp.SUM)
-    total_ms, e2e_ms, decode_ms_max = [float(x) for x in vals.tolist()]
-    job_bytes = float(tot_bytes.item())
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "fma", "mma"])
+    ap.add_argument("--num-splits", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--headline-only", action="store_true", help="skip the short runs of the other workloads")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2609_13285_b200 import binding as gb, build as gbuild, harness, multirank
+
+    info = multirank.rank_info(os.environ)
+    rank, local_rank, world = info["rank"], info["local_rank"], info["world"]
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        gbuild.build()
+    multirank.barrier(dist)
+    gb.load()
+    kernel = {"auto": gb.GVA_KERNEL_AUTO, "fma": gb.GVA_KERNEL_FMA, "mma": gb.GVA_KERNEL_MMA}[args.kernel]
+
+    name = args.workload
+    r = measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with_e2e=True, with_clocks=True)
+    (step_ms, e2e_ms, decode_ms), job_bytes = multirank.reduce_times_and_work(
+        [r["step_ms"], r["e2e_ms"], r["decode_ms"]], r["cache_bytes"], dist, dev)
+
+    others = {}
+    if not args.headline_only and world == 1 and name == "cfg2" and args.kernel == "auto":
+        peak = load_peaks()[0]
+        short = argparse.Namespace(**vars(args))
+        short.steps, short.warmup = max(20, args.steps // 3), 10
+        for other in ("cfg1", "cfg3", "cfg4"):
+            o = measure(other, rank, local_rank, dist, short, kernel, torch, gb, harness, with_e2e=False,
+                        with_clocks=False)
+            per_layer = o["cache_bytes"] / o["layers"]
+            others[other] = {
+                "workload": WORKLOAD_TEXT[other], "ms_per_step": o["step_ms"],
+                "cache_read_GBps": o["cache_bytes"] / (o["step_ms"] * 1e-3) / 1e9,
+                "decode_steps_per_s": 1e3 / o["step_ms"],
+                "gva_decode_ms_per_call": o["decode_ms"],
+                "gva_decode_GBps": per_layer / (o["decode_ms"] * 1e-3) / 1e9,
+                "gva_decode_frac_of_measured_peak": per_layer / (o["decode_ms"] * 1e-3) / 1e9 / peak,
+                "cache_bytes_per_step": o["cache_bytes"], "kernel": o["kernel"], "partitions": o["partitions"],
+                "total_tokens": int(o["case"].seq_lens.astype(np.int64).sum()) * o["layers"], "steps": o["steps"],
+                "device_status": o["status"]}
 
     if rank == 0:
-        ms_step = total_ms / steps
-        value = job_bytes / (ms_step * 1e-3) / 1e9
-        e2e_value = job_bytes / (e2e_ms / steps * 1e-3) / 1e9
+        case = r["case"]
+        value = multirank.job_throughput(job_bytes, step_ms) / 1e9
+        e2e_value = multirank.job_throughput(job_bytes, e2e_ms) / 1e9
         peak, peak_src = load_peaks()
         algo_bytes = case.algorithmic_bytes()
         achieved = algo_bytes / (decode_ms * 1e-3) / 1e9
-        # sanity: end-to-end result equals the device-resident result
-        same = bool(torch.allclose(out_e2e, dc.out.cpu(), atol=1e-5, rtol=1e-5))
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": r["steps"], "warmup": r["warmup"],
+            "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if case.cache_dtype == "bf16" else "f32", "data": "synthetic",
-            "config": dict(workload_description(case), kernel=kernel_used, partitions=n_part, replicas=world),
-            "decode_steps_per_s": world * 1e3 / ms_step,
+            "config": dict(workload_description(name, case, r["layers"]), kernel=r["kernel"],
+                           partitions=r["partitions"], replicas=world),
+            "decode_steps_per_s": world * 1e3 / step_ms,
             "frac_of_8TBs_nominal": value / world / 8000.0,
-            "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": e2e_ms / steps, "matches_device_result": same,
-                    "note": "gva_decode_step_host: pinned host q/v/k_r/pos in, host out; the cache is resident state"},
-            "gpu_launches": 3 * steps,
+            "clocks": r["clocks"],
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"],
+                    "ms_per_step": e2e_ms, "matches_device_result": r["e2e_matches"],
+                    "note": "gva_decode_step_host per step, then a stream sync: pinned host q_c/q_r/v_new/k_r/pos/"
+                            "seq_lens in, host out; the cache and the maps M are resident state"},
+            "gpu_launches": 3 * r["steps"] * r["layers"],
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_source": peak_src,
-                         "kernel": f"gva_decode ({kernel_used} split-KV kernel + LSE combine, timed together)",
+                         "traffic": NCU_TRAFFIC_BYTES.get(name), "peak_source": peak_src,
+                         "kernel": f"gva_decode: {r['kernel']} split-KV decode kernel + LSE combine kernel, timed "
+                                   "together over back-to-back calls (the decode kernel alone is ~0.91 of that time)",
                          "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": decode_ms},
-            "device_status": status,
+            "device_status": r["status"],
         }
-        if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(case)
-        elif not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(case, budget_s=6.0)
+        if others:
+            line["other_workloads"] = others
+        if not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(case, budget_s=12.0 if world == 1 else 6.0)
         print(json.dumps(line))
-    dc.close()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
