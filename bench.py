@@ -396,7 +396,7 @@ def main() -> None:
         short.steps, short.warmup = max(20, args.steps // 3), 10
         for other in ("cfg1", "cfg3", "cfg4"):
             o = measure(other, rank, local_rank, dist, short, kernel, torch, gb, harness, with_e2e=False,
-                        with_clocks=False)
+                        with_clocks=True)
             per_layer = o["cache_bytes"] / o["layers"]
             others[other] = {
                 "workload": WORKLOAD_TEXT[other], "ms_per_step": o["step_ms"],
@@ -407,7 +407,7 @@ def main() -> None:
                 "gva_decode_frac_of_measured_peak": per_layer / (o["decode_ms"] * 1e-3) / 1e9 / peak,
                 "cache_bytes_per_step": o["cache_bytes"], "kernel": o["kernel"], "partitions": o["partitions"],
                 "total_tokens": int(o["case"].seq_lens.astype(np.int64).sum()) * o["layers"], "steps": o["steps"],
-                "device_status": o["status"]}
+                "clocks": o["clocks"], "device_status": o["status"]}
 
     if rank == 0:
         case = r["case"]

@@ -141,7 +141,7 @@ WorkspaceLayout workspace_layout(const gva_handle *h, int B, int num_splits) {
     WorkspaceLayout w;
     // up to two partial records per (block, sequence): the tensor-core kernel may run two warps per group
     w.n_rec = 2 * (num_splits > 0 ? B * num_splits : max_units_balanced(h) + B);
-    w.hdr_bytes = align_up((size_t)(kHdrInts + B + 1) * 4, 256);
+    w.hdr_bytes = align_up((size_t)(kHdrInts + 2 * B) * 4, 256);
     w.rec_o_bytes = align_up((size_t)w.n_rec * h->cfg.H * h->cfg.d_v * 4, 256);
     w.rec_ml_bytes = align_up((size_t)w.n_rec * h->cfg.H * 2 * 4, 256);
     w.total = w.hdr_bytes + w.rec_o_bytes + w.rec_ml_bytes;
@@ -169,6 +169,7 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     p.rec_ml = reinterpret_cast<float *>(ws + w.hdr_bytes + w.rec_o_bytes);
     p.num_splits = num_splits;
     p.rec_mult = 1;
+    p.combine_passes = 2;
     if (B == 0) return GVA_OK;
 
 

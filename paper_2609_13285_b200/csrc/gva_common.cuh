@@ -11,8 +11,8 @@
 namespace gva {
 
 constexpr int kHeadsPerGroup = 4;   // H / G of every instantiated kernel
-// Workspace header (ints): the partition of the flat tile list into units, published by block 0 of
-// the decode kernel for the combine kernel.
+// Workspace header (ints): the partition of the flat tile list into units (for inspection) followed by one
+// (first record, record count) pair per sequence, published by block 0 of the decode kernel for the combine kernel.
 constexpr int kHdrInts = 8;
 constexpr int kHdrTotal = 0;        // total tiles
 constexpr int kHdrRanges = 1;       // equal contiguous ranges the tile list is cut into
@@ -29,7 +29,7 @@ struct DecodeParams {
     const int32_t *block_table;  // nullable
     const int32_t *seq_lens;
     const float *q;              // [B][H][d_q]
-    int32_t *hdr;                // workspace header (kHdrInts + B + 1 ints)
+    int32_t *hdr;                // workspace header (kHdrInts + 2 B ints)
     float *rec_o;                // [n_rec][H][d_v] unnormalised partial outputs
     float *rec_ml;               // [n_rec][H][2]   running max (log2 domain) and sum
     float *out;                  // [B][H][d_v]
@@ -39,6 +39,7 @@ struct DecodeParams {
     int B, H, G, P, num_pages, max_pages;
     int num_splits;              // 0 = balanced flat partition
     int rec_mult;                // partial records per (block, sequence): consumer warps per value group
+    int combine_passes;          // 2: the combine kernel runs its body once dry before its dependency wait
     int early_start;             // 1: launched right behind step_front_kernel (see gva_decode_mma.cuh)
     const int32_t *append_pos;   // early_start: position being appended per sequence (its tile must not be read early)
     float scale_log2;            // softmax scale * log2(e)
@@ -234,7 +235,15 @@ __device__ __forceinline__ void publish_header(const DecodeParams &p, const int 
         p.hdr[kHdrU] = plan.U;
         p.hdr[kHdrK] = plan.K;
     }
-    for (int i = tid; i <= p.B; i += nt) p.hdr[kHdrInts + i] = s_off[i];
+    // per sequence: first record (before the per-warp multiplier) and number of records of its run of units
+    for (int b = tid; b < p.B; b += nt) {
+        int2 seg = make_int2(0, 0);
+        if (s_off[b + 1] > s_off[b]) {
+            const int u0 = unit_of_tile(plan, s_off[b]), u1 = unit_of_tile(plan, s_off[b + 1] - 1);
+            seg = make_int2(u0 + b, u1 - u0 + 1);
+        }
+        reinterpret_cast<int2 *>(p.hdr + kHdrInts)[b] = seg;
+    }
 }
 
 // ---- small PTX wrappers ------------------------------------------------------------------------

@@ -56,18 +56,40 @@ __device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, cons
     const int tid = threadIdx.x;
     const float *Mh = M + (size_t)h * d_v * d_c;
     const int n_elem = d_v * d_c;
+    const int dq = d_v + d_r;
+    const int half = d_r / 2;
+    // Every global load this block needs is requested before the first one is used, so the block pays one
+    // memory round trip instead of one per phase: the query rows, the RoPE inputs, then the map.
+    constexpr int kQPer = (kAbsorbBatch * 256 + kAbsorbThreads - 1) / kAbsorbThreads;   // d_c <= 256
+    float qreg[kQPer];
+#pragma unroll
+    for (int u = 0; u < kQPer; ++u) {
+        const int i = u * kAbsorbThreads + tid;
+        qreg[u] = (i < nb * d_c) ? q_c[((size_t)(b0 + i / d_c) * H + h) * d_c + (i % d_c)] : 0.f;
+    }
+    float r0 = 0.f, r1 = 0.f;
+    int rpos = 0;
+    const bool has_rope = tid < nb * half;      // nb * half <= 8 * 16 < kAbsorbThreads
+    if (has_rope) {
+        const int bb = tid / half, i = tid % half;
+        const size_t src = ((size_t)(b0 + bb) * H + h) * d_r + 2 * i;
+        r0 = q_r[src];
+        r1 = q_r[src + 1];
+        rpos = q_pos[b0 + bb];
+    }
     if ((d_c & 3) == 0) {
         const float4 *M4 = reinterpret_cast<const float4 *>(Mh);    // M is 16-byte aligned per head: d_v*d_c*4 % 16 == 0
         const int n4 = n_elem >> 2;
-        for (int base = 0; base < n4; base += kAbsorbThreads * 4) {
-            float4 v[4];
+        constexpr int kMBatch = 8;
+        for (int base = 0; base < n4; base += kAbsorbThreads * kMBatch) {
+            float4 v[kMBatch];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < kMBatch; ++u) {
                 const int i = base + u * kAbsorbThreads + tid;
                 if (i < n4) v[u] = M4[i];
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < kMBatch; ++u) {
                 const int i = base + u * kAbsorbThreads + tid;
                 if (i < n4) {
                     const int e = i << 2;
@@ -79,24 +101,48 @@ __device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, cons
     } else {
         for (int i = tid; i < n_elem; i += kAbsorbThreads) sM[(i / d_c) * (d_c + 1) + (i % d_c)] = Mh[i];
     }
-    for (int i = tid; i < nb * d_c; i += kAbsorbThreads)
-        sq[i] = q_c[((size_t)(b0 + i / d_c) * H + h) * d_c + (i % d_c)];
-    __syncthreads();
-    const int dq = d_v + d_r;
-    for (int o = tid; o < nb * d_v; o += kAbsorbThreads) {
-        const int bb = o / d_v, i = o % d_v;
-        const float *mrow = sM + i * (d_c + 1);
-        const float *qrow = sq + bb * d_c;
-        float acc = 0.f;
-        for (int j = 0; j < d_c; ++j) acc = fmaf(qrow[j], mrow[j], acc);
-        q_abs[((size_t)(b0 + bb) * H + h) * dq + i] = acc;
+#pragma unroll
+    for (int u = 0; u < kQPer; ++u) {
+        const int i = u * kAbsorbThreads + tid;
+        if (i < nb * d_c) sq[i] = qreg[u];
     }
-    const int half = d_r / 2;
-    for (int o = tid; o < nb * half; o += kAbsorbThreads) {
-        const int bb = o / half, i = o % half;
-        const size_t src = ((size_t)(b0 + bb) * H + h) * d_r + 2 * i;
+    __syncthreads();
+    // Thread t owns map row i = t % d_v for sequences bb0, bb0 + step, ... (kAbsorbThreads % d_v == 0), so one
+    // read of M_h[i][j] feeds up to four independent accumulators.
+    if (kAbsorbThreads % d_v == 0 && kAbsorbBatch * d_v <= 4 * kAbsorbThreads) {
+        const int i = tid % d_v, bb0 = tid / d_v, step = kAbsorbThreads / d_v;
+        const float *mrow = sM + i * (d_c + 1);
+        const float *q0 = sq + min(bb0, nb - 1) * d_c, *q1 = sq + min(bb0 + step, nb - 1) * d_c;
+        const float *q2 = sq + min(bb0 + 2 * step, nb - 1) * d_c, *q3 = sq + min(bb0 + 3 * step, nb - 1) * d_c;
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+        for (int j = 0; j < d_c; ++j) {
+            const float m = mrow[j];
+            a0 = fmaf(q0[j], m, a0);
+            a1 = fmaf(q1[j], m, a1);
+            a2 = fmaf(q2[j], m, a2);
+            a3 = fmaf(q3[j], m, a3);
+        }
+        const float acc[4] = {a0, a1, a2, a3};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int bb = bb0 + k * step;
+            if (bb < nb) q_abs[((size_t)(b0 + bb) * H + h) * dq + i] = acc[k];
+        }
+    } else {
+        for (int o = tid; o < nb * d_v; o += kAbsorbThreads) {
+            const int bb = o / d_v, i = o % d_v;
+            const float *mrow = sM + i * (d_c + 1);
+            const float *qrow = sq + bb * d_c;
+            float acc = 0.f;
+            for (int j = 0; j < d_c; ++j) acc = fmaf(qrow[j], mrow[j], acc);
+            q_abs[((size_t)(b0 + bb) * H + h) * dq + i] = acc;
+        }
+    }
+    if (has_rope) {
+        const int bb = tid / half, i = tid % half;
         double y0, y1;
-        rope_pair((double)q_r[src], (double)q_r[src + 1], q_pos[b0 + bb], rope.inv_freq[i], y0, y1);
+        rope_pair((double)r0, (double)r1, rpos, rope.inv_freq[i], y0, y1);
         float *dst = q_abs + ((size_t)(b0 + bb) * H + h) * dq + d_v + 2 * i;
         dst[0] = __double2float_rn(y0);
         dst[1] = __double2float_rn(y1);
@@ -227,6 +273,11 @@ step_front_kernel(StepFrontParams a, RopeTable rope) {
 // a running (m, L, acc) by the usual rescaling; everything is merged in a fixed order, so the result is
 // reproducible for fixed launch geometry.
 //   m* = max_r m_r ;  L = sum_r l_r 2^(m_r - m*) ;  out = sum_r 2^(m_r - m*) o_r / L ;  lse = (m* + log2 L) ln 2
+// The body runs twice: a first, "dry" pass while the block still waits for the decode kernel (reads of the
+// workspace are discarded, nothing is written), then the real pass after the wait.  Both passes execute the
+// same instructions, so the real pass finds them in the SM's instruction cache; a kernel this short otherwise
+// spends most of its time on cold instruction fetches, because the cache stream has pushed its code out of L2
+// since the previous call.
 template <int DV, int WPH>
 __global__ void __launch_bounds__(128)
 combine_kernel(DecodeParams p) {
@@ -241,38 +292,32 @@ combine_kernel(DecodeParams p) {
     const int h = blockIdx.y * (4 / WPH) + warp / WPH;
     const int part = warp % WPH;
     const bool active = h < p.H;
+    const int hh = active ? h : 0;
 
-    auto read_plan = [&](int &first, int &n) {
-        UnitPlan plan;
-        plan.total = __ldcg(p.hdr + kHdrTotal);
-        plan.n_ranges = __ldcg(p.hdr + kHdrRanges);
-        plan.U = __ldcg(p.hdr + kHdrU);
-        plan.K = __ldcg(p.hdr + kHdrK);
-        const int off0 = __ldcg(p.hdr + kHdrInts + b), off1 = __ldcg(p.hdr + kHdrInts + b + 1);
-        if (off1 == off0) {
-            n = 0;
-            first = 0;
-        } else {
-            const int u0 = unit_of_tile(plan, off0), u1 = unit_of_tile(plan, off1 - 1);
-            first = (u0 + b) * p.rec_mult;
-            n = (u1 - u0 + 1) * p.rec_mult;
+#pragma unroll 1
+    for (int pass = 0; pass < p.combine_passes; ++pass) {
+        const bool dry = pass + 1 < p.combine_passes;
+        if (!dry) {
+            grid_dependency_wait();
+            // the decode kernel is complete: hand the tail-unit ticket back at zero for the next call
+            if (b == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.ticket = 0;
         }
-    };
-    grid_dependency_wait();
-    int first = 0, n = 0;
-    if (p.num_splits > 0) {
-        first = b * p.num_splits * p.rec_mult;
-        n = p.num_splits * p.rec_mult;
-    } else {
-        read_plan(first, n);
-    }
-    // the decode kernel is complete: hand the tail-unit ticket back at zero for the next call
-    if (b == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.ticket = 0;
-
-    float m_w = -INFINITY, L_w = 0.f, acc[DPL];
+        int first, n;
+        if (p.num_splits > 0) {
+            first = b * p.num_splits * p.rec_mult;
+            n = p.num_splits * p.rec_mult;
+        } else {   // this sequence's run of records, worked out by block 0 of the decode kernel
+            const int2 seg = __ldcg(reinterpret_cast<const int2 *>(p.hdr + kHdrInts) + b);
+            first = seg.x * p.rec_mult;
+            n = seg.y * p.rec_mult;
+        }
+        if (dry) {      // whatever the header holds right now, stay inside the workspace
+            first = 0;
+            n = WPH * UNROLL;
+        }
+        float m_w = -INFINITY, L_w = 0.f, acc[DPL];
 #pragma unroll
-    for (int d = 0; d < DPL; ++d) acc[d] = 0.f;
-    if (active) {
+        for (int d = 0; d < DPL; ++d) acc[d] = 0.f;
         for (int r0 = part; r0 < n; r0 += WPH * UNROLL) {
             float2 ml[UNROLL];
             VecT v[UNROLL];
@@ -281,7 +326,7 @@ combine_kernel(DecodeParams p) {
                 const int r = r0 + WPH * u;
                 ml[u] = make_float2(-INFINITY, 0.f);
                 if (r < n) {
-                    const size_t rh = (size_t)(first + r) * p.H + h;
+                    const size_t rh = (size_t)(first + r) * p.H + hh;
                     ml[u] = __ldcg(reinterpret_cast<const float2 *>(p.rec_ml + rh * 2));
                     v[u] = __ldcg(reinterpret_cast<const VecT *>(p.rec_o + rh * DV + lane * DPL));
                 }
@@ -289,7 +334,7 @@ combine_kernel(DecodeParams p) {
             float m_new = m_w;
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) m_new = fmaxf(m_new, ml[u].x);
-            if (m_new == -INFINITY) continue;            // nothing live yet
+            if (!(m_new > -INFINITY)) continue;          // nothing live yet (or, dry, garbage)
             const float corr = exp2f(m_w - m_new);       // 0 when m_w = -inf
             L_w *= corr;
 #pragma unroll
@@ -297,7 +342,7 @@ combine_kernel(DecodeParams p) {
             m_w = m_new;
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
-                if (ml[u].x == -INFINITY) continue;      // empty partition or past the end: its output was never written
+                if (!(ml[u].x > -INFINITY)) continue;    // empty partition or past the end: its output was never written
                 const float w = exp2f(ml[u].x - m_new);
                 L_w = fmaf(ml[u].y, w, L_w);
                 if constexpr (DPL == 2) {
@@ -311,46 +356,44 @@ combine_kernel(DecodeParams p) {
                 }
             }
         }
-    }
-    float mstar = m_w, L = L_w, o[DPL];
+        float mstar = m_w, L = L_w, o[DPL];
 #pragma unroll
-    for (int d = 0; d < DPL; ++d) o[d] = acc[d];
-    if constexpr (WPH > 1) {
+        for (int d = 0; d < DPL; ++d) o[d] = acc[d];
+        if constexpr (WPH > 1) {
+            __syncthreads();                             // previous pass has finished reading shared memory
 #pragma unroll
-        for (int d = 0; d < DPL; ++d) s_acc[warp][lane * DPL + d] = acc[d];
-        if (lane == 0) {
-            s_ml[warp][0] = m_w;
-            s_ml[warp][1] = L_w;
+            for (int d = 0; d < DPL; ++d) s_acc[warp][lane * DPL + d] = acc[d];
+            if (lane == 0) {
+                s_ml[warp][0] = m_w;
+                s_ml[warp][1] = L_w;
+            }
+            __syncthreads();
+            const int w0 = warp - part;
+            mstar = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < WPH; ++w) mstar = fmaxf(mstar, s_ml[w0 + w][0]);
+            L = 0.f;
+#pragma unroll
+            for (int d = 0; d < DPL; ++d) o[d] = 0.f;
+#pragma unroll
+            for (int w = 0; w < WPH; ++w) {
+                if (!(s_ml[w0 + w][0] > -INFINITY)) continue;
+                const float sc = exp2f(s_ml[w0 + w][0] - mstar);
+                L = fmaf(s_ml[w0 + w][1], sc, L);
+#pragma unroll
+                for (int d = 0; d < DPL; ++d) o[d] = fmaf(sc, s_acc[w0 + w][lane * DPL + d], o[d]);
+            }
         }
-        __syncthreads();
-        if (part != 0) return;
-        mstar = -INFINITY;
+        const bool live = mstar > -INFINITY;
+        const float inv = live ? 1.f / L : 0.f;
+        const float lse = live ? (mstar + log2f(L)) * kLn2 : -INFINITY;
+        if (!dry && active && part == 0) {
+            float *o_dst = p.out + ((size_t)b * p.H + h) * DV + lane * DPL;
 #pragma unroll
-        for (int w = 0; w < WPH; ++w) mstar = fmaxf(mstar, s_ml[warp + w][0]);
-        L = 0.f;
-#pragma unroll
-        for (int d = 0; d < DPL; ++d) o[d] = 0.f;
-#pragma unroll
-        for (int w = 0; w < WPH; ++w) {
-            if (s_ml[warp + w][0] == -INFINITY) continue;
-            const float sc = exp2f(s_ml[warp + w][0] - mstar);
-            L = fmaf(s_ml[warp + w][1], sc, L);
-#pragma unroll
-            for (int d = 0; d < DPL; ++d) o[d] = fmaf(sc, s_acc[warp + w][lane * DPL + d], o[d]);
+            for (int d = 0; d < DPL; ++d) o_dst[d] = live ? o[d] * inv : 0.f;
+            if (p.lse && lane == 0) p.lse[(size_t)b * p.H + h] = lse;
         }
     }
-    if (!active) return;
-    float *o_dst = p.out + ((size_t)b * p.H + h) * DV + lane * DPL;
-    if (mstar == -INFINITY) {
-#pragma unroll
-        for (int d = 0; d < DPL; ++d) o_dst[d] = 0.f;
-        if (p.lse && lane == 0) p.lse[(size_t)b * p.H + h] = -INFINITY;
-        return;
-    }
-    const float inv = 1.f / L;
-#pragma unroll
-    for (int d = 0; d < DPL; ++d) o_dst[d] = o[d] * inv;
-    if (p.lse && lane == 0) p.lse[(size_t)b * p.H + h] = (mstar + log2f(L)) * kLn2;
 }
 
 }  // namespace gva
