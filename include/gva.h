@@ -199,7 +199,10 @@ int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const
  * resident on the device (they are state, not per-step input).
  *   [host] q_c_host [B][H][d_c], q_r_host [B][H][d_r], v_new_host [B][G][d_v], kr_new_host [B][d_r] f32,
  *          pos_host [B] i32 (position t of the new token = query position), seq_lens_host [B] i32
- *          (tokens attended, normally t + 1).  Use pinned memory for truly asynchronous copies.
+ *          (tokens attended, normally t + 1).  If the four float inputs and out_host are all pinned
+ *          (page-locked, device-mapped) memory the kernels read and write them in place over the
+ *          interconnect and only pos and seq_lens are copied; otherwise every buffer is staged through
+ *          `scratch` with cudaMemcpyAsync (pageable memory makes those copies synchronous).
  *   [host] out_host [B][H][d_v] f32
  *   M                device, as in gva_absorb_query
  *   scratch          device, at least gva_step_scratch_bytes(h, B, max_seq_len, num_splits) bytes, 256-byte aligned;

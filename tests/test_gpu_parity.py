@@ -333,3 +333,33 @@ def test_fused_steps_back_to_back_generate_tokens(kernel):
         assert np.array_equal(v_gpu, case.v_pool) and np.array_equal(k_gpu, case.kr_pool)
     finally:
         dc.close()
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_step_matches_device_step(pinned):
+    # gva_decode_step_host with pinned buffers (read and written in place by the kernels) and with pageable
+    # buffers (staged copies) must both equal the device-buffer step
+    lens = np.array([700, 64, 1, 2049], dtype=np.int32)
+    mk = lambda: wl.make_case("hstep", wl.SHAPE_A, lens, page_size=64, cache_dtype="bf16", seed=213,
+                              q_pos=lens - 1, append_pos=lens - 1)
+    a, b = harness.upload(mk()), harness.upload(mk())
+    try:
+        a.step()
+        case = b.case
+        mkh = (lambda x: torch.from_numpy(np.ascontiguousarray(x)).pin_memory()) if pinned else \
+            (lambda x: torch.from_numpy(np.ascontiguousarray(x)))
+        h = [mkh(x) for x in (case.q_c, case.q_r, case.v_new, case.kr_new, case.append_pos, case.seq_lens)]
+        out_h = torch.full((case.B, 16, 64), float("nan"))
+        if pinned:
+            out_h = out_h.pin_memory()
+        scratch = torch.empty(gb.gva_step_scratch_bytes(b.handle, case.B, int(lens.max()), 0), dtype=torch.uint8,
+                              device="cuda")
+        for _ in range(2):
+            gb.gva_decode_step_host(b.handle, b.cache, b.M, h[0], h[1], h[2], h[3], h[4], h[5], out_h, scratch, case.B,
+                                    int(lens.max()), 0, b.status)
+            torch.cuda.synchronize()
+        assert int(b.status.item()) == 0
+        assert torch.equal(out_h, a.out.cpu())
+        assert torch.equal(a.v_pool, b.v_pool) and torch.equal(a.kr_pool, b.kr_pool)
+    finally:
+        a.close(); b.close()
