@@ -215,9 +215,22 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
         h->last_kernel = GVA_KERNEL_FMA;
         h->last_tile = 32;
     }
-    const cudaError_t ce = (h->cfg.d_v == 64)
-        ? launch_pdl(combine_kernel<64, 4>, dim3(B, h->cfg.H), dim3(128), 0, stream, p)
-        : launch_pdl(combine_kernel<128, 1>, dim3(B, (h->cfg.H + 3) / 4), dim3(128), 0, stream, p);
+    // Warps per head for the merge: enough that a head's records (about units / B, plus the cuts at both ends)
+    // are fetched in one or two round trips; one warp per head and four heads per block for the wide-head shape
+    // unless a sequence has many records, so that those blocks fit beside the decode kernel's blocks.
+    const long long tiles_ub = (long long)B * ((max_seq_len + h->last_tile - 1) / h->last_tile);
+    const UnitPlan est = make_unit_plan((int)tiles_ub, h->last_num_splits,
+                                        h->cfg.d_v == 64 && h->last_kernel == GVA_KERNEL_MMA);
+    const int units = num_splits > 0 ? num_splits : plan_units(est);
+    const int n_est = (num_splits > 0 ? units : units / B + 8) * p.rec_mult;
+    int wph = h->cfg.d_v == 64 ? 4 : 1;
+    while (wph < 32 && wph * 8 < n_est) wph *= 2;
+    if (h->cfg.d_v == 128 && wph <= 2) wph = 1;
+    const int hpb = wph >= 4 ? 1 : 4 / wph;
+    const size_t csmem = (size_t)wph * hpb * (h->cfg.d_v + 2) * sizeof(float);
+    const dim3 cgrid(B, (h->cfg.H + hpb - 1) / hpb), cblock(32 * wph * hpb);
+    const cudaError_t ce = (h->cfg.d_v == 64) ? launch_pdl(combine_kernel<64>, cgrid, cblock, csmem, stream, p, wph, hpb)
+                                              : launch_pdl(combine_kernel<128>, cgrid, cblock, csmem, stream, p, wph, hpb);
     if (ce != cudaSuccess) {
         (void)cudaGetLastError();
         (void)cudaMemsetAsync(h->ticket, 0, sizeof(int32_t), stream);   // the merge that would have reset it never ran

@@ -264,33 +264,34 @@ step_front_kernel(StepFrontParams a, RopeTable rope) {
 }
 
 // ---- LSE combine ---------------------------------------------------------------------------------
-// block 128 = 4 warps; WPH warps share one (sequence, head), so a block covers 4 / WPH heads:
-//   WPH = 4 (d_v = 64):  grid (B, H).     Warp w takes records w, w+4, ... -- 32 records per memory round trip
-//                        per block -- and the four warp states are merged through shared memory.
-//   WPH = 1 (d_v = 128): grid (B, H / 4). One warp per head, no shared memory, so that every block fits beside
-//                        the decode kernel's blocks and is already resident when that kernel ends.
-// Each warp requests kCombineUnroll records' (max, sum) pairs and partial outputs before using any, and keeps
-// a running (m, L, acc) by the usual rescaling; everything is merged in a fixed order, so the result is
-// reproducible for fixed launch geometry.
+// A block holds hpb heads of one sequence, wph warps per head (blockDim = 32 * wph * hpb, grid (B, H / hpb)).
+// Warp `part` of a head takes records part, part + wph, ...; eight records' (max, sum) pairs and partial outputs
+// are requested before any is used, so a head covers 8 * wph records per memory round trip.  Each warp keeps a
+// running (m, L, acc) by the usual rescaling and the wph warp states are merged through shared memory in a fixed
+// order, so the result is reproducible for fixed launch geometry.  The host picks wph from the number of
+// records a sequence can have (many for a single long sequence, few for a large batch).
 //   m* = max_r m_r ;  L = sum_r l_r 2^(m_r - m*) ;  out = sum_r 2^(m_r - m*) o_r / L ;  lse = (m* + log2 L) ln 2
+//
 // The body runs twice: a first, "dry" pass while the block still waits for the decode kernel (reads of the
 // workspace are discarded, nothing is written), then the real pass after the wait.  Both passes execute the
 // same instructions, so the real pass finds them in the SM's instruction cache; a kernel this short otherwise
 // spends most of its time on cold instruction fetches, because the cache stream has pushed its code out of L2
 // since the previous call.
-template <int DV, int WPH>
-__global__ void __launch_bounds__(128)
-combine_kernel(DecodeParams p) {
+template <int DV>
+__global__ void __launch_bounds__(1024)
+combine_kernel(DecodeParams p, int wph, int hpb) {
     grid_dependency_launch();
     constexpr int DPL = DV / 32;
     constexpr int UNROLL = 8;
     using VecT = typename std::conditional<DPL == 2, float2, float4>::type;
-    __shared__ float s_acc[WPH > 1 ? 4 : 1][WPH > 1 ? DV : 1];
-    __shared__ float s_ml[4][2];
+    extern __shared__ float s_comb[];            // [hpb * wph][DV] partial outputs, then [hpb * wph][2] (m, L)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_warps = wph * hpb;
+    float *s_acc = s_comb;
+    float *s_ml = s_comb + n_warps * DV;
     const int b = blockIdx.x;
-    const int h = blockIdx.y * (4 / WPH) + warp / WPH;
-    const int part = warp % WPH;
+    const int h = blockIdx.y * hpb + warp / wph;
+    const int part = warp % wph;
     const bool active = h < p.H;
     const int hh = active ? h : 0;
 
@@ -313,17 +314,17 @@ combine_kernel(DecodeParams p) {
         }
         if (dry) {      // whatever the header holds right now, stay inside the workspace
             first = 0;
-            n = WPH * UNROLL;
+            n = wph * UNROLL < 32 ? wph * UNROLL : 32;
         }
         float m_w = -INFINITY, L_w = 0.f, acc[DPL];
 #pragma unroll
         for (int d = 0; d < DPL; ++d) acc[d] = 0.f;
-        for (int r0 = part; r0 < n; r0 += WPH * UNROLL) {
+        for (int r0 = part; r0 < n; r0 += wph * UNROLL) {
             float2 ml[UNROLL];
             VecT v[UNROLL];
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
-                const int r = r0 + WPH * u;
+                const int r = r0 + wph * u;
                 ml[u] = make_float2(-INFINITY, 0.f);
                 if (r < n) {
                     const size_t rh = (size_t)(first + r) * p.H + hh;
@@ -359,29 +360,30 @@ combine_kernel(DecodeParams p) {
         float mstar = m_w, L = L_w, o[DPL];
 #pragma unroll
         for (int d = 0; d < DPL; ++d) o[d] = acc[d];
-        if constexpr (WPH > 1) {
-            __syncthreads();                             // previous pass has finished reading shared memory
+        if (wph > 1) {                                   // block-uniform
+            __syncthreads();                             // the previous pass has finished reading shared memory
 #pragma unroll
-            for (int d = 0; d < DPL; ++d) s_acc[warp][lane * DPL + d] = acc[d];
+            for (int d = 0; d < DPL; ++d) s_acc[warp * DV + lane * DPL + d] = acc[d];
             if (lane == 0) {
-                s_ml[warp][0] = m_w;
-                s_ml[warp][1] = L_w;
+                s_ml[warp * 2] = m_w;
+                s_ml[warp * 2 + 1] = L_w;
             }
             __syncthreads();
-            const int w0 = warp - part;
-            mstar = -INFINITY;
+            if (part == 0) {
+                const int w0 = warp;
+                mstar = -INFINITY;
+                for (int w = 0; w < wph; ++w) mstar = fmaxf(mstar, s_ml[(w0 + w) * 2]);
+                L = 0.f;
 #pragma unroll
-            for (int w = 0; w < WPH; ++w) mstar = fmaxf(mstar, s_ml[w0 + w][0]);
-            L = 0.f;
+                for (int d = 0; d < DPL; ++d) o[d] = 0.f;
+                for (int w = 0; w < wph; ++w) {
+                    const float mw = s_ml[(w0 + w) * 2];
+                    if (!(mw > -INFINITY)) continue;
+                    const float sc = exp2f(mw - mstar);
+                    L = fmaf(s_ml[(w0 + w) * 2 + 1], sc, L);
 #pragma unroll
-            for (int d = 0; d < DPL; ++d) o[d] = 0.f;
-#pragma unroll
-            for (int w = 0; w < WPH; ++w) {
-                if (!(s_ml[w0 + w][0] > -INFINITY)) continue;
-                const float sc = exp2f(s_ml[w0 + w][0] - mstar);
-                L = fmaf(s_ml[w0 + w][1], sc, L);
-#pragma unroll
-                for (int d = 0; d < DPL; ++d) o[d] = fmaf(sc, s_acc[w0 + w][lane * DPL + d], o[d]);
+                    for (int d = 0; d < DPL; ++d) o[d] = fmaf(sc, s_acc[(w0 + w) * DV + lane * DPL + d], o[d]);
+                }
             }
         }
         const bool live = mstar > -INFINITY;
