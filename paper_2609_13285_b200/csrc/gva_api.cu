@@ -294,7 +294,7 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
     }
 #endif
     // the absorb kernel may need more than 48 KB for a 128 x 128 map
-    const size_t absorb_smem = ((size_t)cfg->d_v * (cfg->d_c + 1) + (size_t)kAbsorbBatch * cfg->d_c) * 4;
+    const size_t absorb_smem = absorb_smem_bytes(cfg->d_v, cfg->d_c);
     if (absorb_smem > (size_t)optin ||
         cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)absorb_smem) != cudaSuccess ||
         cudaFuncSetAttribute(step_front_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -328,7 +328,7 @@ int gva_absorb_query(gva_handle *h, const float *q_c, const float *q_r, const fl
     if (!aligned(q_c, 4) || !aligned(q_r, 4) || !aligned(M, 4) || !aligned(q_pos, 4) || !aligned(q_abs, 16))
         return GVA_ERR_INVALID_ARG;
     const gva_config &c = h->cfg;
-    const size_t smem = ((size_t)c.d_v * (c.d_c + 1) + (size_t)kAbsorbBatch * c.d_c) * 4;
+    const size_t smem = absorb_smem_bytes(c.d_v, c.d_c);
     dim3 grid(c.H, (B + kAbsorbBatch - 1) / kAbsorbBatch);
     if (launch_pdl(absorb_kernel, grid, dim3(kAbsorbThreads), smem, static_cast<cudaStream_t>(stream), q_c, q_r, M, q_pos,
                    q_abs, B, c.H, c.d_v, c.d_c, c.d_r, h->rope) != cudaSuccess) {
@@ -429,7 +429,7 @@ int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const
     a.B = B; a.H = c.H; a.G = c.G; a.d_v = c.d_v; a.d_c = c.d_c; a.d_r = c.d_r; a.P = c.page_size;
     a.num_pages = cache->num_pages; a.max_pages = cache->max_pages_per_seq;
     a.n_absorb = c.H * ((B + kAbsorbBatch - 1) / kAbsorbBatch);
-    const size_t smem = ((size_t)c.d_v * (c.d_c + 1) + (size_t)kAbsorbBatch * c.d_c) * 4;
+    const size_t smem = absorb_smem_bytes(c.d_v, c.d_c);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const cudaError_t ce = (c.cache_dtype == GVA_BF16)
         ? launch_pdl(step_front_kernel<__nv_bfloat16>, dim3(a.n_absorb + B), dim3(kAbsorbThreads), smem, st, a, h->rope)

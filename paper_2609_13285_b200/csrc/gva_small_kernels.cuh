@@ -40,32 +40,49 @@ __device__ __forceinline__ void rope_pair(double x0, double x1, int pos, double 
 
 // ---- absorb --------------------------------------------------------------------------------------
 // grid (H, ceil(B / kAbsorbBatch)), block 256.  M_h is staged once per block in shared memory
-// (row stride d_c + 1 floats, conflict-free for the row-per-thread dot products) with all of a
-// thread's 16-byte loads in flight at once, and reused for kAbsorbBatch sequences.
+// (row stride d_c + 4 floats: 16-byte aligned for cp.async and conflict-free for 16-byte row-per-thread
+// reads), and reused for kAbsorbBatch sequences.
 constexpr int kAbsorbBatch = 8;
 constexpr int kAbsorbThreads = 256;
 
+// Shared-memory row stride of the staged map, in floats: d_c + 4 keeps rows 16-byte aligned for cp.async.
+__host__ __device__ __forceinline__ int absorb_row_stride(int d_c) { return d_c + 4; }
+__host__ __device__ __forceinline__ size_t absorb_smem_bytes(int d_v, int d_c) {
+    return ((size_t)d_v * absorb_row_stride(d_c) + (size_t)kAbsorbBatch * d_c) * sizeof(float);
+}
+
 // One block's share: head h, sequences [b0, b0 + kAbsorbBatch).  All kAbsorbThreads threads must call it.
+// Every global read is requested up front -- M_h and the query rows as 16-byte cp.async copies straight into
+// shared memory, the RoPE inputs into registers -- so the block pays one memory round trip.
 __device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, const float *__restrict__ q_r,
                                              const float *__restrict__ M, const int32_t *__restrict__ q_pos,
                                              float *__restrict__ q_abs, int B, int H, int d_v, int d_c, int d_r,
                                              const RopeTable &rope, int h, int b0, float *smem_f) {
-    float *sM = smem_f;                            // [d_v][d_c + 1]
-    float *sq = smem_f + d_v * (d_c + 1);          // [kAbsorbBatch][d_c]
+    const int ld = absorb_row_stride(d_c);
+    float *sM = smem_f;                            // [d_v][ld]
+    float *sq = smem_f + d_v * ld;                 // [kAbsorbBatch][d_c]
     const int nb = min(kAbsorbBatch, B - b0);
     const int tid = threadIdx.x;
     const float *Mh = M + (size_t)h * d_v * d_c;
-    const int n_elem = d_v * d_c;
     const int dq = d_v + d_r;
     const int half = d_r / 2;
-    // Every global load this block needs is requested before the first one is used, so the block pays one
-    // memory round trip instead of one per phase: the query rows, the RoPE inputs, then the map.
-    constexpr int kQPer = (kAbsorbBatch * 256 + kAbsorbThreads - 1) / kAbsorbThreads;   // d_c <= 256
-    float qreg[kQPer];
-#pragma unroll
-    for (int u = 0; u < kQPer; ++u) {
-        const int i = u * kAbsorbThreads + tid;
-        qreg[u] = (i < nb * d_c) ? q_c[((size_t)(b0 + i / d_c) * H + h) * d_c + (i % d_c)] : 0.f;
+    const bool vec = (d_c & 3) == 0 && (reinterpret_cast<uintptr_t>(q_c) & 15) == 0 && (reinterpret_cast<uintptr_t>(M) & 15) == 0;
+    if (vec) {
+        const int cpr = d_c >> 2;                  // 16-byte chunks per row
+        const uint32_t sM_u32 = smem_u32(sM), sq_u32 = smem_u32(sq);
+        for (int c = tid; c < d_v * cpr; c += kAbsorbThreads) {
+            const int row = c / cpr, col = c % cpr;
+            cp_async16(sM_u32 + (row * ld + col * 4) * 4, Mh + (size_t)row * d_c + col * 4, 16);
+        }
+        for (int c = tid; c < nb * cpr; c += kAbsorbThreads) {
+            const int bb = c / cpr, col = c % cpr;
+            cp_async16(sq_u32 + (bb * d_c + col * 4) * 4, q_c + ((size_t)(b0 + bb) * H + h) * d_c + col * 4, 16);
+        }
+        cp_async_commit();
+    } else {
+        for (int i = tid; i < d_v * d_c; i += kAbsorbThreads) sM[(i / d_c) * ld + (i % d_c)] = Mh[i];
+        for (int i = tid; i < nb * d_c; i += kAbsorbThreads)
+            sq[i] = q_c[((size_t)(b0 + i / d_c) * H + h) * d_c + (i % d_c)];
     }
     float r0 = 0.f, r1 = 0.f;
     int rpos = 0;
@@ -77,51 +94,45 @@ __device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, cons
         r1 = q_r[src + 1];
         rpos = q_pos[b0 + bb];
     }
-    if ((d_c & 3) == 0) {
-        const float4 *M4 = reinterpret_cast<const float4 *>(Mh);    // M is 16-byte aligned per head: d_v*d_c*4 % 16 == 0
-        const int n4 = n_elem >> 2;
-        constexpr int kMBatch = 8;
-        for (int base = 0; base < n4; base += kAbsorbThreads * kMBatch) {
-            float4 v[kMBatch];
-#pragma unroll
-            for (int u = 0; u < kMBatch; ++u) {
-                const int i = base + u * kAbsorbThreads + tid;
-                if (i < n4) v[u] = M4[i];
-            }
-#pragma unroll
-            for (int u = 0; u < kMBatch; ++u) {
-                const int i = base + u * kAbsorbThreads + tid;
-                if (i < n4) {
-                    const int e = i << 2;
-                    float *dst = sM + (e / d_c) * (d_c + 1) + (e % d_c);
-                    dst[0] = v[u].x; dst[1] = v[u].y; dst[2] = v[u].z; dst[3] = v[u].w;
-                }
-            }
-        }
-    } else {
-        for (int i = tid; i < n_elem; i += kAbsorbThreads) sM[(i / d_c) * (d_c + 1) + (i % d_c)] = Mh[i];
+    if (has_rope) {                             // the rotation overlaps with the copies in flight
+        const int bb = tid / half, i = tid % half;
+        double y0, y1;
+        rope_pair((double)r0, (double)r1, rpos, rope.inv_freq[i], y0, y1);
+        float *dst = q_abs + ((size_t)(b0 + bb) * H + h) * dq + d_v + 2 * i;
+        dst[0] = __double2float_rn(y0);
+        dst[1] = __double2float_rn(y1);
     }
-#pragma unroll
-    for (int u = 0; u < kQPer; ++u) {
-        const int i = u * kAbsorbThreads + tid;
-        if (i < nb * d_c) sq[i] = qreg[u];
-    }
+    if (vec) cp_async_wait<0>();
     __syncthreads();
     // Thread t owns map row i = t % d_v for sequences bb0, bb0 + step, ... (kAbsorbThreads % d_v == 0), so one
     // read of M_h[i][j] feeds up to four independent accumulators.
     if (kAbsorbThreads % d_v == 0 && kAbsorbBatch * d_v <= 4 * kAbsorbThreads) {
         const int i = tid % d_v, bb0 = tid / d_v, step = kAbsorbThreads / d_v;
-        const float *mrow = sM + i * (d_c + 1);
+        const float *mrow = sM + i * ld;
         const float *q0 = sq + min(bb0, nb - 1) * d_c, *q1 = sq + min(bb0 + step, nb - 1) * d_c;
         const float *q2 = sq + min(bb0 + 2 * step, nb - 1) * d_c, *q3 = sq + min(bb0 + 3 * step, nb - 1) * d_c;
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        if (vec) {      // 16-byte shared-memory reads: rows are 16-byte aligned and (d_c + 4) * 4 bytes apart, conflict-free
+            const float4 *m4 = reinterpret_cast<const float4 *>(mrow);
+            const float4 *p0 = reinterpret_cast<const float4 *>(q0), *p1 = reinterpret_cast<const float4 *>(q1);
+            const float4 *p2 = reinterpret_cast<const float4 *>(q2), *p3 = reinterpret_cast<const float4 *>(q3);
+#pragma unroll 2
+            for (int j = 0; j < (d_c >> 2); ++j) {
+                const float4 m = m4[j], x0 = p0[j], x1 = p1[j], x2 = p2[j], x3 = p3[j];
+                a0 = fmaf(x0.x, m.x, a0); a0 = fmaf(x0.y, m.y, a0); a0 = fmaf(x0.z, m.z, a0); a0 = fmaf(x0.w, m.w, a0);
+                a1 = fmaf(x1.x, m.x, a1); a1 = fmaf(x1.y, m.y, a1); a1 = fmaf(x1.z, m.z, a1); a1 = fmaf(x1.w, m.w, a1);
+                a2 = fmaf(x2.x, m.x, a2); a2 = fmaf(x2.y, m.y, a2); a2 = fmaf(x2.z, m.z, a2); a2 = fmaf(x2.w, m.w, a2);
+                a3 = fmaf(x3.x, m.x, a3); a3 = fmaf(x3.y, m.y, a3); a3 = fmaf(x3.z, m.z, a3); a3 = fmaf(x3.w, m.w, a3);
+            }
+        } else {
 #pragma unroll 4
-        for (int j = 0; j < d_c; ++j) {
-            const float m = mrow[j];
-            a0 = fmaf(q0[j], m, a0);
-            a1 = fmaf(q1[j], m, a1);
-            a2 = fmaf(q2[j], m, a2);
-            a3 = fmaf(q3[j], m, a3);
+            for (int j = 0; j < d_c; ++j) {
+                const float m = mrow[j];
+                a0 = fmaf(q0[j], m, a0);
+                a1 = fmaf(q1[j], m, a1);
+                a2 = fmaf(q2[j], m, a2);
+                a3 = fmaf(q3[j], m, a3);
+            }
         }
         const float acc[4] = {a0, a1, a2, a3};
 #pragma unroll
@@ -132,20 +143,12 @@ __device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, cons
     } else {
         for (int o = tid; o < nb * d_v; o += kAbsorbThreads) {
             const int bb = o / d_v, i = o % d_v;
-            const float *mrow = sM + i * (d_c + 1);
+            const float *mrow = sM + i * ld;
             const float *qrow = sq + bb * d_c;
             float acc = 0.f;
             for (int j = 0; j < d_c; ++j) acc = fmaf(qrow[j], mrow[j], acc);
             q_abs[((size_t)(b0 + bb) * H + h) * dq + i] = acc;
         }
-    }
-    if (has_rope) {
-        const int bb = tid / half, i = tid % half;
-        double y0, y1;
-        rope_pair((double)r0, (double)r1, rpos, rope.inv_freq[i], y0, y1);
-        float *dst = q_abs + ((size_t)(b0 + bb) * H + h) * dq + d_v + 2 * i;
-        dst[0] = __double2float_rn(y0);
-        dst[1] = __double2float_rn(y1);
     }
 }
 
