@@ -349,6 +349,46 @@ def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with
     return res
 
 
+def measure_gqa(rank, local_rank, dist, args, kernel, torch, gb, harness):
+    """Matched GQA decode (two cached streams of the same grouping: H=16, G=4, d_h=64, B=32, T=32768, paged) through
+    gqa_decode, for the cache-bytes comparison N_GVA / N_GQA = 1/2 + d_r / (2 G d_h)."""
+    from paper_2609_13285_b200 import multirank, workloads as wl
+    dev = torch.device("cuda", local_rank)
+    g = wl.gqa_case("gqa-cfg2", 16, 4, 64, [32768] * 32, page_size=64, paged=True, cache_dtype="bf16",
+                    seed=wl.MASTER_SEED + 5000 + 7919 * rank)
+    dc = harness.upload_gqa(g, device=dev, kernel=kernel)
+    pools = [(dc.k_pool, dc.v_pool), (dc.k_pool.clone(), dc.v_pool.clone())]
+    caches = [gb.make_gqa_cache(k, v, dc.block_table, g["num_pages"], g["max_pages_per_seq"]) for k, v in pools]
+    B, max_len = g["B"], int(g["seq_lens"].max())
+    ws = torch.empty(gb.gva_decode_workspace_bytes(dc.handle, B, max_len, 0), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    steps, warmup = max(20, args.steps // 3), 10
+
+    def call(i):
+        gb.gqa_decode(dc.handle, caches[i & 1], dc.q, dc.seq_lens, dc.out, dc.lse, ws, B, max_len, 0, dc.status)
+
+    for i in range(warmup):
+        call(i)
+    multirank.barrier(dist)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for i in range(steps):
+        call(i)
+    b.record(stream)
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    nbytes = 2 * int(g["seq_lens"].astype(np.int64).sum()) * g["G"] * g["d_h"] * 2
+    res = {"workload": "matched GQA decode: H=16, G=4, d_h=64, B=32, T=32768, bf16 K and V in 64-token pages",
+           "gqa_decode_ms_per_call": ms, "cache_bytes_per_call": nbytes, "cache_read_GBps": nbytes / (ms * 1e-3) / 1e9,
+           "kernel": {1: "fma", 2: "mma"}.get(gb.gva_last_kernel(dc.handle), "?"), "steps": steps,
+           "device_status": int(dc.status.item())}
+    dc.close()
+    del pools, caches
+    torch.cuda.empty_cache()
+    return res
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -408,6 +448,11 @@ def main() -> None:
                 "cache_bytes_per_step": o["cache_bytes"], "kernel": o["kernel"], "partitions": o["partitions"],
                 "total_tokens": int(o["case"].seq_lens.astype(np.int64).sum()) * o["layers"], "steps": o["steps"],
                 "clocks": o["clocks"], "device_status": o["status"]}
+
+        gq = measure_gqa(rank, local_rank, dist, short, kernel, torch, gb, harness)
+        gq["gva_over_gqa_cache_bytes"] = r["cache_bytes"] / gq["cache_bytes_per_call"]      # 0.53125 = 1/2 + 16/(2*4*64)
+        gq["gva_over_gqa_decode_time"] = decode_ms / gq["gqa_decode_ms_per_call"]
+        others["gqa_matched_cfg2"] = gq
 
     if rank == 0:
         case = r["case"]

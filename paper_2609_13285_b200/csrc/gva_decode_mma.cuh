@@ -272,17 +272,17 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                     }
                     while (f >= s_off[b + 1]) ++b;
                     const int t0 = (f - s_off[b]) * TILE;
-                    if (!waited) {
-                        const int ap = p.append_pos[b];
-                        if (ap >= t0 && ap < t0 + TILE) {   // this tile receives the new token: it must be complete first
-                            grid_dependency_wait();
-                            waited = true;
-                        }
-                    }
-                    int n_valid = min(TILE, p.seq_lens[b] - t0);
                     const int pj = t0 / p.P, slot0 = t0 % p.P;
+                    // the three lookups are independent: request them together, use them afterwards
+                    const int len = p.seq_lens[b];
+                    const int ap = waited ? -1 : p.append_pos[b];
                     long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
                                                    : (long long)b * p.max_pages + pj;
+                    if (!waited && ap >= t0 && ap < t0 + TILE) {   // this tile receives the new token: it must be complete first
+                        grid_dependency_wait();
+                        waited = true;
+                    }
+                    int n_valid = min(TILE, len - t0);
                     if (page < 0 || page >= p.num_pages) {
                         report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
                         page = 0;

@@ -363,3 +363,18 @@ def test_host_buffer_step_matches_device_step(pinned):
         assert torch.equal(a.v_pool, b.v_pool) and torch.equal(a.kr_pool, b.kr_pool)
     finally:
         a.close(); b.close()
+
+
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+def test_odd_page_size_many_short_sequences_and_one_long(kernel):
+    _mma_or_skip(kernel)
+    # 96-token pages (a multiple of 32 but not of 64), 300 short ragged sequences, and one sequence long
+    # enough that every block of the grid holds a piece of it
+    rng = np.random.default_rng(9)
+    case = wl.make_case("p96", wl.SHAPE_A, rng.integers(0, 200, size=300), page_size=96, cache_dtype="bf16", seed=214,
+                        poison_unused=True)
+    U().check_decode(case, kernel)
+    case = wl.make_case("long1", wl.SHAPE_A, [150_001], page_size=64, cache_dtype="bf16", seed=215, poison_unused=True)
+    U().check_decode(case, kernel)
+    case = wl.make_case("long1b", wl.SHAPE_B, [70_003, 5], page_size=64, cache_dtype="bf16", seed=216, poison_unused=True)
+    U().check_decode(case, kernel)
