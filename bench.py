@@ -56,6 +56,9 @@ def make_workload(name: str, rank: int):
         return wl.config3(seed=wl.MASTER_SEED + 3000 + shift)
     if name == "cfg4":
         return wl.config4_layer(0, seed=wl.MASTER_SEED + 4000 + shift)
+    if name == "cfg2-dr24":  # cfg2 with the paper's other tested RoPE width (d_r = 24: 48-byte positional rows)
+        return wl.make_case("cfg2-dr24", wl.SHAPE_C, [32768] * 32, page_size=64, cache_dtype="bf16", paged=True,
+                            seed=wl.MASTER_SEED + 2024 + shift)
     if name == "cfg2-ncu":   # profiler-sized: 143 MB of cache (> L2), same shapes and paging as cfg2
         return wl.config2(seed=wl.MASTER_SEED + 2000 + shift, B=16, T=16384)
     if name == "cfg2-small":
@@ -68,6 +71,7 @@ WORKLOAD_TEXT = {
     "cfg2": "long-context paged decode step (B=32, T=32768, 64-token pages, permuted block table)",
     "cfg3": "wider-head ragged serving batch (B=64, H=32, G=8, d_v=128, seq_lens ~ U[1024,16384], paged)",
     "cfg4": "24-layer decode step (B=128, T=8192 cached + 1 appended per layer, paged, one pool per layer)",
+    "cfg2-dr24": "cfg2 with RoPE width d_r = 24 (B=32, T=32768, paged; N_GVA/N_GQA = 0.546875)",
 }
 
 
@@ -80,7 +84,7 @@ def workload_description(name: str, case, layers: int = 1) -> dict:
         l2 = "cache stream is several times the 126 MB L2 and alternates between two pool copies"
     else:
         l2 = "cache smaller than L2: enough pool copies (>= 300 MB together) are rotated that every step streams from HBM"
-    return {"workload": f"{name}: {WORKLOAD_TEXT.get(name.split('-')[0], name)}; step = absorb + append + "
+    return {"workload": f"{name}: {WORKLOAD_TEXT.get(name, WORKLOAD_TEXT.get(name.split('-')[0], name))}; step = absorb + append + "
                         "split-KV decode + LSE combine" + (f", {layers} layers" if layers > 1 else ""),
             "B": case.B, "H": s.H, "G": s.G, "d_v": s.d_v, "d_c": s.d_c, "d_r": s.d_r, "layers": layers,
             "total_tokens": int(case.seq_lens.astype(np.int64).sum()), "max_seq_len": int(case.seq_lens.max()),
@@ -434,7 +438,7 @@ def main() -> None:
         peak = load_peaks()[0]
         short = argparse.Namespace(**vars(args))
         short.steps, short.warmup = max(20, args.steps // 3), 10
-        for other in ("cfg1", "cfg3", "cfg4"):
+        for other in ("cfg1", "cfg3", "cfg4", "cfg2-dr24"):
             o = measure(other, rank, local_rank, dist, short, kernel, torch, gb, harness, with_e2e=False,
                         with_clocks=True)
             per_layer = o["cache_bytes"] / o["layers"]

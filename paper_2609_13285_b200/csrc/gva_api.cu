@@ -113,6 +113,8 @@ bool plan_fma_t(const gva_handle *h, int B, FmaPlan *out) {
 template <bool GQA>
 bool plan_fma(const gva_handle *h, int B, FmaPlan *out) {
     const bool bf = h->cfg.cache_dtype == GVA_BF16;
+    if (h->cfg.d_v == 64 && h->cfg.d_r == 24 && !GQA)
+        return bf ? plan_fma_t<__nv_bfloat16, 64, 24, false>(h, B, out) : plan_fma_t<float, 64, 24, false>(h, B, out);
     if (h->cfg.d_v == 64)
         return bf ? plan_fma_t<__nv_bfloat16, 64, 16, GQA>(h, B, out) : plan_fma_t<float, 64, 16, GQA>(h, B, out);
     return bf ? plan_fma_t<__nv_bfloat16, 128, 32, GQA>(h, B, out) : plan_fma_t<float, 128, 32, GQA>(h, B, out);
@@ -252,7 +254,8 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
     if (cfg->cache_dtype != GVA_F32 && cfg->cache_dtype != GVA_BF16) return GVA_ERR_INVALID_ARG;
     if (cfg->kernel < GVA_KERNEL_AUTO || cfg->kernel > GVA_KERNEL_MMA) return GVA_ERR_INVALID_ARG;
     if (cfg->H % cfg->G != 0 || cfg->H / cfg->G != kHeadsPerGroup) return GVA_ERR_UNSUPPORTED;
-    if (!((cfg->d_v == 64 && cfg->d_r == 16) || (cfg->d_v == 128 && cfg->d_r == 32))) return GVA_ERR_UNSUPPORTED;
+    if (!((cfg->d_v == 64 && (cfg->d_r == 16 || cfg->d_r == 24)) || (cfg->d_v == 128 && cfg->d_r == 32)))
+        return GVA_ERR_UNSUPPORTED;
     if (cfg->G > 8 || cfg->d_c > 256 || cfg->page_size % 32 != 0) return GVA_ERR_UNSUPPORTED;
     if (cfg->kernel == GVA_KERNEL_MMA && cfg->cache_dtype != GVA_BF16) return GVA_ERR_UNSUPPORTED;
 #ifndef GVA_WITH_MMA

@@ -107,6 +107,15 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void ldsm_x2(uint32_t addr, uint32_t (&r)[2]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];\n" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_k8(float (&c)[4], const uint32_t (&a)[2], uint32_t b0) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(b0));
+}
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
     uint32_t y;
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(y) : "r"(x));
@@ -125,10 +134,11 @@ struct MmaTraits {
     static constexpr int BOXES = DV / 64;                       // 64-dim (128-byte) boxes per value row
     static constexpr int VBOX_BYTES = TILE * 128;               // one box of one group
     static constexpr int VTILE_BYTES = BOXES * VBOX_BYTES;      // one group's tile
-    static constexpr int KR_ROW = DR * 2;                       // 32 or 64 bytes
+    static constexpr int KR_ROW = DR * 2;                       // 32, 48 or 64 bytes
     static constexpr int KR_BYTES = TILE * KR_ROW;
     static constexpr int KSTEPS_V = DV / 16;
-    static constexpr int KSTEPS_R = GQA ? 0 : DR / 16;
+    static constexpr int KSTEPS_R = GQA ? 0 : DR / 16;          // full 16-wide k-steps over the RoPE dims
+    static constexpr bool KREM8 = !GQA && (DR % 16) == 8;       // d_r = 24: one more 8-wide k-step (m16n8k8)
     static constexpr int KSTEPS = KSTEPS_V + KSTEPS_R;
     static constexpr int MT = DV / 16;                          // output m-tiles
     static constexpr int CHUNKS = TILE / 16;
@@ -368,9 +378,13 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         const int row_pv = r7 + (lane >> 4) * 8, hi_pv = (lane >> 3) & 1;          // transposed: (t0-7,d0-7) (t0-7,d8-15) (t8-15,d0-7) (t8-15,d8-15)
         const uint32_t off_qk = row_qk * 128 + ((hi_qk ^ r7) << 4);
         const uint32_t off_pv = row_pv * 128 + ((hi_pv ^ r7) << 4);
-        const uint32_t off_kr = (T::KR_ROW == 32) ? row_qk * 32 + ((hi_qk ^ ((row_qk >> 2) & 1)) << 4)
-                                                  : row_qk * 64 + ((hi_qk ^ ((row_qk >> 1) & 3)) << 4);
+        // positional-key tile: 32-byte rows carry the 32-byte swizzle, 64-byte rows the 64-byte one; 48-byte rows
+        // (d_r = 24) are unswizzled -- a 48-byte stride is conflict-free for ldmatrix as it is
+        const uint32_t off_kr = (T::KR_ROW == 32)   ? row_qk * 32 + ((hi_qk ^ ((row_qk >> 2) & 1)) << 4)
+                                : (T::KR_ROW == 64) ? row_qk * 64 + ((hi_qk ^ ((row_qk >> 1) & 3)) << 4)
+                                                    : row_qk * 48 + (hi_qk << 4);
         uint32_t qf[T::KSTEPS][2];        // B fragments of Q^T: column n = lane/4 = 2*head + {hi, lo}
+        uint32_t qf8 = 0;                 // d_r = 24: B fragment of the last 8 RoPE dims
         float oacc[T::MT][4];
         float m_run = -INFINITY, l_run = 0.f;
         const float scale = p.scale_log2;
@@ -387,6 +401,11 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                     const uint32_t sx = split_hi_lo(v.x), sy = split_hi_lo(v.y);
                     qf[kk][half] = lo_part ? ((sx >> 16) | (sy & 0xffff0000u)) : ((sx & 0xffffu) | (sy << 16));
                 }
+            }
+            if constexpr (T::KREM8) {
+                const float2 v = *reinterpret_cast<const float2 *>(q + T::KSTEPS * 16 + 2 * jh);
+                const uint32_t sx = split_hi_lo(v.x), sy = split_hi_lo(v.y);
+                qf8 = lo_part ? ((sx >> 16) | (sy & 0xffff0000u)) : ((sx & 0xffffu) | (sy << 16));
             }
         };
         if (early) grid_dependency_wait();
@@ -462,6 +481,11 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                         uint32_t a[4];
                         ldsm_x4(kr_u32 + c * 16 * T::KR_ROW + (off_kr ^ (kk << 5)), a);
                         mma_bf16(sacc[c], a, qf[T::KSTEPS_V + kk][0], qf[T::KSTEPS_V + kk][1]);
+                    }
+                    if constexpr (T::KREM8) {     // dims 16..23: rows 0-7 and 8-15, third 16-byte chunk of each row
+                        uint32_t a2[2];
+                        ldsm_x2(kr_u32 + c * 16 * T::KR_ROW + row_qk * T::KR_ROW + 32, a2);
+                        mma_bf16_k8(sacc[c], a2, qf8);
                     }
                 }
             }
@@ -581,7 +605,9 @@ int launch_mma_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
         if (!encode_map(st, &tm_k, p.k_pool, DV, vrows, 64, TILE, CU_TENSOR_MAP_SWIZZLE_128B)) return GVA_ERR_CUDA;
     } else {
         if (!encode_map(st, &tm_k, p.kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, TILE,
-                        DR == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B))
+                        DR == 16   ? CU_TENSOR_MAP_SWIZZLE_32B
+                        : DR == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                   : CU_TENSOR_MAP_SWIZZLE_NONE))
             return GVA_ERR_CUDA;
     }
     const int threads = 32 * (G * WPG + 1);
@@ -616,6 +642,13 @@ int launch_decode_mma(const gva_config &cfg, const MmaHostState &st, int sm_coun
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
     *tile_out = mma_tile_for(cfg, GQA);
     *rec_mult_out = mma_warps_per_group(cfg, GQA);
+    if (cfg.d_v == 64 && cfg.d_r == 24 && !GQA) {
+        if (*tile_out == 64)
+            return launch_mma_t<64, 24, 64, 3, GVA_MMA_WPG64, false>(cfg, st, sm_count, smem_optin, p, B, max_seq_len,
+                                                                     num_splits, max_blocks, stream, n_blocks_out);
+        return launch_mma_t<64, 24, 32, 3, GVA_MMA_WPG64, false>(cfg, st, sm_count, smem_optin, p, B, max_seq_len,
+                                                                 num_splits, max_blocks, stream, n_blocks_out);
+    }
     if (cfg.d_v == 64 && *tile_out == 64)
         return launch_mma_t<64, 16, 64, 3, GVA_MMA_WPG64, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks,
                                                    stream, n_blocks_out);

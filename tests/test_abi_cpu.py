@@ -53,7 +53,8 @@ def test_create_rejects_bad_configs_on_the_host(lib):
     assert _create(H=16, G=3)[0] == gb.GVA_ERR_UNSUPPORTED           # H % G != 0
     assert _create(H=16, G=8)[0] == gb.GVA_ERR_UNSUPPORTED           # H / G != 4
     assert _create(d_v=96)[0] == gb.GVA_ERR_UNSUPPORTED
-    assert _create(d_r=24)[0] == gb.GVA_ERR_UNSUPPORTED
+    assert _create(d_r=20)[0] == gb.GVA_ERR_UNSUPPORTED
+    assert _create(d_v=128, d_r=24)[0] == gb.GVA_ERR_UNSUPPORTED
     assert _create(page_size=48)[0] == gb.GVA_ERR_UNSUPPORTED
     assert _create(cache_dtype=7)[0] == gb.GVA_ERR_INVALID_ARG
     assert _create(rope_base=0.5)[0] == gb.GVA_ERR_INVALID_ARG

@@ -37,7 +37,7 @@ def _mma_or_skip(kernel):
 
 
 # ------------------------------------------------------------------ absorb
-@pytest.mark.parametrize("shape,B", [(wl.SHAPE_A, 1), (wl.SHAPE_A, 19), (wl.SHAPE_B, 9)])
+@pytest.mark.parametrize("shape,B", [(wl.SHAPE_A, 1), (wl.SHAPE_A, 19), (wl.SHAPE_B, 9), (wl.SHAPE_C, 11)])
 def test_absorb_matches_oracle(shape, B):
     lens = np.arange(B) * 37 + 5
     case = wl.make_case("absorb", shape, lens, page_size=64, cache_dtype="bf16", seed=101,
@@ -55,7 +55,7 @@ def test_absorb_matches_oracle(shape, B):
 
 # ------------------------------------------------------------------ append (bit exact)
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C])
 def test_append_is_bit_exact_and_touches_nothing_else(dtype, shape):
     lens = [1, 64, 65, 300, 129, 4000, 8193]
     case = wl.make_case("append", shape, lens, page_size=64, cache_dtype=dtype, seed=102, extra_pages=3)
@@ -137,7 +137,7 @@ EDGE_LENS = [0, 1, 31, 32, 33, 63, 64, 65, 127, 128, 129, 640, 641, 1000]
 
 
 @pytest.mark.parametrize("kernel", KERNELS_BF16)
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C])
 @pytest.mark.parametrize("num_splits", [0, 1, 5, 40])
 def test_ragged_edge_lengths_poisoned(kernel, shape, num_splits):
     # lengths around tile and page boundaries, an empty sequence, more splits than tiles;
@@ -148,7 +148,7 @@ def test_ragged_edge_lengths_poisoned(kernel, shape, num_splits):
     U().check_decode(case, kernel, num_splits=num_splits)
 
 
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C])
 @pytest.mark.parametrize("num_splits", [0, 3])
 def test_ragged_edge_lengths_f32(shape, num_splits):
     case = wl.make_case("edge32", shape, EDGE_LENS, page_size=64, cache_dtype="f32", seed=202, poison_unused=True)
@@ -276,7 +276,7 @@ def test_full_step_follows_algorithm_order(kernel):
 
 # ------------------------------------------------------------------ fused step entry point
 @pytest.mark.parametrize("kernel", KERNELS_BF16)
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C])
 def test_fused_step_is_bitwise_the_three_calls(kernel, shape):
     _mma_or_skip(kernel)
     lens = np.array([1, 64, 65, 1001, 4096, 130], dtype=np.int32)
