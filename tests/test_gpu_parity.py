@@ -378,3 +378,40 @@ def test_odd_page_size_many_short_sequences_and_one_long(kernel):
     U().check_decode(case, kernel)
     case = wl.make_case("long1b", wl.SHAPE_B, [70_003, 5], page_size=64, cache_dtype="bf16", seed=216, poison_unused=True)
     U().check_decode(case, kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS_BF16)
+def test_workspace_and_outputs_stay_inside_their_bounds(kernel):
+    # guard bands around the workspace, the outputs and the absorbed queries must survive every kind of call
+    _mma_or_skip(kernel)
+    lens = np.array([5000, 64, 0, 1, 777], dtype=np.int32)
+    case = wl.make_case("canary", wl.SHAPE_A, lens, page_size=64, cache_dtype="bf16", seed=217,
+                        q_pos=np.maximum(lens - 1, 0), append_pos=np.maximum(lens - 1, 0))
+    dc = harness.upload(case, kernel=kernel)
+    try:
+        B, guard = case.B, 4096
+        def banded(nbytes):
+            buf = torch.full((nbytes + 2 * guard,), 0x5A, dtype=torch.uint8, device="cuda")
+            return buf, buf[guard:guard + nbytes]
+        checks = []
+        for ns in (0, 3):
+            need = gb.gva_decode_workspace_bytes(dc.handle, B, int(lens.max()), ns)
+            ws_full, ws = banded(need)
+            out_full, out_b = banded(B * 16 * 64 * 4)
+            lse_full, lse_b = banded(B * 16 * 4)
+            qa_full, qa_b = banded(B * 16 * 80 * 4)
+            out, lse, q_abs = out_b.view(torch.float32), lse_b.view(torch.float32), qa_b.view(torch.float32)
+            gb.gva_absorb_query(dc.handle, dc.q_c, dc.q_r, dc.M, dc.q_pos, q_abs, B)
+            gb.gva_decode(dc.handle, dc.cache, q_abs, dc.seq_lens, out, lse, ws, B, int(lens.max()), ns, dc.status,
+                          workspace_bytes=need)
+            gb.gva_decode_step(dc.handle, dc.cache, dc.M, dc.q_c, dc.q_r, dc.v_new, dc.kr_new, dc.append_pos, dc.seq_lens,
+                               q_abs, out, lse, ws, B, int(lens.max()), ns, dc.status)
+            torch.cuda.synchronize()
+            for full, n in ((ws_full, need), (out_full, out.numel() * 4), (lse_full, lse.numel() * 4),
+                            (qa_full, q_abs.numel() * 4)):
+                checks.append(bool((full[:guard] == 0x5A).all()) and bool((full[guard + n:] == 0x5A).all()))
+            assert torch.isfinite(out).all()
+        assert all(checks)
+        assert int(dc.status.item()) == 0
+    finally:
+        dc.close()
