@@ -233,6 +233,33 @@ void oracle_gqa_decode(const void *k_pool, const void *v_pool, int dtype, const 
         }
 }
 
+/* ---- the projections around the attention (Algorithm 1: q_t = x_t W_Q, v_t = x_t W_V, x_t W_r; then
+ * "the usual concatenation and output projection") ---------------------------------------------------
+ * Plain matrix product y[b][n] = sum_k x[b][k] W[k][n], fp64. */
+void oracle_matmul(const double *x, const double *W, int B, int K, int N, double *y) {
+#pragma omp parallel for schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int k = 0; k < K; ++k) acc += x[(int64_t)b * K + k] * W[(int64_t)k * N + n];
+            y[(int64_t)b * N + n] = acc;
+        }
+}
+
+/* Weight absorption: because M_h is fixed at inference, q~_h = (x W_Q^{nope,h}) M_h^T = x (W_Q^{nope,h} M_h^T)
+ * (Eq. absorb applied to the projection).  W_q_nope [d_model][H][d_c], M [H][d_v][d_c] ->
+ * W_abs [d_model][H][d_v] with W_abs[m][h][i] = sum_j W_q_nope[m][h][j] M[h][i][j]. */
+void oracle_fold_maps(const double *W_q_nope, const double *M, int d_model, int H, int d_v, int d_c, double *W_abs) {
+    for (int m = 0; m < d_model; ++m)
+        for (int h = 0; h < H; ++h)
+            for (int i = 0; i < d_v; ++i) {
+                double acc = 0.0;
+                for (int j = 0; j < d_c; ++j)
+                    acc += W_q_nope[((int64_t)m * H + h) * d_c + j] * M[((int64_t)h * d_v + i) * d_c + j];
+                W_abs[((int64_t)m * H + h) * d_v + i] = acc;
+            }
+}
+
 #ifdef _OPENMP
 #include <omp.h>
 int oracle_num_threads(void) { return omp_get_max_threads(); }

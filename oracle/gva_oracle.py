@@ -173,6 +173,79 @@ def gqa_decode(k_pool, v_pool, block_table, seq_lens, q, scale: Optional[float] 
     return out, lse
 
 
+# ---- projections around the attention (Algorithm 1's first lines and the output projection) ----
+def matmul(x, W) -> np.ndarray:
+    """y = x W by the plain triple loop in fp64."""
+    x, W = _f64(x), _f64(W)
+    B, K = x.shape
+    K2, N = W.shape
+    assert K == K2
+    y = np.empty((B, N), dtype=np.float64)
+    lib().oracle_matmul(_p(x), _p(W), *map(ctypes.c_int, (B, K, N)), _p(y))
+    return y
+
+
+def fold_maps(W_q_nope, M) -> np.ndarray:
+    """W_abs[m,h,:] = W_q_nope[m,h,:] M_h^T  ([d_model,H,d_c] x [H,d_v,d_c] -> [d_model,H,d_v])."""
+    W_q_nope, M = _f64(W_q_nope), _f64(M)
+    d_model, H, d_c = W_q_nope.shape
+    d_v = M.shape[1]
+    out = np.empty((d_model, H, d_v), dtype=np.float64)
+    lib().oracle_fold_maps(_p(W_q_nope), _p(M), *map(ctypes.c_int, (d_model, H, d_v, d_c)), _p(out))
+    return out
+
+
+def bf16_round(a) -> np.ndarray:
+    """Values rounded to bfloat16 (nearest even, straight from fp64), returned as uint16 bit patterns."""
+    a = _f64(a)
+    out = np.empty(a.shape, dtype=np.uint16)
+    flat, of = a.ravel(), out.ravel()
+    for i in range(flat.size):
+        of[i] = lib().oracle_bf16_from_double(ctypes.c_double(float(flat[i])))
+    return out
+
+
+def pack_input_weights(W_q_nope, W_q_rope, W_v, W_r, M) -> np.ndarray:
+    """The packed input projection [d_model, H*(d_v+d_r) + G*d_v + d_r] in fp64: per head the folded content
+    columns W_q_nope_h M_h^T then the positional query columns, then the value columns, then the positional key."""
+    W_q_nope, W_q_rope, W_v, W_r = _f64(W_q_nope), _f64(W_q_rope), _f64(W_v), _f64(W_r)
+    d_model, H, _ = W_q_nope.shape
+    W_abs = fold_maps(W_q_nope, M)
+    per_head = np.concatenate([W_abs, W_q_rope], axis=2)                  # [d_model, H, d_v + d_r]
+    return np.concatenate([per_head.reshape(d_model, -1), W_v.reshape(d_model, -1), W_r.reshape(d_model, -1)], axis=1)
+
+
+def project_in(x, W_in, H: int, G: int, d_v: int, d_r: int):
+    """x W_in split into (q_tilde [B,H,d_v], q_rope [B,H,d_r] unrotated, v_new [B,G,d_v], kr_new [B,d_r] unrotated)."""
+    y = matmul(x, W_in)
+    B = y.shape[0]
+    nq = H * (d_v + d_r)
+    qh = y[:, :nq].reshape(B, H, d_v + d_r)
+    v = y[:, nq:nq + G * d_v].reshape(B, G, d_v)
+    kr = y[:, nq + G * d_v:]
+    assert kr.shape[1] == d_r
+    return qh[..., :d_v].copy(), qh[..., d_v:].copy(), v.copy(), kr.copy()
+
+
+def layer_step(x, W_in, W_o, v_pool, kr_pool, block_table, pos, seq_lens, H: int, G: int, d_c: int,
+               base: float = 10000.0, max_pages_per_seq: Optional[int] = None):
+    """One whole decode step of a GVA layer from the hidden state (Algorithm 1, then the output projection):
+    project, rotate, append to the cache (in place), attend, concatenate heads, project out.
+    Returns (y [B,d_model], attention output [B,H,d_v], q_abs [B,H,d_v+d_r])."""
+    _, Gp, P, d_v = v_pool.shape
+    d_r = kr_pool.shape[-1]
+    assert Gp == G
+    q_t, q_r, v_new, kr_new = project_in(x, W_in, H, G, d_v, d_r)
+    pos = _i32(pos)
+    q_abs = np.concatenate([q_t, np.stack([rope(q_r[b], int(pos[b]), base) for b in range(len(pos))])], axis=2)
+    rc = append(v_pool, kr_pool, block_table, v_new, kr_new, pos, base, max_pages_per_seq=max_pages_per_seq)
+    assert rc == 0
+    out, _ = decode(v_pool, kr_pool, block_table, seq_lens, q_abs, H, scale=1.0 / np.sqrt(float(d_c + d_r)),
+                    max_pages_per_seq=max_pages_per_seq)
+    y = matmul(out.reshape(out.shape[0], -1), W_o)
+    return y, out, q_abs
+
+
 # ---- convenience over a workloads.DecodeCase-like object (duck-typed; no import of the generator) ----
 def absorb_case(case) -> np.ndarray:
     return absorb(case.q_c, case.q_r, case.M, case.q_pos, case.rope_base)

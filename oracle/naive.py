@@ -2,7 +2,7 @@
 
 TEST INFRASTRUCTURE ONLY.  Used to brute-force hand-sized cases and to cross-check the C oracle
 (oracle/gva_oracle.c); written separately from it, following Algorithm 1 of the paper line by
-line in its notation (1-based steps of the algorithm are noted beside the code).  Cache values are
+line in its notation.  Cache values are
 plain Python floats (already widened from whatever storage type).
 """
 from __future__ import annotations
@@ -99,3 +99,36 @@ def gather_tokens(v_pool, kr_pool, block_table: Optional[Sequence[Sequence[int]]
         V_tokens.append(vt)
         KR_tokens.append(kt)
     return V_tokens, KR_tokens
+
+
+def layer_decode_step(x, W_Q, W_V, W_r, W_O, M, t: int, V_cache, KR_cache, H: int, G: int, d_c: int, d_r: int,
+                      base: float = 10000.0):
+    """Algorithm 1 line by line for ONE sequence, starting from the hidden state x (list of d_model floats).
+
+    W_Q[m][h] = list of d_r + d_c floats (positional slice first, then content slice, as the algorithm's split
+    "q^rope, q^nope" lists them), W_V[m][g] = list of d_v, W_r[m] = list of d_r, W_O[h*d_v + i] = list of d_model.
+    V_cache[g] = list of cached value rows, KR_cache = list of cached rotated positional keys; both are extended
+    in place.  Keys are materialised explicitly (K = V M), nothing is absorbed.  Returns (y, per-head outputs)."""
+    d_model = len(x)
+    d_v = len(M[0])
+    # q_t <- x_t W_Q ; split each head into q^rope, q^nope
+    q = [[sum(x[m] * W_Q[m][h][c] for m in range(d_model)) for c in range(d_r + d_c)] for h in range(H)]
+    q_rope = [q[h][:d_r] for h in range(H)]
+    q_nope = [q[h][d_r:] for h in range(H)]
+    # v_t <- x_t W_V ; append one row per value group
+    for g in range(G):
+        V_cache[g].append([sum(x[m] * W_V[m][g][i] for m in range(d_model)) for i in range(d_v)])
+    # k^rope_t <- (x_t W_r) R_t^T ; append
+    KR_cache.append(rope([sum(x[m] * W_r[m][k] for m in range(d_model)) for k in range(d_r)], t, base))
+    outs = []
+    for h in range(H):
+        g = h // (H // G)
+        qr = rope(q_rope[h], t, base)                                   # q^rope <- q^rope R_t^T
+        keys = [reconstruct_key(v, M[h]) for v in V_cache[g]]           # K^nope = V M_h, materialised
+        s = [(sum(a * b for a, b in zip(q_nope[h], keys[j])) + sum(a * b for a, b in zip(qr, KR_cache[j])))
+             / math.sqrt(d_c + d_r) for j in range(len(keys))]          # scores, with explicit keys instead of q~
+        p = softmax(s)
+        outs.append([sum(p[j] * V_cache[g][j][i] for j in range(len(keys))) for i in range(d_v)])   # o <- softmax(s) V
+    concat = [v for o in outs for v in o]
+    y = [sum(concat[r] * W_O[r][m] for r in range(len(concat))) for m in range(d_model)]
+    return y, outs

@@ -277,3 +277,18 @@ def gqa_case(name: str, H: int, G: int, d_h: int, seq_lens, *, page_size: int = 
     q = rng.standard_normal((B, H, d_h), dtype=np.float32)
     return dict(name=name, H=H, G=G, d_h=d_h, B=B, page_size=P, num_pages=num_pages, max_pages_per_seq=max_pages,
                 k_pool=k_pool, v_pool=v_pool, block_table=bt, seq_lens=seq_lens, q=q, cache_dtype=cache_dtype)
+
+
+def layer_weights(shape: HeadShape, d_model: int, B: int, seed: int = MASTER_SEED + 6000) -> dict:
+    """Seeded projections around the attention of one layer and one hidden state per sequence.
+    Every weight ~ N(0, 1/fan_in) (so projected activations stay unit-scale), x ~ N(0, 1):
+      W_q_nope [d_model, H, d_c], W_q_rope [d_model, H, d_r], W_v [d_model, G, d_v], W_r [d_model, d_r],
+      W_o [H*d_v, d_model], x [B, d_model]."""
+    rng = _rng(seed)
+    sd = np.float32(1.0 / np.sqrt(d_model))
+    n = lambda *sh: (rng.standard_normal(sh, dtype=np.float32) * sd).astype(np.float32)
+    return dict(d_model=d_model, W_q_nope=n(d_model, shape.H, shape.d_c), W_q_rope=n(d_model, shape.H, shape.d_r),
+                W_v=n(d_model, shape.G, shape.d_v), W_r=n(d_model, shape.d_r),
+                W_o=(rng.standard_normal((shape.H * shape.d_v, d_model), dtype=np.float32)
+                     * np.float32(1.0 / np.sqrt(shape.H * shape.d_v))).astype(np.float32),
+                x=rng.standard_normal((B, d_model), dtype=np.float32))

@@ -450,3 +450,76 @@ def test_gqa_oracle_against_sdpa():
 
 def test_c_oracle_thread_count_is_positive():
     assert orc.num_threads() >= 1
+
+
+# ---------------------------------------------------------------- projections around the attention
+def _tiny_layer(seed=31):
+    s = wl.HeadShape(H=4, G=2, d_v=4, d_c=6, d_r=2)
+    lw = wl.layer_weights(s, d_model=10, B=3, seed=seed)
+    rng = np.random.default_rng(seed)
+    M = (rng.standard_normal((s.H, s.d_v, s.d_c)) / 2).astype(np.float32)
+    return s, lw, M
+
+
+def test_matmul_against_library_routine():
+    rng = np.random.default_rng(30)
+    x, W = rng.standard_normal((5, 17)), rng.standard_normal((17, 9))
+    assert np.allclose(orc.matmul(x, W), x @ W, atol=1e-13)
+
+
+def test_weight_absorption_is_associativity():
+    # (x W_Q^nope) M^T == x (W_Q^nope M^T): the folded projection gives the absorbed query directly
+    s, lw, M = _tiny_layer()
+    x = lw["x"].astype(np.float64)
+    W_abs = orc.fold_maps(lw["W_q_nope"], M)
+    for h in range(s.H):
+        q_nope = x @ lw["W_q_nope"][:, h, :].astype(np.float64)               # Algorithm 1: q = x W_Q
+        two_step = q_nope @ M[h].astype(np.float64).T                           # then q~ = q^nope M_h^T
+        assert np.allclose(x @ W_abs[:, h, :], two_step, atol=1e-13)
+    ref = np.einsum("mhj,hij->mhi", lw["W_q_nope"].astype(np.float64), M.astype(np.float64))
+    assert np.allclose(W_abs, ref, atol=1e-14)
+
+
+def test_packed_projection_layout():
+    s, lw, M = _tiny_layer()
+    W_in = orc.pack_input_weights(lw["W_q_nope"], lw["W_q_rope"], lw["W_v"], lw["W_r"], M)
+    assert W_in.shape == (10, s.H * (s.d_v + s.d_r) + s.G * s.d_v + s.d_r)
+    q_t, q_r, v, kr = orc.project_in(lw["x"], W_in, s.H, s.G, s.d_v, s.d_r)
+    x = lw["x"].astype(np.float64)
+    assert np.allclose(q_r, np.einsum("bm,mhr->bhr", x, lw["W_q_rope"].astype(np.float64)), atol=1e-13)
+    assert np.allclose(v, np.einsum("bm,mgd->bgd", x, lw["W_v"].astype(np.float64)), atol=1e-13)
+    assert np.allclose(kr, x @ lw["W_r"].astype(np.float64), atol=1e-13)
+    assert np.allclose(q_t, np.einsum("bm,mhj,hij->bhi", x, lw["W_q_nope"].astype(np.float64), M.astype(np.float64)),
+                       atol=1e-13)
+
+
+def test_layer_step_against_algorithm_line_by_line():
+    # the oracle's layer step (folded weights, absorbed scores, paged cache) against the naive path that follows
+    # Algorithm 1 from the hidden state with explicit keys K = V M, for each sequence separately
+    s, lw, M = _tiny_layer()
+    T = [3, 0, 5]                                        # tokens already cached per sequence
+    case = wl.make_case("layer", s, [t + 1 for t in T], page_size=2, cache_dtype="f32", paged=True, seed=32,
+                        q_pos=T, append_pos=T)
+    V0 = wl.pool_to_f64(case.v_pool).tolist(); K0 = wl.pool_to_f64(case.kr_pool).tolist()
+    Vt, Kt = naive.gather_tokens(V0, K0, case.block_table.tolist(), T, 2, case.max_pages_per_seq)
+    W_in = orc.pack_input_weights(lw["W_q_nope"], lw["W_q_rope"], lw["W_v"], lw["W_r"], M)
+    y, out, _ = orc.layer_step(lw["x"], W_in, lw["W_o"], case.v_pool, case.kr_pool, case.block_table, T,
+                               [t + 1 for t in T], s.H, s.G, s.d_c)
+    W_Q = np.concatenate([lw["W_q_rope"], lw["W_q_nope"]], axis=2).astype(np.float64).tolist()   # [m][h][rope | nope]
+    for b in range(3):
+        V_cache = [[Vt[b][t][g] for t in range(T[b])] for g in range(s.G)]
+        KR_cache = [Kt[b][t] for t in range(T[b])]
+        y_ref, outs = naive.layer_decode_step(lw["x"][b].astype(np.float64).tolist(), W_Q,
+                                              lw["W_v"].astype(np.float64).tolist(), lw["W_r"].astype(np.float64).tolist(),
+                                              lw["W_o"].astype(np.float64).tolist(), M.astype(np.float64).tolist(), T[b],
+                                              V_cache, KR_cache, s.H, s.G, s.d_c, s.d_r)
+        # the cache is f32 in this case: the appended row is rounded to f32 before it is attended
+        assert np.allclose(out[b], np.array(outs), atol=1e-6)
+        assert np.allclose(y[b], np.array(y_ref), atol=1e-6)
+
+
+def test_bf16_round_matches_library_cast():
+    rng = np.random.default_rng(33)
+    a = rng.standard_normal(300).astype(np.float32)
+    ref = torch.from_numpy(a).bfloat16().view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(orc.bf16_round(a), ref)
