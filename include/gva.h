@@ -215,6 +215,37 @@ int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, 
                          size_t scratch_bytes, int B, int max_seq_len, int num_splits, int32_t *dev_status,
                          void *stream);
 
+/* ---- The projections around the attention (Algorithm 1: q_t = x_t W_Q, v_t = x_t W_V, k^rope_t = (x_t W_r) R_t^T;
+ * then "the usual concatenation and output projection"), with the maps folded into the query projection:
+ * because M_h is fixed at inference, q~_h = (x W_Q^{nope,h}) M_h^T = x (W_Q^{nope,h} M_h^T)  (Eq. absorb), so
+ * one product with a packed weight matrix yields the absorbed queries directly and gva_absorb_query drops out.
+ *
+ * Packed input projection W_in: bf16 [d_model][N_in], N_in = gva_input_width() = H*(d_v+d_r) + G*d_v + d_r,
+ * columns per head h: d_v folded content columns (W_Q^{nope,h} M_h^T), then d_r positional-query columns;
+ * then the G*d_v value columns; then the d_r positional-key columns.  d_model must be a multiple of 16. */
+int gva_input_width(const gva_handle *h);
+
+/* [host] Offline packing of one layer's input projection: folds the maps in fp64 and rounds every entry once to
+ * bf16.  W_q_nope [d_model][H][d_c], W_q_rope [d_model][H][d_r], W_v [d_model][G][d_v], W_r [d_model][d_r],
+ * M [H][d_v][d_c] f32 (host); W_in [d_model][N_in] bf16 bit patterns (host, caller uploads it). */
+int gva_pack_input_weights(const gva_handle *h, const float *W_q_nope, const float *W_q_rope, const float *W_v,
+                           const float *W_r, const float *M, int d_model, uint16_t *W_in);
+/* [host] f32 -> bf16 bit patterns, nearest even (for the output projection W_o). */
+int gva_pack_bf16(const float *src, uint16_t *dst, size_t n);
+
+/* x [B][d_model] f32 -> q_abs [B][H][d_v+d_r] f32 (positional slice rotated at pos[b]) and the cache append of the
+ * new token at pos[b] (value rows rounded to the cache dtype from the f32 product, k^rope rotated in fp64), in one
+ * kernel.  Same device-side error rules as gva_append_cache. */
+int gva_project_in(gva_handle *h, const gva_cache *cache, const float *x, const void *W_in, int d_model,
+                   const int32_t *pos, float *q_abs, int B, int32_t *dev_status, void *stream);
+/* attn [B][H*d_v] f32 (heads concatenated, as gva_decode writes them) x W_o bf16 [H*d_v][d_model] -> y [B][d_model] f32. */
+int gva_project_out(gva_handle *h, const float *attn, const void *W_o, int d_model, float *y, int B, void *stream);
+/* A whole layer's decode step from the hidden state: gva_project_in -> gva_decode -> gva_project_out. */
+int gva_layer_step(gva_handle *h, const gva_cache *cache, const float *x, const void *W_in, const void *W_o,
+                   int d_model, const int32_t *pos, const int32_t *seq_lens, float *q_abs, float *attn, float *y,
+                   void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
+                   int32_t *dev_status, void *stream);
+
 /* Geometry of the most recent gva_decode / gqa_decode launch on this handle (reporting only):
  * number of split-KV partitions launched (thread blocks of the decode kernel). */
 int gva_last_num_splits(const gva_handle *h);

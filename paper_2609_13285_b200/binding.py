@@ -22,7 +22,8 @@ GVA_F32, GVA_BF16 = 0, 1
 GVA_KERNEL_AUTO, GVA_KERNEL_FMA, GVA_KERNEL_MMA = 0, 1, 2
 
 EXPORTS = ["gva_create", "gva_destroy", "gva_decode_workspace_bytes", "gva_absorb_query", "gva_append_cache",
-           "gva_decode", "gva_decode_static", "gqa_decode", "gva_decode_step", "gva_step_scratch_bytes", "gva_decode_step_host", "gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens",
+           "gva_decode", "gva_decode_static", "gqa_decode", "gva_decode_step", "gva_step_scratch_bytes", "gva_decode_step_host", "gva_input_width", "gva_pack_input_weights", "gva_pack_bf16",
+           "gva_project_in", "gva_project_out", "gva_layer_step", "gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens",
            "gva_status_string"]
 
 
@@ -76,12 +77,19 @@ def load() -> ctypes.CDLL:
     lib.gva_decode.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, vp, sz, ip, ip, ip, vp, vp]
     lib.gva_decode_static.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, ip, ip, ip, vp, vp]
     lib.gqa_decode.argtypes = [vp, ctypes.POINTER(GqaCache), vp, vp, vp, vp, vp, sz, ip, ip, ip, vp, vp]
+    lib.gva_input_width.argtypes = [vp]
+    lib.gva_pack_input_weights.argtypes = [vp, vp, vp, vp, vp, vp, ip, vp]
+    lib.gva_pack_bf16.argtypes = [vp, vp, sz]
+    lib.gva_project_in.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, ip, vp, vp, ip, vp, vp]
+    lib.gva_project_out.argtypes = [vp, vp, vp, ip, vp, ip, vp]
+    lib.gva_layer_step.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, ip, vp, vp, vp, vp, vp, vp, sz, ip, ip, ip,
+                                   vp, vp]
     for name in ("gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens"):
         getattr(lib, name).argtypes = [vp]
     lib.gva_status_string.argtypes = [ip]
     lib.gva_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("gva_decode_workspace_bytes", "gva_step_scratch_bytes", "gva_status_string"):
+        if name not in ("gva_decode_workspace_bytes", "gva_step_scratch_bytes", "gva_status_string", "gva_pack_bf16"):
             getattr(lib, name).restype = ip
     _lib = lib
     return lib
@@ -205,6 +213,59 @@ def gva_decode_step_host(handle: int, cache: GvaCache, M, q_c_host, q_r_host, v_
                                      int(max_seq_len), int(num_splits), _ptr(dev_status), _stream())
     if check:
         _check(rc, "gva_decode_step_host")
+    return rc
+
+
+def gva_input_width(handle: int) -> int:
+    return int(load().gva_input_width(handle))
+
+
+def _np_ptr(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def gva_pack_input_weights(handle: int, W_q_nope, W_q_rope, W_v, W_r, M, d_model: int):
+    """Host-side offline packing (numpy float32 in, numpy uint16 bf16 bit patterns [d_model, N_in] out)."""
+    import numpy as np
+    arrs = [np.ascontiguousarray(a, dtype=np.float32) for a in (W_q_nope, W_q_rope, W_v, W_r, M)]
+    out = np.empty((d_model, gva_input_width(handle)), dtype=np.uint16)
+    _check(load().gva_pack_input_weights(handle, *[_np_ptr(a) for a in arrs], int(d_model), _np_ptr(out)),
+           "gva_pack_input_weights")
+    return out
+
+
+def gva_pack_bf16(src):
+    import numpy as np
+    src = np.ascontiguousarray(src, dtype=np.float32)
+    out = np.empty(src.shape, dtype=np.uint16)
+    _check(load().gva_pack_bf16(_np_ptr(src), _np_ptr(out), src.size), "gva_pack_bf16")
+    return out
+
+
+def gva_project_in(handle: int, cache: GvaCache, x, W_in, d_model: int, pos, q_abs, B: int, dev_status=None,
+                   check: bool = True) -> int:
+    rc = load().gva_project_in(handle, ctypes.byref(cache), _ptr(x), _ptr(W_in), int(d_model), _ptr(pos), _ptr(q_abs),
+                               int(B), _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gva_project_in")
+    return rc
+
+
+def gva_project_out(handle: int, attn, W_o, d_model: int, y, B: int, check: bool = True) -> int:
+    rc = load().gva_project_out(handle, _ptr(attn), _ptr(W_o), int(d_model), _ptr(y), int(B), _stream())
+    if check:
+        _check(rc, "gva_project_out")
+    return rc
+
+
+def gva_layer_step(handle: int, cache: GvaCache, x, W_in, W_o, d_model: int, pos, seq_lens, q_abs, attn, y, workspace,
+                   B: int, max_seq_len: int, num_splits: int = 0, dev_status=None, check: bool = True) -> int:
+    rc = load().gva_layer_step(handle, ctypes.byref(cache), _ptr(x), _ptr(W_in), _ptr(W_o), int(d_model), _ptr(pos),
+                               _ptr(seq_lens), _ptr(q_abs), _ptr(attn), _ptr(y), _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), int(B), int(max_seq_len), int(num_splits),
+                               _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gva_layer_step")
     return rc
 
 

@@ -10,6 +10,7 @@
 #include "gva_common.cuh"
 #include "gva_decode_fma.cuh"
 #include "gva_small_kernels.cuh"
+#include "gva_project.cuh"
 #ifdef GVA_WITH_MMA
 #include "gva_decode_mma.cuh"
 #endif
@@ -603,6 +604,127 @@ int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, 
     if (cudaMemcpyAsync(out_host, out, (size_t)B * c.H * c.d_v * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return GVA_ERR_CUDA;
     return GVA_OK;
+}
+
+}  // extern "C"
+
+// ---- projections around the attention -----------------------------------------------------------------
+namespace {
+// host: double -> bf16 bits, round to nearest even (via round-to-odd f32, as on the device)
+uint16_t host_bf16_from_double(double x) {
+    float f = (float)x;                                   // nearest-even
+    if ((double)f != x && std::isfinite(f)) {            // make it round-to-odd: step toward x's side, then set the sticky bit
+        uint32_t u;
+        std::memcpy(&u, &f, 4);
+        const bool over = std::fabs((double)f) > std::fabs(x);
+        if (over) u -= 1;                                 // truncate toward zero (magnitude)
+        u |= 1u;
+        std::memcpy(&f, &u, 4);
+    }
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+int input_width(const gva_config &c) { return c.H * (c.d_v + c.d_r) + c.G * c.d_v + c.d_r; }
+
+template <int MODE>
+int launch_project(const gva_handle *h, const ProjParams &p, cudaStream_t stream) {
+    if (p.M <= 0) return GVA_OK;
+    if (p.K % 16 != 0 || p.N % 8 != 0 || p.K <= 0) return GVA_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)p.K * kProjRowBytes;
+    if (smem > (size_t)h->smem_optin) return GVA_ERR_UNSUPPORTED;
+    const dim3 grid((p.N + kProjCols - 1) / kProjCols, (p.M + 16 * kProjWarps - 1) / (16 * kProjWarps));
+    const bool bf = h->cfg.cache_dtype == GVA_BF16;
+    auto fn = (MODE == 1 && !bf) ? project_kernel<MODE, float> : project_kernel<MODE, __nv_bfloat16>;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
+    if (launch_pdl(fn, grid, dim3(32 * kProjWarps), smem, stream, p, h->rope) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GVA_ERR_CUDA;
+    }
+    return GVA_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int gva_input_width(const gva_handle *h) { return h ? input_width(h->cfg) : 0; }
+
+int gva_pack_input_weights(const gva_handle *h, const float *W_q_nope, const float *W_q_rope, const float *W_v,
+                           const float *W_r, const float *M, int d_model, uint16_t *W_in) {
+    if (!h || !W_q_nope || !W_q_rope || !W_v || !W_r || !M || !W_in || d_model <= 0) return GVA_ERR_INVALID_ARG;
+    const gva_config &c = h->cfg;
+    const int dq = c.d_v + c.d_r, nq = c.H * dq, nv = c.G * c.d_v, N = input_width(c);
+    for (int m = 0; m < d_model; ++m) {
+        uint16_t *row = W_in + (size_t)m * N;
+        for (int hh = 0; hh < c.H; ++hh) {
+            const float *wq = W_q_nope + ((size_t)m * c.H + hh) * c.d_c;
+            for (int i = 0; i < c.d_v; ++i) {            // folded content columns: (W_Q^nope M_h^T)[m][i]
+                const float *mi = M + ((size_t)hh * c.d_v + i) * c.d_c;
+                double acc = 0.0;
+                for (int j = 0; j < c.d_c; ++j) acc += (double)wq[j] * (double)mi[j];
+                row[hh * dq + i] = host_bf16_from_double(acc);
+            }
+            for (int r = 0; r < c.d_r; ++r)
+                row[hh * dq + c.d_v + r] = host_bf16_from_double((double)W_q_rope[((size_t)m * c.H + hh) * c.d_r + r]);
+        }
+        for (int i = 0; i < nv; ++i) row[nq + i] = host_bf16_from_double((double)W_v[(size_t)m * nv + i]);
+        for (int r = 0; r < c.d_r; ++r) row[nq + nv + r] = host_bf16_from_double((double)W_r[(size_t)m * c.d_r + r]);
+    }
+    return GVA_OK;
+}
+
+int gva_pack_bf16(const float *src, uint16_t *dst, size_t n) {
+    if (!src || !dst) return GVA_ERR_INVALID_ARG;
+    for (size_t i = 0; i < n; ++i) dst[i] = host_bf16_from_double((double)src[i]);
+    return GVA_OK;
+}
+
+int gva_project_in(gva_handle *h, const gva_cache *cache, const float *x, const void *W_in, int d_model,
+                   const int32_t *pos, float *q_abs, int B, int32_t *dev_status, void *stream) {
+    if (!h || !cache || B < 0 || d_model <= 0) return GVA_ERR_INVALID_ARG;
+    if (B == 0) return GVA_OK;
+    if (!x || !W_in || !pos || !q_abs || !cache->v_pool || !cache->kr_pool) return GVA_ERR_INVALID_ARG;
+    if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
+    if (!aligned(x, 8) || !aligned(W_in, 16) || !aligned(q_abs, 8) || !aligned(cache->v_pool, 16) ||
+        !aligned(cache->kr_pool, 16))
+        return GVA_ERR_INVALID_ARG;
+    const gva_config &c = h->cfg;
+    ProjParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.A = x; p.W = static_cast<const uint16_t *>(W_in);
+    p.M = B; p.K = d_model; p.N = input_width(c);
+    p.q_abs = q_abs; p.v_pool = cache->v_pool; p.kr_pool = cache->kr_pool;
+    p.block_table = cache->block_table; p.pos = pos; p.dev_status = dev_status;
+    p.H = c.H; p.G = c.G; p.d_v = c.d_v; p.d_r = c.d_r; p.P = c.page_size;
+    p.num_pages = cache->num_pages; p.max_pages = cache->max_pages_per_seq;
+    return launch_project<1>(h, p, static_cast<cudaStream_t>(stream));
+}
+
+int gva_project_out(gva_handle *h, const float *attn, const void *W_o, int d_model, float *y, int B, void *stream) {
+    if (!h || B < 0 || d_model <= 0) return GVA_ERR_INVALID_ARG;
+    if (B == 0) return GVA_OK;
+    if (!attn || !W_o || !y) return GVA_ERR_INVALID_ARG;
+    if (!aligned(attn, 8) || !aligned(W_o, 16) || !aligned(y, 8)) return GVA_ERR_INVALID_ARG;
+    ProjParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.A = attn; p.W = static_cast<const uint16_t *>(W_o);
+    p.M = B; p.K = h->cfg.H * h->cfg.d_v; p.N = d_model;
+    p.Y = y;
+    return launch_project<0>(h, p, static_cast<cudaStream_t>(stream));
+}
+
+int gva_layer_step(gva_handle *h, const gva_cache *cache, const float *x, const void *W_in, const void *W_o, int d_model,
+                   const int32_t *pos, const int32_t *seq_lens, float *q_abs, float *attn, float *y, void *workspace,
+                   size_t workspace_bytes, int B, int max_seq_len, int num_splits, int32_t *dev_status, void *stream) {
+    int rc = gva_project_in(h, cache, x, W_in, d_model, pos, q_abs, B, dev_status, stream);
+    if (rc != GVA_OK) return rc;
+    rc = gva_decode(h, cache, q_abs, seq_lens, attn, nullptr, workspace, workspace_bytes, B, max_seq_len, num_splits,
+                    dev_status, stream);
+    if (rc != GVA_OK) return rc;
+    return gva_project_out(h, attn, W_o, d_model, y, B, stream);
 }
 
 int gva_last_num_splits(const gva_handle *h) { return h ? h->last_num_splits : 0; }
