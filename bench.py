@@ -393,6 +393,57 @@ def measure_gqa(rank, local_rank, dist, args, kernel, torch, gb, harness):
     return res
 
 
+def measure_layer(rank, local_rank, dist, args, kernel, torch, gb, harness):
+    """A whole layer's decode step from the hidden state on the headline shapes (d_model = 1024): input projection
+    with the maps folded in + fused append, gva_decode, output projection (gva_layer_step: 4 launches)."""
+    from paper_2609_13285_b200 import multirank, workloads as wl
+    dev = torch.device("cuda", local_rank)
+    case = make_workload("cfg2", rank)
+    pos_np = (case.seq_lens - 1).astype(np.int32)
+    case.q_pos[:] = pos_np
+    case.append_pos[:] = pos_np
+    d_model = 1024
+    lw = wl.layer_weights(case.shape, d_model, case.B, seed=wl.MASTER_SEED + 6000 + 7919 * rank)
+    dc = harness.upload(case, device=dev, kernel=kernel)
+    s, B = case.shape, case.B
+    W_in = torch.from_numpy(gb.gva_pack_input_weights(dc.handle, lw["W_q_nope"], lw["W_q_rope"], lw["W_v"], lw["W_r"],
+                                                      case.M, d_model).view(np.int16)).to(dev)
+    W_o = torch.from_numpy(gb.gva_pack_bf16(lw["W_o"]).view(np.int16)).to(dev)
+    x = torch.from_numpy(lw["x"]).to(dev)
+    attn = torch.empty((B, s.H, s.d_v), dtype=torch.float32, device=dev)
+    y = torch.empty((B, d_model), dtype=torch.float32, device=dev)
+    pools = [(dc.v_pool, dc.kr_pool), (dc.v_pool.clone(), dc.kr_pool.clone())]
+    caches = [gb.make_cache(v, k, dc.block_table, case.num_pages, case.max_pages_per_seq) for v, k in pools]
+    max_len = int(case.seq_lens.max())
+    ws = dc.ensure_workspace(0)
+    stream = torch.cuda.current_stream()
+    steps, warmup = max(20, args.steps // 3), 10
+
+    def call(i):
+        gb.gva_layer_step(dc.handle, caches[i & 1], x, W_in, W_o, d_model, dc.append_pos, dc.seq_lens, dc.q_abs, attn, y,
+                          ws, B, max_len, 0, dc.status)
+
+    for i in range(warmup):
+        call(i)
+    multirank.barrier(dist)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for i in range(steps):
+        call(i)
+    b.record(stream)
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    res = {"workload": "cfg2 shapes from the hidden state: x[32,1024] -> packed input projection (bf16, maps folded in) "
+                       "+ append, gva_decode, output projection",
+           "ms_per_step": ms, "cache_read_GBps": case.cache_bytes() / (ms * 1e-3) / 1e9,
+           "weight_bytes": int(W_in.numel() * 2 + W_o.numel() * 2), "steps": steps, "device_status": int(dc.status.item())}
+    dc.close()
+    del pools, caches
+    torch.cuda.empty_cache()
+    return res
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -457,6 +508,7 @@ def main() -> None:
         gq["gva_over_gqa_cache_bytes"] = r["cache_bytes"] / gq["cache_bytes_per_call"]      # 0.53125 = 1/2 + 16/(2*4*64)
         gq["gva_over_gqa_decode_time"] = decode_ms / gq["gqa_decode_ms_per_call"]
         others["gqa_matched_cfg2"] = gq
+        others["layer_step_cfg2"] = measure_layer(rank, local_rank, dist, short, kernel, torch, gb, harness)
 
     if rank == 0:
         case = r["case"]

@@ -631,12 +631,23 @@ uint16_t host_bf16_from_double(double x) {
 int input_width(const gva_config &c) { return c.H * (c.d_v + c.d_r) + c.G * c.d_v + c.d_r; }
 
 template <int MODE>
-int launch_project(const gva_handle *h, const ProjParams &p, cudaStream_t stream) {
+int launch_project(const gva_handle *h, ProjParams p, cudaStream_t stream) {
     if (p.M <= 0) return GVA_OK;
     if (p.K % 16 != 0 || p.N % 8 != 0 || p.K <= 0) return GVA_ERR_UNSUPPORTED;
-    const size_t smem = (size_t)p.K * kProjRowBytes;
+    // warps of a block: m-tiles first, the rest split K (as far as K allows)
+    int m_tiles = (p.M + 15) / 16;
+    if (m_tiles > kProjWarps) m_tiles = kProjWarps;
+    int mt_pow2 = 1;
+    while (mt_pow2 < m_tiles) mt_pow2 *= 2;
+    p.m_tiles = mt_pow2;
+    p.k_slices = kProjWarps / mt_pow2;
+    while (p.k_slices > 1 && p.K % (16 * p.k_slices) != 0) p.k_slices /= 2;
+    if (p.k_slices * p.m_tiles != kProjWarps) {     // K too ragged to split that far: fewer slices, idle warps
+        p.m_tiles = kProjWarps / p.k_slices;
+    }
+    const size_t smem = (size_t)p.K * kProjRowBytes + (size_t)kProjWarps * 32 * 8 * sizeof(float);
     if (smem > (size_t)h->smem_optin) return GVA_ERR_UNSUPPORTED;
-    const dim3 grid((p.N + kProjCols - 1) / kProjCols, (p.M + 16 * kProjWarps - 1) / (16 * kProjWarps));
+    const dim3 grid((p.N + kProjCols - 1) / kProjCols, (p.M + 16 * p.m_tiles - 1) / (16 * p.m_tiles));
     const bool bf = h->cfg.cache_dtype == GVA_BF16;
     auto fn = (MODE == 1 && !bf) ? project_kernel<MODE, float> : project_kernel<MODE, __nv_bfloat16>;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;

@@ -6,7 +6,9 @@
 // Both are skinny GEMMs  C[M x N] = A[M x K] W[K x N]  with M = batch (tens to hundreds of rows), bf16 weights
 // and f32 activations.  One block owns 16 output columns over the whole K: its 16-column slab of W is staged
 // once in shared memory with cp.async (48-byte rows: conflict-free for ldmatrix without a swizzle); each warp
-// owns a 16-row m-tile, reads its activations straight from global memory in mma A-fragment order, splits every
+// owns a 16-row m-tile and a slice of K (small batches leave most of a block's eight warps without an m-tile
+// of their own, so they split K instead and their partial sums meet in shared memory), reads its activations
+// straight from global memory in mma A-fragment order, splits every
 // f32 activation into three bf16 terms (hi + mid + lo carry all 24 significant bits, so only the weights'
 // own bf16 storage limits accuracy) and issues three m16n8k16 MMAs per fragment with f32 accumulation.
 // The input projection's epilogue writes the absorbed queries (rotating the positional slice in fp64) and
@@ -46,6 +48,7 @@ struct ProjParams {
     const float *A;              // [M][K] activations
     const uint16_t *W;           // [K][N] bf16 weights
     int M, K, N;
+    int m_tiles, k_slices;       // per block: m_tiles * k_slices == kProjWarps, K % (16 * k_slices) == 0
     // plain epilogue
     float *Y;                    // [M][N]
     // input-projection epilogue
@@ -64,7 +67,10 @@ project_kernel(ProjParams p, RopeTable rope) {
     extern __shared__ __align__(16) unsigned char slab[];      // [K][48 bytes]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n0 = blockIdx.x * kProjCols;
-    const int m0 = (blockIdx.y * kProjWarps + warp) * 16;
+    const int mt = warp % p.m_tiles, ks = warp / p.m_tiles;
+    const int m0 = (blockIdx.y * p.m_tiles + mt) * 16;
+    const int k_len = p.K / p.k_slices, k_begin = ks * k_len;
+    float *s_red = reinterpret_cast<float *>(slab + (size_t)p.K * kProjRowBytes);      // [kProjWarps][32][8] partial sums
     grid_dependency_wait();
     // stage this block's 16 columns of W: two 16-byte chunks per k-row
     {
@@ -92,8 +98,8 @@ project_kernel(ProjParams p, RopeTable rope) {
     if (warp_live) {
         // ldmatrix.trans lane addressing: matrices (k0-7, n0-7) (k8-15, n0-7) (k0-7, n8-15) (k8-15, n8-15)
         const uint32_t b_base = smem_u32(slab) + ((lane & 7) + ((lane >> 3) & 1) * 8) * kProjRowBytes + (lane >> 4) * 16;
-#pragma unroll 4
-        for (int k0 = 0; k0 < p.K; k0 += 16) {
+#pragma unroll 8
+        for (int k0 = k_begin; k0 < k_begin + k_len; k0 += 16) {
             const float2 f0 = *reinterpret_cast<const float2 *>(a_lo + k0);
             const float2 f1 = *reinterpret_cast<const float2 *>(a_hi + k0);
             const float2 f2 = *reinterpret_cast<const float2 *>(a_lo + k0 + 8);
@@ -110,6 +116,22 @@ project_kernel(ProjParams p, RopeTable rope) {
                 mma_bf16_p(acc[t], am, b[2 * t], b[2 * t + 1]);
                 mma_bf16_p(acc[t], ah, b[2 * t], b[2 * t + 1]);
             }
+        }
+    }
+    if (p.k_slices > 1) {       // block-uniform: the K slices of an m-tile are summed in slice order by slice 0
+        float *mine = s_red + ((size_t)warp * 32 + lane) * 8;
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) mine[t * 4 + e] = acc[t][e];
+        __syncthreads();
+        if (ks != 0) return;
+        for (int s2 = 1; s2 < p.k_slices; ++s2) {
+            const float *other = s_red + ((size_t)(s2 * p.m_tiles + mt) * 32 + lane) * 8;
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[t][e] += other[t * 4 + e];
         }
     }
     if (!warp_live) return;
