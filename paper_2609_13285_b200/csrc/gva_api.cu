@@ -229,6 +229,9 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     int wph = h->cfg.d_v == 64 ? 4 : 1;
     while (wph < 32 && wph * 8 < n_est) wph *= 2;
     if (h->cfg.d_v == 128 && wph <= 2) wph = 1;
+    // ... but no more than ~4096 warps in the whole grid: beyond that the merge blocks no longer fit beside the decode
+    // blocks and start in waves after them (measured on B = 128: 2 warps per head 94 us, 4 warps 99 us, 8 warps 107 us)
+    while (wph > 1 && (long long)B * h->cfg.H * wph > 4096) wph /= 2;
     const int hpb = wph >= 4 ? 1 : 4 / wph;
     const size_t csmem = (size_t)wph * hpb * (h->cfg.d_v + 2) * sizeof(float);
     const dim3 cgrid(B, (h->cfg.H + hpb - 1) / hpb), cblock(32 * wph * hpb);
