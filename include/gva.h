@@ -222,7 +222,7 @@ int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, 
  *
  * Packed input projection W_in: bf16 [d_model][N_in], N_in = gva_input_width() = H*(d_v+d_r) + G*d_v + d_r,
  * columns per head h: d_v folded content columns (W_Q^{nope,h} M_h^T), then d_r positional-query columns;
- * then the G*d_v value columns; then the d_r positional-key columns.  d_model must be a multiple of 16. */
+ * then the G*d_v value columns; then the d_r positional-key columns.  d_model must be a multiple of 128. */
 int gva_input_width(const gva_handle *h);
 
 /* [host] Offline packing of one layer's input projection: folds the maps in fp64 and rounds every entry once to

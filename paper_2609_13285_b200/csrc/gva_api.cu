@@ -636,25 +636,35 @@ int input_width(const gva_config &c) { return c.H * (c.d_v + c.d_r) + c.G * c.d_
 template <int MODE>
 int launch_project(const gva_handle *h, ProjParams p, cudaStream_t stream) {
     if (p.M <= 0) return GVA_OK;
-    if (p.K % 16 != 0 || p.N % 8 != 0 || p.K <= 0) return GVA_ERR_UNSUPPORTED;
-    // warps of a block: m-tiles first, the rest split K (as far as K allows)
-    int m_tiles = (p.M + 15) / 16;
-    if (m_tiles > kProjWarps) m_tiles = kProjWarps;
-    int mt_pow2 = 1;
-    while (mt_pow2 < m_tiles) mt_pow2 *= 2;
-    p.m_tiles = mt_pow2;
-    p.k_slices = kProjWarps / mt_pow2;
-    while (p.k_slices > 1 && p.K % (16 * p.k_slices) != 0) p.k_slices /= 2;
-    if (p.k_slices * p.m_tiles != kProjWarps) {     // K too ragged to split that far: fewer slices, idle warps
-        p.m_tiles = kProjWarps / p.k_slices;
-    }
-    const size_t smem = (size_t)p.K * kProjRowBytes + (size_t)kProjWarps * 32 * 8 * sizeof(float);
+    if (p.K <= 0 || p.K % (16 * kProjSlices) != 0 || p.N % 8 != 0) return GVA_ERR_UNSUPPORTED;
+    int m_tiles = (std::min(p.M, kProjRows) + 15) / 16, mt = 1;
+    while (mt < m_tiles) mt *= 2;
+    const size_t smem = (size_t)kProjChunk * kProjRowBytes + (size_t)16 * mt * kProjALd * sizeof(float);
     if (smem > (size_t)h->smem_optin) return GVA_ERR_UNSUPPORTED;
-    const dim3 grid((p.N + kProjCols - 1) / kProjCols, (p.M + 16 * p.m_tiles - 1) / (16 * p.m_tiles));
-    const bool bf = h->cfg.cache_dtype == GVA_BF16;
-    auto fn = (MODE == 1 && !bf) ? project_kernel<MODE, float> : project_kernel<MODE, __nv_bfloat16>;
+    const bool f32 = MODE == 1 && h->cfg.cache_dtype != GVA_BF16;
+    void (*fn)(ProjParams, RopeTable) = nullptr;
+    switch (mt) {
+        case 1: fn = f32 ? project_kernel<MODE, float, 1> : project_kernel<MODE, __nv_bfloat16, 1>; break;
+        case 2: fn = f32 ? project_kernel<MODE, float, 2> : project_kernel<MODE, __nv_bfloat16, 2>; break;
+        case 4: fn = f32 ? project_kernel<MODE, float, 4> : project_kernel<MODE, __nv_bfloat16, 4>; break;
+        default: fn = f32 ? project_kernel<MODE, float, 8> : project_kernel<MODE, __nv_bfloat16, 8>; break;
+    }
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
-    if (launch_pdl(fn, grid, dim3(32 * kProjWarps), smem, stream, p, h->rope) != cudaSuccess) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((p.N + kProjStrip - 1) / kProjStrip, kProjSlices, (p.M + kProjRows - 1) / kProjRows);
+    cfg.blockDim = dim3(32 * kProjWarps);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = kProjSlices;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    if (cudaLaunchKernelEx(&cfg, fn, p, h->rope) != cudaSuccess) {
         (void)cudaGetLastError();
         return GVA_ERR_CUDA;
     }
@@ -702,7 +712,7 @@ int gva_project_in(gva_handle *h, const gva_cache *cache, const float *x, const 
     if (B == 0) return GVA_OK;
     if (!x || !W_in || !pos || !q_abs || !cache->v_pool || !cache->kr_pool) return GVA_ERR_INVALID_ARG;
     if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
-    if (!aligned(x, 8) || !aligned(W_in, 16) || !aligned(q_abs, 8) || !aligned(cache->v_pool, 16) ||
+    if (!aligned(x, 16) || !aligned(W_in, 16) || !aligned(q_abs, 8) || !aligned(cache->v_pool, 16) ||
         !aligned(cache->kr_pool, 16))
         return GVA_ERR_INVALID_ARG;
     const gva_config &c = h->cfg;
@@ -721,7 +731,7 @@ int gva_project_out(gva_handle *h, const float *attn, const void *W_o, int d_mod
     if (!h || B < 0 || d_model <= 0) return GVA_ERR_INVALID_ARG;
     if (B == 0) return GVA_OK;
     if (!attn || !W_o || !y) return GVA_ERR_INVALID_ARG;
-    if (!aligned(attn, 8) || !aligned(W_o, 16) || !aligned(y, 8)) return GVA_ERR_INVALID_ARG;
+    if (!aligned(attn, 16) || !aligned(W_o, 16) || !aligned(y, 8)) return GVA_ERR_INVALID_ARG;
     ProjParams p;
     std::memset(&p, 0, sizeof(p));
     p.A = attn; p.W = static_cast<const uint16_t *>(W_o);

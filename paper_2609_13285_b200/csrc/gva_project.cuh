@@ -4,30 +4,37 @@
 // applied to the projection), so no separate absorb step remains.
 //
 // Both are skinny GEMMs  C[M x N] = A[M x K] W[K x N]  with M = batch (tens to hundreds of rows), bf16 weights
-// and f32 activations.  One block owns 16 output columns over the whole K: its 16-column slab of W is staged
-// once in shared memory with cp.async (48-byte rows: conflict-free for ldmatrix without a swizzle); each warp
-// owns a 16-row m-tile and a slice of K (small batches leave most of a block's eight warps without an m-tile
-// of their own, so they split K instead and their partial sums meet in shared memory), reads its activations
-// straight from global memory in mma A-fragment order, splits every
-// f32 activation into three bf16 terms (hi + mid + lo carry all 24 significant bits, so only the weights'
-// own bf16 storage limits accuracy) and issues three m16n8k16 MMAs per fragment with f32 accumulation.
-// The input projection's epilogue writes the absorbed queries (rotating the positional slice in fp64) and
-// appends the new value rows and the rotated positional key to the paged cache.
+// and f32 activations: too few rows to fill the machine by output tiles alone, so K is split eight ways across
+// a thread-block cluster.  Block (n, r) of a cluster computes the partial product of a 64-column strip over
+// K-slice r: its slice of W (K/8 rows of 128 contiguous bytes) is staged with cp.async into 144-byte rows
+// (conflict-free for ldmatrix without a swizzle); each warp owns a 16-row m-tile and some of the strip's eight
+// n-tiles, reads its activations straight from global memory in mma A-fragment order, splits every f32
+// activation into three bf16 terms (hi + mid + lo carry all 24 significant bits, so only the weights' own bf16
+// storage limits accuracy) and issues three m16n8k16 MMAs per fragment with f32 accumulation.  The partial
+// strips meet through distributed shared memory: after a cluster barrier block r sums columns [8r, 8r + 8) of
+// all eight partials in rank order (deterministic) and runs the epilogue for them.  The input projection's
+// epilogue writes the absorbed queries (rotating the positional slice in fp64) and appends the new value rows
+// and the rotated positional key to the paged cache.
 #pragma once
+
+#include <cooperative_groups.h>
 
 #include "gva_common.cuh"
 #include "gva_small_kernels.cuh"
 
 namespace gva {
 
-constexpr int kProjCols = 16;             // output columns per block
-constexpr int kProjRowBytes = 48;         // shared-memory stride of one k-row of the slab (32 bytes used)
-constexpr int kProjWarps = 8;             // m-tiles per block: 128 rows
+namespace cg = cooperative_groups;
 
-__device__ __forceinline__ void ldsm_x4_trans_p(uint32_t addr, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
+constexpr int kProjStrip = 64;            // output columns per cluster
+constexpr int kProjSlices = 8;            // K slices = blocks per cluster
+constexpr int kProjRowBytes = 144;        // shared-memory stride of one k-row of the W slice (128 bytes used)
+constexpr int kProjWarps = 8;             // 256 threads
+constexpr int kProjRows = 128;            // rows (sequences) per block
+constexpr int kProjLd = kProjStrip + 4;   // f32 row stride of the partial strip in shared memory
+
+__device__ __forceinline__ void ldsm_x2_trans_p(uint32_t addr, uint32_t (&r)[2]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];\n" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
 }
 __device__ __forceinline__ void mma_bf16_p(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -48,7 +55,6 @@ struct ProjParams {
     const float *A;              // [M][K] activations
     const uint16_t *W;           // [K][N] bf16 weights
     int M, K, N;
-    int m_tiles, k_slices;       // per block: m_tiles * k_slices == kProjWarps, K % (16 * k_slices) == 0
     // plain epilogue
     float *Y;                    // [M][N]
     // input-projection epilogue
@@ -59,156 +65,185 @@ struct ProjParams {
     int H, G, d_v, d_r, P, num_pages, max_pages;
 };
 
-// MODE 0: Y = A W.   MODE 1: input projection with the fused query / rotation / append epilogue.
+// One finished pair of outputs (row, columns n and n + 1).
+// MODE 0: Y = A W.   MODE 1: input projection: absorbed query / rotated positional query / value append / rotated key append.
 template <int MODE, typename CT>
+__device__ __forceinline__ void project_epilogue(const ProjParams &p, const RopeTable &rope, int row, int n, float c0, float c1,
+                                                 int t_pos) {
+    if constexpr (MODE == 0) {
+        *reinterpret_cast<float2 *>(p.Y + (size_t)row * p.N + n) = make_float2(c0, c1);
+    } else {
+        const int dq = p.d_v + p.d_r, nq = p.H * dq, nv = p.G * p.d_v;
+        if (n < nq) {
+            const int h = n / dq, j = n % dq;
+            float *dst = p.q_abs + ((size_t)row * p.H + h) * dq + j;
+            if (j < p.d_v) {
+                *reinterpret_cast<float2 *>(dst) = make_float2(c0, c1);
+            } else {
+                double y0, y1;
+                rope_pair((double)c0, (double)c1, t_pos, rope.inv_freq[(j - p.d_v) >> 1], y0, y1);
+                *reinterpret_cast<float2 *>(dst) = make_float2(__double2float_rn(y0), __double2float_rn(y1));
+            }
+            return;
+        }
+        // cache slot of this sequence's new token; one thread per (row, strip) reports a bad position
+        const bool reporter = (n & (kProjStrip - 1)) == 0 || n == nq;
+        if (t_pos < 0 || t_pos / p.P >= p.max_pages) {
+            if (reporter) report_error(p.dev_status, GVA_ERR_SEQ_LEN, row);
+            return;
+        }
+        const long long page = p.block_table ? (long long)p.block_table[(size_t)row * p.max_pages + t_pos / p.P]
+                                             : (long long)row * p.max_pages + t_pos / p.P;
+        if (page < 0 || page >= p.num_pages) {
+            if (reporter) report_error(p.dev_status, GVA_ERR_BAD_PAGE, row);
+            return;
+        }
+        const int slot = t_pos % p.P;
+        if (n < nq + nv) {
+            const int idx = n - nq, g = idx / p.d_v, d = idx % p.d_v;
+            const size_t off = (((size_t)page * p.G + g) * p.P + slot) * p.d_v + d;
+            if constexpr (sizeof(CT) == 2) {
+                reinterpret_cast<uint32_t *>(reinterpret_cast<uint16_t *>(p.v_pool) + off)[0] =
+                    (uint32_t)float_to_bf16_bits(c0) | ((uint32_t)float_to_bf16_bits(c1) << 16);
+            } else {
+                *reinterpret_cast<float2 *>(reinterpret_cast<float *>(p.v_pool) + off) = make_float2(c0, c1);
+            }
+        } else {
+            const int i = (n - nq - nv) >> 1;
+            double y0, y1;
+            rope_pair((double)c0, (double)c1, t_pos, rope.inv_freq[i], y0, y1);
+            const size_t off = ((size_t)page * p.P + slot) * p.d_r + 2 * i;
+            if constexpr (sizeof(CT) == 2) {
+                reinterpret_cast<uint32_t *>(reinterpret_cast<uint16_t *>(p.kr_pool) + off)[0] =
+                    (uint32_t)double_to_bf16_bits(y0) | ((uint32_t)double_to_bf16_bits(y1) << 16);
+            } else {
+                *reinterpret_cast<float2 *>(reinterpret_cast<float *>(p.kr_pool) + off) =
+                    make_float2(__double2float_rn(y0), __double2float_rn(y1));
+            }
+        }
+    }
+}
+
+// grid (ceil(N / 64), 8, ceil(M / 128)), cluster (1, 8, 1), block 256.
+// MT = m-tiles per block (power of two); 8 / MT warps share an m-tile and each takes MT of the strip's 8 n-tiles.
+// The K slice is walked in chunks of 128: the chunk of W and the chunk of activations are both staged with
+// cp.async (one memory round trip per chunk) and the k-steps run as a small rolled loop over shared memory --
+// short kernels like this one are dominated by instruction fetch when their code is large, because the cache
+// stream between two calls pushes it out of L2.
+constexpr int kProjChunk = 128;                       // k per staged chunk
+constexpr int kProjALd = kProjChunk + 8;              // f32 row stride of the staged activations (conflict-free float2 reads)
+
+template <int MODE, typename CT, int MT>
 __global__ void __launch_bounds__(32 * kProjWarps)
 project_kernel(ProjParams p, RopeTable rope) {
     grid_dependency_launch();
-    extern __shared__ __align__(16) unsigned char slab[];      // [K][48 bytes]
+    cg::cluster_group cluster = cg::this_cluster();
+    extern __shared__ __align__(16) unsigned char psm[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n0 = blockIdx.x * kProjCols;
-    const int mt = warp % p.m_tiles, ks = warp / p.m_tiles;
-    const int m0 = (blockIdx.y * p.m_tiles + mt) * 16;
-    const int k_len = p.K / p.k_slices, k_begin = ks * k_len;
-    float *s_red = reinterpret_cast<float *>(slab + (size_t)p.K * kProjRowBytes);      // [kProjWarps][32][8] partial sums
+    const int k_len = p.K / kProjSlices;
+    unsigned char *w_s = psm;                                                        // [kProjChunk][144 bytes]
+    float *a_s = reinterpret_cast<float *>(psm + (size_t)kProjChunk * kProjRowBytes);  // [16 MT][kProjALd]
+    float *part = a_s;                                                               // [16 MT][kProjLd], after the last chunk
+    const int n0 = blockIdx.x * kProjStrip;
+    const int rank = blockIdx.y;                  // == cluster rank: the cluster spans y
+    const int k_begin = rank * k_len;
+    const int row0 = blockIdx.z * kProjRows;
+    const int rows = min(kProjRows, p.M - row0);
+    const int mt = warp % MT, ng = warp / MT;
+    const int m0 = mt * 16;
     grid_dependency_wait();
-    // stage this block's 16 columns of W: two 16-byte chunks per k-row
-    {
-        const uint32_t s_u32 = smem_u32(slab);
-        const unsigned char *src = reinterpret_cast<const unsigned char *>(p.W);
-        for (int c = tid; c < p.K * 2; c += 32 * kProjWarps) {
-            const int k = c >> 1, half = c & 1;
-            const bool in = n0 + half * 8 < p.N;       // N is a multiple of 8; a block may hang over the last 8 columns
-            cp_async16(s_u32 + k * kProjRowBytes + half * 16, src + (in ? ((size_t)k * p.N + n0) * 2 + half * 16 : 0),
-                       in ? 16 : 0);
-        }
-        cp_async_commit();
-    }
-    const bool warp_live = m0 < p.M;
-    const int r_lo = min(m0 + (lane >> 2), p.M - 1), r_hi = min(m0 + (lane >> 2) + 8, p.M - 1);
-    const float *a_lo = p.A + (size_t)r_lo * p.K + 2 * (lane & 3);
-    const float *a_hi = p.A + (size_t)r_hi * p.K + 2 * (lane & 3);
-    float acc[2][4];
+    // the epilogue's position lookups travel with the first chunk
+    int ep_pos[2] = {0, 0};
+    if constexpr (MODE == 1) {
 #pragma unroll
-    for (int t = 0; t < 2; ++t)
+        for (int u = 0; u < 2; ++u) {
+            const int item = tid + u * 32 * kProjWarps;
+            if (item < rows * 4) ep_pos[u] = p.pos[row0 + (item >> 2)];
+        }
+    }
+    float acc[MT][4];
+#pragma unroll
+    for (int t = 0; t < MT; ++t)
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[t][e] = 0.f;
-    cp_async_wait<0>();
-    __syncthreads();
-    if (warp_live) {
-        // ldmatrix.trans lane addressing: matrices (k0-7, n0-7) (k8-15, n0-7) (k0-7, n8-15) (k8-15, n8-15)
-        const uint32_t b_base = smem_u32(slab) + ((lane & 7) + ((lane >> 3) & 1) * 8) * kProjRowBytes + (lane >> 4) * 16;
-#pragma unroll 8
-        for (int k0 = k_begin; k0 < k_begin + k_len; k0 += 16) {
+    const uint32_t w_u32 = smem_u32(w_s), a_u32 = smem_u32(a_s);
+    // ldmatrix.x2.trans lane addressing: matrices (k0-7, n-tile) and (k8-15, n-tile); lanes 16-31 repeat 0-15
+    const uint32_t b_base = w_u32 + (lane & 15) * kProjRowBytes + ng * MT * 16;
+    const float *a_lo = a_s + (m0 + (lane >> 2)) * kProjALd + 2 * (lane & 3);
+    const float *a_hi = a_lo + 8 * kProjALd;
+#pragma unroll 1
+    for (int kc = 0; kc < k_len; kc += kProjChunk) {
+        const int kn = min(kProjChunk, k_len - kc);
+        if (kc > 0) __syncthreads();              // everyone is done with the previous chunk
+        {
+            const unsigned char *src = reinterpret_cast<const unsigned char *>(p.W);
+            for (int c = tid; c < kn * 8; c += 32 * kProjWarps) {       // W chunk: kn rows of 8 x 16 bytes
+                const int k = c >> 3, ch = c & 7;
+                const bool in = n0 + ch * 8 < p.N;                     // columns past N read as zero
+                cp_async16(w_u32 + k * kProjRowBytes + ch * 16,
+                           src + (in ? ((size_t)(k_begin + kc + k) * p.N + n0 + ch * 8) * 2 : 0), in ? 16 : 0);
+            }
+            const int cpr = kn >> 2;                                    // 16-byte chunks per activation row
+            for (int c = tid; c < 16 * MT * cpr; c += 32 * kProjWarps) {
+                const int r = c / cpr, ch = c % cpr;
+                const int row = row0 + min(r, rows - 1);                // rows past M repeat the last one (never stored)
+                cp_async16(a_u32 + (r * kProjALd + ch * 4) * 4, p.A + (size_t)row * p.K + k_begin + kc + ch * 4, 16);
+            }
+            cp_async_commit();
+        }
+        cp_async_wait<0>();
+        __syncthreads();
+#pragma unroll 1
+        for (int k0 = 0; k0 < kn; k0 += 16) {
             const float2 f0 = *reinterpret_cast<const float2 *>(a_lo + k0);
             const float2 f1 = *reinterpret_cast<const float2 *>(a_hi + k0);
             const float2 f2 = *reinterpret_cast<const float2 *>(a_lo + k0 + 8);
             const float2 f3 = *reinterpret_cast<const float2 *>(a_hi + k0 + 8);
-            uint32_t ah[4], am[4], al[4], b[4];
+            uint32_t ah[4], am[4], al[4];
             split3(f0.x, f0.y, ah[0], am[0], al[0]);
             split3(f1.x, f1.y, ah[1], am[1], al[1]);
             split3(f2.x, f2.y, ah[2], am[2], al[2]);
             split3(f3.x, f3.y, ah[3], am[3], al[3]);
-            ldsm_x4_trans_p(b_base + k0 * kProjRowBytes, b);
 #pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                mma_bf16_p(acc[t], al, b[2 * t], b[2 * t + 1]);      // smallest terms first
-                mma_bf16_p(acc[t], am, b[2 * t], b[2 * t + 1]);
-                mma_bf16_p(acc[t], ah, b[2 * t], b[2 * t + 1]);
+            for (int t = 0; t < MT; ++t) {
+                uint32_t b[2];
+                ldsm_x2_trans_p(b_base + k0 * kProjRowBytes + t * 16, b);
+                mma_bf16_p(acc[t], al, b[0], b[1]);      // smallest terms first
+                mma_bf16_p(acc[t], am, b[0], b[1]);
+                mma_bf16_p(acc[t], ah, b[0], b[1]);
             }
         }
     }
-    if (p.k_slices > 1) {       // block-uniform: the K slices of an m-tile are summed in slice order by slice 0
-        float *mine = s_red + ((size_t)warp * 32 + lane) * 8;
+    __syncthreads();      // the activation buffer becomes the partial strip
+    // partial strip of this K slice: rows m0 + lane/4 (+8), columns (ng*MT + t)*8 + 2*(lane%4) + {0,1}
 #pragma unroll
-        for (int t = 0; t < 2; ++t)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) mine[t * 4 + e] = acc[t][e];
-        __syncthreads();
-        if (ks != 0) return;
-        for (int s2 = 1; s2 < p.k_slices; ++s2) {
-            const float *other = s_red + ((size_t)(s2 * p.m_tiles + mt) * 32 + lane) * 8;
-#pragma unroll
-            for (int t = 0; t < 2; ++t)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) acc[t][e] += other[t * 4 + e];
-        }
+    for (int t = 0; t < MT; ++t) {
+        const int col = (ng * MT + t) * 8 + 2 * (lane & 3);
+        *reinterpret_cast<float2 *>(part + (m0 + (lane >> 2)) * kProjLd + col) = make_float2(acc[t][0], acc[t][1]);
+        *reinterpret_cast<float2 *>(part + (m0 + (lane >> 2) + 8) * kProjLd + col) = make_float2(acc[t][2], acc[t][3]);
     }
-    if (!warp_live) return;
-    // ---- epilogue: thread holds rows m0 + lane/4 (+8), columns n0 + t*8 + 2*(lane%4) + {0,1} ----
+    cluster.sync();
+    // block `rank` finishes columns [8 rank, 8 rank + 8) of the strip: sum the eight partials in rank order
+    const float *remote[kProjSlices];
 #pragma unroll
-    for (int rr = 0; rr < 2; ++rr) {
-        const int row = m0 + (lane >> 2) + rr * 8;
-        if (row >= p.M) continue;
-        if constexpr (MODE == 0) {
+    for (int q = 0; q < kProjSlices; ++q) remote[q] = cluster.map_shared_rank(part, q);
 #pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                const int n = n0 + t * 8 + 2 * (lane & 3);
-                if (n < p.N)
-                    *reinterpret_cast<float2 *>(p.Y + (size_t)row * p.N + n) = make_float2(acc[t][2 * rr], acc[t][2 * rr + 1]);
-            }
-        } else {
-            const int dq = p.d_v + p.d_r, nq = p.H * dq, nv = p.G * p.d_v;
-            const int t_pos = p.pos[row];
-            // cache slot of this sequence's new token (needed only by the value / positional-key columns)
-            long long page = -1;
-            int slot = 0;
-            const bool cache_cols = n0 + kProjCols > nq;
-            if (cache_cols) {
-                if (t_pos < 0 || t_pos / p.P >= p.max_pages) {
-                    if ((lane & 3) == 0) report_error(p.dev_status, GVA_ERR_SEQ_LEN, row);
-                } else {
-                    page = p.block_table ? (long long)p.block_table[(size_t)row * p.max_pages + t_pos / p.P]
-                                         : (long long)row * p.max_pages + t_pos / p.P;
-                    if (page < 0 || page >= p.num_pages) {
-                        if ((lane & 3) == 0) report_error(p.dev_status, GVA_ERR_BAD_PAGE, row);
-                        page = -1;
-                    }
-                    slot = t_pos % p.P;
-                }
-            }
+    for (int u = 0; u < 2; ++u) {
+        const int item = tid + u * 32 * kProjWarps;     // rows <= 128: at most two items per thread
+        if (item >= rows * 4) continue;
+        const int r = item >> 2, col = rank * 8 + (item & 3) * 2;
+        const int n = n0 + col;
+        if (n >= p.N) continue;
+        float c0 = 0.f, c1 = 0.f;
 #pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                const int n = n0 + t * 8 + 2 * (lane & 3);
-                const float c0 = acc[t][2 * rr], c1 = acc[t][2 * rr + 1];
-                if (n >= p.N) continue;
-                if (n < nq) {
-                    const int h = n / dq, j = n % dq;
-                    float *dst = p.q_abs + ((size_t)row * p.H + h) * dq + j;
-                    if (j < p.d_v) {
-                        *reinterpret_cast<float2 *>(dst) = make_float2(c0, c1);
-                    } else {
-                        double y0, y1;
-                        rope_pair((double)c0, (double)c1, t_pos, rope.inv_freq[(j - p.d_v) >> 1], y0, y1);
-                        *reinterpret_cast<float2 *>(dst) = make_float2(__double2float_rn(y0), __double2float_rn(y1));
-                    }
-                } else if (page >= 0) {
-                    if (n < nq + nv) {
-                        const int idx = n - nq, g = idx / p.d_v, d = idx % p.d_v;
-                        const size_t off = (((size_t)page * p.G + g) * p.P + slot) * p.d_v + d;
-                        if constexpr (sizeof(CT) == 2) {
-                            reinterpret_cast<uint32_t *>(reinterpret_cast<uint16_t *>(p.v_pool) + off)[0] =
-                                (uint32_t)float_to_bf16_bits(c0) | ((uint32_t)float_to_bf16_bits(c1) << 16);
-                        } else {
-                            *reinterpret_cast<float2 *>(reinterpret_cast<float *>(p.v_pool) + off) = make_float2(c0, c1);
-                        }
-                    } else {
-                        const int i = (n - nq - nv) >> 1;
-                        double y0, y1;
-                        rope_pair((double)c0, (double)c1, t_pos, rope.inv_freq[i], y0, y1);
-                        const size_t off = ((size_t)page * p.P + slot) * p.d_r + 2 * i;
-                        if constexpr (sizeof(CT) == 2) {
-                            reinterpret_cast<uint32_t *>(reinterpret_cast<uint16_t *>(p.kr_pool) + off)[0] =
-                                (uint32_t)double_to_bf16_bits(y0) | ((uint32_t)double_to_bf16_bits(y1) << 16);
-                        } else {
-                            *reinterpret_cast<float2 *>(reinterpret_cast<float *>(p.kr_pool) + off) =
-                                make_float2(__double2float_rn(y0), __double2float_rn(y1));
-                        }
-                    }
-                }
-            }
+        for (int q = 0; q < kProjSlices; ++q) {
+            const float2 v = *reinterpret_cast<const float2 *>(remote[q] + r * kProjLd + col);
+            c0 += v.x;
+            c1 += v.y;
         }
+        project_epilogue<MODE, CT>(p, rope, row0 + r, n, c0, c1, ep_pos[u]);
     }
+    cluster.sync();      // nobody leaves while another block may still read its shared memory
 }
 
 }  // namespace gva
