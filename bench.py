@@ -34,7 +34,7 @@ UNIT = "GB/s"
 
 # DRAM traffic of one decode-kernel launch on cfg2 at full size, from ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum, mean of two launches; profiles/decode_mma_kernel_cfg2.md).
-NCU_TRAFFIC_BYTES = {"cfg2": 0.5 * ((571_091_200 + 3_437_056) + (571_084_544 + 409_856))}
+NCU_TRAFFIC_BYTES = {"cfg2": 0.5 * ((571_105_024 + 4_873_216) + (571_087_360 + 387_584))}
 
 
 def load_peaks():
