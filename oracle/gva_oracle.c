@@ -17,6 +17,9 @@
  *   decode    : s_j = q~_h v_{j,g(h)}^T + q^rope_h (k^rope_j)^T ;  o_h = softmax(s/sqrt(d_qk)) V_{g(h)}
  *               with d_qk = d_c + d_r                     (Section 3.3 score equation; Algorithm 1)
  *   gqa       : matched GQA decode over cached K and V    (Section 2, GQA; Section 3.4)
+ *   prefill   : standard causal attention with the same content-position split, keys formed explicitly:
+ *               K_h = V_g(h) M_h (Eq. kvm), k_j = [K_h,j ; k^rope_j], q_i = [q^nope_i ; q^rope_i R_i^T]
+ *               (Section 3.3; the sentence after Algorithm 1 on training / multi-token attention)
  *
  * All arithmetic is double precision.  Cache pools are read in their storage type (bf16 bit
  * patterns or float32) and widened exactly.
@@ -258,6 +261,95 @@ void oracle_fold_maps(const double *W_q_nope, const double *M, int d_model, int 
                     acc += W_q_nope[((int64_t)m * H + h) * d_c + j] * M[((int64_t)h * d_v + i) * d_c + j];
                 W_abs[((int64_t)m * H + h) * d_v + i] = acc;
             }
+}
+
+/* ---- prefill / chunked prefill: standard causal attention with the content-position split --------
+ * Several query tokens per sequence.  Sequence b has ctx_lens[b] tokens cached before the chunk and
+ * q_lens = cu_q[b+1] - cu_q[b] new tokens whose value rows and rotated positional keys are ALREADY in
+ * the cache (appended first, as in Algorithm 1); query token i of sequence b sits at position
+ * t = ctx_lens[b] + i and attends to positions 0..t.  Nothing is absorbed here: the content keys are
+ * formed explicitly, K_h = V_g(h) M_h (Eq. kvm), and the score is the full-key dot product
+ *   s_ij = q^nope_i . K_h,j + (q^rope_i R_t^T) . k^rope_j,   o_i = softmax_j<=t(s_ij / sqrt(d_qk)) V_g(h).
+ * q_c [n_q][H][d_c], q_r [n_q][H][d_r] unrotated, M [H][d_v][d_c]; out [n_q][H][d_v], lse [n_q][H]. */
+void oracle_prefill(const void *v_pool, const void *kr_pool, int dtype, const int32_t *block_table,
+                    int max_pages, int P, const int32_t *cu_q, const int32_t *ctx_lens, const double *q_c,
+                    const double *q_r, const double *M, double base, double scale, int B, int H, int G,
+                    int d_v, int d_c, int d_r, double *out, double *lse) {
+    int hpg = H / G;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            int g = h / hpg;
+            int n_q = cu_q[b + 1] - cu_q[b];
+            int T = ctx_lens[b] + n_q;                     /* tokens in the cache after the chunk's append */
+            if (n_q <= 0) continue;
+            /* explicit keys of this head: K[j][:] = v_j M_h  (d_c wide), and the value rows widened */
+            double *K = (double *)malloc(sizeof(double) * (size_t)T * (size_t)d_c);
+            double *V = (double *)malloc(sizeof(double) * (size_t)T * (size_t)d_v);
+            double *R = (double *)malloc(sizeof(double) * (size_t)T * (size_t)(d_r > 0 ? d_r : 1));
+            double *s = (double *)malloc(sizeof(double) * (size_t)T);
+            double *qrot = (double *)malloc(sizeof(double) * (size_t)(d_r > 0 ? d_r : 1));
+            for (int j = 0; j < T; ++j) {
+                int64_t page = page_of(block_table, max_pages, b, j / P);
+                int slot = j % P;
+                for (int i = 0; i < d_v; ++i) V[(int64_t)j * d_v + i] = load_elem(v_pool, dtype, ((page * G + g) * P + slot) * d_v + i);
+                for (int k = 0; k < d_r; ++k) R[(int64_t)j * d_r + k] = load_elem(kr_pool, dtype, (page * P + slot) * d_r + k);
+                for (int c = 0; c < d_c; ++c) {
+                    double acc = 0.0;
+                    for (int i = 0; i < d_v; ++i) acc += V[(int64_t)j * d_v + i] * M[((int64_t)h * d_v + i) * d_c + c];
+                    K[(int64_t)j * d_c + c] = acc;
+                }
+            }
+            for (int i = 0; i < n_q; ++i) {
+                int64_t row = (int64_t)(cu_q[b] + i) * H + h;
+                int t = ctx_lens[b] + i;
+                const double *qc = q_c + row * d_c;
+                oracle_rope(q_r + row * d_r, d_r, (double)t, base, qrot);
+                double m = -INFINITY;
+                for (int j = 0; j <= t; ++j) {
+                    double acc = 0.0;
+                    for (int c = 0; c < d_c; ++c) acc += qc[c] * K[(int64_t)j * d_c + c];
+                    for (int k = 0; k < d_r; ++k) acc += qrot[k] * R[(int64_t)j * d_r + k];
+                    s[j] = acc * scale;
+                    if (s[j] > m) m = s[j];
+                }
+                double L = 0.0;
+                for (int j = 0; j <= t; ++j) { s[j] = exp(s[j] - m); L += s[j]; }
+                double *o = out + row * d_v;
+                for (int d = 0; d < d_v; ++d) o[d] = 0.0;
+                for (int j = 0; j <= t; ++j) {
+                    double p = s[j] / L;
+                    for (int d = 0; d < d_v; ++d) o[d] += p * V[(int64_t)j * d_v + d];
+                }
+                if (lse) lse[row] = m + log(L);
+            }
+            free(K); free(V); free(R); free(s); free(qrot);
+        }
+}
+
+/* Append of a chunk: token i of sequence b (i < cu_q[b+1]-cu_q[b]) is written at position ctx_lens[b] + i,
+ * exactly as oracle_append writes one token (Algorithm 1's append lines, once per new token).
+ * v_new [n_q][G][d_v], kr_new [n_q][d_r] unrotated.  Returns 0, or 1+b for the first bad page. */
+int oracle_append_chunk(void *v_pool, void *kr_pool, int dtype, const int32_t *block_table, int num_pages,
+                        int max_pages, int P, int G, int d_v, int d_r, double base, const double *v_new,
+                        const double *kr_new, const int32_t *cu_q, const int32_t *ctx_lens, int B) {
+    double *rot = (double *)malloc(sizeof(double) * (size_t)(d_r > 0 ? d_r : 1));
+    int rc = 0;
+    for (int b = 0; b < B && !rc; ++b)
+        for (int i = 0; i < cu_q[b + 1] - cu_q[b]; ++i) {
+            int64_t n = cu_q[b] + i;
+            int t = ctx_lens[b] + i;
+            int64_t page = page_of(block_table, max_pages, b, t / P);
+            int slot = t % P;
+            if (t < 0 || t / P >= max_pages || page < 0 || page >= num_pages) { rc = 1 + b; break; }
+            for (int g = 0; g < G; ++g)
+                for (int d = 0; d < d_v; ++d)
+                    store_elem(v_pool, dtype, ((page * G + g) * P + slot) * d_v + d, v_new[(n * G + g) * d_v + d]);
+            oracle_rope(kr_new + n * d_r, d_r, (double)t, base, rot);
+            for (int k = 0; k < d_r; ++k) store_elem(kr_pool, dtype, (page * P + slot) * d_r + k, rot[k]);
+        }
+    free(rot);
+    return rc;
 }
 
 #ifdef _OPENMP

@@ -39,6 +39,7 @@ def lib() -> ctypes.CDLL:
         _lib.oracle_bf16_from_double.argtypes = [ctypes.c_double]
         _lib.oracle_num_threads.restype = ctypes.c_int
         _lib.oracle_append.restype = ctypes.c_int
+        _lib.oracle_append_chunk.restype = ctypes.c_int
     return _lib
 
 
@@ -244,6 +245,56 @@ def layer_step(x, W_in, W_o, v_pool, kr_pool, block_table, pos, seq_lens, H: int
                     max_pages_per_seq=max_pages_per_seq)
     y = matmul(out.reshape(out.shape[0], -1), W_o)
     return y, out, q_abs
+
+
+def prefill(v_pool, kr_pool, block_table, cu_q, ctx_lens, q_c, q_r, M, base: float = 10000.0,
+            scale: Optional[float] = None, max_pages_per_seq: Optional[int] = None):
+    """Causal attention of a chunk of new tokens per sequence with explicitly formed keys K_h = V_g M_h.
+    q_c [n_q,H,d_c], q_r [n_q,H,d_r] unrotated; query i of sequence b is at position ctx_lens[b] + i and its
+    value rows / positional key are already cached.  Returns (out [n_q,H,d_v], lse [n_q,H])."""
+    dt = _dt(v_pool)
+    assert v_pool.flags.c_contiguous and kr_pool.flags.c_contiguous and _dt(kr_pool) == dt
+    _, G, P, d_v = v_pool.shape
+    d_r = kr_pool.shape[-1]
+    q_c, q_r, M = _f64(q_c), _f64(q_r), _f64(M)
+    cu_q, ctx_lens = _i32(cu_q), _i32(ctx_lens)
+    B = ctx_lens.shape[0]
+    n_q, H, d_c = q_c.shape
+    assert cu_q.shape == (B + 1,) and int(cu_q[-1]) == n_q and q_r.shape == (n_q, H, d_r) and M.shape == (H, d_v, d_c)
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d_c + d_r))
+    bt = None if block_table is None else _i32(block_table)
+    max_pages = bt.shape[1] if bt is not None else int(max_pages_per_seq)
+    out = np.zeros((n_q, H, d_v), dtype=np.float64)
+    lse = np.zeros((n_q, H), dtype=np.float64)
+    lib().oracle_prefill(_p(v_pool), _p(kr_pool), ctypes.c_int(dt), _p(bt), ctypes.c_int(max_pages), ctypes.c_int(P),
+                         _p(cu_q), _p(ctx_lens), _p(q_c), _p(q_r), _p(M), ctypes.c_double(base), ctypes.c_double(scale),
+                         *map(ctypes.c_int, (B, H, G, d_v, d_c, d_r)), _p(out), _p(lse))
+    return out, lse
+
+
+def append_chunk(v_pool, kr_pool, block_table, v_new, kr_new, cu_q, ctx_lens, base: float = 10000.0,
+                 max_pages_per_seq: Optional[int] = None) -> int:
+    """In-place append of a chunk: token i of sequence b goes to position ctx_lens[b] + i."""
+    dt = _dt(v_pool)
+    assert v_pool.flags.c_contiguous and kr_pool.flags.c_contiguous and _dt(kr_pool) == dt
+    num_pages, G, P, d_v = v_pool.shape
+    d_r = kr_pool.shape[-1]
+    v_new, kr_new, cu_q, ctx_lens = _f64(v_new), _f64(kr_new), _i32(cu_q), _i32(ctx_lens)
+    B = ctx_lens.shape[0]
+    bt = None if block_table is None else _i32(block_table)
+    max_pages = bt.shape[1] if bt is not None else int(max_pages_per_seq)
+    return int(lib().oracle_append_chunk(_p(v_pool), _p(kr_pool), ctypes.c_int(dt), _p(bt), ctypes.c_int(num_pages),
+                                         ctypes.c_int(max_pages), ctypes.c_int(P), ctypes.c_int(G), ctypes.c_int(d_v),
+                                         ctypes.c_int(d_r), ctypes.c_double(base), _p(v_new), _p(kr_new), _p(cu_q),
+                                         _p(ctx_lens), ctypes.c_int(B)))
+
+
+def prefill_case(pc):
+    """Oracle outputs of a workloads.PrefillCase-like object (duck-typed)."""
+    c = pc.cache
+    return prefill(c.v_pool, c.kr_pool, c.block_table, pc.cu_q, pc.ctx_lens, pc.q_c, pc.q_r, c.M, c.rope_base,
+                   max_pages_per_seq=c.max_pages_per_seq)
 
 
 # ---- convenience over a workloads.DecodeCase-like object (duck-typed; no import of the generator) ----

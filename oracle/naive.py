@@ -132,3 +132,27 @@ def layer_decode_step(x, W_Q, W_V, W_r, W_O, M, t: int, V_cache, KR_cache, H: in
     concat = [v for o in outs for v in o]
     y = [sum(concat[r] * W_O[r][m] for r in range(len(concat))) for m in range(d_model)]
     return y, outs
+
+
+def prefill_sequence(q_c, q_r, M, ctx: int, V_tokens, KR_tokens, H: int, G: int, base: float = 10000.0):
+    """Causal attention of a chunk for ONE sequence, with explicit keys (nothing absorbed) and plain loops.
+
+    q_c[i][h][d_c], q_r[i][h][d_r] (unrotated) for the chunk's tokens i = 0..n-1 at positions ctx + i;
+    V_tokens[t][g] / KR_tokens[t] as in decode_step, holding ctx + n tokens.  Returns out[i][h][d_v]."""
+    out = []
+    for i in range(len(q_c)):
+        t = ctx + i
+        row = []
+        for h in range(H):
+            g = h // (H // G)
+            d_c, d_r = len(q_c[i][h]), len(q_r[i][h])
+            qr = rope(q_r[i][h], t, base) if d_r else []
+            s = []
+            for j in range(t + 1):
+                k = reconstruct_key(V_tokens[j][g], M[h])
+                s.append((sum(a * b for a, b in zip(q_c[i][h], k)) + sum(a * b for a, b in zip(qr, KR_tokens[j])))
+                         / math.sqrt(d_c + d_r))
+            p = softmax(s)
+            row.append([sum(p[j] * V_tokens[j][g][d] for j in range(t + 1)) for d in range(len(M[h]))])
+        out.append(row)
+    return out

@@ -279,6 +279,67 @@ def gqa_case(name: str, H: int, G: int, d_h: int, seq_lens, *, page_size: int = 
                 k_pool=k_pool, v_pool=v_pool, block_table=bt, seq_lens=seq_lens, q=q, cache_dtype=cache_dtype)
 
 
+# ---- prefill / chunked prefill: several query tokens per sequence ------------------------------------
+@dataclass
+class PrefillCase:
+    """A chunk of new tokens per sequence on top of a (possibly empty) cached context.
+
+    `cache` is a DecodeCase whose pools already hold every token (context and chunk) and whose seq_lens are
+    ctx_lens + q_lens; its per-sequence q_c / q_r / v_new / kr_new fields are not used.  Query token i of
+    sequence b is row cu_q[b] + i of q_c / q_r and sits at position ctx_lens[b] + i."""
+    name: str
+    cache: DecodeCase
+    ctx_lens: np.ndarray                  # int32 [B]   tokens cached before the chunk
+    q_lens: np.ndarray                    # int32 [B]   new tokens
+    cu_q: np.ndarray                      # int32 [B+1] exclusive prefix sums of q_lens
+    q_c: np.ndarray                       # f32 [n_q, H, d_c]
+    q_r: np.ndarray                       # f32 [n_q, H, d_r]   unrotated
+    q_pos: np.ndarray                     # int32 [n_q] position of every query token
+    q_seq: np.ndarray                     # int32 [n_q] sequence of every query token
+    v_new: np.ndarray                     # f32 [n_q, G, d_v]  rows for a chunk append
+    kr_new: np.ndarray                    # f32 [n_q, d_r]     unrotated positional keys for a chunk append
+
+    @property
+    def n_q(self) -> int:
+        return int(self.cu_q[-1])
+
+    def pairs(self) -> int:
+        """(query, key) pairs under the causal mask, summed over sequences (per head)."""
+        c, n = self.ctx_lens.astype(np.int64), self.q_lens.astype(np.int64)
+        return int((n * c + n * (n + 1) // 2).sum())
+
+    def flops(self) -> int:
+        """Multiply-adds x 2 of the absorbed form: per pair and head (d_v + d_r) for the score, d_v for the value sum."""
+        s = self.cache.shape
+        return 2 * self.pairs() * s.H * (2 * s.d_v + s.d_r)
+
+
+def make_prefill_case(name: str, shape: HeadShape, ctx_lens, q_lens, *, page_size: int = 64, cache_dtype: str = "bf16",
+                      paged: bool = True, seed: int = MASTER_SEED + 7000, poison_unused: bool = False,
+                      extra_pages: int = 0, q_gain: float = 1.0) -> PrefillCase:
+    ctx_lens = np.asarray(ctx_lens, dtype=np.int32)
+    q_lens = np.asarray(q_lens, dtype=np.int32)
+    cache = make_case(name, shape, ctx_lens + q_lens, page_size=page_size, cache_dtype=cache_dtype, paged=paged, seed=seed,
+                      extra_pages=extra_pages, poison_unused=poison_unused)
+    rng = _rng(seed + 1)
+    cu_q = np.zeros(len(q_lens) + 1, dtype=np.int32)
+    cu_q[1:] = np.cumsum(q_lens)
+    n_q = int(cu_q[-1])
+    q_c = (q_gain * rng.standard_normal((n_q, shape.H, shape.d_c), dtype=np.float32)).astype(np.float32)
+    q_r = (q_gain * rng.standard_normal((n_q, shape.H, shape.d_r), dtype=np.float32)).astype(np.float32)
+    v_new = rng.standard_normal((n_q, shape.G, shape.d_v), dtype=np.float32)
+    kr_new = rng.standard_normal((n_q, shape.d_r), dtype=np.float32)
+    q_seq = np.repeat(np.arange(len(q_lens), dtype=np.int32), q_lens)
+    q_pos = (ctx_lens[q_seq] + (np.arange(n_q, dtype=np.int32) - cu_q[q_seq])).astype(np.int32)
+    return PrefillCase(name=name, cache=cache, ctx_lens=ctx_lens, q_lens=q_lens, cu_q=cu_q, q_c=q_c, q_r=q_r,
+                       q_pos=q_pos, q_seq=q_seq, v_new=v_new, kr_new=kr_new)
+
+
+def prefill_bench_case(seed: int = MASTER_SEED + 7100, B: int = 8, T: int = 8192) -> PrefillCase:
+    """Whole-prompt prefill on the headline head shape: B prompts of T tokens, empty context, 64-token pages."""
+    return make_prefill_case("prefill", SHAPE_A, [0] * B, [T] * B, page_size=64, seed=seed)
+
+
 def layer_weights(shape: HeadShape, d_model: int, B: int, seed: int = MASTER_SEED + 6000) -> dict:
     """Seeded projections around the attention of one layer and one hidden state per sequence.
     Every weight ~ N(0, 1/fan_in) (so projected activations stay unit-scale), x ~ N(0, 1):

@@ -523,3 +523,125 @@ def test_bf16_round_matches_library_cast():
     a = rng.standard_normal(300).astype(np.float32)
     ref = torch.from_numpy(a).bfloat16().view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(orc.bf16_round(a), ref)
+
+
+# ---------------------------------------------------------------- prefill / chunked prefill (causal, explicit keys)
+def small_prefill(cache_dtype="bf16", paged=True, seed=31):
+    s = wl.HeadShape(H=4, G=2, d_v=8, d_c=6, d_r=4)
+    return wl.make_prefill_case("pf", s, [0, 5, 3, 9], [7, 4, 0, 1], page_size=4, cache_dtype=cache_dtype, paged=paged,
+                                seed=seed, poison_unused=True)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_prefill_causal_sdpa_equivalence(dtype):
+    # library routine with an explicit boolean causal mask over explicitly formed full keys [V M_h | k^rope]
+    pc = small_prefill(dtype)
+    c, s = pc.cache, pc.cache.shape
+    out, lse = orc.prefill_case(pc)
+    V = torch.from_numpy(wl.pool_to_f64(c.v_pool)); KR = torch.from_numpy(wl.pool_to_f64(c.kr_pool))
+    M = torch.from_numpy(c.M.astype(np.float64))
+    for b in range(c.B):
+        n, ctx = int(pc.q_lens[b]), int(pc.ctx_lens[b])
+        if n == 0:
+            continue
+        L = ctx + n
+        pages = [c.page_of(b, t // c.page_size) for t in range(L)]; slots = [t % c.page_size for t in range(L)]
+        rows = slice(int(pc.cu_q[b]), int(pc.cu_q[b + 1]))
+        q_rot = np.stack([orc.rope(pc.q_r[int(pc.cu_q[b]) + i], ctx + i) for i in range(n)])            # [n, H, d_r]
+        q_full = torch.cat([torch.from_numpy(pc.q_c[rows].astype(np.float64)), torch.from_numpy(q_rot)], dim=-1)
+        mask = torch.arange(L)[None, :] <= (ctx + torch.arange(n))[:, None]                              # [n, L]
+        for h in range(s.H):
+            Vg = V[pages, h // (s.H // s.G), slots]
+            K = torch.cat([Vg @ M[h], KR[pages, slots]], dim=-1)
+            ref = torch.nn.functional.scaled_dot_product_attention(
+                q_full[None, None, :, h], K[None, None], Vg[None, None], attn_mask=mask[None, None],
+                scale=1.0 / math.sqrt(s.d_c + s.d_r))[0, 0]
+            assert np.allclose(out[rows, h], ref.numpy(), atol=1e-12)
+            logits = (q_full[:, h] @ K.T) / math.sqrt(s.d_c + s.d_r)
+            ref_lse = torch.logsumexp(logits.masked_fill(~mask, -math.inf), dim=-1)
+            assert np.allclose(lse[rows, h], ref_lse.numpy(), atol=1e-12)
+
+
+def test_prefill_row_equals_decode_of_its_prefix():
+    # each query row is one decode step over the first t+1 tokens (Algorithm 1 applied token by token); the decode
+    # oracle uses the absorbed form, the prefill oracle explicit keys, so this is also the absorption identity
+    pc = small_prefill("bf16", paged=True, seed=32)
+    c, s = pc.cache, pc.cache.shape
+    out, lse = orc.prefill_case(pc)
+    q_abs = orc.absorb(pc.q_c, pc.q_r, c.M, pc.q_pos)
+    for n in range(pc.n_q):
+        b = int(pc.q_seq[n])
+        lens = np.zeros(c.B, dtype=np.int32); lens[b] = pc.q_pos[n] + 1
+        qa = np.zeros((c.B, s.H, s.d_v + s.d_r)); qa[b] = q_abs[n]
+        o, l = orc.decode(c.v_pool, c.kr_pool, c.block_table, lens, qa, s.H, d_c=s.d_c)
+        assert np.allclose(out[n], o[b], atol=1e-13) and np.allclose(lse[n], l[b], atol=1e-13)
+
+
+def test_prefill_brute_force_and_closed_forms():
+    pc = small_prefill("f32", paged=True, seed=33)
+    c, s = pc.cache, pc.cache.shape
+    out, lse = orc.prefill_case(pc)
+    V = wl.pool_to_f64(c.v_pool).tolist(); KR = wl.pool_to_f64(c.kr_pool).tolist()
+    Vt, Kt = naive.gather_tokens(V, KR, c.block_table.tolist(), c.seq_lens.tolist(), c.page_size, c.max_pages_per_seq)
+    for b in range(c.B):
+        rows = slice(int(pc.cu_q[b]), int(pc.cu_q[b + 1]))
+        o2 = naive.prefill_sequence(pc.q_c[rows].astype(np.float64).tolist(), pc.q_r[rows].astype(np.float64).tolist(),
+                                    c.M.astype(np.float64).tolist(), int(pc.ctx_lens[b]), Vt[b], Kt[b], s.H, s.G)
+        if pc.q_lens[b]:
+            assert np.allclose(out[rows], np.array(o2), atol=1e-13)
+    # the first token of a prompt with no context sees only itself: o = its own value row, lse = its own score
+    first = int(pc.cu_q[0])
+    Vd = wl.pool_to_f64(c.v_pool)
+    for h in range(s.H):
+        g = h // (s.H // s.G)
+        assert np.allclose(out[first, h], Vd[c.page_of(0, 0), g, 0], atol=1e-15)
+    # zero queries: uniform weights over the visible prefix -> running mean of the value rows, lse = log(t + 1)
+    pz = small_prefill("f32", paged=False, seed=34)
+    pz.q_c[:] = 0; pz.q_r[:] = 0
+    oz, lz = orc.prefill_case(pz)
+    cz = pz.cache
+    Vz = wl.pool_to_f64(cz.v_pool)
+    for n in range(pz.n_q):
+        b, t = int(pz.q_seq[n]), int(pz.q_pos[n])
+        rowsV = np.stack([Vz[cz.page_of(b, j // cz.page_size), :, j % cz.page_size] for j in range(t + 1)])   # [t+1, G, d_v]
+        for h in range(s.H):
+            assert np.allclose(oz[n, h], rowsV[:, h // (s.H // s.G)].mean(axis=0), atol=1e-14)
+        assert np.allclose(lz[n], math.log(t + 1), atol=1e-14)
+
+
+def test_prefill_is_causal_and_chunking_invariant():
+    # (a) changing a later token's cache rows or queries never changes an earlier row; (b) splitting the same
+    # prompt into [context | chunk] at any point gives the same rows as prefilling it whole
+    s = wl.HeadShape(H=4, G=2, d_v=8, d_c=6, d_r=4)
+    whole = wl.make_prefill_case("w", s, [0], [11], page_size=4, cache_dtype="f32", paged=True, seed=35)
+    out_w, lse_w = orc.prefill_case(whole)
+    for cut in (1, 4, 10):
+        part = wl.make_prefill_case("p", s, [cut], [11 - cut], page_size=4, cache_dtype="f32", paged=True, seed=35)
+        assert np.array_equal(part.cache.v_pool, whole.cache.v_pool)           # same seeded cache
+        part.q_c[:] = whole.q_c[cut:]; part.q_r[:] = whole.q_r[cut:]
+        o, l = orc.prefill_case(part)
+        assert np.allclose(o, out_w[cut:], atol=1e-14) and np.allclose(l, lse_w[cut:], atol=1e-14)
+    c = whole.cache
+    page, slot = c.page_of(0, 7 // 4), 7 % 4
+    c.v_pool[page, :, slot] += 3.0
+    c.kr_pool[page, slot] -= 2.0
+    whole.q_c[8:] *= -1
+    o2, _ = orc.prefill_case(whole)
+    assert np.array_equal(o2[:7], out_w[:7]) and not np.allclose(o2[7], out_w[7])
+
+
+def test_append_chunk_equals_token_by_token_append():
+    pc = small_prefill("bf16", paged=True, seed=36)
+    c = pc.cache
+    v1, k1 = c.v_pool.copy(), c.kr_pool.copy()
+    v2, k2 = c.v_pool.copy(), c.kr_pool.copy()
+    assert orc.append_chunk(v1, k1, c.block_table, pc.v_new, pc.kr_new, pc.cu_q, pc.ctx_lens) == 0
+    for n in range(pc.n_q):                       # Algorithm 1's append, one token at a time
+        b = int(pc.q_seq[n])
+        vn = np.zeros((c.B,) + pc.v_new.shape[1:], dtype=np.float32); kn = np.zeros((c.B, pc.kr_new.shape[1]), dtype=np.float32)
+        vn[b], kn[b] = pc.v_new[n], pc.kr_new[n]
+        # append only sequence b: a one-sequence view of the block table
+        assert orc.append(v2, k2, c.block_table[b:b + 1], vn[b:b + 1], kn[b:b + 1], [int(pc.q_pos[n])]) == 0
+    assert np.array_equal(v1, v2) and np.array_equal(k1, k2)
+    changed = np.argwhere((v1 != c.v_pool).any(axis=(1, 3)))
+    assert len(changed) <= pc.n_q                                  # at most one (page, slot) per new token
