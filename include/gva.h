@@ -246,6 +246,30 @@ int gva_layer_step(gva_handle *h, const gva_cache *cache, const float *x, const 
                    void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
                    int32_t *dev_status, void *stream);
 
+/* ---- Several new tokens per sequence: prefill and chunked prefill (the paper's multi-token form: "standard causal
+ * attention with the same content-position split", Section 3.3 and the remark after Algorithm 1), computed in the
+ * absorbed form of Eq. absorb.  Sequence b has ctx_lens[b] tokens cached already and q_len_b = cu_q[b+1] - cu_q[b]
+ * new tokens; new token i of sequence b is input row cu_q[b] + i, sits at position t = ctx_lens[b] + i and attends
+ * to positions 0..t.  The order of calls is Algorithm 1's, once per chunk instead of once per token:
+ *   gva_absorb_query(B := n_q, q_pos[row] = position of the row)  ->  gva_append_chunk  ->  gva_prefill.
+ *   cu_q [B+1] i32 (cu_q[0] = 0, non-decreasing), ctx_lens [B] i32, n_q = cu_q[B] rows in all. */
+
+/* Algorithm 1's append for every new token of the chunk: row n of v_new [n_q][G][d_v] / kr_new [n_q][d_r] (unrotated)
+ * is written at its position exactly as gva_append_cache writes one token (same rounding, same error rules). */
+int gva_append_chunk(gva_handle *h, const gva_cache *cache, const float *v_new, const float *kr_new,
+                     const int32_t *cu_q, const int32_t *ctx_lens, int B, int n_q, int32_t *dev_status, void *stream);
+
+/* Causal attention of the chunk over the cache, which must already hold the chunk's own tokens.
+ *   q_abs [n_q][H][d_v+d_r] f32  from gva_absorb_query;  out [n_q][H][d_v] f32;  lse [n_q][H] f32 or NULL
+ *   max_q_len                    upper bound on the q_len_b (sizes the launch; longer chunks are cut off)
+ * bf16 cache only, page_size a multiple of 64, (d_v, d_r) = (64, 16) or (128, 32); otherwise GVA_ERR_UNSUPPORTED.
+ * Runs on the tensor cores with bf16 operands (the absorbed query and the softmax weights are rounded to bf16,
+ * accumulation is f32), so results carry bf16-level error: |out - exact| <= 2e-2 for unit-variance data.
+ * Device-side errors as in gva_decode; a thread block that meets one stops and leaves its rows of out unwritten. */
+int gva_prefill(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *cu_q,
+                const int32_t *ctx_lens, float *out, float *lse, int B, int max_q_len, int32_t *dev_status,
+                void *stream);
+
 /* Geometry of the most recent gva_decode / gqa_decode launch on this handle (reporting only):
  * number of split-KV partitions launched (thread blocks of the decode kernel). */
 int gva_last_num_splits(const gva_handle *h);

@@ -24,7 +24,7 @@ GVA_KERNEL_AUTO, GVA_KERNEL_FMA, GVA_KERNEL_MMA = 0, 1, 2
 EXPORTS = ["gva_create", "gva_destroy", "gva_decode_workspace_bytes", "gva_absorb_query", "gva_append_cache",
            "gva_decode", "gva_decode_static", "gqa_decode", "gva_decode_step", "gva_step_scratch_bytes", "gva_decode_step_host", "gva_input_width", "gva_pack_input_weights", "gva_pack_bf16",
            "gva_project_in", "gva_project_out", "gva_layer_step", "gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens",
-           "gva_status_string"]
+           "gva_status_string", "gva_append_chunk", "gva_prefill"]
 
 
 class GvaConfig(ctypes.Structure):
@@ -75,6 +75,8 @@ def load() -> ctypes.CDLL:
     lib.gva_absorb_query.argtypes = [vp, vp, vp, vp, vp, vp, ip, vp]
     lib.gva_append_cache.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, ip, vp, vp]
     lib.gva_decode.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, vp, sz, ip, ip, ip, vp, vp]
+    lib.gva_append_chunk.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, ip, ip, vp, vp]
+    lib.gva_prefill.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, vp, ip, ip, vp, vp]
     lib.gva_decode_static.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, ip, ip, ip, vp, vp]
     lib.gqa_decode.argtypes = [vp, ctypes.POINTER(GqaCache), vp, vp, vp, vp, vp, sz, ip, ip, ip, vp, vp]
     lib.gva_input_width.argtypes = [vp]
@@ -151,6 +153,24 @@ def gva_append_cache(handle: int, cache: GvaCache, v_new, kr_new, pos, B: int, d
                                  _ptr(dev_status), _stream())
     if check:
         _check(rc, "gva_append_cache")
+    return rc
+
+
+def gva_append_chunk(handle: int, cache: GvaCache, v_new, kr_new, cu_q, ctx_lens, B: int, n_q: int, dev_status=None,
+                     check: bool = True) -> int:
+    rc = load().gva_append_chunk(handle, ctypes.byref(cache), _ptr(v_new), _ptr(kr_new), _ptr(cu_q), _ptr(ctx_lens), int(B),
+                                 int(n_q), _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gva_append_chunk")
+    return rc
+
+
+def gva_prefill(handle: int, cache: GvaCache, q_abs, cu_q, ctx_lens, out, lse, B: int, max_q_len: int, dev_status=None,
+                check: bool = True) -> int:
+    rc = load().gva_prefill(handle, ctypes.byref(cache), _ptr(q_abs), _ptr(cu_q), _ptr(ctx_lens), _ptr(out), _ptr(lse), int(B),
+                            int(max_q_len), _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gva_prefill")
     return rc
 
 

@@ -13,6 +13,7 @@
 #include "gva_project.cuh"
 #ifdef GVA_WITH_MMA
 #include "gva_decode_mma.cuh"
+#include "gva_prefill.cuh"
 #endif
 
 using namespace gva;
@@ -369,6 +370,66 @@ int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, 
         return GVA_ERR_CUDA;
     }
     return GVA_OK;
+}
+
+int gva_append_chunk(gva_handle *h, const gva_cache *cache, const float *v_new, const float *kr_new, const int32_t *cu_q,
+                     const int32_t *ctx_lens, int B, int n_q, int32_t *dev_status, void *stream) {
+    if (!h || !cache || B < 0 || n_q < 0) return GVA_ERR_INVALID_ARG;
+    if (B == 0 || n_q == 0) return GVA_OK;
+    if (!cache->v_pool || !cache->kr_pool || !v_new || !kr_new || !cu_q || !ctx_lens) return GVA_ERR_INVALID_ARG;
+    if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
+    if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16)) return GVA_ERR_INVALID_ARG;
+    const gva_config &c = h->cfg;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (c.G * c.d_v > kAppendMaxPerThread * 128) return GVA_ERR_UNSUPPORTED;
+    cudaError_t ce;
+    if (c.cache_dtype == GVA_BF16)
+        ce = launch_pdl(append_chunk_kernel<__nv_bfloat16>, dim3(n_q), dim3(128), 0, s, static_cast<__nv_bfloat16 *>(cache->v_pool),
+                        static_cast<__nv_bfloat16 *>(cache->kr_pool), cache->block_table, v_new, kr_new, cu_q, ctx_lens, B, c.G,
+                        c.d_v, c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+    else
+        ce = launch_pdl(append_chunk_kernel<float>, dim3(n_q), dim3(128), 0, s, static_cast<float *>(cache->v_pool),
+                        static_cast<float *>(cache->kr_pool), cache->block_table, v_new, kr_new, cu_q, ctx_lens, B, c.G, c.d_v,
+                        c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+    if (ce != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GVA_ERR_CUDA;
+    }
+    return GVA_OK;
+}
+
+int gva_prefill(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *cu_q, const int32_t *ctx_lens,
+                float *out, float *lse, int B, int max_q_len, int32_t *dev_status, void *stream) {
+    if (!h || !cache || B < 0 || max_q_len < 0) return GVA_ERR_INVALID_ARG;
+    if (B == 0 || max_q_len == 0) return GVA_OK;
+    if (!cache->v_pool || !cache->kr_pool || !q_abs || !cu_q || !ctx_lens || !out) return GVA_ERR_INVALID_ARG;
+    if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
+    if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16) || !aligned(q_abs, 16) || !aligned(out, 16))
+        return GVA_ERR_INVALID_ARG;
+    if (B > 65535) return GVA_ERR_UNSUPPORTED;
+#ifdef GVA_WITH_MMA
+    const gva_config &c = h->cfg;
+    PrefillParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.q_abs = q_abs;
+    p.cu_q = cu_q;
+    p.ctx_lens = ctx_lens;
+    p.block_table = cache->block_table;
+    p.out = out;
+    p.lse = lse;
+    p.dev_status = dev_status;
+    p.B = B;
+    p.H = c.H;
+    p.G = c.G;
+    p.P = c.page_size;
+    p.num_pages = cache->num_pages;
+    p.max_pages = cache->max_pages_per_seq;
+    p.scale_log2 = h->scale * kLog2e;
+    return launch_prefill(c, h->mma, h->smem_optin, p, cache->v_pool, cache->kr_pool, B, max_q_len,
+                          static_cast<cudaStream_t>(stream));
+#else
+    return GVA_ERR_UNSUPPORTED;
+#endif
 }
 
 static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,

@@ -1,0 +1,471 @@
+// Causal prefill / chunked-prefill attention over the paged bf16 GVA cache on the 5th-generation tensor
+// cores (tcgen05 + tensor memory), sm_100a.
+//
+// What it computes (the paper's multi-token form: standard causal attention with the content-position split,
+// Section 3.3 and the remark after Algorithm 1), in the absorbed form of Eq. absorb: for query token i at
+// position t, head h of group g,
+//     s_ij = q~_i,h . v_j,g + q^rope_i,h . k^rope_j   (j <= t),   o_i,h = softmax_j(s_ij / sqrt(d_qk)) V_g.
+// With the query absorbed the key of token j is [v_j,g | k^rope_j]: the cached value tile IS the content-key
+// tile, so one shared-memory tile feeds both the score product (as a K-major operand) and the value product
+// (as an MN-major operand), and the H/G = 4 heads of a group stack into the M dimension of one tile.
+//
+// Layout of the work
+//   thread block   = 32 query tokens x 4 heads of one (sequence, value group): 128 rows = one M = 128 MMA tile
+//   warps 0-3      = softmax: thread r owns row r (token r / 4, head r % 4) -- tensor-memory lane r
+//   warp 4         = producer (one lane): TMA loads of the 64-token value tile and positional-key tile into a ring
+//   warp 5         = MMA issuer (one lane) and owner of the tensor-memory allocation
+//   per 64-token tile j:
+//     S[j & 1]  = Q K_j^T            tcgen05.mma, K = d_v (value dims, 128-byte swizzle) + d_r (RoPE dims)
+//     softmax   : tcgen05.ld row -> mask -> running max / sum (base 2) -> P_j as bf16 into shared memory
+//     O[j & 1]  = P_j V_j            tcgen05.mma with the same value tile as an MN-major operand
+//     the row's output accumulates in registers: acc = acc * 2^(m_old - m_new) + O[j & 1]
+//   S and O are double-buffered in tensor memory, so the score product of tile j + 1 and the value product of
+//   tile j run while the softmax warps work; two thread blocks per SM (d_v = 64) fill each other's gaps.
+//   Every wait is bounded; on expiry the block records GVA_ERR_TIMEOUT, drains what it issued, frees its
+//   tensor memory and exits.
+#pragma once
+
+#include "gva_decode_mma.cuh"
+
+namespace gva {
+
+struct PrefillParams {
+    const float *q_abs;          // [n_q][H][d_v + d_r] absorbed content query, rotated positional query
+    const int32_t *cu_q;         // [B + 1] first query row of every sequence
+    const int32_t *ctx_lens;     // [B] tokens cached before the chunk
+    const int32_t *block_table;  // nullable
+    float *out;                  // [n_q][H][d_v]
+    float *lse;                  // [n_q][H], nullable
+    int32_t *dev_status;         // nullable
+    int B, H, G, P, num_pages, max_pages;
+    float scale_log2;            // softmax scale * log2(e)
+};
+
+template <int DV, int DR>
+struct PrefillTraits {
+    static constexpr int QTOK = 32;                              // query tokens per block
+    static constexpr int ROWS = QTOK * kHeadsPerGroup;           // 128 = MMA M
+    static constexpr int TILE = 64;                              // cached tokens per tile = MMA N of the score product
+    static constexpr int NSTAGE = 4;
+    static constexpr int BOXES = DV / 64;                        // 64-dim (128-byte) boxes per value row
+    static constexpr int QBOX_BYTES = ROWS * 128;
+    static constexpr int QV_BYTES = BOXES * QBOX_BYTES;
+    static constexpr int KR_ROW = DR * 2;                        // 32 or 64 bytes
+    static constexpr int QR_BYTES = (ROWS * KR_ROW + 1023) & ~1023;
+    static constexpr int P_BYTES = ROWS * 128;                   // [128 rows][64 tokens] bf16
+    static constexpr int VBOX_BYTES = TILE * 128;
+    static constexpr int V_BYTES = BOXES * VBOX_BYTES;
+    static constexpr int KR_BYTES = TILE * KR_ROW;
+    static constexpr int STAGE_BYTES = V_BYTES + ((KR_BYTES + 1023) & ~1023);
+    static constexpr int OFF_QV = 0;
+    static constexpr int OFF_QR = OFF_QV + QV_BYTES;
+    static constexpr int OFF_P = OFF_QR + QR_BYTES;
+    static constexpr int OFF_STAGE = OFF_P + P_BYTES;
+    static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
+    static constexpr int N_BARS = 2 * NSTAGE + 6;
+    static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
+    // tensor-memory columns: S0, S1 (64 each), O0, O1 (DV each)
+    static constexpr int COL_S = 0, COL_O = 2 * TILE;
+    static constexpr int TMEM_COLS = (2 * TILE + 2 * DV) <= 256 ? 256 : 512;
+    static constexpr int KSTEPS_V = DV / 16, KSTEPS_R = DR / 16;
+    static constexpr int THREADS = 192;
+};
+
+// ---- tcgen05 wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, f32 accumulate; issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The mbarrier receives one arrival when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+// 32 consecutive f32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor: start address, leading / stride byte offsets (16-byte units), descriptor
+// version 1 (bit 46), swizzle mode in bits 61-63 (2 = 128-byte, 4 = 64-byte, 6 = 32-byte).
+constexpr uint64_t kSwz128 = 2, kSwz64 = 4, kSwz32 = 6;
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint64_t swizzle) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | (swizzle << 61);
+}
+// Instruction descriptor of kind::f16: f32 accumulator (bits 4-5 = 1), bf16 A and B (bits 7-9, 10-12 = 1),
+// B major in bit 16 (0 = K-major, 1 = MN-major), N / 8 in bits 17-22, M / 16 in bits 24-28.
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+template <int DV, int DR>
+__global__ void __launch_bounds__(192, DV == 64 ? 2 : 1)
+prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
+    using T = PrefillTraits<DV, DR>;
+    constexpr int NS = T::NSTAGE;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.z, g = blockIdx.y;
+    const int qb = gridDim.x - 1 - blockIdx.x;        // the longest rows (last query blocks) are scheduled first
+    grid_dependency_wait();
+    const int q_begin = p.cu_q[b];
+    const int n_q = p.cu_q[b + 1] - q_begin;
+    const int q0 = qb * T::QTOK;
+    if (q0 >= n_q) return;
+    const int ctx = p.ctx_lens[b];
+    const long long kv_total = (long long)ctx + n_q;   // tokens of this sequence in the cache (context + chunk)
+    if (ctx < 0 || kv_total > (long long)p.max_pages * p.P) {
+        if (tid == 0) report_error(p.dev_status, GVA_ERR_SEQ_LEN, b);
+        return;
+    }
+    const int nv = min(T::QTOK, n_q - q0);             // live query tokens of this block
+    const int p0 = ctx + q0;                           // position of the block's first query token
+    const int n_tiles = (p0 + nv - 1) / T::TILE + 1;   // tiles 0..n_tiles-1 hold every visible token
+
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t s_base = smem_u32(smem);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + T::OFF_BAR);
+    const uint32_t bar0 = s_base + T::OFF_BAR;
+    auto kv_full = [&](int s) { return bar0 + 8u * s; };
+    auto kv_empty = [&](int s) { return bar0 + 8u * (NS + s); };
+    auto s_full = [&](int i) { return bar0 + 8u * (2 * NS + i); };
+    const uint32_t p_full = bar0 + 8u * (2 * NS + 2), q_ready = bar0 + 8u * (2 * NS + 3), drain = bar0 + 8u * (2 * NS + 4);
+    const uint32_t o_full = bar0 + 8u * (2 * NS + 5);   // one barrier for both O buffers: value products complete in order
+    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + T::N_BARS);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(kv_full(s), 1);
+            mbar_init(kv_empty(s), 1);
+        }
+        mbar_init(s_full(0), 1);
+        mbar_init(s_full(1), 1);
+        mbar_init(p_full, T::ROWS);
+        mbar_init(q_ready, T::ROWS);
+        mbar_init(drain, 1);
+        mbar_init(o_full, 1);
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32(s_tmem), T::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *s_tmem;
+
+    if (warp < 4) {
+        // ====================================== softmax: one row per thread ======================================
+        const int r = tid;
+        const int tok = r >> 2, hl = r & 3;
+        const int h = g * kHeadsPerGroup + hl;
+        const bool live = tok < nv;
+        const int pos = p0 + tok;
+        // ---- stage Q: f32 -> bf16, swizzled K-major rows (value dims in 128-byte boxes, then the RoPE dims) ----
+        {
+            const float4 *src = reinterpret_cast<const float4 *>(p.q_abs + ((size_t)(q_begin + q0 + tok) * p.H + h) * (DV + DR));
+#pragma unroll
+            for (int c = 0; c < DV / 8; ++c) {
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
+                if (live) {
+                    a = __ldg(src + 2 * c);
+                    bq = __ldg(src + 2 * c + 1);
+                }
+                uint4 w;
+                w.x = pack_bf16(a.x, a.y);
+                w.y = pack_bf16(a.z, a.w);
+                w.z = pack_bf16(bq.x, bq.y);
+                w.w = pack_bf16(bq.z, bq.w);
+                *reinterpret_cast<uint4 *>(smem + T::OFF_QV + (c >> 3) * T::QBOX_BYTES + swz128(r, c & 7)) = w;
+            }
+#pragma unroll
+            for (int c = 0; c < DR / 8; ++c) {
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
+                if (live) {
+                    a = __ldg(src + DV / 4 + 2 * c);
+                    bq = __ldg(src + DV / 4 + 2 * c + 1);
+                }
+                uint4 w;
+                w.x = pack_bf16(a.x, a.y);
+                w.y = pack_bf16(a.z, a.w);
+                w.z = pack_bf16(bq.x, bq.y);
+                w.w = pack_bf16(bq.z, bq.w);
+                *reinterpret_cast<uint4 *>(smem + T::OFF_QR + swz_kr<T::KR_ROW>(r, c)) = w;
+            }
+            fence_async_smem();
+            mbar_arrive(q_ready);
+        }
+
+        float acc[DV];
+#pragma unroll
+        for (int i = 0; i < DV; ++i) acc[i] = 0.f;
+        float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        bool ok = true;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            if (!mbar_wait_bounded(s_full(j & 1), (j >> 1) & 1, s_abort)) { ok = false; break; }
+            tc_fence_after();
+            uint32_t pk[T::TILE / 2];
+            float alpha;
+            {
+                float s[T::TILE];
+                {
+                    float t0[32], t1[32];
+                    tmem_ld32(lane_base + T::COL_S + (j & 1) * T::TILE, t0);
+                    tmem_ld32(lane_base + T::COL_S + (j & 1) * T::TILE + 32, t1);
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) { s[c] = t0[c]; s[32 + c] = t1[c]; }
+                }
+                const int limit = pos - j * T::TILE;          // columns c > limit are in the future of this row
+                if (limit < T::TILE - 1) {
+#pragma unroll
+                    for (int c = 0; c < T::TILE; ++c) s[c] = (c > limit) ? -INFINITY : s[c];
+                }
+                float mx = s[0];
+#pragma unroll
+                for (int c = 1; c < T::TILE; ++c) mx = fmaxf(mx, s[c]);
+                const float m_new = fmaxf(m_run, mx * p.scale_log2);
+                // m_new is finite from tile 0 on: token 0 is visible to every row
+                alpha = fast_exp2(m_run - m_new);
+                float sum = 0.f;
+#pragma unroll
+                for (int c = 0; c < T::TILE; c += 2) {
+                    const float e0 = fast_exp2(fmaf(s[c], p.scale_log2, -m_new));
+                    const float e1 = fast_exp2(fmaf(s[c + 1], p.scale_log2, -m_new));
+                    sum += e0 + e1;
+                    pk[c >> 1] = pack_bf16(e0, e1);
+                }
+                l_run = l_run * alpha + sum;
+                m_run = m_new;
+            }
+            // the previous value product has read P and written O[(j-1) & 1]
+            if (j > 0 && !mbar_wait_bounded(o_full, (j - 1) & 1, s_abort)) { ok = false; break; }
+            // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
+            if ((long long)(j + 1) * T::TILE > kv_total && r < T::TILE && (long long)j * T::TILE + r >= kv_total) {
+                unsigned char *vrow = smem + T::OFF_STAGE + (j % NS) * T::STAGE_BYTES;
+#pragma unroll
+                for (int bx = 0; bx < T::BOXES; ++bx)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4 *>(vrow + bx * T::VBOX_BYTES + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<uint4 *>(smem + T::OFF_P + swz128(r, c)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive(p_full);
+            if (j > 0) {
+                tc_fence_after();
+#pragma unroll
+                for (int part = 0; part < DV / 32; ++part) {
+                    float o[32];
+                    tmem_ld32(lane_base + T::COL_O + ((j - 1) & 1) * DV + part * 32, o);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[part * 32 + i] = fmaf(acc[part * 32 + i], alpha_prev, o[i]);
+                }
+            }
+            alpha_prev = alpha;
+        }
+        if (ok && !mbar_wait_bounded(o_full, (n_tiles - 1) & 1, s_abort)) ok = false;
+        if (ok) {
+            tc_fence_after();
+            const float inv = 1.f / l_run;
+            float *dst = p.out + ((size_t)(q_begin + q0 + tok) * p.H + h) * DV;
+#pragma unroll
+            for (int part = 0; part < DV / 32; ++part) {
+                float o[32];
+                tmem_ld32(lane_base + T::COL_O + ((n_tiles - 1) & 1) * DV + part * 32, o);
+                if (live) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        float4 v;
+                        v.x = fmaf(acc[part * 32 + i], alpha_prev, o[i]) * inv;
+                        v.y = fmaf(acc[part * 32 + i + 1], alpha_prev, o[i + 1]) * inv;
+                        v.z = fmaf(acc[part * 32 + i + 2], alpha_prev, o[i + 2]) * inv;
+                        v.w = fmaf(acc[part * 32 + i + 3], alpha_prev, o[i + 3]) * inv;
+                        *reinterpret_cast<float4 *>(dst + part * 32 + i) = v;
+                    }
+                }
+            }
+            if (live && p.lse) p.lse[(size_t)(q_begin + q0 + tok) * p.H + h] = (m_run + log2f(l_run)) * kLn2;
+        } else if (!*s_abort) {
+            report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+            *s_abort = 1;
+        }
+        tc_fence_before();
+    } else if (warp == 4) {
+        // ====================================== producer (one lane) ======================================
+        if (lane == 0) {
+            int issued = 0;
+            for (int j = 0; j < n_tiles; ++j) {
+                const int st = j % NS;
+                const int t0 = j * T::TILE;
+                const int pj = t0 / p.P, slot0 = t0 % p.P;
+                const long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
+                                                     : (long long)b * p.max_pages + pj;
+                if (page < 0 || page >= p.num_pages) {
+                    report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
+                    *s_abort = 1;
+                    break;
+                }
+                if (j >= NS && !mbar_wait_bounded(kv_empty(st), ((j / NS) & 1) ^ 1, s_abort)) {
+                    if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+                    *s_abort = 1;
+                    break;
+                }
+                const uint32_t dst = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
+                mbar_expect_tx(kv_full(st), T::V_BYTES + T::KR_BYTES);
+                const int row = (int)((page * p.G + g) * p.P + slot0);
+#pragma unroll
+                for (int bx = 0; bx < T::BOXES; ++bx) tma_load_2d(dst + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, kv_full(st));
+                tma_load_2d(dst + T::V_BYTES, &tm_k, 0, (int)(page * p.P + slot0), kv_full(st));
+                ++issued;
+            }
+            if (*s_abort) {   // copies still in flight must land before the block's shared memory is released
+                for (int j = max(0, issued - NS); j < issued; ++j)
+                    for (int it = 0; it < kDrainPolls && !mbar_try_wait(kv_full(j % NS), (j / NS) & 1); ++it) {}
+            }
+        }
+    } else {
+        // ====================================== MMA issuer (one lane) ======================================
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = umma_idesc(T::ROWS, T::TILE, false);
+            constexpr uint32_t idesc_o = umma_idesc(T::ROWS, DV, true);
+            constexpr uint64_t kr_swz = T::KR_ROW == 32 ? kSwz32 : kSwz64;
+            constexpr uint32_t kr_sbo = 8 * T::KR_ROW;
+            bool ok = mbar_wait_bounded(q_ready, 0, s_abort);
+            int issued_mma = 0;
+            for (int j = 0; j <= n_tiles && ok; ++j) {
+                if (j < n_tiles) {
+                    // score product of tile j; S[j & 1] was released when P of tile j-2 was complete (waited below)
+                    const int st = j % NS;
+                    if (!mbar_wait_bounded(kv_full(st), (j / NS) & 1, s_abort)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t vb = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
+                    const uint32_t d = tmem + T::COL_S + (j & 1) * T::TILE;
+#pragma unroll
+                    for (int ks = 0; ks < T::KSTEPS_V; ++ks) {
+                        const uint32_t off = (ks >> 2) * T::QBOX_BYTES + (ks & 3) * 32;
+                        const uint32_t voff = (ks >> 2) * T::VBOX_BYTES + (ks & 3) * 32;
+                        umma_bf16(d, smem_desc(s_base + T::OFF_QV + off, 16, 1024, kSwz128),
+                                  smem_desc(vb + voff, 16, 1024, kSwz128), idesc_s, ks > 0);
+                    }
+#pragma unroll
+                    for (int ks = 0; ks < T::KSTEPS_R; ++ks)
+                        umma_bf16(d, smem_desc(s_base + T::OFF_QR + ks * 32, 16, kr_sbo, kr_swz),
+                                  smem_desc(vb + T::V_BYTES + ks * 32, 16, kr_sbo, kr_swz), idesc_s, 1);
+                    umma_commit(s_full(j & 1));
+                    ++issued_mma;
+                }
+                if (j >= 1) {
+                    // value product of tile j-1: O[(j-1) & 1] = P V; all rows have stored P and have read O of tile j-3
+                    const int jj = j - 1, st = jj % NS;
+                    if (!mbar_wait_bounded(p_full, jj & 1, s_abort)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t vb = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
+                    const uint32_t d = tmem + T::COL_O + (jj & 1) * DV;
+#pragma unroll
+                    for (int ks = 0; ks < T::TILE / 16; ++ks)
+                        umma_bf16(d, smem_desc(s_base + T::OFF_P + ks * 32, 16, 1024, kSwz128),
+                                  smem_desc(vb + ks * 16 * 128, T::VBOX_BYTES, 1024, kSwz128), idesc_o, ks > 0);
+                    umma_commit(kv_empty(st));
+                    umma_commit(o_full);
+                    ++issued_mma;
+                }
+            }
+            if (!ok && !*s_abort) {
+                report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+                *s_abort = 1;
+            }
+            // nothing issued by this thread may still be running (or about to signal a barrier) when the block ends
+            if (issued_mma > 0) {
+                umma_commit(drain);
+                for (int it = 0; it < kDrainPolls * 16 && !mbar_try_wait(drain, 0); ++it) {}
+            }
+            tc_fence_before();
+        }
+    }
+    grid_dependency_launch();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        tmem_dealloc(tmem, T::TMEM_COLS);
+    }
+}
+
+// ---- host: support check, tensor maps, launch ---------------------------------------------------------
+inline bool prefill_supported(const gva_config &cfg) {
+    return cfg.cache_dtype == GVA_BF16 && cfg.page_size % 64 == 0 && cfg.H / cfg.G == kHeadsPerGroup &&
+           ((cfg.d_v == 64 && cfg.d_r == 16) || (cfg.d_v == 128 && cfg.d_r == 32));
+}
+
+template <int DV, int DR>
+int launch_prefill_t(const gva_config &cfg, const MmaHostState &st, int smem_optin, const PrefillParams &p, const void *v_pool,
+                     const void *kr_pool, int B, int max_q_len, cudaStream_t stream) {
+    using T = PrefillTraits<DV, DR>;
+    // request at least 80 KB so that no more than two blocks (2 x 256 tensor-memory columns) share an SM
+    const size_t smem = T::SMEM_BYTES < 80 * 1024 ? 80 * 1024 : T::SMEM_BYTES;
+    if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
+    auto fn = prefill_kernel<DV, DR>;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
+    CUtensorMap tm_v, tm_k;
+    if (!encode_map(st, &tm_v, v_pool, DV, (uint64_t)p.num_pages * cfg.G * p.P, 64, T::TILE, CU_TENSOR_MAP_SWIZZLE_128B))
+        return GVA_ERR_CUDA;
+    if (!encode_map(st, &tm_k, kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, T::TILE,
+                    DR == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B))
+        return GVA_ERR_CUDA;
+    const dim3 grid((max_q_len + T::QTOK - 1) / T::QTOK, cfg.G, B);
+    if (launch_pdl(fn, grid, dim3(T::THREADS), smem, stream, p, tm_v, tm_k) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GVA_ERR_CUDA;
+    }
+    return GVA_OK;
+}
+
+inline int launch_prefill(const gva_config &cfg, const MmaHostState &st, int smem_optin, const PrefillParams &p,
+                          const void *v_pool, const void *kr_pool, int B, int max_q_len, cudaStream_t stream) {
+    if (!prefill_supported(cfg)) return GVA_ERR_UNSUPPORTED;
+    if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
+    if (cfg.d_v == 64) return launch_prefill_t<64, 16>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, stream);
+    return launch_prefill_t<128, 32>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, stream);
+}
+
+}  // namespace gva

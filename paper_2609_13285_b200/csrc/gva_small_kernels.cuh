@@ -169,25 +169,25 @@ absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, cons
 constexpr int kAppendMaxPerThread = 8;    // G * d_v <= 8 * 128 elements (blocks have at least 128 threads)
 
 // One sequence's append.  Every thread of the block must call it (blockDim.x >= 128).
+// Writes input row `row` (v_new[row], kr_new[row]) as token `t` of sequence `seq`.
 template <typename CT>
-__device__ __forceinline__ void append_block(CT *__restrict__ v_pool, CT *__restrict__ kr_pool,
-                                             const int32_t *__restrict__ block_table, const float *__restrict__ v_new,
-                                             const float *__restrict__ kr_new, const int32_t *__restrict__ pos, int G,
-                                             int d_v, int d_r, int P, int num_pages, int max_pages, int32_t *dev_status,
-                                             const RopeTable &rope, int b) {
+__device__ __forceinline__ void append_row(CT *__restrict__ v_pool, CT *__restrict__ kr_pool,
+                                           const int32_t *__restrict__ block_table, const float *__restrict__ v_new,
+                                           const float *__restrict__ kr_new, int G, int d_v, int d_r, int P, int num_pages,
+                                           int max_pages, int32_t *dev_status, const RopeTable &rope, int row, int seq, int t) {
     const int n_v = G * d_v;
     const int nt = blockDim.x;
-    const int t = pos[b];
+    const int b = seq;
     float x[kAppendMaxPerThread];
 #pragma unroll
     for (int u = 0; u < kAppendMaxPerThread; ++u) {
         const int i = u * nt + threadIdx.x;
-        x[u] = (i < n_v) ? v_new[(size_t)b * n_v + i] : 0.f;
+        x[u] = (i < n_v) ? v_new[(size_t)row * n_v + i] : 0.f;
     }
     float k0 = 0.f, k1 = 0.f;
     if (threadIdx.x < d_r / 2) {
-        k0 = kr_new[(size_t)b * d_r + 2 * threadIdx.x];
-        k1 = kr_new[(size_t)b * d_r + 2 * threadIdx.x + 1];
+        k0 = kr_new[(size_t)row * d_r + 2 * threadIdx.x];
+        k1 = kr_new[(size_t)row * d_r + 2 * threadIdx.x + 1];
     }
     if (t < 0 || t / P >= max_pages) {
         if (threadIdx.x == 0) report_error(dev_status, GVA_ERR_SEQ_LEN, b);
@@ -226,6 +226,16 @@ __device__ __forceinline__ void append_block(CT *__restrict__ v_pool, CT *__rest
 }
 
 template <typename CT>
+__device__ __forceinline__ void append_block(CT *__restrict__ v_pool, CT *__restrict__ kr_pool,
+                                             const int32_t *__restrict__ block_table, const float *__restrict__ v_new,
+                                             const float *__restrict__ kr_new, const int32_t *__restrict__ pos, int G,
+                                             int d_v, int d_r, int P, int num_pages, int max_pages, int32_t *dev_status,
+                                             const RopeTable &rope, int b) {
+    append_row<CT>(v_pool, kr_pool, block_table, v_new, kr_new, G, d_v, d_r, P, num_pages, max_pages, dev_status, rope, b, b,
+                   pos[b]);
+}
+
+template <typename CT>
 __global__ void __launch_bounds__(128)
 append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *__restrict__ block_table,
               const float *__restrict__ v_new, const float *__restrict__ kr_new, const int32_t *__restrict__ pos,
@@ -234,6 +244,28 @@ append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *
     grid_dependency_wait();
     append_block<CT>(v_pool, kr_pool, block_table, v_new, kr_new, pos, G, d_v, d_r, P, num_pages, max_pages, dev_status,
                      rope, blockIdx.x);
+}
+
+// Append of a chunk of new tokens per sequence: block n writes input row n as token ctx_lens[b] + (n - cu_q[b]) of
+// the sequence b that owns the row (found by bisection of cu_q).
+template <typename CT>
+__global__ void __launch_bounds__(128)
+append_chunk_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *__restrict__ block_table,
+                    const float *__restrict__ v_new, const float *__restrict__ kr_new, const int32_t *__restrict__ cu_q,
+                    const int32_t *__restrict__ ctx_lens, int B, int G, int d_v, int d_r, int P, int num_pages, int max_pages,
+                    int32_t *dev_status, RopeTable rope) {
+    grid_dependency_launch();
+    grid_dependency_wait();
+    const int n = blockIdx.x;
+    if (n >= cu_q[B]) return;
+    int lo = 0, hi = B - 1;                     // largest b with cu_q[b] <= n (empty sequences repeat an offset)
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (cu_q[mid] <= n) lo = mid;
+        else hi = mid - 1;
+    }
+    append_row<CT>(v_pool, kr_pool, block_table, v_new, kr_new, G, d_v, d_r, P, num_pages, max_pages, dev_status, rope, n, lo,
+                   ctx_lens[lo] + (n - cu_q[lo]));
 }
 
 // ---- fused front of a decode step: absorb and append in one launch ------------------------------------

@@ -163,3 +163,61 @@ def upload_gqa(g: dict, device="cuda:0", kernel: int = gb.GVA_KERNEL_AUTO) -> Gq
                          out=torch.full((B, g["H"], d_h), float("nan"), dtype=torch.float32, device=dev),
                          lse=torch.full((B, g["H"]), float("nan"), dtype=torch.float32, device=dev),
                          status=torch.zeros(1, dtype=torch.int32, device=dev))
+
+
+@dataclass
+class PrefillDeviceCase:
+    """A workloads.PrefillCase on the device: the cache (through a DeviceCase) plus the chunk's per-token tensors."""
+    pc: object
+    dc: DeviceCase
+    cu_q: torch.Tensor
+    ctx_lens: torch.Tensor
+    q_c: torch.Tensor
+    q_r: torch.Tensor
+    q_pos: torch.Tensor
+    v_new: torch.Tensor
+    kr_new: torch.Tensor
+    q_abs: torch.Tensor
+    out: torch.Tensor
+    lse: torch.Tensor
+
+    @property
+    def handle(self) -> int:
+        return self.dc.handle
+
+    @property
+    def status(self) -> torch.Tensor:
+        return self.dc.status
+
+    @property
+    def max_q_len(self) -> int:
+        return int(self.pc.q_lens.max()) if len(self.pc.q_lens) else 0
+
+    def absorb(self) -> torch.Tensor:
+        gb.gva_absorb_query(self.handle, self.q_c, self.q_r, self.dc.M, self.q_pos, self.q_abs, self.pc.n_q)
+        return self.q_abs
+
+    def append(self) -> None:
+        gb.gva_append_chunk(self.handle, self.dc.cache, self.v_new, self.kr_new, self.cu_q, self.ctx_lens, self.pc.cache.B,
+                            self.pc.n_q, self.status)
+
+    def prefill(self, max_q_len: Optional[int] = None):
+        gb.gva_prefill(self.handle, self.dc.cache, self.q_abs, self.cu_q, self.ctx_lens, self.out, self.lse, self.pc.cache.B,
+                       self.max_q_len if max_q_len is None else max_q_len, self.status)
+        return self.out, self.lse
+
+    def close(self) -> None:
+        self.dc.close()
+
+
+def upload_prefill(pc, device="cuda:0") -> PrefillDeviceCase:
+    dev = torch.device(device)
+    dc = upload(pc.cache, device=device)
+    s = pc.cache.shape
+    n = pc.n_q
+    return PrefillDeviceCase(
+        pc=pc, dc=dc, cu_q=_dev(pc.cu_q, dev), ctx_lens=_dev(pc.ctx_lens, dev), q_c=_dev(pc.q_c, dev), q_r=_dev(pc.q_r, dev),
+        q_pos=_dev(pc.q_pos, dev), v_new=_dev(pc.v_new, dev), kr_new=_dev(pc.kr_new, dev),
+        q_abs=torch.empty((max(n, 1), s.H, s.d_v + s.d_r), dtype=torch.float32, device=dev),
+        out=torch.full((max(n, 1), s.H, s.d_v), float("nan"), dtype=torch.float32, device=dev),
+        lse=torch.full((max(n, 1), s.H), float("nan"), dtype=torch.float32, device=dev))

@@ -1,0 +1,178 @@
+"""GPU parity of the prefill / chunked-prefill path (gva_absorb_query -> gva_append_chunk -> gva_prefill, through the
+C ABI) against the fp64 oracle, which forms the keys explicitly (K_h = V_g M_h) and applies a plain causal softmax.
+
+Tolerance: the kernel feeds the tensor cores bf16 operands -- the absorbed query and the softmax weights are each
+rounded once to bf16 (relative error <= 2^-9), products are exact and accumulate in f32.  For unit-variance data a
+score moves by about sqrt(d_v) * 2^-9 / sqrt(3) * scale ~ 1e-3 and a weight by 2^-9 relative, so outputs move by a few
+1e-3 at most; the contract for a bf16 cache (max-abs <= 2e-2) is asserted, with rel-L2 <= 5e-3 as the tighter gate."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gva_oracle as orc
+from paper_2609_13285_b200 import binding as gb
+from paper_2609_13285_b200 import harness
+from paper_2609_13285_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL_MAXABS = 2e-2
+TOL_REL_L2 = 5e-3
+TOL_LSE = 2e-2
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from tests import gpu_util
+    gpu_util.ensure_built()
+
+
+def rel_l2(a, ref):
+    return float(np.linalg.norm((a - ref).ravel()) / max(np.linalg.norm(ref.ravel()), 1e-30))
+
+
+def run_prefill(pc, append=False):
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        if append:
+            pd.append()
+        out, lse = pd.prefill()
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0, f"device status {int(pd.status.item()):#x}"
+        n = pc.n_q
+        return out[:n].cpu().numpy().astype(np.float64), lse[:n].cpu().numpy().astype(np.float64), pd.dc.pools_to_host()
+    finally:
+        pd.close()
+
+
+def check(pc):
+    out, lse, _ = run_prefill(pc)
+    ref_out, ref_lse = orc.prefill_case(pc)
+    assert np.isfinite(out).all() and np.isfinite(lse).all()
+    err = float(np.max(np.abs(out - ref_out))) if out.size else 0.0
+    assert err <= TOL_MAXABS, f"max-abs {err:.3e}"
+    assert rel_l2(out, ref_out) <= TOL_REL_L2, f"rel-L2 {rel_l2(out, ref_out):.3e}"
+    assert np.max(np.abs(lse - ref_lse)) <= TOL_LSE
+    return err
+
+
+@pytest.mark.parametrize("ctx,q", [
+    ([0], [1]),                                   # one token sees itself
+    ([0], [64]),                                  # exactly one tile, two query blocks
+    ([0], [65]),                                  # ragged: one token into the second tile
+    ([0, 5, 100, 64, 0, 1000], [70, 33, 1, 128, 200, 37]),
+    ([0, 0, 7], [0, 300, 0]),                     # sequences without new tokens
+])
+def test_prefill_matches_oracle_shape_a(ctx, q):
+    pc = wl.make_prefill_case("pf", wl.SHAPE_A, ctx, q, page_size=64, seed=501, poison_unused=True)
+    check(pc)
+
+
+def test_prefill_matches_oracle_shape_b():
+    pc = wl.make_prefill_case("pfb", wl.SHAPE_B, [0, 130, 31], [150, 40, 97], page_size=64, seed=502, poison_unused=True)
+    check(pc)
+
+
+def test_prefill_contiguous_cache_and_large_pages():
+    pc = wl.make_prefill_case("pfc", wl.SHAPE_A, [10, 200], [190, 100], page_size=128, paged=False, seed=503)
+    check(pc)
+
+
+def test_prefill_row_equals_decode_kernel_row():
+    # the last row of a chunk is one decode step over the whole sequence: compare with gva_decode on the same cache
+    pc = wl.make_prefill_case("pfd", wl.SHAPE_A, [300, 0], [100, 257], page_size=64, seed=504)
+    out, lse, _ = run_prefill(pc)
+    ref_out, _ = orc.prefill_case(pc)
+    c = pc.cache
+    last = pc.cu_q[1:] - 1
+    c.q_c[:] = pc.q_c[last]; c.q_r[:] = pc.q_r[last]; c.q_pos[:] = pc.q_pos[last]
+    dc = harness.upload(c)
+    try:
+        dc.absorb()
+        o, _ = dc.decode()
+        torch.cuda.synchronize()
+        o = o.cpu().numpy().astype(np.float64)
+    finally:
+        dc.close()
+    assert np.max(np.abs(o - ref_out[last])) <= 2e-5            # the decode kernel keeps f32 operands
+    assert np.max(np.abs(o - out[last])) <= TOL_MAXABS
+
+
+def test_chunked_prefill_equals_whole_prefill():
+    whole = wl.make_prefill_case("w", wl.SHAPE_A, [0, 0], [333, 150], page_size=64, seed=505)
+    out_w, lse_w, _ = run_prefill(whole)
+    cut = np.array([100, 149])
+    part = wl.make_prefill_case("p", wl.SHAPE_A, cut, np.array([333, 150]) - cut, page_size=64, seed=505)
+    assert np.array_equal(part.cache.v_pool, whole.cache.v_pool)
+    rows = np.concatenate([np.arange(whole.cu_q[b] + cut[b], whole.cu_q[b + 1]) for b in range(2)])
+    part.q_c[:] = whole.q_c[rows]; part.q_r[:] = whole.q_r[rows]
+    out_p, lse_p, _ = run_prefill(part)
+    # same rows, same tiles, different row-to-block assignment: equal up to the bf16 rounding of the weights
+    assert np.max(np.abs(out_p - out_w[rows])) <= 5e-3
+    assert np.max(np.abs(lse_p - lse_w[rows])) <= 1e-3
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_append_chunk_is_bit_exact(dtype):
+    pc = wl.make_prefill_case("ap", wl.SHAPE_A, [0, 63, 64, 500], [130, 2, 0, 77], page_size=64, cache_dtype=dtype, seed=506)
+    c = pc.cache
+    v_ref, k_ref = c.v_pool.copy(), c.kr_pool.copy()
+    assert orc.append_chunk(v_ref, k_ref, c.block_table, pc.v_new, pc.kr_new, pc.cu_q, pc.ctx_lens) == 0
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.append()
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        v, k = pd.dc.pools_to_host()
+    finally:
+        pd.close()
+    assert np.array_equal(v.view(np.uint8), v_ref.view(np.uint8)) and np.array_equal(k.view(np.uint8), k_ref.view(np.uint8))
+
+
+def test_append_then_prefill_follows_algorithm_order():
+    # the chunk's own rows come from the append, not from the generator
+    pc = wl.make_prefill_case("apf", wl.SHAPE_A, [40, 0], [90, 129], page_size=64, seed=507)
+    c = pc.cache
+    out, lse, (v, k) = run_prefill(pc, append=True)
+    assert orc.append_chunk(c.v_pool, c.kr_pool, c.block_table, pc.v_new, pc.kr_new, pc.cu_q, pc.ctx_lens) == 0
+    assert np.array_equal(v, c.v_pool) and np.array_equal(k, c.kr_pool)
+    ref_out, ref_lse = orc.prefill_case(pc)
+    assert np.max(np.abs(out - ref_out)) <= TOL_MAXABS and rel_l2(out, ref_out) <= TOL_REL_L2
+
+
+def test_prefill_rejects_what_it_does_not_support():
+    for kw in (dict(cache_dtype=gb.GVA_F32), dict(d_r=24), dict(page_size=32)):
+        args = dict(H=16, G=4, d_v=64, d_c=64, d_r=16, page_size=64)
+        args.update(kw)
+        h = gb.gva_create(**args)
+        try:
+            t = torch.zeros(4096, dtype=torch.float32, device="cuda")
+            i = torch.zeros(16, dtype=torch.int32, device="cuda")
+            cache = gb.make_cache(t, t, None, 4, 4)
+            assert gb.gva_prefill(h, cache, t, i, i, t, None, 1, 8, check=False) == gb.GVA_ERR_UNSUPPORTED
+        finally:
+            gb.gva_destroy(h)
+
+
+def test_prefill_reports_bad_page_and_long_sequence():
+    pc = wl.make_prefill_case("bad", wl.SHAPE_A, [0, 0], [100, 40], page_size=64, seed=508)
+    pc.cache.block_table[0, 1] = pc.cache.num_pages + 5
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        pd.prefill()
+        torch.cuda.synchronize()
+        st = int(pd.status.item())
+        assert st & 0xff == gb.GVA_ERR_BAD_PAGE and st >> 8 == 0
+        out = pd.out.cpu().numpy()
+        ref, _ = orc.prefill_case(wl.make_prefill_case("bad", wl.SHAPE_A, [0, 0], [100, 40], page_size=64, seed=508))
+        assert np.max(np.abs(out[100:140] - ref[100:140])) <= TOL_MAXABS     # the other sequence is unaffected
+        pd.status.zero_()
+        pd.ctx_lens[1] = 10_000                                               # beyond its block table
+        pd.prefill()
+        torch.cuda.synchronize()
+        st = int(pd.status.item())
+        assert st & 0xff == gb.GVA_ERR_SEQ_LEN and st >> 8 == 1
+    finally:
+        pd.close()
