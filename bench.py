@@ -8,7 +8,7 @@ d_r=16, T=32768, bf16 cache in 64-token pages behind a permuted block table).  T
 GB/s: the live cache bytes one step must stream, divided by the step time.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-                    [--workload cfg1|cfg2|cfg3|cfg4] [--kernel auto|fma|mma] [--headline-only]
+                    [--workload cfg1|cfg2|cfg3|cfg4|prefill|layer] [--kernel auto|fma|mma] [--headline-only]
 
 N > 1 runs N independent replicas (one process per GPU under torch.distributed.run): the path has no
 exchange step, so there is no collective on the data path; only the timing barrier and the
@@ -444,6 +444,70 @@ def measure_layer(rank, local_rank, dist, args, kernel, torch, gb, harness):
     return res
 
 
+def load_tensor_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["bf16_tflops"]), "measured (MEASURED_PEAKS.json bf16_tflops, cuBLAS bf16 burst)"
+    return 1590.0, "fallback (1.59 PFLOP/s, earlier measurement on this pool)"
+
+
+def measure_prefill(rank, local_rank, dist, args, torch, gb, harness, B=8, T=8192):
+    """Whole-prompt prefill on the headline head shape: gva_absorb_query + gva_append_chunk + gva_prefill, and the
+    attention kernel alone against the tensor roofline (flops of the absorbed form under the causal mask)."""
+    from paper_2609_13285_b200 import multirank, workloads as wl
+    dev = torch.device("cuda", local_rank)
+    pc = wl.prefill_bench_case(seed=wl.MASTER_SEED + 7100 + 7919 * rank, B=B, T=T)
+    pd = harness.upload_prefill(pc, device=dev)
+    stream = torch.cuda.current_stream()
+    steps, warmup = max(5, min(30, args.steps // 10)), 3
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)     # larger than L2: written between timed kernels
+
+    def attention(i):
+        pd.prefill()
+
+    def whole(i):
+        pd.absorb()
+        pd.append()
+        pd.prefill()
+
+    def timed(fn):
+        for i in range(warmup):
+            fn(i)
+        multirank.barrier(dist)
+        torch.cuda.synchronize()
+        total = 0.0
+        for i in range(steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn(i)
+            b.record(stream)
+            torch.cuda.synchronize()
+            total += a.elapsed_time(b)
+        return total / steps
+
+    pd.absorb()
+    attn_ms = timed(attention)
+    whole_ms = timed(whole)
+    status = int(pd.status.item())
+    peak, src = load_tensor_peak()
+    flops = pc.flops()
+    tf = flops / (attn_ms * 1e-3) / 1e12
+    res = {"workload": f"whole-prompt prefill, H=16 G=4 d_v=64 d_c=64 d_r=16, B={B} prompts of T={T} tokens, bf16 cache in "
+                       "64-token pages (permuted block table), L2 flushed between timed calls",
+           "prefill_tokens_per_s": B * T / (whole_ms * 1e-3), "ms_per_step": whole_ms,
+           "gva_prefill_ms_per_call": attn_ms, "steps": steps, "device_status": status,
+           "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                        "traffic": None, "peak_source": src, "kernel": "prefill_kernel<64,16> (tcgen05 score and value products)",
+                        "algorithmic_flops_per_launch": flops, "avg_launch_ms": attn_ms,
+                        "note": "flops = 2 * causal pairs * H * (2 d_v + d_r); bf16 operands, f32 accumulate"}}
+    pd.close()
+    del flush
+    torch.cuda.empty_cache()
+    return res
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -480,6 +544,18 @@ def main() -> None:
     kernel = {"auto": gb.GVA_KERNEL_AUTO, "fma": gb.GVA_KERNEL_FMA, "mma": gb.GVA_KERNEL_MMA}[args.kernel]
 
     name = args.workload
+    if name in ("prefill", "prefill-ncu", "layer"):      # side workloads on their own (small runs for profiler captures)
+        if rank == 0:
+            if name == "layer":
+                res = measure_layer(rank, local_rank, None, args, kernel, torch, gb, harness)
+            else:
+                res = measure_prefill(rank, local_rank, None, args, torch, gb, harness,
+                                      **({"B": 4, "T": 4096} if name == "prefill-ncu" else {}))
+            print(json.dumps({"workload": name, **res}))
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
     r = measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with_e2e=True, with_clocks=True)
     (step_ms, e2e_ms, decode_ms), job_bytes = multirank.reduce_times_and_work(
         [r["step_ms"], r["e2e_ms"], r["decode_ms"]], r["cache_bytes"], dist, dev)
@@ -509,6 +585,7 @@ def main() -> None:
         gq["gva_over_gqa_decode_time"] = decode_ms / gq["gqa_decode_ms_per_call"]
         others["gqa_matched_cfg2"] = gq
         others["layer_step_cfg2"] = measure_layer(rank, local_rank, dist, short, kernel, torch, gb, harness)
+        others["prefill"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness)
 
     if rank == 0:
         case = r["case"]

@@ -11,16 +11,19 @@
 //
 // Layout of the work
 //   thread block   = 32 query tokens x 4 heads of one (sequence, value group): 128 rows = one M = 128 MMA tile
-//   warps 0-3      = softmax: thread r owns row r (token r / 4, head r % 4) -- tensor-memory lane r
-//   warp 4         = producer (one lane): TMA loads of the 64-token value tile and positional-key tile into a ring
-//   warp 5         = MMA issuer (one lane) and owner of the tensor-memory allocation
+//   warps 0-7      = softmax: row r (token r / 4, head r % 4) = tensor-memory lane r is shared by two threads, one in
+//                    warp w and one in warp w + 4 (both reach lanes 32 (w % 4) ..); each owns half of the tile's score
+//                    columns and half of the output dims, and reads the other half of the scores only for the row maximum
+//   warp 8         = producer (one lane): TMA loads of the 64-token value tile and positional-key tile into a ring
+//   warp 9         = MMA issuer (one lane) and owner of the tensor-memory allocation
 //   per 64-token tile j:
 //     S[j & 1]  = Q K_j^T            tcgen05.mma, K = d_v (value dims, 128-byte swizzle) + d_r (RoPE dims)
-//     softmax   : tcgen05.ld row -> mask -> running max / sum (base 2) -> P_j as bf16 into shared memory
-//     O[j & 1]  = P_j V_j            tcgen05.mma with the same value tile as an MN-major operand
-//     the row's output accumulates in registers: acc = acc * 2^(m_old - m_new) + O[j & 1]
-//   S and O are double-buffered in tensor memory, so the score product of tile j + 1 and the value product of
-//   tile j run while the softmax warps work; two thread blocks per SM (d_v = 64) fill each other's gaps.
+//     softmax   : tcgen05.ld row -> mask -> running max / sum (base 2) -> P_j as bf16 pairs into tensor memory
+//     O         = P_j V_j            tcgen05.mma, A = P from tensor memory, B = the same value tile as an MN-major operand
+//     the row's output accumulates in registers: acc = acc * 2^(m_old - m_new) + O
+//   S is double-buffered in tensor memory, so the score product of tile j + 1 runs while the softmax warps work on
+//   tile j; two thread blocks per SM (d_v = 64) fill each other's gaps.  Shared memory carries only the operands
+//   the tensor core reads (Q and the cache tiles): P never touches it.
 //   Every wait is bounded; on expiry the block records GVA_ERR_TIMEOUT, drains what it issued, frees its
 //   tensor memory and exits.
 #pragma once
@@ -52,23 +55,21 @@ struct PrefillTraits {
     static constexpr int QV_BYTES = BOXES * QBOX_BYTES;
     static constexpr int KR_ROW = DR * 2;                        // 32 or 64 bytes
     static constexpr int QR_BYTES = (ROWS * KR_ROW + 1023) & ~1023;
-    static constexpr int P_BYTES = ROWS * 128;                   // [128 rows][64 tokens] bf16
     static constexpr int VBOX_BYTES = TILE * 128;
     static constexpr int V_BYTES = BOXES * VBOX_BYTES;
     static constexpr int KR_BYTES = TILE * KR_ROW;
     static constexpr int STAGE_BYTES = V_BYTES + ((KR_BYTES + 1023) & ~1023);
     static constexpr int OFF_QV = 0;
     static constexpr int OFF_QR = OFF_QV + QV_BYTES;
-    static constexpr int OFF_P = OFF_QR + QR_BYTES;
-    static constexpr int OFF_STAGE = OFF_P + P_BYTES;
+    static constexpr int OFF_STAGE = OFF_QR + QR_BYTES;
     static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
     static constexpr int N_BARS = 2 * NSTAGE + 6;
-    static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
-    // tensor-memory columns: S0, S1 (64 each), O0, O1 (DV each)
-    static constexpr int COL_S = 0, COL_O = 2 * TILE;
-    static constexpr int TMEM_COLS = (2 * TILE + 2 * DV) <= 256 ? 256 : 512;
+    static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16 + 2 * ROWS * 4;
+    // tensor-memory columns: S0, S1 (64 each), O (DV), P (TILE / 2: bf16 pairs)
+    static constexpr int COL_S = 0, COL_O = 2 * TILE, COL_P = COL_O + DV;
+    static constexpr int TMEM_COLS = (COL_P + TILE / 2) <= 256 ? 256 : 512;
     static constexpr int KSTEPS_V = DV / 16, KSTEPS_R = DR / 16;
-    static constexpr int THREADS = 192;
+    static constexpr int THREADS = 320;
 };
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------------------------
@@ -91,6 +92,22 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Same with A read from tensor memory (rows = lanes, two bf16 per 32-bit column, K-major).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 16 consecutive 32-bit columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n" ::"r"(taddr),
+        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+        "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
+}
 // The mbarrier receives one arrival when every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
@@ -112,6 +129,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, float (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+        : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]), "=f"(v[9]),
+          "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15]), "=f"(v[16]), "=f"(v[17]), "=f"(v[18]),
+          "=f"(v[19]), "=f"(v[20]), "=f"(v[21]), "=f"(v[22]), "=f"(v[23]), "=f"(v[24]), "=f"(v[25]), "=f"(v[26]), "=f"(v[27]),
+          "=f"(v[28]), "=f"(v[29]), "=f"(v[30]), "=f"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+
 // Shared-memory matrix descriptor: start address, leading / stride byte offsets (16-byte units), descriptor
 // version 1 (bit 46), swizzle mode in bits 61-63 (2 = 128-byte, 4 = 64-byte, 6 = 32-byte).
 constexpr uint64_t kSwz128 = 2, kSwz64 = 4, kSwz32 = 6;
@@ -132,7 +162,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 template <int DV, int DR>
-__global__ void __launch_bounds__(192, DV == 64 ? 2 : 1)
+__global__ void __launch_bounds__(320, DV == 64 ? 2 : 1)
 prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = PrefillTraits<DV, DR>;
     constexpr int NS = T::NSTAGE;
@@ -166,6 +196,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     const uint32_t o_full = bar0 + 8u * (2 * NS + 5);   // one barrier for both O buffers: value products complete in order
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + T::N_BARS);
     volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
+    float *s_lsum = reinterpret_cast<float *>(s_tmem + 4);        // [2][ROWS] per-half row sums, exchanged once at the end
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
@@ -174,8 +205,8 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         }
         mbar_init(s_full(0), 1);
         mbar_init(s_full(1), 1);
-        mbar_init(p_full, T::ROWS);
-        mbar_init(q_ready, T::ROWS);
+        mbar_init(p_full, 2 * T::ROWS);
+        mbar_init(q_ready, 2 * T::ROWS);
         mbar_init(drain, 1);
         mbar_init(o_full, 1);
         *s_abort = 0;
@@ -183,7 +214,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
     }
-    if (warp == 5) {
+    if (warp == 9) {
         tmem_alloc(smem_u32(s_tmem), T::TMEM_COLS);
         tmem_relinquish();
     }
@@ -192,146 +223,150 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     tc_fence_after();
     const uint32_t tmem = *s_tmem;
 
-    if (warp < 4) {
-        // ====================================== softmax: one row per thread ======================================
-        const int r = tid;
-        const int tok = r >> 2, hl = r & 3;
-        const int h = g * kHeadsPerGroup + hl;
-        const bool live = tok < nv;
-        const int pos = p0 + tok;
+    // softmax threads (warps 0-7): two per row, each owns half of the tile's score columns and of the output dims
+    const int half = (warp >> 2) & 1;                  // warps w and w + 4 reach the same tensor-memory lanes (32 (w % 4) ..)
+    const int r = (warp & 3) * 32 + lane;
+    const int tok = r >> 2, hl = r & 3;
+    const int h = g * kHeadsPerGroup + hl;
+    const bool live = tok < nv;
+    const int pos = p0 + tok;
+    constexpr int HC = T::TILE / 2;                    // score columns per thread
+    constexpr int HD = DV / 2;                         // output dims per thread
+    float acc[HD];
+    float m_run = -INFINITY;
+
+    if (warp < 8) {
+        // ============================================== softmax ==============================================
         // ---- stage Q: f32 -> bf16, swizzled K-major rows (value dims in 128-byte boxes, then the RoPE dims) ----
         {
             const float4 *src = reinterpret_cast<const float4 *>(p.q_abs + ((size_t)(q_begin + q0 + tok) * p.H + h) * (DV + DR));
 #pragma unroll
-            for (int c = 0; c < DV / 8; ++c) {
+            for (int cc = 0; cc < DV / 16; ++cc) {
+                const int c = half * (DV / 16) + cc;
                 float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
                 if (live) {
                     a = __ldg(src + 2 * c);
                     bq = __ldg(src + 2 * c + 1);
                 }
-                uint4 w;
-                w.x = pack_bf16(a.x, a.y);
-                w.y = pack_bf16(a.z, a.w);
-                w.z = pack_bf16(bq.x, bq.y);
-                w.w = pack_bf16(bq.z, bq.w);
-                *reinterpret_cast<uint4 *>(smem + T::OFF_QV + (c >> 3) * T::QBOX_BYTES + swz128(r, c & 7)) = w;
+                *reinterpret_cast<uint4 *>(smem + T::OFF_QV + (c >> 3) * T::QBOX_BYTES + swz128(r, c & 7)) =
+                    make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(bq.x, bq.y), pack_bf16(bq.z, bq.w));
             }
 #pragma unroll
-            for (int c = 0; c < DR / 8; ++c) {
+            for (int cc = 0; cc < DR / 16; ++cc) {
+                const int c = half * (DR / 16) + cc;
                 float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
                 if (live) {
                     a = __ldg(src + DV / 4 + 2 * c);
                     bq = __ldg(src + DV / 4 + 2 * c + 1);
                 }
-                uint4 w;
-                w.x = pack_bf16(a.x, a.y);
-                w.y = pack_bf16(a.z, a.w);
-                w.z = pack_bf16(bq.x, bq.y);
-                w.w = pack_bf16(bq.z, bq.w);
-                *reinterpret_cast<uint4 *>(smem + T::OFF_QR + swz_kr<T::KR_ROW>(r, c)) = w;
+                *reinterpret_cast<uint4 *>(smem + T::OFF_QR + swz_kr<T::KR_ROW>(r, c)) =
+                    make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(bq.x, bq.y), pack_bf16(bq.z, bq.w));
             }
             fence_async_smem();
             mbar_arrive(q_ready);
         }
 
-        float acc[DV];
 #pragma unroll
-        for (int i = 0; i < DV; ++i) acc[i] = 0.f;
-        float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        for (int i = 0; i < HD; ++i) acc[i] = 0.f;
+        float l_run = 0.f, alpha_prev = 0.f;           // l_run: sum over this thread's columns only
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
             if (!mbar_wait_bounded(s_full(j & 1), (j >> 1) & 1, s_abort)) { ok = false; break; }
             tc_fence_after();
-            uint32_t pk[T::TILE / 2];
+            uint32_t pk[HC / 2];
             float alpha;
             {
-                float s[T::TILE];
-                {
-                    float t0[32], t1[32];
-                    tmem_ld32(lane_base + T::COL_S + (j & 1) * T::TILE, t0);
-                    tmem_ld32(lane_base + T::COL_S + (j & 1) * T::TILE + 32, t1);
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) { s[c] = t0[c]; s[32 + c] = t1[c]; }
-                }
+                // the row maximum needs all 64 columns: read the partner's half too (no exchange between threads)
                 const int limit = pos - j * T::TILE;          // columns c > limit are in the future of this row
-                if (limit < T::TILE - 1) {
+                const bool diag = limit < T::TILE - 1;
+                float mx[4];
+                {
+                    float u[HC];
+                    tmem_ld32_nowait(lane_base + T::COL_S + (j & 1) * T::TILE + (half ^ 1) * HC, u);
+                    tmem_ld_wait();
+                    if (diag) {
 #pragma unroll
-                    for (int c = 0; c < T::TILE; ++c) s[c] = (c > limit) ? -INFINITY : s[c];
+                        for (int c = 0; c < HC; ++c) u[c] = ((half ^ 1) * HC + c > limit) ? -INFINITY : u[c];
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) mx[k] = fmaxf(u[k], u[k + 4]);
+#pragma unroll
+                    for (int c = 8; c < HC; c += 4)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) mx[k] = fmaxf(mx[k], u[c + k]);
                 }
-                float mx = s[0];
+                float s[HC];
+                tmem_ld32_nowait(lane_base + T::COL_S + (j & 1) * T::TILE + half * HC, s);
+                tmem_ld_wait();
+                if (diag) {
 #pragma unroll
-                for (int c = 1; c < T::TILE; ++c) mx = fmaxf(mx, s[c]);
-                const float m_new = fmaxf(m_run, mx * p.scale_log2);
+                    for (int c = 0; c < HC; ++c) s[c] = (half * HC + c > limit) ? -INFINITY : s[c];
+                }
+#pragma unroll
+                for (int c = 0; c < HC; c += 4)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) mx[k] = fmaxf(mx[k], s[c + k]);
+                const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2);
                 // m_new is finite from tile 0 on: token 0 is visible to every row
                 alpha = fast_exp2(m_run - m_new);
-                float sum = 0.f;
+                float sum[2] = {0.f, 0.f};
 #pragma unroll
-                for (int c = 0; c < T::TILE; c += 2) {
+                for (int c = 0; c < HC; c += 2) {
                     const float e0 = fast_exp2(fmaf(s[c], p.scale_log2, -m_new));
                     const float e1 = fast_exp2(fmaf(s[c + 1], p.scale_log2, -m_new));
-                    sum += e0 + e1;
+                    sum[0] += e0;
+                    sum[1] += e1;
                     pk[c >> 1] = pack_bf16(e0, e1);
                 }
-                l_run = l_run * alpha + sum;
+                l_run = l_run * alpha + (sum[0] + sum[1]);
                 m_run = m_new;
             }
-            // the previous value product has read P and written O[(j-1) & 1]
-            if (j > 0 && !mbar_wait_bounded(o_full, (j - 1) & 1, s_abort)) { ok = false; break; }
-            // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
-            if ((long long)(j + 1) * T::TILE > kv_total && r < T::TILE && (long long)j * T::TILE + r >= kv_total) {
-                unsigned char *vrow = smem + T::OFF_STAGE + (j % NS) * T::STAGE_BYTES;
-#pragma unroll
-                for (int bx = 0; bx < T::BOXES; ++bx)
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4 *>(vrow + bx * T::VBOX_BYTES + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
-            }
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<uint4 *>(smem + T::OFF_P + swz128(r, c)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-            fence_async_smem();
-            tc_fence_before();
-            mbar_arrive(p_full);
+            // the previous value product has read P and written O
             if (j > 0) {
+                if (!mbar_wait_bounded(o_full, (j - 1) & 1, s_abort)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
-                for (int part = 0; part < DV / 32; ++part) {
+                for (int part = 0; part < HD / 32; ++part) {
                     float o[32];
-                    tmem_ld32(lane_base + T::COL_O + ((j - 1) & 1) * DV + part * 32, o);
+                    tmem_ld32(lane_base + T::COL_O + half * HD + part * 32, o);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) acc[part * 32 + i] = fmaf(acc[part * 32 + i], alpha_prev, o[i]);
                 }
             }
+            // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
+            if ((long long)(j + 1) * T::TILE > kv_total) {
+                if (tid < T::TILE && (long long)j * T::TILE + tid >= kv_total) {
+                    unsigned char *vrow = smem + T::OFF_STAGE + (j % NS) * T::STAGE_BYTES;
+#pragma unroll
+                    for (int bx = 0; bx < T::BOXES; ++bx)
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4 *>(vrow + bx * T::VBOX_BYTES + tid * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+                }
+                fence_async_smem();
+            }
+            tmem_st16(lane_base + T::COL_P + half * (HC / 2), pk);
+            tc_fence_before();
+            mbar_arrive(p_full);
             alpha_prev = alpha;
         }
         if (ok && !mbar_wait_bounded(o_full, (n_tiles - 1) & 1, s_abort)) ok = false;
         if (ok) {
             tc_fence_after();
-            const float inv = 1.f / l_run;
-            float *dst = p.out + ((size_t)(q_begin + q0 + tok) * p.H + h) * DV;
 #pragma unroll
-            for (int part = 0; part < DV / 32; ++part) {
+            for (int part = 0; part < HD / 32; ++part) {
                 float o[32];
-                tmem_ld32(lane_base + T::COL_O + ((n_tiles - 1) & 1) * DV + part * 32, o);
-                if (live) {
+                tmem_ld32(lane_base + T::COL_O + half * HD + part * 32, o);
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        float4 v;
-                        v.x = fmaf(acc[part * 32 + i], alpha_prev, o[i]) * inv;
-                        v.y = fmaf(acc[part * 32 + i + 1], alpha_prev, o[i + 1]) * inv;
-                        v.z = fmaf(acc[part * 32 + i + 2], alpha_prev, o[i + 2]) * inv;
-                        v.w = fmaf(acc[part * 32 + i + 3], alpha_prev, o[i + 3]) * inv;
-                        *reinterpret_cast<float4 *>(dst + part * 32 + i) = v;
-                    }
-                }
+                for (int i = 0; i < 32; ++i) acc[part * 32 + i] = fmaf(acc[part * 32 + i], alpha_prev, o[i]);
             }
-            if (live && p.lse) p.lse[(size_t)(q_begin + q0 + tok) * p.H + h] = (m_run + log2f(l_run)) * kLn2;
+            s_lsum[half * T::ROWS + r] = l_run;
         } else if (!*s_abort) {
             report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
             *s_abort = 1;
         }
         tc_fence_before();
-    } else if (warp == 4) {
+    } else if (warp == 8) {
         // ====================================== producer (one lane) ======================================
         if (lane == 0) {
             int issued = 0;
@@ -396,16 +431,16 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                     ++issued_mma;
                 }
                 if (j >= 1) {
-                    // value product of tile j-1: O[(j-1) & 1] = P V; all rows have stored P and have read O of tile j-3
+                    // value product of tile j-1: O = P V; all rows have stored P and have read O of tile j-2
                     const int jj = j - 1, st = jj % NS;
                     if (!mbar_wait_bounded(p_full, jj & 1, s_abort)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t vb = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
-                    const uint32_t d = tmem + T::COL_O + (jj & 1) * DV;
+                    const uint32_t d = tmem + T::COL_O;
 #pragma unroll
                     for (int ks = 0; ks < T::TILE / 16; ++ks)
-                        umma_bf16(d, smem_desc(s_base + T::OFF_P + ks * 32, 16, 1024, kSwz128),
-                                  smem_desc(vb + ks * 16 * 128, T::VBOX_BYTES, 1024, kSwz128), idesc_o, ks > 0);
+                        umma_bf16_ts(d, tmem + T::COL_P + ks * 8, smem_desc(vb + ks * 16 * 128, T::VBOX_BYTES, 1024, kSwz128),
+                                     idesc_o, ks > 0);
                     umma_commit(kv_empty(st));
                     umma_commit(o_full);
                     ++issued_mma;
@@ -424,8 +459,17 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         }
     }
     grid_dependency_launch();
-    __syncthreads();
-    if (warp == 5) {
+    __syncthreads();                                   // both halves of every row have published their sums; all MMAs are done
+    if (warp < 8 && !*s_abort && live) {
+        const float l = s_lsum[r] + s_lsum[T::ROWS + r];
+        const float inv = 1.f / l;
+        float *dst = p.out + ((size_t)(q_begin + q0 + tok) * p.H + h) * DV + half * HD;
+#pragma unroll
+        for (int i = 0; i < HD; i += 4)
+            *reinterpret_cast<float4 *>(dst + i) = make_float4(acc[i] * inv, acc[i + 1] * inv, acc[i + 2] * inv, acc[i + 3] * inv);
+        if (half == 0 && p.lse) p.lse[(size_t)(q_begin + q0 + tok) * p.H + h] = (m_run + log2f(l)) * kLn2;
+    }
+    if (warp == 9) {
         tc_fence_after();
         tmem_dealloc(tmem, T::TMEM_COLS);
     }
