@@ -18,11 +18,12 @@
 //   warp 9         = MMA issuer (one lane) and owner of the tensor-memory allocation
 //   per 64-token tile j:
 //     S[j & 1]  = Q K_j^T            tcgen05.mma, K = d_v (value dims, 128-byte swizzle) + d_r (RoPE dims)
-//     softmax   : tcgen05.ld row -> mask -> running max / sum (base 2) -> P_j as bf16 pairs into tensor memory
-//     O         = P_j V_j            tcgen05.mma, A = P from tensor memory, B = the same value tile as an MN-major operand
-//     the row's output accumulates in registers: acc = acc * 2^(m_old - m_new) + O
-//   S is double-buffered in tensor memory, so the score product of tile j + 1 runs while the softmax warps work on
-//   tile j; two thread blocks per SM (d_v = 64) fill each other's gaps.  Shared memory carries only the operands
+//     softmax   : tcgen05.ld row -> mask -> row maximum / sum (base 2) -> P_j as bf16 pairs into tensor memory
+//     O        += P_j V_j            tcgen05.mma, A = P from tensor memory, B = the same value tile as an MN-major operand
+//     O accumulates in tensor memory across tiles.  The softmax reference of a row moves only when the running
+//     maximum grows by more than 2^8; only then is that row of O rescaled (read, multiplied, written back).
+//   S and P are double-buffered in tensor memory, so the score product of tile j + 1 and the value product of tile
+//   j - 1 run while the softmax warps work on tile j; two thread blocks per SM (d_v = 64) fill each other's gaps.  Shared memory carries only the operands
 //   the tensor core reads (Q and the cache tiles): P never touches it.
 //   Every wait is bounded; on expiry the block records GVA_ERR_TIMEOUT, drains what it issued, frees its
 //   tensor memory and exits.
@@ -65,9 +66,9 @@ struct PrefillTraits {
     static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
     static constexpr int N_BARS = 2 * NSTAGE + 6;
     static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16 + 2 * ROWS * 4;
-    // tensor-memory columns: S0, S1 (64 each), O (DV), P (TILE / 2: bf16 pairs)
+    // tensor-memory columns: S0, S1 (64 each), O (DV), P0, P1 (TILE / 2 each: bf16 pairs)
     static constexpr int COL_S = 0, COL_O = 2 * TILE, COL_P = COL_O + DV;
-    static constexpr int TMEM_COLS = (COL_P + TILE / 2) <= 256 ? 256 : 512;
+    static constexpr int TMEM_COLS = (COL_P + TILE) <= 256 ? 256 : 512;
     static constexpr int KSTEPS_V = DV / 16, KSTEPS_R = DR / 16;
     static constexpr int THREADS = 320;
 };
@@ -105,6 +106,17 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n" ::"r"(taddr),
         "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
         "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n" ::"r"(taddr),
+        "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "f"(v[8]), "f"(v[9]), "f"(v[10]),
+        "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]), "f"(v[16]), "f"(v[17]), "f"(v[18]), "f"(v[19]), "f"(v[20]),
+        "f"(v[21]), "f"(v[22]), "f"(v[23]), "f"(v[24]), "f"(v[25]), "f"(v[26]), "f"(v[27]), "f"(v[28]), "f"(v[29]), "f"(v[30]),
+        "f"(v[31])
         : "memory");
     asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
 }
@@ -154,6 +166,53 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 __host__ __device__ constexpr uint32_t umma_idesc(int M, int N, bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
            ((uint32_t)(M >> 4) << 24);
+}
+// Packed pairs of f32 (two lanes of one 64-bit register): one instruction for two multiply-adds / adds.
+__device__ __forceinline__ uint64_t f2_pack(float x, float y) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};\n" : "=l"(d) : "f"(x), "f"(y));
+    return d;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t d, float &x, float &y) { asm("mov.b64 {%0, %1}, %2;\n" : "=f"(x), "=f"(y) : "l"(d)); }
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+constexpr float kRescaleLog2 = 8.f;   // the softmax reference moves only when the running maximum grows by more than 2^8
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// Bounded wait whose polls sleep in hardware (suspend-time hint) instead of spinning through the issue slots.
+__device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    unsigned long long t0 = 0;
+    for (unsigned it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity), "r"(20000u)
+            : "memory");
+        if (ok) return true;
+        if ((it & 7u) == 7u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) return false;
+        }
+    }
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t d;
@@ -266,73 +325,84 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             mbar_arrive(q_ready);
         }
 
-#pragma unroll
-        for (int i = 0; i < HD; ++i) acc[i] = 0.f;
-        float l_run = 0.f, alpha_prev = 0.f;           // l_run: sum over this thread's columns only
+        float l_run = 0.f;                             // sum over this thread's columns only, relative to m_run
         const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
-            if (!mbar_wait_bounded(s_full(j & 1), (j >> 1) & 1, s_abort)) { ok = false; break; }
+            // S[j & 1] is complete; so is every MMA issued before it: the value product of tile j-2, which read P[j & 1]
+            if (!mbar_wait_sleepy(s_full(j & 1), (j >> 1) & 1, s_abort)) { ok = false; break; }
             tc_fence_after();
-            uint32_t pk[HC / 2];
-            float alpha;
+            const int limit = pos - j * T::TILE;              // columns c > limit are in the future of this row
+            const bool diag = limit < T::TILE - 1;
+            float mx[4];
             {
                 // the row maximum needs all 64 columns: read the partner's half too (no exchange between threads)
-                const int limit = pos - j * T::TILE;          // columns c > limit are in the future of this row
-                const bool diag = limit < T::TILE - 1;
-                float mx[4];
-                {
-                    float u[HC];
-                    tmem_ld32_nowait(lane_base + T::COL_S + (j & 1) * T::TILE + (half ^ 1) * HC, u);
-                    tmem_ld_wait();
-                    if (diag) {
-#pragma unroll
-                        for (int c = 0; c < HC; ++c) u[c] = ((half ^ 1) * HC + c > limit) ? -INFINITY : u[c];
-                    }
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) mx[k] = fmaxf(u[k], u[k + 4]);
-#pragma unroll
-                    for (int c = 8; c < HC; c += 4)
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) mx[k] = fmaxf(mx[k], u[c + k]);
-                }
-                float s[HC];
-                tmem_ld32_nowait(lane_base + T::COL_S + (j & 1) * T::TILE + half * HC, s);
+                float u[HC];
+                tmem_ld32_nowait(lane_base + T::COL_S + (j & 1) * T::TILE + (half ^ 1) * HC, u);
                 tmem_ld_wait();
                 if (diag) {
 #pragma unroll
-                    for (int c = 0; c < HC; ++c) s[c] = (half * HC + c > limit) ? -INFINITY : s[c];
+                    for (int c = 0; c < HC; ++c) u[c] = ((half ^ 1) * HC + c > limit) ? -INFINITY : u[c];
                 }
 #pragma unroll
-                for (int c = 0; c < HC; c += 4)
+                for (int k = 0; k < 4; ++k) mx[k] = max3(u[k], u[k + 4], u[k + 8]);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) mx[k] = fmaxf(mx[k], s[c + k]);
-                const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2);
-                // m_new is finite from tile 0 on: token 0 is visible to every row
-                alpha = fast_exp2(m_run - m_new);
-                float sum[2] = {0.f, 0.f};
+                for (int c = 12; c + 8 <= HC; c += 8)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) mx[k] = max3(mx[k], u[c + k], u[c + 4 + k]);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) mx[k] = fmaxf(mx[k], u[HC - 4 + k]);
+            }
+            float s[HC];
+            tmem_ld32_nowait(lane_base + T::COL_S + (j & 1) * T::TILE + half * HC, s);
+            tmem_ld_wait();
+            if (diag) {
+#pragma unroll
+                for (int c = 0; c < HC; ++c) s[c] = (half * HC + c > limit) ? -INFINITY : s[c];
+            }
+#pragma unroll
+            for (int c = 0; c < HC; c += 8)
+#pragma unroll
+                for (int k = 0; k < 4; ++k) mx[k] = max3(mx[k], s[c + k], s[c + 4 + k]);
+            const float m_tile = max3(mx[0], mx[1], fmaxf(mx[2], mx[3])) * p.scale_log2;
+            // The reference m_run of the row only moves when the tile's maximum exceeds it by more than 2^8: the
+            // weights stay below 256 relative to it, the result is the same quotient, and the accumulated O (which
+            // lives in tensor memory) has to be rescaled only then.  Both threads of a row take the same decision.
+            // (m_tile is finite in tile 0: token 0 is visible to every row.)
+            if (m_tile > m_run + kRescaleLog2) {
+                const float alpha = fast_exp2(m_run - m_tile);
+                l_run *= alpha;
+                m_run = m_tile;
+                if (j > 0) {
+                    if (!mbar_wait_sleepy(o_full, (j - 1) & 1, s_abort)) { ok = false; break; }   // O holds tiles 0..j-1
+                    tc_fence_after();
+                    const uint64_t al2 = f2_pack(alpha, alpha);
+#pragma unroll
+                    for (int part = 0; part < HD / 32; ++part) {
+                        float o[32];
+                        tmem_ld32_nowait(lane_base + T::COL_O + half * HD + part * 32, o);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) f2_unpack(f2_mul(f2_pack(o[i], o[i + 1]), al2), o[i], o[i + 1]);
+                        tmem_st32(lane_base + T::COL_O + half * HD + part * 32, o);
+                    }
+                }
+            }
+            uint32_t pk[HC / 2];
+            {
+                const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nm2 = f2_pack(-m_run, -m_run);
+                uint64_t sum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
 #pragma unroll
                 for (int c = 0; c < HC; c += 2) {
-                    const float e0 = fast_exp2(fmaf(s[c], p.scale_log2, -m_new));
-                    const float e1 = fast_exp2(fmaf(s[c + 1], p.scale_log2, -m_new));
-                    sum[0] += e0;
-                    sum[1] += e1;
+                    float t0, t1;
+                    f2_unpack(f2_fma(f2_pack(s[c], s[c + 1]), sc2, nm2), t0, t1);
+                    const float e0 = fast_exp2(t0), e1 = fast_exp2(t1);
+                    sum2[(c >> 1) & 1] = f2_add(sum2[(c >> 1) & 1], f2_pack(e0, e1));
                     pk[c >> 1] = pack_bf16(e0, e1);
                 }
-                l_run = l_run * alpha + (sum[0] + sum[1]);
-                m_run = m_new;
-            }
-            // the previous value product has read P and written O
-            if (j > 0) {
-                if (!mbar_wait_bounded(o_full, (j - 1) & 1, s_abort)) { ok = false; break; }
-                tc_fence_after();
-#pragma unroll
-                for (int part = 0; part < HD / 32; ++part) {
-                    float o[32];
-                    tmem_ld32(lane_base + T::COL_O + half * HD + part * 32, o);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) acc[part * 32 + i] = fmaf(acc[part * 32 + i], alpha_prev, o[i]);
-                }
+                float sa, sb;
+                f2_unpack(f2_add(sum2[0], sum2[1]), sa, sb);
+                l_run += sa + sb;
             }
             // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
             if ((long long)(j + 1) * T::TILE > kv_total) {
@@ -345,20 +415,20 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                 }
                 fence_async_smem();
             }
-            tmem_st16(lane_base + T::COL_P + half * (HC / 2), pk);
+            tmem_st16(lane_base + T::COL_P + (j & 1) * (T::TILE / 2) + half * (HC / 2), pk);
             tc_fence_before();
             mbar_arrive(p_full);
-            alpha_prev = alpha;
         }
-        if (ok && !mbar_wait_bounded(o_full, (n_tiles - 1) & 1, s_abort)) ok = false;
+        if (ok && !mbar_wait_sleepy(o_full, (n_tiles - 1) & 1, s_abort)) ok = false;
         if (ok) {
             tc_fence_after();
 #pragma unroll
             for (int part = 0; part < HD / 32; ++part) {
                 float o[32];
-                tmem_ld32(lane_base + T::COL_O + half * HD + part * 32, o);
+                tmem_ld32_nowait(lane_base + T::COL_O + half * HD + part * 32, o);
+                tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) acc[part * 32 + i] = fmaf(acc[part * 32 + i], alpha_prev, o[i]);
+                for (int i = 0; i < 32; ++i) acc[part * 32 + i] = o[i];
             }
             s_lsum[half * T::ROWS + r] = l_run;
         } else if (!*s_abort) {
@@ -381,7 +451,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                     *s_abort = 1;
                     break;
                 }
-                if (j >= NS && !mbar_wait_bounded(kv_empty(st), ((j / NS) & 1) ^ 1, s_abort)) {
+                if (j >= NS && !mbar_wait_sleepy(kv_empty(st), ((j / NS) & 1) ^ 1, s_abort)) {
                     if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
                     *s_abort = 1;
                     break;
@@ -406,13 +476,13 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             constexpr uint32_t idesc_o = umma_idesc(T::ROWS, DV, true);
             constexpr uint64_t kr_swz = T::KR_ROW == 32 ? kSwz32 : kSwz64;
             constexpr uint32_t kr_sbo = 8 * T::KR_ROW;
-            bool ok = mbar_wait_bounded(q_ready, 0, s_abort);
+            bool ok = mbar_wait_sleepy(q_ready, 0, s_abort);
             int issued_mma = 0;
             for (int j = 0; j <= n_tiles && ok; ++j) {
                 if (j < n_tiles) {
                     // score product of tile j; S[j & 1] was released when P of tile j-2 was complete (waited below)
                     const int st = j % NS;
-                    if (!mbar_wait_bounded(kv_full(st), (j / NS) & 1, s_abort)) { ok = false; break; }
+                    if (!mbar_wait_sleepy(kv_full(st), (j / NS) & 1, s_abort)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t vb = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
                     const uint32_t d = tmem + T::COL_S + (j & 1) * T::TILE;
@@ -431,16 +501,16 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                     ++issued_mma;
                 }
                 if (j >= 1) {
-                    // value product of tile j-1: O = P V; all rows have stored P and have read O of tile j-2
+                    // value product of tile j-1: O += P V; all rows have stored P[(j-1) & 1] and finished any rescaling of O
                     const int jj = j - 1, st = jj % NS;
-                    if (!mbar_wait_bounded(p_full, jj & 1, s_abort)) { ok = false; break; }
+                    if (!mbar_wait_sleepy(p_full, jj & 1, s_abort)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t vb = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
                     const uint32_t d = tmem + T::COL_O;
 #pragma unroll
                     for (int ks = 0; ks < T::TILE / 16; ++ks)
-                        umma_bf16_ts(d, tmem + T::COL_P + ks * 8, smem_desc(vb + ks * 16 * 128, T::VBOX_BYTES, 1024, kSwz128),
-                                     idesc_o, ks > 0);
+                        umma_bf16_ts(d, tmem + T::COL_P + (jj & 1) * (T::TILE / 2) + ks * 8,
+                                     smem_desc(vb + ks * 16 * 128, T::VBOX_BYTES, 1024, kSwz128), idesc_o, (jj > 0 || ks > 0) ? 1u : 0u);
                     umma_commit(kv_empty(st));
                     umma_commit(o_full);
                     ++issued_mma;
