@@ -11,20 +11,20 @@
 //
 // Layout of the work
 //   thread block   = 32 query tokens x 4 heads of one (sequence, value group): 128 rows = one M = 128 MMA tile
-//   warps 0-7      = softmax: row r (token r / 4, head r % 4) = tensor-memory lane r is shared by two threads, one in
-//                    warp w and one in warp w + 4 (both reach lanes 32 (w % 4) ..); each owns half of the tile's score
-//                    columns and half of the output dims, and reads the other half of the scores only for the row maximum
-//   warp 8         = producer (one lane): TMA loads of the 64-token value tile and positional-key tile into a ring
-//   warp 9         = MMA issuer (one lane) and owner of the tensor-memory allocation
+//   warps 0-3      = softmax: thread r owns row r (token r / 4, head r % 4) = tensor-memory lane r
+//   warp 4         = producer (one lane): TMA loads of the 64-token value tile and positional-key tile into a ring
+//   warp 5         = MMA issuer (one lane) and owner of the tensor-memory allocation
 //   per 64-token tile j:
-//     S[j & 1]  = Q K_j^T            tcgen05.mma, K = d_v (value dims, 128-byte swizzle) + d_r (RoPE dims)
-//     softmax   : tcgen05.ld row -> mask -> row maximum / sum (base 2) -> P_j as bf16 pairs into tensor memory
+//     S         = Q K_j^T            tcgen05.mma, K = d_v (value dims, 128-byte swizzle) + d_r (RoPE dims)
+//     softmax   : tcgen05.ld row -> mask -> row maximum / sum (base 2) -> P_j as bf16 pairs, written over the first
+//                 half of the row's own S columns (a row has one reader, so nothing else can still need them)
 //     O        += P_j V_j            tcgen05.mma, A = P from tensor memory, B = the same value tile as an MN-major operand
 //     O accumulates in tensor memory across tiles.  The softmax reference of a row moves only when the running
 //     maximum grows by more than 2^8; only then is that row of O rescaled (read, multiplied, written back).
-//   S and P are double-buffered in tensor memory, so the score product of tile j + 1 and the value product of tile
-//   j - 1 run while the softmax warps work on tile j; two thread blocks per SM (d_v = 64) fill each other's gaps.  Shared memory carries only the operands
-//   the tensor core reads (Q and the cache tiles): P never touches it.
+//   A block holds 64 + d_v tensor-memory columns and little shared memory, so four blocks (d_v = 64) share an SM:
+//   inside a block the score product, the softmax and the value product of a tile follow one another, and the
+//   other blocks fill the gaps.  Shared memory carries only the operands the tensor core reads (Q and the cache
+//   tiles): P never touches it.
 //   Every wait is bounded; on expiry the block records GVA_ERR_TIMEOUT, drains what it issued, frees its
 //   tensor memory and exits.
 #pragma once
@@ -50,7 +50,7 @@ struct PrefillTraits {
     static constexpr int QTOK = 32;                              // query tokens per block
     static constexpr int ROWS = QTOK * kHeadsPerGroup;           // 128 = MMA M
     static constexpr int TILE = 64;                              // cached tokens per tile = MMA N of the score product
-    static constexpr int NSTAGE = 4;
+    static constexpr int NSTAGE = 3;
     static constexpr int BOXES = DV / 64;                        // 64-dim (128-byte) boxes per value row
     static constexpr int QBOX_BYTES = ROWS * 128;
     static constexpr int QV_BYTES = BOXES * QBOX_BYTES;
@@ -64,13 +64,14 @@ struct PrefillTraits {
     static constexpr int OFF_QR = OFF_QV + QV_BYTES;
     static constexpr int OFF_STAGE = OFF_QR + QR_BYTES;
     static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
-    static constexpr int N_BARS = 2 * NSTAGE + 6;
-    static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16 + 2 * ROWS * 4;
-    // tensor-memory columns: S0, S1 (64 each), O (DV), P0, P1 (TILE / 2 each: bf16 pairs)
-    static constexpr int COL_S = 0, COL_O = 2 * TILE, COL_P = COL_O + DV;
-    static constexpr int TMEM_COLS = (COL_P + TILE) <= 256 ? 256 : 512;
+    static constexpr int N_BARS = 2 * NSTAGE + 5;
+    static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
+    // tensor-memory columns: S (64; P overwrites its first 32), O (DV)
+    static constexpr int COL_S = 0, COL_O = TILE;
+    static constexpr int TMEM_COLS = (TILE + DV) <= 128 ? 128 : 256;
+    static constexpr int BLOCKS_PER_SM = 512 / TMEM_COLS;
     static constexpr int KSTEPS_V = DV / 16, KSTEPS_R = DR / 16;
-    static constexpr int THREADS = 320;
+    static constexpr int THREADS = 192;
 };
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------------------------
@@ -109,6 +110,14 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
         : "memory");
     asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
 }
+__device__ __forceinline__ void tmem_st16_nowait(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n" ::"r"(taddr),
+        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+        "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -221,7 +230,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 template <int DV, int DR>
-__global__ void __launch_bounds__(320, DV == 64 ? 2 : 1)
+__global__ void __launch_bounds__(192, PrefillTraits<DV, DR>::BLOCKS_PER_SM)
 prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = PrefillTraits<DV, DR>;
     constexpr int NS = T::NSTAGE;
@@ -250,22 +259,19 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     const uint32_t bar0 = s_base + T::OFF_BAR;
     auto kv_full = [&](int s) { return bar0 + 8u * s; };
     auto kv_empty = [&](int s) { return bar0 + 8u * (NS + s); };
-    auto s_full = [&](int i) { return bar0 + 8u * (2 * NS + i); };
-    const uint32_t p_full = bar0 + 8u * (2 * NS + 2), q_ready = bar0 + 8u * (2 * NS + 3), drain = bar0 + 8u * (2 * NS + 4);
-    const uint32_t o_full = bar0 + 8u * (2 * NS + 5);   // one barrier for both O buffers: value products complete in order
+    const uint32_t s_full = bar0 + 8u * (2 * NS), p_full = bar0 + 8u * (2 * NS + 1), q_ready = bar0 + 8u * (2 * NS + 2),
+                   drain = bar0 + 8u * (2 * NS + 3), o_full = bar0 + 8u * (2 * NS + 4);
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + T::N_BARS);
     volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
-    float *s_lsum = reinterpret_cast<float *>(s_tmem + 4);        // [2][ROWS] per-half row sums, exchanged once at the end
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(kv_full(s), 1);
             mbar_init(kv_empty(s), 1);
         }
-        mbar_init(s_full(0), 1);
-        mbar_init(s_full(1), 1);
-        mbar_init(p_full, 2 * T::ROWS);
-        mbar_init(q_ready, 2 * T::ROWS);
+        mbar_init(s_full, 1);
+        mbar_init(p_full, T::ROWS);
+        mbar_init(q_ready, T::ROWS);
         mbar_init(drain, 1);
         mbar_init(o_full, 1);
         *s_abort = 0;
@@ -273,7 +279,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
     }
-    if (warp == 9) {
+    if (warp == 5) {
         tmem_alloc(smem_u32(s_tmem), T::TMEM_COLS);
         tmem_relinquish();
     }
@@ -282,26 +288,18 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     tc_fence_after();
     const uint32_t tmem = *s_tmem;
 
-    // softmax threads (warps 0-7): two per row, each owns half of the tile's score columns and of the output dims
-    const int half = (warp >> 2) & 1;                  // warps w and w + 4 reach the same tensor-memory lanes (32 (w % 4) ..)
-    const int r = (warp & 3) * 32 + lane;
-    const int tok = r >> 2, hl = r & 3;
-    const int h = g * kHeadsPerGroup + hl;
-    const bool live = tok < nv;
-    const int pos = p0 + tok;
-    constexpr int HC = T::TILE / 2;                    // score columns per thread
-    constexpr int HD = DV / 2;                         // output dims per thread
-    float acc[HD];
-    float m_run = -INFINITY;
-
-    if (warp < 8) {
-        // ============================================== softmax ==============================================
+    if (warp < 4) {
+        // ====================================== softmax: one row per thread ======================================
+        const int r = tid;
+        const int tok = r >> 2, hl = r & 3;
+        const int h = g * kHeadsPerGroup + hl;
+        const bool live = tok < nv;
+        const int pos = p0 + tok;
         // ---- stage Q: f32 -> bf16, swizzled K-major rows (value dims in 128-byte boxes, then the RoPE dims) ----
         {
             const float4 *src = reinterpret_cast<const float4 *>(p.q_abs + ((size_t)(q_begin + q0 + tok) * p.H + h) * (DV + DR));
 #pragma unroll
-            for (int cc = 0; cc < DV / 16; ++cc) {
-                const int c = half * (DV / 16) + cc;
+            for (int c = 0; c < DV / 8; ++c) {
                 float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
                 if (live) {
                     a = __ldg(src + 2 * c);
@@ -311,8 +309,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                     make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(bq.x, bq.y), pack_bf16(bq.z, bq.w));
             }
 #pragma unroll
-            for (int cc = 0; cc < DR / 16; ++cc) {
-                const int c = half * (DR / 16) + cc;
+            for (int c = 0; c < DR / 8; ++c) {
                 float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
                 if (live) {
                     a = __ldg(src + DV / 4 + 2 * c);
@@ -325,85 +322,102 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             mbar_arrive(q_ready);
         }
 
-        float l_run = 0.f;                             // sum over this thread's columns only, relative to m_run
-        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        float m_run = -INFINITY, l_run = 0.f;          // softmax reference (log2 domain) and sum relative to it
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        const uint32_t s_addr = lane_base + T::COL_S, o_addr = lane_base + T::COL_O;
         bool ok = true;
-        for (int j = 0; j < n_tiles && ok; ++j) {
-            // S[j & 1] is complete; so is every MMA issued before it: the value product of tile j-2, which read P[j & 1]
-            if (!mbar_wait_sleepy(s_full(j & 1), (j >> 1) & 1, s_abort)) { ok = false; break; }
+        for (int j = 0; j < n_tiles; ++j) {
+            // S of tile j is complete, and with it every MMA issued before it: O holds tiles 0..j-1
+            if (!mbar_wait_sleepy(s_full, j & 1, s_abort)) { ok = false; break; }
             tc_fence_after();
             const int limit = pos - j * T::TILE;              // columns c > limit are in the future of this row
             const bool diag = limit < T::TILE - 1;
+            // ---- pass 1: the row maximum ----
             float mx[4];
-            {
-                // the row maximum needs all 64 columns: read the partner's half too (no exchange between threads)
-                float u[HC];
-                tmem_ld32_nowait(lane_base + T::COL_S + (j & 1) * T::TILE + (half ^ 1) * HC, u);
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                float u[32];
+                tmem_ld32_nowait(s_addr + hf * 32, u);
                 tmem_ld_wait();
                 if (diag) {
 #pragma unroll
-                    for (int c = 0; c < HC; ++c) u[c] = ((half ^ 1) * HC + c > limit) ? -INFINITY : u[c];
+                    for (int c = 0; c < 32; ++c) u[c] = (hf * 32 + c > limit) ? -INFINITY : u[c];
                 }
+                if (hf == 0) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k) mx[k] = max3(u[k], u[k + 4], u[k + 8]);
+                    for (int k = 0; k < 4; ++k) mx[k] = max3(u[k], u[k + 4], u[k + 8]);
 #pragma unroll
-                for (int c = 12; c + 8 <= HC; c += 8)
+                    for (int c = 12; c + 8 <= 32; c += 8)
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) mx[k] = max3(mx[k], u[c + k], u[c + 4 + k]);
+                        for (int k = 0; k < 4; ++k) mx[k] = max3(mx[k], u[c + k], u[c + 4 + k]);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) mx[k] = fmaxf(mx[k], u[HC - 4 + k]);
+                    for (int k = 0; k < 4; ++k) mx[k] = fmaxf(mx[k], u[28 + k]);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 8)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) mx[k] = max3(mx[k], u[c + k], u[c + 4 + k]);
+                }
             }
-            float s[HC];
-            tmem_ld32_nowait(lane_base + T::COL_S + (j & 1) * T::TILE + half * HC, s);
-            tmem_ld_wait();
-            if (diag) {
-#pragma unroll
-                for (int c = 0; c < HC; ++c) s[c] = (half * HC + c > limit) ? -INFINITY : s[c];
-            }
-#pragma unroll
-            for (int c = 0; c < HC; c += 8)
-#pragma unroll
-                for (int k = 0; k < 4; ++k) mx[k] = max3(mx[k], s[c + k], s[c + 4 + k]);
             const float m_tile = max3(mx[0], mx[1], fmaxf(mx[2], mx[3])) * p.scale_log2;
             // The reference m_run of the row only moves when the tile's maximum exceeds it by more than 2^8: the
             // weights stay below 256 relative to it, the result is the same quotient, and the accumulated O (which
-            // lives in tensor memory) has to be rescaled only then.  Both threads of a row take the same decision.
-            // (m_tile is finite in tile 0: token 0 is visible to every row.)
-            if (m_tile > m_run + kRescaleLog2) {
-                const float alpha = fast_exp2(m_run - m_tile);
+            // lives in tensor memory) has to be rescaled only then.  (m_tile is finite in tile 0: token 0 is
+            // visible to every row.)
+            const bool move = m_tile > m_run + kRescaleLog2;
+            float alpha = 1.f;
+            if (move) {
+                alpha = fast_exp2(m_run - m_tile);
                 l_run *= alpha;
                 m_run = m_tile;
-                if (j > 0) {
-                    if (!mbar_wait_sleepy(o_full, (j - 1) & 1, s_abort)) { ok = false; break; }   // O holds tiles 0..j-1
-                    tc_fence_after();
-                    const uint64_t al2 = f2_pack(alpha, alpha);
+            }
+            // tcgen05.ld / tcgen05.st are warp-wide instructions: when any row of the warp moves its reference, every
+            // lane rescales its row of O (by 1 where nothing moved)
+            if (j > 0 && __any_sync(0xffffffffu, move)) {
+                const uint64_t al2 = f2_pack(alpha, alpha);
 #pragma unroll
-                    for (int part = 0; part < HD / 32; ++part) {
-                        float o[32];
-                        tmem_ld32_nowait(lane_base + T::COL_O + half * HD + part * 32, o);
-                        tmem_ld_wait();
+                for (int part = 0; part < DV / 32; ++part) {
+                    float o[32];
+                    tmem_ld32_nowait(o_addr + part * 32, o);
+                    tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2) f2_unpack(f2_mul(f2_pack(o[i], o[i + 1]), al2), o[i], o[i + 1]);
-                        tmem_st32(lane_base + T::COL_O + half * HD + part * 32, o);
-                    }
+                    for (int i = 0; i < 32; i += 2) f2_unpack(f2_mul(f2_pack(o[i], o[i + 1]), al2), o[i], o[i + 1]);
+                    tmem_st32(o_addr + part * 32, o);
                 }
             }
-            uint32_t pk[HC / 2];
-            {
-                const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nm2 = f2_pack(-m_run, -m_run);
-                uint64_t sum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
+            // ---- pass 2: weights, row sum, P over the first 32 columns of S (both halves of S are in registers or
+            //      consumed before their columns are overwritten: half 0 is read before P of half 0 is stored, and
+            //      P of half 1 lands in columns 16..31, which belong to half 0) ----
+            const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nm2 = f2_pack(-m_run, -m_run);
+            uint64_t sum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
 #pragma unroll
-                for (int c = 0; c < HC; c += 2) {
+            for (int hf = 0; hf < 2; ++hf) {
+                float s[32];
+                tmem_ld32_nowait(s_addr + hf * 32, s);
+                tmem_ld_wait();
+                if (diag) {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) s[c] = (hf * 32 + c > limit) ? -INFINITY : s[c];
+                }
+                uint32_t pk[16];
+#pragma unroll
+                for (int c = 0; c < 32; c += 2) {
                     float t0, t1;
                     f2_unpack(f2_fma(f2_pack(s[c], s[c + 1]), sc2, nm2), t0, t1);
                     const float e0 = fast_exp2(t0), e1 = fast_exp2(t1);
                     sum2[(c >> 1) & 1] = f2_add(sum2[(c >> 1) & 1], f2_pack(e0, e1));
                     pk[c >> 1] = pack_bf16(e0, e1);
                 }
-                float sa, sb;
-                f2_unpack(f2_add(sum2[0], sum2[1]), sa, sb);
-                l_run += sa + sb;
+                if (hf == 0) {
+                    // half 1 of S must be in registers before columns 16..31 can be overwritten; columns 0..15 are free now
+                    tmem_st16_nowait(s_addr, pk);
+                } else {
+                    tmem_st16_nowait(s_addr + 16, pk);
+                }
             }
+            float sa, sb;
+            f2_unpack(f2_add(sum2[0], sum2[1]), sa, sb);
+            l_run += sa + sb;
             // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
             if ((long long)(j + 1) * T::TILE > kv_total) {
                 if (tid < T::TILE && (long long)j * T::TILE + tid >= kv_total) {
@@ -415,28 +429,34 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                 }
                 fence_async_smem();
             }
-            tmem_st16(lane_base + T::COL_P + (j & 1) * (T::TILE / 2) + half * (HC / 2), pk);
+            tmem_st_wait();
             tc_fence_before();
             mbar_arrive(p_full);
         }
-        if (ok && !mbar_wait_sleepy(o_full, (n_tiles - 1) & 1, s_abort)) ok = false;
+        if (ok && !mbar_wait_sleepy(o_full, 0, s_abort)) ok = false;
         if (ok) {
             tc_fence_after();
+            // (tcgen05.ld is a warp-wide instruction: every lane takes part, dead rows only skip the stores)
+            const float inv = 1.f / l_run;
+            float *dst = p.out + ((size_t)(q_begin + q0 + tok) * p.H + h) * DV;
 #pragma unroll
-            for (int part = 0; part < HD / 32; ++part) {
+            for (int part = 0; part < DV / 32; ++part) {
                 float o[32];
-                tmem_ld32_nowait(lane_base + T::COL_O + half * HD + part * 32, o);
+                tmem_ld32_nowait(o_addr + part * 32, o);
                 tmem_ld_wait();
+                if (live) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) acc[part * 32 + i] = o[i];
+                    for (int i = 0; i < 32; i += 4)
+                        *reinterpret_cast<float4 *>(dst + part * 32 + i) = make_float4(o[i] * inv, o[i + 1] * inv, o[i + 2] * inv, o[i + 3] * inv);
+                }
             }
-            s_lsum[half * T::ROWS + r] = l_run;
+            if (live && p.lse) p.lse[(size_t)(q_begin + q0 + tok) * p.H + h] = (m_run + log2f(l_run)) * kLn2;
         } else if (!*s_abort) {
             report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
             *s_abort = 1;
         }
         tc_fence_before();
-    } else if (warp == 8) {
+    } else if (warp == 4) {
         // ====================================== producer (one lane) ======================================
         if (lane == 0) {
             int issued = 0;
@@ -478,44 +498,37 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             constexpr uint32_t kr_sbo = 8 * T::KR_ROW;
             bool ok = mbar_wait_sleepy(q_ready, 0, s_abort);
             int issued_mma = 0;
-            for (int j = 0; j <= n_tiles && ok; ++j) {
-                if (j < n_tiles) {
-                    // score product of tile j; S[j & 1] was released when P of tile j-2 was complete (waited below)
-                    const int st = j % NS;
-                    if (!mbar_wait_sleepy(kv_full(st), (j / NS) & 1, s_abort)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t vb = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
-                    const uint32_t d = tmem + T::COL_S + (j & 1) * T::TILE;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                // score product of tile j: overwrites S and the P of tile j-1 inside it, so the value product of tile
+                // j-1 must have completed (MMAs with different accumulators are not ordered among themselves)
+                const int st = j % NS;
+                if (!mbar_wait_sleepy(kv_full(st), (j / NS) & 1, s_abort)) { ok = false; break; }
+                if (j > 0 && !mbar_wait_sleepy(kv_empty((j - 1) % NS), ((j - 1) / NS) & 1, s_abort)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t vb = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
 #pragma unroll
-                    for (int ks = 0; ks < T::KSTEPS_V; ++ks) {
-                        const uint32_t off = (ks >> 2) * T::QBOX_BYTES + (ks & 3) * 32;
-                        const uint32_t voff = (ks >> 2) * T::VBOX_BYTES + (ks & 3) * 32;
-                        umma_bf16(d, smem_desc(s_base + T::OFF_QV + off, 16, 1024, kSwz128),
-                                  smem_desc(vb + voff, 16, 1024, kSwz128), idesc_s, ks > 0);
-                    }
-#pragma unroll
-                    for (int ks = 0; ks < T::KSTEPS_R; ++ks)
-                        umma_bf16(d, smem_desc(s_base + T::OFF_QR + ks * 32, 16, kr_sbo, kr_swz),
-                                  smem_desc(vb + T::V_BYTES + ks * 32, 16, kr_sbo, kr_swz), idesc_s, 1);
-                    umma_commit(s_full(j & 1));
-                    ++issued_mma;
+                for (int ks = 0; ks < T::KSTEPS_V; ++ks) {
+                    const uint32_t off = (ks >> 2) * T::QBOX_BYTES + (ks & 3) * 32;
+                    const uint32_t voff = (ks >> 2) * T::VBOX_BYTES + (ks & 3) * 32;
+                    umma_bf16(tmem + T::COL_S, smem_desc(s_base + T::OFF_QV + off, 16, 1024, kSwz128),
+                              smem_desc(vb + voff, 16, 1024, kSwz128), idesc_s, ks > 0);
                 }
-                if (j >= 1) {
-                    // value product of tile j-1: O += P V; all rows have stored P[(j-1) & 1] and finished any rescaling of O
-                    const int jj = j - 1, st = jj % NS;
-                    if (!mbar_wait_sleepy(p_full, jj & 1, s_abort)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t vb = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
-                    const uint32_t d = tmem + T::COL_O;
 #pragma unroll
-                    for (int ks = 0; ks < T::TILE / 16; ++ks)
-                        umma_bf16_ts(d, tmem + T::COL_P + (jj & 1) * (T::TILE / 2) + ks * 8,
-                                     smem_desc(vb + ks * 16 * 128, T::VBOX_BYTES, 1024, kSwz128), idesc_o, (jj > 0 || ks > 0) ? 1u : 0u);
-                    umma_commit(kv_empty(st));
-                    umma_commit(o_full);
-                    ++issued_mma;
-                }
+                for (int ks = 0; ks < T::KSTEPS_R; ++ks)
+                    umma_bf16(tmem + T::COL_S, smem_desc(s_base + T::OFF_QR + ks * 32, 16, kr_sbo, kr_swz),
+                              smem_desc(vb + T::V_BYTES + ks * 32, 16, kr_sbo, kr_swz), idesc_s, 1);
+                umma_commit(s_full);
+                ++issued_mma;
+                // value product of tile j: O += P V once every row has stored P (and finished any rescaling of O)
+                if (!mbar_wait_sleepy(p_full, j & 1, s_abort)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < T::TILE / 16; ++ks)
+                    umma_bf16_ts(tmem + T::COL_O, tmem + T::COL_S + ks * 8,
+                                 smem_desc(vb + ks * 16 * 128, T::VBOX_BYTES, 1024, kSwz128), idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
+                umma_commit(kv_empty(st));
             }
+            if (ok) umma_commit(o_full);
             if (!ok && !*s_abort) {
                 report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
                 *s_abort = 1;
@@ -529,17 +542,8 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         }
     }
     grid_dependency_launch();
-    __syncthreads();                                   // both halves of every row have published their sums; all MMAs are done
-    if (warp < 8 && !*s_abort && live) {
-        const float l = s_lsum[r] + s_lsum[T::ROWS + r];
-        const float inv = 1.f / l;
-        float *dst = p.out + ((size_t)(q_begin + q0 + tok) * p.H + h) * DV + half * HD;
-#pragma unroll
-        for (int i = 0; i < HD; i += 4)
-            *reinterpret_cast<float4 *>(dst + i) = make_float4(acc[i] * inv, acc[i + 1] * inv, acc[i + 2] * inv, acc[i + 3] * inv);
-        if (half == 0 && p.lse) p.lse[(size_t)(q_begin + q0 + tok) * p.H + h] = (m_run + log2f(l)) * kLn2;
-    }
-    if (warp == 9) {
+    __syncthreads();
+    if (warp == 5) {
         tc_fence_after();
         tmem_dealloc(tmem, T::TMEM_COLS);
     }
@@ -555,8 +559,9 @@ template <int DV, int DR>
 int launch_prefill_t(const gva_config &cfg, const MmaHostState &st, int smem_optin, const PrefillParams &p, const void *v_pool,
                      const void *kr_pool, int B, int max_q_len, cudaStream_t stream) {
     using T = PrefillTraits<DV, DR>;
-    // request at least 80 KB so that no more than two blocks (2 x 256 tensor-memory columns) share an SM
-    const size_t smem = T::SMEM_BYTES < 80 * 1024 ? 80 * 1024 : T::SMEM_BYTES;
+    // never more blocks on an SM than its 512 tensor-memory columns can serve: pad the request if need be
+    const size_t floor_bytes = (size_t)227 * 1024 / (T::BLOCKS_PER_SM + 1) + 1024;
+    const size_t smem = (size_t)T::SMEM_BYTES < floor_bytes ? floor_bytes : (size_t)T::SMEM_BYTES;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
     auto fn = prefill_kernel<DV, DR>;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;

@@ -169,6 +169,8 @@ def test_prefill_reports_bad_page_and_long_sequence():
         ref, _ = orc.prefill_case(wl.make_prefill_case("bad", wl.SHAPE_A, [0, 0], [100, 40], page_size=64, seed=508))
         assert np.max(np.abs(out[100:140] - ref[100:140])) <= TOL_MAXABS     # the other sequence is unaffected
         pd.status.zero_()
+        pd.dc.block_table.copy_(torch.from_numpy(wl.make_prefill_case("bad", wl.SHAPE_A, [0, 0], [100, 40], page_size=64,
+                                                                      seed=508).cache.block_table).to(pd.dc.block_table.device))
         pd.ctx_lens[1] = 10_000                                               # beyond its block table
         pd.prefill()
         torch.cuda.synchronize()
