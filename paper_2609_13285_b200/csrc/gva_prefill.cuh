@@ -15,16 +15,15 @@
 //   warp 4         = producer (one lane): TMA loads of the 64-token value tile and positional-key tile into a ring
 //   warp 5         = MMA issuer (one lane) and owner of the tensor-memory allocation
 //   per 64-token tile j:
-//     S         = Q K_j^T            tcgen05.mma, K = d_v (value dims, 128-byte swizzle) + d_r (RoPE dims)
+//     S[j & 1]  = Q K_j^T            tcgen05.mma, K = d_v (value dims, 128-byte swizzle) + d_r (RoPE dims)
 //     softmax   : tcgen05.ld row -> mask -> row maximum / sum (base 2) -> P_j as bf16 pairs, written over the first
 //                 half of the row's own S columns (a row has one reader, so nothing else can still need them)
 //     O        += P_j V_j            tcgen05.mma, A = P from tensor memory, B = the same value tile as an MN-major operand
 //     O accumulates in tensor memory across tiles.  The softmax reference of a row moves only when the running
 //     maximum grows by more than 2^8; only then is that row of O rescaled (read, multiplied, written back).
-//   A block holds 64 + d_v tensor-memory columns and little shared memory, so four blocks (d_v = 64) share an SM:
-//   inside a block the score product, the softmax and the value product of a tile follow one another, and the
-//   other blocks fill the gaps.  Shared memory carries only the operands the tensor core reads (Q and the cache
-//   tiles): P never touches it.
+//   S is double-buffered, so the score product of tile j + 1 and the value product of tile j - 1 run while the
+//   softmax warps work on tile j; two blocks share an SM (256 tensor-memory columns each).  Shared memory carries
+//   only the operands the tensor core reads (Q and the cache tiles): P never touches it.
 //   Every wait is bounded; on expiry the block records GVA_ERR_TIMEOUT, drains what it issued, frees its
 //   tensor memory and exits.
 #pragma once
@@ -50,7 +49,7 @@ struct PrefillTraits {
     static constexpr int QTOK = 32;                              // query tokens per block
     static constexpr int ROWS = QTOK * kHeadsPerGroup;           // 128 = MMA M
     static constexpr int TILE = 64;                              // cached tokens per tile = MMA N of the score product
-    static constexpr int NSTAGE = 3;
+    static constexpr int NSTAGE = 4;
     static constexpr int BOXES = DV / 64;                        // 64-dim (128-byte) boxes per value row
     static constexpr int QBOX_BYTES = ROWS * 128;
     static constexpr int QV_BYTES = BOXES * QBOX_BYTES;
@@ -64,11 +63,12 @@ struct PrefillTraits {
     static constexpr int OFF_QR = OFF_QV + QV_BYTES;
     static constexpr int OFF_STAGE = OFF_QR + QR_BYTES;
     static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
-    static constexpr int N_BARS = 2 * NSTAGE + 5;
+    static constexpr int N_BARS = 2 * NSTAGE + 6;
     static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
-    // tensor-memory columns: S (64; P overwrites its first 32), O (DV)
-    static constexpr int COL_S = 0, COL_O = TILE;
-    static constexpr int TMEM_COLS = (TILE + DV) <= 128 ? 128 : 256;
+    // tensor-memory columns: S0, S1 (64 each; P overwrites the first 32 of its S), O (DV)
+    static constexpr int COL_S = 0, COL_O = 2 * TILE;
+    static constexpr int TMEM_COLS = 256;
+    static_assert(2 * TILE + DV <= TMEM_COLS, "S0, S1 and O must fit the allocation");
     static constexpr int BLOCKS_PER_SM = 512 / TMEM_COLS;
     static constexpr int KSTEPS_V = DV / 16, KSTEPS_R = DR / 16;
     static constexpr int THREADS = 192;
@@ -115,6 +115,16 @@ __device__ __forceinline__ void tmem_st16_nowait(uint32_t taddr, const uint32_t 
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n" ::"r"(taddr),
         "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
         "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32u_nowait(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n" ::"r"(taddr),
+        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+        "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]),
+        "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]),
+        "r"(v[31])
         : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
@@ -204,6 +214,11 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
+// Bounded wait for the softmax warps, whose barriers are normally complete already: a bare poll first.
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_bounded(bar, parity, abort_flag);
+}
 // Bounded wait whose polls sleep in hardware (suspend-time hint) instead of spinning through the issue slots.
 __device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     unsigned long long t0 = 0;
@@ -215,6 +230,7 @@ __device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, 
             : "r"(bar), "r"(parity), "r"(20000u)
             : "memory");
         if (ok) return true;
+        __nanosleep(64);
         if ((it & 7u) == 7u) {
             if (*abort_flag) return false;
             const unsigned long long now = global_timer_ns();
@@ -259,8 +275,9 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     const uint32_t bar0 = s_base + T::OFF_BAR;
     auto kv_full = [&](int s) { return bar0 + 8u * s; };
     auto kv_empty = [&](int s) { return bar0 + 8u * (NS + s); };
-    const uint32_t s_full = bar0 + 8u * (2 * NS), p_full = bar0 + 8u * (2 * NS + 1), q_ready = bar0 + 8u * (2 * NS + 2),
-                   drain = bar0 + 8u * (2 * NS + 3), o_full = bar0 + 8u * (2 * NS + 4);
+    auto s_full = [&](int i) { return bar0 + 8u * (2 * NS + i); };
+    const uint32_t p_full = bar0 + 8u * (2 * NS + 2), q_ready = bar0 + 8u * (2 * NS + 3), drain = bar0 + 8u * (2 * NS + 4),
+                   o_full = bar0 + 8u * (2 * NS + 5);
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + T::N_BARS);
     volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
 
@@ -269,7 +286,8 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             mbar_init(kv_full(s), 1);
             mbar_init(kv_empty(s), 1);
         }
-        mbar_init(s_full, 1);
+        mbar_init(s_full(0), 1);
+        mbar_init(s_full(1), 1);
         mbar_init(p_full, T::ROWS);
         mbar_init(q_ready, T::ROWS);
         mbar_init(drain, 1);
@@ -324,41 +342,35 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
 
         float m_run = -INFINITY, l_run = 0.f;          // softmax reference (log2 domain) and sum relative to it
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        const uint32_t s_addr = lane_base + T::COL_S, o_addr = lane_base + T::COL_O;
+        const uint32_t o_addr = lane_base + T::COL_O;
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
-            // S of tile j is complete, and with it every MMA issued before it: O holds tiles 0..j-1
-            if (!mbar_wait_sleepy(s_full, j & 1, s_abort)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait_spin(s_full(j & 1), (j >> 1) & 1, s_abort))) { ok = false; break; }   // warp-uniform
             tc_fence_after();
+            const uint32_t s_addr = lane_base + T::COL_S + (j & 1) * T::TILE;
+            float s[T::TILE];
+            {
+                float lo[32], hi[32];
+                tmem_ld32_nowait(s_addr, lo);
+                tmem_ld32_nowait(s_addr + 32, hi);
+                tmem_ld_wait();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) { s[c] = lo[c]; s[32 + c] = hi[c]; }
+            }
             const int limit = pos - j * T::TILE;              // columns c > limit are in the future of this row
-            const bool diag = limit < T::TILE - 1;
-            // ---- pass 1: the row maximum ----
+            if (limit < T::TILE - 1) {
+#pragma unroll
+                for (int c = 0; c < T::TILE; ++c) s[c] = (c > limit) ? -INFINITY : s[c];
+            }
             float mx[4];
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                float u[32];
-                tmem_ld32_nowait(s_addr + hf * 32, u);
-                tmem_ld_wait();
-                if (diag) {
+            for (int k = 0; k < 4; ++k) mx[k] = max3(s[k], s[k + 4], s[k + 8]);
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) u[c] = (hf * 32 + c > limit) ? -INFINITY : u[c];
-                }
-                if (hf == 0) {
+            for (int c = 12; c + 8 <= T::TILE; c += 8)
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) mx[k] = max3(u[k], u[k + 4], u[k + 8]);
+                for (int k = 0; k < 4; ++k) mx[k] = max3(mx[k], s[c + k], s[c + 4 + k]);
 #pragma unroll
-                    for (int c = 12; c + 8 <= 32; c += 8)
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) mx[k] = max3(mx[k], u[c + k], u[c + 4 + k]);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) mx[k] = fmaxf(mx[k], u[28 + k]);
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 32; c += 8)
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) mx[k] = max3(mx[k], u[c + k], u[c + 4 + k]);
-                }
-            }
+            for (int k = 0; k < 4; ++k) mx[k] = fmaxf(mx[k], s[T::TILE - 4 + k]);
             const float m_tile = max3(mx[0], mx[1], fmaxf(mx[2], mx[3])) * p.scale_log2;
             // The reference m_run of the row only moves when the tile's maximum exceeds it by more than 2^8: the
             // weights stay below 256 relative to it, the result is the same quotient, and the accumulated O (which
@@ -372,8 +384,10 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                 m_run = m_tile;
             }
             // tcgen05.ld / tcgen05.st are warp-wide instructions: when any row of the warp moves its reference, every
-            // lane rescales its row of O (by 1 where nothing moved)
+            // lane rescales its row of O (by 1 where nothing moved), once the value product of tile j-1 has landed
             if (j > 0 && __any_sync(0xffffffffu, move)) {
+                if (!__all_sync(0xffffffffu, mbar_wait_spin(kv_empty((j - 1) % NS), ((j - 1) / NS) & 1, s_abort))) { ok = false; break; }
+                tc_fence_after();
                 const uint64_t al2 = f2_pack(alpha, alpha);
 #pragma unroll
                 for (int part = 0; part < DV / 32; ++part) {
@@ -385,36 +399,19 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                     tmem_st32(o_addr + part * 32, o);
                 }
             }
-            // ---- pass 2: weights, row sum, P over the first 32 columns of S (both halves of S are in registers or
-            //      consumed before their columns are overwritten: half 0 is read before P of half 0 is stored, and
-            //      P of half 1 lands in columns 16..31, which belong to half 0) ----
+            // ---- weights, row sum, P over the first 32 columns of this tile's S (the row's only reader is this thread) ----
             const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nm2 = f2_pack(-m_run, -m_run);
             uint64_t sum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
+            uint32_t pk[T::TILE / 2];
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                float s[32];
-                tmem_ld32_nowait(s_addr + hf * 32, s);
-                tmem_ld_wait();
-                if (diag) {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) s[c] = (hf * 32 + c > limit) ? -INFINITY : s[c];
-                }
-                uint32_t pk[16];
-#pragma unroll
-                for (int c = 0; c < 32; c += 2) {
-                    float t0, t1;
-                    f2_unpack(f2_fma(f2_pack(s[c], s[c + 1]), sc2, nm2), t0, t1);
-                    const float e0 = fast_exp2(t0), e1 = fast_exp2(t1);
-                    sum2[(c >> 1) & 1] = f2_add(sum2[(c >> 1) & 1], f2_pack(e0, e1));
-                    pk[c >> 1] = pack_bf16(e0, e1);
-                }
-                if (hf == 0) {
-                    // half 1 of S must be in registers before columns 16..31 can be overwritten; columns 0..15 are free now
-                    tmem_st16_nowait(s_addr, pk);
-                } else {
-                    tmem_st16_nowait(s_addr + 16, pk);
-                }
+            for (int c = 0; c < T::TILE; c += 2) {
+                float t0, t1;
+                f2_unpack(f2_fma(f2_pack(s[c], s[c + 1]), sc2, nm2), t0, t1);
+                const float e0 = fast_exp2(t0), e1 = fast_exp2(t1);
+                sum2[(c >> 1) & 1] = f2_add(sum2[(c >> 1) & 1], f2_pack(e0, e1));
+                pk[c >> 1] = pack_bf16(e0, e1);
             }
+            tmem_st32u_nowait(s_addr, pk);
             float sa, sb;
             f2_unpack(f2_add(sum2[0], sum2[1]), sa, sb);
             l_run += sa + sb;
@@ -433,7 +430,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             tc_fence_before();
             mbar_arrive(p_full);
         }
-        if (ok && !mbar_wait_sleepy(o_full, 0, s_abort)) ok = false;
+        if (ok && !__all_sync(0xffffffffu, mbar_wait_spin(o_full, 0, s_abort))) ok = false;
         if (ok) {
             tc_fence_after();
             // (tcgen05.ld is a warp-wide instruction: every lane takes part, dead rows only skip the stores)
@@ -498,35 +495,42 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             constexpr uint32_t kr_sbo = 8 * T::KR_ROW;
             bool ok = mbar_wait_sleepy(q_ready, 0, s_abort);
             int issued_mma = 0;
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                // score product of tile j: overwrites S and the P of tile j-1 inside it, so the value product of tile
-                // j-1 must have completed (MMAs with different accumulators are not ordered among themselves)
-                const int st = j % NS;
-                if (!mbar_wait_sleepy(kv_full(st), (j / NS) & 1, s_abort)) { ok = false; break; }
-                if (j > 0 && !mbar_wait_sleepy(kv_empty((j - 1) % NS), ((j - 1) / NS) & 1, s_abort)) { ok = false; break; }
+            // score product of tile t into S[t & 1].  That buffer also holds the P of tile t-2, so the value product of
+            // tile t-2 must have completed (MMAs with different accumulators are not ordered among themselves).
+            auto score = [&](int t) -> bool {
+                const int st = t % NS;
+                if (!mbar_wait_sleepy(kv_full(st), (t / NS) & 1, s_abort)) return false;
+                if (t >= 2 && !mbar_wait_sleepy(kv_empty((t - 2) % NS), ((t - 2) / NS) & 1, s_abort)) return false;
                 tc_fence_after();
                 const uint32_t vb = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
+                const uint32_t d = tmem + T::COL_S + (t & 1) * T::TILE;
 #pragma unroll
                 for (int ks = 0; ks < T::KSTEPS_V; ++ks) {
                     const uint32_t off = (ks >> 2) * T::QBOX_BYTES + (ks & 3) * 32;
                     const uint32_t voff = (ks >> 2) * T::VBOX_BYTES + (ks & 3) * 32;
-                    umma_bf16(tmem + T::COL_S, smem_desc(s_base + T::OFF_QV + off, 16, 1024, kSwz128),
-                              smem_desc(vb + voff, 16, 1024, kSwz128), idesc_s, ks > 0);
+                    umma_bf16(d, smem_desc(s_base + T::OFF_QV + off, 16, 1024, kSwz128), smem_desc(vb + voff, 16, 1024, kSwz128),
+                              idesc_s, ks > 0);
                 }
 #pragma unroll
                 for (int ks = 0; ks < T::KSTEPS_R; ++ks)
-                    umma_bf16(tmem + T::COL_S, smem_desc(s_base + T::OFF_QR + ks * 32, 16, kr_sbo, kr_swz),
+                    umma_bf16(d, smem_desc(s_base + T::OFF_QR + ks * 32, 16, kr_sbo, kr_swz),
                               smem_desc(vb + T::V_BYTES + ks * 32, 16, kr_sbo, kr_swz), idesc_s, 1);
-                umma_commit(s_full);
+                umma_commit(s_full(t & 1));
                 ++issued_mma;
+                return true;
+            };
+            if (ok) ok = score(0);
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                if (j + 1 < n_tiles && !score(j + 1)) { ok = false; break; }   // runs while the softmax warps work on tile j
                 // value product of tile j: O += P V once every row has stored P (and finished any rescaling of O)
                 if (!mbar_wait_sleepy(p_full, j & 1, s_abort)) { ok = false; break; }
                 tc_fence_after();
+                const uint32_t vb = s_base + T::OFF_STAGE + (j % NS) * T::STAGE_BYTES;
 #pragma unroll
                 for (int ks = 0; ks < T::TILE / 16; ++ks)
-                    umma_bf16_ts(tmem + T::COL_O, tmem + T::COL_S + ks * 8,
+                    umma_bf16_ts(tmem + T::COL_O, tmem + T::COL_S + (j & 1) * T::TILE + ks * 8,
                                  smem_desc(vb + ks * 16 * 128, T::VBOX_BYTES, 1024, kSwz128), idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
-                umma_commit(kv_empty(st));
+                umma_commit(kv_empty(j % NS));
             }
             if (ok) umma_commit(o_full);
             if (!ok && !*s_abort) {
