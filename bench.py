@@ -452,12 +452,16 @@ def load_tensor_peak():
     return 1590.0, "fallback (1.59 PFLOP/s, earlier measurement on this pool)"
 
 
-def measure_prefill(rank, local_rank, dist, args, torch, gb, harness, B=8, T=8192):
+def measure_prefill(rank, local_rank, dist, args, torch, gb, harness, B=8, T=8192, wide=False):
     """Whole-prompt prefill on the headline head shape: gva_absorb_query + gva_append_chunk + gva_prefill, and the
     attention kernel alone against the tensor roofline (flops of the absorbed form under the causal mask)."""
     from paper_2609_13285_b200 import multirank, workloads as wl
     dev = torch.device("cuda", local_rank)
-    pc = wl.prefill_bench_case(seed=wl.MASTER_SEED + 7100 + 7919 * rank, B=B, T=T)
+    if wide:
+        pc = wl.prefill_bench_case_b(seed=wl.MASTER_SEED + 7200 + 7919 * rank, B=B, T=T)
+    else:
+        pc = wl.prefill_bench_case(seed=wl.MASTER_SEED + 7100 + 7919 * rank, B=B, T=T)
+    sh = pc.cache.shape
     pd = harness.upload_prefill(pc, device=dev)
     stream = torch.cuda.current_stream()
     steps, warmup = max(5, min(30, args.steps // 10)), 3
@@ -494,12 +498,12 @@ def measure_prefill(rank, local_rank, dist, args, torch, gb, harness, B=8, T=819
     peak, src = load_tensor_peak()
     flops = pc.flops()
     tf = flops / (attn_ms * 1e-3) / 1e12
-    res = {"workload": f"whole-prompt prefill, H=16 G=4 d_v=64 d_c=64 d_r=16, B={B} prompts of T={T} tokens, bf16 cache in "
+    res = {"workload": f"whole-prompt prefill, H={sh.H} G={sh.G} d_v={sh.d_v} d_c={sh.d_c} d_r={sh.d_r}, B={B} prompts of T={T} tokens, bf16 cache in "
                        "64-token pages (permuted block table), L2 flushed between timed calls",
            "prefill_tokens_per_s": B * T / (whole_ms * 1e-3), "ms_per_step": whole_ms,
            "gva_prefill_ms_per_call": attn_ms, "steps": steps, "device_status": status,
            "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
-                        "traffic": None, "peak_source": src, "kernel": "prefill_kernel<64,16> (tcgen05 score and value products)",
+                        "traffic": None, "peak_source": src, "kernel": f"prefill_kernel<{sh.d_v},{sh.d_r}> (tcgen05 score and value products)",
                         "algorithmic_flops_per_launch": flops, "avg_launch_ms": attn_ms,
                         "note": "flops = 2 * causal pairs * H * (2 d_v + d_r); bf16 operands, f32 accumulate"}}
     pd.close()
@@ -544,13 +548,14 @@ def main() -> None:
     kernel = {"auto": gb.GVA_KERNEL_AUTO, "fma": gb.GVA_KERNEL_FMA, "mma": gb.GVA_KERNEL_MMA}[args.kernel]
 
     name = args.workload
-    if name in ("prefill", "prefill-ncu", "layer"):      # side workloads on their own (small runs for profiler captures)
+    if name in ("prefill", "prefill-ncu", "prefill-wide", "layer"):      # side workloads on their own (small runs for profiler captures)
         if rank == 0:
             if name == "layer":
                 res = measure_layer(rank, local_rank, None, args, kernel, torch, gb, harness)
             else:
                 res = measure_prefill(rank, local_rank, None, args, torch, gb, harness,
-                                      **({"B": 4, "T": 4096} if name == "prefill-ncu" else {}))
+                                      **({"B": 4, "T": 4096} if name == "prefill-ncu" else
+                                         {"B": 4, "T": 8192, "wide": True} if name == "prefill-wide" else {}))
             print(json.dumps({"workload": name, **res}))
         if dist is not None:
             dist.barrier()
@@ -586,6 +591,7 @@ def main() -> None:
         others["gqa_matched_cfg2"] = gq
         others["layer_step_cfg2"] = measure_layer(rank, local_rank, dist, short, kernel, torch, gb, harness)
         others["prefill"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness)
+        others["prefill_wide"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness, B=4, T=8192, wide=True)
 
     if rank == 0:
         case = r["case"]

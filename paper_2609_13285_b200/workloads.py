@@ -340,6 +340,11 @@ def prefill_bench_case(seed: int = MASTER_SEED + 7100, B: int = 8, T: int = 8192
     return make_prefill_case("prefill", SHAPE_A, [0] * B, [T] * B, page_size=64, seed=seed)
 
 
+def prefill_bench_case_b(seed: int = MASTER_SEED + 7200, B: int = 4, T: int = 8192) -> PrefillCase:
+    """Whole-prompt prefill on the wider head shape (H=32, G=8, d_v=128, d_c=128, d_r=32)."""
+    return make_prefill_case("prefill_b", SHAPE_B, [0] * B, [T] * B, page_size=64, seed=seed)
+
+
 def layer_weights(shape: HeadShape, d_model: int, B: int, seed: int = MASTER_SEED + 6000) -> dict:
     """Seeded projections around the attention of one layer and one hidden state per sequence.
     Every weight ~ N(0, 1/fan_in) (so projected activations stay unit-scale), x ~ N(0, 1):

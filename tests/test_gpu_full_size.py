@@ -90,3 +90,43 @@ def test_config4_two_layers_full_batch():
             assert np.max(np.abs(o[sample] - ref[sample])) <= 5e-5
         finally:
             dc.close()
+
+
+@pytest.mark.parametrize("shape_name", ["A", "B"])
+def test_prefill_bench_size_sampled_rows(shape_name):
+    # bench.py's prefill workload, same launch: a sample of query rows (first / last rows, tile and block edges, random
+    # ones) is checked one by one against the decode oracle over the row's prefix (a prefill row IS one decode step over
+    # its prefix -- pinned in the CPU tests); every other row is covered by finiteness and the Gaussian-tilting statistic
+    from oracle import gva_oracle as orc
+    pc = wl.prefill_bench_case() if shape_name == "A" else wl.prefill_bench_case_b()
+    c, s = pc.cache, pc.cache.shape
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        out, lse = pd.prefill()
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out.cpu().numpy().astype(np.float64)
+        l = lse.cpu().numpy().astype(np.float64)
+        q_abs = pd.q_abs.cpu().numpy().astype(np.float64)
+    finally:
+        pd.close()
+    assert np.isfinite(o).all() and np.isfinite(l).all()
+    T = int(pc.q_lens[0])
+    rng = np.random.default_rng(7)
+    for b in (0, c.B - 1):
+        toks = sorted(set([0, 1, 31, 32, 63, 64, 65, 127, 128, 4095, 4096, T - 33, T - 32, T - 2, T - 1] +
+                          rng.integers(0, T, size=6).tolist()))
+        for t in toks:
+            n = int(pc.cu_q[b]) + t
+            lens = np.zeros(c.B, dtype=np.int32); lens[b] = t + 1
+            qa = np.zeros((c.B, s.H, s.d_v + s.d_r)); qa[b] = q_abs[n]
+            ref_o, ref_l = orc.decode(c.v_pool, c.kr_pool, c.block_table, lens, qa, s.H, d_c=s.d_c)
+            assert np.max(np.abs(o[n] - ref_o[b])) <= 2e-2, (b, t)
+            assert np.max(np.abs(l[n] - ref_l[b])) <= 2e-2, (b, t)
+    # rows with a long prefix: the softmax-weighted mean of N(0, I) rows sits near q~ / sqrt(d_qk)
+    target = q_abs[..., :s.d_v] / np.sqrt(s.d_c + s.d_r)
+    # (tens of millions of components here, so the bound is on a high quantile and the maximum only has to stay sane)
+    far = pc.q_pos >= 4096
+    dev = np.abs(o[far] - target[far])
+    assert np.quantile(dev, 0.9999) < 0.2 and dev.max() < 1.0
