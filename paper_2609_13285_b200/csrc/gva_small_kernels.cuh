@@ -162,6 +162,92 @@ absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, cons
     absorb_block(q_c, q_r, M, q_pos, q_abs, B, H, d_v, d_c, d_r, rope, blockIdx.x, blockIdx.y * kAbsorbBatch, smem_f);
 }
 
+// ---- absorb for many rows (prefill: one row per new token) -----------------------------------------
+// grid (H, blocks per head), block 256.  Thread t keeps row i = t % DV of M_h in registers for the whole block and
+// serves the rows r with r % (256 / DV) == t / DV of every chunk; query rows stream through a double-buffered
+// shared-memory chunk (cp.async) and are read as broadcasts.  Each output is the same j-ordered chain of fused
+// multiply-adds as in absorb_block, so both kernels give identical bits.
+constexpr int kAbsorbChunk = 32;          // query rows per chunk
+template <int DV, int DC>
+__global__ void __launch_bounds__(kAbsorbThreads)
+absorb_rows_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, const float *__restrict__ M,
+                   const int32_t *__restrict__ q_pos, float *__restrict__ q_abs, int B, int H, int d_r, int rows_per_block,
+                   RopeTable rope) {
+    constexpr int NG = kAbsorbThreads / DV;            // row groups
+    constexpr int RPT = kAbsorbChunk / NG;             // rows per thread and chunk
+    static_assert(kAbsorbThreads % DV == 0 && kAbsorbChunk % NG == 0 && RPT % 4 == 0 && DC % 4 == 0, "tiling");
+    grid_dependency_launch();
+    __shared__ __align__(16) float sq[2][kAbsorbChunk][DC];
+    const int tid = threadIdx.x, h = blockIdx.x;
+    const int i = tid % DV, grp = tid / DV;
+    const int row0 = blockIdx.y * rows_per_block;
+    const int row1 = min(B, row0 + rows_per_block);
+    grid_dependency_wait();
+    if (row0 >= row1) return;
+    float m[DC];
+    {
+        const float4 *src = reinterpret_cast<const float4 *>(M + ((size_t)h * DV + i) * DC);
+#pragma unroll
+        for (int j = 0; j < DC / 4; ++j) {
+            const float4 v = __ldg(src + j);
+            m[4 * j] = v.x; m[4 * j + 1] = v.y; m[4 * j + 2] = v.z; m[4 * j + 3] = v.w;
+        }
+    }
+    const int dq = DV + d_r, half = d_r / 2;
+    auto stage = [&](int buf, int r0) {
+        const int n = min(kAbsorbChunk, row1 - r0);
+        const uint32_t dst = smem_u32(&sq[buf][0][0]);
+        for (int c = tid; c < n * (DC / 4); c += kAbsorbThreads) {
+            const int rr = c / (DC / 4), col = c % (DC / 4);
+            cp_async16(dst + (rr * DC + col * 4) * 4, q_c + ((size_t)(r0 + rr) * H + h) * DC + col * 4, 16);
+        }
+        cp_async_commit();
+    };
+    stage(0, row0);
+    int buf = 0;
+    for (int r0 = row0; r0 < row1; r0 += kAbsorbChunk, buf ^= 1) {
+        const int n = min(kAbsorbChunk, row1 - r0);
+        if (r0 + kAbsorbChunk < row1) stage(buf ^ 1, r0 + kAbsorbChunk);
+        else cp_async_commit();
+        // the positional slices of this chunk: one rotation pair per thread and pass, in fp64
+        for (int e = tid; e < n * half; e += kAbsorbThreads) {
+            const int rr = e / half, k = e % half;
+            const size_t src = ((size_t)(r0 + rr) * H + h) * d_r + 2 * k;
+            double y0, y1;
+            rope_pair((double)q_r[src], (double)q_r[src + 1], q_pos[r0 + rr], rope.inv_freq[k], y0, y1);
+            float *dst = q_abs + ((size_t)(r0 + rr) * H + h) * dq + DV + 2 * k;
+            dst[0] = __double2float_rn(y0);
+            dst[1] = __double2float_rn(y1);
+        }
+        cp_async_wait<1>();
+        __syncthreads();
+#pragma unroll
+        for (int pass = 0; pass < RPT / 4; ++pass) {
+            float a[4] = {0.f, 0.f, 0.f, 0.f};
+            const float4 *p[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) p[k] = reinterpret_cast<const float4 *>(&sq[buf][min(grp + NG * (pass * 4 + k), n - 1)][0]);
+#pragma unroll
+            for (int j = 0; j < DC / 4; ++j) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float4 x = p[k][j];
+                    a[k] = fmaf(x.x, m[4 * j], a[k]);
+                    a[k] = fmaf(x.y, m[4 * j + 1], a[k]);
+                    a[k] = fmaf(x.z, m[4 * j + 2], a[k]);
+                    a[k] = fmaf(x.w, m[4 * j + 3], a[k]);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int rr = grp + NG * (pass * 4 + k);
+                if (rr < n) q_abs[((size_t)(r0 + rr) * H + h) * dq + i] = a[k];
+            }
+        }
+        __syncthreads();        // the chunk is consumed before the copy after next overwrites it
+    }
+}
+
 // ---- append --------------------------------------------------------------------------------------
 // grid B, block 128.  Integer page arithmetic, round-to-nearest-even stores, nothing else touched.
 // The new rows are loaded before the page lookup so that the two dependent lookups (position, then

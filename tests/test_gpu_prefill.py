@@ -178,3 +178,25 @@ def test_prefill_reports_bad_page_and_long_sequence():
         assert st & 0xff == gb.GVA_ERR_SEQ_LEN and st >> 8 == 1
     finally:
         pd.close()
+
+
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+def test_absorb_many_rows_matches_oracle_and_the_small_batch_kernel(shape):
+    # prefill absorbs one row per new token: above 512 rows a kernel that streams the rows takes over; it must give
+    # the oracle's values and the very bits of the decode-batch kernel (same chain of fused multiply-adds per output)
+    n = 1000 + 37
+    pc = wl.make_prefill_case("abs", shape, [3], [n], page_size=64, seed=509)
+    pd = harness.upload_prefill(pc)
+    try:
+        q = pd.absorb().cpu().numpy()
+        ref = orc.absorb(pc.q_c, pc.q_r, pc.cache.M, pc.q_pos)
+        assert np.max(np.abs(q.astype(np.float64) - ref)) <= 1e-5
+        assert np.array_equal(q[..., shape.d_v:], ref[..., shape.d_v:].astype(np.float32))      # fp64 rotation, one rounding
+        small = torch.empty_like(pd.q_abs)
+        for lo in range(0, n, 100):
+            hi = min(n, lo + 100)
+            gb.gva_absorb_query(pd.handle, pd.q_c[lo:hi], pd.q_r[lo:hi], pd.dc.M, pd.q_pos[lo:hi], small[lo:hi], hi - lo)
+        torch.cuda.synchronize()
+        assert np.array_equal(small.cpu().numpy().view(np.uint32), q.view(np.uint32))
+    finally:
+        pd.close()
