@@ -21,8 +21,9 @@
 //     O        += P_j V_j            tcgen05.mma, A = P from tensor memory, B = the same value tile as an MN-major operand
 //     O accumulates in tensor memory across tiles.  The softmax reference of a row moves only when the running
 //     maximum grows by more than 2^8; only then is that row of O rescaled (read, multiplied, written back).
-//   S is double-buffered, so the score product of tile j + 1 and the value product of tile j - 1 run while the
-//   softmax warps work on tile j; two blocks share an SM (256 tensor-memory columns each).  Shared memory carries
+//   S has two buffers, so the score product of tile j + 1 runs while the softmax warps work on tile j; for d_v = 64
+//   the query tile lives in tensor memory too, so every MMA reads only its B operand (the cache tile) from shared
+//   memory; two blocks share an SM (256 tensor-memory columns each).  Shared memory carries
 //   only the operands the tensor core reads (Q and the cache tiles): P never touches it.
 //   Every wait is bounded; on expiry the block records GVA_ERR_TIMEOUT, drains what it issued, frees its
 //   tensor memory and exits.
@@ -63,12 +64,17 @@ struct PrefillTraits {
     static constexpr int OFF_QR = OFF_QV + QV_BYTES;
     static constexpr int OFF_STAGE = OFF_QR + QR_BYTES;
     static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
-    static constexpr int N_BARS = 2 * NSTAGE + 6;
+    static constexpr int N_BARS = 2 * NSTAGE + 7;
     static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
-    // tensor-memory columns: S0, S1 (64 each; P overwrites the first 32 of its S), O (DV)
-    static constexpr int COL_S = 0, COL_O = 2 * TILE;
+    // tensor-memory columns: two score buffers (64 each; P overwrites the first 32 of its S), O (DV) and, where it
+    // fits (d_v = 64), the query tile Q as bf16 pairs ((DV + DR) / 2): an MMA whose A operand comes from tensor memory
+    // reads only B from shared memory (measured: 128 x 64 x 16 MMAs with both operands in shared memory run at 62
+    // cycles each -- the 6 KB of operands per MMA at ~97 B/clk -- against 32 with A in tensor memory)
     static constexpr int TMEM_COLS = 256;
-    static_assert(2 * TILE + DV <= TMEM_COLS, "S0, S1 and O must fit the allocation");
+    static constexpr int NSBUF = 2;
+    static constexpr int COL_S = 0, COL_O = NSBUF * TILE, COL_Q = COL_O + DV;
+    static constexpr bool Q_IN_TMEM = COL_Q + (DV + DR) / 2 <= TMEM_COLS;
+    static_assert(NSBUF * TILE + DV <= TMEM_COLS, "the score buffers and O must fit the allocation");
     static constexpr int BLOCKS_PER_SM = 512 / TMEM_COLS;
     static constexpr int KSTEPS_V = DV / 16, KSTEPS_R = DR / 16;
     static constexpr int THREADS = 192;
@@ -126,6 +132,11 @@ __device__ __forceinline__ void tmem_st32u_nowait(uint32_t taddr, const uint32_t
         "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]),
         "r"(v[31])
         : "memory");
+}
+__device__ __forceinline__ void tmem_st8_nowait(uint32_t taddr, const uint32_t (&v)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n" ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]),
+                 "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
@@ -208,6 +219,31 @@ __device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
     asm("mul.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+// 2^t for a pair of arguments without the special-function unit: t = n + f with n the nearest integer (magic-number
+// rounding), 2^f by a cubic on [-1/2, 1/2] (relative error 7.5e-5, far below the bf16 rounding of the weights that
+// follows), 2^n by adding n to the exponent field.  Arguments are clamped at -126 (the result is then ~1e-38, i.e. 0
+// for a softmax weight); the caller guarantees t <= 8 + log2(64).
+__device__ __forceinline__ void exp2_pair_fma(float t0, float t1, float &e0, float &e1) {
+    const float kMagic = 12582912.f;                         // 1.5 * 2^23: adding it rounds to the nearest integer
+    t0 = fmaxf(t0, -126.f);
+    t1 = fmaxf(t1, -126.f);
+    const uint64_t t2 = f2_pack(t0, t1);
+    const uint64_t r2 = f2_add(t2, f2_pack(kMagic, kMagic));
+    const uint64_t n2 = f2_add(r2, f2_pack(-kMagic, -kMagic));
+    const uint64_t f2 = f2_fma(n2, f2_pack(-1.f, -1.f), t2);
+    uint64_t p2 = f2_fma(f2, f2_pack(0.0551716648f, 0.0551716648f), f2_pack(0.2426111251f, 0.2426111251f));
+    p2 = f2_fma(p2, f2, f2_pack(0.6932609677f, 0.6932609677f));
+    p2 = f2_fma(p2, f2, f2_pack(0.9999280572f, 0.9999280572f));
+    float r0, r1, p0, p1;
+    f2_unpack(r2, r0, r1);
+    f2_unpack(p2, p0, p1);
+    e0 = __uint_as_float(__float_as_uint(r0) * 0x00800000u + __float_as_uint(p0));   // low mantissa bits of r hold n
+    e1 = __uint_as_float(__float_as_uint(r1) * 0x00800000u + __float_as_uint(p1));
+}
+#ifndef GVA_PREFILL_EMU_EVERY
+#define GVA_PREFILL_EMU_EVERY 0     // build-time knob: every n-th pair of exponentials runs on the FMA pipe (0 = none;
+                                    // measured slower at 4, 3 and 2: the XU pipe is not what the warps wait for)
+#endif
 constexpr float kRescaleLog2 = 8.f;   // the softmax reference moves only when the running maximum grows by more than 2^8
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
@@ -276,8 +312,9 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     auto kv_full = [&](int s) { return bar0 + 8u * s; };
     auto kv_empty = [&](int s) { return bar0 + 8u * (NS + s); };
     auto s_full = [&](int i) { return bar0 + 8u * (2 * NS + i); };
-    const uint32_t p_full = bar0 + 8u * (2 * NS + 2), q_ready = bar0 + 8u * (2 * NS + 3), drain = bar0 + 8u * (2 * NS + 4),
-                   o_full = bar0 + 8u * (2 * NS + 5);
+    const uint32_t p_full = bar0 + 8u * (2 * NS + 3), q_ready = bar0 + 8u * (2 * NS + 4), drain = bar0 + 8u * (2 * NS + 5),
+                   o_full = bar0 + 8u * (2 * NS + 6);
+    constexpr int NB = T::NSBUF;
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + T::N_BARS);
     volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
 
@@ -288,6 +325,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         }
         mbar_init(s_full(0), 1);
         mbar_init(s_full(1), 1);
+        mbar_init(s_full(2), 1);
         mbar_init(p_full, T::ROWS);
         mbar_init(q_ready, T::ROWS);
         mbar_init(drain, 1);
@@ -313,41 +351,59 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         const int h = g * kHeadsPerGroup + hl;
         const bool live = tok < nv;
         const int pos = p0 + tok;
-        // ---- stage Q: f32 -> bf16, swizzled K-major rows (value dims in 128-byte boxes, then the RoPE dims) ----
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        // ---- stage Q as bf16: into tensor memory (row = lane, two values per column) or, where that does not fit,
+        //      into shared memory as swizzled K-major rows (value dims in 128-byte boxes, then the RoPE dims) ----
         {
             const float4 *src = reinterpret_cast<const float4 *>(p.q_abs + ((size_t)(q_begin + q0 + tok) * p.H + h) * (DV + DR));
+            if constexpr (T::Q_IN_TMEM) {
 #pragma unroll
-            for (int c = 0; c < DV / 8; ++c) {
-                float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
-                if (live) {
-                    a = __ldg(src + 2 * c);
-                    bq = __ldg(src + 2 * c + 1);
-                }
-                *reinterpret_cast<uint4 *>(smem + T::OFF_QV + (c >> 3) * T::QBOX_BYTES + swz128(r, c & 7)) =
-                    make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(bq.x, bq.y), pack_bf16(bq.z, bq.w));
-            }
+                for (int part = 0; part < (DV + DR) / 16; ++part) {      // 16 values = 8 columns per step
+                    uint32_t w[8];
 #pragma unroll
-            for (int c = 0; c < DR / 8; ++c) {
-                float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
-                if (live) {
-                    a = __ldg(src + DV / 4 + 2 * c);
-                    bq = __ldg(src + DV / 4 + 2 * c + 1);
+                    for (int c = 0; c < 4; ++c) {
+                        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (live) a = __ldg(src + part * 4 + c);
+                        w[2 * c] = pack_bf16(a.x, a.y);
+                        w[2 * c + 1] = pack_bf16(a.z, a.w);
+                    }
+                    tmem_st8_nowait(lane_base + T::COL_Q + part * 8, w);
                 }
-                *reinterpret_cast<uint4 *>(smem + T::OFF_QR + swz_kr<T::KR_ROW>(r, c)) =
-                    make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(bq.x, bq.y), pack_bf16(bq.z, bq.w));
+                tmem_st_wait();
+                tc_fence_before();
+            } else {
+#pragma unroll
+                for (int c = 0; c < DV / 8; ++c) {
+                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
+                    if (live) {
+                        a = __ldg(src + 2 * c);
+                        bq = __ldg(src + 2 * c + 1);
+                    }
+                    *reinterpret_cast<uint4 *>(smem + T::OFF_QV + (c >> 3) * T::QBOX_BYTES + swz128(r, c & 7)) =
+                        make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(bq.x, bq.y), pack_bf16(bq.z, bq.w));
+                }
+#pragma unroll
+                for (int c = 0; c < DR / 8; ++c) {
+                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
+                    if (live) {
+                        a = __ldg(src + DV / 4 + 2 * c);
+                        bq = __ldg(src + DV / 4 + 2 * c + 1);
+                    }
+                    *reinterpret_cast<uint4 *>(smem + T::OFF_QR + swz_kr<T::KR_ROW>(r, c)) =
+                        make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(bq.x, bq.y), pack_bf16(bq.z, bq.w));
+                }
+                fence_async_smem();
             }
-            fence_async_smem();
             mbar_arrive(q_ready);
         }
 
         float m_run = -INFINITY, l_run = 0.f;          // softmax reference (log2 domain) and sum relative to it
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
         const uint32_t o_addr = lane_base + T::COL_O;
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
-            if (!__all_sync(0xffffffffu, mbar_wait_spin(s_full(j & 1), (j >> 1) & 1, s_abort))) { ok = false; break; }   // warp-uniform
+            if (!__all_sync(0xffffffffu, mbar_wait_spin(s_full(j % NB), (j / NB) & 1, s_abort))) { ok = false; break; }   // warp-uniform
             tc_fence_after();
-            const uint32_t s_addr = lane_base + T::COL_S + (j & 1) * T::TILE;
+            const uint32_t s_addr = lane_base + T::COL_S + (j % NB) * T::TILE;
             float s[T::TILE];
             {
                 float lo[32], hi[32];
@@ -362,6 +418,33 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
 #pragma unroll
                 for (int c = 0; c < T::TILE; ++c) s[c] = (c > limit) ? -INFINITY : s[c];
             }
+            uint32_t pk[T::TILE / 2];
+            float tile_sum = 0.f;
+            // weights and their sum relative to the reference m_ref; P as bf16 pairs
+            auto weights = [&](float m_ref) {
+                const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nm2 = f2_pack(-m_ref, -m_ref);
+                uint64_t sum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
+#pragma unroll
+                for (int c = 0; c < T::TILE; c += 2) {
+                    float t0, t1, e0, e1;
+                    f2_unpack(f2_fma(f2_pack(s[c], s[c + 1]), sc2, nm2), t0, t1);
+                    if (GVA_PREFILL_EMU_EVERY > 0 && ((c >> 1) % (GVA_PREFILL_EMU_EVERY > 0 ? GVA_PREFILL_EMU_EVERY : 1)) == 1) {
+                        exp2_pair_fma(t0, t1, e0, e1);       // a share of the exponentials can bypass the XU pipe
+                    } else {
+                        e0 = fast_exp2(t0);
+                        e1 = fast_exp2(t1);
+                    }
+                    sum2[(c >> 1) & 1] = f2_add(sum2[(c >> 1) & 1], f2_pack(e0, e1));
+                    pk[c >> 1] = pack_bf16(e0, e1);
+                }
+                float sa, sb;
+                f2_unpack(f2_add(sum2[0], sum2[1]), sa, sb);
+                tile_sum = sa + sb;
+            };
+            // From the second tile on the weights are computed against the current reference at once, while the row
+            // maximum is still being reduced (the two instruction streams are independent); the rare tile whose
+            // maximum moves the reference is redone.
+            if (j > 0) weights(m_run);
             float mx[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) mx[k] = max3(s[k], s[k + 4], s[k + 8]);
@@ -377,44 +460,34 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             // lives in tensor memory) has to be rescaled only then.  (m_tile is finite in tile 0: token 0 is
             // visible to every row.)
             const bool move = m_tile > m_run + kRescaleLog2;
-            float alpha = 1.f;
-            if (move) {
-                alpha = fast_exp2(m_run - m_tile);
-                l_run *= alpha;
-                m_run = m_tile;
-            }
             // tcgen05.ld / tcgen05.st are warp-wide instructions: when any row of the warp moves its reference, every
             // lane rescales its row of O (by 1 where nothing moved), once the value product of tile j-1 has landed
-            if (j > 0 && __any_sync(0xffffffffu, move)) {
-                if (!__all_sync(0xffffffffu, mbar_wait_spin(kv_empty((j - 1) % NS), ((j - 1) / NS) & 1, s_abort))) { ok = false; break; }
-                tc_fence_after();
-                const uint64_t al2 = f2_pack(alpha, alpha);
-#pragma unroll
-                for (int part = 0; part < DV / 32; ++part) {
-                    float o[32];
-                    tmem_ld32_nowait(o_addr + part * 32, o);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) f2_unpack(f2_mul(f2_pack(o[i], o[i + 1]), al2), o[i], o[i + 1]);
-                    tmem_st32(o_addr + part * 32, o);
+            if (j == 0 || __any_sync(0xffffffffu, move)) {
+                float alpha = 1.f;
+                if (move) {
+                    alpha = fast_exp2(m_run - m_tile);
+                    l_run *= alpha;
+                    m_run = m_tile;
                 }
-            }
-            // ---- weights, row sum, P over the first 32 columns of this tile's S (the row's only reader is this thread) ----
-            const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nm2 = f2_pack(-m_run, -m_run);
-            uint64_t sum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
-            uint32_t pk[T::TILE / 2];
+                if (j > 0) {
+                    if (!__all_sync(0xffffffffu, mbar_wait_spin(kv_empty((j - 1) % NS), ((j - 1) / NS) & 1, s_abort))) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t al2 = f2_pack(alpha, alpha);
 #pragma unroll
-            for (int c = 0; c < T::TILE; c += 2) {
-                float t0, t1;
-                f2_unpack(f2_fma(f2_pack(s[c], s[c + 1]), sc2, nm2), t0, t1);
-                const float e0 = fast_exp2(t0), e1 = fast_exp2(t1);
-                sum2[(c >> 1) & 1] = f2_add(sum2[(c >> 1) & 1], f2_pack(e0, e1));
-                pk[c >> 1] = pack_bf16(e0, e1);
+                    for (int part = 0; part < DV / 32; ++part) {
+                        float o[32];
+                        tmem_ld32_nowait(o_addr + part * 32, o);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) f2_unpack(f2_mul(f2_pack(o[i], o[i + 1]), al2), o[i], o[i + 1]);
+                        tmem_st32(o_addr + part * 32, o);
+                    }
+                }
+                weights(m_run);
             }
+            // P goes over the first 32 columns of this tile's S (the row's only reader is this thread)
             tmem_st32u_nowait(s_addr, pk);
-            float sa, sb;
-            f2_unpack(f2_add(sum2[0], sum2[1]), sa, sb);
-            l_run += sa + sb;
+            l_run += tile_sum;
             // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
             if ((long long)(j + 1) * T::TILE > kv_total) {
                 if (tid < T::TILE && (long long)j * T::TILE + tid >= kv_total) {
@@ -493,44 +566,90 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             constexpr uint32_t idesc_o = umma_idesc(T::ROWS, DV, true);
             constexpr uint64_t kr_swz = T::KR_ROW == 32 ? kSwz32 : kSwz64;
             constexpr uint32_t kr_sbo = 8 * T::KR_ROW;
-            bool ok = mbar_wait_sleepy(q_ready, 0, s_abort);
+            bool ok = mbar_wait_spin(q_ready, 0, s_abort);
             int issued_mma = 0;
-            // score product of tile t into S[t & 1].  That buffer also holds the P of tile t-2, so the value product of
-            // tile t-2 must have completed (MMAs with different accumulators are not ordered among themselves).
-            auto score = [&](int t) -> bool {
-                const int st = t % NS;
-                if (!mbar_wait_sleepy(kv_full(st), (t / NS) & 1, s_abort)) return false;
-                if (t >= 2 && !mbar_wait_sleepy(kv_empty((t - 2) % NS), ((t - 2) / NS) & 1, s_abort)) return false;
-                tc_fence_after();
-                const uint32_t vb = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
-                const uint32_t d = tmem + T::COL_S + (t & 1) * T::TILE;
-#pragma unroll
-                for (int ks = 0; ks < T::KSTEPS_V; ++ks) {
-                    const uint32_t off = (ks >> 2) * T::QBOX_BYTES + (ks & 3) * 32;
-                    const uint32_t voff = (ks >> 2) * T::VBOX_BYTES + (ks & 3) * 32;
-                    umma_bf16(d, smem_desc(s_base + T::OFF_QV + off, 16, 1024, kSwz128), smem_desc(vb + voff, 16, 1024, kSwz128),
-                              idesc_s, ks > 0);
+            // One MMA of the score product of tile t (k-step ks) into S[t % NB], and one of the value product of tile t.
+            // Consecutive MMAs on one accumulator wait for each other inside the tensor pipe (measured: ~80 cycles per
+            // 128 x 64 x 16 MMA in a chain against 32 at full rate), so with three score buffers the two chains are
+            // issued interleaved.
+            // Descriptors differ only in their 14-bit start-address field (low word): the high words and the other low
+            // bits are compile-time constants, so one issue costs an add per operand, not a descriptor build.
+            constexpr uint32_t hi128 = (1024u >> 4) | (1u << 14) | ((uint32_t)kSwz128 << 29);      // SBO 1024, version 1, 128-byte swizzle
+            constexpr uint32_t hikr = (kr_sbo >> 4) | (1u << 14) | ((uint32_t)kr_swz << 29);
+            constexpr uint32_t lo_k = (16u >> 4) << 16;                                           // LBO 16 (K-major operands)
+            constexpr uint32_t lo_mn = ((uint32_t)T::VBOX_BYTES >> 4) << 16;                      // LBO = box stride (MN-major value tile)
+            const uint32_t a_qv = ((s_base + T::OFF_QV) & 0x3FFFFu) >> 4, a_qr = ((s_base + T::OFF_QR) & 0x3FFFFu) >> 4;
+            const uint32_t a_st = ((s_base + T::OFF_STAGE) & 0x3FFFFu) >> 4;
+            auto mk = [](uint32_t lo, uint32_t hi) { return (uint64_t)lo | ((uint64_t)hi << 32); };
+            auto score_mma = [&](int t, int ks) {
+                const uint32_t vb = a_st + (uint32_t)(t % NS) * (T::STAGE_BYTES >> 4);
+                const uint32_t d = tmem + T::COL_S + (t % NB) * T::TILE;
+                if (ks < T::KSTEPS_V) {
+                    const uint32_t off = ((ks >> 2) * T::QBOX_BYTES + (ks & 3) * 32) >> 4;
+                    const uint32_t voff = ((ks >> 2) * T::VBOX_BYTES + (ks & 3) * 32) >> 4;
+                    if constexpr (T::Q_IN_TMEM) umma_bf16_ts(d, tmem + T::COL_Q + ks * 8, mk((vb + voff) | lo_k, hi128), idesc_s, ks > 0);
+                    else umma_bf16(d, mk((a_qv + off) | lo_k, hi128), mk((vb + voff) | lo_k, hi128), idesc_s, ks > 0);
+                } else {
+                    const uint32_t kr = (uint32_t)(ks - T::KSTEPS_V) * 2;
+                    if constexpr (T::Q_IN_TMEM) umma_bf16_ts(d, tmem + T::COL_Q + ks * 8, mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
+                    else umma_bf16(d, mk((a_qr + kr) | lo_k, hikr), mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
                 }
-#pragma unroll
-                for (int ks = 0; ks < T::KSTEPS_R; ++ks)
-                    umma_bf16(d, smem_desc(s_base + T::OFF_QR + ks * 32, 16, kr_sbo, kr_swz),
-                              smem_desc(vb + T::V_BYTES + ks * 32, 16, kr_sbo, kr_swz), idesc_s, 1);
-                umma_commit(s_full(t & 1));
-                ++issued_mma;
+            };
+            auto value_mma = [&](int t, int ks) {
+                const uint32_t vb = a_st + (uint32_t)(t % NS) * (T::STAGE_BYTES >> 4);
+                umma_bf16_ts(tmem + T::COL_O, tmem + T::COL_S + (t % NB) * T::TILE + ks * 8,
+                             mk((vb + ks * (16 * 128 >> 4)) | lo_mn, hi128), idesc_o, (t > 0 || ks > 0) ? 1u : 0u);
+            };
+            constexpr int KS_S = T::KSTEPS_V + T::KSTEPS_R, KS_O = T::TILE / 16;
+            // S[t % NB] also holds the P of tile t - NB, so the value product of that tile must have completed before the
+            // score product of tile t is issued (MMAs with different accumulators are not ordered among themselves).
+            auto score_ready = [&](int t) -> bool {
+                if (!mbar_wait_spin(kv_full(t % NS), (t / NS) & 1, s_abort)) return false;
+                if (t >= NB && !mbar_wait_spin(kv_empty((t - NB) % NS), ((t - NB) / NS) & 1, s_abort)) return false;
+                tc_fence_after();
                 return true;
             };
-            if (ok) ok = score(0);
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                if (j + 1 < n_tiles && !score(j + 1)) { ok = false; break; }   // runs while the softmax warps work on tile j
-                // value product of tile j: O += P V once every row has stored P (and finished any rescaling of O)
-                if (!mbar_wait_sleepy(p_full, j & 1, s_abort)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t vb = s_base + T::OFF_STAGE + (j % NS) * T::STAGE_BYTES;
+            // prologue: the score products that run ahead of the softmax
+            for (int t = 0; t < NB - 1 && t < n_tiles && ok; ++t) {
+                ok = score_ready(t);
+                if (!ok) break;
 #pragma unroll
-                for (int ks = 0; ks < T::TILE / 16; ++ks)
-                    umma_bf16_ts(tmem + T::COL_O, tmem + T::COL_S + (j & 1) * T::TILE + ks * 8,
-                                 smem_desc(vb + ks * 16 * 128, T::VBOX_BYTES, 1024, kSwz128), idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
-                umma_commit(kv_empty(j % NS));
+                for (int ks = 0; ks < KS_S; ++ks) score_mma(t, ks);
+                umma_commit(s_full(t % NB));
+                ++issued_mma;
+            }
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int t = j + NB - 1;                     // the score product issued together with the value product of tile j
+                const bool ahead = t < n_tiles;
+                if constexpr (NB == 2) {
+                    // two score buffers: S[t % 2] is free as soon as the value product of tile j-1 has completed, before
+                    // the softmax of tile j ends, so the score product goes first and runs under that softmax
+                    if (ahead) {
+                        if (!score_ready(t)) { ok = false; break; }
+#pragma unroll
+                        for (int ks = 0; ks < KS_S; ++ks) score_mma(t, ks);
+                        umma_commit(s_full(t % NB));
+                    }
+                    if (!mbar_wait_spin(p_full, j & 1, s_abort)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < KS_O; ++ks) value_mma(j, ks);
+                    umma_commit(kv_empty(j % NS));
+                } else {
+                    // three score buffers: once every row has stored P of tile j (and finished any rescaling of O), the value
+                    // product of tile j and the score product of tile j+2 are issued as two interleaved chains
+                    if (!mbar_wait_spin(p_full, j & 1, s_abort)) { ok = false; break; }
+                    if (ahead && !score_ready(t)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < (KS_S > KS_O ? KS_S : KS_O); ++ks) {
+                        if (ks < KS_O) value_mma(j, ks);
+                        if (ahead && ks < KS_S) score_mma(t, ks);
+                        if (ks == KS_O - 1) umma_commit(kv_empty(j % NS));    // (also covers the score MMAs issued so far)
+                    }
+                    if (ahead) umma_commit(s_full(t % NB));
+                }
+                ++issued_mma;
             }
             if (ok) umma_commit(o_full);
             if (!ok && !*s_abort) {
