@@ -12,8 +12,9 @@
 // Layout of the work
 //   thread block   = 32 query tokens x 4 heads of one (sequence, value group): 128 rows = one M = 128 MMA tile
 //   warps 0-3      = softmax: thread r owns row r (token r / 4, head r % 4) = tensor-memory lane r
-//   warp 4         = producer (one lane): TMA loads of the 64-token value tile and positional-key tile into a ring
-//   warp 5         = MMA issuer (one lane) and owner of the tensor-memory allocation
+//   warp 4         = one lane: TMA loads of the 64-token value tile and positional-key tile into a ring, and issuer of
+//                    the value products
+//   warp 5         = one lane: issuer of the score products; the warp owns the tensor-memory allocation
 //   per 64-token tile j:
 //     S[j & 1]  = Q K_j^T            tcgen05.mma, K = d_v (value dims, 128-byte swizzle) + d_r (RoPE dims)
 //     softmax   : tcgen05.ld row -> mask -> row maximum / sum (base 2) -> P_j as bf16 pairs, written over the first
@@ -64,7 +65,7 @@ struct PrefillTraits {
     static constexpr int OFF_QR = OFF_QV + QV_BYTES;
     static constexpr int OFF_STAGE = OFF_QR + QR_BYTES;
     static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
-    static constexpr int N_BARS = 2 * NSTAGE + 7;
+    static constexpr int N_BARS = 2 * NSTAGE + 9;
     static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
     // tensor-memory columns: two score buffers (64 each; P overwrites the first 32 of its S), O (DV) and, where it
     // fits (d_v = 64), the query tile Q as bf16 pairs ((DV + DR) / 2): an MMA whose A operand comes from tensor memory
@@ -312,8 +313,11 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     auto kv_full = [&](int s) { return bar0 + 8u * s; };
     auto kv_empty = [&](int s) { return bar0 + 8u * (NS + s); };
     auto s_full = [&](int i) { return bar0 + 8u * (2 * NS + i); };
-    const uint32_t p_full = bar0 + 8u * (2 * NS + 3), q_ready = bar0 + 8u * (2 * NS + 4), drain = bar0 + 8u * (2 * NS + 5),
-                   o_full = bar0 + 8u * (2 * NS + 6);
+    // one P barrier per score buffer: the softmax of tile j+1 can end before the value-product issuer has observed tile j,
+    // and a single barrier waited on by parity would then be two phases ahead of its waiter
+    auto p_full = [&](int i) { return bar0 + 8u * (2 * NS + ((i & 1) ? 8 : 3)); };
+    const uint32_t q_ready = bar0 + 8u * (2 * NS + 4), drain = bar0 + 8u * (2 * NS + 5),
+                   o_full = bar0 + 8u * (2 * NS + 6), drain2 = bar0 + 8u * (2 * NS + 7);
     constexpr int NB = T::NSBUF;
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + T::N_BARS);
     volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
@@ -326,9 +330,11 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         mbar_init(s_full(0), 1);
         mbar_init(s_full(1), 1);
         mbar_init(s_full(2), 1);
-        mbar_init(p_full, T::ROWS);
+        mbar_init(p_full(0), T::ROWS);
+        mbar_init(p_full(1), T::ROWS);
         mbar_init(q_ready, T::ROWS);
         mbar_init(drain, 1);
+        mbar_init(drain2, 1);
         mbar_init(o_full, 1);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -501,7 +507,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             }
             tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(p_full);
+            mbar_arrive(p_full(j));
         }
         if (ok && !__all_sync(0xffffffffu, mbar_wait_spin(o_full, 0, s_abort))) ok = false;
         if (ok) {
@@ -526,52 +532,15 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             *s_abort = 1;
         }
         tc_fence_before();
-    } else if (warp == 4) {
-        // ====================================== producer (one lane) ======================================
-        if (lane == 0) {
-            int issued = 0;
-            for (int j = 0; j < n_tiles; ++j) {
-                const int st = j % NS;
-                const int t0 = j * T::TILE;
-                const int pj = t0 / p.P, slot0 = t0 % p.P;
-                const long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
-                                                     : (long long)b * p.max_pages + pj;
-                if (page < 0 || page >= p.num_pages) {
-                    report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
-                    *s_abort = 1;
-                    break;
-                }
-                if (j >= NS && !mbar_wait_sleepy(kv_empty(st), ((j / NS) & 1) ^ 1, s_abort)) {
-                    if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
-                    *s_abort = 1;
-                    break;
-                }
-                const uint32_t dst = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
-                mbar_expect_tx(kv_full(st), T::V_BYTES + T::KR_BYTES);
-                const int row = (int)((page * p.G + g) * p.P + slot0);
-#pragma unroll
-                for (int bx = 0; bx < T::BOXES; ++bx) tma_load_2d(dst + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, kv_full(st));
-                tma_load_2d(dst + T::V_BYTES, &tm_k, 0, (int)(page * p.P + slot0), kv_full(st));
-                ++issued;
-            }
-            if (*s_abort) {   // copies still in flight must land before the block's shared memory is released
-                for (int j = max(0, issued - NS); j < issued; ++j)
-                    for (int it = 0; it < kDrainPolls && !mbar_try_wait(kv_full(j % NS), (j / NS) & 1); ++it) {}
-            }
-        }
     } else {
-        // ====================================== MMA issuer (one lane) ======================================
+        // ========== MMA issuers: warp 5 the score products, warp 4 the value products (and the TMA loads) ==========
+        // One thread sustains about one tcgen05.mma per 110 cycles (measured), and a 128 x 64 x 16 MMA occupies the tensor
+        // pipe for 32: two issuing threads per block (and two blocks per SM) are needed to keep the pipe fed.
         if (lane == 0) {
             constexpr uint32_t idesc_s = umma_idesc(T::ROWS, T::TILE, false);
             constexpr uint32_t idesc_o = umma_idesc(T::ROWS, DV, true);
             constexpr uint64_t kr_swz = T::KR_ROW == 32 ? kSwz32 : kSwz64;
             constexpr uint32_t kr_sbo = 8 * T::KR_ROW;
-            bool ok = mbar_wait_spin(q_ready, 0, s_abort);
-            int issued_mma = 0;
-            // One MMA of the score product of tile t (k-step ks) into S[t % NB], and one of the value product of tile t.
-            // Consecutive MMAs on one accumulator wait for each other inside the tensor pipe (measured: ~80 cycles per
-            // 128 x 64 x 16 MMA in a chain against 32 at full rate), so with three score buffers the two chains are
-            // issued interleaved.
             // Descriptors differ only in their 14-bit start-address field (low word): the high words and the other low
             // bits are compile-time constants, so one issue costs an add per operand, not a descriptor build.
             constexpr uint32_t hi128 = (1024u >> 4) | (1u << 14) | ((uint32_t)kSwz128 << 29);      // SBO 1024, version 1, 128-byte swizzle
@@ -581,85 +550,91 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             const uint32_t a_qv = ((s_base + T::OFF_QV) & 0x3FFFFu) >> 4, a_qr = ((s_base + T::OFF_QR) & 0x3FFFFu) >> 4;
             const uint32_t a_st = ((s_base + T::OFF_STAGE) & 0x3FFFFu) >> 4;
             auto mk = [](uint32_t lo, uint32_t hi) { return (uint64_t)lo | ((uint64_t)hi << 32); };
-            auto score_mma = [&](int t, int ks) {
-                const uint32_t vb = a_st + (uint32_t)(t % NS) * (T::STAGE_BYTES >> 4);
-                const uint32_t d = tmem + T::COL_S + (t % NB) * T::TILE;
-                if (ks < T::KSTEPS_V) {
-                    const uint32_t off = ((ks >> 2) * T::QBOX_BYTES + (ks & 3) * 32) >> 4;
-                    const uint32_t voff = ((ks >> 2) * T::VBOX_BYTES + (ks & 3) * 32) >> 4;
-                    if constexpr (T::Q_IN_TMEM) umma_bf16_ts(d, tmem + T::COL_Q + ks * 8, mk((vb + voff) | lo_k, hi128), idesc_s, ks > 0);
-                    else umma_bf16(d, mk((a_qv + off) | lo_k, hi128), mk((vb + voff) | lo_k, hi128), idesc_s, ks > 0);
-                } else {
-                    const uint32_t kr = (uint32_t)(ks - T::KSTEPS_V) * 2;
-                    if constexpr (T::Q_IN_TMEM) umma_bf16_ts(d, tmem + T::COL_Q + ks * 8, mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
-                    else umma_bf16(d, mk((a_qr + kr) | lo_k, hikr), mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
-                }
-            };
-            auto value_mma = [&](int t, int ks) {
-                const uint32_t vb = a_st + (uint32_t)(t % NS) * (T::STAGE_BYTES >> 4);
-                umma_bf16_ts(tmem + T::COL_O, tmem + T::COL_S + (t % NB) * T::TILE + ks * 8,
-                             mk((vb + ks * (16 * 128 >> 4)) | lo_mn, hi128), idesc_o, (t > 0 || ks > 0) ? 1u : 0u);
-            };
             constexpr int KS_S = T::KSTEPS_V + T::KSTEPS_R, KS_O = T::TILE / 16;
-            // S[t % NB] also holds the P of tile t - NB, so the value product of that tile must have completed before the
-            // score product of tile t is issued (MMAs with different accumulators are not ordered among themselves).
-            auto score_ready = [&](int t) -> bool {
-                if (!mbar_wait_spin(kv_full(t % NS), (t / NS) & 1, s_abort)) return false;
-                if (t >= NB && !mbar_wait_spin(kv_empty((t - NB) % NS), ((t - NB) / NS) & 1, s_abort)) return false;
-                tc_fence_after();
-                return true;
-            };
-            // prologue: the score products that run ahead of the softmax
-            for (int t = 0; t < NB - 1 && t < n_tiles && ok; ++t) {
-                ok = score_ready(t);
-                if (!ok) break;
-#pragma unroll
-                for (int ks = 0; ks < KS_S; ++ks) score_mma(t, ks);
-                umma_commit(s_full(t % NB));
-                ++issued_mma;
-            }
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int t = j + NB - 1;                     // the score product issued together with the value product of tile j
-                const bool ahead = t < n_tiles;
-                if constexpr (NB == 2) {
-                    // two score buffers: S[t % 2] is free as soon as the value product of tile j-1 has completed, before
-                    // the softmax of tile j ends, so the score product goes first and runs under that softmax
-                    if (ahead) {
-                        if (!score_ready(t)) { ok = false; break; }
-#pragma unroll
-                        for (int ks = 0; ks < KS_S; ++ks) score_mma(t, ks);
-                        umma_commit(s_full(t % NB));
-                    }
-                    if (!mbar_wait_spin(p_full, j & 1, s_abort)) { ok = false; break; }
+            bool ok = true;
+            int issued_mma = 0;
+            if (warp == 5) {
+                ok = mbar_wait_spin(q_ready, 0, s_abort);
+                for (int t = 0; t < n_tiles && ok; ++t) {
+                    // S[t & 1] also holds the P of tile t-2, so the value product of that tile must have completed before the
+                    // score product of tile t is issued (MMAs with different accumulators are not ordered among themselves)
+                    if (!mbar_wait_spin(kv_full(t % NS), (t / NS) & 1, s_abort)) { ok = false; break; }
+                    if (t >= NB && !mbar_wait_spin(kv_empty((t - NB) % NS), ((t - NB) / NS) & 1, s_abort)) { ok = false; break; }
                     tc_fence_after();
+                    const uint32_t vb = a_st + (uint32_t)(t % NS) * (T::STAGE_BYTES >> 4);
+                    const uint32_t d = tmem + T::COL_S + (t % NB) * T::TILE;
 #pragma unroll
-                    for (int ks = 0; ks < KS_O; ++ks) value_mma(j, ks);
-                    umma_commit(kv_empty(j % NS));
-                } else {
-                    // three score buffers: once every row has stored P of tile j (and finished any rescaling of O), the value
-                    // product of tile j and the score product of tile j+2 are issued as two interleaved chains
-                    if (!mbar_wait_spin(p_full, j & 1, s_abort)) { ok = false; break; }
-                    if (ahead && !score_ready(t)) { ok = false; break; }
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < (KS_S > KS_O ? KS_S : KS_O); ++ks) {
-                        if (ks < KS_O) value_mma(j, ks);
-                        if (ahead && ks < KS_S) score_mma(t, ks);
-                        if (ks == KS_O - 1) umma_commit(kv_empty(j % NS));    // (also covers the score MMAs issued so far)
+                    for (int ks = 0; ks < KS_S; ++ks) {
+                        if (ks < T::KSTEPS_V) {
+                            const uint32_t off = ((ks >> 2) * T::QBOX_BYTES + (ks & 3) * 32) >> 4;
+                            const uint32_t voff = ((ks >> 2) * T::VBOX_BYTES + (ks & 3) * 32) >> 4;
+                            if constexpr (T::Q_IN_TMEM) umma_bf16_ts(d, tmem + T::COL_Q + ks * 8, mk((vb + voff) | lo_k, hi128), idesc_s, ks > 0);
+                            else umma_bf16(d, mk((a_qv + off) | lo_k, hi128), mk((vb + voff) | lo_k, hi128), idesc_s, ks > 0);
+                        } else {
+                            const uint32_t kr = (uint32_t)(ks - T::KSTEPS_V) * 2;
+                            if constexpr (T::Q_IN_TMEM) umma_bf16_ts(d, tmem + T::COL_Q + ks * 8, mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
+                            else umma_bf16(d, mk((a_qr + kr) | lo_k, hikr), mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
+                        }
                     }
-                    if (ahead) umma_commit(s_full(t % NB));
+                    umma_commit(s_full(t % NB));
+                    ++issued_mma;
                 }
-                ++issued_mma;
+            } else {
+                // This thread is also the producer: it fills the ring first, and after each value product it refills the
+                // stage that the previous value product has released.
+                int loaded = 0;
+                auto load_tile = [&](int t) -> bool {
+                    const int st = t % NS;
+                    const int t0 = t * T::TILE;
+                    const int pj = t0 / p.P, slot0 = t0 % p.P;
+                    const long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
+                                                         : (long long)b * p.max_pages + pj;
+                    if (page < 0 || page >= p.num_pages) {
+                        report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
+                        *s_abort = 1;
+                        return false;
+                    }
+                    const uint32_t dst = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
+                    mbar_expect_tx(kv_full(st), T::V_BYTES + T::KR_BYTES);
+                    const int row = (int)((page * p.G + g) * p.P + slot0);
+#pragma unroll
+                    for (int bx = 0; bx < T::BOXES; ++bx) tma_load_2d(dst + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, kv_full(st));
+                    tma_load_2d(dst + T::V_BYTES, &tm_k, 0, (int)(page * p.P + slot0), kv_full(st));
+                    ++loaded;
+                    return true;
+                };
+                for (int t = 0; t < NS && t < n_tiles && ok; ++t) ok = load_tile(t);
+                for (int j = 0; j < n_tiles && ok; ++j) {
+                    // every row has stored P of tile j and finished any rescaling of O
+                    if (!mbar_wait_spin(p_full(j), (j >> 1) & 1, s_abort)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t vb = a_st + (uint32_t)(j % NS) * (T::STAGE_BYTES >> 4);
+#pragma unroll
+                    for (int ks = 0; ks < KS_O; ++ks)
+                        umma_bf16_ts(tmem + T::COL_O, tmem + T::COL_S + (j % NB) * T::TILE + ks * 8,
+                                     mk((vb + ks * (16 * 128 >> 4)) | lo_mn, hi128), idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
+                    umma_commit(kv_empty(j % NS));
+                    ++issued_mma;
+                    if (j >= 1 && j - 1 + NS < n_tiles) {      // tile j-1 was consumed a tile ago: its stage takes tile j-1+NS
+                        if (!mbar_wait_spin(kv_empty((j - 1) % NS), ((j - 1) / NS) & 1, s_abort)) { ok = false; break; }
+                        ok = load_tile(j - 1 + NS);
+                    }
+                }
+                if (ok) umma_commit(o_full);
+                if (*s_abort) {   // copies still in flight must land before the block's shared memory is released
+                    for (int t = max(0, loaded - NS); t < loaded; ++t)
+                        for (int it = 0; it < kDrainPolls && !mbar_try_wait(kv_full(t % NS), (t / NS) & 1); ++it) {}
+                }
             }
-            if (ok) umma_commit(o_full);
             if (!ok && !*s_abort) {
                 report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
                 *s_abort = 1;
             }
             // nothing issued by this thread may still be running (or about to signal a barrier) when the block ends
             if (issued_mma > 0) {
-                umma_commit(drain);
-                for (int it = 0; it < kDrainPolls * 16 && !mbar_try_wait(drain, 0); ++it) {}
+                const uint32_t dr = warp == 5 ? drain : drain2;
+                umma_commit(dr);
+                for (int it = 0; it < kDrainPolls * 16 && !mbar_try_wait(dr, 0); ++it) {}
             }
             tc_fence_before();
         }
