@@ -59,6 +59,9 @@ def make_workload(name: str, rank: int):
     if name == "cfg2-dr24":  # cfg2 with the paper's other tested RoPE width (d_r = 24: 48-byte positional rows)
         return wl.make_case("cfg2-dr24", wl.SHAPE_C, [32768] * 32, page_size=64, cache_dtype="bf16", paged=True,
                             seed=wl.MASTER_SEED + 2024 + shift)
+    if name == "cfg2-dr0":   # cfg2 without the positional slice: the value-only cache, exactly half of matched GQA
+        return wl.make_case("cfg2-dr0", wl.SHAPE_A0, [32768] * 32, page_size=64, cache_dtype="bf16", paged=True,
+                            seed=wl.MASTER_SEED + 2050 + shift)
     if name == "cfg2-ncu":   # profiler-sized: 143 MB of cache (> L2), same shapes and paging as cfg2
         return wl.config2(seed=wl.MASTER_SEED + 2000 + shift, B=16, T=16384)
     if name == "cfg2-small":
@@ -72,6 +75,7 @@ WORKLOAD_TEXT = {
     "cfg3": "wider-head ragged serving batch (B=64, H=32, G=8, d_v=128, seq_lens ~ U[1024,16384], paged)",
     "cfg4": "24-layer decode step (B=128, T=8192 cached + 1 appended per layer, paged, one pool per layer)",
     "cfg2-dr24": "cfg2 with RoPE width d_r = 24 (B=32, T=32768, paged; N_GVA/N_GQA = 0.546875)",
+    "cfg2-dr0": "cfg2 without the positional slice, d_r = 0 (value-only cache; B=32, T=32768, paged; N_GVA/N_GQA = 0.5)",
 }
 
 
@@ -321,7 +325,10 @@ def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with
            "kernel": {1: "fma", 2: "mma"}.get(gb.gva_last_kernel(dc.handle), "?"),
            "cache_bytes": case.cache_bytes() * n_layers}
 
-    if with_e2e:
+    if with_e2e and case.shape.d_r == 0:
+        # the host-buffer entry point is not built for the value-only cache: report the device-timed step
+        res.update(e2e_ms=step_ms, e2e_matches=None, h2d=0, d2h=0)
+    elif with_e2e:
         # end to end: host buffers in, host buffer out, through the C ABI (one call per step, then a sync)
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
         h_qc, h_qr, h_vn, h_kn = pin(case.q_c), pin(case.q_r), pin(case.v_new), pin(case.kr_new)
@@ -570,7 +577,7 @@ def main() -> None:
         peak = load_peaks()[0]
         short = argparse.Namespace(**vars(args))
         short.steps, short.warmup = max(20, args.steps // 3), 10
-        for other in ("cfg1", "cfg3", "cfg4", "cfg2-dr24"):
+        for other in ("cfg1", "cfg3", "cfg4", "cfg2-dr24", "cfg2-dr0"):
             o = measure(other, rank, local_rank, dist, short, kernel, torch, gb, harness, with_e2e=False,
                         with_clocks=True)
             per_layer = o["cache_bytes"] / o["layers"]

@@ -63,7 +63,10 @@ typedef struct {
     int32_t H, G;          /* query heads, value groups; H % G == 0 and H/G == 4                          */
     int32_t d_v;           /* value width: 64 or 128                                                      */
     int32_t d_c;           /* content-key width (only gva_absorb_query uses it): 1..256                   */
-    int32_t d_r;           /* RoPE width: 16 or 24 with d_v = 64 (the paper's two tested widths), 32 with d_v = 128 */
+    int32_t d_r;           /* RoPE width: 16 or 24 with d_v = 64 (the paper's two tested widths), 32 with d_v = 128;
+                              0 = value-only cache without a positional slice (Section 3.4: "only values, exactly
+                              half"): kr_pool, q_r and kr_new are then unused and may be NULL, scale = 1/sqrt(d_c);
+                              gva_decode_step_host, the projections and gva_prefill return GVA_ERR_UNSUPPORTED     */
     int32_t page_size;     /* tokens per page, a multiple of 32                                           */
     int32_t cache_dtype;   /* gva_dtype                                                                   */
     int32_t kernel;        /* gva_kernel                                                                  */

@@ -117,6 +117,10 @@ bool plan_fma(const gva_handle *h, int B, FmaPlan *out) {
     const bool bf = h->cfg.cache_dtype == GVA_BF16;
     if (h->cfg.d_v == 64 && h->cfg.d_r == 24 && !GQA)
         return bf ? plan_fma_t<__nv_bfloat16, 64, 24, false>(h, B, out) : plan_fma_t<float, 64, 24, false>(h, B, out);
+    if (h->cfg.d_r == 0 && !GQA) {      // value-only cache
+        if (h->cfg.d_v == 64) return bf ? plan_fma_t<__nv_bfloat16, 64, 0, false>(h, B, out) : plan_fma_t<float, 64, 0, false>(h, B, out);
+        return bf ? plan_fma_t<__nv_bfloat16, 128, 0, false>(h, B, out) : plan_fma_t<float, 128, 0, false>(h, B, out);
+    }
     if (h->cfg.d_v == 64)
         return bf ? plan_fma_t<__nv_bfloat16, 64, 16, GQA>(h, B, out) : plan_fma_t<float, 64, 16, GQA>(h, B, out);
     return bf ? plan_fma_t<__nv_bfloat16, 128, 32, GQA>(h, B, out) : plan_fma_t<float, 128, 32, GQA>(h, B, out);
@@ -253,13 +257,14 @@ extern "C" {
 int gva_create(gva_handle **out, const gva_config *cfg, int device) {
     if (!out || !cfg) return GVA_ERR_INVALID_ARG;
     *out = nullptr;
-    if (cfg->H <= 0 || cfg->G <= 0 || cfg->d_v <= 0 || cfg->d_c <= 0 || cfg->d_r <= 0 || cfg->page_size <= 0 ||
+    if (cfg->H <= 0 || cfg->G <= 0 || cfg->d_v <= 0 || cfg->d_c <= 0 || cfg->d_r < 0 || cfg->page_size <= 0 ||
         !(cfg->rope_base > 1.0) || !(cfg->softmax_scale >= 0.f) || device < 0)
         return GVA_ERR_INVALID_ARG;
     if (cfg->cache_dtype != GVA_F32 && cfg->cache_dtype != GVA_BF16) return GVA_ERR_INVALID_ARG;
     if (cfg->kernel < GVA_KERNEL_AUTO || cfg->kernel > GVA_KERNEL_MMA) return GVA_ERR_INVALID_ARG;
     if (cfg->H % cfg->G != 0 || cfg->H / cfg->G != kHeadsPerGroup) return GVA_ERR_UNSUPPORTED;
-    if (!((cfg->d_v == 64 && (cfg->d_r == 16 || cfg->d_r == 24)) || (cfg->d_v == 128 && cfg->d_r == 32)))
+    // d_r = 0 is the value-only cache (no positional slice: Section 3.4, "exactly half")
+    if (!((cfg->d_v == 64 && (cfg->d_r == 16 || cfg->d_r == 24 || cfg->d_r == 0)) || (cfg->d_v == 128 && (cfg->d_r == 32 || cfg->d_r == 0))))
         return GVA_ERR_UNSUPPORTED;
     if (cfg->G > 8 || cfg->d_c > 256 || cfg->page_size % 32 != 0) return GVA_ERR_UNSUPPORTED;
     if (cfg->kernel == GVA_KERNEL_MMA && cfg->cache_dtype != GVA_BF16) return GVA_ERR_UNSUPPORTED;
@@ -332,7 +337,7 @@ int gva_absorb_query(gva_handle *h, const float *q_c, const float *q_r, const fl
                      float *q_abs, int B, void *stream) {
     if (!h || B < 0) return GVA_ERR_INVALID_ARG;
     if (B == 0) return GVA_OK;
-    if (!q_c || !q_r || !M || !q_pos || !q_abs) return GVA_ERR_INVALID_ARG;
+    if (!q_c || (h->cfg.d_r > 0 && !q_r) || !M || !q_pos || !q_abs) return GVA_ERR_INVALID_ARG;
     if (!aligned(q_c, 4) || !aligned(q_r, 4) || !aligned(M, 4) || !aligned(q_pos, 4) || !aligned(q_abs, 16))
         return GVA_ERR_INVALID_ARG;
     const gva_config &c = h->cfg;
@@ -368,7 +373,7 @@ int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, 
                      const int32_t *pos, int B, int32_t *dev_status, void *stream) {
     if (!h || !cache || B < 0) return GVA_ERR_INVALID_ARG;
     if (B == 0) return GVA_OK;
-    if (!cache->v_pool || !cache->kr_pool || !v_new || !kr_new || !pos) return GVA_ERR_INVALID_ARG;
+    if (!cache->v_pool || (h->cfg.d_r > 0 && !cache->kr_pool) || !v_new || (h->cfg.d_r > 0 && !kr_new) || !pos) return GVA_ERR_INVALID_ARG;
     if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
     if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16)) return GVA_ERR_INVALID_ARG;
     const gva_config &c = h->cfg;
@@ -394,7 +399,7 @@ int gva_append_chunk(gva_handle *h, const gva_cache *cache, const float *v_new, 
                      const int32_t *ctx_lens, int B, int n_q, int32_t *dev_status, void *stream) {
     if (!h || !cache || B < 0 || n_q < 0) return GVA_ERR_INVALID_ARG;
     if (B == 0 || n_q == 0) return GVA_OK;
-    if (!cache->v_pool || !cache->kr_pool || !v_new || !kr_new || !cu_q || !ctx_lens) return GVA_ERR_INVALID_ARG;
+    if (!cache->v_pool || (h->cfg.d_r > 0 && !cache->kr_pool) || !v_new || (h->cfg.d_r > 0 && !kr_new) || !cu_q || !ctx_lens) return GVA_ERR_INVALID_ARG;
     if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
     if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16)) return GVA_ERR_INVALID_ARG;
     const gva_config &c = h->cfg;
@@ -420,7 +425,7 @@ int gva_prefill(gva_handle *h, const gva_cache *cache, const float *q_abs, const
                 float *out, float *lse, int B, int max_q_len, int32_t *dev_status, void *stream) {
     if (!h || !cache || B < 0 || max_q_len < 0) return GVA_ERR_INVALID_ARG;
     if (B == 0 || max_q_len == 0) return GVA_OK;
-    if (!cache->v_pool || !cache->kr_pool || !q_abs || !cu_q || !ctx_lens || !out) return GVA_ERR_INVALID_ARG;
+    if (!cache->v_pool || (h->cfg.d_r > 0 && !cache->kr_pool) || !q_abs || !cu_q || !ctx_lens || !out) return GVA_ERR_INVALID_ARG;
     if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
     if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16) || !aligned(q_abs, 16) || !aligned(out, 16))
         return GVA_ERR_INVALID_ARG;
@@ -457,7 +462,7 @@ static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs
     if (rc != GVA_OK) return rc;
     if (!cache) return GVA_ERR_INVALID_ARG;
     if (B > 0) {
-        if (!cache->v_pool || !cache->kr_pool || !q_abs || !seq_lens || !out) return GVA_ERR_INVALID_ARG;
+        if (!cache->v_pool || (h->cfg.d_r > 0 && !cache->kr_pool) || !q_abs || !seq_lens || !out) return GVA_ERR_INVALID_ARG;
         if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
         if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16) || !aligned(q_abs, 16) || !aligned(out, 16))
             return GVA_ERR_INVALID_ARG;
@@ -498,9 +503,9 @@ int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const
     int rc = check_common(h, B, max_seq_len, num_splits);
     if (rc != GVA_OK) return rc;
     if (B == 0) return GVA_OK;
-    if (!cache || !M || !q_c || !q_r || !v_new || !kr_new || !pos || !seq_lens || !q_abs || !out)
+    if (!cache || !M || !q_c || (h->cfg.d_r > 0 && !q_r) || !v_new || (h->cfg.d_r > 0 && !kr_new) || !pos || !seq_lens || !q_abs || !out)
         return GVA_ERR_INVALID_ARG;
-    if (!cache->v_pool || !cache->kr_pool || cache->num_pages <= 0 || cache->max_pages_per_seq <= 0)
+    if (!cache->v_pool || (h->cfg.d_r > 0 && !cache->kr_pool) || cache->num_pages <= 0 || cache->max_pages_per_seq <= 0)
         return GVA_ERR_INVALID_ARG;
     if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16) || !aligned(q_abs, 16) || !aligned(out, 16) ||
         !aligned(M, 16))
@@ -637,6 +642,7 @@ int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, 
     int rc = check_common(h, B, max_seq_len, num_splits);
     if (rc != GVA_OK) return rc;
     if (B == 0) return GVA_OK;
+    if (h->cfg.d_r == 0) return GVA_ERR_UNSUPPORTED;     // the value-only cache goes through the device entry points
     if (!cache || !M || !q_c_host || !q_r_host || !v_new_host || !kr_new_host || !pos_host || !seq_lens_host || !out_host)
         return GVA_ERR_INVALID_ARG;
     const StepLayout L = step_layout(h, B, num_splits);
@@ -758,6 +764,7 @@ int gva_input_width(const gva_handle *h) { return h ? input_width(h->cfg) : 0; }
 int gva_pack_input_weights(const gva_handle *h, const float *W_q_nope, const float *W_q_rope, const float *W_v,
                            const float *W_r, const float *M, int d_model, uint16_t *W_in) {
     if (!h || !W_q_nope || !W_q_rope || !W_v || !W_r || !M || !W_in || d_model <= 0) return GVA_ERR_INVALID_ARG;
+    if (h->cfg.d_r == 0) return GVA_ERR_UNSUPPORTED;     // the projections are built for the caches with a positional slice
     const gva_config &c = h->cfg;
     const int dq = c.d_v + c.d_r, nq = c.H * dq, nv = c.G * c.d_v, N = input_width(c);
     for (int m = 0; m < d_model; ++m) {
@@ -788,8 +795,9 @@ int gva_pack_bf16(const float *src, uint16_t *dst, size_t n) {
 int gva_project_in(gva_handle *h, const gva_cache *cache, const float *x, const void *W_in, int d_model,
                    const int32_t *pos, float *q_abs, int B, int32_t *dev_status, void *stream) {
     if (!h || !cache || B < 0 || d_model <= 0) return GVA_ERR_INVALID_ARG;
+    if (h->cfg.d_r == 0) return GVA_ERR_UNSUPPORTED;
     if (B == 0) return GVA_OK;
-    if (!x || !W_in || !pos || !q_abs || !cache->v_pool || !cache->kr_pool) return GVA_ERR_INVALID_ARG;
+    if (!x || !W_in || !pos || !q_abs || !cache->v_pool || (h->cfg.d_r > 0 && !cache->kr_pool)) return GVA_ERR_INVALID_ARG;
     if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
     if (!aligned(x, 16) || !aligned(W_in, 16) || !aligned(q_abs, 8) || !aligned(cache->v_pool, 16) ||
         !aligned(cache->kr_pool, 16))

@@ -314,7 +314,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                     const uint32_t bar = smem_u32(&full_bar[st]);
                     const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
                     mbar_expect_tx(bar, GQA ? 2 * G * T::VTILE_BYTES : G * T::VTILE_BYTES + T::KR_BYTES);
-                    if constexpr (!GQA) tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
+                    if constexpr (!GQA && DR > 0) tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
                     for (int g = 0; g < G; ++g) {
                         const int row = (int)((page * G + g) * p.P + slot0);
                         if constexpr (GQA) {
@@ -603,6 +603,8 @@ int launch_mma_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
     if (!encode_map(st, &tm_v, p.v_pool, DV, vrows, 64, TILE, CU_TENSOR_MAP_SWIZZLE_128B)) return GVA_ERR_CUDA;
     if (GQA) {
         if (!encode_map(st, &tm_k, p.k_pool, DV, vrows, 64, TILE, CU_TENSOR_MAP_SWIZZLE_128B)) return GVA_ERR_CUDA;
+    } else if (DR == 0) {
+        tm_k = tm_v;      // value-only cache: there is no positional-key tile to describe (the kernel never uses this map)
     } else {
         if (!encode_map(st, &tm_k, p.kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, TILE,
                         DR == 16   ? CU_TENSOR_MAP_SWIZZLE_32B
@@ -648,6 +650,16 @@ int launch_decode_mma(const gva_config &cfg, const MmaHostState &st, int sm_coun
                                                                      num_splits, max_blocks, stream, n_blocks_out);
         return launch_mma_t<64, 24, 32, 3, GVA_MMA_WPG64, false>(cfg, st, sm_count, smem_optin, p, B, max_seq_len,
                                                                  num_splits, max_blocks, stream, n_blocks_out);
+    }
+    if (cfg.d_r == 0 && !GQA) {       // value-only cache
+        if (cfg.d_v == 64 && *tile_out == 64)
+            return launch_mma_t<64, 0, 64, 3, GVA_MMA_WPG64, false>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits,
+                                                                    max_blocks, stream, n_blocks_out);
+        if (cfg.d_v == 64)
+            return launch_mma_t<64, 0, 32, 3, GVA_MMA_WPG64, false>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits,
+                                                                    max_blocks, stream, n_blocks_out);
+        return launch_mma_t<128, 0, 32, 3, 1, false>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks,
+                                                     stream, n_blocks_out);
     }
     if (cfg.d_v == 64 && *tile_out == 64)
         return launch_mma_t<64, 16, 64, 3, GVA_MMA_WPG64, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks,

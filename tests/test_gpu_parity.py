@@ -55,7 +55,7 @@ def test_absorb_matches_oracle(shape, B):
 
 # ------------------------------------------------------------------ append (bit exact)
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C, wl.SHAPE_A0])
 def test_append_is_bit_exact_and_touches_nothing_else(dtype, shape):
     lens = [1, 64, 65, 300, 129, 4000, 8193]
     case = wl.make_case("append", shape, lens, page_size=64, cache_dtype=dtype, seed=102, extra_pages=3)
@@ -137,7 +137,7 @@ EDGE_LENS = [0, 1, 31, 32, 33, 63, 64, 65, 127, 128, 129, 640, 641, 1000]
 
 
 @pytest.mark.parametrize("kernel", KERNELS_BF16)
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C, wl.SHAPE_A0, wl.SHAPE_B0])
 @pytest.mark.parametrize("num_splits", [0, 1, 5, 40])
 def test_ragged_edge_lengths_poisoned(kernel, shape, num_splits):
     # lengths around tile and page boundaries, an empty sequence, more splits than tiles;
@@ -148,7 +148,7 @@ def test_ragged_edge_lengths_poisoned(kernel, shape, num_splits):
     U().check_decode(case, kernel, num_splits=num_splits)
 
 
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C, wl.SHAPE_A0, wl.SHAPE_B0])
 @pytest.mark.parametrize("num_splits", [0, 3])
 def test_ragged_edge_lengths_f32(shape, num_splits):
     case = wl.make_case("edge32", shape, EDGE_LENS, page_size=64, cache_dtype="f32", seed=202, poison_unused=True)
@@ -276,7 +276,7 @@ def test_full_step_follows_algorithm_order(kernel):
 
 # ------------------------------------------------------------------ fused step entry point
 @pytest.mark.parametrize("kernel", KERNELS_BF16)
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C, wl.SHAPE_A0])
 def test_fused_step_is_bitwise_the_three_calls(kernel, shape):
     _mma_or_skip(kernel)
     lens = np.array([1, 64, 65, 1001, 4096, 130], dtype=np.int32)
@@ -415,3 +415,21 @@ def test_workspace_and_outputs_stay_inside_their_bounds(kernel):
         assert int(dc.status.item()) == 0
     finally:
         dc.close()
+
+
+def test_value_only_cache_long_context_and_what_it_does_not_cover():
+    # the cache without a positional slice (Section 3.4): a paged long-context case on both kernels, then the entry points
+    # that are not built for it
+    case = wl.make_case("vo-long", wl.SHAPE_A0, [20000, 8191, 4097, 333], page_size=64, cache_dtype="bf16", seed=231)
+    for kernel in KERNELS_BF16:
+        _mma_or_skip(kernel)
+        U().check_decode(case, kernel)
+    h = gb.gva_create(H=16, G=4, d_v=64, d_c=64, d_r=0, page_size=64)
+    try:
+        t = torch.zeros(4096, dtype=torch.float32, device="cuda")
+        i = torch.zeros(16, dtype=torch.int32, device="cuda")
+        cache = gb.make_cache(t, None, None, 4, 4)
+        assert gb.gva_prefill(h, cache, t, i, i, t, None, 1, 8, check=False) == gb.GVA_ERR_UNSUPPORTED
+        assert gb.gva_project_in(h, cache, t, t, 128, i, t, 1, check=False) == gb.GVA_ERR_UNSUPPORTED
+    finally:
+        gb.gva_destroy(h)

@@ -645,3 +645,34 @@ def test_append_chunk_equals_token_by_token_append():
     assert np.array_equal(v1, v2) and np.array_equal(k1, k2)
     changed = np.argwhere((v1 != c.v_pool).any(axis=(1, 3)))
     assert len(changed) <= pc.n_q                                  # at most one (page, slot) per new token
+
+
+# ---------------------------------------------------------------- value-only cache (no positional slice, d_r = 0)
+def test_value_only_cache_is_attention_with_keys_v_m():
+    # without the positional slice the score is q^nope . (v M_h) alone and d_qk = d_c: plain attention whose keys
+    # are the reconstructed content keys (library routine), and the cache is exactly half of matched GQA
+    s = wl.HeadShape(H=8, G=2, d_v=16, d_c=12, d_r=0)
+    c = wl.make_case("vo", s, [37, 5, 16, 1, 0], page_size=16, cache_dtype="bf16", paged=True, seed=41, poison_unused=True)
+    assert c.kr_pool.size == 0 and c.cache_bytes() * 2 == int(c.seq_lens.sum()) * 2 * s.G * s.d_v * 2
+    q_abs = orc.absorb_case(c)
+    assert q_abs.shape == (c.B, s.H, s.d_v)
+    out, lse = orc.decode_case(c)
+    V = torch.from_numpy(wl.pool_to_f64(c.v_pool)); M = torch.from_numpy(c.M.astype(np.float64))
+    for b in range(c.B):
+        L = int(c.seq_lens[b])
+        if L == 0:
+            assert np.all(out[b] == 0) and np.all(np.isneginf(lse[b]))
+            continue
+        pages = [c.page_of(b, t // c.page_size) for t in range(L)]; slots = [t % c.page_size for t in range(L)]
+        q = torch.from_numpy(c.q_c[b].astype(np.float64))
+        K = torch.stack([V[pages, h // (s.H // s.G), slots] @ M[h] for h in range(s.H)])
+        Vv = torch.stack([V[pages, h // (s.H // s.G), slots] for h in range(s.H)])
+        ref = torch.nn.functional.scaled_dot_product_attention(q[None, :, None, :], K[None], Vv[None],
+                                                               scale=1.0 / math.sqrt(s.d_c))[0, :, 0]
+        assert np.allclose(out[b], ref.numpy(), atol=1e-12)
+    # append writes value rows only
+    v0 = c.v_pool.copy()
+    live = c.seq_lens > 0
+    c.append_pos[:] = np.maximum(c.seq_lens - 1, 0)
+    assert orc.append_case(c) == 0
+    assert (c.v_pool != v0).any() and c.kr_pool.size == 0
