@@ -273,6 +273,22 @@ int gva_prefill(gva_handle *h, const gva_cache *cache, const float *q_abs, const
                 const int32_t *ctx_lens, float *out, float *lse, int B, int max_q_len, int32_t *dev_status,
                 void *stream);
 
+/* Decode of several new tokens per sequence over a long cached context (speculative / multi-token decode; not in the
+ * paper -- Algorithm 1 applied to q_len_b tokens at once, i.e. gva_prefill's computation) with split-KV: every block of
+ * 32 query tokens is handled by several thread blocks, each over a contiguous range of 64-token tiles, and a second
+ * kernel merges their partial results by log-sum-exp weights, so that small batches still fill the GPU.
+ *   arguments as gva_prefill, plus
+ *   n_q                          cu_q[B]: query rows in all (sizes the merge)
+ *   max_seq_len                  upper bound on ctx_lens[b] + q_len_b
+ *   num_splits                   0 = enough splits for two thread blocks per SM; n >= 1 = exactly n (at most one per tile, 64)
+ *   workspace / workspace_bytes  at least gva_decode_multi_workspace_bytes(...) bytes, 256-byte aligned
+ * Same support, tolerance and error rules as gva_prefill. */
+size_t gva_decode_multi_workspace_bytes(const gva_handle *h, int B, int n_q, int max_q_len, int max_seq_len,
+                                        int num_splits);
+int gva_decode_multi(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *cu_q,
+                     const int32_t *ctx_lens, float *out, float *lse, void *workspace, size_t workspace_bytes, int B,
+                     int n_q, int max_q_len, int max_seq_len, int num_splits, int32_t *dev_status, void *stream);
+
 /* Geometry of the most recent gva_decode / gqa_decode launch on this handle (reporting only):
  * number of split-KV partitions launched (thread blocks of the decode kernel). */
 int gva_last_num_splits(const gva_handle *h);

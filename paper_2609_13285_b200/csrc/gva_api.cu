@@ -421,9 +421,10 @@ int gva_append_chunk(gva_handle *h, const gva_cache *cache, const float *v_new, 
     return GVA_OK;
 }
 
-int gva_prefill(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *cu_q, const int32_t *ctx_lens,
-                float *out, float *lse, int B, int max_q_len, int32_t *dev_status, void *stream) {
-    if (!h || !cache || B < 0 || max_q_len < 0) return GVA_ERR_INVALID_ARG;
+static int prefill_impl(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *cu_q, const int32_t *ctx_lens,
+                        float *out, float *lse, void *workspace, size_t workspace_bytes, int B, int n_q, int max_q_len,
+                        int num_splits, int32_t *dev_status, void *stream) {
+    if (!h || !cache || B < 0 || max_q_len < 0 || n_q < 0 || num_splits < 1) return GVA_ERR_INVALID_ARG;
     if (B == 0 || max_q_len == 0) return GVA_OK;
     if (!cache->v_pool || (h->cfg.d_r > 0 && !cache->kr_pool) || !q_abs || !cu_q || !ctx_lens || !out) return GVA_ERR_INVALID_ARG;
     if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;
@@ -448,11 +449,54 @@ int gva_prefill(gva_handle *h, const gva_cache *cache, const float *q_abs, const
     p.num_pages = cache->num_pages;
     p.max_pages = cache->max_pages_per_seq;
     p.scale_log2 = h->scale * kLog2e;
-    return launch_prefill(c, h->mma, h->smem_optin, p, cache->v_pool, cache->kr_pool, B, max_q_len,
+    p.num_splits = num_splits;
+    if (num_splits > 1) {
+        const size_t o_bytes = align_up((size_t)n_q * c.H * num_splits * c.d_v * sizeof(float), 256);
+        const size_t ml_bytes = (size_t)n_q * c.H * num_splits * 2 * sizeof(float);
+        if (!workspace || !aligned(workspace, 256) || workspace_bytes < o_bytes + ml_bytes) return GVA_ERR_WORKSPACE;
+        p.part_o = static_cast<float *>(workspace);
+        p.part_ml = reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + o_bytes);
+    }
+    return launch_prefill(c, h->mma, h->smem_optin, p, cache->v_pool, cache->kr_pool, B, max_q_len, n_q,
                           static_cast<cudaStream_t>(stream));
 #else
     return GVA_ERR_UNSUPPORTED;
 #endif
+}
+
+int gva_prefill(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *cu_q, const int32_t *ctx_lens,
+                float *out, float *lse, int B, int max_q_len, int32_t *dev_status, void *stream) {
+    return prefill_impl(h, cache, q_abs, cu_q, ctx_lens, out, lse, nullptr, 0, B, 0, max_q_len, 1, dev_status, stream);
+}
+
+// Splits per query block for gva_decode_multi: enough thread blocks for two per SM, never more than tiles.
+static int multi_splits(const gva_handle *h, int B, int max_q_len, int max_seq_len, int num_splits) {
+    const int tiles = (max_seq_len + 63) / 64;
+    int s = num_splits;
+    if (s <= 0) {
+        const long long blocks = (long long)B * h->cfg.G * ((max_q_len + 31) / 32);
+        s = (int)((2LL * h->sm_count + blocks - 1) / (blocks > 0 ? blocks : 1));
+    }
+    if (s > tiles) s = tiles;
+    if (s > 64) s = 64;
+    return s < 1 ? 1 : s;
+}
+
+size_t gva_decode_multi_workspace_bytes(const gva_handle *h, int B, int n_q, int max_q_len, int max_seq_len, int num_splits) {
+    if (!h || B < 0 || n_q < 0 || max_q_len < 0 || max_seq_len < 0) return 0;
+    const int s = multi_splits(h, B, max_q_len, max_seq_len, num_splits);
+    if (s == 1) return 256;
+    return align_up((size_t)n_q * h->cfg.H * s * h->cfg.d_v * sizeof(float), 256) +
+           align_up((size_t)n_q * h->cfg.H * s * 2 * sizeof(float), 256);
+}
+
+int gva_decode_multi(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *cu_q, const int32_t *ctx_lens,
+                     float *out, float *lse, void *workspace, size_t workspace_bytes, int B, int n_q, int max_q_len,
+                     int max_seq_len, int num_splits, int32_t *dev_status, void *stream) {
+    if (!h || max_seq_len < 0 || num_splits < 0) return GVA_ERR_INVALID_ARG;
+    const int s = multi_splits(h, B > 0 ? B : 1, max_q_len, max_seq_len, num_splits);
+    return prefill_impl(h, cache, q_abs, cu_q, ctx_lens, out, lse, workspace, workspace_bytes, B, n_q, max_q_len, s, dev_status,
+                        stream);
 }
 
 static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,

@@ -126,7 +126,7 @@ decode_fma_kernel(DecodeParams p) {
                 cp_async16(kb + (g * TILE + t) * T::VROW + ch * 16,
                            ksrc + (ok ? row * (DV * sizeof(CT)) + ch * 16 : 0), ok ? 16 : 0);
             }
-        } else {
+        } else if constexpr (DR > 0) {      // (the value-only cache has no positional tile)
             const unsigned char *ksrc = reinterpret_cast<const unsigned char *>(p.kr_pool);
             const uint32_t kb = st_u32 + G * TILE * T::VROW;
             for (int c = tid; c < TILE * T::KCH; c += nt) {

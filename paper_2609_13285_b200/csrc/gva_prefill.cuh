@@ -44,6 +44,11 @@ struct PrefillParams {
     int32_t *dev_status;         // nullable
     int B, H, G, P, num_pages, max_pages;
     float scale_log2;            // softmax scale * log2(e)
+    // split-KV (multi-token decode over a long cached context): every query block is handled by num_splits thread
+    // blocks, each over a contiguous range of tiles, which leave unnormalised partial results for merge_splits_kernel
+    int num_splits;              // 1 = no split: the kernel writes out / lse itself
+    float *part_o;               // [n_q][H][num_splits][d_v]   partial O relative to part_ml[..][0]
+    float *part_ml;              // [n_q][H][num_splits][2]     reference (log2 domain) and sum; (-inf, 0) for an empty range
 };
 
 template <int DV, int DR>
@@ -289,7 +294,8 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     constexpr int NS = T::NSTAGE;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int b = blockIdx.z, g = blockIdx.y;
-    const int qb = gridDim.x - 1 - blockIdx.x;        // the longest rows (last query blocks) are scheduled first
+    const int S = p.num_splits, split = blockIdx.x % S;
+    const int qb = gridDim.x / S - 1 - blockIdx.x / S;   // the longest rows (last query blocks) are scheduled first
     grid_dependency_wait();
     const int q_begin = p.cu_q[b];
     const int n_q = p.cu_q[b + 1] - q_begin;
@@ -303,7 +309,18 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     }
     const int nv = min(T::QTOK, n_q - q0);             // live query tokens of this block
     const int p0 = ctx + q0;                           // position of the block's first query token
-    const int n_tiles = (p0 + nv - 1) / T::TILE + 1;   // tiles 0..n_tiles-1 hold every visible token
+    const int n_all = (p0 + nv - 1) / T::TILE + 1;     // tiles 0..n_all-1 hold every visible token
+    const int per_split = (n_all + S - 1) / S;
+    const int t_lo = split * per_split;                // this block's tiles: t_lo .. t_lo + n_tiles - 1 (tile j below is local)
+    const int n_tiles = min(n_all, t_lo + per_split) - t_lo;
+    if (n_tiles <= 0) {                                // more splits than tiles: an empty range weighs nothing in the merge
+        if (tid < T::ROWS && (tid >> 2) < nv) {
+            float *ml = p.part_ml + (((size_t)(q_begin + q0 + (tid >> 2)) * p.H + g * kHeadsPerGroup + (tid & 3)) * S + split) * 2;
+            ml[0] = -INFINITY;
+            ml[1] = 0.f;
+        }
+        return;
+    }
 
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -419,7 +436,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
 #pragma unroll
                 for (int c = 0; c < 32; ++c) { s[c] = lo[c]; s[32 + c] = hi[c]; }
             }
-            const int limit = pos - j * T::TILE;              // columns c > limit are in the future of this row
+            const int limit = pos - (t_lo + j) * T::TILE;     // columns c > limit are in the future of this row
             if (limit < T::TILE - 1) {
 #pragma unroll
                 for (int c = 0; c < T::TILE; ++c) s[c] = (c > limit) ? -INFINITY : s[c];
@@ -428,7 +445,8 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             float tile_sum = 0.f;
             // weights and their sum relative to the reference m_ref; P as bf16 pairs
             auto weights = [&](float m_ref) {
-                const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nm2 = f2_pack(-m_ref, -m_ref);
+                const float nm = (m_ref == -INFINITY) ? 0.f : -m_ref;   // a row that has seen nothing yet: all weights 0, not NaN
+                const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nm2 = f2_pack(nm, nm);
                 uint64_t sum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
 #pragma unroll
                 for (int c = 0; c < T::TILE; c += 2) {
@@ -463,8 +481,9 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             const float m_tile = max3(mx[0], mx[1], fmaxf(mx[2], mx[3])) * p.scale_log2;
             // The reference m_run of the row only moves when the tile's maximum exceeds it by more than 2^8: the
             // weights stay below 256 relative to it, the result is the same quotient, and the accumulated O (which
-            // lives in tensor memory) has to be rescaled only then.  (m_tile is finite in tile 0: token 0 is
-            // visible to every row.)
+            // lives in tensor memory) has to be rescaled only then.  (Token 0 is visible to every row, so m_tile is
+            // finite in global tile 0; a later split can start with tiles a row does not see at all: its reference
+            // stays -inf and its weights are 0 until it sees something.)
             const bool move = m_tile > m_run + kRescaleLog2;
             // tcgen05.ld / tcgen05.st are warp-wide instructions: when any row of the warp moves its reference, every
             // lane rescales its row of O (by 1 where nothing moved), once the value product of tile j-1 has landed
@@ -495,8 +514,8 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             tmem_st32u_nowait(s_addr, pk);
             l_run += tile_sum;
             // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
-            if ((long long)(j + 1) * T::TILE > kv_total) {
-                if (tid < T::TILE && (long long)j * T::TILE + tid >= kv_total) {
+            if ((long long)(t_lo + j + 1) * T::TILE > kv_total) {
+                if (tid < T::TILE && (long long)(t_lo + j) * T::TILE + tid >= kv_total) {
                     unsigned char *vrow = smem + T::OFF_STAGE + (j % NS) * T::STAGE_BYTES;
 #pragma unroll
                     for (int bx = 0; bx < T::BOXES; ++bx)
@@ -513,8 +532,10 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         if (ok) {
             tc_fence_after();
             // (tcgen05.ld is a warp-wide instruction: every lane takes part, dead rows only skip the stores)
-            const float inv = 1.f / l_run;
-            float *dst = p.out + ((size_t)(q_begin + q0 + tok) * p.H + h) * DV;
+            const size_t row_h = (size_t)(q_begin + q0 + tok) * p.H + h;
+            const bool whole = S == 1;
+            const float inv = whole ? 1.f / l_run : 1.f;          // a split leaves O unnormalised for the merge
+            float *dst = whole ? p.out + row_h * DV : p.part_o + (row_h * S + split) * DV;
 #pragma unroll
             for (int part = 0; part < DV / 32; ++part) {
                 float o[32];
@@ -526,7 +547,14 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                         *reinterpret_cast<float4 *>(dst + part * 32 + i) = make_float4(o[i] * inv, o[i + 1] * inv, o[i + 2] * inv, o[i + 3] * inv);
                 }
             }
-            if (live && p.lse) p.lse[(size_t)(q_begin + q0 + tok) * p.H + h] = (m_run + log2f(l_run)) * kLn2;
+            if (live) {
+                if (whole) {
+                    if (p.lse) p.lse[row_h] = (m_run + log2f(l_run)) * kLn2;
+                } else {
+                    p.part_ml[(row_h * S + split) * 2] = m_run;
+                    p.part_ml[(row_h * S + split) * 2 + 1] = l_run;
+                }
+            }
         } else if (!*s_abort) {
             report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
             *s_abort = 1;
@@ -585,7 +613,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                 int loaded = 0;
                 auto load_tile = [&](int t) -> bool {
                     const int st = t % NS;
-                    const int t0 = t * T::TILE;
+                    const int t0 = (t_lo + t) * T::TILE;
                     const int pj = t0 / p.P, slot0 = t0 % p.P;
                     const long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
                                                          : (long long)b * p.max_pages + pj;
@@ -647,6 +675,37 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     }
 }
 
+// ---- merge of split-KV partial results: one warp per (query row, head) -----------------------------------
+template <int DV>
+__global__ void __launch_bounds__(128)
+merge_splits_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, float *__restrict__ out,
+                    float *__restrict__ lse, int rows, int S) {
+    grid_dependency_launch();
+    grid_dependency_wait();
+    const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const float *ml = part_ml + (size_t)row * S * 2;
+    float m_max = -INFINITY;
+    for (int s = 0; s < S; ++s) m_max = fmaxf(m_max, ml[2 * s]);
+    float acc[DV / 32];
+#pragma unroll
+    for (int i = 0; i < DV / 32; ++i) acc[i] = 0.f;
+    float L = 0.f;
+    for (int s = 0; s < S; ++s) {
+        const float l = ml[2 * s + 1];
+        if (!(l > 0.f)) continue;                      // an empty range left its O unwritten
+        const float w = fast_exp2(ml[2 * s] - m_max);
+        L += w * l;
+        const float *o = part_o + ((size_t)row * S + s) * DV;
+#pragma unroll
+        for (int i = 0; i < DV / 32; ++i) acc[i] = fmaf(w, o[i * 32 + lane], acc[i]);
+    }
+    const float inv = 1.f / L;
+#pragma unroll
+    for (int i = 0; i < DV / 32; ++i) out[(size_t)row * DV + i * 32 + lane] = acc[i] * inv;
+    if (lse && lane == 0) lse[row] = (m_max + log2f(L)) * kLn2;
+}
+
 // ---- host: support check, tensor maps, launch ---------------------------------------------------------
 inline bool prefill_supported(const gva_config &cfg) {
     return cfg.cache_dtype == GVA_BF16 && cfg.page_size % 64 == 0 && cfg.H / cfg.G == kHeadsPerGroup &&
@@ -655,7 +714,7 @@ inline bool prefill_supported(const gva_config &cfg) {
 
 template <int DV, int DR>
 int launch_prefill_t(const gva_config &cfg, const MmaHostState &st, int smem_optin, const PrefillParams &p, const void *v_pool,
-                     const void *kr_pool, int B, int max_q_len, cudaStream_t stream) {
+                     const void *kr_pool, int B, int max_q_len, int n_q, cudaStream_t stream) {
     using T = PrefillTraits<DV, DR>;
     // never more blocks on an SM than its 512 tensor-memory columns can serve: pad the request if need be
     const size_t floor_bytes = (size_t)227 * 1024 / (T::BLOCKS_PER_SM + 1) + 1024;
@@ -669,20 +728,28 @@ int launch_prefill_t(const gva_config &cfg, const MmaHostState &st, int smem_opt
     if (!encode_map(st, &tm_k, kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, T::TILE,
                     DR == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B))
         return GVA_ERR_CUDA;
-    const dim3 grid((max_q_len + T::QTOK - 1) / T::QTOK, cfg.G, B);
+    const dim3 grid(((max_q_len + T::QTOK - 1) / T::QTOK) * p.num_splits, cfg.G, B);
     if (launch_pdl(fn, grid, dim3(T::THREADS), smem, stream, p, tm_v, tm_k) != cudaSuccess) {
         (void)cudaGetLastError();
         return GVA_ERR_CUDA;
+    }
+    if (p.num_splits > 1) {
+        const int rows = n_q * cfg.H;
+        if (launch_pdl(merge_splits_kernel<DV>, dim3((rows + 3) / 4), dim3(128), 0, stream, (const float *)p.part_o,
+                       (const float *)p.part_ml, p.out, p.lse, rows, p.num_splits) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return GVA_ERR_CUDA;
+        }
     }
     return GVA_OK;
 }
 
 inline int launch_prefill(const gva_config &cfg, const MmaHostState &st, int smem_optin, const PrefillParams &p,
-                          const void *v_pool, const void *kr_pool, int B, int max_q_len, cudaStream_t stream) {
+                          const void *v_pool, const void *kr_pool, int B, int max_q_len, int n_q, cudaStream_t stream) {
     if (!prefill_supported(cfg)) return GVA_ERR_UNSUPPORTED;
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
-    if (cfg.d_v == 64) return launch_prefill_t<64, 16>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, stream);
-    return launch_prefill_t<128, 32>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, stream);
+    if (cfg.d_v == 64) return launch_prefill_t<64, 16>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
+    return launch_prefill_t<128, 32>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
 }
 
 }  // namespace gva

@@ -180,6 +180,7 @@ class PrefillDeviceCase:
     q_abs: torch.Tensor
     out: torch.Tensor
     lse: torch.Tensor
+    _ws: Optional[torch.Tensor] = None
 
     @property
     def handle(self) -> int:
@@ -204,6 +205,17 @@ class PrefillDeviceCase:
     def prefill(self, max_q_len: Optional[int] = None):
         gb.gva_prefill(self.handle, self.dc.cache, self.q_abs, self.cu_q, self.ctx_lens, self.out, self.lse, self.pc.cache.B,
                        self.max_q_len if max_q_len is None else max_q_len, self.status)
+        return self.out, self.lse
+
+    def decode_multi(self, num_splits: int = 0):
+        """The same attention with split-KV (gva_decode_multi): for few new tokens over a long cached context."""
+        c = self.pc.cache
+        max_len = int(c.seq_lens.max()) if c.B else 0
+        need = gb.gva_decode_multi_workspace_bytes(self.handle, c.B, self.pc.n_q, self.max_q_len, max_len, num_splits)
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=self.q_abs.device)
+        gb.gva_decode_multi(self.handle, self.dc.cache, self.q_abs, self.cu_q, self.ctx_lens, self.out, self.lse, ws, c.B,
+                            self.pc.n_q, self.max_q_len, max_len, num_splits, self.status)
+        self._ws = ws          # keep the workspace alive until the stream has run
         return self.out, self.lse
 
     def close(self) -> None:

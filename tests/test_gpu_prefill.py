@@ -200,3 +200,49 @@ def test_absorb_many_rows_matches_oracle_and_the_small_batch_kernel(shape):
         assert np.array_equal(small.cpu().numpy().view(np.uint32), q.view(np.uint32))
     finally:
         pd.close()
+
+
+# ------------------------------------------------------------------ multi-token decode with split-KV
+@pytest.mark.parametrize("num_splits", [0, 1, 2, 7, 64])
+def test_decode_multi_matches_oracle_and_prefill(num_splits):
+    # a few new tokens per sequence over a long cached context: the oracle's chunked-prefill rows, computed by several
+    # thread blocks per query block and merged; more splits than some sequences have tiles; a sequence without new tokens
+    ctx = [5000, 130, 64, 0, 2047, 700]
+    q = [4, 1, 8, 3, 33, 0]
+    pc = wl.make_prefill_case("multi", wl.SHAPE_A, ctx, q, page_size=64, seed=510, poison_unused=True)
+    ref_out, ref_lse = orc.prefill_case(pc)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        out, lse = pd.decode_multi(num_splits=num_splits)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out[:pc.n_q].cpu().numpy().astype(np.float64); l = lse[:pc.n_q].cpu().numpy().astype(np.float64)
+        assert np.isfinite(o).all() and np.isfinite(l).all()
+        assert np.max(np.abs(o - ref_out)) <= TOL_MAXABS and rel_l2(o, ref_out) <= TOL_REL_L2
+        assert np.max(np.abs(l - ref_lse)) <= TOL_LSE
+        pd.out.fill_(float("nan"))
+        o1, _ = pd.prefill()
+        torch.cuda.synchronize()
+        assert np.max(np.abs(o1[:pc.n_q].cpu().numpy() - o)) <= 5e-3
+    finally:
+        pd.close()
+
+
+def test_decode_multi_wide_shape_and_workspace_check():
+    pc = wl.make_prefill_case("multi-b", wl.SHAPE_B, [1500, 90], [5, 2], page_size=64, seed=511)
+    ref_out, _ = orc.prefill_case(pc)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        out, _ = pd.decode_multi(num_splits=0)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out[:pc.n_q].cpu().numpy().astype(np.float64)
+        assert np.max(np.abs(o - ref_out)) <= TOL_MAXABS and rel_l2(o, ref_out) <= TOL_REL_L2
+        small = torch.empty(256, dtype=torch.uint8, device="cuda")
+        rc = gb.gva_decode_multi(pd.handle, pd.dc.cache, pd.q_abs, pd.cu_q, pd.ctx_lens, pd.out, pd.lse, small, 2, pc.n_q, 5, 1505, 4,
+                                 check=False)
+        assert rc == gb.GVA_ERR_WORKSPACE
+    finally:
+        pd.close()
