@@ -469,13 +469,25 @@ int gva_prefill(gva_handle *h, const gva_cache *cache, const float *q_abs, const
     return prefill_impl(h, cache, q_abs, cu_q, ctx_lens, out, lse, nullptr, 0, B, 0, max_q_len, 1, dev_status, stream);
 }
 
-// Splits per query block for gva_decode_multi: enough thread blocks for two per SM, never more than tiles.
+// Splits per query block for gva_decode_multi.  Automatic choice: the split count that minimises
+// (waves of thread blocks over the 2-per-SM slots) x (tiles per block + a fixed per-block cost of about 6 tiles),
+// so that the last wave is not left mostly empty; never more splits than tiles, at most 64.
 static int multi_splits(const gva_handle *h, int B, int max_q_len, int max_seq_len, int num_splits) {
     const int tiles = (max_seq_len + 63) / 64;
     int s = num_splits;
     if (s <= 0) {
         const long long blocks = (long long)B * h->cfg.G * ((max_q_len + 31) / 32);
-        s = (int)((2LL * h->sm_count + blocks - 1) / (blocks > 0 ? blocks : 1));
+        const long long slots = 2LL * h->sm_count;
+        long long best = -1;
+        s = 1;
+        for (int c = 1; c <= 64 && c <= (tiles > 0 ? tiles : 1); ++c) {
+            const long long waves = (blocks * c + slots - 1) / slots;
+            const long long cost = waves * ((tiles + c - 1) / c + 6);
+            if (best < 0 || cost < best) {
+                best = cost;
+                s = c;
+            }
+        }
     }
     if (s > tiles) s = tiles;
     if (s > 64) s = 64;
