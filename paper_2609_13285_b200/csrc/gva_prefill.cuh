@@ -423,8 +423,28 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         float m_run = -INFINITY, l_run = 0.f;          // softmax reference (log2 domain) and sum relative to it
         const uint32_t o_addr = lane_base + T::COL_O;
         bool ok = true;
+        // A warp none of whose 8 query tokens is live (short chunks, multi-token decode) only keeps the barrier protocol
+        // going: its rows of S, P and O are never used.  (S of tile j complete implies the P barrier of tile j-2 has
+        // completed, so an arrival for tile j cannot fall into an earlier phase.)
+        const bool warp_dead = warp * 8 >= nv;
         for (int j = 0; j < n_tiles; ++j) {
             if (!__all_sync(0xffffffffu, mbar_wait_spin(s_full(j % NB), (j / NB) & 1, s_abort))) { ok = false; break; }   // warp-uniform
+            // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
+            // (the score product of this tile has completed, the value product starts only after the arrivals below)
+            if ((long long)(t_lo + j + 1) * T::TILE > kv_total) {
+                if (tid < T::TILE && (long long)(t_lo + j) * T::TILE + tid >= kv_total) {
+                    unsigned char *vrow = smem + T::OFF_STAGE + (j % NS) * T::STAGE_BYTES;
+#pragma unroll
+                    for (int bx = 0; bx < T::BOXES; ++bx)
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4 *>(vrow + bx * T::VBOX_BYTES + tid * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+                }
+                fence_async_smem();
+            }
+            if (warp_dead) {
+                mbar_arrive(p_full(j));
+                continue;
+            }
             tc_fence_after();
             const uint32_t s_addr = lane_base + T::COL_S + (j % NB) * T::TILE;
             float s[T::TILE];
@@ -513,23 +533,12 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             // P goes over the first 32 columns of this tile's S (the row's only reader is this thread)
             tmem_st32u_nowait(s_addr, pk);
             l_run += tile_sum;
-            // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
-            if ((long long)(t_lo + j + 1) * T::TILE > kv_total) {
-                if (tid < T::TILE && (long long)(t_lo + j) * T::TILE + tid >= kv_total) {
-                    unsigned char *vrow = smem + T::OFF_STAGE + (j % NS) * T::STAGE_BYTES;
-#pragma unroll
-                    for (int bx = 0; bx < T::BOXES; ++bx)
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4 *>(vrow + bx * T::VBOX_BYTES + tid * 128 + c * 16) = make_uint4(0, 0, 0, 0);
-                }
-                fence_async_smem();
-            }
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(p_full(j));
         }
         if (ok && !__all_sync(0xffffffffu, mbar_wait_spin(o_full, 0, s_abort))) ok = false;
-        if (ok) {
+        if (ok && !warp_dead) {
             tc_fence_after();
             // (tcgen05.ld is a warp-wide instruction: every lane takes part, dead rows only skip the stores)
             const size_t row_h = (size_t)(q_begin + q0 + tok) * p.H + h;
@@ -555,7 +564,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                     p.part_ml[(row_h * S + split) * 2 + 1] = l_run;
                 }
             }
-        } else if (!*s_abort) {
+        } else if (!ok && !*s_abort) {
             report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
             *s_abort = 1;
         }
