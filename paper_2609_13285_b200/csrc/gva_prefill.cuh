@@ -24,10 +24,15 @@
 //     maximum grows by more than 2^8; only then is that row of O rescaled (read, multiplied, written back).
 //   S has two buffers, so the score product of tile j + 1 runs while the softmax warps work on tile j; for d_v = 64
 //   the query tile lives in tensor memory too, so every MMA reads only its B operand (the cache tile) from shared
-//   memory; two blocks share an SM (256 tensor-memory columns each).  Shared memory carries
-//   only the operands the tensor core reads (Q and the cache tiles): P never touches it.
-//   Every wait is bounded; on expiry the block records GVA_ERR_TIMEOUT, drains what it issued, frees its
-//   tensor memory and exits.
+//   memory; two blocks share an SM (256 tensor-memory columns each).  Shared memory carries only operands the tensor
+//   core reads (the cache tiles, and Q for d_v = 128): P never touches it.
+//   Split-KV (gva_decode_multi: few new tokens over a long context): a query block is shared by several thread
+//   blocks, each over a contiguous range of tiles, which leave unnormalised (O, reference, sum) per row for
+//   merge_splits_kernel.
+//   Rules this file keeps: (1) tcgen05.ld / tcgen05.st are warp-wide (.sync.aligned): they never sit inside a per-lane
+//   branch, and every wait that guards them returns a warp-uniform result; (2) every barrier that is waited on by
+//   parity is argued, at its wait, never to be two phases ahead of that waiter; (3) every wait is bounded: on expiry
+//   the block records GVA_ERR_TIMEOUT, drains what it issued, frees its tensor memory and exits.
 #pragma once
 
 #include "gva_decode_mma.cuh"
