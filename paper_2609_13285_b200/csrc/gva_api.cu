@@ -407,11 +407,11 @@ int gva_append_chunk(gva_handle *h, const gva_cache *cache, const float *v_new, 
     if (c.G * c.d_v > kAppendMaxPerThread * 128) return GVA_ERR_UNSUPPORTED;
     cudaError_t ce;
     if (c.cache_dtype == GVA_BF16)
-        ce = launch_pdl(append_chunk_kernel<__nv_bfloat16>, dim3(n_q), dim3(128), 0, s, static_cast<__nv_bfloat16 *>(cache->v_pool),
+        ce = launch_pdl(append_chunk_kernel<__nv_bfloat16>, dim3((n_q + kAppendChunkRows - 1) / kAppendChunkRows), dim3(128), 0, s, static_cast<__nv_bfloat16 *>(cache->v_pool),
                         static_cast<__nv_bfloat16 *>(cache->kr_pool), cache->block_table, v_new, kr_new, cu_q, ctx_lens, B, c.G,
                         c.d_v, c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
     else
-        ce = launch_pdl(append_chunk_kernel<float>, dim3(n_q), dim3(128), 0, s, static_cast<float *>(cache->v_pool),
+        ce = launch_pdl(append_chunk_kernel<float>, dim3((n_q + kAppendChunkRows - 1) / kAppendChunkRows), dim3(128), 0, s, static_cast<float *>(cache->v_pool),
                         static_cast<float *>(cache->kr_pool), cache->block_table, v_new, kr_new, cu_q, ctx_lens, B, c.G, c.d_v,
                         c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
     if (ce != cudaSuccess) {

@@ -332,8 +332,9 @@ append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *
                      rope, blockIdx.x);
 }
 
-// Append of a chunk of new tokens per sequence: block n writes input row n as token ctx_lens[b] + (n - cu_q[b]) of
-// the sequence b that owns the row (found by bisection of cu_q).
+// Append of a chunk of new tokens per sequence: input row n becomes token ctx_lens[b] + (n - cu_q[b]) of the sequence b
+// that owns the row (found by bisection of cu_q).  A block writes kAppendChunkRows consecutive rows.
+constexpr int kAppendChunkRows = 8;
 template <typename CT>
 __global__ void __launch_bounds__(128)
 append_chunk_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *__restrict__ block_table,
@@ -342,16 +343,23 @@ append_chunk_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int
                     int32_t *dev_status, RopeTable rope) {
     grid_dependency_launch();
     grid_dependency_wait();
-    const int n = blockIdx.x;
-    if (n >= cu_q[B]) return;
-    int lo = 0, hi = B - 1;                     // largest b with cu_q[b] <= n (empty sequences repeat an offset)
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (cu_q[mid] <= n) lo = mid;
-        else hi = mid - 1;
+    const int total = cu_q[B];
+    int b = -1;
+    for (int k = 0; k < kAppendChunkRows; ++k) {
+        const int n = blockIdx.x * kAppendChunkRows + k;
+        if (n >= total) return;
+        if (b < 0 || n >= cu_q[b + 1]) {        // largest b with cu_q[b] <= n (empty sequences repeat an offset)
+            int lo = 0, hi = B - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (cu_q[mid] <= n) lo = mid;
+                else hi = mid - 1;
+            }
+            b = lo;
+        }
+        append_row<CT>(v_pool, kr_pool, block_table, v_new, kr_new, G, d_v, d_r, P, num_pages, max_pages, dev_status, rope, n, b,
+                       ctx_lens[b] + (n - cu_q[b]));
     }
-    append_row<CT>(v_pool, kr_pool, block_table, v_new, kr_new, G, d_v, d_r, P, num_pages, max_pages, dev_status, rope, n, lo,
-                   ctx_lens[lo] + (n - cu_q[lo]));
 }
 
 // ---- fused front of a decode step: absorb and append in one launch ------------------------------------
