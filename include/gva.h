@@ -204,7 +204,8 @@ int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const
  *          pos_host [B] i32 (position t of the new token = query position), seq_lens_host [B] i32
  *          (tokens attended, normally t + 1).  If the four float inputs and out_host are all pinned
  *          (page-locked, device-mapped) memory the kernels read and write them in place over the
- *          interconnect and only pos and seq_lens are copied; otherwise every buffer is staged through
+ *          interconnect and only pos and seq_lens are brought to the device (by a one-block kernel when they are
+ *          pinned too, else by two copies); otherwise every buffer is staged through
  *          `scratch` with cudaMemcpyAsync (pageable memory makes those copies synchronous).
  *   [host] out_host [B][H][d_v] f32
  *   M                device, as in gva_absorb_query

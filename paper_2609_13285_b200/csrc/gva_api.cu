@@ -727,7 +727,34 @@ int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, 
             mapped[i] = attr.devicePointer;
         }
     }
-    if (!h2d(L.pos, pos_host, (size_t)B * 4) || !h2d(L.lens, seq_lens_host, (size_t)B * 4)) return GVA_ERR_CUDA;
+    // positions and lengths go to device scratch (every decode block reads them): by one small kernel when they are
+    // pinned, else by two copies
+    {
+        void *ints[2] = {nullptr, nullptr};
+        const void *src[2] = {pos_host, seq_lens_host};
+        bool ints_mapped = host_mapped;
+        for (int i = 0; i < 2 && ints_mapped; ++i) {
+            cudaPointerAttributes attr;
+            if (cudaPointerGetAttributes(&attr, src[i]) != cudaSuccess) {
+                (void)cudaGetLastError();
+                ints_mapped = false;
+            } else if (attr.type != cudaMemoryTypeHost || attr.devicePointer == nullptr) {
+                ints_mapped = false;
+            } else {
+                ints[i] = attr.devicePointer;
+            }
+        }
+        if (ints_mapped) {
+            if (launch_pdl(stage_ints_kernel, dim3(1), dim3(128), 0, st, static_cast<const int32_t *>(ints[0]),
+                           static_cast<const int32_t *>(ints[1]), reinterpret_cast<int32_t *>(s + L.pos),
+                           reinterpret_cast<int32_t *>(s + L.lens), B) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return GVA_ERR_CUDA;
+            }
+        } else if (!h2d(L.pos, pos_host, (size_t)B * 4) || !h2d(L.lens, seq_lens_host, (size_t)B * 4)) {
+            return GVA_ERR_CUDA;
+        }
+    }
     const int32_t *pos = reinterpret_cast<const int32_t *>(s + L.pos);
     const int32_t *lens = reinterpret_cast<const int32_t *>(s + L.lens);
     float *q_abs = reinterpret_cast<float *>(s + L.q_abs);

@@ -362,6 +362,20 @@ append_chunk_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int
     }
 }
 
+// Brings two small int32 arrays that live in pinned host memory into device scratch: one block reading them over the
+// interconnect costs less stream time than two copy-engine transfers.
+__global__ void __launch_bounds__(128)
+stage_ints_kernel(const int32_t *__restrict__ a_src, const int32_t *__restrict__ b_src, int32_t *__restrict__ a_dst,
+                  int32_t *__restrict__ b_dst, int n) {
+    grid_dependency_launch();
+    grid_dependency_wait();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const int32_t x = a_src[i], y = b_src[i];
+        a_dst[i] = x;
+        b_dst[i] = y;
+    }
+}
+
 // ---- fused front of a decode step: absorb and append in one launch ------------------------------------
 // Blocks [0, n_absorb) run absorb_block (head = block % H, batch tile = block / H); blocks
 // [n_absorb, n_absorb + B) run append_block.  The two are independent of each other.  This kernel
