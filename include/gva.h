@@ -290,6 +290,22 @@ int gva_decode_multi(gva_handle *h, const gva_cache *cache, const float *q_abs, 
                      const int32_t *ctx_lens, float *out, float *lse, void *workspace, size_t workspace_bytes, int B,
                      int n_q, int max_q_len, int max_seq_len, int num_splits, int32_t *dev_status, void *stream);
 
+/* Decode of q_len = 2 or 4 new tokens per sequence at the single-token kernel's cache-stream rate (speculative /
+ * multi-token decode; not in the paper -- Algorithm 1 applied to q_len tokens at once).  The split-KV tensor-core decode
+ * kernel of gva_decode carries the 4 * q_len (head, token) pairs of a value group as its MMA columns, so the cache is
+ * streamed once for all of them.  Every sequence has exactly q_len new tokens, already appended.
+ *   q_abs    [B * q_len][H][d_v+d_r] f32  row b * q_len + i = new token i of sequence b (from gva_absorb_query)
+ *   seq_lens [B] i32                      tokens attended by the LAST new token; new token i attends seq_lens[b] - (q_len-1-i)
+ *   out      [B * q_len][H][d_v] f32, lse [B * q_len][H] f32 or NULL
+ *   workspace                             at least gva_decode_tokens_workspace_bytes(...) bytes, 256-byte aligned
+ * bf16 cache, (d_v, d_r) = (64, 16) or (128, 32), tensor-core kernel only; otherwise GVA_ERR_UNSUPPORTED.  The queries
+ * and the softmax weights go to the tensor cores as bf16 (their hi/lo halves of the single-token layout carry the second
+ * token instead), so results carry bf16-level error like gva_prefill: |out - exact| <= 2e-2 for unit-variance data. */
+size_t gva_decode_tokens_workspace_bytes(const gva_handle *h, int B, int q_len, int max_seq_len, int num_splits);
+int gva_decode_tokens(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
+                      float *lse, void *workspace, size_t workspace_bytes, int B, int q_len, int max_seq_len,
+                      int num_splits, int32_t *dev_status, void *stream);
+
 /* Geometry of the most recent gva_decode / gqa_decode launch on this handle (reporting only):
  * number of split-KV partitions launched (thread blocks of the decode kernel). */
 int gva_last_num_splits(const gva_handle *h);

@@ -145,13 +145,13 @@ int max_units_balanced(const gva_handle *h) {
     return a > b ? a : b;
 }
 
-WorkspaceLayout workspace_layout(const gva_handle *h, int B, int num_splits) {
+WorkspaceLayout workspace_layout(const gva_handle *h, int B, int num_splits, int q_len = 1) {
     WorkspaceLayout w;
     // up to two partial records per (block, sequence): the tensor-core kernel may run two warps per group
     w.n_rec = 2 * (num_splits > 0 ? B * num_splits : max_units_balanced(h) + B);
     w.hdr_bytes = align_up((size_t)(kHdrInts + 2 * B) * 4, 256);
-    w.rec_o_bytes = align_up((size_t)w.n_rec * h->cfg.H * h->cfg.d_v * 4, 256);
-    w.rec_ml_bytes = align_up((size_t)w.n_rec * h->cfg.H * 2 * 4, 256);
+    w.rec_o_bytes = align_up((size_t)w.n_rec * h->cfg.H * q_len * h->cfg.d_v * 4, 256);     // q_len * H pseudo-heads per record
+    w.rec_ml_bytes = align_up((size_t)w.n_rec * h->cfg.H * q_len * 2 * 4, 256);
     w.total = w.hdr_bytes + w.rec_o_bytes + w.rec_ml_bytes;
     return w;
 }
@@ -167,8 +167,8 @@ int check_common(const gva_handle *h, int B, int max_seq_len, int num_splits) {
 
 template <bool GQA>
 int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspace_bytes, int B, int max_seq_len,
-                  int num_splits, cudaStream_t stream) {
-    const WorkspaceLayout w = workspace_layout(h, B, num_splits);
+                  int num_splits, cudaStream_t stream, int q_len = 1) {
+    const WorkspaceLayout w = workspace_layout(h, B, num_splits, q_len);
     if (!workspace || workspace_bytes < w.total) return GVA_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return GVA_ERR_INVALID_ARG;
     unsigned char *ws = static_cast<unsigned char *>(workspace);
@@ -189,9 +189,12 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
         kernel = GVA_KERNEL_FMA;
 #endif
     }
+    if (q_len > 1 && (GQA || kernel != GVA_KERNEL_MMA)) return GVA_ERR_UNSUPPORTED;   // multi-token decode: tensor-core kernel only
     if (kernel == GVA_KERNEL_MMA) {
 #ifdef GVA_WITH_MMA
-        int rc = launch_decode_mma<GQA>(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, max_seq_len, num_splits,
+        int rc = q_len > 1 ? launch_decode_mma_multi(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, q_len, max_seq_len, num_splits,
+                                                     max_blocks_balanced(h), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult)
+                           : launch_decode_mma<GQA>(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, max_seq_len, num_splits,
                                         max_blocks_balanced(h), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult);
         if (rc != GVA_OK) return rc;
         h->last_kernel = GVA_KERNEL_MMA;
@@ -236,10 +239,12 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     if (h->cfg.d_v == 128 && wph <= 2) wph = 1;
     // ... but no more than ~4096 warps in the whole grid: beyond that the merge blocks no longer fit beside the decode
     // blocks and start in waves after them (measured on B = 128: 2 warps per head 94 us, 4 warps 99 us, 8 warps 107 us)
-    while (wph > 1 && (long long)B * h->cfg.H * wph > 4096) wph /= 2;
+    const int HQ = h->cfg.H * q_len;           // the merge sees q_len * H pseudo-heads: out rows are [b][slot][head]
+    p.H = HQ;
+    while (wph > 1 && (long long)B * HQ * wph > 4096) wph /= 2;
     const int hpb = wph >= 4 ? 1 : 4 / wph;
     const size_t csmem = (size_t)wph * hpb * (h->cfg.d_v + 2) * sizeof(float);
-    const dim3 cgrid(B, (h->cfg.H + hpb - 1) / hpb), cblock(32 * wph * hpb);
+    const dim3 cgrid(B, (HQ + hpb - 1) / hpb), cblock(32 * wph * hpb);
     const cudaError_t ce = (h->cfg.d_v == 64) ? launch_pdl(combine_kernel<64>, cgrid, cblock, csmem, stream, p, wph, hpb)
                                               : launch_pdl(combine_kernel<128>, cgrid, cblock, csmem, stream, p, wph, hpb);
     if (ce != cudaSuccess) {
@@ -513,7 +518,7 @@ int gva_decode_multi(gva_handle *h, const gva_cache *cache, const float *q_abs, 
 
 static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
                        float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
-                       int32_t *dev_status, void *stream, int early_start, const int32_t *append_pos) {
+                       int32_t *dev_status, void *stream, int early_start, const int32_t *append_pos, int q_len = 1) {
     int rc = check_common(h, B, max_seq_len, num_splits);
     if (rc != GVA_OK) return rc;
     if (!cache) return GVA_ERR_INVALID_ARG;
@@ -542,7 +547,7 @@ static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs
     p.append_pos = append_pos;
     p.ticket = h->ticket;
     return launch_decode<false>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
-                                static_cast<cudaStream_t>(stream));
+                                static_cast<cudaStream_t>(stream), q_len);
 }
 
 int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
@@ -550,6 +555,20 @@ int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const 
                int32_t *dev_status, void *stream) {
     return decode_impl(h, cache, q_abs, seq_lens, out, lse, workspace, workspace_bytes, B, max_seq_len, num_splits,
                        dev_status, stream, 0, nullptr);
+}
+
+size_t gva_decode_tokens_workspace_bytes(const gva_handle *h, int B, int q_len, int max_seq_len, int num_splits) {
+    if (check_common(h, B, max_seq_len, num_splits) != GVA_OK || (q_len != 2 && q_len != 4)) return 0;
+    return workspace_layout(h, B, num_splits, q_len).total;
+}
+
+int gva_decode_tokens(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out, float *lse,
+                      void *workspace, size_t workspace_bytes, int B, int q_len, int max_seq_len, int num_splits,
+                      int32_t *dev_status, void *stream) {
+    if (!h) return GVA_ERR_INVALID_ARG;
+    if (q_len != 2 && q_len != 4) return GVA_ERR_UNSUPPORTED;
+    return decode_impl(h, cache, q_abs, seq_lens, out, lse, workspace, workspace_bytes, B, max_seq_len, num_splits, dev_status,
+                       stream, 0, nullptr, q_len);
 }
 
 int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const float *q_c, const float *q_r,

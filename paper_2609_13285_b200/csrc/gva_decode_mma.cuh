@@ -178,7 +178,11 @@ struct StageMeta {
     int flags;     // bit 0: first tile of its segment, bit 1: last tile of its segment
 };
 
-template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA>
+// QL > 1 (multi-token decode, QL = 2 or 4 new tokens per sequence): the 4 heads x QL tokens of a group are the N
+// columns, 8 per N-block, column c = slot * 4 + head with slot the token's index among the new ones; the queries and
+// the weights go in as plain bf16 (the hi/lo halves of the single-token layout have become the second token), slot s
+// attends to seq_len - (QL - 1 - s) tokens, and the partial records and outputs use QL * H pseudo-heads, slot * H + head.
+template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA, int QL = 1>
 __global__ void __launch_bounds__(32 * 9)
 decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = MmaTraits<DV, DR, TILE, GQA>;
@@ -188,7 +192,10 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     // dynamic shared memory is only guaranteed 16-byte aligned: round up to the swizzle atom
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    static_assert(QL == 1 || ((QL == 2 || QL == 4) && !GQA && (DR % 16) == 0), "multi-token decode: 2 or 4 new tokens, GVA cache, d_r a multiple of 16");
+    constexpr int NBK = QL == 1 ? 1 : QL / 2;     // N-blocks of 8 columns
     const int G = p.G, H = p.H;
+    const int HQ = H * QL;                        // pseudo-heads of the partial records
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int n_consumers = G * WPG;
@@ -237,9 +244,9 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         rg = block_range(p, s_off);
         if (rg.hi <= rg.lo) {   // an empty split still owns its records (weight 0 in the merge)
             if (early) grid_dependency_wait();
-            for (int i = tid; i < H * WPG; i += blockDim.x) {
-                p.rec_ml[((size_t)rg.rec_fixed * WPG * H + i) * 2] = -INFINITY;
-                p.rec_ml[((size_t)rg.rec_fixed * WPG * H + i) * 2 + 1] = 0.f;
+            for (int i = tid; i < HQ * WPG; i += blockDim.x) {
+                p.rec_ml[((size_t)rg.rec_fixed * WPG * HQ + i) * 2] = -INFINITY;
+                p.rec_ml[((size_t)rg.rec_fixed * WPG * HQ + i) * 2 + 1] = 0.f;
             }
             return;
         }
@@ -310,6 +317,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                     m.b = b;
                     m.rec = uniform ? rg.rec_fixed : unit + b;
                     m.flags = ((f == lo || f == s_off[b]) ? 1 : 0) | ((f + 1 == hi || f + 1 >= s_off[b + 1]) ? 2 : 0);
+                    if constexpr (QL > 1) m.flags |= min(max(len - t0 - TILE, 0), QL - 1) << 8;   // tokens of the sequence beyond this tile, capped
                     s_meta[st] = m;
                     const uint32_t bar = smem_u32(&full_bar[st]);
                     const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
@@ -383,6 +391,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         const uint32_t off_kr = (T::KR_ROW == 32)   ? row_qk * 32 + ((hi_qk ^ ((row_qk >> 2) & 1)) << 4)
                                 : (T::KR_ROW == 64) ? row_qk * 64 + ((hi_qk ^ ((row_qk >> 1) & 3)) << 4)
                                                     : row_qk * 48 + (hi_qk << 4);
+        if constexpr (QL == 1) {
         uint32_t qf[T::KSTEPS][2];        // B fragments of Q^T: column n = lane/4 = 2*head + {hi, lo}
         uint32_t qf8 = 0;                 // d_r = 24: B fragment of the last 8 RoPE dims
         float oacc[T::MT][4];
@@ -557,6 +566,202 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 }
             }
         }
+    
+        } else {
+            // ================= multi-token decode: QL new tokens per sequence, columns = slot * 4 + head =================
+            uint32_t qf[T::KSTEPS][NBK][2];   // B fragments of Q^T (plain bf16): column n = lane / 4 of N-block nb
+            float oacc[T::MT][NBK][4];
+            float m_run[NBK][2], l_run[NBK][2];   // per column of this lane: columns 2 jh, 2 jh + 1 of every N-block
+            const float scale = p.scale_log2;
+            // the lane's B-fragment column n = lane / 4 = r8 is (slot 2 nb + n / 4, head n % 4)
+            auto load_query = [&](int b) {
+#pragma unroll
+                for (int nb = 0; nb < NBK; ++nb) {
+                    const int slot = 2 * nb + (r8 >> 2), head = r8 & 3;
+                    const float *q = p.q + (((size_t)b * QL + slot) * H + g * kHeadsPerGroup + head) * T::DQ;
+#pragma unroll
+                    for (int kk = 0; kk < T::KSTEPS; ++kk)
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            const float2 v = *reinterpret_cast<const float2 *>(q + kk * 16 + half * 8 + 2 * jh);
+                            uint32_t w;
+                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(w) : "f"(v.y), "f"(v.x));
+                            qf[kk][nb][half] = w;
+                        }
+                }
+            };
+            if (early) grid_dependency_wait();
+            publish_header(p, s_off, plan, tid, n_consumers * 32);
+            int cur_b = -1;
+            if (rg.lo < rg.hi) {
+                cur_b = rg.b_first;
+                load_query(cur_b);
+            }
+#pragma unroll 1
+            for (int i = 0;; ++i) {
+                const int st = i % NSTAGE;
+                if (!mbar_wait_bounded(smem_u32(&full_bar[st]), (i / NSTAGE) & 1, s_abort)) {
+                    if (!*s_abort && lane == 0) report_error(p.dev_status, GVA_ERR_TIMEOUT, cur_b < 0 ? 0 : cur_b);
+                    *s_abort = 1;
+                    break;
+                }
+                const StageMeta meta = s_meta[st];
+                const int n_valid = meta.n_valid;
+                if (n_valid < 0) break;       // producer is done
+                const int b = meta.b;
+                if (meta.flags & 1) {         // a new segment: its own softmax state (and queries, if the sequence changed)
+                    if (b != cur_b) {
+                        cur_b = b;
+                        load_query(b);
+                    }
+#pragma unroll
+                    for (int nb = 0; nb < NBK; ++nb) {
+                        m_run[nb][0] = m_run[nb][1] = -INFINITY;
+                        l_run[nb][0] = l_run[nb][1] = 0.f;
+#pragma unroll
+                        for (int mt = 0; mt < T::MT; ++mt)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) oacc[mt][nb][e] = 0.f;
+                    }
+                }
+                unsigned char *stage = smem + (size_t)st * stage_bytes;
+                unsigned char *vt = stage + (size_t)g * T::VTILE_BYTES;
+                const int row0 = part * CPW * 16;
+                // tokens of this tile that slot s may see: n_valid + (tokens of the sequence beyond the tile, capped) - (QL - 1 - s)
+                const int reach = n_valid + ((meta.flags >> 8) & 0xff) - (QL - 1);
+                const bool ragged = n_valid < row0 + CPW * 16;
+                if (ragged) {
+                    const int z0 = max(n_valid, row0);
+                    const int n_zero_chunks = (row0 + CPW * 16 - z0) * 8;
+                    for (int c = lane; c < n_zero_chunks * T::BOXES; c += 32) {
+                        const int bx = c / n_zero_chunks, cc = c % n_zero_chunks;
+                        *reinterpret_cast<uint4 *>(vt + bx * T::VBOX_BYTES + (z0 + cc / 8) * 128 + (cc % 8) * 16) =
+                            make_uint4(0, 0, 0, 0);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                    __syncwarp();
+                }
+                const bool masked = reach < row0 + CPW * 16;      // some slot does not see the whole share of this warp
+                const uint32_t vt_u32 = smem_u32(vt) + row0 * 128;
+                const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES) + row0 * T::KR_ROW;
+
+                // ---- S^T = V_tile . Q^T (+ positional part): 16 tokens per m-tile, 8 columns per N-block ----
+                float sacc[CPW][NBK][4];
+#pragma unroll
+                for (int c = 0; c < CPW; ++c) {
+#pragma unroll
+                    for (int nb = 0; nb < NBK; ++nb)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) sacc[c][nb][e] = 0.f;
+#pragma unroll
+                    for (int kk = 0; kk < T::KSTEPS_V; ++kk) {
+                        uint32_t a[4];
+                        ldsm_x4(vt_u32 + (kk >> 2) * T::VBOX_BYTES + c * 2048 + (off_qk ^ ((kk & 3) << 5)), a);
+#pragma unroll
+                        for (int nb = 0; nb < NBK; ++nb) mma_bf16(sacc[c][nb], a, qf[kk][nb][0], qf[kk][nb][1]);
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < T::KSTEPS_R; ++kk) {
+                        uint32_t a[4];
+                        ldsm_x4(kr_u32 + c * 16 * T::KR_ROW + (off_kr ^ (kk << 5)), a);
+#pragma unroll
+                        for (int nb = 0; nb < NBK; ++nb)
+                            mma_bf16(sacc[c][nb], a, qf[T::KSTEPS_V + kk][nb][0], qf[T::KSTEPS_V + kk][nb][1]);
+                    }
+                }
+                // ---- online softmax per column: this lane holds columns 2 jh, 2 jh + 1 of every N-block at token rows
+                //      r8 and r8 + 8 of every m-tile; both columns belong to slot 2 nb + jh / 2 ----
+                float corr[NBK][2], m_use[NBK][2];
+#pragma unroll
+                for (int nb = 0; nb < NBK; ++nb) {
+                    const int lim = reach + 2 * nb + (jh >> 1);           // tokens of the tile this slot sees
+                    float tmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+                    for (int c = 0; c < CPW; ++c) {
+                        if (masked) {
+                            const int t_lo = row0 + c * 16 + r8;
+                            if (t_lo >= lim) sacc[c][nb][0] = sacc[c][nb][1] = -INFINITY;
+                            if (t_lo + 8 >= lim) sacc[c][nb][2] = sacc[c][nb][3] = -INFINITY;
+                        }
+                        tmax[0] = fmaxf(tmax[0], fmaxf(sacc[c][nb][0], sacc[c][nb][2]));
+                        tmax[1] = fmaxf(tmax[1], fmaxf(sacc[c][nb][1], sacc[c][nb][3]));
+                    }
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        float t = tmax[e];
+                        t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 4));
+                        t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 8));
+                        t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 16));
+                        const float m_new = fmaxf(m_run[nb][e], t * scale);
+                        m_use[nb][e] = (m_new != -INFINITY) ? m_new : 0.f;    // keeps (-inf) - (-inf) out of the exponent
+                        corr[nb][e] = fast_exp2(m_run[nb][e] - m_use[nb][e]);
+                        m_run[nb][e] = m_new;
+                        l_run[nb][e] *= corr[nb][e];
+                    }
+#pragma unroll
+                    for (int mt = 0; mt < T::MT; ++mt) {
+                        oacc[mt][nb][0] *= corr[nb][0];
+                        oacc[mt][nb][1] *= corr[nb][1];
+                        oacc[mt][nb][2] *= corr[nb][0];
+                        oacc[mt][nb][3] *= corr[nb][1];
+                    }
+                }
+                // ---- O^T += V_tile^T . P^T ----
+#pragma unroll
+                for (int c = 0; c < CPW; ++c) {
+                    uint32_t pb[NBK][2];
+#pragma unroll
+                    for (int nb = 0; nb < NBK; ++nb) {
+                        const float p00 = fast_exp2(fmaf(sacc[c][nb][0], scale, -m_use[nb][0]));   // row r8,     column 2 jh
+                        const float p01 = fast_exp2(fmaf(sacc[c][nb][1], scale, -m_use[nb][1]));   // row r8,     column 2 jh + 1
+                        const float p10 = fast_exp2(fmaf(sacc[c][nb][2], scale, -m_use[nb][0]));   // row r8 + 8, column 2 jh
+                        const float p11 = fast_exp2(fmaf(sacc[c][nb][3], scale, -m_use[nb][1]));
+                        l_run[nb][0] += p00 + p10;
+                        l_run[nb][1] += p01 + p11;
+                        uint32_t w0, w1;
+                        asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(w0) : "f"(p01), "f"(p00));
+                        asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(w1) : "f"(p11), "f"(p10));
+                        pb[nb][0] = movmatrix_trans(w0);
+                        pb[nb][1] = movmatrix_trans(w1);
+                    }
+#pragma unroll
+                    for (int mt = 0; mt < T::MT; ++mt) {
+                        uint32_t a[4];
+                        ldsm_x4_trans(vt_u32 + (mt >> 2) * T::VBOX_BYTES + c * 2048 + (off_pv ^ ((mt & 3) << 5)), a);
+#pragma unroll
+                        for (int nb = 0; nb < NBK; ++nb) mma_bf16(oacc[mt][nb], a, pb[nb][0], pb[nb][1]);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&empty_bar[st]));
+
+                // ---- segment end: one partial per (unit, sequence, part) and pseudo-head slot * H + head ----
+                if (meta.flags & 2) {
+                    const int rec = meta.rec * WPG + part;
+#pragma unroll
+                    for (int nb = 0; nb < NBK; ++nb)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            float l = l_run[nb][e];
+                            l += __shfl_xor_sync(0xffffffffu, l, 4);
+                            l += __shfl_xor_sync(0xffffffffu, l, 8);
+                            l += __shfl_xor_sync(0xffffffffu, l, 16);
+                            const int col = 2 * jh + e;                       // column of N-block nb: slot 2 nb + col / 4, head col % 4
+                            const size_t rh = (size_t)rec * HQ + (size_t)(2 * nb + (col >> 2)) * H + g * kHeadsPerGroup + (col & 3);
+                            float *o_dst = p.rec_o + rh * DV;
+#pragma unroll
+                            for (int mt = 0; mt < T::MT; ++mt) {
+                                o_dst[mt * 16 + r8] = oacc[mt][nb][e];
+                                o_dst[mt * 16 + r8 + 8] = oacc[mt][nb][2 + e];
+                            }
+                            if (r8 == 0) {
+                                p.rec_ml[rh * 2] = m_run[nb][e];
+                                p.rec_ml[rh * 2 + 1] = l;
+                            }
+                        }
+                }
+            }
+        }
     }
     // keep shared memory alive until every warp (and every copy in flight) is done
     __syncthreads();
@@ -589,14 +794,14 @@ inline bool encode_map(const MmaHostState &st, CUtensorMap *map, const void *bas
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA>
+template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA, int QL = 1>
 int launch_mma_t(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
                  int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream, int *n_blocks_out) {
     using T = MmaTraits<DV, DR, TILE, GQA>;
     const int G = cfg.G;
     const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
-    auto fn = decode_mma_kernel<DV, DR, TILE, NSTAGE, WPG, GQA>;
+    auto fn = decode_mma_kernel<DV, DR, TILE, NSTAGE, WPG, GQA, QL>;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
     CUtensorMap tm_v, tm_k;
     const uint64_t vrows = (uint64_t)p.num_pages * G * p.P;
@@ -669,6 +874,31 @@ int launch_decode_mma(const gva_config &cfg, const MmaHostState &st, int sm_coun
                                                    stream, n_blocks_out);
     return launch_mma_t<128, 32, GQA ? 16 : 32, 3, 1, GQA>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits,
                                                            max_blocks, stream, n_blocks_out);
+}
+
+// Multi-token decode (q_len = 2 or 4 new tokens per sequence) on the same kernel: see decode_mma_kernel.
+inline int launch_decode_mma_multi(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p,
+                                   int B, int q_len, int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream,
+                                   int *n_blocks_out, int *tile_out, int *rec_mult_out) {
+    if (!mma_supported(cfg, false) || (q_len != 2 && q_len != 4)) return GVA_ERR_UNSUPPORTED;
+    if (!((cfg.d_v == 64 && cfg.d_r == 16) || (cfg.d_v == 128 && cfg.d_r == 32))) return GVA_ERR_UNSUPPORTED;
+    if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
+    *tile_out = mma_tile_for(cfg, false);
+    *rec_mult_out = 1;
+#define GVA_MULTI(DV_, DR_, TILE_, QL_)                                                                                       \
+    return launch_mma_t<DV_, DR_, TILE_, 3, 1, false, QL_>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, \
+                                                            stream, n_blocks_out)
+    if (cfg.d_v == 64 && *tile_out == 64) {
+        if (q_len == 2) GVA_MULTI(64, 16, 64, 2);
+        GVA_MULTI(64, 16, 64, 4);
+    }
+    if (cfg.d_v == 64) {
+        if (q_len == 2) GVA_MULTI(64, 16, 32, 2);
+        GVA_MULTI(64, 16, 32, 4);
+    }
+    if (q_len == 2) GVA_MULTI(128, 32, 32, 2);
+    GVA_MULTI(128, 32, 32, 4);
+#undef GVA_MULTI
 }
 
 }  // namespace gva

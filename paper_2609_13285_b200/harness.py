@@ -218,6 +218,17 @@ class PrefillDeviceCase:
         self._ws = ws          # keep the workspace alive until the stream has run
         return self.out, self.lse
 
+    def decode_tokens(self, q_len: int, num_splits: int = 0):
+        """The same attention for exactly q_len new tokens per sequence on the split-KV decode kernel (gva_decode_tokens)."""
+        c = self.pc.cache
+        max_len = int(c.seq_lens.max()) if c.B else 0
+        need = gb.gva_decode_tokens_workspace_bytes(self.handle, c.B, q_len, max_len, num_splits)
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=self.q_abs.device)
+        gb.gva_decode_tokens(self.handle, self.dc.cache, self.q_abs, self.dc.seq_lens, self.out, self.lse, ws, c.B, q_len, max_len,
+                             num_splits, self.status)
+        self._ws = ws
+        return self.out, self.lse
+
     def close(self) -> None:
         self.dc.close()
 

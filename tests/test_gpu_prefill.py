@@ -246,3 +246,45 @@ def test_decode_multi_wide_shape_and_workspace_check():
         assert rc == gb.GVA_ERR_WORKSPACE
     finally:
         pd.close()
+
+
+# ------------------------------------------------------------------ q_len new tokens on the split-KV decode kernel
+@pytest.mark.parametrize("q_len", [2, 4])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+@pytest.mark.parametrize("num_splits", [0, 1, 5])
+def test_decode_tokens_matches_oracle(q_len, shape, num_splits):
+    # exactly q_len new tokens per sequence over contexts around tile and page boundaries (a context of 0 too: the first
+    # new token then sees only itself), poisoned unused slots; the oracle is the chunked-prefill oracle
+    ctx = [0, 1, 61, 62, 63, 64, 65, 127, 128, 700, 2047, 5000]
+    pc = wl.make_prefill_case("tok", shape, ctx, [q_len] * len(ctx), page_size=64, seed=520 + q_len, poison_unused=True)
+    ref_out, ref_lse = orc.prefill_case(pc)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        out, lse = pd.decode_tokens(q_len, num_splits=num_splits)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out[:pc.n_q].cpu().numpy().astype(np.float64); l = lse[:pc.n_q].cpu().numpy().astype(np.float64)
+        assert np.isfinite(o).all() and np.isfinite(l).all()
+        assert np.max(np.abs(o - ref_out)) <= TOL_MAXABS, np.max(np.abs(o - ref_out))
+        assert rel_l2(o, ref_out) <= TOL_REL_L2
+        assert np.max(np.abs(l - ref_lse)) <= TOL_LSE
+    finally:
+        pd.close()
+
+
+def test_decode_tokens_unsupported_and_page_size_32():
+    pc = wl.make_prefill_case("tok32", wl.SHAPE_A, [300, 31], [2, 2], page_size=32, seed=530)
+    ref_out, _ = orc.prefill_case(pc)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        out, _ = pd.decode_tokens(2)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        assert np.max(np.abs(out[:pc.n_q].cpu().numpy().astype(np.float64) - ref_out)) <= TOL_MAXABS
+        ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+        rc = gb.gva_decode_tokens(pd.handle, pd.dc.cache, pd.q_abs, pd.dc.seq_lens, pd.out, pd.lse, ws, 2, 3, 302, 0, check=False)
+        assert rc == gb.GVA_ERR_UNSUPPORTED
+    finally:
+        pd.close()
