@@ -519,7 +519,7 @@ def measure_prefill(rank, local_rank, dist, args, torch, gb, harness, B=8, T=819
     return res
 
 
-def measure_multi(rank, local_rank, dist, args, torch, gb, harness, q_len=4):
+def measure_multi(rank, local_rank, dist, args, torch, gb, harness, q_len=4, on_decode_kernel=False):
     """Multi-token decode on the headline workload's shape: q_len new tokens per sequence over the long cached context
     (gva_decode_multi: the tcgen05 kernel with split-KV + merge); the cache stream is the same as cfg2's."""
     from paper_2609_13285_b200 import multirank, workloads as wl
@@ -535,12 +535,18 @@ def measure_multi(rank, local_rank, dist, args, torch, gb, harness, q_len=4):
     pools = [(pd.dc.v_pool, pd.dc.kr_pool), (pd.dc.v_pool.clone(), pd.dc.kr_pool.clone())]
     c = pc.cache
     caches = [gb.make_cache(v, k, pd.dc.block_table, c.num_pages, c.max_pages_per_seq) for v, k in pools]
-    need = gb.gva_decode_multi_workspace_bytes(pd.handle, B, pc.n_q, q_len, T, 0)
+    if on_decode_kernel:
+        need = gb.gva_decode_tokens_workspace_bytes(pd.handle, B, q_len, T, 0)
+    else:
+        need = gb.gva_decode_multi_workspace_bytes(pd.handle, B, pc.n_q, q_len, T, 0)
     ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
 
     def call(i):
-        gb.gva_decode_multi(pd.handle, caches[i & 1], pd.q_abs, pd.cu_q, pd.ctx_lens, pd.out, pd.lse, ws, B, pc.n_q, q_len, T, 0,
-                            pd.status)
+        if on_decode_kernel:
+            gb.gva_decode_tokens(pd.handle, caches[i & 1], pd.q_abs, pd.dc.seq_lens, pd.out, pd.lse, ws, B, q_len, T, 0, pd.status)
+        else:
+            gb.gva_decode_multi(pd.handle, caches[i & 1], pd.q_abs, pd.cu_q, pd.ctx_lens, pd.out, pd.lse, ws, B, pc.n_q, q_len, T,
+                                0, pd.status)
 
     for i in range(warmup):
         call(i)
@@ -556,7 +562,9 @@ def measure_multi(rank, local_rank, dist, args, torch, gb, harness, q_len=4):
     peak = load_peaks()[0]
     gbps = c.cache_bytes() / (ms * 1e-3) / 1e9
     res = {"workload": f"multi-token decode, cfg2 shapes: {q_len} new tokens per sequence over T = {T} cached tokens, B = {B}, "
-                       "bf16 paged cache (two pool copies alternate: every call streams from HBM)",
+                       "bf16 paged cache (two pool copies alternate: every call streams from HBM); "
+                       + ("gva_decode_tokens (split-KV mma.sync decode kernel)" if on_decode_kernel else
+                          "gva_decode_multi (tcgen05 kernel with split-KV)"),
            "q_len": q_len, "ms_per_call": ms, "cache_read_GBps": gbps, "frac_of_measured_peak": gbps / peak,
            "tokens_per_s": B * q_len / (ms * 1e-3), "steps": steps, "device_status": int(pd.status.item())}
     pd.close()
@@ -601,10 +609,13 @@ def main() -> None:
     kernel = {"auto": gb.GVA_KERNEL_AUTO, "fma": gb.GVA_KERNEL_FMA, "mma": gb.GVA_KERNEL_MMA}[args.kernel]
 
     name = args.workload
-    if name in ("prefill", "prefill-ncu", "prefill-wide", "layer", "multi", "multi-q1", "multi-q8", "multi-q32"):      # side workloads on their own (small runs for profiler captures)
+    if name in ("prefill", "prefill-ncu", "prefill-wide", "layer", "multi", "multi-q1", "multi-q8", "multi-q32", "tokens-q2", "tokens-q4"):      # side workloads on their own (small runs for profiler captures)
         if rank == 0:
             if name == "layer":
                 res = measure_layer(rank, local_rank, None, args, kernel, torch, gb, harness)
+            elif name.startswith("tokens"):
+                res = measure_multi(rank, local_rank, None, args, torch, gb, harness, q_len=int(name.split("-q")[1]),
+                                    on_decode_kernel=True)
             elif name.startswith("multi"):
                 res = measure_multi(rank, local_rank, None, args, torch, gb, harness,
                                     q_len=int(name.split("-q")[1]) if "-q" in name else 4)
@@ -647,6 +658,8 @@ def main() -> None:
         others["gqa_matched_cfg2"] = gq
         others["layer_step_cfg2"] = measure_layer(rank, local_rank, dist, short, kernel, torch, gb, harness)
         others["decode_multi_cfg2_q4"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=4)
+        others["decode_tokens_cfg2_q2"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=2, on_decode_kernel=True)
+        others["decode_tokens_cfg2_q4"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=4, on_decode_kernel=True)
         others["prefill"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness)
         others["prefill_wide"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness, B=4, T=8192, wide=True)
 

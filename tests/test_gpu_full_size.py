@@ -159,3 +159,33 @@ def test_decode_multi_bench_size_sampled_rows():
             ref_o, ref_l = orc.decode(c.v_pool, c.kr_pool, c.block_table, lens, qa, s.H, d_c=s.d_c)
             assert np.max(np.abs(o[n] - ref_o[b])) <= 2e-2, (b, i)
             assert np.max(np.abs(l[n] - ref_l[b])) <= 2e-2, (b, i)
+
+
+@pytest.mark.parametrize("q_len", [2, 4])
+def test_decode_tokens_bench_size_sampled_rows(q_len):
+    # bench.py's gva_decode_tokens workload (cfg2 shapes), same launch: every new token of a sample of sequences against
+    # the decode oracle over its prefix; finiteness for the rest
+    from oracle import gva_oracle as orc
+    B, T = 32, 32768
+    pc = wl.make_prefill_case("multi", wl.SHAPE_A, [T - q_len] * B, [q_len] * B, page_size=64, seed=wl.MASTER_SEED + 7300)
+    c, s = pc.cache, pc.cache.shape
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        out, lse = pd.decode_tokens(q_len)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out.cpu().numpy().astype(np.float64)
+        l = lse.cpu().numpy().astype(np.float64)
+        q_abs = pd.q_abs.cpu().numpy().astype(np.float64)
+    finally:
+        pd.close()
+    assert np.isfinite(o).all() and np.isfinite(l).all()
+    for b in (0, 17, B - 1):
+        for i in range(q_len):
+            n = int(pc.cu_q[b]) + i
+            lens = np.zeros(c.B, dtype=np.int32); lens[b] = T - q_len + i + 1
+            qa = np.zeros((c.B, s.H, s.d_v + s.d_r)); qa[b] = q_abs[n]
+            ref_o, ref_l = orc.decode(c.v_pool, c.kr_pool, c.block_table, lens, qa, s.H, d_c=s.d_c)
+            assert np.max(np.abs(o[n] - ref_o[b])) <= 2e-2, (b, i)
+            assert np.max(np.abs(l[n] - ref_l[b])) <= 2e-2, (b, i)
