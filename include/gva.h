@@ -290,7 +290,7 @@ int gva_decode_multi(gva_handle *h, const gva_cache *cache, const float *q_abs, 
                      const int32_t *ctx_lens, float *out, float *lse, void *workspace, size_t workspace_bytes, int B,
                      int n_q, int max_q_len, int max_seq_len, int num_splits, int32_t *dev_status, void *stream);
 
-/* Decode of q_len = 2 or 4 new tokens per sequence at the single-token kernel's cache-stream rate (speculative /
+/* Decode of q_len = 2, 3 or 4 new tokens per sequence at the single-token kernel's cache-stream rate (speculative /
  * multi-token decode; not in the paper -- Algorithm 1 applied to q_len tokens at once).  The split-KV tensor-core decode
  * kernel of gva_decode carries the 4 * q_len (head, token) pairs of a value group as its MMA columns, so the cache is
  * streamed once for all of them.  Every sequence has exactly q_len new tokens, already appended.

@@ -546,6 +546,7 @@ static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs
     p.early_start = early_start;
     p.append_pos = append_pos;
     p.ticket = h->ticket;
+    p.q_len = q_len;
     return launch_decode<false>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
                                 static_cast<cudaStream_t>(stream), q_len);
 }
@@ -558,7 +559,7 @@ int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const 
 }
 
 size_t gva_decode_tokens_workspace_bytes(const gva_handle *h, int B, int q_len, int max_seq_len, int num_splits) {
-    if (check_common(h, B, max_seq_len, num_splits) != GVA_OK || (q_len != 2 && q_len != 4)) return 0;
+    if (check_common(h, B, max_seq_len, num_splits) != GVA_OK || q_len < 2 || q_len > 4) return 0;
     return workspace_layout(h, B, num_splits, q_len).total;
 }
 
@@ -566,7 +567,7 @@ int gva_decode_tokens(gva_handle *h, const gva_cache *cache, const float *q_abs,
                       void *workspace, size_t workspace_bytes, int B, int q_len, int max_seq_len, int num_splits,
                       int32_t *dev_status, void *stream) {
     if (!h) return GVA_ERR_INVALID_ARG;
-    if (q_len != 2 && q_len != 4) return GVA_ERR_UNSUPPORTED;
+    if (q_len < 2 || q_len > 4) return GVA_ERR_UNSUPPORTED;
     return decode_impl(h, cache, q_abs, seq_lens, out, lse, workspace, workspace_bytes, B, max_seq_len, num_splits, dev_status,
                        stream, 0, nullptr, q_len);
 }

@@ -43,6 +43,7 @@ struct DecodeParams {
     int early_start;             // 1: launched right behind step_front_kernel (see gva_decode_mma.cuh)
     const int32_t *append_pos;   // early_start: position being appended per sequence (its tile must not be read early)
     float scale_log2;            // softmax scale * log2(e)
+    int q_len;                   // multi-token decode: new tokens per sequence (2..4); 0 or 1 otherwise
 };
 
 __device__ __forceinline__ void report_error(int32_t *dev_status, int code, int b) {

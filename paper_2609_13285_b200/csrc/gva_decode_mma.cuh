@@ -195,7 +195,8 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     static_assert(QL == 1 || ((QL == 2 || QL == 4) && !GQA && (DR % 16) == 0), "multi-token decode: 2 or 4 new tokens, GVA cache, d_r a multiple of 16");
     constexpr int NBK = QL == 1 ? 1 : QL / 2;     // N-blocks of 8 columns
     const int G = p.G, H = p.H;
-    const int HQ = H * QL;                        // pseudo-heads of the partial records
+    const int ql = QL == 1 ? 1 : p.q_len;         // new tokens per sequence actually present (<= QL; the other slots stay empty)
+    const int HQ = H * ql;                        // pseudo-heads of the partial records
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int n_consumers = G * WPG;
@@ -317,7 +318,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                     m.b = b;
                     m.rec = uniform ? rg.rec_fixed : unit + b;
                     m.flags = ((f == lo || f == s_off[b]) ? 1 : 0) | ((f + 1 == hi || f + 1 >= s_off[b + 1]) ? 2 : 0);
-                    if constexpr (QL > 1) m.flags |= min(max(len - t0 - TILE, 0), QL - 1) << 8;   // tokens of the sequence beyond this tile, capped
+                    if constexpr (QL > 1) m.flags |= min(max(len - t0 - TILE, 0), ql - 1) << 8;   // tokens of the sequence beyond this tile, capped
                     s_meta[st] = m;
                     const uint32_t bar = smem_u32(&full_bar[st]);
                     const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
@@ -578,12 +579,14 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 #pragma unroll
                 for (int nb = 0; nb < NBK; ++nb) {
                     const int slot = 2 * nb + (r8 >> 2), head = r8 & 3;
-                    const float *q = p.q + (((size_t)b * QL + slot) * H + g * kHeadsPerGroup + head) * T::DQ;
+                    const bool present = slot < ql;       // an absent slot gets a zero query; its columns are masked everywhere
+                    const float *q = p.q + (((size_t)b * ql + (present ? slot : 0)) * H + g * kHeadsPerGroup + head) * T::DQ;
 #pragma unroll
                     for (int kk = 0; kk < T::KSTEPS; ++kk)
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
-                            const float2 v = *reinterpret_cast<const float2 *>(q + kk * 16 + half * 8 + 2 * jh);
+                            float2 v = *reinterpret_cast<const float2 *>(q + kk * 16 + half * 8 + 2 * jh);
+                            if (!present) v = make_float2(0.f, 0.f);
                             uint32_t w;
                             asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(w) : "f"(v.y), "f"(v.x));
                             qf[kk][nb][half] = w;
@@ -628,7 +631,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 unsigned char *vt = stage + (size_t)g * T::VTILE_BYTES;
                 const int row0 = part * CPW * 16;
                 // tokens of this tile that slot s may see: n_valid + (tokens of the sequence beyond the tile, capped) - (QL - 1 - s)
-                const int reach = n_valid + ((meta.flags >> 8) & 0xff) - (QL - 1);
+                const int reach = n_valid + ((meta.flags >> 8) & 0xff) - (ql - 1);
                 const bool ragged = n_valid < row0 + CPW * 16;
                 if (ragged) {
                     const int z0 = max(n_valid, row0);
@@ -641,7 +644,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                     __syncwarp();
                 }
-                const bool masked = reach < row0 + CPW * 16;      // some slot does not see the whole share of this warp
+                const bool masked = reach < row0 + CPW * 16 || ql < QL;      // some slot does not see the whole share of this warp
                 const uint32_t vt_u32 = smem_u32(vt) + row0 * 128;
                 const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES) + row0 * T::KR_ROW;
 
@@ -674,7 +677,8 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 float corr[NBK][2], m_use[NBK][2];
 #pragma unroll
                 for (int nb = 0; nb < NBK; ++nb) {
-                    const int lim = reach + 2 * nb + (jh >> 1);           // tokens of the tile this slot sees
+                    const int slot_l = 2 * nb + (jh >> 1);
+                    const int lim = slot_l < ql ? reach + slot_l : 0;     // tokens of the tile this slot sees (an absent slot: none)
                     float tmax[2] = {-INFINITY, -INFINITY};
 #pragma unroll
                     for (int c = 0; c < CPW; ++c) {
@@ -747,6 +751,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                             l += __shfl_xor_sync(0xffffffffu, l, 8);
                             l += __shfl_xor_sync(0xffffffffu, l, 16);
                             const int col = 2 * jh + e;                       // column of N-block nb: slot 2 nb + col / 4, head col % 4
+                            if (2 * nb + (col >> 2) >= ql) continue;           // (uniform over the lanes that reduce together)
                             const size_t rh = (size_t)rec * HQ + (size_t)(2 * nb + (col >> 2)) * H + g * kHeadsPerGroup + (col & 3);
                             float *o_dst = p.rec_o + rh * DV;
 #pragma unroll
@@ -880,7 +885,7 @@ int launch_decode_mma(const gva_config &cfg, const MmaHostState &st, int sm_coun
 inline int launch_decode_mma_multi(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p,
                                    int B, int q_len, int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream,
                                    int *n_blocks_out, int *tile_out, int *rec_mult_out) {
-    if (!mma_supported(cfg, false) || (q_len != 2 && q_len != 4)) return GVA_ERR_UNSUPPORTED;
+    if (!mma_supported(cfg, false) || q_len < 2 || q_len > 4) return GVA_ERR_UNSUPPORTED;
     if (!((cfg.d_v == 64 && cfg.d_r == 16) || (cfg.d_v == 128 && cfg.d_r == 32))) return GVA_ERR_UNSUPPORTED;
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
     *tile_out = mma_tile_for(cfg, false);
@@ -890,7 +895,7 @@ inline int launch_decode_mma_multi(const gva_config &cfg, const MmaHostState &st
                                                             stream, n_blocks_out)
     if (cfg.d_v == 64 && *tile_out == 64) {
         if (q_len == 2) GVA_MULTI(64, 16, 64, 2);
-        GVA_MULTI(64, 16, 64, 4);
+        GVA_MULTI(64, 16, 64, 4);       // three tokens run in the four-token kernel with one slot empty
     }
     if (cfg.d_v == 64) {
         if (q_len == 2) GVA_MULTI(64, 16, 32, 2);

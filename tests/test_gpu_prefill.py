@@ -249,7 +249,7 @@ def test_decode_multi_wide_shape_and_workspace_check():
 
 
 # ------------------------------------------------------------------ q_len new tokens on the split-KV decode kernel
-@pytest.mark.parametrize("q_len", [2, 4])
+@pytest.mark.parametrize("q_len", [2, 3, 4])
 @pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
 @pytest.mark.parametrize("num_splits", [0, 1, 5])
 def test_decode_tokens_matches_oracle(q_len, shape, num_splits):
@@ -284,7 +284,7 @@ def test_decode_tokens_unsupported_and_page_size_32():
         assert int(pd.status.item()) == 0
         assert np.max(np.abs(out[:pc.n_q].cpu().numpy().astype(np.float64) - ref_out)) <= TOL_MAXABS
         ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
-        rc = gb.gva_decode_tokens(pd.handle, pd.dc.cache, pd.q_abs, pd.dc.seq_lens, pd.out, pd.lse, ws, 2, 3, 302, 0, check=False)
+        rc = gb.gva_decode_tokens(pd.handle, pd.dc.cache, pd.q_abs, pd.dc.seq_lens, pd.out, pd.lse, ws, 2, 5, 302, 0, check=False)
         assert rc == gb.GVA_ERR_UNSUPPORTED
     finally:
         pd.close()
