@@ -8,7 +8,7 @@ d_r=16, T=32768, bf16 cache in 64-token pages behind a permuted block table).  T
 GB/s: the live cache bytes one step must stream, divided by the step time.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-                    [--workload cfg1|cfg2|cfg3|cfg4|prefill|layer] [--kernel auto|fma|mma] [--headline-only]
+                    [--workload cfg0|cfg1|cfg2|cfg3|cfg4|prefill|layer|...] [--kernel auto|fma|mma] [--headline-only]
 
 N > 1 runs N independent replicas (one process per GPU under torch.distributed.run): the path has no
 exchange step, so there is no collective on the data path; only the timing barrier and the
@@ -48,6 +48,8 @@ def load_peaks():
 def make_workload(name: str, rank: int):
     from paper_2609_13285_b200 import workloads as wl
     shift = 7919 * rank
+    if name == "cfg0":
+        return wl.config0(seed=wl.MASTER_SEED + shift)
     if name == "cfg1":
         return wl.config1(seed=wl.MASTER_SEED + 1000 + shift)
     if name == "cfg2":
@@ -70,6 +72,7 @@ def make_workload(name: str, rank: int):
 
 
 WORKLOAD_TEXT = {
+    "cfg0": "single decode step, contiguous f32 cache (B=1, T=128): latency-bound, the CUDA-core kernel",
     "cfg1": "batched decode step, contiguous bf16 cache (B=8, T=4096)",
     "cfg2": "long-context paged decode step (B=32, T=32768, 64-token pages, permuted block table)",
     "cfg3": "wider-head ragged serving batch (B=64, H=32, G=8, d_v=128, seq_lens ~ U[1024,16384], paged)",
@@ -319,7 +322,28 @@ def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with
     d0, d1 = timed(decode_only, steps)                # the dominant kernel: K gva_decode calls back to back
     sync_all()
     clocks = sampler.finish() if sampler else None
+    # Small workloads are bound by the host's launch rate when launched one call at a time: replay the same steps from a
+    # CUDA graph as well (programmatic dependent launches survive capture) to show the device-side time per step.
+    graph_ms = None
+    if n_layers == 1 and case.cache_bytes() < 100e6:
+        n_rep = min(64, len(layers[0].caches))
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(n_rep):
+                step(i)
+        g.replay()
+        torch.cuda.synchronize()
+        reps = max(3, steps // n_rep)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(torch.cuda.current_stream())
+        for _ in range(reps):
+            g.replay()
+        b.record(torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        graph_ms = a.elapsed_time(b) / (reps * n_rep)
+        del g
     res = {"case": case, "layers": n_layers, "step_ms": step_ms, "decode_ms": d0.elapsed_time(d1) / steps / n_layers,
+           "graph_step_ms": graph_ms,
            "steps": steps, "warmup": warmup, "clocks": clocks, "status": int(dc.status.item()),
            "partitions": gb.gva_last_num_splits(dc.handle),
            "kernel": {1: "fma", 2: "mma"}.get(gb.gva_last_kernel(dc.handle), "?"),
@@ -637,7 +661,7 @@ def main() -> None:
         peak = load_peaks()[0]
         short = argparse.Namespace(**vars(args))
         short.steps, short.warmup = max(20, args.steps // 3), 10
-        for other in ("cfg1", "cfg3", "cfg4", "cfg2-dr24", "cfg2-dr0"):
+        for other in ("cfg0", "cfg1", "cfg3", "cfg4", "cfg2-dr24", "cfg2-dr0"):
             o = measure(other, rank, local_rank, dist, short, kernel, torch, gb, harness, with_e2e=False,
                         with_clocks=True)
             per_layer = o["cache_bytes"] / o["layers"]
@@ -646,6 +670,7 @@ def main() -> None:
                 "cache_read_GBps": o["cache_bytes"] / (o["step_ms"] * 1e-3) / 1e9,
                 "decode_steps_per_s": 1e3 / o["step_ms"],
                 "gva_decode_ms_per_call": o["decode_ms"],
+                "ms_per_step_graph_replay": o["graph_step_ms"],
                 "gva_decode_GBps": per_layer / (o["decode_ms"] * 1e-3) / 1e9,
                 "gva_decode_frac_of_measured_peak": per_layer / (o["decode_ms"] * 1e-3) / 1e9 / peak,
                 "cache_bytes_per_step": o["cache_bytes"], "kernel": o["kernel"], "partitions": o["partitions"],
