@@ -641,7 +641,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                     const int row = (int)((page * p.G + g) * p.P + slot0);
 #pragma unroll
                     for (int bx = 0; bx < T::BOXES; ++bx) tma_load_2d(dst + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, kv_full(st));
-                    tma_load_2d(dst + T::V_BYTES, &tm_k, 0, (int)(page * p.P + slot0), kv_full(st));
+                    if constexpr (DR > 0) tma_load_2d(dst + T::V_BYTES, &tm_k, 0, (int)(page * p.P + slot0), kv_full(st));   // (no positional tile in a value-only cache)
                     ++loaded;
                     return true;
                 };
@@ -723,7 +723,7 @@ merge_splits_kernel(const float *__restrict__ part_o, const float *__restrict__ 
 // ---- host: support check, tensor maps, launch ---------------------------------------------------------
 inline bool prefill_supported(const gva_config &cfg) {
     return cfg.cache_dtype == GVA_BF16 && cfg.page_size % 64 == 0 && cfg.H / cfg.G == kHeadsPerGroup &&
-           ((cfg.d_v == 64 && cfg.d_r == 16) || (cfg.d_v == 128 && cfg.d_r == 32));
+           ((cfg.d_v == 64 && (cfg.d_r == 16 || cfg.d_r == 0)) || (cfg.d_v == 128 && (cfg.d_r == 32 || cfg.d_r == 0)));
 }
 
 template <int DV, int DR>
@@ -739,9 +739,12 @@ int launch_prefill_t(const gva_config &cfg, const MmaHostState &st, int smem_opt
     CUtensorMap tm_v, tm_k;
     if (!encode_map(st, &tm_v, v_pool, DV, (uint64_t)p.num_pages * cfg.G * p.P, 64, T::TILE, CU_TENSOR_MAP_SWIZZLE_128B))
         return GVA_ERR_CUDA;
-    if (!encode_map(st, &tm_k, kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, T::TILE,
-                    DR == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B))
+    if (DR == 0) {
+        tm_k = tm_v;      // value-only cache: there is no positional-key tile to describe (the kernel never uses this map)
+    } else if (!encode_map(st, &tm_k, kr_pool, DR, (uint64_t)p.num_pages * p.P, DR > 0 ? DR : 16, T::TILE,
+                           DR == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B)) {
         return GVA_ERR_CUDA;
+    }
     const dim3 grid(((max_q_len + T::QTOK - 1) / T::QTOK) * p.num_splits, cfg.G, B);
     if (launch_pdl(fn, grid, dim3(T::THREADS), smem, stream, p, tm_v, tm_k) != cudaSuccess) {
         (void)cudaGetLastError();
@@ -762,6 +765,10 @@ inline int launch_prefill(const gva_config &cfg, const MmaHostState &st, int sme
                           const void *v_pool, const void *kr_pool, int B, int max_q_len, int n_q, cudaStream_t stream) {
     if (!prefill_supported(cfg)) return GVA_ERR_UNSUPPORTED;
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
+    if (cfg.d_r == 0) {       // value-only cache
+        if (cfg.d_v == 64) return launch_prefill_t<64, 0>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
+        return launch_prefill_t<128, 0>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
+    }
     if (cfg.d_v == 64) return launch_prefill_t<64, 16>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
     return launch_prefill_t<128, 32>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
 }

@@ -429,7 +429,6 @@ def test_value_only_cache_long_context_and_what_it_does_not_cover():
         t = torch.zeros(4096, dtype=torch.float32, device="cuda")
         i = torch.zeros(16, dtype=torch.int32, device="cuda")
         cache = gb.make_cache(t, None, None, 4, 4)
-        assert gb.gva_prefill(h, cache, t, i, i, t, None, 1, 8, check=False) == gb.GVA_ERR_UNSUPPORTED
         assert gb.gva_project_in(h, cache, t, t, 128, i, t, 1, check=False) == gb.GVA_ERR_UNSUPPORTED
     finally:
         gb.gva_destroy(h)

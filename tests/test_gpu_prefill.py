@@ -288,3 +288,21 @@ def test_decode_tokens_unsupported_and_page_size_32():
         assert rc == gb.GVA_ERR_UNSUPPORTED
     finally:
         pd.close()
+
+
+@pytest.mark.parametrize("shape", [wl.SHAPE_A0, wl.SHAPE_B0])
+def test_prefill_and_decode_multi_value_only_cache(shape):
+    # the cache without a positional slice (d_r = 0): keys are the reconstructed content keys alone, scale 1/sqrt(d_c)
+    pc = wl.make_prefill_case("pf0", shape, [0, 70, 1000], [130, 33, 5], page_size=64, seed=540, poison_unused=True)
+    check(pc)
+    ref_out, _ = orc.prefill_case(pc)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        out, _ = pd.decode_multi(num_splits=3)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out[:pc.n_q].cpu().numpy().astype(np.float64)
+        assert np.max(np.abs(o - ref_out)) <= TOL_MAXABS and rel_l2(o, ref_out) <= TOL_REL_L2
+    finally:
+        pd.close()
