@@ -306,3 +306,26 @@ def test_prefill_and_decode_multi_value_only_cache(shape):
         assert np.max(np.abs(o - ref_out)) <= TOL_MAXABS and rel_l2(o, ref_out) <= TOL_REL_L2
     finally:
         pd.close()
+
+
+def test_append_then_decode_tokens_follows_algorithm_order():
+    # Algorithm 1 for three new tokens at once: absorb, append all three, then attend; the new tokens' own rows come
+    # from the append (bit-exact against the oracle's), each new token sees its predecessors and itself
+    q_len = 3
+    pc = wl.make_prefill_case("atok", wl.SHAPE_A, [63, 640, 0, 4095], [q_len] * 4, page_size=64, seed=541)
+    c = pc.cache
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        pd.append()
+        out, lse = pd.decode_tokens(q_len)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        v, k = pd.dc.pools_to_host()
+        o = out[:pc.n_q].cpu().numpy().astype(np.float64)
+    finally:
+        pd.close()
+    assert orc.append_chunk(c.v_pool, c.kr_pool, c.block_table, pc.v_new, pc.kr_new, pc.cu_q, pc.ctx_lens) == 0
+    assert np.array_equal(v, c.v_pool) and np.array_equal(k, c.kr_pool)
+    ref_out, _ = orc.prefill_case(pc)
+    assert np.max(np.abs(o - ref_out)) <= TOL_MAXABS and rel_l2(o, ref_out) <= TOL_REL_L2
