@@ -354,3 +354,41 @@ def test_prefill_and_decode_tokens_flat_and_peaked_scores(q_gain):
         assert np.max(np.abs(out2[:pc.n_q].cpu().numpy().astype(np.float64) - o)) <= (5e-3 if q_gain == 0 else 0.06)
     finally:
         pd.close()
+
+
+@pytest.mark.parametrize("it", range(16))
+def test_random_cases_through_every_multi_token_entry_point(it):
+    # seeded random batches (shape, batch, contexts, chunk lengths, page size, paged or contiguous, poisoned slots) through
+    # gva_prefill, gva_decode_multi (given and automatic split counts) and gva_decode_tokens, against the oracle
+    rng = np.random.default_rng(7000 + it)
+    shape = wl.SHAPE_A if it % 3 else wl.SHAPE_B
+    B = int(rng.integers(1, 7))
+    ctx = rng.integers(0, 1500, size=B)
+    mode = it % 4
+    if mode == 3:
+        q = np.full(B, int(rng.integers(2, 5)))
+    else:
+        q = rng.integers(0, 200, size=B)
+        if q.sum() == 0:
+            q[0] = 5
+    pc = wl.make_prefill_case("rnd", shape, ctx, q, page_size=64 if it % 5 else 128, seed=9000 + it, poison_unused=True,
+                              paged=bool(it % 2))
+    ref, ref_l = orc.prefill_case(pc)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        if mode == 0:
+            out, lse = pd.prefill()
+        elif mode == 1:
+            out, lse = pd.decode_multi(num_splits=int(rng.integers(1, 9)))
+        elif mode == 2:
+            out, lse = pd.decode_multi(num_splits=0)
+        else:
+            out, lse = pd.decode_tokens(int(q[0]), num_splits=int(rng.integers(0, 4)))
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out[:pc.n_q].cpu().numpy().astype(np.float64); l = lse[:pc.n_q].cpu().numpy().astype(np.float64)
+        assert np.isfinite(o).all() and np.isfinite(l).all()
+        assert np.max(np.abs(o - ref)) <= TOL_MAXABS and np.max(np.abs(l - ref_l)) <= TOL_LSE
+    finally:
+        pd.close()
