@@ -31,9 +31,20 @@
 
 #define ORACLE_F32 0
 #define ORACLE_BF16 1
+#define ORACLE_E4M3 2   /* 8-bit float: 1 sign, 4 exponent (bias 7), 3 mantissa bits; no infinity, 0x7F / 0xFF = NaN, largest finite 448 */
 
 /* ---- storage <-> double ---------------------------------------------------------------------- */
+/* value of an e4m3 code, exactly */
+double oracle_e4m3_to_double(uint8_t c) {
+    int e = (c >> 3) & 15, m = c & 7;
+    double v;
+    if ((c & 0x7F) == 0x7F) return NAN;
+    v = e == 0 ? ldexp((double)m, -9) : ldexp(1.0 + m / 8.0, e - 7);
+    return (c & 0x80) ? -v : v;
+}
+
 static double load_elem(const void *pool, int dtype, int64_t idx) {
+    if (dtype == ORACLE_E4M3) return oracle_e4m3_to_double(((const uint8_t *)pool)[idx]);
     if (dtype == ORACLE_BF16) {
         uint32_t u = ((uint32_t)((const uint16_t *)pool)[idx]) << 16;
         float f;
@@ -67,8 +78,34 @@ uint16_t oracle_bf16_from_double(double x) {
     return (uint16_t)(sign | (uint16_t)(u >> 16));
 }
 
+/* Round a double to e4m3, nearest with ties to even, straight from the fp64 value; magnitudes beyond the largest finite
+ * value 448 saturate to it (there is no infinity to round to), NaN stays NaN.  Same construction as above: scale so
+ * that the representable numbers near |x| are the integers (quantum 2^(e-3) for |x| in [2^e, 2^(e+1)), fixed quantum
+ * 2^-9 below the smallest normal 2^-6), round with nearbyint, scale back, then read off exponent and mantissa. */
+uint8_t oracle_e4m3_from_double(double x) {
+    if (x != x) return 0x7F;
+    uint8_t sign = signbit(x) ? 0x80 : 0;
+    double a = fabs(x);
+    if (a > 448.0) return (uint8_t)(sign | 0x7E);
+    if (a == 0.0) return sign;
+    int e;
+    (void)frexp(a, &e);
+    int exp_unb = e - 1;                       /* floor(log2 a) */
+    if (exp_unb < -6) exp_unb = -6;            /* subnormal range: quantum 2^-9 */
+    double r = nearbyint(ldexp(a, 3 - exp_unb));   /* in [8, 16] for normals, [0, 8] for subnormals */
+    double y = ldexp(r, exp_unb - 3);          /* exact */
+    if (y == 0.0) return sign;
+    if (y < ldexp(1.0, -6)) return (uint8_t)(sign | (uint8_t)r);          /* subnormal: mantissa = r */
+    (void)frexp(y, &e);
+    exp_unb = e - 1;                           /* rounding may have carried into the next binade */
+    int m = (int)(ldexp(y, 3 - exp_unb) - 8.0);
+    return (uint8_t)(sign | ((exp_unb + 7) << 3) | m);
+}
+
 static void store_elem(void *pool, int dtype, int64_t idx, double x) {
-    if (dtype == ORACLE_BF16)
+    if (dtype == ORACLE_E4M3)
+        ((uint8_t *)pool)[idx] = oracle_e4m3_from_double(x);
+    else if (dtype == ORACLE_BF16)
         ((uint16_t *)pool)[idx] = oracle_bf16_from_double(x);
     else
         ((float *)pool)[idx] = (float)x;  /* IEEE nearest-even conversion */

@@ -20,7 +20,7 @@ _SRC = os.path.join(_HERE, "gva_oracle.c")
 _LIB = os.path.join(_HERE, "libgva_oracle.so")
 _lib = None
 
-F32, BF16 = 0, 1
+F32, BF16, E4M3 = 0, 1, 2
 
 
 def build(force: bool = False) -> str:
@@ -37,6 +37,10 @@ def lib() -> ctypes.CDLL:
         _lib = ctypes.CDLL(build())
         _lib.oracle_bf16_from_double.restype = ctypes.c_uint16
         _lib.oracle_bf16_from_double.argtypes = [ctypes.c_double]
+        _lib.oracle_e4m3_from_double.restype = ctypes.c_uint8
+        _lib.oracle_e4m3_from_double.argtypes = [ctypes.c_double]
+        _lib.oracle_e4m3_to_double.restype = ctypes.c_double
+        _lib.oracle_e4m3_to_double.argtypes = [ctypes.c_uint8]
         _lib.oracle_num_threads.restype = ctypes.c_int
         _lib.oracle_append.restype = ctypes.c_int
         _lib.oracle_append_chunk.restype = ctypes.c_int
@@ -52,7 +56,9 @@ def _dt(pool: np.ndarray) -> int:
         return BF16
     if pool.dtype == np.float32:
         return F32
-    raise TypeError("cache pools must be uint16 (bf16 bits) or float32")
+    if pool.dtype == np.uint8:
+        return E4M3
+    raise TypeError("cache pools must be uint16 (bf16 bits), uint8 (e4m3 codes) or float32")
 
 
 def _f64(a) -> np.ndarray:
@@ -73,6 +79,14 @@ def set_threads(n: int) -> None:
 
 def bf16_from_double(x: float) -> int:
     return int(lib().oracle_bf16_from_double(ctypes.c_double(float(x))))
+
+
+def e4m3_from_double(x: float) -> int:
+    return int(lib().oracle_e4m3_from_double(float(x)))
+
+
+def e4m3_to_double(code: int) -> float:
+    return float(lib().oracle_e4m3_to_double(int(code)))
 
 
 def rope(x, pos: float, base: float = 10000.0) -> np.ndarray:

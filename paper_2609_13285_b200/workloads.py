@@ -45,10 +45,40 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
     return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
+def f32_to_e4m3_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 values to the 8-bit e4m3 format (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; nearest,
+    ties to even; magnitudes beyond the largest finite value 448 saturate to it); returns uint8 codes."""
+    x = np.ascontiguousarray(x, dtype=np.float32).astype(np.float64)
+    sign = np.where(np.signbit(x), 0x80, 0).astype(np.uint8)
+    a = np.minimum(np.abs(x), 448.0)
+    _, e = np.frexp(np.where(a > 0, a, 1.0))
+    eu = np.maximum(e - 1, -6)                                  # below 2^-6 the quantum is fixed at 2^-9
+    y = np.ldexp(np.rint(np.ldexp(a, 3 - eu)), eu - 3)         # rint: ties to even
+    _, e2 = np.frexp(np.where(y > 0, y, 1.0))
+    eu2 = e2 - 1
+    normal = y >= 2.0 ** -6
+    mant = np.where(normal, np.ldexp(y, 3 - eu2) - 8.0, np.ldexp(y, 9)).astype(np.int64)
+    expo = np.where(normal, eu2 + 7, 0).astype(np.int64)
+    code = ((expo << 3) | mant).astype(np.uint8)
+    code = np.where(np.isnan(x), np.uint8(0x7F), code | sign)
+    return code.astype(np.uint8)
+
+
+def e4m3_bits_to_f64(b: np.ndarray) -> np.ndarray:
+    """Widen e4m3 codes (uint8) exactly to float64."""
+    b = np.ascontiguousarray(b, dtype=np.uint8).astype(np.int64)
+    e, m = (b >> 3) & 15, b & 7
+    v = np.where(e == 0, np.ldexp(m.astype(np.float64), -9), np.ldexp(1.0 + m / 8.0, e - 7))
+    v = np.where((b & 0x7F) == 0x7F, np.nan, v)
+    return np.where(b & 0x80, -v, v)
+
+
 def pool_to_f64(pool: np.ndarray) -> np.ndarray:
-    """Cache pool (uint16 bf16 bits or float32) widened exactly to float64."""
+    """Cache pool (uint16 bf16 bits, uint8 e4m3 codes or float32) widened exactly to float64."""
     if pool.dtype == np.uint16:
         return bf16_bits_to_f32(pool).astype(np.float64)
+    if pool.dtype == np.uint8:
+        return e4m3_bits_to_f64(pool)
     return pool.astype(np.float64)
 
 
@@ -84,7 +114,7 @@ class DecodeCase:
     shape: HeadShape
     B: int
     page_size: int
-    cache_dtype: str                      # "bf16" | "f32"
+    cache_dtype: str                      # "bf16" | "f32" | "fp8" (e4m3 codes)
     num_pages: int
     max_pages_per_seq: int
     v_pool: np.ndarray                    # [num_pages, G, page_size, d_v]  uint16 (bf16 bits) | float32
@@ -103,7 +133,7 @@ class DecodeCase:
 
     @property
     def elem_size(self) -> int:
-        return 2 if self.cache_dtype == "bf16" else 4
+        return {"bf16": 2, "fp8": 1}.get(self.cache_dtype, 4)
 
     def cache_bytes(self) -> int:
         """Live cache bytes a decode step must stream: sum_b seq_len * (G*d_v + d_r) * elem."""
@@ -129,10 +159,14 @@ def _normal_pool(rng: np.random.Generator, shape, cache_dtype: str, chunk_elems:
     n = int(np.prod(shape))
     if cache_dtype == "f32":
         return rng.standard_normal(n, dtype=np.float32).reshape(shape)
-    out = np.empty(n, dtype=np.uint16)
+    fp8 = cache_dtype == "fp8"
+    out = np.empty(n, dtype=np.uint8 if fp8 else np.uint16)
+    if fp8:
+        chunk_elems = min(chunk_elems, 1 << 22)         # the e4m3 cast works in float64 temporaries
     for lo in range(0, n, chunk_elems):
         hi = min(n, lo + chunk_elems)
-        out[lo:hi] = f32_to_bf16_bits(rng.standard_normal(hi - lo, dtype=np.float32))
+        draw = rng.standard_normal(hi - lo, dtype=np.float32)
+        out[lo:hi] = f32_to_e4m3_bits(draw) if fp8 else f32_to_bf16_bits(draw)
     return out.reshape(shape)
 
 
@@ -209,6 +243,9 @@ def poison_unused_slots(case: DecodeCase) -> None:
     if case.cache_dtype == "bf16":
         case.v_pool[np.broadcast_to(dead[:, None, :], case.v_pool.shape[:3])] = BF16_NAN_BITS
         case.kr_pool[dead] = BF16_NAN_BITS
+    elif case.cache_dtype == "fp8":
+        case.v_pool[np.broadcast_to(dead[:, None, :], case.v_pool.shape[:3])] = np.uint8(0x7F)     # the e4m3 NaN code
+        case.kr_pool[dead] = np.uint8(0x7F)
     else:
         case.v_pool[np.broadcast_to(dead[:, None, :], case.v_pool.shape[:3])] = np.nan
         case.kr_pool[dead] = np.nan

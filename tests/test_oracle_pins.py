@@ -676,3 +676,56 @@ def test_value_only_cache_is_attention_with_keys_v_m():
     c.append_pos[:] = np.maximum(c.seq_lens - 1, 0)
     assert orc.append_case(c) == 0
     assert (c.v_pool != v0).any() and c.kr_pool.size == 0
+
+
+# ---------------------------------------------------------------- 8-bit (e4m3) cache codes
+def test_e4m3_codec_against_library_cast_and_by_hand():
+    codes = np.arange(256, dtype=np.uint8)
+    lib_vals = torch.from_numpy(codes).view(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+    mine = np.array([orc.e4m3_to_double(int(c)) for c in codes])
+    gen = wl.e4m3_bits_to_f64(codes)
+    finite = ~np.isnan(lib_vals)
+    assert finite.sum() == 254 and np.isnan(mine[~finite]).all() and np.isnan(gen[~finite]).all()
+    assert np.array_equal(mine[finite], lib_vals[finite]) and np.array_equal(gen[finite], lib_vals[finite])
+    # every finite code survives a round trip through both encoders (0x80 is -0)
+    for c in codes[finite]:
+        assert orc.e4m3_from_double(mine[c]) == c
+    assert np.array_equal(wl.f32_to_e4m3_bits(lib_vals[finite].astype(np.float32)), codes[finite])
+    # random float32 values inside the finite range: both encoders agree with the library's cast
+    rng = np.random.default_rng(61)
+    x = np.concatenate([rng.standard_normal(20000), rng.uniform(-448, 448, 5000), rng.standard_normal(5000) * 1e-2]).astype(np.float32)
+    lib_codes = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(wl.f32_to_e4m3_bits(x), lib_codes)
+    assert np.array_equal(np.array([orc.e4m3_from_double(float(v)) for v in x[:4000]], dtype=np.uint8), lib_codes[:4000])
+    # by hand: ties go to the even mantissa, the subnormal quantum is 2^-9, magnitudes beyond 448 saturate
+    assert orc.e4m3_from_double(1.0625) == 0x38 and orc.e4m3_from_double(1.1875) == 0x3A        # 1.0 and 1.25
+    assert orc.e4m3_from_double(2.0 ** -10) == 0x00 and orc.e4m3_from_double(3 * 2.0 ** -10) == 0x02
+    assert orc.e4m3_from_double(2.0 ** -6 - 2.0 ** -10) == 0x08                                   # rounds up into the normals
+    assert orc.e4m3_from_double(1e6) == 0x7E and orc.e4m3_from_double(-449.0) == 0xFE and orc.e4m3_from_double(float("nan")) == 0x7F
+
+
+def test_fp8_cache_decode_and_append_through_the_oracle():
+    # the oracle reads e4m3 codes exactly and appends with one rounding; the decode over such a cache is the same plain
+    # attention over the widened values
+    c = small_case(cache_dtype="fp8")
+    assert c.v_pool.dtype == np.uint8 and c.cache_bytes() == int(c.seq_lens.sum()) * c.shape.row_elems
+    out, lse = orc.decode_case(c)
+    V = wl.pool_to_f64(c.v_pool); KR = wl.pool_to_f64(c.kr_pool)
+    q_abs = orc.absorb_case(c)
+    s = c.shape
+    for b in range(c.B):
+        L = int(c.seq_lens[b])
+        for h in range(s.H):
+            g = h // (s.H // s.G)
+            rows = [(c.page_of(b, t // c.page_size), t % c.page_size) for t in range(L)]
+            sc = np.array([q_abs[b, h, :s.d_v] @ V[p, g, sl] + q_abs[b, h, s.d_v:] @ KR[p, sl] for p, sl in rows]) / math.sqrt(s.d_c + s.d_r)
+            w = np.exp(sc - sc.max()); w /= w.sum()
+            assert np.allclose(out[b, h], sum(w[t] * V[rows[t][0], g, rows[t][1]] for t in range(L)), atol=1e-13)
+    v0, k0 = c.v_pool.copy(), c.kr_pool.copy()
+    assert orc.append_case(c) == 0
+    for b in range(c.B):
+        t = int(c.append_pos[b]); p, sl = c.page_of(b, t // c.page_size), t % c.page_size
+        assert np.array_equal(c.v_pool[p, :, sl], wl.f32_to_e4m3_bits(c.v_new[b]))
+        rot = orc.rope(c.kr_new[b], t)
+        assert np.array_equal(c.kr_pool[p, sl], np.array([orc.e4m3_from_double(float(v)) for v in rot], dtype=np.uint8))
+    assert (c.v_pool != v0).sum() <= c.B * s.G * s.d_v and (c.kr_pool != k0).sum() <= c.B * s.d_r
