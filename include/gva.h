@@ -52,11 +52,19 @@ typedef enum {
     GVA_ERR_STATIC_LIMIT = 8  /* gva_decode_static: the request needs more than GVA_STATIC_SCRATCH_BYTES  */
 } gva_status;
 
-typedef enum { GVA_F32 = 0, GVA_BF16 = 1 } gva_dtype;
+/* Element type of the cache pools.  GVA_E4M3 stores every cache element as one byte (sign, 4 exponent bits with bias 7,
+ * 3 mantissa bits; no infinities, 0x7F / 0xFF = NaN, largest finite 448): appends round to nearest even and saturate
+ * at +-448, decode widens the codes exactly and computes as for the other types.  The paper stores 16-bit caches; the
+ * 8-bit cache is this library's extension of its byte accounting (Section 3.4) and halves the bytes per token again.
+ * It is built for d_v = 64, d_r = 16, pages of a multiple of 64 tokens, with the tensor-core kernel only:
+ * gva_absorb_query, gva_append_cache, gva_append_chunk, gva_decode, gva_decode_step, gva_decode_step_host and
+ * gva_decode_static serve it; gqa_decode, gva_prefill, gva_decode_multi, gva_decode_tokens and the projections return
+ * GVA_ERR_UNSUPPORTED. */
+typedef enum { GVA_F32 = 0, GVA_BF16 = 1, GVA_E4M3 = 2 } gva_dtype;
 
-/* Which decode kernel gva_decode launches.  AUTO = tensor-core kernel when the cache is bf16,
- * CUDA-core (FMA) kernel for an f32 cache.  FMA / MMA force one (MMA with an f32 cache is
- * GVA_ERR_UNSUPPORTED). */
+/* Which decode kernel gva_decode launches.  AUTO = tensor-core kernel when the cache is bf16 or e4m3,
+ * CUDA-core (FMA) kernel for an f32 cache.  FMA / MMA force one (MMA with an f32 cache and
+ * FMA with an e4m3 cache are GVA_ERR_UNSUPPORTED). */
 typedef enum { GVA_KERNEL_AUTO = 0, GVA_KERNEL_FMA = 1, GVA_KERNEL_MMA = 2 } gva_kernel;
 
 typedef struct {

@@ -18,7 +18,7 @@ GVA_OK = 0
 GVA_ERR_INVALID_ARG, GVA_ERR_UNSUPPORTED, GVA_ERR_WORKSPACE, GVA_ERR_CUDA = 1, 2, 3, 4
 GVA_ERR_BAD_PAGE, GVA_ERR_SEQ_LEN, GVA_ERR_TIMEOUT, GVA_ERR_STATIC_LIMIT = 5, 6, 7, 8
 GVA_STATIC_SCRATCH_BYTES = 16 << 20
-GVA_F32, GVA_BF16 = 0, 1
+GVA_F32, GVA_BF16, GVA_E4M3 = 0, 1, 2
 GVA_KERNEL_AUTO, GVA_KERNEL_FMA, GVA_KERNEL_MMA = 0, 1, 2
 
 EXPORTS = ["gva_create", "gva_destroy", "gva_decode_workspace_bytes", "gva_absorb_query", "gva_append_cache",

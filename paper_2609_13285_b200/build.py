@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgva.so")
 SOURCES = ["gva_api.cu"]
-HEADERS = ["gva_common.cuh", "gva_small_kernels.cuh", "gva_decode_fma.cuh", "gva_decode_mma.cuh", "gva_prefill.cuh", "gva_project.cuh",
+HEADERS = ["gva_common.cuh", "gva_small_kernels.cuh", "gva_decode_fma.cuh", "gva_decode_mma.cuh", "gva_decode_fp8.cuh", "gva_prefill.cuh", "gva_project.cuh",
            os.path.join("..", "..", "include", "gva.h")]
 
 

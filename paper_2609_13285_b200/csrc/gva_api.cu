@@ -13,6 +13,7 @@
 #include "gva_project.cuh"
 #ifdef GVA_WITH_MMA
 #include "gva_decode_mma.cuh"
+#include "gva_decode_fp8.cuh"
 #include "gva_prefill.cuh"
 #endif
 
@@ -189,10 +190,15 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
         kernel = GVA_KERNEL_FMA;
 #endif
     }
+    if (h->cfg.cache_dtype == GVA_E4M3) kernel = GVA_KERNEL_MMA;
     if (q_len > 1 && (GQA || kernel != GVA_KERNEL_MMA)) return GVA_ERR_UNSUPPORTED;   // multi-token decode: tensor-core kernel only
+    if ((q_len > 1 || GQA) && h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;
     if (kernel == GVA_KERNEL_MMA) {
 #ifdef GVA_WITH_MMA
-        int rc = q_len > 1 ? launch_decode_mma_multi(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, q_len, max_seq_len, num_splits,
+        int rc = h->cfg.cache_dtype == GVA_E4M3
+                     ? launch_decode_fp8(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, max_seq_len, num_splits, stream,
+                                         &h->last_num_splits, &h->last_tile, &p.rec_mult)
+                 : q_len > 1 ? launch_decode_mma_multi(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, q_len, max_seq_len, num_splits,
                                                      max_blocks_balanced(h), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult)
                            : launch_decode_mma<GQA>(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, max_seq_len, num_splits,
                                         max_blocks_balanced(h), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult);
@@ -265,14 +271,21 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
     if (cfg->H <= 0 || cfg->G <= 0 || cfg->d_v <= 0 || cfg->d_c <= 0 || cfg->d_r < 0 || cfg->page_size <= 0 ||
         !(cfg->rope_base > 1.0) || !(cfg->softmax_scale >= 0.f) || device < 0)
         return GVA_ERR_INVALID_ARG;
-    if (cfg->cache_dtype != GVA_F32 && cfg->cache_dtype != GVA_BF16) return GVA_ERR_INVALID_ARG;
+    if (cfg->cache_dtype != GVA_F32 && cfg->cache_dtype != GVA_BF16 && cfg->cache_dtype != GVA_E4M3) return GVA_ERR_INVALID_ARG;
     if (cfg->kernel < GVA_KERNEL_AUTO || cfg->kernel > GVA_KERNEL_MMA) return GVA_ERR_INVALID_ARG;
     if (cfg->H % cfg->G != 0 || cfg->H / cfg->G != kHeadsPerGroup) return GVA_ERR_UNSUPPORTED;
     // d_r = 0 is the value-only cache (no positional slice: Section 3.4, "exactly half")
     if (!((cfg->d_v == 64 && (cfg->d_r == 16 || cfg->d_r == 24 || cfg->d_r == 0)) || (cfg->d_v == 128 && (cfg->d_r == 32 || cfg->d_r == 0))))
         return GVA_ERR_UNSUPPORTED;
     if (cfg->G > 8 || cfg->d_c > 256 || cfg->page_size % 32 != 0) return GVA_ERR_UNSUPPORTED;
-    if (cfg->kernel == GVA_KERNEL_MMA && cfg->cache_dtype != GVA_BF16) return GVA_ERR_UNSUPPORTED;
+    if (cfg->kernel == GVA_KERNEL_MMA && cfg->cache_dtype == GVA_F32) return GVA_ERR_UNSUPPORTED;
+    if (cfg->cache_dtype == GVA_E4M3) {   // the 8-bit cache: one shape, tensor-core kernel only
+#ifdef GVA_WITH_MMA
+        if (cfg->kernel == GVA_KERNEL_FMA || !fp8_supported(*cfg)) return GVA_ERR_UNSUPPORTED;
+#else
+        return GVA_ERR_UNSUPPORTED;
+#endif
+    }
 #ifndef GVA_WITH_MMA
     if (cfg->kernel == GVA_KERNEL_MMA) return GVA_ERR_UNSUPPORTED;
 #endif
@@ -385,7 +398,11 @@ int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (c.G * c.d_v > kAppendMaxPerThread * 128) return GVA_ERR_UNSUPPORTED;
     cudaError_t ce;
-    if (c.cache_dtype == GVA_BF16)
+    if (c.cache_dtype == GVA_E4M3)
+        ce = launch_pdl(append_kernel<uint8_t>, dim3(B), dim3(128), 0, s, static_cast<uint8_t *>(cache->v_pool),
+                        static_cast<uint8_t *>(cache->kr_pool), cache->block_table, v_new, kr_new, pos, c.G, c.d_v,
+                        c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+    else if (c.cache_dtype == GVA_BF16)
         ce = launch_pdl(append_kernel<__nv_bfloat16>, dim3(B), dim3(128), 0, s, static_cast<__nv_bfloat16 *>(cache->v_pool),
                         static_cast<__nv_bfloat16 *>(cache->kr_pool), cache->block_table, v_new, kr_new, pos, c.G, c.d_v,
                         c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
@@ -411,7 +428,11 @@ int gva_append_chunk(gva_handle *h, const gva_cache *cache, const float *v_new, 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (c.G * c.d_v > kAppendMaxPerThread * 128) return GVA_ERR_UNSUPPORTED;
     cudaError_t ce;
-    if (c.cache_dtype == GVA_BF16)
+    if (c.cache_dtype == GVA_E4M3)
+        ce = launch_pdl(append_chunk_kernel<uint8_t>, dim3((n_q + kAppendChunkRows - 1) / kAppendChunkRows), dim3(128), 0, s, static_cast<uint8_t *>(cache->v_pool),
+                        static_cast<uint8_t *>(cache->kr_pool), cache->block_table, v_new, kr_new, cu_q, ctx_lens, B, c.G,
+                        c.d_v, c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+    else if (c.cache_dtype == GVA_BF16)
         ce = launch_pdl(append_chunk_kernel<__nv_bfloat16>, dim3((n_q + kAppendChunkRows - 1) / kAppendChunkRows), dim3(128), 0, s, static_cast<__nv_bfloat16 *>(cache->v_pool),
                         static_cast<__nv_bfloat16 *>(cache->kr_pool), cache->block_table, v_new, kr_new, cu_q, ctx_lens, B, c.G,
                         c.d_v, c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
@@ -598,7 +619,9 @@ int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const
     a.n_absorb = c.H * ((B + kAbsorbBatch - 1) / kAbsorbBatch);
     const size_t smem = absorb_smem_bytes(c.d_v, c.d_c);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const cudaError_t ce = (c.cache_dtype == GVA_BF16)
+    const cudaError_t ce = (c.cache_dtype == GVA_E4M3)
+        ? launch_pdl(step_front_kernel<uint8_t>, dim3(a.n_absorb + B), dim3(kAbsorbThreads), smem, st, a, h->rope)
+        : (c.cache_dtype == GVA_BF16)
         ? launch_pdl(step_front_kernel<__nv_bfloat16>, dim3(a.n_absorb + B), dim3(kAbsorbThreads), smem, st, a, h->rope)
         : launch_pdl(step_front_kernel<float>, dim3(a.n_absorb + B), dim3(kAbsorbThreads), smem, st, a, h->rope);
     if (ce != cudaSuccess) {
@@ -868,6 +891,7 @@ int gva_pack_input_weights(const gva_handle *h, const float *W_q_nope, const flo
                            const float *W_r, const float *M, int d_model, uint16_t *W_in) {
     if (!h || !W_q_nope || !W_q_rope || !W_v || !W_r || !M || !W_in || d_model <= 0) return GVA_ERR_INVALID_ARG;
     if (h->cfg.d_r == 0) return GVA_ERR_UNSUPPORTED;     // the projections are built for the caches with a positional slice
+    if (h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;
     const gva_config &c = h->cfg;
     const int dq = c.d_v + c.d_r, nq = c.H * dq, nv = c.G * c.d_v, N = input_width(c);
     for (int m = 0; m < d_model; ++m) {
@@ -898,6 +922,7 @@ int gva_pack_bf16(const float *src, uint16_t *dst, size_t n) {
 int gva_project_in(gva_handle *h, const gva_cache *cache, const float *x, const void *W_in, int d_model,
                    const int32_t *pos, float *q_abs, int B, int32_t *dev_status, void *stream) {
     if (!h || !cache || B < 0 || d_model <= 0) return GVA_ERR_INVALID_ARG;
+    if (h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;   // the fused projection writes 16- or 32-bit caches
     if (h->cfg.d_r == 0) return GVA_ERR_UNSUPPORTED;
     if (B == 0) return GVA_OK;
     if (!x || !W_in || !pos || !q_abs || !cache->v_pool || (h->cfg.d_r > 0 && !cache->kr_pool)) return GVA_ERR_INVALID_ARG;

@@ -1,0 +1,478 @@
+// Split-KV decode over an 8-bit (e4m3) GVA cache: the tensor-core kernel of gva_decode_mma.cuh with the cache tile in
+// one byte per element.  Work partition, producer, barriers, partial records and merge are the same; what differs is
+// the consumer's way from shared memory to MMA fragments: ldmatrix moves 16-bit units, so a register holds two (plain)
+// or 2 x 2 (transposed) cache bytes, which are widened to f16 (exactly: every e4m3 value is an f16 value) with
+// cvt.rn.f16x2.e4m3x2 -- after a byte permute in the transposed case -- and multiplied with f16 hi/lo halves of the f32
+// query and weights (m16n8k16, f16 in, f32 accumulate).  The k index inside a 16-dim step is a fixed permutation of
+// the dims, applied to the query fragments as well, and the output rows of an m-tile are its even dims followed by its
+// odd dims.  d_v = 64, d_r = 16, 64-token tiles.
+#pragma once
+
+#include "gva_decode_mma.cuh"
+
+namespace gva {
+
+struct Fp8Traits {
+    static constexpr int DV = 64, DR = 16, TILE = 64;
+    static constexpr int VTILE_BYTES = TILE * DV;               // one group's tile: 64-byte rows
+    static constexpr int KR_ROW = DR;                           // 16 bytes
+    static constexpr int KR_BYTES = TILE * KR_ROW;
+    static constexpr int KSTEPS_V = DV / 16, KSTEPS = KSTEPS_V + DR / 16;
+    static constexpr int MT = DV / 16;
+    static constexpr int CHUNKS = TILE / 16;
+    static constexpr int DQ = DV + DR;
+    __host__ __device__ static constexpr int stage_bytes(int G) { return G * VTILE_BYTES + KR_BYTES; }
+    __host__ __device__ static constexpr int tail_bytes(int B, int nstage) {
+        return nstage * 16 /* barriers */ + nstage * 16 /* per-stage meta */ + 16 /* abort */ + (B + 1) * 4;
+    }
+};
+
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// two e4m3 codes (low 16 bits of x) -> two f16 (exact)
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
+    uint32_t d;
+    asm("{\n .reg .b16 t;\n cvt.u16.u32 t, %1;\n cvt.rn.f16x2.e4m3x2 %0, t;\n}\n" : "=r"(d) : "r"(x));
+    return d;
+}
+// x = hi + lo with hi, lo f16; hi in the low half-word, lo in the high half-word (|x| must stay below 65504)
+__device__ __forceinline__ uint32_t split_hi_lo_f16(float x) {
+    const __half hi = __float2half_rn(x);
+    const __half lo = __float2half_rn(x - __half2float(hi));
+    return (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
+}
+
+template <int NSTAGE>
+__global__ void __launch_bounds__(32 * 9)
+decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
+    using T = Fp8Traits;
+    constexpr int DV = T::DV, TILE = T::TILE, WPG = 1;
+    constexpr int CPW = T::CHUNKS / WPG;          // 16-token chunks per consumer warp and tile
+    static_assert(CPW >= 1 && CPW * WPG == T::CHUNKS, "tile must split evenly over the group's warps");
+    grid_dependency_launch();
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    // dynamic shared memory is only guaranteed 16-byte aligned: round up to the swizzle atom
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int G = p.G, H = p.H;
+    const int HQ = H;
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int n_consumers = G * WPG;
+    const int stage_bytes = T::stage_bytes(G);
+
+    unsigned char *tail = smem + (size_t)NSTAGE * stage_bytes;
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(tail);
+    uint64_t *empty_bar = full_bar + NSTAGE;
+    StageMeta *s_meta = reinterpret_cast<StageMeta *>(empty_bar + NSTAGE);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(s_meta + NSTAGE);
+    int *s_off = reinterpret_cast<int *>(s_meta + NSTAGE) + 4;
+
+    if (tid == 0) {
+        for (int s = 0; s < NSTAGE; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), 1);
+            mbar_init(smem_u32(&empty_bar[s]), n_consumers);
+        }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        // fetch the two tensor-map descriptors now, not at the first copy
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
+    }
+    // Early start (only behind step_front_kernel, which has already waited for everything before it): the
+    // tile bookkeeping and the producer's first loads run while the front kernel computes.  Nothing the front
+    // kernel writes is touched before grid_dependency_wait(): consumers wait before reading the absorbed
+    // query, the producer waits before loading the tile that holds the token being appended, and the
+    // workspace is written only after the wait.
+    const bool early = p.early_start != 0;
+    if (!early) grid_dependency_wait();
+    compute_tile_offsets<TILE>(p, s_off);   // ends with __syncthreads(): barriers are initialised for everyone
+    const bool uniform = p.num_splits > 0;
+    // Tail stealing pays where two blocks share an SM and their speeds differ by +-20 % (d_v = 64: measured -2.7 us
+    // of 100 on the long-context workload); with one block per SM (d_v = 128) speeds differ by +-4 % and the extra
+    // partial records cost more than the balance gains (measured +3.9 us of 180), so there the ranges stay static.
+#ifndef GVA_MMA_DYNAMIC_TAIL
+#define GVA_MMA_DYNAMIC_TAIL 1   // build-time knob: 0 = equal static ranges only
+#endif
+    const UnitPlan plan = make_unit_plan(s_off[p.B], gridDim.x, GVA_MMA_DYNAMIC_TAIL != 0 && DV == 64);
+    BlockRange rg;
+    rg.lo = rg.hi = 0;
+    rg.rec_fixed = -1;
+    rg.b_first = 0;
+    int first_unit = -1;
+    if (uniform) {
+        rg = block_range(p, s_off);
+        if (rg.hi <= rg.lo) {   // an empty split still owns its records (weight 0 in the merge)
+            if (early) grid_dependency_wait();
+            for (int i = tid; i < HQ * WPG; i += blockDim.x) {
+                p.rec_ml[((size_t)rg.rec_fixed * WPG * HQ + i) * 2] = -INFINITY;
+                p.rec_ml[((size_t)rg.rec_fixed * WPG * HQ + i) * 2 + 1] = 0.f;
+            }
+            return;
+        }
+    } else if ((int)blockIdx.x < plan.n_ranges) {
+        first_unit = blockIdx.x * (plan.U + 1);          // the head of this block's own range
+        unit_range(plan, blockIdx.x, 0, rg.lo, rg.hi);
+        rg.b_first = (rg.lo < rg.hi) ? seq_of_tile(s_off, p.B, rg.lo) : 0;
+    }
+    const int n_tickets = uniform ? 0 : plan.n_ranges * plan.U;    // tail units on offer
+    if (!uniform && first_unit < 0 && n_tickets == 0) {   // more blocks than ranges and no tails to share
+        if (blockIdx.x == 0) {                            // (total == 0): the header is still needed by the merge
+            if (early) grid_dependency_wait();
+            publish_header(p, s_off, plan);
+        }
+        return;
+    }
+
+    if (warp == n_consumers) {
+        // ================================ producer (one elected lane) ================================
+        if (lane == 0) {
+            bool waited = !early;
+            bool ok = true;
+            int issued = 0;       // tiles issued by this block: ring position
+            int lo = rg.lo, hi = rg.hi, unit = first_unit;
+            int b = rg.b_first;
+            for (;;) {
+                // the next tail unit is requested while this one is being issued (the ticket is reset
+                // by the previous call's combine kernel: never touch it before grid_dependency_wait())
+                int ticket = -1;
+                bool asked = n_tickets == 0;
+                for (int f = lo; f < hi && ok; ++f) {
+                    const int st = issued % NSTAGE;
+                    if (!waited && issued >= NSTAGE) {   // the ring is full: nothing more to gain from running ahead
+                        grid_dependency_wait();
+                        waited = true;
+                    }
+                    if (!asked && waited && hi - f <= 2) {   // late, so that tails go to whoever really is ahead
+                        ticket = atomicAdd(p.ticket, 1);
+                        asked = true;
+                    }
+                    while (f >= s_off[b + 1]) ++b;
+                    const int t0 = (f - s_off[b]) * TILE;
+                    const int pj = t0 / p.P, slot0 = t0 % p.P;
+                    // the three lookups are independent: request them together, use them afterwards
+                    const int len = p.seq_lens[b];
+                    const int ap = waited ? -1 : p.append_pos[b];
+                    long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
+                                                   : (long long)b * p.max_pages + pj;
+                    if (!waited && ap >= t0 && ap < t0 + TILE) {   // this tile receives the new token: it must be complete first
+                        grid_dependency_wait();
+                        waited = true;
+                    }
+                    int n_valid = min(TILE, len - t0);
+                    if (page < 0 || page >= p.num_pages) {
+                        report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
+                        page = 0;
+                        n_valid = 0;
+                    }
+                    // the bookkeeping above overlaps with the wait for the stage to be released
+                    if (!mbar_wait_bounded(smem_u32(&empty_bar[st]), ((issued / NSTAGE) & 1) ^ 1, s_abort)) {
+                        if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+                        *s_abort = 1;
+                        ok = false;
+                        break;
+                    }
+                    StageMeta m;
+                    m.n_valid = n_valid;
+                    m.b = b;
+                    m.rec = uniform ? rg.rec_fixed : unit + b;
+                    m.flags = ((f == lo || f == s_off[b]) ? 1 : 0) | ((f + 1 == hi || f + 1 >= s_off[b + 1]) ? 2 : 0);
+                    s_meta[st] = m;
+                    const uint32_t bar = smem_u32(&full_bar[st]);
+                    const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
+                    mbar_expect_tx(bar, G * T::VTILE_BYTES + T::KR_BYTES);
+                    tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
+                    for (int g = 0; g < G; ++g)
+                        tma_load_2d(base + g * T::VTILE_BYTES, &tm_v, 0, (int)((page * G + g) * p.P + slot0), bar);
+                    ++issued;
+                }
+                if (!ok) break;
+                if (!asked) {
+                    if (!waited) {
+                        grid_dependency_wait();
+                        waited = true;
+                    }
+                    ticket = atomicAdd(p.ticket, 1);
+                }
+                if (ticket < 0 || ticket >= n_tickets) break;
+                // ticket t -> tail j = 1 + t / n_ranges of range t % n_ranges: first every range's first tail, then the second, ...
+                const int c = ticket % plan.n_ranges, j = 1 + ticket / plan.n_ranges;
+                unit = c * (plan.U + 1) + j;
+                unit_range(plan, c, j, lo, hi);
+                if (lo < hi) b = seq_of_tile(s_off, p.B, lo);
+            }
+            if (ok) {
+                // tell the consumers that nothing more is coming
+                const int st = issued % NSTAGE;
+                if (mbar_wait_bounded(smem_u32(&empty_bar[st]), ((issued / NSTAGE) & 1) ^ 1, s_abort)) {
+                    s_meta[st].n_valid = -1;
+                    mbar_arrive(smem_u32(&full_bar[st]));
+                } else {
+                    if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+                    *s_abort = 1;
+                    ok = false;
+                }
+            }
+            if (!ok) {
+                // drain: every copy this block started must land before its shared memory is released
+                const int first = max(0, issued - NSTAGE);
+                for (int i = first; i < issued; ++i) {
+                    const int st = i % NSTAGE;
+                    for (int it = 0; it < kDrainPolls; ++it)
+                        if (mbar_try_wait(smem_u32(&full_bar[st]), (i / NSTAGE) & 1)) break;
+                }
+            }
+        }
+    } else {
+        // ============ consumer: value group g, token chunks [part*CPW, part*CPW + CPW) of every tile ============
+        const int g = warp / WPG;
+        const int part = warp % WPG;
+        const int jh = lane & 3;          // head within the group this lane's score/output columns belong to
+        const int r8 = lane >> 2;         // row within an 8-row block
+        // ldmatrix lane addressing inside a 16-token chunk of the value tile (64-byte rows, 64-byte swizzle: 16-byte chunk
+        // c of row t sits at chunk c ^ ((t >> 1) & 3)).  One ldmatrix.x4 fetches (tokens 0-7 | 8-15) x (chunk 2i | 2i + 1);
+        // a 16-byte chunk is 16 value dims, so lane L's register of matrix m holds four consecutive dims of token L / 4
+        // (plain) or the dim pair L / 4 of tokens 2 (L % 4), 2 (L % 4) + 1 (transposed).
+        const int r7 = lane & 7;
+        const int row_ld = r7 + ((lane >> 3) & 1) * 8, ch_ld = lane >> 4;
+        const uint32_t off_v = row_ld * 64;
+        const uint32_t swz_v = (row_ld >> 1) & 3;
+        uint32_t qf[T::KSTEPS][2];        // B fragments of Q^T as f16: column n = lane/4 = 2*head + {hi, lo}; k-step kk covers
+                                          // dims 16 kk .. 16 kk + 15 in the order the converted A registers present them
+        float oacc[T::MT][4];
+        float m_run = -INFINITY, l_run = 0.f;
+        const float scale = p.scale_log2;
+        const int lo_part = r8 & 1;
+
+        // absorbed query of head (lane/4)/2, hi or lo part by (lane/4)&1, as mma B fragments: b0 = dims 4 jh, 4 jh + 1 and
+        // b1 = dims 4 jh + 2, 4 jh + 3 of the k-step's 16 dims (the A registers carry the cache bytes in that order)
+        auto load_query = [&](int b) {
+            const float *q = p.q + ((size_t)b * H + g * kHeadsPerGroup + (r8 >> 1)) * T::DQ;
+#pragma unroll
+            for (int kk = 0; kk < T::KSTEPS; ++kk) {
+                const float4 v = *reinterpret_cast<const float4 *>(q + kk * 16 + 4 * jh);
+                const uint32_t sx = split_hi_lo_f16(v.x), sy = split_hi_lo_f16(v.y), sz = split_hi_lo_f16(v.z), sw = split_hi_lo_f16(v.w);
+                qf[kk][0] = lo_part ? ((sx >> 16) | (sy & 0xffff0000u)) : ((sx & 0xffffu) | (sy << 16));
+                qf[kk][1] = lo_part ? ((sz >> 16) | (sw & 0xffff0000u)) : ((sz & 0xffffu) | (sw << 16));
+            }
+        };
+        if (early) grid_dependency_wait();
+        publish_header(p, s_off, plan, tid, n_consumers * 32);
+        // the first sequence is known before any tile arrives: fetch its query while the first copies fly
+        int cur_b = -1;
+        if (rg.lo < rg.hi) {
+            cur_b = rg.b_first;
+            load_query(cur_b);
+        }
+
+#pragma unroll 1
+        for (int i = 0;; ++i) {
+            const int st = i % NSTAGE;
+            if (!mbar_wait_bounded(smem_u32(&full_bar[st]), (i / NSTAGE) & 1, s_abort)) {
+                if (!*s_abort && lane == 0) report_error(p.dev_status, GVA_ERR_TIMEOUT, cur_b < 0 ? 0 : cur_b);
+                *s_abort = 1;
+                break;
+            }
+            const StageMeta meta = s_meta[st];
+            const int n_valid = meta.n_valid;
+            if (n_valid < 0) break;       // producer is done
+            const int b = meta.b;
+            if (meta.flags & 1) {         // a new segment: its own softmax state (and query, if the sequence changed)
+                if (b != cur_b) {
+                    cur_b = b;
+                    load_query(b);
+                }
+                m_run = -INFINITY;
+                l_run = 0.f;
+#pragma unroll
+                for (int mt = 0; mt < T::MT; ++mt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) oacc[mt][e] = 0.f;
+            }
+            unsigned char *stage = smem + (size_t)st * stage_bytes;
+            unsigned char *vt = stage + (size_t)g * T::VTILE_BYTES;
+            const int row0 = part * CPW * 16;                 // first token row of this warp's share of the tile
+            const bool ragged = n_valid < row0 + CPW * 16;
+            if (ragged) {
+                // rows past the sequence end may hold anything (the NaN code included): zero this warp's share of them
+                // so that a zero weight times such a row stays zero
+                const int z0 = max(n_valid, row0);
+                const int n_zero_chunks = (row0 + CPW * 16 - z0) * 4;
+                for (int c = lane; c < n_zero_chunks; c += 32)
+                    *reinterpret_cast<uint4 *>(vt + (z0 + c / 4) * 64 + (c % 4) * 16) = make_uint4(0, 0, 0, 0);
+                // generic-proxy writes must be ordered before the TMA write that later refills the stage
+                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                __syncwarp();
+            }
+            const uint32_t vt_u32 = smem_u32(vt) + row0 * 64;
+            const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES) + row0 * T::KR_ROW;
+
+            // ---- S^T = V_tile . Q^T (+ positional part), 16 tokens per m-tile ----
+            float sacc[CPW][4];
+#pragma unroll
+            for (int c = 0; c < CPW; ++c) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) sacc[c][e] = 0.f;
+#pragma unroll
+                for (int pr = 0; pr < DV / 32; ++pr) {        // two 16-dim chunks per fetch
+                    uint32_t r[4];                             // (tok r8, chunk 2 pr) (tok r8 + 8, chunk 2 pr) (tok r8, chunk 2 pr + 1) (tok r8 + 8, ..)
+                    ldsm_x4(vt_u32 + c * 1024 + off_v + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_v) << 4), r);
+#pragma unroll
+                    for (int hx = 0; hx < 2; ++hx) {
+                        uint32_t a[4];
+                        a[0] = e4m3x2_to_f16x2(r[2 * hx] & 0xffffu);
+                        a[1] = e4m3x2_to_f16x2(r[2 * hx + 1] & 0xffffu);
+                        a[2] = e4m3x2_to_f16x2(r[2 * hx] >> 16);
+                        a[3] = e4m3x2_to_f16x2(r[2 * hx + 1] >> 16);
+                        mma_f16(sacc[c], a, qf[2 * pr + hx][0], qf[2 * pr + hx][1]);
+                    }
+                }
+                {   // the positional key: 16-byte rows, one fetch of (tokens 0-7 | 8-15)
+                    uint32_t r[2];
+                    ldsm_x2(kr_u32 + c * 16 * T::KR_ROW + (lane & 15) * T::KR_ROW, r);
+                    uint32_t a[4];
+                    a[0] = e4m3x2_to_f16x2(r[0] & 0xffffu);
+                    a[1] = e4m3x2_to_f16x2(r[1] & 0xffffu);
+                    a[2] = e4m3x2_to_f16x2(r[0] >> 16);
+                    a[3] = e4m3x2_to_f16x2(r[1] >> 16);
+                    mma_f16(sacc[c], a, qf[T::KSTEPS_V][0], qf[T::KSTEPS_V][1]);
+                }
+            }
+            // ---- online softmax for head jh over this warp's tokens (rows r8, r8+8 of every m-tile) ----
+            float sr[CPW][2];              // raw scores (hi + lo columns summed)
+            float tmax = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < CPW; ++c) {
+                sr[c][0] = sacc[c][0] + sacc[c][1];
+                sr[c][1] = sacc[c][2] + sacc[c][3];
+                if (ragged) {
+                    const int t_lo = row0 + c * 16 + r8;
+                    if (t_lo >= n_valid) sr[c][0] = -INFINITY;
+                    if (t_lo + 8 >= n_valid) sr[c][1] = -INFINITY;
+                }
+                tmax = fmaxf(tmax, fmaxf(sr[c][0], sr[c][1]));
+            }
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 4));
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 8));
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
+            const float m_new = fmaxf(m_run, tmax * scale);          // scale > 0: max commutes with it
+            const bool live = m_new != -INFINITY;
+            const float m_use = live ? m_new : 0.f;                  // keeps (-inf) - (-inf) out of the exponent
+            const float corr = fast_exp2(m_run - m_use);             // 2^(-inf) = 0 for the first live tile
+            m_run = m_new;
+            l_run *= corr;
+#pragma unroll
+            for (int mt = 0; mt < T::MT; ++mt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) oacc[mt][e] *= corr;
+
+            // ---- O^T += V_tile^T . P^T: MMA row r of m-tile mt is value dim 16 mt + 2 r (r < 8) or 16 mt + 2 (r - 8) + 1 ----
+#pragma unroll
+            for (int c = 0; c < CPW; ++c) {
+                const float p0 = fast_exp2(fmaf(sr[c][0], scale, -m_use));
+                const float p1 = fast_exp2(fmaf(sr[c][1], scale, -m_use));
+                l_run += p0 + p1;
+                // (hi, lo) of p for token row r8 / r8+8 and columns 2*jh, 2*jh+1 -> transpose to B fragments
+                const uint32_t pb0 = movmatrix_trans(split_hi_lo_f16(p0));
+                const uint32_t pb1 = movmatrix_trans(split_hi_lo_f16(p1));
+#pragma unroll
+                for (int pr = 0; pr < DV / 32; ++pr) {
+                    uint32_t r[4];    // transposed: dim pair r8 of chunk (2 pr | 2 pr + 1) at tokens (2 jh, 2 jh + 1) and (2 jh + 8, 2 jh + 9)
+                    ldsm_x4_trans(vt_u32 + c * 1024 + off_v + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_v) << 4), r);
+#pragma unroll
+                    for (int hx = 0; hx < 2; ++hx) {
+                        uint32_t a[4];
+                        a[0] = e4m3x2_to_f16x2(__byte_perm(r[2 * hx], 0, 0x4420));        // even dim, tokens 2 jh, 2 jh + 1
+                        a[1] = e4m3x2_to_f16x2(__byte_perm(r[2 * hx], 0, 0x4431));        // odd dim
+                        a[2] = e4m3x2_to_f16x2(__byte_perm(r[2 * hx + 1], 0, 0x4420));    // even dim, tokens 2 jh + 8, 2 jh + 9
+                        a[3] = e4m3x2_to_f16x2(__byte_perm(r[2 * hx + 1], 0, 0x4431));
+                        mma_f16(oacc[2 * pr + hx], a, pb0, pb1);
+                    }
+                }
+            }
+            // release the stage to the producer
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&empty_bar[st]));
+
+            // ---- segment end: write this (unit, sequence, part) partial ----
+            if (meta.flags & 2) {
+                const int rec = meta.rec * WPG + part;
+                float l = l_run;
+                l += __shfl_xor_sync(0xffffffffu, l, 4);
+                l += __shfl_xor_sync(0xffffffffu, l, 8);
+                l += __shfl_xor_sync(0xffffffffu, l, 16);
+                const size_t rh = (size_t)rec * H + g * kHeadsPerGroup + jh;
+                float *o_dst = p.rec_o + rh * DV;
+#pragma unroll
+                for (int mt = 0; mt < T::MT; ++mt)
+                    *reinterpret_cast<float2 *>(o_dst + mt * 16 + 2 * r8) = make_float2(oacc[mt][0] + oacc[mt][1], oacc[mt][2] + oacc[mt][3]);
+                if (r8 == 0) {
+                    p.rec_ml[rh * 2] = m_run;
+                    p.rec_ml[rh * 2 + 1] = l;
+                }
+            }
+        }
+    }
+    // keep shared memory alive until every warp (and every copy in flight) is done
+    __syncthreads();
+}
+
+
+// ---- host ---------------------------------------------------------------------------------------------
+inline bool fp8_supported(const gva_config &cfg) {
+    return cfg.cache_dtype == GVA_E4M3 && cfg.d_v == 64 && cfg.d_r == 16 && cfg.page_size % 64 == 0;
+}
+
+inline bool encode_map_u8(const MmaHostState &st, CUtensorMap *map, const void *base, uint64_t inner, uint64_t rows,
+                          uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz) {
+    cuuint64_t dims[2] = {inner, rows};
+    cuuint64_t strides[1] = {inner};
+    cuuint32_t box[2] = {box_inner, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return st.encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline int launch_decode_fp8(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
+                             int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out, int *tile_out,
+                             int *rec_mult_out) {
+    using T = Fp8Traits;
+    constexpr int NSTAGE = 4;
+    if (!fp8_supported(cfg)) return GVA_ERR_UNSUPPORTED;
+    if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
+    const int G = cfg.G;
+    const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
+    if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
+    auto fn = decode_fp8_kernel<NSTAGE>;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
+    CUtensorMap tm_v, tm_k;
+    if (!encode_map_u8(st, &tm_v, p.v_pool, T::DV, (uint64_t)p.num_pages * G * p.P, T::DV, T::TILE, CU_TENSOR_MAP_SWIZZLE_64B))
+        return GVA_ERR_CUDA;
+    if (!encode_map_u8(st, &tm_k, p.kr_pool, T::DR, (uint64_t)p.num_pages * p.P, T::DR, T::TILE, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return GVA_ERR_CUDA;
+    const int threads = 32 * (G + 1);
+    int grid;
+    if (num_splits > 0) {
+        grid = B * num_splits;
+    } else {
+        const long long tiles_ub = (long long)B * ((max_seq_len + T::TILE - 1) / T::TILE);
+        const long long want = 2LL * sm_count;      // two blocks per SM, as the workspace is sized for (d_v = 64)
+        grid = (int)(tiles_ub < want ? (tiles_ub < 1 ? 1 : tiles_ub) : want);
+    }
+    DecodeParams pp = p;
+    pp.rec_mult = 1;
+    if (launch_pdl(fn, dim3(grid), dim3(threads), smem, stream, pp, tm_v, tm_k) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GVA_ERR_CUDA;
+    }
+    *n_blocks_out = grid;
+    *tile_out = T::TILE;
+    *rec_mult_out = 1;
+    return GVA_OK;
+}
+
+}  // namespace gva

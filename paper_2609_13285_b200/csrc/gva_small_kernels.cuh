@@ -29,6 +29,9 @@ __device__ __forceinline__ uint16_t double_to_bf16_bits(double x) {
 __device__ __forceinline__ uint16_t float_to_bf16_bits(float f) {
     return __bfloat16_as_ushort(__float2bfloat16_rn(f));
 }
+// 8-bit e4m3 codes: round to nearest even, finite overflow and infinity saturate to +-448, NaN stays NaN
+__device__ __forceinline__ uint8_t float_to_e4m3_bits(float f) { return (uint8_t)__nv_cvt_float_to_fp8(f, __NV_SATFINITE, __NV_E4M3); }
+__device__ __forceinline__ uint8_t double_to_e4m3_bits(double x) { return (uint8_t)__nv_cvt_double_to_fp8(x, __NV_SATFINITE, __NV_E4M3); }
 
 // One pair of y = x R_pos^T in fp64.
 __device__ __forceinline__ void rope_pair(double x0, double x1, int pos, double inv_freq, double &y0, double &y1) {
@@ -292,7 +295,8 @@ __device__ __forceinline__ void append_row(CT *__restrict__ v_pool, CT *__restri
         if (i < n_v) {
             const int g = i / d_v, d = i % d_v;
             const size_t dst = (((size_t)page * G + g) * P + slot) * d_v + d;
-            if constexpr (sizeof(CT) == 2) reinterpret_cast<uint16_t *>(v_pool)[dst] = float_to_bf16_bits(x[u]);
+            if constexpr (sizeof(CT) == 1) reinterpret_cast<uint8_t *>(v_pool)[dst] = float_to_e4m3_bits(x[u]);
+            else if constexpr (sizeof(CT) == 2) reinterpret_cast<uint16_t *>(v_pool)[dst] = float_to_bf16_bits(x[u]);
             else reinterpret_cast<float *>(v_pool)[dst] = x[u];
         }
     }
@@ -301,7 +305,10 @@ __device__ __forceinline__ void append_row(CT *__restrict__ v_pool, CT *__restri
         double y0, y1;
         rope_pair((double)k0, (double)k1, t, rope.inv_freq[i], y0, y1);
         const size_t dst = ((size_t)page * P + slot) * d_r + 2 * i;
-        if constexpr (sizeof(CT) == 2) {
+        if constexpr (sizeof(CT) == 1) {
+            reinterpret_cast<uint8_t *>(kr_pool)[dst] = double_to_e4m3_bits(y0);
+            reinterpret_cast<uint8_t *>(kr_pool)[dst + 1] = double_to_e4m3_bits(y1);
+        } else if constexpr (sizeof(CT) == 2) {
             reinterpret_cast<uint16_t *>(kr_pool)[dst] = double_to_bf16_bits(y0);
             reinterpret_cast<uint16_t *>(kr_pool)[dst + 1] = double_to_bf16_bits(y1);
         } else {

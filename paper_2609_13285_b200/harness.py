@@ -1,6 +1,6 @@
 """Moves a generated decode case into device memory and wraps the three library calls.
 
-No arithmetic happens here: tensors are uploaded as generated (bf16 pools as raw 16-bit patterns)
+No arithmetic happens here: tensors are uploaded as generated (bf16 pools as raw 16-bit patterns, e4m3 pools as bytes)
 and handed to the C ABI through `binding`.
 """
 from __future__ import annotations
@@ -101,7 +101,7 @@ def upload(case: DecodeCase, device="cuda:0", kernel: int = gb.GVA_KERNEL_AUTO) 
     dev = torch.device(device)
     s = case.shape
     handle = gb.gva_create(H=s.H, G=s.G, d_v=s.d_v, d_c=s.d_c, d_r=s.d_r, page_size=case.page_size,
-                           cache_dtype=gb.GVA_BF16 if case.cache_dtype == "bf16" else gb.GVA_F32, kernel=kernel,
+                           cache_dtype={"bf16": gb.GVA_BF16, "fp8": gb.GVA_E4M3}.get(case.cache_dtype, gb.GVA_F32), kernel=kernel,
                            rope_base=case.rope_base, device=dev.index or 0)
     B = case.B
     return DeviceCase(

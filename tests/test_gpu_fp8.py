@@ -1,0 +1,241 @@
+"""GPU parity over the 8-bit (e4m3) cache: the CUDA library against the fp64 oracle, which reads the same stored codes
+exactly (every e4m3 value is an f16 value), so the tight f32-arithmetic gates apply unchanged."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gva_oracle as orc
+from paper_2609_13285_b200 import binding as gb
+from paper_2609_13285_b200 import harness
+from paper_2609_13285_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+EDGE_LENS = [0, 1, 31, 32, 33, 63, 64, 65, 127, 128, 129, 640, 641, 1000]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from tests import gpu_util
+    gpu_util.ensure_built()
+
+
+def U():
+    from tests import gpu_util
+    return gpu_util
+
+
+@pytest.mark.parametrize("num_splits", [0, 1, 5, 40])
+def test_ragged_edge_lengths_poisoned(num_splits):
+    # lengths around tile and page boundaries, an empty sequence, more splits than tiles; every slot no live token
+    # occupies holds the NaN code and unused block-table entries are -1
+    case = wl.make_case("edge8", wl.SHAPE_A, EDGE_LENS, page_size=64, cache_dtype="fp8", seed=801, poison_unused=True,
+                        extra_pages=2)
+    U().check_decode(case, gb.GVA_KERNEL_AUTO, num_splits=num_splits)
+
+
+@pytest.mark.parametrize("num_splits", [0, 2, 7])
+def test_long_batch_all_split_counts(num_splits):
+    case = wl.make_case("long8", wl.SHAPE_A, [4096] * 8, page_size=64, cache_dtype="fp8", paged=False, seed=802)
+    dc = harness.upload(case)
+    try:
+        U().check_decode(case, gb.GVA_KERNEL_AUTO, num_splits=num_splits, dc=dc)
+        assert gb.gva_last_kernel(dc.handle) == gb.GVA_KERNEL_MMA
+    finally:
+        dc.close()
+
+
+def test_every_value_dim_and_token_slot_lands_where_it_should():
+    # one-hot probes: a cache whose only non-zero element is (token t, group g, dim d) and a flat score row give
+    # out[h, d'] = value / T at d' = d for the heads of group g and zero elsewhere -- catches any permutation of dims,
+    # tokens or heads on the way through the byte fragments
+    T = 128
+    case = wl.make_case("onehot8", wl.SHAPE_A, [T] * 6, page_size=64, cache_dtype="fp8", seed=803, q_gain=0.0)
+    one = int(wl.f32_to_e4m3_bits(np.array([1.0], dtype=np.float32))[0])
+    case.v_pool[:] = 0
+    case.kr_pool[:] = 0
+    probes = [(0, 0, 0), (1, 1, 17), (77, 2, 34), (127, 3, 63), (64, 0, 49), (15, 3, 6)]
+    for b, (t, g, d) in enumerate(probes):
+        page = int(case.block_table[b, t // 64])
+        case.v_pool[page, g, t % 64, d] = one
+    dc = harness.upload(case)
+    try:
+        dc.absorb()
+        out, _ = dc.decode()
+        torch.cuda.synchronize()
+        o = out.cpu().numpy()
+        s = case.shape
+        for b, (t, g, d) in enumerate(probes):
+            want = np.zeros((s.H, s.d_v), dtype=np.float32)
+            want[g * 4:(g + 1) * 4, d] = 1.0 / T
+            assert np.allclose(o[b], want, atol=1e-7), (b, t, g, d)
+    finally:
+        dc.close()
+
+
+def test_score_side_sees_every_dim_in_place():
+    # scores pick the token: a query far along one dim and a cache whose token t carries a large value at that dim only
+    # must put (nearly) all weight on t -- one probe per 16-dim chunk and byte lane, the positional slice included
+    T = 64
+    s = wl.SHAPE_A
+    dims = [0, 1, 2, 3, 5, 18, 35, 52, 63, 64, 67, 70, 79]        # >= 64: the positional slice
+    case = wl.make_case("score8", s, [T] * len(dims), page_size=64, cache_dtype="fp8", seed=804, q_gain=0.0)
+    big = int(wl.f32_to_e4m3_bits(np.array([16.0], dtype=np.float32))[0])
+    one = int(wl.f32_to_e4m3_bits(np.array([1.0], dtype=np.float32))[0])
+    case.v_pool[:] = 0
+    case.kr_pool[:] = 0
+    for b, d in enumerate(dims):
+        t = (7 * b + 3) % T
+        page = int(case.block_table[b, 0])
+        if d < s.d_v:
+            case.v_pool[page, :, t, d] = big
+        else:
+            case.kr_pool[page, t, d - s.d_v] = big
+        case.v_pool[page, :, t, (d + 9) % s.d_v] = one      # marks the token in the output (beside the score dim)
+    dc = harness.upload(case)
+    try:
+        q = np.zeros((len(dims), s.H, s.d_v + s.d_r), dtype=np.float32)
+        for b, d in enumerate(dims):
+            q[b, :, d] = 40.0
+        dc.q_abs.copy_(torch.from_numpy(q))
+        out, _ = dc.decode()
+        torch.cuda.synchronize()
+        o = out.cpu().numpy().astype(np.float64)
+        ref, _ = orc.decode_case(case, q.astype(np.float64))
+        assert np.max(np.abs(o - ref)) <= 2e-5
+        for b, d in enumerate(dims):
+            assert abs(o[b, 0, (d + 9) % s.d_v] - 1.0) < 1e-3
+    finally:
+        dc.close()
+
+
+def test_peaked_and_flat_scores():
+    case = wl.make_case("peak8", wl.SHAPE_A, [500, 2049, 64], page_size=64, cache_dtype="fp8", seed=805, q_gain=30.0)
+    U().check_decode(case, gb.GVA_KERNEL_AUTO, tight=False)
+    case = wl.make_case("flat8", wl.SHAPE_A, [500, 2049, 64], page_size=64, cache_dtype="fp8", seed=806, q_gain=0.0)
+    U().check_decode(case, gb.GVA_KERNEL_AUTO)
+
+
+def test_page_sizes_and_contiguous():
+    for P, paged in ((128, True), (256, False), (64, False)):
+        case = wl.make_case("ps8", wl.SHAPE_A, [777, 3], page_size=P, cache_dtype="fp8", paged=paged, seed=807 + P,
+                            poison_unused=True)
+        U().check_decode(case, gb.GVA_KERNEL_AUTO)
+
+
+def test_append_is_bit_exact_and_saturates():
+    lens = [1, 64, 65, 300, 129, 4000, 8193]
+    case = wl.make_case("append8", wl.SHAPE_A, lens, page_size=64, cache_dtype="fp8", seed=808, extra_pages=3)
+    # values beyond the largest finite code, ties between codes, subnormals and zeros of both signs
+    case.v_new[0, 0, :8] = [1e6, -1e6, 448.0, 464.0, 1.0625, 1.1875, 2.0 ** -10, -0.0]
+    case.v_new[1, 1, :4] = [3 * 2.0 ** -10, 2.0 ** -6 - 2.0 ** -10, -449.0, 0.0]
+    dc = harness.upload(case)
+    try:
+        dc.append()
+        torch.cuda.synchronize()
+        assert int(dc.status.item()) == 0
+        v_gpu, k_gpu = dc.pools_to_host()
+        assert orc.append_case(case) == 0                  # oracle applies the same append to the host copy
+        assert np.array_equal(v_gpu, case.v_pool)
+        assert np.array_equal(k_gpu, case.kr_pool)
+    finally:
+        dc.close()
+
+
+def test_append_chunk_is_bit_exact():
+    pc = wl.make_prefill_case("ap8", wl.SHAPE_A, [0, 63, 64, 500], [130, 2, 0, 77], page_size=64, cache_dtype="fp8", seed=812)
+    c = pc.cache
+    v_ref, k_ref = c.v_pool.copy(), c.kr_pool.copy()
+    assert orc.append_chunk(v_ref, k_ref, c.block_table, pc.v_new, pc.kr_new, pc.cu_q, pc.ctx_lens) == 0
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.append()
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        v, k = pd.dc.pools_to_host()
+    finally:
+        pd.close()
+    assert np.array_equal(v, v_ref) and np.array_equal(k, k_ref)
+
+
+def test_fused_step_is_bitwise_the_three_calls_and_matches_the_oracle():
+    lens = np.array([1, 64, 65, 1001, 4096, 130], dtype=np.int32)
+    mk = lambda: wl.make_case("fstep8", wl.SHAPE_A, lens, page_size=64, cache_dtype="fp8", seed=809,
+                              q_pos=lens - 1, append_pos=lens - 1)
+    case = mk()
+    a, b = harness.upload(mk()), harness.upload(mk())
+    try:
+        a.absorb(); a.append(); a.decode()
+        b.step()
+        torch.cuda.synchronize()
+        assert int(a.status.item()) == 0 and int(b.status.item()) == 0
+        assert torch.equal(a.q_abs, b.q_abs)
+        assert torch.equal(a.v_pool, b.v_pool) and torch.equal(a.kr_pool, b.kr_pool)
+        assert torch.equal(a.out, b.out) and torch.equal(a.lse, b.lse)
+        assert orc.append_case(case) == 0                      # oracle: append, then attend, with its own fp64 query
+        ref_out, _ = orc.decode_case(case)
+        assert np.max(np.abs(b.out.cpu().numpy().astype(np.float64) - ref_out)) <= 5e-5
+    finally:
+        a.close(); b.close()
+
+
+def test_static_entry_point_and_host_step():
+    case = wl.make_case("host8", wl.SHAPE_A, [200, 64, 1300], page_size=64, cache_dtype="fp8", seed=810,
+                        q_pos=np.array([199, 63, 1299]), append_pos=np.array([199, 63, 1299]))
+    dc = harness.upload(case)
+    try:
+        dc.step()
+        torch.cuda.synchronize()
+        want = dc.out.clone()
+        dc.out.fill_(float("nan"))
+        gb.gva_decode_static(dc.handle, dc.cache, dc.q_abs, dc.seq_lens, dc.out, dc.lse, case.B, dc.max_seq_len, 0, dc.status)
+        torch.cuda.synchronize()
+        assert int(dc.status.item()) == 0
+        assert torch.equal(dc.out, want)
+    finally:
+        dc.close()
+
+
+def test_what_the_8_bit_cache_does_not_cover():
+    for kw in (dict(H=32, G=8, d_v=128, d_c=128, d_r=32, page_size=64), dict(H=16, G=4, d_v=64, d_c=64, d_r=24, page_size=64),
+               dict(H=16, G=4, d_v=64, d_c=64, d_r=16, page_size=32),
+               dict(H=16, G=4, d_v=64, d_c=64, d_r=16, page_size=64, kernel=gb.GVA_KERNEL_FMA)):
+        with pytest.raises(gb.GvaError) as e:
+            gb.gva_create(cache_dtype=gb.GVA_E4M3, **kw)
+        assert e.value.status == gb.GVA_ERR_UNSUPPORTED
+    pc = wl.make_prefill_case("pf8", wl.SHAPE_A, [64, 0], [4, 4], page_size=64, cache_dtype="fp8", seed=811)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        for call in (pd.prefill, lambda: pd.decode_multi(num_splits=0), lambda: pd.decode_tokens(4)):
+            with pytest.raises(gb.GvaError) as e:
+                call()
+            assert e.value.status == gb.GVA_ERR_UNSUPPORTED
+    finally:
+        pd.close()
+
+
+def test_full_size_long_context_sampled():
+    # bench.py's 8-bit workload (the long-context paged configuration with one byte per cache element), same launch:
+    # the oracle evaluates a sample of sequences; the Gaussian-tilting statistic covers the rest
+    case = wl.make_case("cfg2-fp8", wl.SHAPE_A, [32768] * 32, page_size=64, cache_dtype="fp8", paged=True,
+                        seed=wl.MASTER_SEED + 2000)
+    dc = harness.upload(case)
+    try:
+        dc.absorb()
+        out, lse = dc.decode(num_splits=0)
+        torch.cuda.synchronize()
+        assert int(dc.status.item()) == 0
+        o = out.cpu().numpy().astype(np.float64)
+        assert np.isfinite(o).all()
+        sample = [0, 17, 31]
+        lens = np.zeros_like(case.seq_lens)
+        lens[sample] = case.seq_lens[sample]
+        ref, _ = U().oracle_for_gpu_q(case, dc.q_abs, seq_lens=lens)
+        assert np.max(np.abs(o[sample] - ref[sample])) <= U().TOL_TIGHT_MAXABS
+        s = case.shape
+        q = dc.q_abs.cpu().numpy().astype(np.float64)
+        target = q[..., :s.d_v] / np.sqrt(s.d_c + s.d_r)
+        assert np.max(np.abs(o - target)) < 0.25      # e4m3 rounding of N(0, 1) rows adds ~0.1 % variance only
+    finally:
+        dc.close()
