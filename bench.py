@@ -64,6 +64,12 @@ def make_workload(name: str, rank: int):
     if name == "cfg2-dr0":   # cfg2 without the positional slice: the value-only cache, exactly half of matched GQA
         return wl.make_case("cfg2-dr0", wl.SHAPE_A0, [32768] * 32, page_size=64, cache_dtype="bf16", paged=True,
                             seed=wl.MASTER_SEED + 2050 + shift)
+    if name == "cfg2-fp8":   # cfg2 over the 8-bit (e4m3) cache: half the bytes per token again
+        return wl.make_case("cfg2-fp8", wl.SHAPE_A, [32768] * 32, page_size=64, cache_dtype="fp8", paged=True,
+                            seed=wl.MASTER_SEED + 2000 + shift)
+    if name == "cfg2-fp8-ncu":   # profiler-sized: 143 MB of 8-bit cache (> L2)
+        return wl.make_case("cfg2-fp8-ncu", wl.SHAPE_A, [32768] * 16, page_size=64, cache_dtype="fp8", paged=True,
+                            seed=wl.MASTER_SEED + 2000 + shift)
     if name == "cfg2-ncu":   # profiler-sized: 143 MB of cache (> L2), same shapes and paging as cfg2
         return wl.config2(seed=wl.MASTER_SEED + 2000 + shift, B=16, T=16384)
     if name == "cfg2-small":
@@ -79,6 +85,7 @@ WORKLOAD_TEXT = {
     "cfg4": "24-layer decode step (B=128, T=8192 cached + 1 appended per layer, paged, one pool per layer)",
     "cfg2-dr24": "cfg2 with RoPE width d_r = 24 (B=32, T=32768, paged; N_GVA/N_GQA = 0.546875)",
     "cfg2-dr0": "cfg2 without the positional slice, d_r = 0 (value-only cache; B=32, T=32768, paged; N_GVA/N_GQA = 0.5)",
+    "cfg2-fp8": "cfg2 over an 8-bit e4m3 cache (B=32, T=32768, paged; 272 bytes per token: half of the bf16 GVA cache)",
 }
 
 
@@ -661,7 +668,7 @@ def main() -> None:
         peak = load_peaks()[0]
         short = argparse.Namespace(**vars(args))
         short.steps, short.warmup = max(20, args.steps // 3), 10
-        for other in ("cfg0", "cfg1", "cfg3", "cfg4", "cfg2-dr24", "cfg2-dr0"):
+        for other in ("cfg0", "cfg1", "cfg3", "cfg4", "cfg2-dr24", "cfg2-dr0", "cfg2-fp8"):
             o = measure(other, rank, local_rank, dist, short, kernel, torch, gb, harness, with_e2e=False,
                         with_clocks=True)
             per_layer = o["cache_bytes"] / o["layers"]
@@ -698,7 +705,7 @@ def main() -> None:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": r["steps"], "warmup": r["warmup"],
             "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if case.cache_dtype == "bf16" else "f32", "data": "synthetic",
+            "dtype": {"bf16": "bf16", "fp8": "e4m3"}.get(case.cache_dtype, "f32"), "data": "synthetic",
             "config": dict(workload_description(name, case, r["layers"]), kernel=r["kernel"],
                            partitions=r["partitions"], replicas=world),
             "decode_steps_per_s": world * 1e3 / step_ms,

@@ -141,15 +141,20 @@ int max_blocks_balanced(const gva_handle *h) {
 // Upper bound on units (records per sequence come on top): the CUDA-core kernel uses one unit per block; the
 // tensor-core kernel runs at most 2 blocks per SM (d_v = 64) or 1 (d_v = 128), each range with up to 4 tail units.
 int max_units_balanced(const gva_handle *h) {
-    const int mma_blocks = (h->cfg.d_v == 64 ? 2 : 1) * h->sm_count;
+#ifdef GVA_WITH_MMA
+    const int per_sm = h->cfg.cache_dtype == GVA_E4M3 ? GVA_FP8_BLOCKS_PER_SM : (h->cfg.d_v == 64 ? 2 : 1);
+#else
+    const int per_sm = h->cfg.d_v == 64 ? 2 : 1;
+#endif
+    const int mma_blocks = per_sm * h->sm_count;
     const int a = max_blocks_balanced(h), b = unit_bound(mma_blocks);
     return a > b ? a : b;
 }
 
 WorkspaceLayout workspace_layout(const gva_handle *h, int B, int num_splits, int q_len = 1) {
     WorkspaceLayout w;
-    // up to two partial records per (block, sequence): the tensor-core kernel may run two warps per group
-    w.n_rec = 2 * (num_splits > 0 ? B * num_splits : max_units_balanced(h) + B);
+    // up to two partial records per (block, sequence): the 16-bit tensor-core kernel may run two warps per group
+    w.n_rec = (h->cfg.cache_dtype == GVA_E4M3 ? 1 : 2) * (num_splits > 0 ? B * num_splits : max_units_balanced(h) + B);
     w.hdr_bytes = align_up((size_t)(kHdrInts + 2 * B) * 4, 256);
     w.rec_o_bytes = align_up((size_t)w.n_rec * h->cfg.H * q_len * h->cfg.d_v * 4, 256);     // q_len * H pseudo-heads per record
     w.rec_ml_bytes = align_up((size_t)w.n_rec * h->cfg.H * q_len * 2 * 4, 256);

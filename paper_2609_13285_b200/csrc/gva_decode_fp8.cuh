@@ -1,14 +1,28 @@
 // Split-KV decode over an 8-bit (e4m3) GVA cache: the tensor-core kernel of gva_decode_mma.cuh with the cache tile in
 // one byte per element.  Work partition, producer, barriers, partial records and merge are the same; what differs is
-// the consumer's way from shared memory to MMA fragments: ldmatrix moves 16-bit units, so a register holds two (plain)
-// or 2 x 2 (transposed) cache bytes, which are widened to f16 (exactly: every e4m3 value is an f16 value) with
-// cvt.rn.f16x2.e4m3x2 -- after a byte permute in the transposed case -- and multiplied with f16 hi/lo halves of the f32
-// query and weights (m16n8k16, f16 in, f32 accumulate).  The k index inside a 16-dim step is a fixed permutation of
-// the dims, applied to the query fragments as well, and the output rows of an m-tile are its even dims followed by its
-// odd dims.  d_v = 64, d_r = 16, 64-token tiles.
+// the consumer's way from shared memory to MMA fragments.  The byte MMA (m16n8k32, e4m3 operands) is not a native
+// warp-level instruction on this architecture (the compiler widens its operands and splits it: measured slower), so
+// the cache bytes are widened to f16 -- exactly: every e4m3 value is an f16 value -- with cvt.rn.f16x2.e4m3x2, two
+// codes per instruction, and multiplied with f16 hi/lo halves of the f32 query and weights (m16n8k16, f16 in, f32
+// accumulate).  For the score product ldmatrix delivers four consecutive dims of one token per register; for the
+// value product the byte-transposing 16x16 ldmatrix delivers four tokens of one dim per register, so both sides
+// need nothing but the two conversions per register.  The k index inside an MMA is then a fixed permutation of the
+// dims (score product) or tokens (value product); the other operand's fragments are built in the same order.
+// d_v = 64, d_r = 16, 64-token tiles.
 #pragma once
 
 #include "gva_decode_mma.cuh"
+
+// build-time knobs: ring depth, warps per value group (G <= 4), resident blocks per SM the grid is sized for
+#ifndef GVA_FP8_NSTAGE
+#define GVA_FP8_NSTAGE 3
+#endif
+#ifndef GVA_FP8_WPG
+#define GVA_FP8_WPG 1
+#endif
+#ifndef GVA_FP8_BLOCKS_PER_SM
+#define GVA_FP8_BLOCKS_PER_SM 4
+#endif
 
 namespace gva {
 
@@ -33,11 +47,26 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], u
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-// two e4m3 codes (low 16 bits of x) -> two f16 (exact)
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
-    uint32_t d;
-    asm("{\n .reg .b16 t;\n cvt.u16.u32 t, %1;\n cvt.rn.f16x2.e4m3x2 %0, t;\n}\n" : "=r"(d) : "r"(x));
-    return d;
+// four e4m3 codes -> f16 pairs (exact) of the low and of the high half-word
+__device__ __forceinline__ void e4m3x4_to_f16x2(uint32_t x, uint32_t &lo, uint32_t &hi) {
+    asm("{\n .reg .b16 l, h;\n mov.b32 {l, h}, %2;\n cvt.rn.f16x2.e4m3x2 %0, l;\n cvt.rn.f16x2.e4m3x2 %1, h;\n}\n" : "=r"(lo), "=r"(hi) : "r"(x));
+}
+// Two 16x16 byte matrices, transposed on the way: lanes 0-15 give the row addresses (16 bytes each) of the first,
+// lanes 16-31 of the second.  Lane (g = lane / 4, t = lane % 4) receives bytes [column g | g + 8][rows 4 t .. 4 t + 3]
+// of the first matrix in r[0] | r[1] and of the second in r[2] | r[3].
+__device__ __forceinline__ void ldsm_b8_x2_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m16n16.x2.trans.shared.b8 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// (x0, x1) -> (hi, lo) f16 pairs of each, two values per conversion instruction
+__device__ __forceinline__ void split_pair_hi_lo_f16(float x0, float x1, uint32_t &s0, uint32_t &s1) {
+    const __half2 h = __floats2half2_rn(x0, x1);
+    const float2 f = __half22float2(h);
+    const __half2 l = __floats2half2_rn(x0 - f.x, x1 - f.y);
+    const uint32_t hu = *reinterpret_cast<const uint32_t *>(&h), lu = *reinterpret_cast<const uint32_t *>(&l);
+    s0 = __byte_perm(hu, lu, 0x5410);
+    s1 = __byte_perm(hu, lu, 0x7632);
 }
 // x = hi + lo with hi, lo f16; hi in the low half-word, lo in the high half-word (|x| must stay below 65504)
 __device__ __forceinline__ uint32_t split_hi_lo_f16(float x) {
@@ -46,11 +75,11 @@ __device__ __forceinline__ uint32_t split_hi_lo_f16(float x) {
     return (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
 }
 
-template <int NSTAGE>
+template <int NSTAGE, int WPG>
 __global__ void __launch_bounds__(32 * 9)
 decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = Fp8Traits;
-    constexpr int DV = T::DV, TILE = T::TILE, WPG = 1;
+    constexpr int DV = T::DV, TILE = T::TILE;
     constexpr int CPW = T::CHUNKS / WPG;          // 16-token chunks per consumer warp and tile
     static_assert(CPW >= 1 && CPW * WPG == T::CHUNKS, "tile must split evenly over the group's warps");
     grid_dependency_launch();
@@ -232,14 +261,23 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         const int part = warp % WPG;
         const int jh = lane & 3;          // head within the group this lane's score/output columns belong to
         const int r8 = lane >> 2;         // row within an 8-row block
-        // ldmatrix lane addressing inside a 16-token chunk of the value tile (64-byte rows, 64-byte swizzle: 16-byte chunk
-        // c of row t sits at chunk c ^ ((t >> 1) & 3)).  One ldmatrix.x4 fetches (tokens 0-7 | 8-15) x (chunk 2i | 2i + 1);
-        // a 16-byte chunk is 16 value dims, so lane L's register of matrix m holds four consecutive dims of token L / 4
-        // (plain) or the dim pair L / 4 of tokens 2 (L % 4), 2 (L % 4) + 1 (transposed).
+        // Fragment addressing inside a 16-token chunk of the value tile (64-byte rows, 64-byte swizzle: 16-byte piece c
+        // of row t sits at piece c ^ ((t >> 1) & 3)).  The token order inside a chunk is free on both products as long as
+        // they agree; it is chosen so that every 8 rows fetched together differ in t mod 8 (no bank conflicts).  With
+        // pi(j) = j (j < 8), j ^ 2 (j >= 8):
+        //   value product: the transposing load's row j is token pi(j); a register holds tokens pi(4t .. 4t + 3) of one dim,
+        //                  its low half becomes k = 2t, 2t + 1 and its high half k = 2t + 8, 2t + 9 of the MMA
+        //   score product: MMA row g is token pi(4 (g / 2) + g % 2), row g + 8 is token pi(4 (g / 2) + 2 + g % 2), so that the
+        //                  weights of rows (2t, 2t + 1), which the register transpose brings together, are k = 2t, 2t + 1
+        //                  (from the low rows) and k = 2t + 8, 2t + 9 (from the high rows)
         const int r7 = lane & 7;
-        const int row_ld = r7 + ((lane >> 3) & 1) * 8, ch_ld = lane >> 4;
-        const uint32_t off_v = row_ld * 64;
-        const uint32_t swz_v = (row_ld >> 1) & 3;
+        auto pi = [](int j) { return j < 8 ? j : (j ^ 2); };
+        const int row_qk = pi(4 * (r7 >> 1) + 2 * ((lane >> 3) & 1) + (r7 & 1));    // x4: (low | high rows) x (piece 2i | 2i + 1)
+        const int ch_ld = lane >> 4;
+        const uint32_t off_qk = row_qk * 64, swz_qk = (row_qk >> 1) & 3;
+        const int row_pv = pi(lane & 15);                                            // x2: (piece 2i | 2i + 1), 16 tokens each
+        const uint32_t off_pv = row_pv * 64, swz_pv = (row_pv >> 1) & 3;
+        const int tok_lo = pi(4 * (r8 >> 1) + (r8 & 1)), tok_hi = pi(4 * (r8 >> 1) + 2 + (r8 & 1));   // this lane's two score rows
         uint32_t qf[T::KSTEPS][2];        // B fragments of Q^T as f16: column n = lane/4 = 2*head + {hi, lo}; k-step kk covers
                                           // dims 16 kk .. 16 kk + 15 in the order the converted A registers present them
         float oacc[T::MT][4];
@@ -319,25 +357,21 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 #pragma unroll
                 for (int pr = 0; pr < DV / 32; ++pr) {        // two 16-dim chunks per fetch
                     uint32_t r[4];                             // (tok r8, chunk 2 pr) (tok r8 + 8, chunk 2 pr) (tok r8, chunk 2 pr + 1) (tok r8 + 8, ..)
-                    ldsm_x4(vt_u32 + c * 1024 + off_v + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_v) << 4), r);
+                    ldsm_x4(vt_u32 + c * 1024 + off_qk + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_qk) << 4), r);
 #pragma unroll
                     for (int hx = 0; hx < 2; ++hx) {
                         uint32_t a[4];
-                        a[0] = e4m3x2_to_f16x2(r[2 * hx] & 0xffffu);
-                        a[1] = e4m3x2_to_f16x2(r[2 * hx + 1] & 0xffffu);
-                        a[2] = e4m3x2_to_f16x2(r[2 * hx] >> 16);
-                        a[3] = e4m3x2_to_f16x2(r[2 * hx + 1] >> 16);
+                        e4m3x4_to_f16x2(r[2 * hx], a[0], a[2]);
+                        e4m3x4_to_f16x2(r[2 * hx + 1], a[1], a[3]);
                         mma_f16(sacc[c], a, qf[2 * pr + hx][0], qf[2 * pr + hx][1]);
                     }
                 }
                 {   // the positional key: 16-byte rows, one fetch of (tokens 0-7 | 8-15)
                     uint32_t r[2];
-                    ldsm_x2(kr_u32 + c * 16 * T::KR_ROW + (lane & 15) * T::KR_ROW, r);
+                    ldsm_x2(kr_u32 + (c * 16 + row_qk) * T::KR_ROW, r);      // lanes 0-7: low rows, 8-15: high rows
                     uint32_t a[4];
-                    a[0] = e4m3x2_to_f16x2(r[0] & 0xffffu);
-                    a[1] = e4m3x2_to_f16x2(r[1] & 0xffffu);
-                    a[2] = e4m3x2_to_f16x2(r[0] >> 16);
-                    a[3] = e4m3x2_to_f16x2(r[1] >> 16);
+                    e4m3x4_to_f16x2(r[0], a[0], a[2]);
+                    e4m3x4_to_f16x2(r[1], a[1], a[3]);
                     mma_f16(sacc[c], a, qf[T::KSTEPS_V][0], qf[T::KSTEPS_V][1]);
                 }
             }
@@ -349,9 +383,8 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 sr[c][0] = sacc[c][0] + sacc[c][1];
                 sr[c][1] = sacc[c][2] + sacc[c][3];
                 if (ragged) {
-                    const int t_lo = row0 + c * 16 + r8;
-                    if (t_lo >= n_valid) sr[c][0] = -INFINITY;
-                    if (t_lo + 8 >= n_valid) sr[c][1] = -INFINITY;
+                    if (row0 + c * 16 + tok_lo >= n_valid) sr[c][0] = -INFINITY;
+                    if (row0 + c * 16 + tok_hi >= n_valid) sr[c][1] = -INFINITY;
                 }
                 tmax = fmaxf(tmax, fmaxf(sr[c][0], sr[c][1]));
             }
@@ -369,26 +402,26 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 #pragma unroll
                 for (int e = 0; e < 4; ++e) oacc[mt][e] *= corr;
 
-            // ---- O^T += V_tile^T . P^T: MMA row r of m-tile mt is value dim 16 mt + 2 r (r < 8) or 16 mt + 2 (r - 8) + 1 ----
+            // ---- O^T += V_tile^T . P^T: m-tile mt holds value dims 16 mt .. 16 mt + 15 ----
 #pragma unroll
             for (int c = 0; c < CPW; ++c) {
                 const float p0 = fast_exp2(fmaf(sr[c][0], scale, -m_use));
                 const float p1 = fast_exp2(fmaf(sr[c][1], scale, -m_use));
                 l_run += p0 + p1;
-                // (hi, lo) of p for token row r8 / r8+8 and columns 2*jh, 2*jh+1 -> transpose to B fragments
-                const uint32_t pb0 = movmatrix_trans(split_hi_lo_f16(p0));
-                const uint32_t pb1 = movmatrix_trans(split_hi_lo_f16(p1));
+                // (hi, lo) of p for this lane's two token rows and columns 2*jh, 2*jh+1 -> transpose to B fragments
+                uint32_t s0, s1;
+                split_pair_hi_lo_f16(p0, p1, s0, s1);
+                const uint32_t pb0 = movmatrix_trans(s0);
+                const uint32_t pb1 = movmatrix_trans(s1);
 #pragma unroll
                 for (int pr = 0; pr < DV / 32; ++pr) {
-                    uint32_t r[4];    // transposed: dim pair r8 of chunk (2 pr | 2 pr + 1) at tokens (2 jh, 2 jh + 1) and (2 jh + 8, 2 jh + 9)
-                    ldsm_x4_trans(vt_u32 + c * 1024 + off_v + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_v) << 4), r);
+                    uint32_t r[4];    // dims 32 pr + (r8 | r8 + 8) and 32 pr + 16 + (r8 | r8 + 8), tokens pi(4 jh .. 4 jh + 3) each
+                    ldsm_b8_x2_trans(vt_u32 + c * 1024 + off_pv + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_pv) << 4), r);
 #pragma unroll
                     for (int hx = 0; hx < 2; ++hx) {
                         uint32_t a[4];
-                        a[0] = e4m3x2_to_f16x2(__byte_perm(r[2 * hx], 0, 0x4420));        // even dim, tokens 2 jh, 2 jh + 1
-                        a[1] = e4m3x2_to_f16x2(__byte_perm(r[2 * hx], 0, 0x4431));        // odd dim
-                        a[2] = e4m3x2_to_f16x2(__byte_perm(r[2 * hx + 1], 0, 0x4420));    // even dim, tokens 2 jh + 8, 2 jh + 9
-                        a[3] = e4m3x2_to_f16x2(__byte_perm(r[2 * hx + 1], 0, 0x4431));
+                        e4m3x4_to_f16x2(r[2 * hx], a[0], a[2]);
+                        e4m3x4_to_f16x2(r[2 * hx + 1], a[1], a[3]);
                         mma_f16(oacc[2 * pr + hx], a, pb0, pb1);
                     }
                 }
@@ -408,7 +441,10 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 float *o_dst = p.rec_o + rh * DV;
 #pragma unroll
                 for (int mt = 0; mt < T::MT; ++mt)
-                    *reinterpret_cast<float2 *>(o_dst + mt * 16 + 2 * r8) = make_float2(oacc[mt][0] + oacc[mt][1], oacc[mt][2] + oacc[mt][3]);
+                {
+                    o_dst[mt * 16 + r8] = oacc[mt][0] + oacc[mt][1];
+                    o_dst[mt * 16 + r8 + 8] = oacc[mt][2] + oacc[mt][3];
+                }
                 if (r8 == 0) {
                     p.rec_ml[rh * 2] = m_run;
                     p.rec_ml[rh * 2 + 1] = l;
@@ -441,37 +477,39 @@ inline int launch_decode_fp8(const gva_config &cfg, const MmaHostState &st, int 
                              int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out, int *tile_out,
                              int *rec_mult_out) {
     using T = Fp8Traits;
-    constexpr int NSTAGE = 4;
+    constexpr int NSTAGE = GVA_FP8_NSTAGE;
     if (!fp8_supported(cfg)) return GVA_ERR_UNSUPPORTED;
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
     const int G = cfg.G;
     const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
-    auto fn = decode_fp8_kernel<NSTAGE>;
+    constexpr int wpg = GVA_FP8_WPG;      // warps per group (each takes 1 / wpg of a tile's tokens); one measured fastest
+    if (cfg.G * wpg + 1 > 9) return GVA_ERR_UNSUPPORTED;
+    auto fn = decode_fp8_kernel<NSTAGE, wpg>;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
     CUtensorMap tm_v, tm_k;
     if (!encode_map_u8(st, &tm_v, p.v_pool, T::DV, (uint64_t)p.num_pages * G * p.P, T::DV, T::TILE, CU_TENSOR_MAP_SWIZZLE_64B))
         return GVA_ERR_CUDA;
     if (!encode_map_u8(st, &tm_k, p.kr_pool, T::DR, (uint64_t)p.num_pages * p.P, T::DR, T::TILE, CU_TENSOR_MAP_SWIZZLE_NONE))
         return GVA_ERR_CUDA;
-    const int threads = 32 * (G + 1);
+    const int threads = 32 * (G * wpg + 1);
     int grid;
     if (num_splits > 0) {
         grid = B * num_splits;
     } else {
         const long long tiles_ub = (long long)B * ((max_seq_len + T::TILE - 1) / T::TILE);
-        const long long want = 2LL * sm_count;      // two blocks per SM, as the workspace is sized for (d_v = 64)
+        const long long want = (long long)GVA_FP8_BLOCKS_PER_SM * sm_count;      // two blocks per SM, as the workspace is sized for (d_v = 64)
         grid = (int)(tiles_ub < want ? (tiles_ub < 1 ? 1 : tiles_ub) : want);
     }
     DecodeParams pp = p;
-    pp.rec_mult = 1;
+    pp.rec_mult = wpg;
     if (launch_pdl(fn, dim3(grid), dim3(threads), smem, stream, pp, tm_v, tm_k) != cudaSuccess) {
         (void)cudaGetLastError();
         return GVA_ERR_CUDA;
     }
     *n_blocks_out = grid;
     *tile_out = T::TILE;
-    *rec_mult_out = 1;
+    *rec_mult_out = wpg;
     return GVA_OK;
 }
 
