@@ -34,7 +34,8 @@ UNIT = "GB/s"
 
 # DRAM traffic of one decode-kernel launch on cfg2 at full size, from ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum, mean of two launches; profiles/decode_mma_kernel_cfg2.md).
-NCU_TRAFFIC_BYTES = {"cfg2": 0.5 * ((571_105_024 + 4_873_216) + (571_087_360 + 387_584))}
+NCU_TRAFFIC_BYTES = {"cfg2": 0.5 * ((571_105_024 + 4_873_216) + (571_087_360 + 387_584)),
+                     "cfg2-fp8": 0.5 * ((285_778_688 + 3_652_864) + (285_774_592 + 776_192))}
 
 
 def load_peaks():
