@@ -68,6 +68,10 @@ def make_workload(name: str, rank: int):
     if name == "cfg2-fp8":   # cfg2 over the 8-bit (e4m3) cache: half the bytes per token again
         return wl.make_case("cfg2-fp8", wl.SHAPE_A, [32768] * 32, page_size=64, cache_dtype="fp8", paged=True,
                             seed=wl.MASTER_SEED + 2000 + shift)
+    if name == "cfg3-fp8":   # cfg3 (wide heads, ragged batch) over the 8-bit cache
+        seed = wl.MASTER_SEED + 3000 + shift
+        return wl.make_case("cfg3-fp8", wl.SHAPE_B, wl.config3_seq_lens(seed), page_size=64, cache_dtype="fp8", paged=True,
+                            seed=seed)
     if name == "cfg2-fp8-ncu":   # profiler-sized: 143 MB of 8-bit cache (> L2)
         return wl.make_case("cfg2-fp8-ncu", wl.SHAPE_A, [32768] * 16, page_size=64, cache_dtype="fp8", paged=True,
                             seed=wl.MASTER_SEED + 2000 + shift)
@@ -87,6 +91,7 @@ WORKLOAD_TEXT = {
     "cfg2-dr24": "cfg2 with RoPE width d_r = 24 (B=32, T=32768, paged; N_GVA/N_GQA = 0.546875)",
     "cfg2-dr0": "cfg2 without the positional slice, d_r = 0 (value-only cache; B=32, T=32768, paged; N_GVA/N_GQA = 0.5)",
     "cfg2-fp8": "cfg2 over an 8-bit e4m3 cache (B=32, T=32768, paged; 272 bytes per token: half of the bf16 GVA cache)",
+    "cfg3-fp8": "cfg3 over an 8-bit e4m3 cache (B=64, H=32, G=8, d_v=128, seq_lens ~ U[1024,16384], paged; 1056 bytes per token)",
 }
 
 
@@ -669,7 +674,7 @@ def main() -> None:
         peak = load_peaks()[0]
         short = argparse.Namespace(**vars(args))
         short.steps, short.warmup = max(20, args.steps // 3), 10
-        for other in ("cfg0", "cfg1", "cfg3", "cfg4", "cfg2-dr24", "cfg2-dr0", "cfg2-fp8"):
+        for other in ("cfg0", "cfg1", "cfg3", "cfg4", "cfg2-dr24", "cfg2-dr0", "cfg2-fp8", "cfg3-fp8"):
             o = measure(other, rank, local_rank, dist, short, kernel, torch, gb, harness, with_e2e=False,
                         with_clocks=True)
             per_layer = o["cache_bytes"] / o["layers"]

@@ -56,7 +56,8 @@ typedef enum {
  * 3 mantissa bits; no infinities, 0x7F / 0xFF = NaN, largest finite 448): appends round to nearest even and saturate
  * at +-448, decode widens the codes exactly and computes as for the other types.  The paper stores 16-bit caches; the
  * 8-bit cache is this library's extension of its byte accounting (Section 3.4) and halves the bytes per token again.
- * It is built for d_v = 64, d_r = 16, pages of a multiple of 64 tokens, with the tensor-core kernel only:
+ * It is built for (d_v, d_r) = (64, 16), (64, 0), (128, 32), (128, 0), G <= 8, pages of a multiple of 64 tokens, with the
+ * tensor-core kernel only:
  * gva_absorb_query, gva_append_cache, gva_append_chunk, gva_decode, gva_decode_step, gva_decode_step_host and
  * gva_decode_static serve it; gqa_decode, gva_prefill, gva_decode_multi, gva_decode_tokens and the projections return
  * GVA_ERR_UNSUPPORTED. */

@@ -142,7 +142,7 @@ int max_blocks_balanced(const gva_handle *h) {
 // tensor-core kernel runs at most 2 blocks per SM (d_v = 64) or 1 (d_v = 128), each range with up to 4 tail units.
 int max_units_balanced(const gva_handle *h) {
 #ifdef GVA_WITH_MMA
-    const int per_sm = h->cfg.cache_dtype == GVA_E4M3 ? GVA_FP8_BLOCKS_PER_SM : (h->cfg.d_v == 64 ? 2 : 1);
+    const int per_sm = h->cfg.cache_dtype == GVA_E4M3 ? fp8_blocks_per_sm(h->cfg) : (h->cfg.d_v == 64 ? 2 : 1);
 #else
     const int per_sm = h->cfg.d_v == 64 ? 2 : 1;
 #endif
@@ -336,6 +336,8 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
         cudaFuncSetAttribute(step_front_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)absorb_smem) != cudaSuccess ||
         cudaFuncSetAttribute(step_front_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)absorb_smem) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(step_front_kernel<uint8_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)absorb_smem) !=
             cudaSuccess) {
         delete h;
         return GVA_ERR_CUDA;

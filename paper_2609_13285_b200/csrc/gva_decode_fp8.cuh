@@ -8,7 +8,7 @@
 // value product the byte-transposing 16x16 ldmatrix delivers four tokens of one dim per register, so both sides
 // need nothing but the two conversions per register.  The k index inside an MMA is then a fixed permutation of the
 // dims (score product) or tokens (value product); the other operand's fragments are built in the same order.
-// d_v = 64, d_r = 16, 64-token tiles.
+// Shapes: (d_v, d_r) = (64, 16), (64, 0) with 64-token tiles; (128, 32), (128, 0) with 32-token tiles.
 #pragma once
 
 #include "gva_decode_mma.cuh"
@@ -26,16 +26,23 @@
 
 namespace gva {
 
+template <int DV_, int DR_, int TILE_>
 struct Fp8Traits {
-    static constexpr int DV = 64, DR = 16, TILE = 64;
-    static constexpr int VTILE_BYTES = TILE * DV;               // one group's tile: 64-byte rows
-    static constexpr int KR_ROW = DR;                           // 16 bytes
+    static constexpr int DV = DV_, DR = DR_, TILE = TILE_;
+    static_assert((DV == 64 || DV == 128) && (DR == 0 || DR == 16 || DR == 32) && TILE % 16 == 0, "shape not built");
+    static constexpr int VTILE_BYTES = TILE * DV;               // one group's tile: rows of d_v bytes, swizzled over the row width
+    static constexpr int KR_ROW = DR;                           // 16 bytes (unswizzled) or 32 bytes (32-byte swizzle)
     static constexpr int KR_BYTES = TILE * KR_ROW;
     static constexpr int KSTEPS_V = DV / 16, KSTEPS = KSTEPS_V + DR / 16;
     static constexpr int MT = DV / 16;
     static constexpr int CHUNKS = TILE / 16;
     static constexpr int DQ = DV + DR;
-    __host__ __device__ static constexpr int stage_bytes(int G) { return G * VTILE_BYTES + KR_BYTES; }
+    // the positional tile is padded to a multiple of 1 KB so that every stage starts on the swizzle period
+    __host__ __device__ static constexpr int stage_bytes(int G) { return G * VTILE_BYTES + (KR_BYTES + 1023) / 1024 * 1024; }
+    // 16-byte piece c of value row t sits at piece c ^ swz(t): the 64- and 128-byte TMA swizzles
+    __host__ __device__ static constexpr uint32_t swz(int t) { return DV == 64 ? ((t >> 1) & 3) : (t & 7); }
+    // ... and of positional row t (32-byte rows, 32-byte swizzle; 16-byte rows are one piece)
+    __host__ __device__ static constexpr uint32_t swz_kr(int t) { return DR == 32 ? ((t >> 2) & 1) : 0; }
     __host__ __device__ static constexpr int tail_bytes(int B, int nstage) {
         return nstage * 16 /* barriers */ + nstage * 16 /* per-stage meta */ + 16 /* abort */ + (B + 1) * 4;
     }
@@ -75,11 +82,10 @@ __device__ __forceinline__ uint32_t split_hi_lo_f16(float x) {
     return (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
 }
 
-template <int NSTAGE, int WPG>
-__global__ void __launch_bounds__(32 * 9)
+template <int DV, int DR, int TILE, int NSTAGE, int WPG>
+__global__ void __launch_bounds__(32 * 9, DV == 128 ? 2 : 3)      // register caps: 4 five-warp blocks (d_v = 64) or 2 nine-warp blocks (d_v = 128) per SM
 decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
-    using T = Fp8Traits;
-    constexpr int DV = T::DV, TILE = T::TILE;
+    using T = Fp8Traits<DV, DR, TILE>;
     constexpr int CPW = T::CHUNKS / WPG;          // 16-token chunks per consumer warp and tile
     static_assert(CPW >= 1 && CPW * WPG == T::CHUNKS, "tile must split evenly over the group's warps");
     grid_dependency_launch();
@@ -213,7 +219,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                     const uint32_t bar = smem_u32(&full_bar[st]);
                     const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
                     mbar_expect_tx(bar, G * T::VTILE_BYTES + T::KR_BYTES);
-                    tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
+                    if constexpr (DR > 0) tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
                     for (int g = 0; g < G; ++g)
                         tma_load_2d(base + g * T::VTILE_BYTES, &tm_v, 0, (int)((page * G + g) * p.P + slot0), bar);
                     ++issued;
@@ -274,9 +280,10 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         auto pi = [](int j) { return j < 8 ? j : (j ^ 2); };
         const int row_qk = pi(4 * (r7 >> 1) + 2 * ((lane >> 3) & 1) + (r7 & 1));    // x4: (low | high rows) x (piece 2i | 2i + 1)
         const int ch_ld = lane >> 4;
-        const uint32_t off_qk = row_qk * 64, swz_qk = (row_qk >> 1) & 3;
+        const uint32_t off_qk = row_qk * DV, swz_qk = T::swz(row_qk);
+        const uint32_t off_kr = row_qk * T::KR_ROW, swz_kr = T::swz_kr(row_qk);
         const int row_pv = pi(lane & 15);                                            // x2: (piece 2i | 2i + 1), 16 tokens each
-        const uint32_t off_pv = row_pv * 64, swz_pv = (row_pv >> 1) & 3;
+        const uint32_t off_pv = row_pv * DV, swz_pv = T::swz(row_pv);
         const int tok_lo = pi(4 * (r8 >> 1) + (r8 & 1)), tok_hi = pi(4 * (r8 >> 1) + 2 + (r8 & 1));   // this lane's two score rows
         uint32_t qf[T::KSTEPS][2];        // B fragments of Q^T as f16: column n = lane/4 = 2*head + {hi, lo}; k-step kk covers
                                           // dims 16 kk .. 16 kk + 15 in the order the converted A registers present them
@@ -338,14 +345,14 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 // rows past the sequence end may hold anything (the NaN code included): zero this warp's share of them
                 // so that a zero weight times such a row stays zero
                 const int z0 = max(n_valid, row0);
-                const int n_zero_chunks = (row0 + CPW * 16 - z0) * 4;
+                const int n_zero_chunks = (row0 + CPW * 16 - z0) * (DV / 16);
                 for (int c = lane; c < n_zero_chunks; c += 32)
-                    *reinterpret_cast<uint4 *>(vt + (z0 + c / 4) * 64 + (c % 4) * 16) = make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4 *>(vt + (z0 + c / (DV / 16)) * DV + (c % (DV / 16)) * 16) = make_uint4(0, 0, 0, 0);
                 // generic-proxy writes must be ordered before the TMA write that later refills the stage
                 asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                 __syncwarp();
             }
-            const uint32_t vt_u32 = smem_u32(vt) + row0 * 64;
+            const uint32_t vt_u32 = smem_u32(vt) + row0 * DV;
             const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES) + row0 * T::KR_ROW;
 
             // ---- S^T = V_tile . Q^T (+ positional part), 16 tokens per m-tile ----
@@ -357,7 +364,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 #pragma unroll
                 for (int pr = 0; pr < DV / 32; ++pr) {        // two 16-dim chunks per fetch
                     uint32_t r[4];                             // (tok r8, chunk 2 pr) (tok r8 + 8, chunk 2 pr) (tok r8, chunk 2 pr + 1) (tok r8 + 8, ..)
-                    ldsm_x4(vt_u32 + c * 1024 + off_qk + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_qk) << 4), r);
+                    ldsm_x4(vt_u32 + c * 16 * DV + off_qk + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_qk) << 4), r);
 #pragma unroll
                     for (int hx = 0; hx < 2; ++hx) {
                         uint32_t a[4];
@@ -366,13 +373,23 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                         mma_f16(sacc[c], a, qf[2 * pr + hx][0], qf[2 * pr + hx][1]);
                     }
                 }
-                {   // the positional key: 16-byte rows, one fetch of (tokens 0-7 | 8-15)
+                if constexpr (DR == 16) {   // the positional key: 16-byte rows, one fetch of (low | high rows)
                     uint32_t r[2];
-                    ldsm_x2(kr_u32 + (c * 16 + row_qk) * T::KR_ROW, r);      // lanes 0-7: low rows, 8-15: high rows
+                    ldsm_x2(kr_u32 + c * 16 * T::KR_ROW + off_kr, r);        // lanes 0-7: low rows, 8-15: high rows
                     uint32_t a[4];
                     e4m3x4_to_f16x2(r[0], a[0], a[2]);
                     e4m3x4_to_f16x2(r[1], a[1], a[3]);
                     mma_f16(sacc[c], a, qf[T::KSTEPS_V][0], qf[T::KSTEPS_V][1]);
+                } else if constexpr (DR == 32) {   // 32-byte rows: (low | high rows) x (piece 0 | 1)
+                    uint32_t r[4];
+                    ldsm_x4(kr_u32 + c * 16 * T::KR_ROW + off_kr + ((((uint32_t)ch_ld) ^ swz_kr) << 4), r);
+#pragma unroll
+                    for (int hx = 0; hx < 2; ++hx) {
+                        uint32_t a[4];
+                        e4m3x4_to_f16x2(r[2 * hx], a[0], a[2]);
+                        e4m3x4_to_f16x2(r[2 * hx + 1], a[1], a[3]);
+                        mma_f16(sacc[c], a, qf[T::KSTEPS_V + hx][0], qf[T::KSTEPS_V + hx][1]);
+                    }
                 }
             }
             // ---- online softmax for head jh over this warp's tokens (rows r8, r8+8 of every m-tile) ----
@@ -416,7 +433,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 #pragma unroll
                 for (int pr = 0; pr < DV / 32; ++pr) {
                     uint32_t r[4];    // dims 32 pr + (r8 | r8 + 8) and 32 pr + 16 + (r8 | r8 + 8), tokens pi(4 jh .. 4 jh + 3) each
-                    ldsm_b8_x2_trans(vt_u32 + c * 1024 + off_pv + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_pv) << 4), r);
+                    ldsm_b8_x2_trans(vt_u32 + c * 16 * DV + off_pv + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_pv) << 4), r);
 #pragma unroll
                     for (int hx = 0; hx < 2; ++hx) {
                         uint32_t a[4];
@@ -459,8 +476,12 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 
 // ---- host ---------------------------------------------------------------------------------------------
 inline bool fp8_supported(const gva_config &cfg) {
-    return cfg.cache_dtype == GVA_E4M3 && cfg.d_v == 64 && cfg.d_r == 16 && cfg.page_size % 64 == 0;
+    const bool shape = (cfg.d_v == 64 && (cfg.d_r == 16 || cfg.d_r == 0)) || (cfg.d_v == 128 && (cfg.d_r == 32 || cfg.d_r == 0));
+    return cfg.cache_dtype == GVA_E4M3 && shape && cfg.page_size % 64 == 0 && cfg.G <= 8;
 }
+// resident blocks per SM the grid (and the workspace) is sized for: as many as measured best where the rings fit
+inline int fp8_blocks_per_sm(const gva_config &cfg) { return (cfg.d_v == 128 && cfg.G > 4) ? 2 : GVA_FP8_BLOCKS_PER_SM; }
+inline int fp8_tile(const gva_config &cfg) { return cfg.d_v == 64 ? 64 : 32; }
 
 inline bool encode_map_u8(const MmaHostState &st, CUtensorMap *map, const void *base, uint64_t inner, uint64_t rows,
                           uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz) {
@@ -473,32 +494,35 @@ inline bool encode_map_u8(const MmaHostState &st, CUtensorMap *map, const void *
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-inline int launch_decode_fp8(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
-                             int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out, int *tile_out,
-                             int *rec_mult_out) {
-    using T = Fp8Traits;
+template <int DV, int DR, int TILE>
+int launch_fp8_t(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
+                 int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out) {
+    using T = Fp8Traits<DV, DR, TILE>;
     constexpr int NSTAGE = GVA_FP8_NSTAGE;
-    if (!fp8_supported(cfg)) return GVA_ERR_UNSUPPORTED;
-    if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
+    constexpr int wpg = GVA_FP8_WPG;      // warps per group (each takes 1 / wpg of a tile's tokens); one measured fastest
     const int G = cfg.G;
+    if (G * wpg + 1 > 9) return GVA_ERR_UNSUPPORTED;
     const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
-    constexpr int wpg = GVA_FP8_WPG;      // warps per group (each takes 1 / wpg of a tile's tokens); one measured fastest
-    if (cfg.G * wpg + 1 > 9) return GVA_ERR_UNSUPPORTED;
-    auto fn = decode_fp8_kernel<NSTAGE, wpg>;
+    auto fn = decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg>;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
     CUtensorMap tm_v, tm_k;
-    if (!encode_map_u8(st, &tm_v, p.v_pool, T::DV, (uint64_t)p.num_pages * G * p.P, T::DV, T::TILE, CU_TENSOR_MAP_SWIZZLE_64B))
+    if (!encode_map_u8(st, &tm_v, p.v_pool, DV, (uint64_t)p.num_pages * G * p.P, DV, TILE,
+                       DV == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B))
         return GVA_ERR_CUDA;
-    if (!encode_map_u8(st, &tm_k, p.kr_pool, T::DR, (uint64_t)p.num_pages * p.P, T::DR, T::TILE, CU_TENSOR_MAP_SWIZZLE_NONE))
+    if (DR == 0) {
+        tm_k = tm_v;      // value-only cache: no positional tile (the kernel never uses this map)
+    } else if (!encode_map_u8(st, &tm_k, p.kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, TILE,
+                              DR == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE)) {
         return GVA_ERR_CUDA;
+    }
     const int threads = 32 * (G * wpg + 1);
     int grid;
     if (num_splits > 0) {
         grid = B * num_splits;
     } else {
-        const long long tiles_ub = (long long)B * ((max_seq_len + T::TILE - 1) / T::TILE);
-        const long long want = (long long)GVA_FP8_BLOCKS_PER_SM * sm_count;      // two blocks per SM, as the workspace is sized for (d_v = 64)
+        const long long tiles_ub = (long long)B * ((max_seq_len + TILE - 1) / TILE);
+        const long long want = (long long)fp8_blocks_per_sm(cfg) * sm_count;      // what the workspace is sized for
         grid = (int)(tiles_ub < want ? (tiles_ub < 1 ? 1 : tiles_ub) : want);
     }
     DecodeParams pp = p;
@@ -508,9 +532,21 @@ inline int launch_decode_fp8(const gva_config &cfg, const MmaHostState &st, int 
         return GVA_ERR_CUDA;
     }
     *n_blocks_out = grid;
-    *tile_out = T::TILE;
-    *rec_mult_out = wpg;
     return GVA_OK;
+}
+
+inline int launch_decode_fp8(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
+                             int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out, int *tile_out,
+                             int *rec_mult_out) {
+    if (!fp8_supported(cfg)) return GVA_ERR_UNSUPPORTED;
+    if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
+    *tile_out = fp8_tile(cfg);
+    *rec_mult_out = GVA_FP8_WPG;
+    if (cfg.d_v == 64)
+        return cfg.d_r == 16 ? launch_fp8_t<64, 16, 64>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, stream, n_blocks_out)
+                             : launch_fp8_t<64, 0, 64>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, stream, n_blocks_out);
+    return cfg.d_r == 32 ? launch_fp8_t<128, 32, 32>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, stream, n_blocks_out)
+                         : launch_fp8_t<128, 0, 32>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, stream, n_blocks_out);
 }
 
 }  // namespace gva

@@ -25,18 +25,23 @@ def U():
     return gpu_util
 
 
+SHAPES = [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_A0, wl.SHAPE_B0]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
 @pytest.mark.parametrize("num_splits", [0, 1, 5, 40])
-def test_ragged_edge_lengths_poisoned(num_splits):
+def test_ragged_edge_lengths_poisoned(shape, num_splits):
     # lengths around tile and page boundaries, an empty sequence, more splits than tiles; every slot no live token
     # occupies holds the NaN code and unused block-table entries are -1
-    case = wl.make_case("edge8", wl.SHAPE_A, EDGE_LENS, page_size=64, cache_dtype="fp8", seed=801, poison_unused=True,
+    case = wl.make_case("edge8", shape, EDGE_LENS, page_size=64, cache_dtype="fp8", seed=801, poison_unused=True,
                         extra_pages=2)
     U().check_decode(case, gb.GVA_KERNEL_AUTO, num_splits=num_splits)
 
 
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
 @pytest.mark.parametrize("num_splits", [0, 2, 7])
-def test_long_batch_all_split_counts(num_splits):
-    case = wl.make_case("long8", wl.SHAPE_A, [4096] * 8, page_size=64, cache_dtype="fp8", paged=False, seed=802)
+def test_long_batch_all_split_counts(shape, num_splits):
+    case = wl.make_case("long8", shape, [4096] * 8, page_size=64, cache_dtype="fp8", paged=False, seed=802)
     dc = harness.upload(case)
     try:
         U().check_decode(case, gb.GVA_KERNEL_AUTO, num_splits=num_splits, dc=dc)
@@ -45,16 +50,19 @@ def test_long_batch_all_split_counts(num_splits):
         dc.close()
 
 
-def test_every_value_dim_and_token_slot_lands_where_it_should():
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+def test_every_value_dim_and_token_slot_lands_where_it_should(shape):
     # one-hot probes: a cache whose only non-zero element is (token t, group g, dim d) and a flat score row give
     # out[h, d'] = value / T at d' = d for the heads of group g and zero elsewhere -- catches any permutation of dims,
     # tokens or heads on the way through the byte fragments
     T = 128
-    case = wl.make_case("onehot8", wl.SHAPE_A, [T] * 6, page_size=64, cache_dtype="fp8", seed=803, q_gain=0.0)
+    case = wl.make_case("onehot8", shape, [T] * 6, page_size=64, cache_dtype="fp8", seed=803, q_gain=0.0)
     one = int(wl.f32_to_e4m3_bits(np.array([1.0], dtype=np.float32))[0])
     case.v_pool[:] = 0
     case.kr_pool[:] = 0
     probes = [(0, 0, 0), (1, 1, 17), (77, 2, 34), (127, 3, 63), (64, 0, 49), (15, 3, 6)]
+    if shape.d_v == 128:
+        probes = [(0, 0, 0), (1, 5, 17 + 64), (77, 2, 34), (127, 7, 127), (33, 4, 49 + 64), (47, 3, 6 + 64)]
     for b, (t, g, d) in enumerate(probes):
         page = int(case.block_table[b, t // 64])
         case.v_pool[page, g, t % 64, d] = one
@@ -73,12 +81,14 @@ def test_every_value_dim_and_token_slot_lands_where_it_should():
         dc.close()
 
 
-def test_score_side_sees_every_dim_in_place():
+@pytest.mark.parametrize("s", [wl.SHAPE_A, wl.SHAPE_B])
+def test_score_side_sees_every_dim_in_place(s):
     # scores pick the token: a query far along one dim and a cache whose token t carries a large value at that dim only
     # must put (nearly) all weight on t -- one probe per 16-dim chunk and byte lane, the positional slice included
     T = 64
-    s = wl.SHAPE_A
-    dims = [0, 1, 2, 3, 5, 18, 35, 52, 63, 64, 67, 70, 79]        # >= 64: the positional slice
+    dims = [0, 1, 2, 3, 5, 18, 35, 52, 63, 64, 67, 70, 79]        # >= d_v: the positional slice
+    if s.d_v == 128:
+        dims = [0, 3, 18, 63, 64, 77, 100, 127, 128, 131, 141, 146, 159]
     case = wl.make_case("score8", s, [T] * len(dims), page_size=64, cache_dtype="fp8", seed=804, q_gain=0.0)
     big = int(wl.f32_to_e4m3_bits(np.array([16.0], dtype=np.float32))[0])
     one = int(wl.f32_to_e4m3_bits(np.array([1.0], dtype=np.float32))[0])
@@ -123,9 +133,10 @@ def test_page_sizes_and_contiguous():
         U().check_decode(case, gb.GVA_KERNEL_AUTO)
 
 
-def test_append_is_bit_exact_and_saturates():
+@pytest.mark.parametrize("shape", SHAPES)
+def test_append_is_bit_exact_and_saturates(shape):
     lens = [1, 64, 65, 300, 129, 4000, 8193]
-    case = wl.make_case("append8", wl.SHAPE_A, lens, page_size=64, cache_dtype="fp8", seed=808, extra_pages=3)
+    case = wl.make_case("append8", shape, lens, page_size=64, cache_dtype="fp8", seed=808, extra_pages=3)
     # values beyond the largest finite code, ties between codes, subnormals and zeros of both signs
     case.v_new[0, 0, :8] = [1e6, -1e6, 448.0, 464.0, 1.0625, 1.1875, 2.0 ** -10, -0.0]
     case.v_new[1, 1, :4] = [3 * 2.0 ** -10, 2.0 ** -6 - 2.0 ** -10, -449.0, 0.0]
@@ -158,9 +169,10 @@ def test_append_chunk_is_bit_exact():
     assert np.array_equal(v, v_ref) and np.array_equal(k, k_ref)
 
 
-def test_fused_step_is_bitwise_the_three_calls_and_matches_the_oracle():
+@pytest.mark.parametrize("shape", SHAPES)
+def test_fused_step_is_bitwise_the_three_calls_and_matches_the_oracle(shape):
     lens = np.array([1, 64, 65, 1001, 4096, 130], dtype=np.int32)
-    mk = lambda: wl.make_case("fstep8", wl.SHAPE_A, lens, page_size=64, cache_dtype="fp8", seed=809,
+    mk = lambda: wl.make_case("fstep8", shape, lens, page_size=64, cache_dtype="fp8", seed=809,
                               q_pos=lens - 1, append_pos=lens - 1)
     case = mk()
     a, b = harness.upload(mk()), harness.upload(mk())
@@ -197,7 +209,7 @@ def test_static_entry_point_and_host_step():
 
 
 def test_what_the_8_bit_cache_does_not_cover():
-    for kw in (dict(H=32, G=8, d_v=128, d_c=128, d_r=32, page_size=64), dict(H=16, G=4, d_v=64, d_c=64, d_r=24, page_size=64),
+    for kw in (dict(H=16, G=4, d_v=64, d_c=64, d_r=24, page_size=64),
                dict(H=16, G=4, d_v=64, d_c=64, d_r=16, page_size=32),
                dict(H=16, G=4, d_v=64, d_c=64, d_r=16, page_size=64, kernel=gb.GVA_KERNEL_FMA)):
         with pytest.raises(gb.GvaError) as e:
