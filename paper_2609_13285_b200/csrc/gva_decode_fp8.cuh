@@ -82,8 +82,8 @@ __device__ __forceinline__ uint32_t split_hi_lo_f16(float x) {
     return (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
 }
 
-template <int DV, int DR, int TILE, int NSTAGE, int WPG>
-__global__ void __launch_bounds__(32 * 9, DV == 128 ? 2 : 3)      // register caps: 4 five-warp blocks (d_v = 64) or 2 nine-warp blocks (d_v = 128) per SM
+template <int DV, int DR, int TILE, int NSTAGE, int WPG, int GMAX>
+__global__ void __launch_bounds__(32 * (GMAX * WPG + 1), GMAX <= 4 ? 4 : 2)      // register caps: 4 five-warp blocks (d_v = 64) or 2 nine-warp blocks (d_v = 128) per SM
 decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = Fp8Traits<DV, DR, TILE>;
     constexpr int CPW = T::CHUNKS / WPG;          // 16-token chunks per consumer warp and tile
@@ -353,6 +353,12 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 __syncwarp();
             }
             const uint32_t vt_u32 = smem_u32(vt) + row0 * DV;
+            uint32_t a_qk[DV / 32], a_pv[DV / 32];            // per pair of pieces: this lane's row address within a chunk
+#pragma unroll
+            for (int pr = 0; pr < DV / 32; ++pr) {
+                a_qk[pr] = vt_u32 + off_qk + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_qk) << 4);
+                a_pv[pr] = vt_u32 + off_pv + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_pv) << 4);
+            }
             const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES) + row0 * T::KR_ROW;
 
             // ---- S^T = V_tile . Q^T (+ positional part), 16 tokens per m-tile ----
@@ -364,7 +370,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 #pragma unroll
                 for (int pr = 0; pr < DV / 32; ++pr) {        // two 16-dim chunks per fetch
                     uint32_t r[4];                             // (tok r8, chunk 2 pr) (tok r8 + 8, chunk 2 pr) (tok r8, chunk 2 pr + 1) (tok r8 + 8, ..)
-                    ldsm_x4(vt_u32 + c * 16 * DV + off_qk + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_qk) << 4), r);
+                    ldsm_x4(a_qk[pr] + c * 16 * DV, r);
 #pragma unroll
                     for (int hx = 0; hx < 2; ++hx) {
                         uint32_t a[4];
@@ -411,13 +417,15 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             const float m_new = fmaxf(m_run, tmax * scale);          // scale > 0: max commutes with it
             const bool live = m_new != -INFINITY;
             const float m_use = live ? m_new : 0.f;                  // keeps (-inf) - (-inf) out of the exponent
-            const float corr = fast_exp2(m_run - m_use);             // 2^(-inf) = 0 for the first live tile
+            if (__any_sync(0xffffffffu, m_new != m_run)) {           // rare once the running maxima have settled
+                const float corr = fast_exp2(m_run - m_use);         // 2^(-inf) = 0 for the first live tile
+                l_run *= corr;
+#pragma unroll
+                for (int mt = 0; mt < T::MT; ++mt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) oacc[mt][e] *= corr;
+            }
             m_run = m_new;
-            l_run *= corr;
-#pragma unroll
-            for (int mt = 0; mt < T::MT; ++mt)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) oacc[mt][e] *= corr;
 
             // ---- O^T += V_tile^T . P^T: m-tile mt holds value dims 16 mt .. 16 mt + 15 ----
 #pragma unroll
@@ -433,7 +441,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 #pragma unroll
                 for (int pr = 0; pr < DV / 32; ++pr) {
                     uint32_t r[4];    // dims 32 pr + (r8 | r8 + 8) and 32 pr + 16 + (r8 | r8 + 8), tokens pi(4 jh .. 4 jh + 3) each
-                    ldsm_b8_x2_trans(vt_u32 + c * 16 * DV + off_pv + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_pv) << 4), r);
+                    ldsm_b8_x2_trans(a_pv[pr] + c * 16 * DV, r);
 #pragma unroll
                     for (int hx = 0; hx < 2; ++hx) {
                         uint32_t a[4];
@@ -504,7 +512,7 @@ int launch_fp8_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
     if (G * wpg + 1 > 9) return GVA_ERR_UNSUPPORTED;
     const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
-    auto fn = decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg>;
+    auto fn = G <= 4 ? decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 4> : decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 8>;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
     CUtensorMap tm_v, tm_k;
     if (!encode_map_u8(st, &tm_v, p.v_pool, DV, (uint64_t)p.num_pages * G * p.P, DV, TILE,
