@@ -251,3 +251,27 @@ def test_full_size_long_context_sampled():
         assert np.max(np.abs(o - target)) < 0.25      # e4m3 rounding of N(0, 1) rows adds ~0.1 % variance only
     finally:
         dc.close()
+
+
+def test_full_size_ragged_wide_heads_sampled():
+    # bench.py's cfg3-fp8 workload (64 ragged sequences, H=32, d_v=128, one byte per cache element), same launch: the
+    # shortest, a median and the longest sequence against the oracle; finiteness for the rest
+    seed = wl.MASTER_SEED + 3000
+    case = wl.make_case("cfg3-fp8", wl.SHAPE_B, wl.config3_seq_lens(seed), page_size=64, cache_dtype="fp8", paged=True,
+                        seed=seed, poison_unused=True)
+    order = np.argsort(case.seq_lens)
+    sample = [int(order[0]), int(order[len(order) // 2]), int(order[-1])]
+    dc = harness.upload(case)
+    try:
+        dc.absorb()
+        out, lse = dc.decode(num_splits=0)
+        torch.cuda.synchronize()
+        assert int(dc.status.item()) == 0
+        o = out.cpu().numpy().astype(np.float64)
+        assert np.isfinite(o).all()
+        lens = np.zeros_like(case.seq_lens)
+        lens[sample] = case.seq_lens[sample]
+        ref, _ = U().oracle_for_gpu_q(case, dc.q_abs, seq_lens=lens)
+        assert np.max(np.abs(o[sample] - ref[sample])) <= U().TOL_TIGHT_MAXABS
+    finally:
+        dc.close()
