@@ -367,19 +367,21 @@ int gva_absorb_query(gva_handle *h, const float *q_c, const float *q_r, const fl
         return GVA_ERR_INVALID_ARG;
     const gva_config &c = h->cfg;
     const size_t smem = absorb_smem_bytes(c.d_v, c.d_c);
-    // many rows (prefill): the map row lives in registers and the rows stream through shared memory
-    const bool vec_ok = aligned(q_c, 16) && aligned(M, 16);
+    // many rows (prefill): a batch of small GEMMs on the tensor cores (f16 hi/lo operands, f32-level accuracy)
+    const bool vec_ok = aligned(q_c, 16) && aligned(M, 16) && aligned(q_r, 8);
     if (B >= 512 && vec_ok && ((c.d_v == 64 && c.d_c == 64) || (c.d_v == 128 && c.d_c == 128))) {
+        const int chunk = kAbsorbMmaRows;
+        const size_t smem_mma = c.d_v == 64 ? AbsorbMmaTraits<64, 64>::smem_bytes() : AbsorbMmaTraits<128, 128>::smem_bytes();
         int per_head = (4 * h->sm_count + c.H - 1) / c.H;                 // about four blocks per SM in all
         int rows_per_block = (B + per_head - 1) / per_head;
-        rows_per_block = (rows_per_block + kAbsorbChunk - 1) / kAbsorbChunk * kAbsorbChunk;
+        rows_per_block = (rows_per_block + chunk - 1) / chunk * chunk;
         const dim3 g2(c.H, (B + rows_per_block - 1) / rows_per_block);
-        cudaError_t ce = c.d_v == 64
-            ? launch_pdl(absorb_rows_kernel<64, 64>, g2, dim3(kAbsorbThreads), 0, static_cast<cudaStream_t>(stream), q_c, q_r, M,
-                         q_pos, q_abs, B, c.H, c.d_r, rows_per_block, h->rope)
-            : launch_pdl(absorb_rows_kernel<128, 128>, g2, dim3(kAbsorbThreads), 0, static_cast<cudaStream_t>(stream), q_c, q_r,
-                         M, q_pos, q_abs, B, c.H, c.d_r, rows_per_block, h->rope);
-        if (ce != cudaSuccess) {
+        auto fn = c.d_v == 64 ? absorb_rows_mma_kernel<64, 64> : absorb_rows_mma_kernel<128, 128>;
+        if (smem_mma > (size_t)h->smem_optin ||
+            cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_mma) != cudaSuccess)
+            return GVA_ERR_CUDA;
+        if (launch_pdl(fn, g2, dim3(kAbsorbMmaThreads), smem_mma, static_cast<cudaStream_t>(stream), q_c, q_r, M, q_pos, q_abs,
+                       B, c.H, c.d_r, rows_per_block, h->rope) != cudaSuccess) {
             (void)cudaGetLastError();
             return GVA_ERR_CUDA;
         }

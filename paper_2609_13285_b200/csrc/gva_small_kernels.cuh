@@ -165,89 +165,141 @@ absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, cons
     absorb_block(q_c, q_r, M, q_pos, q_abs, B, H, d_v, d_c, d_r, rope, blockIdx.x, blockIdx.y * kAbsorbBatch, smem_f);
 }
 
-// ---- absorb for many rows (prefill: one row per new token) -----------------------------------------
-// grid (H, blocks per head), block 256.  Thread t keeps row i = t % DV of M_h in registers for the whole block and
-// serves the rows r with r % (256 / DV) == t / DV of every chunk; query rows stream through a double-buffered
-// shared-memory chunk (cp.async) and are read as broadcasts.  Each output is the same j-ordered chain of fused
-// multiply-adds as in absorb_block, so both kernels give identical bits.
-constexpr int kAbsorbChunk = 32;          // query rows per chunk
+// ---- absorb for many rows on the tensor cores --------------------------------------------------------
+// The same product as a batch of small GEMMs, Q_abs[:, h, :d_v] = Q_c[:, h, :] M_h^T, with f32-level accuracy from f16
+// MMAs: both operands are split x = hi + lo (f16 each, 22 significant bits together) and hi*hi + hi*lo + lo*hi is
+// accumulated in f32 (the dropped lo*lo term is below 2^-22 relative).  grid (H, blocks per head), block 128: M_h's two
+// halves sit in shared memory as f16 [d_v][d_c] (rows padded by 8 so that fragment loads are conflict-free); each warp
+// walks its own 16-row tiles of the block's strip, fetching the A fragments straight from global memory (a warp-wide
+// load covers whole 32-byte sectors) one tile ahead, so that no barrier and no staging buffer sits on the stream.
+// The rotated positional slice is computed as in the other absorb kernels (fp64, one rounding), but once per row for all
+// heads: the H blocks that share a strip of rows split its rows among themselves.
+__device__ __forceinline__ void mma_m16n8k16_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void split_f16x2(float x, float y, uint32_t &hi, uint32_t &lo) {
+    const __half2 h = __floats2half2_rn(x, y);
+    const float2 f = __half22float2(h);
+    const __half2 l = __floats2half2_rn(x - f.x, y - f.y);
+    hi = *reinterpret_cast<const uint32_t *>(&h);
+    lo = *reinterpret_cast<const uint32_t *>(&l);
+}
+constexpr int kAbsorbMmaThreads = 128;
+constexpr int kAbsorbMmaRows = (kAbsorbMmaThreads / 32) * 16;       // rows a block covers per round of its warps
 template <int DV, int DC>
-__global__ void __launch_bounds__(kAbsorbThreads)
-absorb_rows_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, const float *__restrict__ M,
-                   const int32_t *__restrict__ q_pos, float *__restrict__ q_abs, int B, int H, int d_r, int rows_per_block,
-                   RopeTable rope) {
-    constexpr int NG = kAbsorbThreads / DV;            // row groups
-    constexpr int RPT = kAbsorbChunk / NG;             // rows per thread and chunk
-    static_assert(kAbsorbThreads % DV == 0 && kAbsorbChunk % NG == 0 && RPT % 4 == 0 && DC % 4 == 0, "tiling");
+struct AbsorbMmaTraits {
+    static constexpr int MLD = DC + 8;                              // f16 elements per row of a map half
+    static constexpr size_t smem_bytes() { return (size_t)2 * DV * MLD * 2; }
+};
+template <int DV, int DC>
+__global__ void __launch_bounds__(kAbsorbMmaThreads)
+absorb_rows_mma_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, const float *__restrict__ M,
+                       const int32_t *__restrict__ q_pos, float *__restrict__ q_abs, int B, int H, int d_r, int rows_per_block,
+                       RopeTable rope) {
+    using T = AbsorbMmaTraits<DV, DC>;
+    constexpr int MLD = T::MLD, NT = DV / 8, KS = DC / 16;
     grid_dependency_launch();
-    __shared__ __align__(16) float sq[2][kAbsorbChunk][DC];
-    const int tid = threadIdx.x, h = blockIdx.x;
-    const int i = tid % DV, grp = tid / DV;
+    extern __shared__ __align__(16) unsigned char absorb_smem[];
+    __half *m_hi = reinterpret_cast<__half *>(absorb_smem);
+    __half *m_lo = m_hi + DV * MLD;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, h = blockIdx.x;
+    const int g = lane >> 2, t = lane & 3;
     const int row0 = blockIdx.y * rows_per_block;
     const int row1 = min(B, row0 + rows_per_block);
     grid_dependency_wait();
     if (row0 >= row1) return;
-    float m[DC];
-    {
-        const float4 *src = reinterpret_cast<const float4 *>(M + ((size_t)h * DV + i) * DC);
-#pragma unroll
-        for (int j = 0; j < DC / 4; ++j) {
-            const float4 v = __ldg(src + j);
-            m[4 * j] = v.x; m[4 * j + 1] = v.y; m[4 * j + 2] = v.z; m[4 * j + 3] = v.w;
-        }
+    // the map, split once per block
+    for (int e = tid; e < DV * DC / 2; e += kAbsorbMmaThreads) {
+        const int i = e / (DC / 2), j = (e % (DC / 2)) * 2;
+        const float2 v = *reinterpret_cast<const float2 *>(M + ((size_t)h * DV + i) * DC + j);
+        uint32_t hi, lo;
+        split_f16x2(v.x, v.y, hi, lo);
+        *reinterpret_cast<uint32_t *>(m_hi + i * MLD + j) = hi;
+        *reinterpret_cast<uint32_t *>(m_lo + i * MLD + j) = lo;
     }
     const int dq = DV + d_r, half = d_r / 2;
-    auto stage = [&](int buf, int r0) {
-        const int n = min(kAbsorbChunk, row1 - r0);
-        const uint32_t dst = smem_u32(&sq[buf][0][0]);
-        for (int c = tid; c < n * (DC / 4); c += kAbsorbThreads) {
-            const int rr = c / (DC / 4), col = c % (DC / 4);
-            cp_async16(dst + (rr * DC + col * 4) * 4, q_c + ((size_t)(r0 + rr) * H + h) * DC + col * 4, 16);
-        }
-        cp_async_commit();
-    };
-    stage(0, row0);
-    int buf = 0;
-    for (int r0 = row0; r0 < row1; r0 += kAbsorbChunk, buf ^= 1) {
-        const int n = min(kAbsorbChunk, row1 - r0);
-        if (r0 + kAbsorbChunk < row1) stage(buf ^ 1, r0 + kAbsorbChunk);
-        else cp_async_commit();
-        // the positional slices of this chunk: one rotation pair per thread and pass, in fp64
-        for (int e = tid; e < n * half; e += kAbsorbThreads) {
-            const int rr = e / half, k = e % half;
-            const size_t src = ((size_t)(r0 + rr) * H + h) * d_r + 2 * k;
-            double y0, y1;
-            rope_pair((double)q_r[src], (double)q_r[src + 1], q_pos[r0 + rr], rope.inv_freq[k], y0, y1);
-            float *dst = q_abs + ((size_t)(r0 + rr) * H + h) * dq + DV + 2 * k;
-            dst[0] = __double2float_rn(y0);
-            dst[1] = __double2float_rn(y1);
-        }
-        cp_async_wait<1>();
-        __syncthreads();
+    // the positional slices of this block's share of the strip: one (row, pair) per thread and pass, all heads
+    {
+        const int n = row1 - row0, per = (n + H - 1) / H, lo = min(n, h * per), cnt = min(n, lo + per) - lo;
+        for (int e = tid; e < cnt * half; e += kAbsorbMmaThreads) {
+            const int row = row0 + lo + e / half, k = e % half;
+            double sn, cs;
+            sincos((double)q_pos[row] * rope.inv_freq[k], &sn, &cs);
+            const float *src = q_r + (size_t)row * H * d_r + 2 * k;
+            float *dst = q_abs + (size_t)row * H * dq + DV + 2 * k;
+            for (int h0 = 0; h0 < H; h0 += 8) {
+                float2 x[8];
 #pragma unroll
-        for (int pass = 0; pass < RPT / 4; ++pass) {
-            float a[4] = {0.f, 0.f, 0.f, 0.f};
-            const float4 *p[4];
+                for (int u = 0; u < 8; ++u)      // eight independent loads in flight
+                    x[u] = (h0 + u < H) ? *reinterpret_cast<const float2 *>(src + (size_t)(h0 + u) * d_r) : make_float2(0.f, 0.f);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) p[k] = reinterpret_cast<const float4 *>(&sq[buf][min(grp + NG * (pass * 4 + k), n - 1)][0]);
-#pragma unroll
-            for (int j = 0; j < DC / 4; ++j) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float4 x = p[k][j];
-                    a[k] = fmaf(x.x, m[4 * j], a[k]);
-                    a[k] = fmaf(x.y, m[4 * j + 1], a[k]);
-                    a[k] = fmaf(x.z, m[4 * j + 2], a[k]);
-                    a[k] = fmaf(x.w, m[4 * j + 3], a[k]);
+                for (int u = 0; u < 8; ++u) {
+                    const double x0 = (double)x[u].x, x1 = (double)x[u].y;
+                    if (h0 + u < H)
+                        *reinterpret_cast<float2 *>(dst + (size_t)(h0 + u) * dq) =
+                            make_float2(__double2float_rn(x0 * cs - x1 * sn), __double2float_rn(x0 * sn + x1 * cs));
                 }
             }
+        }
+    }
+    __syncthreads();                // the split map is visible to every warp
+    // A fragments of one 16-row tile: rows g and g + 8, k = 16 ks + 2t, +1 and + 8, + 9 -- 8 bytes per lane and load
+    auto fetch = [&](int r0, float2 (&x)[KS][4]) {
+        const int ra = min(r0 + g, row1 - 1), rb = min(r0 + g + 8, row1 - 1);      // rows past the end repeat the last one
+        const float *pa = q_c + ((size_t)ra * H + h) * DC + 2 * t;
+        const float *pb = q_c + ((size_t)rb * H + h) * DC + 2 * t;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int rr = grp + NG * (pass * 4 + k);
-                if (rr < n) q_abs[((size_t)(r0 + rr) * H + h) * dq + i] = a[k];
+        for (int ks = 0; ks < KS; ++ks) {
+            x[ks][0] = *reinterpret_cast<const float2 *>(pa + ks * 16);
+            x[ks][1] = *reinterpret_cast<const float2 *>(pb + ks * 16);
+            x[ks][2] = *reinterpret_cast<const float2 *>(pa + ks * 16 + 8);
+            x[ks][3] = *reinterpret_cast<const float2 *>(pb + ks * 16 + 8);
+        }
+    };
+    float2 cur[KS][4], nxt[KS][4];
+    int r0 = row0 + warp * 16;
+    if (r0 < row1) fetch(r0, cur);
+    for (; r0 < row1; r0 += kAbsorbMmaRows) {
+        const int rn = r0 + kAbsorbMmaRows;
+        if (rn < row1) fetch(rn, nxt);
+        float acc[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            uint32_t a_hi[4], a_lo[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) split_f16x2(cur[ks][e].x, cur[ks][e].y, a_hi[e], a_lo[e]);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                // B = M_h^T: element (k, n) is M_h[n][k]; a fragment register is two consecutive k of one n
+                const int off = (nt * 8 + g) * MLD + ks * 16 + 2 * t;
+                const uint32_t bh0 = *reinterpret_cast<const uint32_t *>(m_hi + off);
+                const uint32_t bh1 = *reinterpret_cast<const uint32_t *>(m_hi + off + 8);
+                const uint32_t bl0 = *reinterpret_cast<const uint32_t *>(m_lo + off);
+                const uint32_t bl1 = *reinterpret_cast<const uint32_t *>(m_lo + off + 8);
+                mma_m16n8k16_f16(acc[nt], a_lo, bh0, bh1);      // small terms first
+                mma_m16n8k16_f16(acc[nt], a_hi, bl0, bl1);
+                mma_m16n8k16_f16(acc[nt], a_hi, bh0, bh1);
             }
         }
-        __syncthreads();        // the chunk is consumed before the copy after next overwrites it
+        const int ra = r0 + g, rb = ra + 8;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            if (ra < row1)
+                *reinterpret_cast<float2 *>(q_abs + ((size_t)ra * H + h) * dq + nt * 8 + 2 * t) = make_float2(acc[nt][0], acc[nt][1]);
+            if (rb < row1)
+                *reinterpret_cast<float2 *>(q_abs + ((size_t)rb * H + h) * dq + nt * 8 + 2 * t) = make_float2(acc[nt][2], acc[nt][3]);
+        }
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) cur[ks][e] = nxt[ks][e];
     }
 }
 
@@ -340,7 +392,9 @@ append_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *
 }
 
 // Append of a chunk of new tokens per sequence: input row n becomes token ctx_lens[b] + (n - cu_q[b]) of the sequence b
-// that owns the row (found by bisection of cu_q).  A block writes kAppendChunkRows consecutive rows.
+// that owns the row (found by bisection of cu_q).  A block writes kAppendChunkRows consecutive rows, all at once: 16
+// threads per row first resolve the row's page and slot and write its rotated positional key (one pair each, fp64), then
+// the whole block copies the value rows with every load independent of the others.
 constexpr int kAppendChunkRows = 8;
 template <typename CT>
 __global__ void __launch_bounds__(128)
@@ -348,24 +402,74 @@ append_chunk_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int
                     const float *__restrict__ v_new, const float *__restrict__ kr_new, const int32_t *__restrict__ cu_q,
                     const int32_t *__restrict__ ctx_lens, int B, int G, int d_v, int d_r, int P, int num_pages, int max_pages,
                     int32_t *dev_status, RopeTable rope) {
+    static_assert(kAppendChunkRows * kMaxRopePairs == 128, "16 threads per row");
     grid_dependency_launch();
+    __shared__ long long s_page[kAppendChunkRows];      // -1: the row is not written
+    __shared__ int s_slot[kAppendChunkRows];
     grid_dependency_wait();
     const int total = cu_q[B];
-    int b = -1;
-    for (int k = 0; k < kAppendChunkRows; ++k) {
-        const int n = blockIdx.x * kAppendChunkRows + k;
-        if (n >= total) return;
-        if (b < 0 || n >= cu_q[b + 1]) {        // largest b with cu_q[b] <= n (empty sequences repeat an offset)
-            int lo = 0, hi = B - 1;
+    {
+        const int r = threadIdx.x / kMaxRopePairs, k = threadIdx.x % kMaxRopePairs;
+        const int n = blockIdx.x * kAppendChunkRows + r;
+        long long page = -1;
+        int slot = 0;
+        if (n < total) {
+            int lo = 0, hi = B - 1;                     // largest b with cu_q[b] <= n (empty sequences repeat an offset)
             while (lo < hi) {
                 const int mid = (lo + hi + 1) >> 1;
                 if (cu_q[mid] <= n) lo = mid;
                 else hi = mid - 1;
             }
-            b = lo;
+            const int b = lo, t = ctx_lens[b] + (n - cu_q[b]);
+            float k0 = 0.f, k1 = 0.f;
+            if (k < d_r / 2) {
+                k0 = kr_new[(size_t)n * d_r + 2 * k];
+                k1 = kr_new[(size_t)n * d_r + 2 * k + 1];
+            }
+            if (t < 0 || t / P >= max_pages) {
+                if (k == 0) report_error(dev_status, GVA_ERR_SEQ_LEN, b);
+            } else {
+                page = block_table ? (long long)block_table[(size_t)b * max_pages + t / P] : (long long)b * max_pages + t / P;
+                slot = t % P;
+                if (page < 0 || page >= num_pages) {
+                    if (k == 0) report_error(dev_status, GVA_ERR_BAD_PAGE, b);
+                    page = -1;
+                } else if (k < d_r / 2) {
+                    double y0, y1;
+                    rope_pair((double)k0, (double)k1, t, rope.inv_freq[k], y0, y1);
+                    const size_t dst = ((size_t)page * P + slot) * d_r + 2 * k;
+                    if constexpr (sizeof(CT) == 1) {
+                        reinterpret_cast<uint8_t *>(kr_pool)[dst] = double_to_e4m3_bits(y0);
+                        reinterpret_cast<uint8_t *>(kr_pool)[dst + 1] = double_to_e4m3_bits(y1);
+                    } else if constexpr (sizeof(CT) == 2) {
+                        reinterpret_cast<uint16_t *>(kr_pool)[dst] = double_to_bf16_bits(y0);
+                        reinterpret_cast<uint16_t *>(kr_pool)[dst + 1] = double_to_bf16_bits(y1);
+                    } else {
+                        reinterpret_cast<float *>(kr_pool)[dst] = __double2float_rn(y0);
+                        reinterpret_cast<float *>(kr_pool)[dst + 1] = __double2float_rn(y1);
+                    }
+                }
+            }
         }
-        append_row<CT>(v_pool, kr_pool, block_table, v_new, kr_new, G, d_v, d_r, P, num_pages, max_pages, dev_status, rope, n, b,
-                       ctx_lens[b] + (n - cu_q[b]));
+        if (k == 0) {
+            s_page[r] = page;
+            s_slot[r] = slot;
+        }
+    }
+    __syncthreads();
+    const int n_v = G * d_v;
+    const int rows = min(kAppendChunkRows, total - (int)blockIdx.x * kAppendChunkRows);
+    const float *src = v_new + (size_t)blockIdx.x * kAppendChunkRows * n_v;
+    for (int e = threadIdx.x; e < rows * n_v; e += 128) {
+        const int r = e / n_v, i = e % n_v;
+        const long long page = s_page[r];
+        if (page < 0) continue;
+        const int g = i / d_v, d = i % d_v;
+        const size_t dst = (((size_t)page * G + g) * P + s_slot[r]) * d_v + d;
+        const float x = src[e];
+        if constexpr (sizeof(CT) == 1) reinterpret_cast<uint8_t *>(v_pool)[dst] = float_to_e4m3_bits(x);
+        else if constexpr (sizeof(CT) == 2) reinterpret_cast<uint16_t *>(v_pool)[dst] = float_to_bf16_bits(x);
+        else reinterpret_cast<float *>(v_pool)[dst] = x;
     }
 }
 

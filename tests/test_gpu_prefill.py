@@ -182,8 +182,9 @@ def test_prefill_reports_bad_page_and_long_sequence():
 
 @pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
 def test_absorb_many_rows_matches_oracle_and_the_small_batch_kernel(shape):
-    # prefill absorbs one row per new token: above 512 rows a kernel that streams the rows takes over; it must give
-    # the oracle's values and the very bits of the decode-batch kernel (same chain of fused multiply-adds per output)
+    # prefill absorbs one row per new token: above 512 rows a tensor-core kernel takes over (f16 hi/lo operands); it must
+    # give the oracle's values within the same bound, the same rotated slice bit for bit (fp64 rotation, one rounding),
+    # and agree with the decode-batch kernel to f32 rounding level
     n = 1000 + 37
     pc = wl.make_prefill_case("abs", shape, [3], [n], page_size=64, seed=509)
     pd = harness.upload_prefill(pc)
@@ -197,7 +198,9 @@ def test_absorb_many_rows_matches_oracle_and_the_small_batch_kernel(shape):
             hi = min(n, lo + 100)
             gb.gva_absorb_query(pd.handle, pd.q_c[lo:hi], pd.q_r[lo:hi], pd.dc.M, pd.q_pos[lo:hi], small[lo:hi], hi - lo)
         torch.cuda.synchronize()
-        assert np.array_equal(small.cpu().numpy().view(np.uint32), q.view(np.uint32))
+        sm = small.cpu().numpy()
+        assert np.array_equal(sm[..., shape.d_v:].view(np.uint32), q[..., shape.d_v:].view(np.uint32))
+        assert np.max(np.abs(sm.astype(np.float64) - q.astype(np.float64))) <= 2e-5      # each is within 1e-5 of the oracle
     finally:
         pd.close()
 
