@@ -38,6 +38,15 @@ def test_ragged_edge_lengths_poisoned(shape, num_splits):
     U().check_decode(case, gb.GVA_KERNEL_AUTO, num_splits=num_splits)
 
 
+def test_eight_groups_of_narrow_heads():
+    # d_v = 64 with G = 8 (nine-warp blocks, two per SM instead of four): ragged, poisoned, balanced and split
+    shape = wl.HeadShape(H=32, G=8, d_v=64, d_c=64, d_r=16)
+    for num_splits in (0, 3):
+        case = wl.make_case("g8", shape, [5, 64, 700, 2049, 0, 333], page_size=64, cache_dtype="fp8", seed=813,
+                            poison_unused=True)
+        U().check_decode(case, gb.GVA_KERNEL_AUTO, num_splits=num_splits)
+
+
 @pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
 @pytest.mark.parametrize("num_splits", [0, 2, 7])
 def test_long_batch_all_split_counts(shape, num_splits):
