@@ -169,7 +169,7 @@ absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, cons
 // The same product as a batch of small GEMMs, Q_abs[:, h, :d_v] = Q_c[:, h, :] M_h^T, with f32-level accuracy from f16
 // MMAs: both operands are split x = hi + lo (f16 each, 22 significant bits together) and hi*hi + hi*lo + lo*hi is
 // accumulated in f32 (the dropped lo*lo term is below 2^-22 relative).  grid (H, blocks per head), block 128: M_h's two
-// halves sit in shared memory as f16 [d_v][d_c] (rows padded by 8 so that fragment loads are conflict-free); each warp
+// halves sit in shared memory as f16 [d_v][d_c] (rows padded by 8 so that the ldmatrix fetches of B fragments are conflict-free); each warp
 // walks its own 16-row tiles of the block's strip, fetching the A fragments straight from global memory (a warp-wide
 // load covers whole 32-byte sectors) one tile ahead, so that no barrier and no staging buffer sits on the stream.
 // The rotated positional slice is computed as in the other absorb kernels (fp64, one rounding), but once per row for all
@@ -187,6 +187,11 @@ __device__ __forceinline__ void split_f16x2(float x, float y, uint32_t &hi, uint
     hi = *reinterpret_cast<const uint32_t *>(&h);
     lo = *reinterpret_cast<const uint32_t *>(&l);
 }
+__device__ __forceinline__ void absorb_ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
 constexpr int kAbsorbMmaThreads = 128;
 constexpr int kAbsorbMmaRows = (kAbsorbMmaThreads / 32) * 16;       // rows a block covers per round of its warps
 template <int DV, int DC>
@@ -195,7 +200,7 @@ struct AbsorbMmaTraits {
     static constexpr size_t smem_bytes() { return (size_t)2 * DV * MLD * 2; }
 };
 template <int DV, int DC>
-__global__ void __launch_bounds__(kAbsorbMmaThreads)
+__global__ void __launch_bounds__(kAbsorbMmaThreads, DV == 64 ? 4 : 2)
 absorb_rows_mma_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, const float *__restrict__ M,
                        const int32_t *__restrict__ q_pos, float *__restrict__ q_abs, int B, int H, int d_r, int rows_per_block,
                        RopeTable rope) {
@@ -259,6 +264,9 @@ absorb_rows_mma_kernel(const float *__restrict__ q_c, const float *__restrict__ 
             x[ks][3] = *reinterpret_cast<const float2 *>(pb + ks * 16 + 8);
         }
     };
+    // ldmatrix row address of this lane: matrices (n-tile, k 0-7), (n-tile, k 8-15), (n-tile + 1, k 0-7), (n-tile + 1, k 8-15)
+    const int b_off = (((lane >> 4) * 8 + (lane & 7)) * MLD + ((lane >> 3) & 1) * 8) * 2;
+    const uint32_t b_hi_addr = smem_u32(m_hi) + b_off, b_lo_addr = smem_u32(m_lo) + b_off;
     float2 cur[KS][4], nxt[KS][4];
     int r0 = row0 + warp * 16;
     if (r0 < row1) fetch(r0, cur);
@@ -276,16 +284,18 @@ absorb_rows_mma_kernel(const float *__restrict__ q_c, const float *__restrict__ 
 #pragma unroll
             for (int e = 0; e < 4; ++e) split_f16x2(cur[ks][e].x, cur[ks][e].y, a_hi[e], a_lo[e]);
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                // B = M_h^T: element (k, n) is M_h[n][k]; a fragment register is two consecutive k of one n
-                const int off = (nt * 8 + g) * MLD + ks * 16 + 2 * t;
-                const uint32_t bh0 = *reinterpret_cast<const uint32_t *>(m_hi + off);
-                const uint32_t bh1 = *reinterpret_cast<const uint32_t *>(m_hi + off + 8);
-                const uint32_t bl0 = *reinterpret_cast<const uint32_t *>(m_lo + off);
-                const uint32_t bl1 = *reinterpret_cast<const uint32_t *>(m_lo + off + 8);
-                mma_m16n8k16_f16(acc[nt], a_lo, bh0, bh1);      // small terms first
-                mma_m16n8k16_f16(acc[nt], a_hi, bl0, bl1);
-                mma_m16n8k16_f16(acc[nt], a_hi, bh0, bh1);
+            for (int nt = 0; nt < NT; nt += 2) {
+                // B = M_h^T: element (k, n) is M_h[n][k]; a fragment register is two consecutive k of one n, which is what
+                // ldmatrix hands out from the [n][k] rows: one fetch = (k 0-7 | k 8-15) of n-tiles nt and nt + 1
+                uint32_t bh[4], bl[4];
+                absorb_ldsm_x4(b_hi_addr + (nt * 8 * MLD + ks * 16) * 2, bh);
+                absorb_ldsm_x4(b_lo_addr + (nt * 8 * MLD + ks * 16) * 2, bl);
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    mma_m16n8k16_f16(acc[nt + u], a_lo, bh[2 * u], bh[2 * u + 1]);      // small terms first
+                    mma_m16n8k16_f16(acc[nt + u], a_hi, bl[2 * u], bl[2 * u + 1]);
+                    mma_m16n8k16_f16(acc[nt + u], a_hi, bh[2 * u], bh[2 * u + 1]);
+                }
             }
         }
         const int ra = r0 + g, rb = ra + 8;
