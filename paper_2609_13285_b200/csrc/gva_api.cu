@@ -197,11 +197,11 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     }
     if (h->cfg.cache_dtype == GVA_E4M3) kernel = GVA_KERNEL_MMA;
     if (q_len > 1 && (GQA || kernel != GVA_KERNEL_MMA)) return GVA_ERR_UNSUPPORTED;   // multi-token decode: tensor-core kernel only
-    if ((q_len > 1 || GQA) && h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;
+    if (GQA && h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;
     if (kernel == GVA_KERNEL_MMA) {
 #ifdef GVA_WITH_MMA
         int rc = h->cfg.cache_dtype == GVA_E4M3
-                     ? launch_decode_fp8(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, max_seq_len, num_splits, stream,
+                     ? launch_decode_fp8(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, q_len, max_seq_len, num_splits, stream,
                                          &h->last_num_splits, &h->last_tile, &p.rec_mult)
                  : q_len > 1 ? launch_decode_mma_multi(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, q_len, max_seq_len, num_splits,
                                                      max_blocks_balanced(h), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult)

@@ -82,8 +82,11 @@ __device__ __forceinline__ uint32_t split_hi_lo_f16(float x) {
     return (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
 }
 
-template <int DV, int DR, int TILE, int NSTAGE, int WPG, int GMAX>
-__global__ void __launch_bounds__(32 * (GMAX * WPG + 1), GMAX <= 4 ? 4 : 2)      // register caps: 4 five-warp blocks (d_v = 64) or 2 nine-warp blocks (d_v = 128) per SM
+// QL > 1 (multi-token decode, QL = 2 or 4 new tokens per sequence): as in the 16-bit kernel, the 4 heads x QL tokens of a
+// group are the MMA columns (plain f16 queries and weights, no hi/lo halves), slot s attends to seq_len - (QL - 1 - s)
+// tokens, and the partial records and outputs use QL * H pseudo-heads, slot * H + head.
+template <int DV, int DR, int TILE, int NSTAGE, int WPG, int GMAX, int QL = 1>
+__global__ void __launch_bounds__(32 * (GMAX * WPG + 1), GMAX <= 4 ? (QL == 1 ? 4 : 3) : (QL == 1 ? 2 : 1))      // register caps: 4 five-warp blocks (d_v = 64) or 2 nine-warp blocks (d_v = 128) per SM
 decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = Fp8Traits<DV, DR, TILE>;
     constexpr int CPW = T::CHUNKS / WPG;          // 16-token chunks per consumer warp and tile
@@ -93,7 +96,10 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     // dynamic shared memory is only guaranteed 16-byte aligned: round up to the swizzle atom
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int G = p.G, H = p.H;
-    const int HQ = H;
+    static_assert(QL == 1 || QL == 2 || QL == 4, "multi-token decode: 2 or 4 new tokens");
+    constexpr int NBK = QL == 1 ? 1 : QL / 2;     // N-blocks of 8 columns
+    const int ql = QL == 1 ? 1 : p.q_len;         // new tokens per sequence actually present (<= QL; the other slots stay empty)
+    const int HQ = H * ql;                        // pseudo-heads of the partial records
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int n_consumers = G * WPG;
@@ -215,6 +221,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                     m.b = b;
                     m.rec = uniform ? rg.rec_fixed : unit + b;
                     m.flags = ((f == lo || f == s_off[b]) ? 1 : 0) | ((f + 1 == hi || f + 1 >= s_off[b + 1]) ? 2 : 0);
+                    if constexpr (QL > 1) m.flags |= min(max(len - t0 - TILE, 0), ql - 1) << 8;   // tokens of the sequence beyond this tile, capped
                     s_meta[st] = m;
                     const uint32_t bar = smem_u32(&full_bar[st]);
                     const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
@@ -285,6 +292,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         const int row_pv = pi(lane & 15);                                            // x2: (piece 2i | 2i + 1), 16 tokens each
         const uint32_t off_pv = row_pv * DV, swz_pv = T::swz(row_pv);
         const int tok_lo = pi(4 * (r8 >> 1) + (r8 & 1)), tok_hi = pi(4 * (r8 >> 1) + 2 + (r8 & 1));   // this lane's two score rows
+        if constexpr (QL == 1) {
         uint32_t qf[T::KSTEPS][2];        // B fragments of Q^T as f16: column n = lane/4 = 2*head + {hi, lo}; k-step kk covers
                                           // dims 16 kk .. 16 kk + 15 in the order the converted A registers present them
         float oacc[T::MT][4];
@@ -476,6 +484,229 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 }
             }
         }
+        } else {
+            // ================= multi-token decode: QL new tokens per sequence, columns = slot * 4 + head =================
+            uint32_t qf[T::KSTEPS][NBK][2];   // B fragments of Q^T (plain f16): column n = lane / 4 of N-block nb, dims in the
+                                              // order the converted A registers present them
+            float oacc[T::MT][NBK][4];
+            float m_run[NBK][2], l_run[NBK][2];   // per column of this lane: columns 2 jh, 2 jh + 1 of every N-block
+            const float scale = p.scale_log2;
+            // the lane's B-fragment column n = lane / 4 = r8 is (slot 2 nb + n / 4, head n % 4)
+            auto load_query = [&](int b) {
+#pragma unroll
+                for (int nb = 0; nb < NBK; ++nb) {
+                    const int slot = 2 * nb + (r8 >> 2), head = r8 & 3;
+                    const bool present = slot < ql;       // an absent slot gets a zero query; its columns are masked everywhere
+                    const float *q = p.q + (((size_t)b * ql + (present ? slot : 0)) * H + g * kHeadsPerGroup + head) * T::DQ;
+#pragma unroll
+                    for (int kk = 0; kk < T::KSTEPS; ++kk) {
+                        float4 v = *reinterpret_cast<const float4 *>(q + kk * 16 + 4 * jh);
+                        if (!present) v = make_float4(0.f, 0.f, 0.f, 0.f);
+                        const __half2 w0 = __floats2half2_rn(v.x, v.y), w1 = __floats2half2_rn(v.z, v.w);
+                        qf[kk][nb][0] = *reinterpret_cast<const uint32_t *>(&w0);
+                        qf[kk][nb][1] = *reinterpret_cast<const uint32_t *>(&w1);
+                    }
+                }
+            };
+            if (early) grid_dependency_wait();
+            publish_header(p, s_off, plan, tid, n_consumers * 32);
+            int cur_b = -1;
+            if (rg.lo < rg.hi) {
+                cur_b = rg.b_first;
+                load_query(cur_b);
+            }
+#pragma unroll 1
+            for (int i = 0;; ++i) {
+                const int st = i % NSTAGE;
+                if (!mbar_wait_bounded(smem_u32(&full_bar[st]), (i / NSTAGE) & 1, s_abort)) {
+                    if (!*s_abort && lane == 0) report_error(p.dev_status, GVA_ERR_TIMEOUT, cur_b < 0 ? 0 : cur_b);
+                    *s_abort = 1;
+                    break;
+                }
+                const StageMeta meta = s_meta[st];
+                const int n_valid = meta.n_valid;
+                if (n_valid < 0) break;       // producer is done
+                const int b = meta.b;
+                if (meta.flags & 1) {         // a new segment: its own softmax state (and queries, if the sequence changed)
+                    if (b != cur_b) {
+                        cur_b = b;
+                        load_query(b);
+                    }
+#pragma unroll
+                    for (int nb = 0; nb < NBK; ++nb) {
+                        m_run[nb][0] = m_run[nb][1] = -INFINITY;
+                        l_run[nb][0] = l_run[nb][1] = 0.f;
+#pragma unroll
+                        for (int mt = 0; mt < T::MT; ++mt)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) oacc[mt][nb][e] = 0.f;
+                    }
+                }
+                unsigned char *stage = smem + (size_t)st * stage_bytes;
+                unsigned char *vt = stage + (size_t)g * T::VTILE_BYTES;
+                const int row0 = part * CPW * 16;
+                // tokens of this tile that slot s may see: n_valid + (tokens of the sequence beyond the tile, capped) - (QL - 1 - s)
+                const int reach = n_valid + ((meta.flags >> 8) & 0xff) - (ql - 1);
+                const bool ragged = n_valid < row0 + CPW * 16;
+                if (ragged) {
+                    const int z0 = max(n_valid, row0);
+                    const int n_zero_chunks = (row0 + CPW * 16 - z0) * (DV / 16);
+                    for (int c = lane; c < n_zero_chunks; c += 32)
+                        *reinterpret_cast<uint4 *>(vt + (z0 + c / (DV / 16)) * DV + (c % (DV / 16)) * 16) = make_uint4(0, 0, 0, 0);
+                    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                    __syncwarp();
+                }
+                const bool masked = reach < row0 + CPW * 16 || ql < QL;      // some slot does not see the whole share of this warp
+                const uint32_t vt_u32 = smem_u32(vt) + row0 * DV;
+                const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES) + row0 * T::KR_ROW;
+                uint32_t a_qk[DV / 32], a_pv[DV / 32];
+#pragma unroll
+                for (int pr = 0; pr < DV / 32; ++pr) {
+                    a_qk[pr] = vt_u32 + off_qk + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_qk) << 4);
+                    a_pv[pr] = vt_u32 + off_pv + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_pv) << 4);
+                }
+
+                // ---- S^T = V_tile . Q^T (+ positional part): 16 tokens per m-tile, 8 columns per N-block ----
+                float sacc[CPW][NBK][4];
+#pragma unroll
+                for (int c = 0; c < CPW; ++c) {
+#pragma unroll
+                    for (int nb = 0; nb < NBK; ++nb)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) sacc[c][nb][e] = 0.f;
+#pragma unroll
+                    for (int pr = 0; pr < DV / 32; ++pr) {
+                        uint32_t r[4];
+                        ldsm_x4(a_qk[pr] + c * 16 * DV, r);
+#pragma unroll
+                        for (int hx = 0; hx < 2; ++hx) {
+                            uint32_t a[4];
+                            e4m3x4_to_f16x2(r[2 * hx], a[0], a[2]);
+                            e4m3x4_to_f16x2(r[2 * hx + 1], a[1], a[3]);
+#pragma unroll
+                            for (int nb = 0; nb < NBK; ++nb) mma_f16(sacc[c][nb], a, qf[2 * pr + hx][nb][0], qf[2 * pr + hx][nb][1]);
+                        }
+                    }
+                    if constexpr (DR == 16) {
+                        uint32_t r[2];
+                        ldsm_x2(kr_u32 + c * 16 * T::KR_ROW + off_kr, r);
+                        uint32_t a[4];
+                        e4m3x4_to_f16x2(r[0], a[0], a[2]);
+                        e4m3x4_to_f16x2(r[1], a[1], a[3]);
+#pragma unroll
+                        for (int nb = 0; nb < NBK; ++nb) mma_f16(sacc[c][nb], a, qf[T::KSTEPS_V][nb][0], qf[T::KSTEPS_V][nb][1]);
+                    } else if constexpr (DR == 32) {
+                        uint32_t r[4];
+                        ldsm_x4(kr_u32 + c * 16 * T::KR_ROW + off_kr + ((((uint32_t)ch_ld) ^ swz_kr) << 4), r);
+#pragma unroll
+                        for (int hx = 0; hx < 2; ++hx) {
+                            uint32_t a[4];
+                            e4m3x4_to_f16x2(r[2 * hx], a[0], a[2]);
+                            e4m3x4_to_f16x2(r[2 * hx + 1], a[1], a[3]);
+#pragma unroll
+                            for (int nb = 0; nb < NBK; ++nb)
+                                mma_f16(sacc[c][nb], a, qf[T::KSTEPS_V + hx][nb][0], qf[T::KSTEPS_V + hx][nb][1]);
+                        }
+                    }
+                }
+                // ---- online softmax per column: this lane holds columns 2 jh, 2 jh + 1 of every N-block at its two token
+                //      rows of every m-tile; both columns belong to slot 2 nb + jh / 2 ----
+                float corr[NBK][2], m_use[NBK][2];
+#pragma unroll
+                for (int nb = 0; nb < NBK; ++nb) {
+                    const int slot_l = 2 * nb + (jh >> 1);
+                    const int lim = slot_l < ql ? reach + slot_l : 0;     // tokens of the tile this slot sees (an absent slot: none)
+                    float tmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+                    for (int c = 0; c < CPW; ++c) {
+                        if (masked) {
+                            if (row0 + c * 16 + tok_lo >= lim) sacc[c][nb][0] = sacc[c][nb][1] = -INFINITY;
+                            if (row0 + c * 16 + tok_hi >= lim) sacc[c][nb][2] = sacc[c][nb][3] = -INFINITY;
+                        }
+                        tmax[0] = fmaxf(tmax[0], fmaxf(sacc[c][nb][0], sacc[c][nb][2]));
+                        tmax[1] = fmaxf(tmax[1], fmaxf(sacc[c][nb][1], sacc[c][nb][3]));
+                    }
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        float t = tmax[e];
+                        t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 4));
+                        t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 8));
+                        t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 16));
+                        const float m_new = fmaxf(m_run[nb][e], t * scale);
+                        m_use[nb][e] = (m_new != -INFINITY) ? m_new : 0.f;    // keeps (-inf) - (-inf) out of the exponent
+                        corr[nb][e] = fast_exp2(m_run[nb][e] - m_use[nb][e]);
+                        m_run[nb][e] = m_new;
+                        l_run[nb][e] *= corr[nb][e];
+                    }
+#pragma unroll
+                    for (int mt = 0; mt < T::MT; ++mt) {
+                        oacc[mt][nb][0] *= corr[nb][0];
+                        oacc[mt][nb][1] *= corr[nb][1];
+                        oacc[mt][nb][2] *= corr[nb][0];
+                        oacc[mt][nb][3] *= corr[nb][1];
+                    }
+                }
+                // ---- O^T += V_tile^T . P^T ----
+#pragma unroll
+                for (int c = 0; c < CPW; ++c) {
+                    uint32_t pb[NBK][2];
+#pragma unroll
+                    for (int nb = 0; nb < NBK; ++nb) {
+                        const float p00 = fast_exp2(fmaf(sacc[c][nb][0], scale, -m_use[nb][0]));   // low row,  column 2 jh
+                        const float p01 = fast_exp2(fmaf(sacc[c][nb][1], scale, -m_use[nb][1]));   // low row,  column 2 jh + 1
+                        const float p10 = fast_exp2(fmaf(sacc[c][nb][2], scale, -m_use[nb][0]));   // high row, column 2 jh
+                        const float p11 = fast_exp2(fmaf(sacc[c][nb][3], scale, -m_use[nb][1]));
+                        l_run[nb][0] += p00 + p10;
+                        l_run[nb][1] += p01 + p11;
+                        const __half2 w0 = __floats2half2_rn(p00, p01), w1 = __floats2half2_rn(p10, p11);
+                        pb[nb][0] = movmatrix_trans(*reinterpret_cast<const uint32_t *>(&w0));
+                        pb[nb][1] = movmatrix_trans(*reinterpret_cast<const uint32_t *>(&w1));
+                    }
+#pragma unroll
+                    for (int pr = 0; pr < DV / 32; ++pr) {
+                        uint32_t r[4];
+                        ldsm_b8_x2_trans(a_pv[pr] + c * 16 * DV, r);
+#pragma unroll
+                        for (int hx = 0; hx < 2; ++hx) {
+                            uint32_t a[4];
+                            e4m3x4_to_f16x2(r[2 * hx], a[0], a[2]);
+                            e4m3x4_to_f16x2(r[2 * hx + 1], a[1], a[3]);
+#pragma unroll
+                            for (int nb = 0; nb < NBK; ++nb) mma_f16(oacc[2 * pr + hx][nb], a, pb[nb][0], pb[nb][1]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&empty_bar[st]));
+
+                // ---- segment end: one partial per (unit, sequence, part) and pseudo-head slot * H + head ----
+                if (meta.flags & 2) {
+                    const int rec = meta.rec * WPG + part;
+#pragma unroll
+                    for (int nb = 0; nb < NBK; ++nb)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            float l = l_run[nb][e];
+                            l += __shfl_xor_sync(0xffffffffu, l, 4);
+                            l += __shfl_xor_sync(0xffffffffu, l, 8);
+                            l += __shfl_xor_sync(0xffffffffu, l, 16);
+                            const int col = 2 * jh + e;                       // column of N-block nb: slot 2 nb + col / 4, head col % 4
+                            if (2 * nb + (col >> 2) >= ql) continue;           // (uniform over the lanes that reduce together)
+                            const size_t rh = (size_t)rec * HQ + (size_t)(2 * nb + (col >> 2)) * H + g * kHeadsPerGroup + (col & 3);
+                            float *o_dst = p.rec_o + rh * DV;
+#pragma unroll
+                            for (int mt = 0; mt < T::MT; ++mt) {
+                                o_dst[mt * 16 + r8] = oacc[mt][nb][e];
+                                o_dst[mt * 16 + r8 + 8] = oacc[mt][nb][2 + e];
+                            }
+                            if (r8 == 0) {
+                                p.rec_ml[rh * 2] = m_run[nb][e];
+                                p.rec_ml[rh * 2 + 1] = l;
+                            }
+                        }
+                }
+            }
+        }
     }
     // keep shared memory alive until every warp (and every copy in flight) is done
     __syncthreads();
@@ -502,7 +733,7 @@ inline bool encode_map_u8(const MmaHostState &st, CUtensorMap *map, const void *
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int DV, int DR, int TILE>
+template <int DV, int DR, int TILE, int QL = 1>
 int launch_fp8_t(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
                  int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out) {
     using T = Fp8Traits<DV, DR, TILE>;
@@ -512,7 +743,7 @@ int launch_fp8_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
     if (G * wpg + 1 > 9) return GVA_ERR_UNSUPPORTED;
     const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
-    auto fn = G <= 4 ? decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 4> : decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 8>;
+    auto fn = G <= 4 ? decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 4, QL> : decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 8, QL>;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
     CUtensorMap tm_v, tm_k;
     if (!encode_map_u8(st, &tm_v, p.v_pool, DV, (uint64_t)p.num_pages * G * p.P, DV, TILE,
@@ -530,7 +761,10 @@ int launch_fp8_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
         grid = B * num_splits;
     } else {
         const long long tiles_ub = (long long)B * ((max_seq_len + TILE - 1) / TILE);
-        const long long want = (long long)fp8_blocks_per_sm(cfg) * sm_count;      // what the workspace is sized for
+        // what the workspace is sized for; the multi-token variants hold more registers: three five-warp blocks or one
+        // nine-warp block per SM
+        const int per_sm = QL == 1 ? fp8_blocks_per_sm(cfg) : (G > 4 ? 1 : 3);
+        const long long want = (long long)per_sm * sm_count;
         grid = (int)(tiles_ub < want ? (tiles_ub < 1 ? 1 : tiles_ub) : want);
     }
     DecodeParams pp = p;
@@ -544,12 +778,24 @@ int launch_fp8_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
 }
 
 inline int launch_decode_fp8(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
-                             int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out, int *tile_out,
+                             int q_len, int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out, int *tile_out,
                              int *rec_mult_out) {
     if (!fp8_supported(cfg)) return GVA_ERR_UNSUPPORTED;
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
     *tile_out = fp8_tile(cfg);
     *rec_mult_out = GVA_FP8_WPG;
+    if (q_len > 1) {       // multi-token decode: 2..4 new tokens per sequence, caches with a positional slice
+        if (q_len > 4 || cfg.d_r == 0) return GVA_ERR_UNSUPPORTED;
+#define GVA_FP8_MULTI(DV_, DR_, TILE_, QL_) \
+    return launch_fp8_t<DV_, DR_, TILE_, QL_>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, stream, n_blocks_out)
+        if (cfg.d_v == 64) {
+            if (q_len == 2) GVA_FP8_MULTI(64, 16, 64, 2);
+            GVA_FP8_MULTI(64, 16, 64, 4);
+        }
+        if (q_len == 2) GVA_FP8_MULTI(128, 32, 32, 2);
+        GVA_FP8_MULTI(128, 32, 32, 4);
+#undef GVA_FP8_MULTI
+    }
     if (cfg.d_v == 64)
         return cfg.d_r == 16 ? launch_fp8_t<64, 16, 64>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, stream, n_blocks_out)
                              : launch_fp8_t<64, 0, 64>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, stream, n_blocks_out);

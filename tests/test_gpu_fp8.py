@@ -228,7 +228,7 @@ def test_what_the_8_bit_cache_does_not_cover():
     pd = harness.upload_prefill(pc)
     try:
         pd.absorb()
-        for call in (pd.prefill, lambda: pd.decode_multi(num_splits=0), lambda: pd.decode_tokens(4)):
+        for call in (pd.prefill, lambda: pd.decode_multi(num_splits=0)):
             with pytest.raises(gb.GvaError) as e:
                 call()
             assert e.value.status == gb.GVA_ERR_UNSUPPORTED
@@ -284,3 +284,51 @@ def test_full_size_ragged_wide_heads_sampled():
         assert np.max(np.abs(o[sample] - ref[sample])) <= U().TOL_TIGHT_MAXABS
     finally:
         dc.close()
+
+
+@pytest.mark.parametrize("q_len", [2, 3, 4])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+@pytest.mark.parametrize("num_splits", [0, 3])
+def test_decode_tokens_matches_oracle(q_len, shape, num_splits):
+    # exactly q_len new tokens per sequence over contexts around tile and page boundaries (a context of 0 too: the first
+    # new token then sees only itself), poisoned unused slots; the oracle is the chunked-prefill oracle over the same
+    # codes.  Queries and weights enter the MMAs as single f16 values (relative 2^-12): tolerances of the 16-bit
+    # multi-token kernels
+    ctx = [0, 1, 61, 62, 63, 64, 65, 127, 128, 700, 2047, 5000]
+    pc = wl.make_prefill_case("tok8", shape, ctx, [q_len] * len(ctx), page_size=64, cache_dtype="fp8", seed=820 + q_len,
+                              poison_unused=True)
+    ref_out, ref_lse = orc.prefill_case(pc)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        out, lse = pd.decode_tokens(q_len, num_splits=num_splits)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out[:pc.n_q].cpu().numpy().astype(np.float64); l = lse[:pc.n_q].cpu().numpy().astype(np.float64)
+        assert np.isfinite(o).all() and np.isfinite(l).all()
+        assert np.max(np.abs(o - ref_out)) <= 5e-3, np.max(np.abs(o - ref_out))
+        assert U().rel_l2(o, ref_out) <= 2e-3
+        assert np.max(np.abs(l - ref_lse)) <= 5e-3
+    finally:
+        pd.close()
+
+
+def test_append_then_decode_tokens_follows_algorithm_order():
+    # Algorithm 1 for three new tokens at once over the 8-bit cache: absorb, append all three (bit-exact codes), attend
+    q_len = 3
+    pc = wl.make_prefill_case("atok8", wl.SHAPE_A, [63, 640, 0, 4095], [q_len] * 4, page_size=64, cache_dtype="fp8", seed=841)
+    c = pc.cache
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        pd.append()
+        out, _ = pd.decode_tokens(q_len)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        v, k = pd.dc.pools_to_host()
+        assert orc.append_chunk(c.v_pool, c.kr_pool, c.block_table, pc.v_new, pc.kr_new, pc.cu_q, pc.ctx_lens) == 0
+        assert np.array_equal(v, c.v_pool) and np.array_equal(k, c.kr_pool)
+        ref_out, _ = orc.prefill_case(pc)
+        assert np.max(np.abs(out[:pc.n_q].cpu().numpy().astype(np.float64) - ref_out)) <= 5e-3
+    finally:
+        pd.close()
