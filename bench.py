@@ -556,13 +556,13 @@ def measure_prefill(rank, local_rank, dist, args, torch, gb, harness, B=8, T=819
     return res
 
 
-def measure_multi(rank, local_rank, dist, args, torch, gb, harness, q_len=4, on_decode_kernel=False):
+def measure_multi(rank, local_rank, dist, args, torch, gb, harness, q_len=4, on_decode_kernel=False, cache_dtype="bf16"):
     """Multi-token decode on the headline workload's shape: q_len new tokens per sequence over the long cached context
     (gva_decode_multi: the tcgen05 kernel with split-KV + merge); the cache stream is the same as cfg2's."""
     from paper_2609_13285_b200 import multirank, workloads as wl
     dev = torch.device("cuda", local_rank)
     B, T = 32, 32768
-    pc = wl.make_prefill_case("multi", wl.SHAPE_A, [T - q_len] * B, [q_len] * B, page_size=64,
+    pc = wl.make_prefill_case("multi", wl.SHAPE_A, [T - q_len] * B, [q_len] * B, page_size=64, cache_dtype=cache_dtype,
                               seed=wl.MASTER_SEED + 7300 + 7919 * rank)
     pd = harness.upload_prefill(pc, device=dev)
     pd.absorb()
@@ -599,7 +599,7 @@ def measure_multi(rank, local_rank, dist, args, torch, gb, harness, q_len=4, on_
     peak = load_peaks()[0]
     gbps = c.cache_bytes() / (ms * 1e-3) / 1e9
     res = {"workload": f"multi-token decode, cfg2 shapes: {q_len} new tokens per sequence over T = {T} cached tokens, B = {B}, "
-                       "bf16 paged cache (two pool copies alternate: every call streams from HBM); "
+                       + ("bf16" if cache_dtype == "bf16" else "8-bit e4m3") + " paged cache (two pool copies alternate: every call streams from HBM); "
                        + ("gva_decode_tokens (split-KV mma.sync decode kernel)" if on_decode_kernel else
                           "gva_decode_multi (tcgen05 kernel with split-KV)"),
            "q_len": q_len, "ms_per_call": ms, "cache_read_GBps": gbps, "frac_of_measured_peak": gbps / peak,
@@ -646,13 +646,13 @@ def main() -> None:
     kernel = {"auto": gb.GVA_KERNEL_AUTO, "fma": gb.GVA_KERNEL_FMA, "mma": gb.GVA_KERNEL_MMA}[args.kernel]
 
     name = args.workload
-    if name in ("prefill", "prefill-ncu", "prefill-wide", "layer", "multi", "multi-q1", "multi-q8", "multi-q32", "tokens-q2", "tokens-q4"):      # side workloads on their own (small runs for profiler captures)
+    if name in ("prefill", "prefill-ncu", "prefill-wide", "layer", "multi", "multi-q1", "multi-q8", "multi-q32", "tokens-q2", "tokens-q4", "tokens-q2-fp8", "tokens-q4-fp8"):      # side workloads on their own (small runs for profiler captures)
         if rank == 0:
             if name == "layer":
                 res = measure_layer(rank, local_rank, None, args, kernel, torch, gb, harness)
             elif name.startswith("tokens"):
-                res = measure_multi(rank, local_rank, None, args, torch, gb, harness, q_len=int(name.split("-q")[1]),
-                                    on_decode_kernel=True)
+                res = measure_multi(rank, local_rank, None, args, torch, gb, harness, q_len=int(name.split("-q")[1].split("-")[0]),
+                                    on_decode_kernel=True, cache_dtype="fp8" if name.endswith("-fp8") else "bf16")
             elif name.startswith("multi"):
                 res = measure_multi(rank, local_rank, None, args, torch, gb, harness,
                                     q_len=int(name.split("-q")[1]) if "-q" in name else 4)
@@ -698,6 +698,8 @@ def main() -> None:
         others["decode_multi_cfg2_q4"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=4)
         others["decode_tokens_cfg2_q2"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=2, on_decode_kernel=True)
         others["decode_tokens_cfg2_q4"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=4, on_decode_kernel=True)
+        others["decode_tokens_cfg2_q4_fp8"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=4,
+                                                            on_decode_kernel=True, cache_dtype="fp8")
         others["prefill"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness)
         others["prefill_wide"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness, B=4, T=8192, wide=True)
 
