@@ -20,6 +20,9 @@
 #ifndef GVA_FP8_WPG
 #define GVA_FP8_WPG 1
 #endif
+// resident five-warp blocks per SM of the multi-token variants (measured on the long-context workload: 2 tokens
+// 79 / 79 / 68 us with 2 / 3 / 4 blocks, 4 tokens 98 / 128 / 142 us: the 4-token variant needs its 168 registers)
+#define GVA_FP8_QL_BLOCKS(QL_) ((QL_) == 2 ? 4 : 2)
 #ifndef GVA_FP8_BLOCKS_PER_SM
 #define GVA_FP8_BLOCKS_PER_SM 4
 #endif
@@ -86,7 +89,7 @@ __device__ __forceinline__ uint32_t split_hi_lo_f16(float x) {
 // group are the MMA columns (plain f16 queries and weights, no hi/lo halves), slot s attends to seq_len - (QL - 1 - s)
 // tokens, and the partial records and outputs use QL * H pseudo-heads, slot * H + head.
 template <int DV, int DR, int TILE, int NSTAGE, int WPG, int GMAX, int QL = 1>
-__global__ void __launch_bounds__(32 * (GMAX * WPG + 1), GMAX <= 4 ? (QL == 1 ? 4 : 3) : (QL == 1 ? 2 : 1))      // register caps: 4 five-warp blocks (d_v = 64) or 2 nine-warp blocks (d_v = 128) per SM
+__global__ void __launch_bounds__(32 * (GMAX * WPG + 1), GMAX <= 4 ? (QL == 1 ? 4 : GVA_FP8_QL_BLOCKS(QL)) : (QL == 1 ? 2 : 1))      // register caps: 4 five-warp blocks (d_v = 64) or 2 nine-warp blocks (d_v = 128) per SM
 decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = Fp8Traits<DV, DR, TILE>;
     constexpr int CPW = T::CHUNKS / WPG;          // 16-token chunks per consumer warp and tile
@@ -761,9 +764,9 @@ int launch_fp8_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
         grid = B * num_splits;
     } else {
         const long long tiles_ub = (long long)B * ((max_seq_len + TILE - 1) / TILE);
-        // what the workspace is sized for; the multi-token variants hold more registers: three five-warp blocks or one
-        // nine-warp block per SM
-        const int per_sm = QL == 1 ? fp8_blocks_per_sm(cfg) : (G > 4 ? 1 : 3);
+        // what the workspace is sized for; the multi-token variants: four (2 tokens) or two (4 tokens) five-warp blocks,
+        // or one nine-warp block per SM
+        const int per_sm = QL == 1 ? fp8_blocks_per_sm(cfg) : (G > 4 ? 1 : GVA_FP8_QL_BLOCKS(QL));
         const long long want = (long long)per_sm * sm_count;
         grid = (int)(tiles_ub < want ? (tiles_ub < 1 ? 1 : tiles_ub) : want);
     }
