@@ -89,7 +89,7 @@ __device__ __forceinline__ uint32_t split_hi_lo_f16(float x) {
 // group are the MMA columns (plain f16 queries and weights, no hi/lo halves), slot s attends to seq_len - (QL - 1 - s)
 // tokens, and the partial records and outputs use QL * H pseudo-heads, slot * H + head.
 template <int DV, int DR, int TILE, int NSTAGE, int WPG, int GMAX, int QL = 1>
-__global__ void __launch_bounds__(32 * (GMAX * WPG + 1), GMAX <= 4 ? (QL == 1 ? 4 : GVA_FP8_QL_BLOCKS(QL)) : (QL == 1 ? 2 : 1))      // register caps: 4 five-warp blocks (d_v = 64) or 2 nine-warp blocks (d_v = 128) per SM
+__global__ void __launch_bounds__(32 * (GMAX * WPG + 1), GMAX <= 4 ? (QL == 1 ? GVA_FP8_BLOCKS_PER_SM : GVA_FP8_QL_BLOCKS(QL)) : (QL == 1 ? 2 : 1))      // register caps: 4 five-warp blocks (d_v = 64) or 2 nine-warp blocks (d_v = 128) per SM
 decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = Fp8Traits<DV, DR, TILE>;
     constexpr int CPW = T::CHUNKS / WPG;          // 16-token chunks per consumer warp and tile
