@@ -436,19 +436,20 @@ int gva_append_chunk(gva_handle *h, const gva_cache *cache, const float *v_new, 
     const gva_config &c = h->cfg;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (c.G * c.d_v > kAppendMaxPerThread * 128) return GVA_ERR_UNSUPPORTED;
+    const int vec4 = (aligned(v_new, 16) && (c.G * c.d_v) % 4 == 0) ? 1 : 0;
     cudaError_t ce;
     if (c.cache_dtype == GVA_E4M3)
         ce = launch_pdl(append_chunk_kernel<uint8_t>, dim3((n_q + kAppendChunkRows - 1) / kAppendChunkRows), dim3(128), 0, s, static_cast<uint8_t *>(cache->v_pool),
                         static_cast<uint8_t *>(cache->kr_pool), cache->block_table, v_new, kr_new, cu_q, ctx_lens, B, c.G,
-                        c.d_v, c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+                        c.d_v, c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope, vec4);
     else if (c.cache_dtype == GVA_BF16)
         ce = launch_pdl(append_chunk_kernel<__nv_bfloat16>, dim3((n_q + kAppendChunkRows - 1) / kAppendChunkRows), dim3(128), 0, s, static_cast<__nv_bfloat16 *>(cache->v_pool),
                         static_cast<__nv_bfloat16 *>(cache->kr_pool), cache->block_table, v_new, kr_new, cu_q, ctx_lens, B, c.G,
-                        c.d_v, c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+                        c.d_v, c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope, vec4);
     else
         ce = launch_pdl(append_chunk_kernel<float>, dim3((n_q + kAppendChunkRows - 1) / kAppendChunkRows), dim3(128), 0, s, static_cast<float *>(cache->v_pool),
                         static_cast<float *>(cache->kr_pool), cache->block_table, v_new, kr_new, cu_q, ctx_lens, B, c.G, c.d_v,
-                        c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope);
+                        c.d_r, c.page_size, cache->num_pages, cache->max_pages_per_seq, dev_status, h->rope, vec4);
     if (ce != cudaSuccess) {
         (void)cudaGetLastError();
         return GVA_ERR_CUDA;

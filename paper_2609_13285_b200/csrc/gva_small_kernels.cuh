@@ -411,7 +411,7 @@ __global__ void __launch_bounds__(128)
 append_chunk_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int32_t *__restrict__ block_table,
                     const float *__restrict__ v_new, const float *__restrict__ kr_new, const int32_t *__restrict__ cu_q,
                     const int32_t *__restrict__ ctx_lens, int B, int G, int d_v, int d_r, int P, int num_pages, int max_pages,
-                    int32_t *dev_status, RopeTable rope) {
+                    int32_t *dev_status, RopeTable rope, int vec4) {
     static_assert(kAppendChunkRows * kMaxRopePairs == 128, "16 threads per row");
     grid_dependency_launch();
     __shared__ long long s_page[kAppendChunkRows];      // -1: the row is not written
@@ -470,16 +470,61 @@ append_chunk_kernel(CT *__restrict__ v_pool, CT *__restrict__ kr_pool, const int
     const int n_v = G * d_v;
     const int rows = min(kAppendChunkRows, total - (int)blockIdx.x * kAppendChunkRows);
     const float *src = v_new + (size_t)blockIdx.x * kAppendChunkRows * n_v;
-    for (int e = threadIdx.x; e < rows * n_v; e += 128) {
-        const int r = e / n_v, i = e % n_v;
+    // element e = r * n_v + i walks the rows in steps of 128 without a division (d_v is a power of two: 64 or 128)
+    const int sh = 31 - __clz(d_v);
+    if (vec4) {     // v_new is 16-byte aligned: four elements per thread and pass
+        const int n4 = n_v >> 2;
+        int r = 0, i = threadIdx.x;
+        while (i >= n4) {
+            i -= n4;
+            ++r;
+        }
+        while (r < rows) {
+            const long long page = s_page[r];
+            if (page >= 0) {
+                const int g = (4 * i) >> sh, d = (4 * i) & (d_v - 1);
+                const size_t dst = (((size_t)page * G + g) * P + s_slot[r]) * d_v + d;
+                const float4 x = *reinterpret_cast<const float4 *>(src + (size_t)r * n_v + 4 * i);
+                if constexpr (sizeof(CT) == 1) {
+                    *reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(v_pool) + dst) =
+                        (uint32_t)float_to_e4m3_bits(x.x) | ((uint32_t)float_to_e4m3_bits(x.y) << 8) |
+                        ((uint32_t)float_to_e4m3_bits(x.z) << 16) | ((uint32_t)float_to_e4m3_bits(x.w) << 24);
+                } else if constexpr (sizeof(CT) == 2) {
+                    *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(v_pool) + dst) =
+                        make_uint2((uint32_t)float_to_bf16_bits(x.x) | ((uint32_t)float_to_bf16_bits(x.y) << 16),
+                                   (uint32_t)float_to_bf16_bits(x.z) | ((uint32_t)float_to_bf16_bits(x.w) << 16));
+                } else {
+                    *reinterpret_cast<float4 *>(reinterpret_cast<float *>(v_pool) + dst) = x;
+                }
+            }
+            i += 128;
+            while (i >= n4) {
+                i -= n4;
+                ++r;
+            }
+        }
+        return;
+    }
+    int r = 0, i = threadIdx.x;
+    while (i >= n_v) {
+        i -= n_v;
+        ++r;
+    }
+    while (r < rows) {
         const long long page = s_page[r];
-        if (page < 0) continue;
-        const int g = i / d_v, d = i % d_v;
-        const size_t dst = (((size_t)page * G + g) * P + s_slot[r]) * d_v + d;
-        const float x = src[e];
-        if constexpr (sizeof(CT) == 1) reinterpret_cast<uint8_t *>(v_pool)[dst] = float_to_e4m3_bits(x);
-        else if constexpr (sizeof(CT) == 2) reinterpret_cast<uint16_t *>(v_pool)[dst] = float_to_bf16_bits(x);
-        else reinterpret_cast<float *>(v_pool)[dst] = x;
+        if (page >= 0) {
+            const int g = i >> sh, d = i & (d_v - 1);
+            const size_t dst = (((size_t)page * G + g) * P + s_slot[r]) * d_v + d;
+            const float x = src[(size_t)r * n_v + i];
+            if constexpr (sizeof(CT) == 1) reinterpret_cast<uint8_t *>(v_pool)[dst] = float_to_e4m3_bits(x);
+            else if constexpr (sizeof(CT) == 2) reinterpret_cast<uint16_t *>(v_pool)[dst] = float_to_bf16_bits(x);
+            else reinterpret_cast<float *>(v_pool)[dst] = x;
+        }
+        i += 128;
+        while (i >= n_v) {
+            i -= n_v;
+            ++r;
+        }
     }
 }
 

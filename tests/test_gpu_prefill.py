@@ -130,6 +130,29 @@ def test_append_chunk_is_bit_exact(dtype):
     assert np.array_equal(v.view(np.uint8), v_ref.view(np.uint8)) and np.array_equal(k.view(np.uint8), k_ref.view(np.uint8))
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32", "fp8"])
+def test_append_chunk_from_rows_that_are_only_4_byte_aligned(dtype):
+    # the copy loop takes four elements per thread when the new rows are 16-byte aligned and one otherwise: same bits
+    pc = wl.make_prefill_case("apu", wl.SHAPE_A, [5, 63, 500], [67, 2, 77], page_size=64, cache_dtype=dtype, seed=531)
+    c = pc.cache
+    v_ref, k_ref = c.v_pool.copy(), c.kr_pool.copy()
+    assert orc.append_chunk(v_ref, k_ref, c.block_table, pc.v_new, pc.kr_new, pc.cu_q, pc.ctx_lens) == 0
+    pd = harness.upload_prefill(pc)
+    try:
+        buf = torch.empty(pd.v_new.numel() + 1, dtype=torch.float32, device=pd.v_new.device)
+        shifted = buf[1:].view(pd.v_new.shape)
+        shifted.copy_(pd.v_new)
+        assert shifted.data_ptr() % 16 == 4
+        pd.v_new = shifted
+        pd.append()
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        v, k = pd.dc.pools_to_host()
+    finally:
+        pd.close()
+    assert np.array_equal(v.view(np.uint8), v_ref.view(np.uint8)) and np.array_equal(k.view(np.uint8), k_ref.view(np.uint8))
+
+
 def test_append_then_prefill_follows_algorithm_order():
     # the chunk's own rows come from the append, not from the generator
     pc = wl.make_prefill_case("apf", wl.SHAPE_A, [40, 0], [90, 129], page_size=64, seed=507)
