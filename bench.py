@@ -77,8 +77,6 @@ def make_workload(name: str, rank: int):
                             seed=wl.MASTER_SEED + 2000 + shift)
     if name == "cfg2-ncu":   # profiler-sized: 143 MB of cache (> L2), same shapes and paging as cfg2
         return wl.config2(seed=wl.MASTER_SEED + 2000 + shift, B=16, T=16384)
-    if name == "cfg2-small":
-        return wl.config2(seed=wl.MASTER_SEED + 2000 + shift, B=8, T=8192)
     raise SystemExit(f"unknown workload {name}")
 
 

@@ -148,7 +148,8 @@ static int64_t page_of(const int32_t *block_table, int max_pages, int b, int j) 
 
 /* ---- append: write the new token's G value rows and its rotated positional key -----------------
  * v_pool [num_pages][G][P][d_v], kr_pool [num_pages][P][d_r].  v_new [B][G][d_v], kr_new [B][d_r]
- * (unrotated), pos [B].  Returns 0, or 1+b for the first sequence whose page id is out of range. */
+ * (unrotated), pos [B].  Returns 0, or 1+b for the first sequence whose position lies outside its block table or whose page id is out of range
+ * (that sequence and the ones after it are not written). */
 int oracle_append(void *v_pool, void *kr_pool, int dtype, const int32_t *block_table, int num_pages,
                   int max_pages, int P, int G, int d_v, int d_r, double base, const double *v_new,
                   const double *kr_new, const int32_t *pos, int B) {
@@ -156,9 +157,10 @@ int oracle_append(void *v_pool, void *kr_pool, int dtype, const int32_t *block_t
     int rc = 0;
     for (int b = 0; b < B && !rc; ++b) {
         int t = pos[b];
+        if (t < 0 || t / P >= max_pages) { rc = 1 + b; break; }   /* position outside the block table: no lookup */
         int64_t page = page_of(block_table, max_pages, b, t / P);
         int slot = t % P;
-        if (t < 0 || t / P >= max_pages || page < 0 || page >= num_pages) { rc = 1 + b; break; }
+        if (page < 0 || page >= num_pages) { rc = 1 + b; break; }
         for (int g = 0; g < G; ++g)
             for (int i = 0; i < d_v; ++i)
                 store_elem(v_pool, dtype, ((page * G + g) * P + slot) * d_v + i,
@@ -366,7 +368,7 @@ void oracle_prefill(const void *v_pool, const void *kr_pool, int dtype, const in
 
 /* Append of a chunk: token i of sequence b (i < cu_q[b+1]-cu_q[b]) is written at position ctx_lens[b] + i,
  * exactly as oracle_append writes one token (Algorithm 1's append lines, once per new token).
- * v_new [n_q][G][d_v], kr_new [n_q][d_r] unrotated.  Returns 0, or 1+b for the first bad page. */
+ * v_new [n_q][G][d_v], kr_new [n_q][d_r] unrotated.  Returns 0, or 1+b for the first sequence with a position outside its block table or a bad page id. */
 int oracle_append_chunk(void *v_pool, void *kr_pool, int dtype, const int32_t *block_table, int num_pages,
                         int max_pages, int P, int G, int d_v, int d_r, double base, const double *v_new,
                         const double *kr_new, const int32_t *cu_q, const int32_t *ctx_lens, int B) {
@@ -376,9 +378,10 @@ int oracle_append_chunk(void *v_pool, void *kr_pool, int dtype, const int32_t *b
         for (int i = 0; i < cu_q[b + 1] - cu_q[b]; ++i) {
             int64_t n = cu_q[b] + i;
             int t = ctx_lens[b] + i;
+            if (t < 0 || t / P >= max_pages) { rc = 1 + b; break; }   /* position outside the block table: no lookup */
             int64_t page = page_of(block_table, max_pages, b, t / P);
             int slot = t % P;
-            if (t < 0 || t / P >= max_pages || page < 0 || page >= num_pages) { rc = 1 + b; break; }
+            if (page < 0 || page >= num_pages) { rc = 1 + b; break; }
             for (int g = 0; g < G; ++g)
                 for (int d = 0; d < d_v; ++d)
                     store_elem(v_pool, dtype, ((page * G + g) * P + slot) * d_v + d, v_new[(n * G + g) * d_v + d]);

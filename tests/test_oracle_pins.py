@@ -214,12 +214,18 @@ def test_dominant_score_selects_row_and_constant_shift():
     s = wl.HeadShape(H=2, G=1, d_v=4, d_c=4, d_r=2)
     c = wl.make_case("dom", s, [8], page_size=8, cache_dtype="f32", paged=False, seed=6)
     q_abs = np.zeros((1, 2, 6))
+    # make row 5 twice as long as the longest other row: with q along it, Cauchy-Schwarz bounds every other
+    # score by half of row 5's, so the gap is guaranteed rather than hoped for
+    norms = np.linalg.norm(wl.pool_to_f64(c.v_pool)[0, 0, :8], axis=1)
+    c.v_pool[0, 0, 5] *= np.float32(2.0 * np.delete(norms, 5).max() / norms[5])
     v5 = wl.pool_to_f64(c.v_pool)[0, 0, 5]
     q_abs[0, 0, :4] = 400.0 * v5 / np.linalg.norm(v5)          # hugely aligned with token 5
     out, _ = orc.decode_case(c, q_abs)
-    scores = wl.pool_to_f64(c.v_pool)[0, 0] @ q_abs[0, 0, :4]
-    if np.argmax(scores) == 5 and np.sort(scores)[-1] - np.sort(scores)[-2] > 200:
-        assert np.allclose(out[0, 0], v5, atol=1e-12)
+    scores = (wl.pool_to_f64(c.v_pool)[0, 0, :8] @ q_abs[0, 0, :4]) / math.sqrt(s.d_c + s.d_r)
+    assert np.argmax(scores) == 5 and np.sort(scores)[-1] - np.sort(scores)[-2] > 40     # exp(-40) ~ 4e-18
+    assert np.allclose(out[0, 0], v5, atol=1e-12)
+    # the other head of the group has a zero query and must still see the mean of the (changed) rows
+    assert np.allclose(out[0, 1], wl.pool_to_f64(c.v_pool)[0, 0, :8].mean(0), atol=1e-13)
     # adding a constant to every score (via a constant k_r channel) leaves out unchanged, shifts lse
     c.kr_pool[:] = 0
     c.kr_pool[..., 0] = 1.0
@@ -430,6 +436,36 @@ def test_append_reports_bad_page():
     c = small_case()
     c.block_table[1, 0] = c.num_pages + 3
     assert orc.append_case(c) == 2
+
+
+@pytest.mark.parametrize("bad", [-1, -64, "first_beyond", "far_beyond"])
+def test_append_refuses_positions_outside_the_block_table(bad):
+    # a position that is negative or at/after max_pages * P has no block-table entry: the sequence is reported
+    # (1 + b), nothing of it or of later sequences is written, and earlier sequences are written as usual
+    c = small_case()
+    cap = c.max_pages_per_seq * c.page_size
+    t_bad = {"first_beyond": cap, "far_beyond": cap + 5 * c.page_size + 3}.get(bad, bad)
+    good = small_case()
+    assert orc.append_case(good) == 0
+    v0, k0 = c.v_pool.copy(), c.kr_pool.copy()
+    c.append_pos[1] = t_bad
+    assert orc.append_case(c) == 2
+    t0 = int(c.append_pos[0])
+    page, slot = c.page_of(0, t0 // c.page_size), t0 % c.page_size
+    mask_v = np.zeros(c.v_pool.shape[:3], dtype=bool); mask_v[page, :, slot] = True
+    mask_k = np.zeros(c.kr_pool.shape[:2], dtype=bool); mask_k[page, slot] = True
+    assert np.array_equal(c.v_pool[mask_v], good.v_pool[mask_v]) and np.array_equal(c.kr_pool[mask_k], good.kr_pool[mask_k])
+    assert np.array_equal(c.v_pool[~mask_v], v0[~mask_v]) and np.array_equal(c.kr_pool[~mask_k], k0[~mask_k])
+    # the chunked form takes the same decision (context length such that the chunk's first token is the bad position)
+    pc = small_prefill("bf16", paged=True, seed=36)
+    pcap = pc.cache.max_pages_per_seq * pc.cache.page_size
+    ctx = np.array(pc.ctx_lens, dtype=np.int32)
+    ctx[0] = {"first_beyond": pcap, "far_beyond": pcap + 5 * pc.cache.page_size + 3}.get(bad, bad)
+    v1, k1 = pc.cache.v_pool.copy(), pc.cache.kr_pool.copy()
+    q0 = int(pc.cu_q[1] - pc.cu_q[0])
+    assert q0 > 0
+    assert orc.append_chunk(v1, k1, pc.cache.block_table, pc.v_new, pc.kr_new, pc.cu_q, ctx) == 1
+    assert np.array_equal(v1, pc.cache.v_pool) and np.array_equal(k1, pc.cache.kr_pool)
 
 
 # ---------------------------------------------------------------- GQA companion
