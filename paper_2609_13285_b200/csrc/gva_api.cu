@@ -24,50 +24,93 @@ struct gva_handle {
     int device;
     int sm_count;
     int smem_optin;          // max dynamic shared memory per block
+    int smem_per_sm;         // shared memory of one SM
     float scale;             // softmax scale of gva_decode
     RopeTable rope;
     int last_num_splits;
     int last_kernel;
     int last_tile;
-    int32_t *ticket;         // this handle's dynamic-unit ticket (device, inside the library image)
-    int ticket_slot;
+    int epoch;               // number of the last decode call on this handle (see kSync* in gva_common.cuh)
+    int32_t *sync_base;      // device address of the sync arena on this handle's device
+    int sync_off, sync_cap;  // the region of the arena in use (words)
+    int n_regions;           // regions reserved so far (the earlier, smaller ones are kept until gva_destroy)
+    int region_off[24], region_cap[24];
 #ifdef GVA_WITH_MMA
     MmaHostState mma;
 #endif
 };
 
-// ---- dynamic-unit tickets --------------------------------------------------------------------------
-// The tensor-core kernel hands out the tail of the tile list through an atomic counter that must be zero
-// when a decode kernel starts.  The counters live inside the library image (zero at load, reset by the
-// combine kernel after every call), one per handle, so no caller buffer has to be initialised and no
-// caller can overwrite them.  Calls on one handle are stream-ordered by contract, so a counter has one user at a time.
-constexpr int kMaxHandles = 4096;
-static __device__ int32_t g_tickets[kMaxHandles];
+// ---- device-side scheduling state ------------------------------------------------------------------
+// The decode and combine kernels coordinate through a few int32 words per handle (gva_common.cuh, kSync*): the tickets
+// that hand out tail units and the per-sequence arrival counters the combine kernel polls.  They live in an arena
+// inside the library image (zero at load), so no caller buffer has to be initialised and no caller can overwrite them;
+// a handle reserves a region of it sized for its largest batch so far.  Calls on one handle are stream-ordered by
+// contract, so a region has one user at a time.
+constexpr int kSyncArenaInts = 1 << 20;          // 4 MiB of device memory per GPU that loads the library
+static __device__ int32_t g_sync_arena[kSyncArenaInts];
 
 namespace {
-std::mutex g_slot_mutex;
-bool g_slot_used[kMaxHandles] = {};
+std::mutex g_arena_mutex;
+struct FreeRange { int off, len; };
+constexpr int kMaxFreeRanges = 4096;
+FreeRange g_free[kMaxFreeRanges] = {{0, kSyncArenaInts}};
+int g_n_free = 1;
 
-// Reserves a slot and resolves its device address (the device must be current).  -1 on failure.
-int acquire_ticket_slot(int /*device*/, int32_t **addr) {
-    void *base = nullptr;
-    if (cudaGetSymbolAddress(&base, g_tickets) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return -1;
-    }
-    std::lock_guard<std::mutex> lock(g_slot_mutex);
-    for (int i = 0; i < kMaxHandles; ++i)
-        if (!g_slot_used[i]) {
-            g_slot_used[i] = true;
-            *addr = static_cast<int32_t *>(base) + i;
-            return i;
+// first fit; -1 when the arena is exhausted
+int arena_reserve(int len) {
+    std::lock_guard<std::mutex> lock(g_arena_mutex);
+    for (int i = 0; i < g_n_free; ++i)
+        if (g_free[i].len >= len) {
+            const int off = g_free[i].off;
+            g_free[i].off += len;
+            g_free[i].len -= len;
+            if (g_free[i].len == 0) {
+                for (int j = i + 1; j < g_n_free; ++j) g_free[j - 1] = g_free[j];
+                --g_n_free;
+            }
+            return off;
         }
     return -1;
 }
-void release_ticket_slot(int slot) {
-    if (slot < 0 || slot >= kMaxHandles) return;
-    std::lock_guard<std::mutex> lock(g_slot_mutex);
-    g_slot_used[slot] = false;
+void arena_release(int off, int len) {
+    std::lock_guard<std::mutex> lock(g_arena_mutex);
+    int i = 0;
+    while (i < g_n_free && g_free[i].off < off) ++i;
+    if (g_n_free >= kMaxFreeRanges) return;             // table of holes full: the range is dropped (lost until the library is reloaded)
+    for (int j = g_n_free; j > i; --j) g_free[j] = g_free[j - 1];
+    g_free[i] = FreeRange{off, len};
+    ++g_n_free;
+    if (i + 1 < g_n_free && g_free[i].off + g_free[i].len == g_free[i + 1].off) {       // merge with the next hole
+        g_free[i].len += g_free[i + 1].len;
+        for (int j = i + 2; j < g_n_free; ++j) g_free[j - 1] = g_free[j];
+        --g_n_free;
+    }
+    if (i > 0 && g_free[i - 1].off + g_free[i - 1].len == g_free[i].off) {               // ... and with the previous one
+        g_free[i - 1].len += g_free[i].len;
+        for (int j = i + 1; j < g_n_free; ++j) g_free[j - 1] = g_free[j];
+        --g_n_free;
+    }
+}
+
+// Makes sure the handle's region holds `need` words; a new, larger region is cleared on `stream` before first use.
+int ensure_sync(gva_handle *h, int need, cudaStream_t stream) {
+    if (need <= h->sync_cap) return GVA_OK;
+    if (h->n_regions >= 24) return GVA_ERR_UNSUPPORTED;
+    int cap = 64;
+    while (cap < need) cap *= 2;
+    const int off = arena_reserve(cap);
+    if (off < 0) return GVA_ERR_UNSUPPORTED;            // too many live handles with very large batches
+    if (cudaMemsetAsync(h->sync_base + off, 0, (size_t)cap * sizeof(int32_t), stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        arena_release(off, cap);
+        return GVA_ERR_CUDA;
+    }
+    h->region_off[h->n_regions] = off;
+    h->region_cap[h->n_regions] = cap;
+    ++h->n_regions;
+    h->sync_off = off;
+    h->sync_cap = cap;
+    return GVA_OK;
 }
 }  // namespace
 
@@ -130,35 +173,57 @@ bool plan_fma(const gva_handle *h, int B, FmaPlan *out) {
 // Workspace: header ints, then partial outputs, then (max, sum) pairs.
 struct WorkspaceLayout {
     size_t hdr_bytes, rec_o_bytes, rec_ml_bytes, total;
-    int n_rec;
+    int n_rec, sync_ints;
 };
 
-int max_blocks_balanced(const gva_handle *h) {
-    // an upper bound on resident decode blocks that any kernel variant launches: 4 per SM
-    return 4 * h->sm_count;
-}
-
-// Upper bound on units (records per sequence come on top): the CUDA-core kernel uses one unit per block; the
-// tensor-core kernel runs at most 2 blocks per SM (d_v = 64) or 1 (d_v = 128), each range with up to 4 tail units.
-int max_units_balanced(const gva_handle *h) {
+// Thread blocks the balanced partition launches at most, per kernel family; the workspace is sized from the same numbers
+// the launchers use.
+int mma_grid_cap(const gva_handle *h, bool gqa) {
 #ifdef GVA_WITH_MMA
-    const int per_sm = h->cfg.cache_dtype == GVA_E4M3 ? fp8_blocks_per_sm(h->cfg) : (h->cfg.d_v == 64 ? 2 : 1);
+    if (h->cfg.cache_dtype == GVA_E4M3) return fp8_blocks_per_sm(h->cfg) * h->sm_count;
+    return mma_blocks_per_sm_cap(h->cfg, gqa, h->smem_per_sm) * h->sm_count;
 #else
-    const int per_sm = h->cfg.d_v == 64 ? 2 : 1;
+    (void)gqa;
+    return 0;
 #endif
-    const int mma_blocks = per_sm * h->sm_count;
-    const int a = max_blocks_balanced(h), b = unit_bound(mma_blocks);
-    return a > b ? a : b;
+}
+int fma_grid_cap(const gva_handle *h) { return 4 * h->sm_count; }
+
+// Upper bound on units of the balanced partition (records per sequence come on top): the CUDA-core kernel uses one unit
+// per block; the tensor-core kernels cut every range into a head and, for d_v = 64, GVA_TAIL_UNITS tails.
+int max_units_balanced(const gva_handle *h) {
+    int units = 0;
+#ifdef GVA_WITH_MMA
+    const int per_range = h->cfg.d_v == 64 ? GVA_TAIL_UNITS + 1 : 1;
+    const int cap = std::max(mma_grid_cap(h, false), mma_grid_cap(h, true));
+    units = cap * per_range;
+    const bool fma_possible = h->cfg.cache_dtype == GVA_F32 || h->cfg.kernel == GVA_KERNEL_FMA ||
+                              (h->cfg.cache_dtype == GVA_BF16 && !(mma_supported(h->cfg, false) && mma_supported(h->cfg, true)));
+#else
+    const bool fma_possible = true;
+#endif
+    if (fma_possible) units = std::max(units, fma_grid_cap(h));
+    return units;
+}
+int max_rec_mult(const gva_handle *h) {
+#ifdef GVA_WITH_MMA
+    if (h->cfg.cache_dtype == GVA_E4M3) return GVA_FP8_WPG;
+    return h->cfg.d_v == 64 ? GVA_MMA_WPG64 : 1;
+#else
+    return 1;
+#endif
 }
 
 WorkspaceLayout workspace_layout(const gva_handle *h, int B, int num_splits, int q_len = 1) {
     WorkspaceLayout w;
-    // up to two partial records per (block, sequence): the 16-bit tensor-core kernel may run two warps per group
-    w.n_rec = (h->cfg.cache_dtype == GVA_E4M3 ? 1 : 2) * (num_splits > 0 ? B * num_splits : max_units_balanced(h) + B);
+    w.n_rec = max_rec_mult(h) * (num_splits > 0 ? B * num_splits : max_units_balanced(h) + B);
+    if (w.n_rec < 1) w.n_rec = 1;
+    const size_t HQ = (size_t)h->cfg.H * q_len;             // q_len * H pseudo-heads per record
     w.hdr_bytes = align_up((size_t)(kHdrInts + 2 * B) * 4, 256);
-    w.rec_o_bytes = align_up((size_t)w.n_rec * h->cfg.H * q_len * h->cfg.d_v * 4, 256);     // q_len * H pseudo-heads per record
-    w.rec_ml_bytes = align_up((size_t)w.n_rec * h->cfg.H * q_len * 2 * 4, 256);
+    w.rec_o_bytes = align_up((size_t)w.n_rec * HQ * h->cfg.d_v * 4, 256);
+    w.rec_ml_bytes = align_up((size_t)w.n_rec * HQ * 2 * 4, 256);
     w.total = w.hdr_bytes + w.rec_o_bytes + w.rec_ml_bytes;
+    w.sync_ints = kSyncWords;
     return w;
 }
 
@@ -171,9 +236,12 @@ int check_common(const gva_handle *h, int B, int max_seq_len, int num_splits) {
     return GVA_OK;
 }
 
+// Validates and launches one decode kernel (which also merges its partial results).  dry = true runs every host-side
+// check and preparation (workspace, kernel choice, shared-memory fit, tensor maps, sync region) but launches nothing, so
+// that a caller can make sure a later launch cannot fail for a reason known in advance.
 template <bool GQA>
 int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspace_bytes, int B, int max_seq_len,
-                  int num_splits, cudaStream_t stream, int q_len = 1) {
+                  int num_splits, cudaStream_t stream, int q_len = 1, bool dry = false) {
     const WorkspaceLayout w = workspace_layout(h, B, num_splits, q_len);
     if (!workspace || workspace_bytes < w.total) return GVA_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return GVA_ERR_INVALID_ARG;
@@ -181,11 +249,10 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     p.hdr = reinterpret_cast<int32_t *>(ws);
     p.rec_o = reinterpret_cast<float *>(ws + w.hdr_bytes);
     p.rec_ml = reinterpret_cast<float *>(ws + w.hdr_bytes + w.rec_o_bytes);
+    p.n_rec = w.n_rec;
     p.num_splits = num_splits;
     p.rec_mult = 1;
-    p.combine_passes = 2;
     if (B == 0) return GVA_OK;
-
 
     int kernel = h->cfg.kernel;
     if (kernel == GVA_KERNEL_AUTO) {
@@ -198,15 +265,22 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     if (h->cfg.cache_dtype == GVA_E4M3) kernel = GVA_KERNEL_MMA;
     if (q_len > 1 && (GQA || kernel != GVA_KERNEL_MMA)) return GVA_ERR_UNSUPPORTED;   // multi-token decode: tensor-core kernel only
     if (GQA && h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;
+    const int rc_sync = ensure_sync(h, w.sync_ints, stream);
+    if (rc_sync != GVA_OK) return rc_sync;
+    p.sync = h->sync_base + h->sync_off;
+    p.epoch = dry ? h->epoch : ++h->epoch;      // a dry run prepares, it does not consume an epoch
+    if (h->epoch >= (1 << 30)) h->epoch = 2 + (h->epoch & 1);      // wrap, keeping the parity sequence
     if (kernel == GVA_KERNEL_MMA) {
 #ifdef GVA_WITH_MMA
+        h->mma.dry = dry;
         int rc = h->cfg.cache_dtype == GVA_E4M3
                      ? launch_decode_fp8(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, q_len, max_seq_len, num_splits, stream,
                                          &h->last_num_splits, &h->last_tile, &p.rec_mult)
                  : q_len > 1 ? launch_decode_mma_multi(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, q_len, max_seq_len, num_splits,
-                                                     max_blocks_balanced(h), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult)
+                                                     mma_grid_cap(h, false), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult)
                            : launch_decode_mma<GQA>(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, max_seq_len, num_splits,
-                                        max_blocks_balanced(h), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult);
+                                        mma_grid_cap(h, GQA), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult);
+        h->mma.dry = false;
         if (rc != GVA_OK) return rc;
         h->last_kernel = GVA_KERNEL_MMA;
 #else
@@ -225,18 +299,20 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, plan.fn, plan.threads, plan.smem) != cudaSuccess)
                 return GVA_ERR_CUDA;
             if (per_sm < 1) per_sm = 1;
-            if (per_sm > 4) per_sm = 4;
             const long long tiles_ub = (long long)B * ((max_seq_len + 31) / 32);
-            grid = (int)std::min<long long>((long long)per_sm * h->sm_count, std::max<long long>(tiles_ub, 1));
-        }
-        if (launch_pdl(plan.fn, dim3(grid), dim3(plan.threads), plan.smem, stream, p) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return GVA_ERR_CUDA;
+            grid = (int)std::min<long long>(std::min<long long>((long long)per_sm * h->sm_count, fma_grid_cap(h)),
+                                            std::max<long long>(tiles_ub, 1));
         }
         h->last_num_splits = grid;
         h->last_kernel = GVA_KERNEL_FMA;
         h->last_tile = 32;
+        if (dry) return GVA_OK;
+        if (launch_pdl(plan.fn, dim3(grid), dim3(plan.threads), plan.smem, stream, p) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return GVA_ERR_CUDA;
+        }
     }
+    if (dry) return GVA_OK;
     // Warps per head for the merge: enough that a head's records (about units / B, plus the cuts at both ends)
     // are fetched in one or two round trips; one warp per head and four heads per block for the wide-head shape
     // unless a sequence has many records, so that those blocks fit beside the decode kernel's blocks.
@@ -248,8 +324,11 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     int wph = h->cfg.d_v == 64 ? 4 : 1;
     while (wph < 32 && wph * 8 < n_est) wph *= 2;
     if (h->cfg.d_v == 128 && wph <= 2) wph = 1;
-    // ... but no more than ~4096 warps in the whole grid: beyond that the merge blocks no longer fit beside the decode
-    // blocks and start in waves after them (measured on B = 128: 2 warps per head 94 us, 4 warps 99 us, 8 warps 107 us)
+    // ... but no more warps in the whole grid than fit beside the decode blocks (64 registers per merge thread next to
+    // two 160-thread decode blocks of ~72 registers: about 27 warps per SM at the 48 registers of the small instantiation): merge blocks that are not resident start
+    // only when decode blocks leave, a launch latency after the last tile instead of a poll after it
+    // (measured on the 32-sequence long-context workload: the last poll succeeds 2.7 us after the last arrival when
+    // part of the merge grid is not resident, 1.4 us when all of it is)
     const int HQ = h->cfg.H * q_len;           // the merge sees q_len * H pseudo-heads: out rows are [b][slot][head]
     p.H = HQ;
     while (wph > 1 && (long long)B * HQ * wph > 4096) wph /= 2;
@@ -260,7 +339,6 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
                                               : launch_pdl(combine_kernel<128>, cgrid, cblock, csmem, stream, p, wph, hpb);
     if (ce != cudaSuccess) {
         (void)cudaGetLastError();
-        (void)cudaMemsetAsync(h->ticket, 0, sizeof(int32_t), stream);   // the merge that would have reset it never ran
         return GVA_ERR_CUDA;
     }
     return GVA_OK;
@@ -298,10 +376,11 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device >= n_dev) return GVA_ERR_CUDA;
     if (cudaSetDevice(device) != cudaSuccess) return GVA_ERR_CUDA;
-    int major = 0, sms = 0, optin = 0;
+    int major = 0, sms = 0, optin = 0, per_sm = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
-        cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
+        cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, device) != cudaSuccess)
         return GVA_ERR_CUDA;
     if (major != 10) return GVA_ERR_CUDA;   // the kernels are built for sm_100a only
 
@@ -311,19 +390,26 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
     h->device = device;
     h->sm_count = sms;
     h->smem_optin = optin;
+    h->smem_per_sm = per_sm;
     h->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : (float)(1.0 / std::sqrt((double)(cfg->d_c + cfg->d_r)));
     for (int i = 0; i < kMaxRopePairs; ++i)
         h->rope.inv_freq[i] = (2 * i < cfg->d_r) ? std::pow(cfg->rope_base, -2.0 * (double)i / (double)cfg->d_r) : 0.0;
     h->last_num_splits = 0;
     h->last_kernel = 0;
     h->last_tile = 0;
-    h->ticket_slot = acquire_ticket_slot(device, &h->ticket);
-    if (h->ticket_slot < 0) {
-        delete h;
-        return GVA_ERR_CUDA;
+    {
+        void *base = nullptr;
+        if (cudaGetSymbolAddress(&base, g_sync_arena) != cudaSuccess) {     // `device` is current
+            (void)cudaGetLastError();
+            delete h;
+            return GVA_ERR_CUDA;
+        }
+        h->sync_base = static_cast<int32_t *>(base);
+        h->sync_off = h->sync_cap = h->n_regions = 0;
+        h->epoch = 0;
     }
 #ifdef GVA_WITH_MMA
-    int rc = mma_host_init(&h->mma);
+    int rc = mma_host_init(&h->mma, device);
     if (rc != GVA_OK) {
         delete h;
         return rc;
@@ -348,7 +434,7 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
 
 int gva_destroy(gva_handle *h) {
     if (!h) return GVA_ERR_INVALID_ARG;
-    release_ticket_slot(h->ticket_slot);
+    for (int i = 0; i < h->n_regions; ++i) arena_release(h->region_off[i], h->region_cap[i]);
     delete h;
     return GVA_OK;
 }
@@ -549,7 +635,8 @@ int gva_decode_multi(gva_handle *h, const gva_cache *cache, const float *q_abs, 
 
 static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
                        float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
-                       int32_t *dev_status, void *stream, int early_start, const int32_t *append_pos, int q_len = 1) {
+                       int32_t *dev_status, void *stream, int early_start, const int32_t *append_pos, int q_len = 1,
+                       bool dry = false) {
     int rc = check_common(h, B, max_seq_len, num_splits);
     if (rc != GVA_OK) return rc;
     if (!cache) return GVA_ERR_INVALID_ARG;
@@ -576,10 +663,9 @@ static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs
     p.scale_log2 = h->scale * kLog2e;
     p.early_start = early_start;
     p.append_pos = append_pos;
-    p.ticket = h->ticket;
     p.q_len = q_len;
     return launch_decode<false>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
-                                static_cast<cudaStream_t>(stream), q_len);
+                                static_cast<cudaStream_t>(stream), q_len, dry);
 }
 
 int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
@@ -617,9 +703,15 @@ int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const
     if (!aligned(cache->v_pool, 16) || !aligned(cache->kr_pool, 16) || !aligned(q_abs, 16) || !aligned(out, 16) ||
         !aligned(M, 16))
         return GVA_ERR_INVALID_ARG;
-    if (!workspace || workspace_bytes < workspace_layout(h, B, num_splits).total) return GVA_ERR_WORKSPACE;
     const gva_config &c = h->cfg;
     if (c.G * c.d_v > kAppendMaxPerThread * 128) return GVA_ERR_UNSUPPORTED;
+    // every host-side check of the decode launch comes first, so that an error return means nothing was enqueued and
+    // the cache was not advanced
+#ifndef GVA_NO_DRY
+    rc = decode_impl(h, cache, q_abs, seq_lens, out, lse, workspace, workspace_bytes, B, max_seq_len, num_splits, dev_status,
+                     stream, 1, pos, 1, true);
+    if (rc != GVA_OK) return rc;
+#endif
     StepFrontParams a;
     a.q_c = q_c; a.q_r = q_r; a.M = M; a.v_new = v_new; a.kr_new = kr_new;
     a.pos = pos; a.block_table = cache->block_table; a.q_abs = q_abs;
@@ -627,6 +719,7 @@ int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const
     a.B = B; a.H = c.H; a.G = c.G; a.d_v = c.d_v; a.d_c = c.d_c; a.d_r = c.d_r; a.P = c.page_size;
     a.num_pages = cache->num_pages; a.max_pages = cache->max_pages_per_seq;
     a.n_absorb = c.H * ((B + kAbsorbBatch - 1) / kAbsorbBatch);
+    a.trace_call = h->epoch + 1;
     const size_t smem = absorb_smem_bytes(c.d_v, c.d_c);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const cudaError_t ce = (c.cache_dtype == GVA_E4M3)
@@ -709,7 +802,6 @@ int gqa_decode(gva_handle *h, const gqa_cache *cache, const float *q, const int3
     p.num_pages = cache->num_pages;
     p.max_pages = cache->max_pages_per_seq;
     p.scale_log2 = (float)(1.0 / std::sqrt((double)c.d_v)) * kLog2e;
-    p.ticket = h->ticket;
     return launch_decode<true>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
                                static_cast<cudaStream_t>(stream));
 }
@@ -968,7 +1060,11 @@ int gva_project_out(gva_handle *h, const float *attn, const void *W_o, int d_mod
 int gva_layer_step(gva_handle *h, const gva_cache *cache, const float *x, const void *W_in, const void *W_o, int d_model,
                    const int32_t *pos, const int32_t *seq_lens, float *q_abs, float *attn, float *y, void *workspace,
                    size_t workspace_bytes, int B, int max_seq_len, int num_splits, int32_t *dev_status, void *stream) {
-    int rc = gva_project_in(h, cache, x, W_in, d_model, pos, q_abs, B, dev_status, stream);
+    // the decode launch's host-side checks first: an error return then means the cache was not advanced
+    int rc = decode_impl(h, cache, q_abs, seq_lens, attn, nullptr, workspace, workspace_bytes, B, max_seq_len, num_splits,
+                         dev_status, stream, 0, nullptr, 1, true);
+    if (rc != GVA_OK) return rc;
+    rc = gva_project_in(h, cache, x, W_in, d_model, pos, q_abs, B, dev_status, stream);
     if (rc != GVA_OK) return rc;
     rc = gva_decode(h, cache, q_abs, seq_lens, attn, nullptr, workspace, workspace_bytes, B, max_seq_len, num_splits,
                     dev_status, stream);
@@ -979,6 +1075,19 @@ int gva_layer_step(gva_handle *h, const gva_cache *cache, const float *x, const 
 int gva_last_num_splits(const gva_handle *h) { return h ? h->last_num_splits : 0; }
 int gva_last_kernel(const gva_handle *h) { return h ? h->last_kernel : 0; }
 int gva_last_tile_tokens(const gva_handle *h) { return h ? h->last_tile : 0; }
+
+#ifdef GVA_TRACE
+// Development builds only: copies the in-kernel timeline stamps (kTrCalls x kTrSlots) to the host and clears them
+// (synchronises the device).
+int gva_debug_trace(unsigned long long *out) {
+    unsigned long long init[kTrCalls * kTrSlots];
+    if (cudaDeviceSynchronize() != cudaSuccess) return GVA_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(out, g_trace, sizeof(init)) != cudaSuccess) return GVA_ERR_CUDA;
+    for (int i = 0; i < kTrCalls * kTrSlots; ++i) init[i] = (i & 1) ? 0ull : ~0ull;
+    if (cudaMemcpyToSymbol(g_trace, init, sizeof(init)) != cudaSuccess) return GVA_ERR_CUDA;
+    return GVA_OK;
+}
+#endif
 
 const char *gva_status_string(int status) {
     switch (status) {

@@ -20,10 +20,16 @@ constexpr int kHdrTotal = 0;        // total tiles
 constexpr int kHdrRanges = 1;       // equal contiguous ranges the tile list is cut into
 constexpr int kHdrU = 2;            // tail units per range
 constexpr int kHdrK = 3;            // tiles per tail unit
+// Device-side scheduling state of one handle ("sync region": int32 words inside the library image).  Every call has an
+// epoch number (1, 2, 3, ...); the call with epoch e uses the words of parity e & 1, and block 0 of its decode kernel
+// clears the words of the other parity for the call after it, so nothing has to be reset at the end of a call and a
+// call that gave up half-way leaves nothing behind that later calls would trip over.
+constexpr int kSyncTicket = 0;      // [2] next tail unit to hand out
+constexpr int kSyncWords = 2;       // (the fused decode step adds its own words behind these: see gva_decode_mma.cuh)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-// Everything a decode / combine launch needs, passed by value.
+// Everything a decode launch needs, passed by value.
 struct DecodeParams {
     const void *v_pool;          // GVA: values.  GQA: values.
     const void *kr_pool;         // GVA: shared rotated positional keys.  GQA: unused.
@@ -32,16 +38,17 @@ struct DecodeParams {
     const int32_t *seq_lens;
     const float *q;              // [B][H][d_q]
     int32_t *hdr;                // workspace header (kHdrInts + 2 B ints)
-    float *rec_o;                // [n_rec][H][d_v] unnormalised partial outputs
-    float *rec_ml;               // [n_rec][H][2]   running max (log2 domain) and sum
+    float *rec_o;                // [n_rec][H * q_len][d_v] unnormalised partial outputs
+    float *rec_ml;               // [n_rec][H * q_len][2]   running max (log2 domain) and sum
     float *out;                  // [B][H][d_v]
     float *lse;                  // nullable
     int32_t *dev_status;         // nullable
-    int32_t *ticket;             // next dynamic unit to hand out; zero between calls
+    int32_t *sync;               // this handle's sync region (see kSync*)
+    int epoch;                   // this call's number on its handle (>= 1)
+    int n_rec;                   // records the workspace holds
     int B, H, G, P, num_pages, max_pages;
     int num_splits;              // 0 = balanced flat partition
     int rec_mult;                // partial records per (block, sequence): consumer warps per value group
-    int combine_passes;          // 2: the combine kernel runs its body once dry before its dependency wait
     int early_start;             // 1: launched right behind step_front_kernel (see gva_decode_mma.cuh)
     const int32_t *append_pos;   // early_start: position being appended per sequence (its tile must not be read early)
     float scale_log2;            // softmax scale * log2(e)
@@ -228,26 +235,51 @@ __device__ __forceinline__ BlockRange block_range(const DecodeParams &p, const i
     return r;
 }
 
-// Block 0 publishes the tile offsets and the unit plan for the combine kernel.
-__device__ __forceinline__ void publish_header(const DecodeParams &p, const int *s_off, const UnitPlan &plan,
-                                               int tid = threadIdx.x, int nt = blockDim.x) {
-    if (blockIdx.x != 0) return;
+// Block 0 of a decode kernel, threads [0, nt), after the block's dependency wait: clears the other parity's ticket and
+// publishes the tile offsets and the unit plan for the combine kernel: per sequence the first record (per-warp
+// multiplier applied) and the number of records of its run of units.
+__device__ __forceinline__ void block0_duties(const DecodeParams &p, const int *s_off, const UnitPlan &plan, int tid, int nt) {
+    if (blockIdx.x != 0 || tid >= nt) return;
     if (tid == 0) {
+        p.sync[kSyncTicket + ((p.epoch & 1) ^ 1)] = 0;
         p.hdr[kHdrTotal] = plan.total;
         p.hdr[kHdrRanges] = plan.n_ranges;
         p.hdr[kHdrU] = plan.U;
         p.hdr[kHdrK] = plan.K;
     }
-    // per sequence: first record (before the per-warp multiplier) and number of records of its run of units
     for (int b = tid; b < p.B; b += nt) {
         int2 seg = make_int2(0, 0);
-        if (s_off[b + 1] > s_off[b]) {
+        if (p.num_splits > 0) {
+            seg = make_int2(b * p.num_splits * p.rec_mult, p.num_splits * p.rec_mult);
+        } else if (s_off[b + 1] > s_off[b]) {
             const int u0 = unit_of_tile(plan, s_off[b]), u1 = unit_of_tile(plan, s_off[b + 1] - 1);
-            seg = make_int2(u0 + b, u1 - u0 + 1);
+            seg = make_int2((u0 + b) * p.rec_mult, (u1 - u0 + 1) * p.rec_mult);
         }
         reinterpret_cast<int2 *>(p.hdr + kHdrInts)[b] = seg;
     }
 }
+
+// ---- optional in-kernel timeline (build with -DGVA_TRACE) ---------------------------------------------------
+// Slots of %globaltimer stamps (ns), kept as a minimum (even slots) or a maximum (odd slots) over all threads that
+// report; read and cleared by gva_debug_trace().  Compiled out of normal builds.
+enum TraceSlot {
+    kTrFrontEnterMin = 0, kTrFrontExitMax = 1, kTrDecodeEnterMin = 2, kTrDecodeEnterMax = 3, kTrFirstTileMin = 4,
+    kTrFirstTileMax = 5, kTrLastTileMin = 6, kTrLastTileMax = 7, kTrArriveMin = 8, kTrArriveMax = 9, kTrCombineEnterMin = 10,
+    kTrCombinePollMax = 11, kTrCombineOutMin = 12, kTrCombineOutMax = 13, kTrDecodeExitMin = 14, kTrDecodeExitMax = 15, kTrSlots = 16
+};
+constexpr int kTrCalls = 8;      // stamps of the last kTrCalls calls are kept apart (slot set = call number % kTrCalls)
+#ifdef GVA_TRACE
+__device__ unsigned long long g_trace[kTrCalls * kTrSlots];
+__device__ __forceinline__ void trace(int slot, int call) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
+    unsigned long long *dst = &g_trace[(call % kTrCalls) * kTrSlots + slot];
+    if (slot & 1) atomicMax(dst, t);
+    else atomicMin(dst, t);
+}
+#else
+__device__ __forceinline__ void trace(int, int) {}
+#endif
 
 // ---- small PTX wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *ptr) {

@@ -73,7 +73,8 @@ decode_fma_kernel(DecodeParams p) {
 
     grid_dependency_wait();
     compute_tile_offsets<TILE>(p, s_off);
-    publish_header(p, s_off, make_unit_plan(s_off[p.B], gridDim.x, false));
+    const UnitPlan plan = make_unit_plan(s_off[p.B], gridDim.x, false);     // one unit per block: unit id = block index
+    block0_duties(p, s_off, plan, tid, nt);
     const BlockRange rg = block_range(p, s_off);
     const int n_tiles = rg.hi - rg.lo;
 

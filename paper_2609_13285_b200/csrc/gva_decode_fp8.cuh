@@ -126,150 +126,37 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
     }
-    // Early start (only behind step_front_kernel, which has already waited for everything before it): the
-    // tile bookkeeping and the producer's first loads run while the front kernel computes.  Nothing the front
-    // kernel writes is touched before grid_dependency_wait(): consumers wait before reading the absorbed
-    // query, the producer waits before loading the tile that holds the token being appended, and the
-    // workspace is written only after the wait.
+    // Early start: as in the 16-bit kernel (see decode_mma_kernel).
     const bool early = p.early_start != 0;
     if (!early) grid_dependency_wait();
     compute_tile_offsets<TILE>(p, s_off);   // ends with __syncthreads(): barriers are initialised for everyone
-    const bool uniform = p.num_splits > 0;
-    // Tail stealing pays where two blocks share an SM and their speeds differ by +-20 % (d_v = 64: measured -2.7 us
-    // of 100 on the long-context workload); with one block per SM (d_v = 128) speeds differ by +-4 % and the extra
-    // partial records cost more than the balance gains (measured +3.9 us of 180), so there the ranges stay static.
-#ifndef GVA_MMA_DYNAMIC_TAIL
-#define GVA_MMA_DYNAMIC_TAIL 1   // build-time knob: 0 = equal static ranges only
-#endif
-    const UnitPlan plan = make_unit_plan(s_off[p.B], gridDim.x, GVA_MMA_DYNAMIC_TAIL != 0 && DV == 64);
-    BlockRange rg;
-    rg.lo = rg.hi = 0;
-    rg.rec_fixed = -1;
-    rg.b_first = 0;
-    int first_unit = -1;
-    if (uniform) {
-        rg = block_range(p, s_off);
-        if (rg.hi <= rg.lo) {   // an empty split still owns its records (weight 0 in the merge)
-            if (early) grid_dependency_wait();
+    const BlockWork w = decode_block_work<DV>(p, s_off);
+    const UnitPlan &plan = w.plan;
+    const BlockRange &rg = w.rg;
+    if (w.uniform ? rg.hi <= rg.lo : (w.first_unit < 0 && w.n_tickets == 0)) {
+        // nothing to stream: an empty split still owns its records (weight 0 in the merge)
+        if (early) grid_dependency_wait();
+        block0_duties(p, s_off, plan, tid, blockDim.x);
+        if (w.uniform)
             for (int i = tid; i < HQ * WPG; i += blockDim.x) {
                 p.rec_ml[((size_t)rg.rec_fixed * WPG * HQ + i) * 2] = -INFINITY;
                 p.rec_ml[((size_t)rg.rec_fixed * WPG * HQ + i) * 2 + 1] = 0.f;
             }
-            return;
-        }
-    } else if ((int)blockIdx.x < plan.n_ranges) {
-        first_unit = blockIdx.x * (plan.U + 1);          // the head of this block's own range
-        unit_range(plan, blockIdx.x, 0, rg.lo, rg.hi);
-        rg.b_first = (rg.lo < rg.hi) ? seq_of_tile(s_off, p.B, rg.lo) : 0;
-    }
-    const int n_tickets = uniform ? 0 : plan.n_ranges * plan.U;    // tail units on offer
-    if (!uniform && first_unit < 0 && n_tickets == 0) {   // more blocks than ranges and no tails to share
-        if (blockIdx.x == 0) {                            // (total == 0): the header is still needed by the merge
-            if (early) grid_dependency_wait();
-            publish_header(p, s_off, plan);
-        }
         return;
     }
 
     if (warp == n_consumers) {
         // ================================ producer (one elected lane) ================================
         if (lane == 0) {
-            bool waited = !early;
-            bool ok = true;
-            int issued = 0;       // tiles issued by this block: ring position
-            int lo = rg.lo, hi = rg.hi, unit = first_unit;
-            int b = rg.b_first;
-            for (;;) {
-                // the next tail unit is requested while this one is being issued (the ticket is reset
-                // by the previous call's combine kernel: never touch it before grid_dependency_wait())
-                int ticket = -1;
-                bool asked = n_tickets == 0;
-                for (int f = lo; f < hi && ok; ++f) {
-                    const int st = issued % NSTAGE;
-                    if (!waited && issued >= NSTAGE) {   // the ring is full: nothing more to gain from running ahead
-                        grid_dependency_wait();
-                        waited = true;
-                    }
-                    if (!asked && waited && hi - f <= 2) {   // late, so that tails go to whoever really is ahead
-                        ticket = atomicAdd(p.ticket, 1);
-                        asked = true;
-                    }
-                    while (f >= s_off[b + 1]) ++b;
-                    const int t0 = (f - s_off[b]) * TILE;
-                    const int pj = t0 / p.P, slot0 = t0 % p.P;
-                    // the three lookups are independent: request them together, use them afterwards
-                    const int len = p.seq_lens[b];
-                    const int ap = waited ? -1 : p.append_pos[b];
-                    long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
-                                                   : (long long)b * p.max_pages + pj;
-                    if (!waited && ap >= t0 && ap < t0 + TILE) {   // this tile receives the new token: it must be complete first
-                        grid_dependency_wait();
-                        waited = true;
-                    }
-                    int n_valid = min(TILE, len - t0);
-                    if (page < 0 || page >= p.num_pages) {
-                        report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
-                        page = 0;
-                        n_valid = 0;
-                    }
-                    // the bookkeeping above overlaps with the wait for the stage to be released
-                    if (!mbar_wait_bounded(smem_u32(&empty_bar[st]), ((issued / NSTAGE) & 1) ^ 1, s_abort)) {
-                        if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
-                        *s_abort = 1;
-                        ok = false;
-                        break;
-                    }
-                    StageMeta m;
-                    m.n_valid = n_valid;
-                    m.b = b;
-                    m.rec = uniform ? rg.rec_fixed : unit + b;
-                    m.flags = ((f == lo || f == s_off[b]) ? 1 : 0) | ((f + 1 == hi || f + 1 >= s_off[b + 1]) ? 2 : 0);
-                    if constexpr (QL > 1) m.flags |= min(max(len - t0 - TILE, 0), ql - 1) << 8;   // tokens of the sequence beyond this tile, capped
-                    s_meta[st] = m;
-                    const uint32_t bar = smem_u32(&full_bar[st]);
+            const uint64_t pol = l2_policy_evict_first();
+            decode_producer<TILE, NSTAGE, (QL > 1)>(p, w, s_off, full_bar, empty_bar, s_meta, s_abort, ql,
+                [&](int st, long long page, int slot0, uint32_t bar) {
                     const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
                     mbar_expect_tx(bar, G * T::VTILE_BYTES + T::KR_BYTES);
-                    if constexpr (DR > 0) tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
+                    if constexpr (DR > 0) tma_load_2d_stream(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar, pol);
                     for (int g = 0; g < G; ++g)
-                        tma_load_2d(base + g * T::VTILE_BYTES, &tm_v, 0, (int)((page * G + g) * p.P + slot0), bar);
-                    ++issued;
-                }
-                if (!ok) break;
-                if (!asked) {
-                    if (!waited) {
-                        grid_dependency_wait();
-                        waited = true;
-                    }
-                    ticket = atomicAdd(p.ticket, 1);
-                }
-                if (ticket < 0 || ticket >= n_tickets) break;
-                // ticket t -> tail j = 1 + t / n_ranges of range t % n_ranges: first every range's first tail, then the second, ...
-                const int c = ticket % plan.n_ranges, j = 1 + ticket / plan.n_ranges;
-                unit = c * (plan.U + 1) + j;
-                unit_range(plan, c, j, lo, hi);
-                if (lo < hi) b = seq_of_tile(s_off, p.B, lo);
-            }
-            if (ok) {
-                // tell the consumers that nothing more is coming
-                const int st = issued % NSTAGE;
-                if (mbar_wait_bounded(smem_u32(&empty_bar[st]), ((issued / NSTAGE) & 1) ^ 1, s_abort)) {
-                    s_meta[st].n_valid = -1;
-                    mbar_arrive(smem_u32(&full_bar[st]));
-                } else {
-                    if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
-                    *s_abort = 1;
-                    ok = false;
-                }
-            }
-            if (!ok) {
-                // drain: every copy this block started must land before its shared memory is released
-                const int first = max(0, issued - NSTAGE);
-                for (int i = first; i < issued; ++i) {
-                    const int st = i % NSTAGE;
-                    for (int it = 0; it < kDrainPolls; ++it)
-                        if (mbar_try_wait(smem_u32(&full_bar[st]), (i / NSTAGE) & 1)) break;
-                }
-            }
+                        tma_load_2d_stream(base + g * T::VTILE_BYTES, &tm_v, 0, (int)((page * G + g) * p.P + slot0), bar, pol);
+                });
         }
     } else {
         // ============ consumer: value group g, token chunks [part*CPW, part*CPW + CPW) of every tile ============
@@ -316,7 +203,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             }
         };
         if (early) grid_dependency_wait();
-        publish_header(p, s_off, plan, tid, n_consumers * 32);
+        block0_duties(p, s_off, plan, tid, n_consumers * 32);
         // the first sequence is known before any tile arrives: fetch its query while the first copies fly
         int cur_b = -1;
         if (rg.lo < rg.hi) {
@@ -512,7 +399,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 }
             };
             if (early) grid_dependency_wait();
-            publish_header(p, s_off, plan, tid, n_consumers * 32);
+            block0_duties(p, s_off, plan, tid, n_consumers * 32);
             int cur_b = -1;
             if (rg.lo < rg.hi) {
                 cur_b = rg.b_first;
@@ -737,7 +624,7 @@ inline bool encode_map_u8(const MmaHostState &st, CUtensorMap *map, const void *
 }
 
 template <int DV, int DR, int TILE, int QL = 1>
-int launch_fp8_t(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
+int launch_fp8_t(const gva_config &cfg, MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
                  int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out) {
     using T = Fp8Traits<DV, DR, TILE>;
     constexpr int NSTAGE = GVA_FP8_NSTAGE;
@@ -747,16 +634,25 @@ int launch_fp8_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
     const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
     auto fn = G <= 4 ? decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 4, QL> : decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 8, QL>;
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
-    CUtensorMap tm_v, tm_k;
-    if (!encode_map_u8(st, &tm_v, p.v_pool, DV, (uint64_t)p.num_pages * G * p.P, DV, TILE,
-                       DV == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B))
-        return GVA_ERR_CUDA;
-    if (DR == 0) {
-        tm_k = tm_v;      // value-only cache: no positional tile (the kernel never uses this map)
-    } else if (!encode_map_u8(st, &tm_k, p.kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, TILE,
-                              DR == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE)) {
-        return GVA_ERR_CUDA;
+    static int s_smem_set[2][kMaxDevicesCached] = {};      // per (G <= 4 or not, device): the attribute is set once, not per call
+    const int dev = st.device >= 0 && st.device < kMaxDevicesCached ? st.device : 0;
+    if (s_smem_set[G <= 4][dev] != (int)smem || st.device >= kMaxDevicesCached) {
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
+        s_smem_set[G <= 4][dev] = (int)smem;
+    }
+    const MapPair *mp = st.find(p.v_pool, p.kr_pool, p.num_pages, 2);
+    if (!mp) {
+        MapPair *m = st.slot_for(p.v_pool, p.kr_pool, p.num_pages, 2);
+        bool ok = encode_map_u8(st, &m->tm_v, p.v_pool, DV, (uint64_t)p.num_pages * G * p.P, DV, TILE,
+                                DV == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
+        if (ok && DR == 0) m->tm_k = m->tm_v;      // value-only cache: no positional tile (the kernel never uses this map)
+        else if (ok) ok = encode_map_u8(st, &m->tm_k, p.kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, TILE,
+                                        DR == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE);
+        if (!ok) {
+            st.forget_last();
+            return GVA_ERR_CUDA;
+        }
+        mp = m;
     }
     const int threads = 32 * (G * wpg + 1);
     int grid;
@@ -770,17 +666,18 @@ int launch_fp8_t(const gva_config &cfg, const MmaHostState &st, int sm_count, in
         const long long want = (long long)per_sm * sm_count;
         grid = (int)(tiles_ub < want ? (tiles_ub < 1 ? 1 : tiles_ub) : want);
     }
+    *n_blocks_out = grid;
+    if (st.dry) return GVA_OK;
     DecodeParams pp = p;
     pp.rec_mult = wpg;
-    if (launch_pdl(fn, dim3(grid), dim3(threads), smem, stream, pp, tm_v, tm_k) != cudaSuccess) {
+    if (launch_pdl(fn, dim3(grid), dim3(threads), smem, stream, pp, mp->tm_v, mp->tm_k) != cudaSuccess) {
         (void)cudaGetLastError();
         return GVA_ERR_CUDA;
     }
-    *n_blocks_out = grid;
     return GVA_OK;
 }
 
-inline int launch_decode_fp8(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
+inline int launch_decode_fp8(const gva_config &cfg, MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
                              int q_len, int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out, int *tile_out,
                              int *rec_mult_out) {
     if (!fp8_supported(cfg)) return GVA_ERR_UNSUPPORTED;

@@ -31,17 +31,47 @@ namespace gva {
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+// Tensor maps depend only on the pools' addresses and sizes: they are encoded once per (pools, kernel kind) and kept in
+// the handle, so a call in steady state pays no driver call for them.
+struct alignas(64) MapPair {
+    CUtensorMap tm_v, tm_k;
+};
+constexpr int kMaxDevicesCached = 64;
 struct MmaHostState {
     EncodeTiledFn encode;
+    int device;                      // the handle's device
+    bool dry;                        // true: check support, set attributes and encode maps, but launch nothing
+    static constexpr int kMaps = 8;
+    struct Key {
+        const void *v, *k;
+        int num_pages, kind;
+    } keys[kMaps];
+    MapPair maps[kMaps];
+    int n_maps, next_map;
+    const MapPair *find(const void *v, const void *k, int num_pages, int kind) const {
+        for (int i = 0; i < n_maps; ++i)
+            if (keys[i].v == v && keys[i].k == k && keys[i].num_pages == num_pages && keys[i].kind == kind) return &maps[i];
+        return nullptr;
+    }
+    MapPair *slot_for(const void *v, const void *k, int num_pages, int kind) {      // oldest entry is replaced
+        const int i = n_maps < kMaps ? n_maps++ : (next_map++ % kMaps);
+        keys[i] = Key{v, k, num_pages, kind};
+        return &maps[i];
+    }
+    void forget_last() { if (n_maps > 0) keys[n_maps < kMaps ? --n_maps : ((next_map - 1) % kMaps)].v = nullptr; }
 };
 
-inline int mma_host_init(MmaHostState *st) {
+inline int mma_host_init(MmaHostState *st, int device) {
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
         qres != cudaDriverEntryPointSuccess || !fn)
         return GVA_ERR_CUDA;
     st->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    st->dry = false;
+    st->device = device;
+    st->n_maps = 0;
+    st->next_map = 0;
     return GVA_OK;
 }
 
@@ -90,6 +120,27 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n" ::"r"(dst),
         "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
+}
+// The decode kernels read every cache byte exactly once per call: their loads carry an evict-first L2 policy, so the
+// stream does not push the small things every call needs again (lengths, block table, queries, partial records, the
+// kernels' own instructions) out of L2.
+#ifndef GVA_STREAM_EVICT_FIRST
+#define GVA_STREAM_EVICT_FIRST 1   // build-time knob: 0 = default L2 policy for the cache stream
+#endif
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_load_2d_stream(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar, uint64_t pol) {
+#if GVA_STREAM_EVICT_FIRST
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;\n" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar), "l"(pol)
+        : "memory");
+#else
+    tma_load_2d(dst, map, x, y, bar);
+#endif
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
@@ -170,13 +221,151 @@ __device__ __forceinline__ uint32_t split_hi_lo_fast(float x) {
     return d;
 }
 
+// ---- what a thread block works on ------------------------------------------------------------------------
+struct BlockWork {
+    UnitPlan plan;
+    BlockRange rg;        // first range of tiles (balanced: the head of the block's own range; uniform: its split)
+    int first_unit;       // balanced: unit id of that range, -1 if the block has none
+    int n_tickets;        // balanced: tail units on offer to whoever asks first
+    bool uniform;
+};
+
+#ifndef GVA_MMA_DYNAMIC_TAIL
+#define GVA_MMA_DYNAMIC_TAIL 1   // build-time knob: 0 = equal static ranges only
+#endif
+// Tail stealing pays where two or more blocks share an SM and their speeds differ by +-20 % (d_v = 64: measured -2.7 us
+// of 100 on the long-context workload); with one block per SM (d_v = 128) speeds differ by +-4 % and the extra
+// partial records cost more than the balance gains (measured +3.9 us of 180), so there the ranges stay static.
+template <int DV>
+__device__ __forceinline__ BlockWork decode_block_work(const DecodeParams &p, const int *s_off) {
+    BlockWork w;
+    w.uniform = p.num_splits > 0;
+    w.plan = make_unit_plan(s_off[p.B], gridDim.x, GVA_MMA_DYNAMIC_TAIL != 0 && DV == 64);
+    w.rg.lo = w.rg.hi = 0;
+    w.rg.rec_fixed = -1;
+    w.rg.b_first = 0;
+    w.first_unit = -1;
+    if (w.uniform) {
+        w.rg = block_range(p, s_off);
+    } else if ((int)blockIdx.x < w.plan.n_ranges) {
+        w.first_unit = blockIdx.x * (w.plan.U + 1);          // the head of this block's own range
+        unit_range(w.plan, blockIdx.x, 0, w.rg.lo, w.rg.hi);
+        w.rg.b_first = (w.rg.lo < w.rg.hi) ? seq_of_tile(s_off, p.B, w.rg.lo) : 0;
+    }
+    w.n_tickets = w.uniform ? 0 : w.plan.n_ranges * w.plan.U;
+    return w;
+}
+
 // Per-stage message from the producer to the consumers.
 struct StageMeta {
     int n_valid;   // live tokens in the tile; -1 = no more tiles for this block
     int b;         // sequence
     int rec;       // partial record this tile's segment belongs to (before the per-warp multiplier)
-    int flags;     // bit 0: first tile of its segment, bit 1: last tile of its segment
+    int flags;     // bit 0: first tile of its segment, bit 1: last tile of its segment; bits 8..: see QL > 1
 };
+
+// The producer lane of a tensor-core decode block: walks the block's tiles (its own range, then the tail units it
+// wins), and for each one resolves the page, waits (bounded) for the ring slot, posts the stage message and calls
+// issue(stage, page, first slot, full barrier), which posts the expected byte count and starts the copies.
+// Early start (p.early_start, only behind step_front_kernel): nothing that kernel writes is touched before
+// grid_dependency_wait() -- the tile that receives the token being appended is loaded only after the wait, and so is
+// the ticket, which belongs to the previous call until then.
+template <int TILE, int NSTAGE, bool MULTI, class Issue>
+__device__ __forceinline__ void decode_producer(const DecodeParams &p, const BlockWork &w, const int *s_off, uint64_t *full_bar,
+                                                uint64_t *empty_bar, StageMeta *s_meta, volatile int *s_abort, int ql,
+                                                Issue issue) {
+    bool waited = p.early_start == 0;
+    bool ok = true;
+    int issued = 0;       // tiles issued by this block: ring position
+    int lo = w.rg.lo, hi = w.rg.hi, unit = w.first_unit;
+    int b = w.rg.b_first;
+    int32_t *ticket_ctr = p.sync + kSyncTicket + (p.epoch & 1);
+    for (;;) {
+        // the next tail unit is requested while this one is being issued
+        int ticket = -1;
+        bool asked = w.n_tickets == 0;
+        for (int f = lo; f < hi && ok; ++f) {
+            const int st = issued % NSTAGE;
+            if (!waited && issued >= NSTAGE) {   // the ring is full: nothing more to gain from running ahead
+                grid_dependency_wait();
+                waited = true;
+            }
+            if (!asked && waited && hi - f <= 2) {   // late, so that tails go to whoever really is ahead
+                ticket = atomicAdd(ticket_ctr, 1);
+                asked = true;
+            }
+            while (f >= s_off[b + 1]) ++b;
+            const int t0 = (f - s_off[b]) * TILE;
+            const int pj = t0 / p.P, slot0 = t0 % p.P;
+            // the three lookups are independent: request them together, use them afterwards
+            const int len = p.seq_lens[b];
+            const int ap = waited ? -1 : p.append_pos[b];
+            long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
+                                           : (long long)b * p.max_pages + pj;
+            if (!waited && ap >= t0 && ap < t0 + TILE) {   // this tile receives the new token: it must be complete first
+                grid_dependency_wait();
+                waited = true;
+            }
+            int n_valid = min(TILE, len - t0);
+            if (page < 0 || page >= p.num_pages) {
+                report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
+                page = 0;
+                n_valid = 0;
+            }
+            // the bookkeeping above overlaps with the wait for the stage to be released
+            if (!mbar_wait_bounded(smem_u32(&empty_bar[st]), ((issued / NSTAGE) & 1) ^ 1, s_abort)) {
+                if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+                *s_abort = 1;
+                ok = false;
+                break;
+            }
+            StageMeta m;
+            m.n_valid = n_valid;
+            m.b = b;
+            m.rec = w.uniform ? w.rg.rec_fixed : unit + b;
+            m.flags = ((f == lo || f == s_off[b]) ? 1 : 0) | ((f + 1 == hi || f + 1 >= s_off[b + 1]) ? 2 : 0);
+            if constexpr (MULTI) m.flags |= min(max(len - t0 - TILE, 0), ql - 1) << 8;   // tokens of the sequence beyond this tile, capped
+            s_meta[st] = m;
+            issue(st, page, slot0, smem_u32(&full_bar[st]));
+            ++issued;
+        }
+        if (!ok) break;
+        if (!asked) {
+            if (!waited) {
+                grid_dependency_wait();
+                waited = true;
+            }
+            ticket = atomicAdd(ticket_ctr, 1);
+        }
+        if (ticket < 0 || ticket >= w.n_tickets) break;
+        // ticket t -> tail j = 1 + t / n_ranges of range t % n_ranges: first every range's first tail, then the second, ...
+        const int c = ticket % w.plan.n_ranges, j = 1 + ticket / w.plan.n_ranges;
+        unit = c * (w.plan.U + 1) + j;
+        unit_range(w.plan, c, j, lo, hi);
+        if (lo < hi) b = seq_of_tile(s_off, p.B, lo);
+    }
+    if (ok) {
+        // tell the consumers that nothing more is coming
+        const int st = issued % NSTAGE;
+        if (mbar_wait_bounded(smem_u32(&empty_bar[st]), ((issued / NSTAGE) & 1) ^ 1, s_abort)) {
+            s_meta[st].n_valid = -1;
+            mbar_arrive(smem_u32(&full_bar[st]));
+        } else {
+            if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+            *s_abort = 1;
+            ok = false;
+        }
+    }
+    if (!ok) {
+        // drain: every copy this block started must land before its shared memory is released
+        const int first = max(0, issued - NSTAGE);
+        for (int i = first; i < issued; ++i) {
+            const int st = i % NSTAGE;
+            for (int it = 0; it < kDrainPolls; ++it)
+                if (mbar_try_wait(smem_u32(&full_bar[st]), (i / NSTAGE) & 1)) break;
+        }
+    }
+}
 
 // QL > 1 (multi-token decode, QL = 2 or 4 new tokens per sequence): the 4 heads x QL tokens of a group are the N
 // columns, 8 per N-block, column c = slot * 4 + head with slot the token's index among the new ones; the queries and
@@ -226,153 +415,49 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     // query, the producer waits before loading the tile that holds the token being appended, and the
     // workspace is written only after the wait.
     const bool early = p.early_start != 0;
+    if (tid == 0) {
+        trace(kTrDecodeEnterMin, p.epoch);
+        trace(kTrDecodeEnterMax, p.epoch);
+    }
     if (!early) grid_dependency_wait();
     compute_tile_offsets<TILE>(p, s_off);   // ends with __syncthreads(): barriers are initialised for everyone
-    const bool uniform = p.num_splits > 0;
-    // Tail stealing pays where two blocks share an SM and their speeds differ by +-20 % (d_v = 64: measured -2.7 us
-    // of 100 on the long-context workload); with one block per SM (d_v = 128) speeds differ by +-4 % and the extra
-    // partial records cost more than the balance gains (measured +3.9 us of 180), so there the ranges stay static.
-#ifndef GVA_MMA_DYNAMIC_TAIL
-#define GVA_MMA_DYNAMIC_TAIL 1   // build-time knob: 0 = equal static ranges only
-#endif
-    const UnitPlan plan = make_unit_plan(s_off[p.B], gridDim.x, GVA_MMA_DYNAMIC_TAIL != 0 && DV == 64);
-    BlockRange rg;
-    rg.lo = rg.hi = 0;
-    rg.rec_fixed = -1;
-    rg.b_first = 0;
-    int first_unit = -1;
-    if (uniform) {
-        rg = block_range(p, s_off);
-        if (rg.hi <= rg.lo) {   // an empty split still owns its records (weight 0 in the merge)
-            if (early) grid_dependency_wait();
+    const BlockWork w = decode_block_work<DV>(p, s_off);
+    const UnitPlan &plan = w.plan;
+    const BlockRange &rg = w.rg;
+    if (w.uniform ? rg.hi <= rg.lo : (w.first_unit < 0 && w.n_tickets == 0)) {
+        // nothing to stream.  Uniform mode: an empty split still owns its records (weight 0 in the merge); balanced
+        // mode: more blocks than ranges and no tails to share.
+        if (early) grid_dependency_wait();
+        block0_duties(p, s_off, plan, tid, blockDim.x);
+        if (w.uniform)
             for (int i = tid; i < HQ * WPG; i += blockDim.x) {
                 p.rec_ml[((size_t)rg.rec_fixed * WPG * HQ + i) * 2] = -INFINITY;
                 p.rec_ml[((size_t)rg.rec_fixed * WPG * HQ + i) * 2 + 1] = 0.f;
             }
-            return;
-        }
-    } else if ((int)blockIdx.x < plan.n_ranges) {
-        first_unit = blockIdx.x * (plan.U + 1);          // the head of this block's own range
-        unit_range(plan, blockIdx.x, 0, rg.lo, rg.hi);
-        rg.b_first = (rg.lo < rg.hi) ? seq_of_tile(s_off, p.B, rg.lo) : 0;
-    }
-    const int n_tickets = uniform ? 0 : plan.n_ranges * plan.U;    // tail units on offer
-    if (!uniform && first_unit < 0 && n_tickets == 0) {   // more blocks than ranges and no tails to share
-        if (blockIdx.x == 0) {                            // (total == 0): the header is still needed by the merge
-            if (early) grid_dependency_wait();
-            publish_header(p, s_off, plan);
-        }
         return;
     }
 
     if (warp == n_consumers) {
         // ================================ producer (one elected lane) ================================
         if (lane == 0) {
-            bool waited = !early;
-            bool ok = true;
-            int issued = 0;       // tiles issued by this block: ring position
-            int lo = rg.lo, hi = rg.hi, unit = first_unit;
-            int b = rg.b_first;
-            for (;;) {
-                // the next tail unit is requested while this one is being issued (the ticket is reset
-                // by the previous call's combine kernel: never touch it before grid_dependency_wait())
-                int ticket = -1;
-                bool asked = n_tickets == 0;
-                for (int f = lo; f < hi && ok; ++f) {
-                    const int st = issued % NSTAGE;
-                    if (!waited && issued >= NSTAGE) {   // the ring is full: nothing more to gain from running ahead
-                        grid_dependency_wait();
-                        waited = true;
-                    }
-                    if (!asked && waited && hi - f <= 2) {   // late, so that tails go to whoever really is ahead
-                        ticket = atomicAdd(p.ticket, 1);
-                        asked = true;
-                    }
-                    while (f >= s_off[b + 1]) ++b;
-                    const int t0 = (f - s_off[b]) * TILE;
-                    const int pj = t0 / p.P, slot0 = t0 % p.P;
-                    // the three lookups are independent: request them together, use them afterwards
-                    const int len = p.seq_lens[b];
-                    const int ap = waited ? -1 : p.append_pos[b];
-                    long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
-                                                   : (long long)b * p.max_pages + pj;
-                    if (!waited && ap >= t0 && ap < t0 + TILE) {   // this tile receives the new token: it must be complete first
-                        grid_dependency_wait();
-                        waited = true;
-                    }
-                    int n_valid = min(TILE, len - t0);
-                    if (page < 0 || page >= p.num_pages) {
-                        report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
-                        page = 0;
-                        n_valid = 0;
-                    }
-                    // the bookkeeping above overlaps with the wait for the stage to be released
-                    if (!mbar_wait_bounded(smem_u32(&empty_bar[st]), ((issued / NSTAGE) & 1) ^ 1, s_abort)) {
-                        if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
-                        *s_abort = 1;
-                        ok = false;
-                        break;
-                    }
-                    StageMeta m;
-                    m.n_valid = n_valid;
-                    m.b = b;
-                    m.rec = uniform ? rg.rec_fixed : unit + b;
-                    m.flags = ((f == lo || f == s_off[b]) ? 1 : 0) | ((f + 1 == hi || f + 1 >= s_off[b + 1]) ? 2 : 0);
-                    if constexpr (QL > 1) m.flags |= min(max(len - t0 - TILE, 0), ql - 1) << 8;   // tokens of the sequence beyond this tile, capped
-                    s_meta[st] = m;
-                    const uint32_t bar = smem_u32(&full_bar[st]);
+            const uint64_t pol = l2_policy_evict_first();
+            decode_producer<TILE, NSTAGE, (QL > 1)>(p, w, s_off, full_bar, empty_bar, s_meta, s_abort, ql,
+                [&](int st, long long page, int slot0, uint32_t bar) {
                     const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
                     mbar_expect_tx(bar, GQA ? 2 * G * T::VTILE_BYTES : G * T::VTILE_BYTES + T::KR_BYTES);
-                    if constexpr (!GQA && DR > 0) tma_load_2d(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar);
+                    if constexpr (!GQA && DR > 0) tma_load_2d_stream(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar, pol);
                     for (int g = 0; g < G; ++g) {
                         const int row = (int)((page * G + g) * p.P + slot0);
                         if constexpr (GQA) {
 #pragma unroll
                             for (int bx = 0; bx < T::BOXES; ++bx)
-                                tma_load_2d(base + (G + g) * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_k, bx * 64, row, bar);
+                                tma_load_2d_stream(base + (G + g) * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_k, bx * 64, row, bar, pol);
                         }
 #pragma unroll
                         for (int bx = 0; bx < T::BOXES; ++bx)
-                            tma_load_2d(base + g * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, bar);
+                            tma_load_2d_stream(base + g * T::VTILE_BYTES + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, bar, pol);
                     }
-                    ++issued;
-                }
-                if (!ok) break;
-                if (!asked) {
-                    if (!waited) {
-                        grid_dependency_wait();
-                        waited = true;
-                    }
-                    ticket = atomicAdd(p.ticket, 1);
-                }
-                if (ticket < 0 || ticket >= n_tickets) break;
-                // ticket t -> tail j = 1 + t / n_ranges of range t % n_ranges: first every range's first tail, then the second, ...
-                const int c = ticket % plan.n_ranges, j = 1 + ticket / plan.n_ranges;
-                unit = c * (plan.U + 1) + j;
-                unit_range(plan, c, j, lo, hi);
-                if (lo < hi) b = seq_of_tile(s_off, p.B, lo);
-            }
-            if (ok) {
-                // tell the consumers that nothing more is coming
-                const int st = issued % NSTAGE;
-                if (mbar_wait_bounded(smem_u32(&empty_bar[st]), ((issued / NSTAGE) & 1) ^ 1, s_abort)) {
-                    s_meta[st].n_valid = -1;
-                    mbar_arrive(smem_u32(&full_bar[st]));
-                } else {
-                    if (!*s_abort) report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
-                    *s_abort = 1;
-                    ok = false;
-                }
-            }
-            if (!ok) {
-                // drain: every copy this block started must land before its shared memory is released
-                const int first = max(0, issued - NSTAGE);
-                for (int i = first; i < issued; ++i) {
-                    const int st = i % NSTAGE;
-                    for (int it = 0; it < kDrainPolls; ++it)
-                        if (mbar_try_wait(smem_u32(&full_bar[st]), (i / NSTAGE) & 1)) break;
-                }
-            }
+                });
         }
     } else {
         // ============ consumer: value group g, token chunks [part*CPW, part*CPW + CPW) of every tile ============
@@ -419,7 +504,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             }
         };
         if (early) grid_dependency_wait();
-        publish_header(p, s_off, plan, tid, n_consumers * 32);
+        block0_duties(p, s_off, plan, tid, n_consumers * 32);
         // the first sequence is known before any tile arrives: fetch its query while the first copies fly
         int cur_b = -1;
         if (rg.lo < rg.hi) {
@@ -438,6 +523,10 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             const StageMeta meta = s_meta[st];
             const int n_valid = meta.n_valid;
             if (n_valid < 0) break;       // producer is done
+            if (i == 0 && tid == 0) {
+                trace(kTrFirstTileMin, p.epoch);
+                trace(kTrFirstTileMax, p.epoch);
+            }
             const int b = meta.b;
             if (meta.flags & 1) {         // a new segment: its own softmax state (and query, if the sequence changed)
                 if (b != cur_b) {
@@ -567,7 +656,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 }
             }
         }
-    
+
         } else {
             // ================= multi-token decode: QL new tokens per sequence, columns = slot * 4 + head =================
             uint32_t qf[T::KSTEPS][NBK][2];   // B fragments of Q^T (plain bf16): column n = lane / 4 of N-block nb
@@ -594,7 +683,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 }
             };
             if (early) grid_dependency_wait();
-            publish_header(p, s_off, plan, tid, n_consumers * 32);
+            block0_duties(p, s_off, plan, tid, n_consumers * 32);
             int cur_b = -1;
             if (rg.lo < rg.hi) {
                 cur_b = rg.b_first;
@@ -770,6 +859,10 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     }
     // keep shared memory alive until every warp (and every copy in flight) is done
     __syncthreads();
+    if (tid == 0) {
+        trace(kTrDecodeExitMin, p.epoch);
+        trace(kTrDecodeExitMax, p.epoch);
+    }
 }
 
 // ---- host: support check, tensor maps, launch ------------------------------------------------------
@@ -799,54 +892,83 @@ inline bool encode_map(const MmaHostState &st, CUtensorMap *map, const void *bas
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Resident blocks per SM that the grid of the 16-bit tensor-core kernel is sized for at most: what the shared memory
+// of an SM holds of its three-stage rings, at most 4.  The workspace bound uses the same number.
+inline int mma_blocks_per_sm_cap(const gva_config &cfg, bool gqa, int smem_per_sm) {
+    const int tile = (cfg.d_v == 64) ? (cfg.page_size % 64 == 0 ? 64 : 32) : (gqa ? 16 : 32);
+    const int vtile = (cfg.d_v / 64) * tile * 128;
+    const int kr = (tile * cfg.d_r * 2 + 1023) & ~1023;
+    const int stage = gqa ? 2 * cfg.G * vtile : cfg.G * vtile + (cfg.d_r > 0 ? kr : 0);
+    const int per_block = 1024 + 3 * stage + 1024;      // alignment slack + rings + the per-block reservation of the hardware
+    const int n = smem_per_sm / per_block;
+    return n < 1 ? 1 : (n > 4 ? 4 : n);
+}
+
 template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA, int QL = 1>
-int launch_mma_t(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
+int launch_mma_t(const gva_config &cfg, MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
                  int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream, int *n_blocks_out) {
     using T = MmaTraits<DV, DR, TILE, GQA>;
     const int G = cfg.G;
     const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
     auto fn = decode_mma_kernel<DV, DR, TILE, NSTAGE, WPG, GQA, QL>;
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
-    CUtensorMap tm_v, tm_k;
-    const uint64_t vrows = (uint64_t)p.num_pages * G * p.P;
-    if (!encode_map(st, &tm_v, p.v_pool, DV, vrows, 64, TILE, CU_TENSOR_MAP_SWIZZLE_128B)) return GVA_ERR_CUDA;
-    if (GQA) {
-        if (!encode_map(st, &tm_k, p.k_pool, DV, vrows, 64, TILE, CU_TENSOR_MAP_SWIZZLE_128B)) return GVA_ERR_CUDA;
-    } else if (DR == 0) {
-        tm_k = tm_v;      // value-only cache: there is no positional-key tile to describe (the kernel never uses this map)
-    } else {
-        if (!encode_map(st, &tm_k, p.kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, TILE,
-                        DR == 16   ? CU_TENSOR_MAP_SWIZZLE_32B
-                        : DR == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
-                                   : CU_TENSOR_MAP_SWIZZLE_NONE))
-            return GVA_ERR_CUDA;
-    }
+    // the attribute and the occupancy figure are asked for once per (kernel, device, shared-memory size), not per call
+    static int s_smem_set[kMaxDevicesCached] = {}, s_occupancy[kMaxDevicesCached] = {};
+    const int dev = st.device >= 0 && st.device < kMaxDevicesCached ? st.device : 0;
     const int threads = 32 * (G * WPG + 1);
+    if (s_smem_set[dev] != (int)smem || st.device >= kMaxDevicesCached) {
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, smem) != cudaSuccess) return GVA_ERR_CUDA;
+        s_occupancy[dev] = per_sm;
+        s_smem_set[dev] = (int)smem;
+    }
+    const void *kptr = GQA ? p.k_pool : p.kr_pool;
+    const MapPair *mp = st.find(p.v_pool, kptr, p.num_pages, GQA ? 1 : 0);
+    if (!mp) {
+        MapPair *m = st.slot_for(p.v_pool, kptr, p.num_pages, GQA ? 1 : 0);
+        const uint64_t vrows = (uint64_t)p.num_pages * G * p.P;
+        bool ok = encode_map(st, &m->tm_v, p.v_pool, DV, vrows, 64, TILE, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (ok && GQA) {
+            ok = encode_map(st, &m->tm_k, p.k_pool, DV, vrows, 64, TILE, CU_TENSOR_MAP_SWIZZLE_128B);
+        } else if (ok && DR == 0) {
+            m->tm_k = m->tm_v;      // value-only cache: there is no positional-key tile to describe (the kernel never uses this map)
+        } else if (ok) {
+            ok = encode_map(st, &m->tm_k, p.kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, TILE,
+                            DR == 16   ? CU_TENSOR_MAP_SWIZZLE_32B
+                            : DR == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                       : CU_TENSOR_MAP_SWIZZLE_NONE);
+        }
+        if (!ok) {
+            st.forget_last();
+            return GVA_ERR_CUDA;
+        }
+        mp = m;
+    }
     int grid;
     if (num_splits > 0) {
         grid = B * num_splits;
     } else {
-        int per_sm = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, smem) != cudaSuccess) return GVA_ERR_CUDA;
+        int per_sm = s_occupancy[dev];
         per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);
         const long long tiles_ub = (long long)B * ((max_seq_len + TILE - 1) / TILE);
         long long want = (long long)per_sm * sm_count;
-        if (want > max_blocks) want = max_blocks;
+        if (want > max_blocks) want = max_blocks;      // never more blocks than the workspace was sized for
         grid = (int)(tiles_ub < want ? (tiles_ub < 1 ? 1 : tiles_ub) : want);
     }
+    *n_blocks_out = grid;
+    if (st.dry) return GVA_OK;
     DecodeParams pp = p;
     pp.rec_mult = WPG;
-    if (launch_pdl(fn, dim3(grid), dim3(threads), smem, stream, pp, tm_v, tm_k) != cudaSuccess) {
+    if (launch_pdl(fn, dim3(grid), dim3(threads), smem, stream, pp, mp->tm_v, mp->tm_k) != cudaSuccess) {
         (void)cudaGetLastError();
         return GVA_ERR_CUDA;
     }
-    *n_blocks_out = grid;
     return GVA_OK;
 }
 
 template <bool GQA>
-int launch_decode_mma(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p,
+int launch_decode_mma(const gva_config &cfg, MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p,
                       int B, int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream, int *n_blocks_out,
                       int *tile_out, int *rec_mult_out) {
     if (!mma_supported(cfg, GQA)) return GVA_ERR_UNSUPPORTED;
@@ -882,7 +1004,7 @@ int launch_decode_mma(const gva_config &cfg, const MmaHostState &st, int sm_coun
 }
 
 // Multi-token decode (q_len = 2 or 4 new tokens per sequence) on the same kernel: see decode_mma_kernel.
-inline int launch_decode_mma_multi(const gva_config &cfg, const MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p,
+inline int launch_decode_mma_multi(const gva_config &cfg, MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p,
                                    int B, int q_len, int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream,
                                    int *n_blocks_out, int *tile_out, int *rec_mult_out) {
     if (!mma_supported(cfg, false) || q_len < 2 || q_len > 4) return GVA_ERR_UNSUPPORTED;

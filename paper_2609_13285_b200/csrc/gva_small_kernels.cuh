@@ -554,6 +554,7 @@ struct StepFrontParams {
     void *v_pool, *kr_pool;
     int32_t *dev_status;
     int B, H, G, d_v, d_c, d_r, P, num_pages, max_pages, n_absorb;
+    int trace_call;      // number of the decode call this launch belongs to (timeline builds only)
 };
 
 template <typename CT>
@@ -562,6 +563,7 @@ step_front_kernel(StepFrontParams a, RopeTable rope) {
     extern __shared__ float smem_f[];
     grid_dependency_wait();
     grid_dependency_launch();
+    if (threadIdx.x == 0) trace(kTrFrontEnterMin, a.trace_call);
     if ((int)blockIdx.x < a.n_absorb) {
         absorb_block(a.q_c, a.q_r, a.M, a.pos, a.q_abs, a.B, a.H, a.d_v, a.d_c, a.d_r, rope, blockIdx.x % a.H,
                      (blockIdx.x / a.H) * kAbsorbBatch, smem_f);
@@ -570,6 +572,7 @@ step_front_kernel(StepFrontParams a, RopeTable rope) {
                          a.pos, a.G, a.d_v, a.d_r, a.P, a.num_pages, a.max_pages, a.dev_status, rope,
                          blockIdx.x - a.n_absorb);
     }
+    if (threadIdx.x == 0) trace(kTrFrontExitMax, a.trace_call);
 }
 
 // ---- LSE combine ---------------------------------------------------------------------------------
@@ -581,11 +584,10 @@ step_front_kernel(StepFrontParams a, RopeTable rope) {
 // records a sequence can have (many for a single long sequence, few for a large batch).
 //   m* = max_r m_r ;  L = sum_r l_r 2^(m_r - m*) ;  out = sum_r 2^(m_r - m*) o_r / L ;  lse = (m* + log2 L) ln 2
 //
-// The body runs twice: a first, "dry" pass while the block still waits for the decode kernel (reads of the
-// workspace are discarded, nothing is written), then the real pass after the wait.  Both passes execute the
-// same instructions, so the real pass finds them in the SM's instruction cache; a kernel this short otherwise
-// spends most of its time on cold instruction fetches, because the cache stream has pushed its code out of L2
-// since the previous call.
+// The kernel is launched right behind the decode kernel and its blocks become resident while that kernel streams.
+// The body runs twice: a first, "dry" pass over record 0 while the block still waits for the decode kernel (loads
+// discarded, nothing written), then the real pass after the wait.  Both passes execute the same instructions, so the
+// real pass finds them in the SM's instruction cache instead of fetching them cold at the one moment that counts.
 template <int DV>
 __global__ void __launch_bounds__(1024)
 combine_kernel(DecodeParams p, int wph, int hpb) {
@@ -603,27 +605,23 @@ combine_kernel(DecodeParams p, int wph, int hpb) {
     const int part = warp % wph;
     const bool active = h < p.H;
     const int hh = active ? h : 0;
+    if (threadIdx.x == 0) trace(kTrCombineEnterMin, p.epoch);
 
 #pragma unroll 1
-    for (int pass = 0; pass < p.combine_passes; ++pass) {
-        const bool dry = pass + 1 < p.combine_passes;
+    for (int pass = 0; pass < 2; ++pass) {
+        const bool dry = pass == 0;
+        int first = 0, n = 1;                    // dry: record 0 only (always inside the workspace)
         if (!dry) {
             grid_dependency_wait();
-            // the decode kernel is complete: hand the tail-unit ticket back at zero for the next call
-            if (b == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.ticket = 0;
-        }
-        int first, n;
-        if (p.num_splits > 0) {
-            first = b * p.num_splits * p.rec_mult;
-            n = p.num_splits * p.rec_mult;
-        } else {   // this sequence's run of records, worked out by block 0 of the decode kernel
-            const int2 seg = __ldcg(reinterpret_cast<const int2 *>(p.hdr + kHdrInts) + b);
-            first = seg.x * p.rec_mult;
-            n = seg.y * p.rec_mult;
-        }
-        if (dry) {      // whatever the header holds right now, stay inside the workspace
-            first = 0;
-            n = wph * UNROLL < 32 ? wph * UNROLL : 32;
+            if (p.num_splits > 0) {
+                first = b * p.num_splits * p.rec_mult;
+                n = p.num_splits * p.rec_mult;
+            } else {   // this sequence's run of records, worked out by block 0 of the decode kernel
+                const int2 seg = __ldcg(reinterpret_cast<const int2 *>(p.hdr + kHdrInts) + b);
+                first = seg.x;
+                n = seg.y;
+            }
+            if (n < 0 || first < 0 || first + n > p.n_rec) n = 0;      // a header that cannot be right (a decode kernel that gave up): read nothing
         }
         float m_w = -INFINITY, L_w = 0.f, acc[DPL];
 #pragma unroll
@@ -703,6 +701,10 @@ combine_kernel(DecodeParams p, int wph, int hpb) {
 #pragma unroll
             for (int d = 0; d < DPL; ++d) o_dst[d] = live ? o[d] * inv : 0.f;
             if (p.lse && lane == 0) p.lse[(size_t)b * p.H + h] = lse;
+            if (lane == 0) {
+                trace(kTrCombineOutMin, p.epoch);
+                trace(kTrCombineOutMax, p.epoch);
+            }
         }
     }
 }
