@@ -71,12 +71,6 @@ struct PrefillTraits {
     static constexpr int V_BYTES = BOXES * VBOX_BYTES;
     static constexpr int KR_BYTES = TILE * KR_ROW;
     static constexpr int STAGE_BYTES = V_BYTES + ((KR_BYTES + 1023) & ~1023);
-    static constexpr int OFF_QV = 0;
-    static constexpr int OFF_QR = OFF_QV + QV_BYTES;
-    static constexpr int OFF_STAGE = OFF_QR + QR_BYTES;
-    static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
-    static constexpr int N_BARS = 2 * NSTAGE + 9;
-    static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
     // tensor-memory columns: two score buffers (64 each; P overwrites the first 32 of its S), O (DV) and, where it
     // fits (d_v = 64), the query tile Q as bf16 pairs ((DV + DR) / 2): an MMA whose A operand comes from tensor memory
     // reads only B from shared memory (measured: 128 x 64 x 16 MMAs with both operands in shared memory run at 62
@@ -85,6 +79,16 @@ struct PrefillTraits {
     static constexpr int NSBUF = 2;
     static constexpr int COL_S = 0, COL_O = NSBUF * TILE, COL_Q = COL_O + DV;
     static constexpr bool Q_IN_TMEM = COL_Q + (DV + DR) / 2 <= TMEM_COLS;
+    // Shared memory: the query as two bf16 tiles, q = hi + lo (see the kernel).  hi sits in tensor memory where it fits,
+    // else at OFF_QV / OFF_QR; lo always sits in shared memory.
+    static constexpr int OFF_QV = 0;
+    static constexpr int OFF_QR = OFF_QV + QV_BYTES;
+    static constexpr int OFF_LOV = Q_IN_TMEM ? OFF_QV : OFF_QR + QR_BYTES;
+    static constexpr int OFF_LOR = OFF_LOV + QV_BYTES;
+    static constexpr int OFF_STAGE = OFF_LOR + QR_BYTES;
+    static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
+    static constexpr int N_BARS = 2 * NSTAGE + 9;
+    static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
     static_assert(NSBUF * TILE + DV <= TMEM_COLS, "the score buffers and O must fit the allocation");
     static constexpr int BLOCKS_PER_SM = 512 / TMEM_COLS;
     static constexpr int KSTEPS_V = DV / 16, KSTEPS_R = DR / 16;
@@ -148,6 +152,9 @@ __device__ __forceinline__ void tmem_st8_nowait(uint32_t taddr, const uint32_t (
     asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n" ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]),
                  "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
                  : "memory");
+}
+__device__ __forceinline__ void tmem_st4_nowait(uint32_t taddr, const uint32_t (&v)[4]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
@@ -383,45 +390,52 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         // ---- stage Q as bf16: into tensor memory (row = lane, two values per column) or, where that does not fit,
         //      into shared memory as swizzled K-major rows (value dims in 128-byte boxes, then the RoPE dims) ----
         {
+            // q = hi + lo with hi = bf16(q), lo = bf16(q - hi): the score product is taken with both, so the absorbed
+            // query enters with ~16 significant bits and a score of any size is as exact as the cache's own bf16 values
+            // allow (with hi alone a score s is off by about |s| 2^-9, which is what limits accuracy on peaked rows).
             const float4 *src = reinterpret_cast<const float4 *>(p.q_abs + ((size_t)(q_begin + q0 + tok) * p.H + h) * (DV + DR));
-            if constexpr (T::Q_IN_TMEM) {
+            auto split4 = [](const float4 &a, uint32_t &h01, uint32_t &h23, uint32_t &l01, uint32_t &l23) {
+                h01 = pack_bf16(a.x, a.y);
+                h23 = pack_bf16(a.z, a.w);
+                l01 = pack_bf16(a.x - __uint_as_float(h01 << 16), a.y - __uint_as_float(h01 & 0xffff0000u));
+                l23 = pack_bf16(a.z - __uint_as_float(h23 << 16), a.w - __uint_as_float(h23 & 0xffff0000u));
+            };
+            // value dims: 16-byte piece c (8 values) of the row, as swizzled K-major rows in 128-byte boxes; then the RoPE dims
 #pragma unroll
-                for (int part = 0; part < (DV + DR) / 16; ++part) {      // 16 values = 8 columns per step
-                    uint32_t w[8];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (live) a = __ldg(src + part * 4 + c);
-                        w[2 * c] = pack_bf16(a.x, a.y);
-                        w[2 * c + 1] = pack_bf16(a.z, a.w);
-                    }
-                    tmem_st8_nowait(lane_base + T::COL_Q + part * 8, w);
+            for (int c = 0; c < DV / 8; ++c) {
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
+                if (live) {
+                    a = __ldg(src + 2 * c);
+                    bq = __ldg(src + 2 * c + 1);
                 }
+                uint32_t hw[4], lw[4];
+                split4(a, hw[0], hw[1], lw[0], lw[1]);
+                split4(bq, hw[2], hw[3], lw[2], lw[3]);
+                const uint32_t off = (c >> 3) * T::QBOX_BYTES + swz128(r, c & 7);
+                *reinterpret_cast<uint4 *>(smem + T::OFF_LOV + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                if constexpr (!T::Q_IN_TMEM) *reinterpret_cast<uint4 *>(smem + T::OFF_QV + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                else tmem_st4_nowait(lane_base + T::COL_Q + c * 4, hw);
+            }
+#pragma unroll
+            for (int c = 0; c < DR / 8; ++c) {
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
+                if (live) {
+                    a = __ldg(src + DV / 4 + 2 * c);
+                    bq = __ldg(src + DV / 4 + 2 * c + 1);
+                }
+                uint32_t hw[4], lw[4];
+                split4(a, hw[0], hw[1], lw[0], lw[1]);
+                split4(bq, hw[2], hw[3], lw[2], lw[3]);
+                const uint32_t off = swz_kr<T::KR_ROW>(r, c);
+                *reinterpret_cast<uint4 *>(smem + T::OFF_LOR + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                if constexpr (!T::Q_IN_TMEM) *reinterpret_cast<uint4 *>(smem + T::OFF_QR + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                else tmem_st4_nowait(lane_base + T::COL_Q + DV / 2 + c * 4, hw);
+            }
+            if constexpr (T::Q_IN_TMEM) {
                 tmem_st_wait();
                 tc_fence_before();
-            } else {
-#pragma unroll
-                for (int c = 0; c < DV / 8; ++c) {
-                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
-                    if (live) {
-                        a = __ldg(src + 2 * c);
-                        bq = __ldg(src + 2 * c + 1);
-                    }
-                    *reinterpret_cast<uint4 *>(smem + T::OFF_QV + (c >> 3) * T::QBOX_BYTES + swz128(r, c & 7)) =
-                        make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(bq.x, bq.y), pack_bf16(bq.z, bq.w));
-                }
-#pragma unroll
-                for (int c = 0; c < DR / 8; ++c) {
-                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
-                    if (live) {
-                        a = __ldg(src + DV / 4 + 2 * c);
-                        bq = __ldg(src + DV / 4 + 2 * c + 1);
-                    }
-                    *reinterpret_cast<uint4 *>(smem + T::OFF_QR + swz_kr<T::KR_ROW>(r, c)) =
-                        make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(bq.x, bq.y), pack_bf16(bq.z, bq.w));
-                }
-                fence_async_smem();
             }
+            fence_async_smem();
             mbar_arrive(q_ready);
         }
 
@@ -590,6 +604,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             constexpr uint32_t lo_k = (16u >> 4) << 16;                                           // LBO 16 (K-major operands)
             constexpr uint32_t lo_mn = ((uint32_t)T::VBOX_BYTES >> 4) << 16;                      // LBO = box stride (MN-major value tile)
             const uint32_t a_qv = ((s_base + T::OFF_QV) & 0x3FFFFu) >> 4, a_qr = ((s_base + T::OFF_QR) & 0x3FFFFu) >> 4;
+            const uint32_t a_lov = ((s_base + T::OFF_LOV) & 0x3FFFFu) >> 4, a_lor = ((s_base + T::OFF_LOR) & 0x3FFFFu) >> 4;
             const uint32_t a_st = ((s_base + T::OFF_STAGE) & 0x3FFFFu) >> 4;
             auto mk = [](uint32_t lo, uint32_t hi) { return (uint64_t)lo | ((uint64_t)hi << 32); };
             constexpr int KS_S = T::KSTEPS_V + T::KSTEPS_R, KS_O = T::TILE / 16;
@@ -616,6 +631,18 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                             const uint32_t kr = (uint32_t)(ks - T::KSTEPS_V) * 2;
                             if constexpr (T::Q_IN_TMEM) umma_bf16_ts(d, tmem + T::COL_Q + ks * 8, mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
                             else umma_bf16(d, mk((a_qr + kr) | lo_k, hikr), mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
+                        }
+                    }
+                    // ... and the same k-steps again with the low-order halves of the query (always from shared memory)
+#pragma unroll
+                    for (int ks = 0; ks < KS_S; ++ks) {
+                        if (ks < T::KSTEPS_V) {
+                            const uint32_t off = ((ks >> 2) * T::QBOX_BYTES + (ks & 3) * 32) >> 4;
+                            const uint32_t voff = ((ks >> 2) * T::VBOX_BYTES + (ks & 3) * 32) >> 4;
+                            umma_bf16(d, mk((a_lov + off) | lo_k, hi128), mk((vb + voff) | lo_k, hi128), idesc_s, 1);
+                        } else {
+                            const uint32_t kr = (uint32_t)(ks - T::KSTEPS_V) * 2;
+                            umma_bf16(d, mk((a_lor + kr) | lo_k, hikr), mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
                         }
                     }
                     umma_commit(s_full(t % NB));

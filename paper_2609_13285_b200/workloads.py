@@ -35,9 +35,20 @@ MASTER_SEED = 20260913
 # ----------------------------------------------------------------------------
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """Round float32 values to bfloat16 (nearest, ties to even); returns uint16 bit patterns."""
-    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
-    r = (u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))) >> np.uint32(16)
-    return r.astype(np.uint16)
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).reshape(-1)
+    out = np.empty(u.shape, dtype=np.uint16)
+    blk = 1 << 20                                   # small blocks: the temporaries stay in cache and are reused
+    t = np.empty(min(blk, max(u.size, 1)), dtype=np.uint32)
+    for lo in range(0, u.size, blk):
+        hi = min(u.size, lo + blk)
+        tv = t[:hi - lo]
+        np.right_shift(u[lo:hi], np.uint32(16), out=tv)
+        np.bitwise_and(tv, np.uint32(1), out=tv)
+        np.add(tv, np.uint32(0x7FFF), out=tv)
+        np.add(tv, u[lo:hi], out=tv)
+        np.right_shift(tv, np.uint32(16), out=tv)
+        out[lo:hi] = tv
+    return out.reshape(np.shape(x))
 
 
 def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
@@ -155,18 +166,34 @@ def _rng(seed: int) -> np.random.Generator:
 
 
 def _normal_pool(rng: np.random.Generator, shape, cache_dtype: str, chunk_elems: int = 1 << 25) -> np.ndarray:
-    """N(0,1) pool in storage dtype, generated in slabs so the f32 temporary stays small."""
+    """N(0,1) pool in storage dtype, generated in slabs so the f32 temporary stays small.
+
+    A pool of more than one slab is drawn slab by slab from independent streams -- slab k from the caller's Philox
+    generator jumped k + 1 times (2^128 draws apart each) -- on a few threads; a pool of one slab is drawn from the
+    caller's generator itself."""
     n = int(np.prod(shape))
-    if cache_dtype == "f32":
+    if cache_dtype == "f32" and n <= chunk_elems:
         return rng.standard_normal(n, dtype=np.float32).reshape(shape)
     fp8 = cache_dtype == "fp8"
-    out = np.empty(n, dtype=np.uint8 if fp8 else np.uint16)
+    out = np.empty(n, dtype=np.float32 if cache_dtype == "f32" else (np.uint8 if fp8 else np.uint16))
     if fp8:
         chunk_elems = min(chunk_elems, 1 << 22)         # the e4m3 cast works in float64 temporaries
-    for lo in range(0, n, chunk_elems):
-        hi = min(n, lo + chunk_elems)
-        draw = rng.standard_normal(hi - lo, dtype=np.float32)
-        out[lo:hi] = f32_to_e4m3_bits(draw) if fp8 else f32_to_bf16_bits(draw)
+    cast = (lambda d: d) if cache_dtype == "f32" else (f32_to_e4m3_bits if fp8 else f32_to_bf16_bits)
+    if n <= chunk_elems:
+        out[:] = cast(rng.standard_normal(n, dtype=np.float32))
+        return out.reshape(shape)
+    slabs = [(k, lo, min(n, lo + chunk_elems)) for k, lo in enumerate(range(0, n, chunk_elems))]
+    base = rng.bit_generator
+
+    def fill(job):
+        k, lo, hi = job
+        sub = np.random.Generator(base.jumped(k + 1))
+        out[lo:hi] = cast(sub.standard_normal(hi - lo, dtype=np.float32))
+
+    from concurrent.futures import ThreadPoolExecutor
+    import os
+    with ThreadPoolExecutor(max_workers=max(1, min(8, len(os.sched_getaffinity(0))))) as pool:
+        list(pool.map(fill, slabs))
     return out.reshape(shape)
 
 

@@ -1,5 +1,6 @@
-"""Parity at the benchmark's full sizes, in the launch configuration bench.py times: the oracle
-evaluates a sample of sequences one by one; Gaussian-tilting statistics cover the rest."""
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.  The decode workloads are
+compared with the oracle on every sequence of the batch (and, for the 24-layer workload, on every layer), through the
+three separate calls and through the fused step; the prefill and multi-token workloads on sampled rows."""
 import numpy as np
 import pytest
 import torch
@@ -17,7 +18,9 @@ def _built():
     gpu_util.ensure_built()
 
 
-def _sampled_check(case, kernel, sample):
+def _whole_batch_check(case, kernel):
+    """absorb -> decode and the fused step on every sequence of the batch, against the oracle fed the GPU's own
+    absorbed queries (tight gates), plus the Gaussian-tilting statistic on the long sequences."""
     from tests import gpu_util as U
     dc = harness.upload(case, kernel=kernel)
     try:
@@ -26,20 +29,35 @@ def _sampled_check(case, kernel, sample):
         torch.cuda.synchronize()
         assert int(dc.status.item()) == 0
         o = out.cpu().numpy().astype(np.float64)
+        l = lse.cpu().numpy().astype(np.float64)
         assert np.isfinite(o).all()
-        lens = np.zeros_like(case.seq_lens)
-        lens[sample] = case.seq_lens[sample]
-        ref, ref_lse = U.oracle_for_gpu_q(case, dc.q_abs, seq_lens=lens)
-        err = np.max(np.abs(o[sample] - ref[sample]))
+        ref, ref_lse = U.oracle_for_gpu_q(case, dc.q_abs)
+        err = np.max(np.abs(o - ref))
         assert err <= U.TOL_TIGHT_MAXABS, err
-        assert U.rel_l2(o[sample], ref[sample]) <= U.TOL_TIGHT_REL_L2
+        assert U.rel_l2(o, ref) <= U.TOL_TIGHT_REL_L2
+        assert np.max(np.abs(l - ref_lse)) <= 1e-4 * max(1.0, np.max(np.abs(ref_lse)))
         # every sequence: the softmax-weighted mean of N(0, I) rows sits near q~ / sqrt(d_qk)
         s = case.shape
         q = dc.q_abs.cpu().numpy().astype(np.float64)
         target = q[..., :s.d_v] / np.sqrt(s.d_c + s.d_r)
         long_enough = np.asarray(case.seq_lens) >= 4096
         assert np.max(np.abs(o[long_enough] - target[long_enough])) < 0.2
-        return gb.gva_last_num_splits(dc.handle)
+        n_blocks = gb.gva_last_num_splits(dc.handle)
+        # the call bench.py times: the fused step (append position = last attended token; the appended row differs
+        # from the generated one, so the oracle appends too before it attends)
+        from oracle import gva_oracle as orc
+        out1 = out.clone()
+        out2, _ = dc.step()
+        torch.cuda.synchronize()
+        assert int(dc.status.item()) == 0
+        v_gpu, k_gpu = dc.pools_to_host()
+        assert orc.append_case(case) == 0
+        assert np.array_equal(v_gpu, case.v_pool) and np.array_equal(k_gpu, case.kr_pool)       # bit-exact append, whole pool
+        ref2, _ = U.oracle_for_gpu_q(case, dc.q_abs)
+        o2 = out2.cpu().numpy().astype(np.float64)
+        assert np.max(np.abs(o2 - ref2)) <= U.TOL_TIGHT_MAXABS
+        assert not torch.equal(out1, out2)                  # (the step really attended the newly appended rows)
+        return n_blocks
     finally:
         dc.close()
 
@@ -57,39 +75,52 @@ def _auto_kernel():
     return gb.GVA_KERNEL_AUTO
 
 
-def test_config2_long_context_paged_sampled():
-    _sampled_check(wl.config2(), _auto_kernel(), [0, 17, 31])
+def test_config2_long_context_paged_whole_batch():
+    case = wl.config2()
+    case.append_pos[:] = case.seq_lens - 1          # the step appends at the last attended position (Algorithm 1's order)
+    case.q_pos[:] = case.seq_lens - 1
+    _whole_batch_check(case, _auto_kernel())
 
 
-def test_config3_ragged_wide_heads_sampled():
+def test_config3_ragged_wide_heads_whole_batch():
     case = wl.config3(poison=True)
-    order = np.argsort(case.seq_lens)
-    _sampled_check(case, _auto_kernel(), [int(order[0]), int(order[len(order) // 2]), int(order[-1])])
+    case.append_pos[:] = case.seq_lens - 1
+    case.q_pos[:] = case.seq_lens - 1
+    _whole_batch_check(case, _auto_kernel())
 
 
-def test_config4_two_layers_full_batch():
+def test_config4_every_layer_whole_batch():
+    # the 24-layer step, one layer on the host at a time: bit-exact append on every layer (whole pool), every
+    # sequence's output against the oracle end to end (the oracle's own fp64 absorbed query), first through the three
+    # separate calls, then through the fused step, whose outputs must equal the three calls' bit for bit
     from oracle import gva_oracle as orc
-    from tests import gpu_util as U
-    for layer in (0, 23):
+    for layer in range(wl.CONFIG4_LAYERS):
         case = wl.config4_layer(layer)
         dc = harness.upload(case, kernel=_auto_kernel())
         try:
             dc.absorb()
             dc.append()
-            out, _ = dc.decode()
+            out, lse = dc.decode()
             torch.cuda.synchronize()
-            assert int(dc.status.item()) == 0
+            assert int(dc.status.item()) == 0, layer
             v_gpu, k_gpu = dc.pools_to_host()
             assert orc.append_case(case) == 0
-            assert np.array_equal(v_gpu, case.v_pool) and np.array_equal(k_gpu, case.kr_pool)   # bit-exact append
-            sample = [0, 64, 127]
-            lens = np.zeros_like(case.seq_lens)
-            lens[sample] = case.seq_lens[sample]
-            ref, _ = orc.decode_case(case, seq_lens=lens)       # oracle's own fp64 absorbed query: end to end
+            assert np.array_equal(v_gpu, case.v_pool) and np.array_equal(k_gpu, case.kr_pool), layer   # bit-exact append
+            ref, ref_lse = orc.decode_case(case)                # oracle's own fp64 absorbed query: end to end
             o = out.cpu().numpy().astype(np.float64)
-            assert np.max(np.abs(o[sample] - ref[sample])) <= 5e-5
+            assert np.max(np.abs(o - ref)) <= 5e-5, layer
+            assert np.max(np.abs(lse.cpu().numpy().astype(np.float64) - ref_lse)) <= 1e-4 * max(1.0, np.max(np.abs(ref_lse))), layer
+            q1, o1, l1 = dc.q_abs.clone(), out.clone(), lse.clone()
+            dc.q_abs.fill_(float("nan")); dc.out.fill_(float("nan")); dc.lse.fill_(float("nan"))
+            out2, lse2 = dc.step()                              # appends the same rows again: the pools must not change
+            torch.cuda.synchronize()
+            assert int(dc.status.item()) == 0, layer
+            assert torch.equal(dc.q_abs, q1) and torch.equal(out2, o1) and torch.equal(lse2, l1), layer
+            v2, k2 = dc.pools_to_host()
+            assert np.array_equal(v2, case.v_pool) and np.array_equal(k2, case.kr_pool), layer
         finally:
             dc.close()
+        del case
 
 
 @pytest.mark.parametrize("shape_name", ["A", "B"])
