@@ -659,7 +659,10 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 
         } else {
             // ================= multi-token decode: QL new tokens per sequence, columns = slot * 4 + head =================
-            uint32_t qf[T::KSTEPS][NBK][2];   // B fragments of Q^T (plain bf16): column n = lane / 4 of N-block nb
+            // B fragments of Q^T: column n = lane / 4 of N-block nb.  The f32 query goes in as two bf16 numbers, q = hi + lo, and
+            // the score product is taken with both (twice the score MMAs): with hi alone a score s is off by about |s| 2^-9,
+            // which on sharply peaked rows is what limits the accuracy of the output.
+            uint32_t qf[T::KSTEPS][NBK][2], qlo[T::KSTEPS][NBK][2];
             float oacc[T::MT][NBK][4];
             float m_run[NBK][2], l_run[NBK][2];   // per column of this lane: columns 2 jh, 2 jh + 1 of every N-block
             const float scale = p.scale_log2;
@@ -676,9 +679,11 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                         for (int half = 0; half < 2; ++half) {
                             float2 v = *reinterpret_cast<const float2 *>(q + kk * 16 + half * 8 + 2 * jh);
                             if (!present) v = make_float2(0.f, 0.f);
-                            uint32_t w;
+                            uint32_t w, wl;
                             asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(w) : "f"(v.y), "f"(v.x));
+                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(wl) : "f"(v.y - __uint_as_float(w & 0xffff0000u)), "f"(v.x - __uint_as_float(w << 16)));
                             qf[kk][nb][half] = w;
+                            qlo[kk][nb][half] = wl;
                         }
                 }
             };
@@ -750,15 +755,20 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                         uint32_t a[4];
                         ldsm_x4(vt_u32 + (kk >> 2) * T::VBOX_BYTES + c * 2048 + (off_qk ^ ((kk & 3) << 5)), a);
 #pragma unroll
-                        for (int nb = 0; nb < NBK; ++nb) mma_bf16(sacc[c][nb], a, qf[kk][nb][0], qf[kk][nb][1]);
+                        for (int nb = 0; nb < NBK; ++nb) {
+                            mma_bf16(sacc[c][nb], a, qlo[kk][nb][0], qlo[kk][nb][1]);
+                            mma_bf16(sacc[c][nb], a, qf[kk][nb][0], qf[kk][nb][1]);
+                        }
                     }
 #pragma unroll
                     for (int kk = 0; kk < T::KSTEPS_R; ++kk) {
                         uint32_t a[4];
                         ldsm_x4(kr_u32 + c * 16 * T::KR_ROW + (off_kr ^ (kk << 5)), a);
 #pragma unroll
-                        for (int nb = 0; nb < NBK; ++nb)
+                        for (int nb = 0; nb < NBK; ++nb) {
+                            mma_bf16(sacc[c][nb], a, qlo[T::KSTEPS_V + kk][nb][0], qlo[T::KSTEPS_V + kk][nb][1]);
                             mma_bf16(sacc[c][nb], a, qf[T::KSTEPS_V + kk][nb][0], qf[T::KSTEPS_V + kk][nb][1]);
+                        }
                     }
                 }
                 // ---- online softmax per column: this lane holds columns 2 jh, 2 jh + 1 of every N-block at token rows
