@@ -71,21 +71,23 @@ struct PrefillTraits {
     static constexpr int V_BYTES = BOXES * VBOX_BYTES;
     static constexpr int KR_BYTES = TILE * KR_ROW;
     static constexpr int STAGE_BYTES = V_BYTES + ((KR_BYTES + 1023) & ~1023);
-    // tensor-memory columns: two score buffers (64 each; P overwrites the first 32 of its S), O (DV) and, where it
-    // fits (d_v = 64), the query tile Q as bf16 pairs ((DV + DR) / 2): an MMA whose A operand comes from tensor memory
-    // reads only B from shared memory (measured: 128 x 64 x 16 MMAs with both operands in shared memory run at 62
-    // cycles each -- the 6 KB of operands per MMA at ~97 B/clk -- against 32 with A in tensor memory)
-    static constexpr int TMEM_COLS = 256;
+    // Tensor-memory columns: two score buffers (64 each; P overwrites the first 32 of its S), O (DV), and the query as bf16
+    // pairs -- q = hi + lo, (DV + DR) / 2 columns each: an MMA whose A operand comes from tensor memory reads only B
+    // from shared memory (measured: 128 x 64 x 16 MMAs with both operands in shared memory run at 62 cycles each -- the
+    // 6 KB of operands per MMA at ~97 B/clk -- against 32 with A in tensor memory).  d_v = 64: two blocks per SM with 256
+    // columns each hold hi; lo (40 more columns) does not fit and sits in shared memory.  d_v = 128: the stages alone
+    // allow one block per SM, which then takes all 512 columns and holds hi and lo.
+    static constexpr int TMEM_COLS = DV == 64 ? 256 : 512;
     static constexpr int NSBUF = 2;
-    static constexpr int COL_S = 0, COL_O = NSBUF * TILE, COL_Q = COL_O + DV;
+    static constexpr int COL_S = 0, COL_O = NSBUF * TILE, COL_Q = COL_O + DV, COL_QLO = COL_Q + (DV + DR) / 2;
     static constexpr bool Q_IN_TMEM = COL_Q + (DV + DR) / 2 <= TMEM_COLS;
-    // Shared memory: the query as two bf16 tiles, q = hi + lo (see the kernel).  hi sits in tensor memory where it fits,
-    // else at OFF_QV / OFF_QR; lo always sits in shared memory.
+    static constexpr bool LO_IN_TMEM = Q_IN_TMEM && COL_QLO + (DV + DR) / 2 <= TMEM_COLS;
+    // Shared memory: whichever of hi (OFF_QV / OFF_QR) and lo (OFF_LOV / OFF_LOR) is not in tensor memory.
     static constexpr int OFF_QV = 0;
-    static constexpr int OFF_QR = OFF_QV + QV_BYTES;
-    static constexpr int OFF_LOV = Q_IN_TMEM ? OFF_QV : OFF_QR + QR_BYTES;
-    static constexpr int OFF_LOR = OFF_LOV + QV_BYTES;
-    static constexpr int OFF_STAGE = OFF_LOR + QR_BYTES;
+    static constexpr int OFF_QR = OFF_QV + (Q_IN_TMEM ? 0 : QV_BYTES);
+    static constexpr int OFF_LOV = OFF_QR + (Q_IN_TMEM ? 0 : QR_BYTES);
+    static constexpr int OFF_LOR = OFF_LOV + (LO_IN_TMEM ? 0 : QV_BYTES);
+    static constexpr int OFF_STAGE = OFF_LOR + (LO_IN_TMEM ? 0 : QR_BYTES);
     static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
     static constexpr int N_BARS = 2 * NSTAGE + 9;
     static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
@@ -412,7 +414,8 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                 split4(a, hw[0], hw[1], lw[0], lw[1]);
                 split4(bq, hw[2], hw[3], lw[2], lw[3]);
                 const uint32_t off = (c >> 3) * T::QBOX_BYTES + swz128(r, c & 7);
-                *reinterpret_cast<uint4 *>(smem + T::OFF_LOV + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                if constexpr (!T::LO_IN_TMEM) *reinterpret_cast<uint4 *>(smem + T::OFF_LOV + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                else tmem_st4_nowait(lane_base + T::COL_QLO + c * 4, lw);
                 if constexpr (!T::Q_IN_TMEM) *reinterpret_cast<uint4 *>(smem + T::OFF_QV + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
                 else tmem_st4_nowait(lane_base + T::COL_Q + c * 4, hw);
             }
@@ -427,7 +430,8 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                 split4(a, hw[0], hw[1], lw[0], lw[1]);
                 split4(bq, hw[2], hw[3], lw[2], lw[3]);
                 const uint32_t off = swz_kr<T::KR_ROW>(r, c);
-                *reinterpret_cast<uint4 *>(smem + T::OFF_LOR + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                if constexpr (!T::LO_IN_TMEM) *reinterpret_cast<uint4 *>(smem + T::OFF_LOR + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                else tmem_st4_nowait(lane_base + T::COL_QLO + DV / 2 + c * 4, lw);
                 if constexpr (!T::Q_IN_TMEM) *reinterpret_cast<uint4 *>(smem + T::OFF_QR + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
                 else tmem_st4_nowait(lane_base + T::COL_Q + DV / 2 + c * 4, hw);
             }
@@ -633,16 +637,18 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                             else umma_bf16(d, mk((a_qr + kr) | lo_k, hikr), mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
                         }
                     }
-                    // ... and the same k-steps again with the low-order halves of the query (always from shared memory)
+                    // ... and the same k-steps again with the low-order halves of the query
 #pragma unroll
                     for (int ks = 0; ks < KS_S; ++ks) {
                         if (ks < T::KSTEPS_V) {
                             const uint32_t off = ((ks >> 2) * T::QBOX_BYTES + (ks & 3) * 32) >> 4;
                             const uint32_t voff = ((ks >> 2) * T::VBOX_BYTES + (ks & 3) * 32) >> 4;
-                            umma_bf16(d, mk((a_lov + off) | lo_k, hi128), mk((vb + voff) | lo_k, hi128), idesc_s, 1);
+                            if constexpr (T::LO_IN_TMEM) umma_bf16_ts(d, tmem + T::COL_QLO + ks * 8, mk((vb + voff) | lo_k, hi128), idesc_s, 1);
+                            else umma_bf16(d, mk((a_lov + off) | lo_k, hi128), mk((vb + voff) | lo_k, hi128), idesc_s, 1);
                         } else {
                             const uint32_t kr = (uint32_t)(ks - T::KSTEPS_V) * 2;
-                            umma_bf16(d, mk((a_lor + kr) | lo_k, hikr), mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
+                            if constexpr (T::LO_IN_TMEM) umma_bf16_ts(d, tmem + T::COL_QLO + ks * 8, mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
+                            else umma_bf16(d, mk((a_lor + kr) | lo_k, hikr), mk((vb + (T::V_BYTES >> 4) + kr) | lo_k, hikr), idesc_s, 1);
                         }
                     }
                     umma_commit(s_full(t % NB));
