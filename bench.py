@@ -32,10 +32,14 @@ if ROOT not in sys.path:
 METRIC = "gva_decode_cache_read_bandwidth"
 UNIT = "GB/s"
 
-# DRAM traffic of one decode-kernel launch on cfg2 at full size, from ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum, mean of two launches; profiles/decode_mma_kernel_cfg2.md).
-NCU_TRAFFIC_BYTES = {"cfg2": 0.5 * ((571_105_024 + 4_873_216) + (571_087_360 + 387_584)),
-                     "cfg2-fp8": 0.5 * ((285_778_688 + 3_652_864) + (285_774_592 + 776_192))}
+# DRAM traffic of one decode-kernel launch at full size, from ncu (dram__bytes_read.sum + dram__bytes_write.sum, mean of
+# two launches).  A profiler figure cannot be taken inside a timed run: the numbers are those of the named profile,
+# which was captured with the kernels as they are in this tree; the line says where they come from.
+NCU_TRAFFIC = {"cfg2": (0.5 * ((571_105_024 + 4_873_216) + (571_087_360 + 387_584)), "profiles/decode_mma_kernel_cfg2.md"),
+               "cfg2-fp8": (0.5 * ((285_778_688 + 3_652_864) + (285_774_592 + 776_192)), "profiles/decode_fp8_kernel_cfg2.md")}
+NOMINAL_HBM_GBPS = 8000.0          # the ~8 TB/s the target quotes (context; the roofline denominator is the measured copy rate)
+MIN_TIMED_WALL_S = 0.5             # every timed loop runs at least this long ...
+MIN_REPEATS = 5                    # ... and at least this many repeats of exactly --steps calls each
 
 
 def load_peaks():
@@ -188,13 +192,22 @@ def oracle_sample(case, n_seq: int):
 
 
 def cpu_baseline(case, budget_s: float = 12.0) -> dict:
-    """The oracle as it stands, timed on this host's cores on a bounded sample of the workload."""
+    """The oracle as it stands, timed on this host's cores on a bounded sample of the workload; the same oracle on one
+    thread beside it."""
+    from oracle import gva_oracle as orc
     dt1, _, threads = oracle_sample(case, 1)
     n = int(max(1, min(case.B, budget_s / max(dt1, 1e-3))))
     dt, nbytes, threads = oracle_sample(case, n)
+    orc.set_threads(1)
+    try:
+        dts, nbs, _ = oracle_sample(case, 1)
+    finally:
+        orc.set_threads(threads)
     return {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"fp64 two-pass oracle (absorb + decode) on the first {n} of {case.B} sequences of the same "
-                      f"workload, {nbytes} cache bytes in {dt:.2f} s"}
+                      f"workload, {nbytes} cache bytes in {dt:.2f} s",
+            "single_thread": {"value": nbs / dts / 1e9, "unit": UNIT, "cores": 1,
+                              "sample": f"the same oracle on one thread, first sequence only: {nbs} cache bytes in {dts:.2f} s"}}
 
 
 def run_reference(args) -> None:
@@ -222,6 +235,72 @@ def run_reference(args) -> None:
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+def timed_repeats(torch, stream, fn, steps: int, sync, min_wall_s: float = MIN_TIMED_WALL_S, min_repeats: int = MIN_REPEATS,
+                  max_repeats: int = 4000):
+    """Times `fn(i)` in repeats of exactly `steps` back-to-back calls each, CUDA events on the launching stream at every
+    repeat boundary; keeps going until at least `min_repeats` repeats and `min_wall_s` seconds of timed device work are
+    in.  `sync()` (barrier + device synchronise) brackets each batch of repeats.  Returns the per-call milliseconds of
+    every repeat."""
+    per_call, i = [], 0
+
+    def batch(n_rep: int):
+        nonlocal i
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_rep + 1)]
+        sync()
+        evs[0].record(stream)
+        for r in range(n_rep):
+            for _ in range(steps):
+                fn(i)
+                i += 1
+            evs[r + 1].record(stream)
+        sync()
+        per_call.extend(evs[r].elapsed_time(evs[r + 1]) / steps for r in range(n_rep))
+
+    batch(min_repeats)
+    done_s = sum(per_call) * steps * 1e-3
+    while done_s < min_wall_s and len(per_call) < max_repeats:
+        per_rep = max(done_s / len(per_call), 1e-6)
+        n_more = int(min(max_repeats - len(per_call), 200, max(1, np.ceil((min_wall_s - done_s) / per_rep))))
+        batch(n_more)
+        done_s = sum(per_call) * steps * 1e-3
+    return per_call
+
+
+def read_ceiling(torch, stream, dev, nbytes: int, steps: int, sync):
+    """Read-only streaming rate of this GPU over `nbytes` bytes (two buffers alternate, as the pool copies do), measured
+    with the probe kernel of csrc/stream_probe.cu under the same repeat protocol.  None if the probe is not built."""
+    import ctypes
+    from paper_2609_13285_b200 import build as gbuild
+    try:
+        lib = ctypes.CDLL(gbuild.build_probe())
+    except Exception:
+        return None
+    lib.gva_probe_stream_read.argtypes = [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p]
+    lib.gva_probe_stream_read.restype = ctypes.c_int
+    nbytes = (nbytes // 32768) * 32768
+    bufs = torch.zeros((2, nbytes), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def call(i: int):
+        if lib.gva_probe_stream_read(bufs[i & 1].data_ptr(), nbytes, status.data_ptr(), stream.cuda_stream) != 0:
+            raise RuntimeError("stream probe launch failed")
+
+    for i in range(5):
+        call(i)
+    ms = timed_repeats(torch, stream, call, steps, sync)
+    ok = int(status.item()) == 0
+    del bufs
+    torch.cuda.empty_cache()
+    if not ok:
+        return None
+    med = float(np.median(ms))
+    return {"GBps": nbytes / (med * 1e-3) / 1e9, "GBps_best": nbytes / (min(ms) * 1e-3) / 1e9, "bytes": nbytes,
+            "ms_per_read": med, "repeats": len(ms),
+            "kernel": "stream_read_kernel (csrc/stream_probe.cu): 32 KB bulk copies into a 3-stage shared-memory ring, "
+                      "2 blocks per SM, evict-first, no arithmetic"}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -310,29 +389,18 @@ def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with
         multirank.barrier(dist)
         torch.cuda.synchronize()
 
-    def timed(fn, n):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for i in range(n):
-            fn(i)
-        b.record(stream)
-        return a, b
-
     for i in range(warmup):
         step(i)
     sync_all()
     sampler = ClockSampler(physical_gpu_index(local_rank)) if with_clocks else None
     if sampler:
         sampler.start()
-    ev0, ev1 = timed(step, steps)                     # K whole steps between two events
-    sync_all()
-    step_ms = ev0.elapsed_time(ev1) / steps
+    step_all = timed_repeats(torch, stream, step, steps, sync_all)             # repeats of exactly K whole steps
     for i in range(warmup):
         decode_only(i)
-    sync_all()
-    d0, d1 = timed(decode_only, steps)                # the dominant kernel: K gva_decode calls back to back
-    sync_all()
+    dec_all = timed_repeats(torch, stream, decode_only, steps, sync_all)       # the dominant kernel: K gva_decode calls back to back
     clocks = sampler.finish() if sampler else None
+    step_ms, decode_ms = float(np.median(step_all)), float(np.median(dec_all)) / n_layers
     # Small workloads are bound by the host's launch rate when launched one call at a time: replay the same steps from a
     # CUDA graph as well (programmatic dependent launches survive capture) to show the device-side time per step.
     graph_ms = None
@@ -353,7 +421,9 @@ def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with
         torch.cuda.synchronize()
         graph_ms = a.elapsed_time(b) / (reps * n_rep)
         del g
-    res = {"case": case, "layers": n_layers, "step_ms": step_ms, "decode_ms": d0.elapsed_time(d1) / steps / n_layers,
+    res = {"case": case, "layers": n_layers, "step_ms": step_ms, "decode_ms": decode_ms,
+           "step_ms_min": float(min(step_all)), "decode_ms_min": float(min(dec_all)) / n_layers,
+           "step_repeats": len(step_all), "decode_repeats": len(dec_all),
            "graph_step_ms": graph_ms,
            "steps": steps, "warmup": warmup, "clocks": clocks, "status": int(dc.status.item()),
            "partitions": gb.gva_last_num_splits(dc.handle),
@@ -362,7 +432,7 @@ def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with
 
     if with_e2e and case.shape.d_r == 0:
         # the host-buffer entry point is not built for the value-only cache: report the device-timed step
-        res.update(e2e_ms=step_ms, e2e_matches=None, h2d=0, d2h=0)
+        res.update(e2e_ms=step_ms, e2e_ms_min=res["step_ms_min"], e2e_repeats=0, e2e_matches=None, h2d=0, d2h=0)
     elif with_e2e:
         # end to end: host buffers in, host buffer out, through the C ABI (one call per step, then a sync)
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
@@ -379,11 +449,10 @@ def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with
 
         for i in range(warmup):
             e2e_step(i)
-        sync_all()
-        t0 = time.perf_counter()
-        e0, e1 = timed(e2e_step, steps)
-        sync_all()
-        res["e2e_ms"] = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / steps
+        e2e_all = timed_repeats(torch, stream, e2e_step, steps, sync_all)
+        res["e2e_ms"] = float(np.median(e2e_all))
+        res["e2e_ms_min"] = float(min(e2e_all))
+        res["e2e_repeats"] = len(e2e_all)
         res["h2d"] = sum(t.numel() * t.element_size() for t in (h_qc, h_qr, h_vn, h_kn, h_pos, h_len))
         res["d2h"] = h_out.numel() * 4
         step(steps - 1)
@@ -392,6 +461,8 @@ def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with
     dc.close()
     del keep, layers
     torch.cuda.empty_cache()
+    if with_e2e:      # the headline workload: the read-only ceiling over the same number of bytes, in the same run
+        res["read_ceiling"] = read_ceiling(torch, stream, dev, case.cache_bytes(), steps, sync_all)
     return res
 
 
@@ -413,17 +484,14 @@ def measure_gqa(rank, local_rank, dist, args, kernel, torch, gb, harness):
     def call(i):
         gb.gqa_decode(dc.handle, caches[i & 1], dc.q, dc.seq_lens, dc.out, dc.lse, ws, B, max_len, 0, dc.status)
 
+    def sync_all():
+        multirank.barrier(dist)
+        torch.cuda.synchronize()
+
     for i in range(warmup):
         call(i)
-    multirank.barrier(dist)
-    torch.cuda.synchronize()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    for i in range(steps):
-        call(i)
-    b.record(stream)
-    torch.cuda.synchronize()
-    ms = a.elapsed_time(b) / steps
+    all_ms = timed_repeats(torch, stream, call, steps, sync_all, min_wall_s=0.25)
+    ms = float(np.median(all_ms))
     nbytes = 2 * int(g["seq_lens"].astype(np.int64).sum()) * g["G"] * g["d_h"] * 2
     res = {"workload": "matched GQA decode: H=16, G=4, d_h=64, B=32, T=32768, bf16 K and V in 64-token pages",
            "gqa_decode_ms_per_call": ms, "cache_bytes_per_call": nbytes, "cache_read_GBps": nbytes / (ms * 1e-3) / 1e9,
@@ -465,17 +533,14 @@ def measure_layer(rank, local_rank, dist, args, kernel, torch, gb, harness):
         gb.gva_layer_step(dc.handle, caches[i & 1], x, W_in, W_o, d_model, dc.append_pos, dc.seq_lens, dc.q_abs, attn, y,
                           ws, B, max_len, 0, dc.status)
 
+    def sync_all():
+        multirank.barrier(dist)
+        torch.cuda.synchronize()
+
     for i in range(warmup):
         call(i)
-    multirank.barrier(dist)
-    torch.cuda.synchronize()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    for i in range(steps):
-        call(i)
-    b.record(stream)
-    torch.cuda.synchronize()
-    ms = a.elapsed_time(b) / steps
+    all_ms = timed_repeats(torch, stream, call, steps, sync_all, min_wall_s=0.25)
+    ms = float(np.median(all_ms))
     res = {"workload": "cfg2 shapes from the hidden state: x[32,1024] -> packed input projection (bf16, maps folded in) "
                        "+ append, gva_decode, output projection",
            "ms_per_step": ms, "cache_read_GBps": case.cache_bytes() / (ms * 1e-3) / 1e9,
@@ -583,17 +648,14 @@ def measure_multi(rank, local_rank, dist, args, torch, gb, harness, q_len=4, on_
             gb.gva_decode_multi(pd.handle, caches[i & 1], pd.q_abs, pd.cu_q, pd.ctx_lens, pd.out, pd.lse, ws, B, pc.n_q, q_len, T,
                                 0, pd.status)
 
+    def sync_all():
+        multirank.barrier(dist)
+        torch.cuda.synchronize()
+
     for i in range(warmup):
         call(i)
-    multirank.barrier(dist)
-    torch.cuda.synchronize()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    for i in range(steps):
-        call(i)
-    b.record(stream)
-    torch.cuda.synchronize()
-    ms = a.elapsed_time(b) / steps
+    all_ms = timed_repeats(torch, stream, call, steps, sync_all, min_wall_s=0.25)
+    ms = float(np.median(all_ms))
     peak = load_peaks()[0]
     gbps = c.cache_bytes() / (ms * 1e-3) / 1e9
     res = {"workload": f"multi-token decode, cfg2 shapes: {q_len} new tokens per sequence over T = {T} cached tokens, B = {B}, "
@@ -667,7 +729,7 @@ def main() -> None:
     (step_ms, e2e_ms, decode_ms), job_bytes = multirank.reduce_times_and_work(
         [r["step_ms"], r["e2e_ms"], r["decode_ms"]], r["cache_bytes"], dist, dev)
 
-    others = {}
+    others, by_workload = {}, {}
     if not args.headline_only and world == 1 and name == "cfg2" and args.kernel == "auto":
         peak = load_peaks()[0]
         short = argparse.Namespace(**vars(args))
@@ -676,17 +738,26 @@ def main() -> None:
             o = measure(other, rank, local_rank, dist, short, kernel, torch, gb, harness, with_e2e=False,
                         with_clocks=True)
             per_layer = o["cache_bytes"] / o["layers"]
+            dec_gbps = per_layer / (o["decode_ms"] * 1e-3) / 1e9
+            step_gbps = o["cache_bytes"] / (o["step_ms"] * 1e-3) / 1e9
             others[other] = {
-                "workload": WORKLOAD_TEXT[other], "ms_per_step": o["step_ms"],
-                "cache_read_GBps": o["cache_bytes"] / (o["step_ms"] * 1e-3) / 1e9,
+                "workload": WORKLOAD_TEXT[other], "ms_per_step": o["step_ms"], "ms_per_step_min": o["step_ms_min"],
+                "cache_read_GBps": step_gbps,
                 "decode_steps_per_s": 1e3 / o["step_ms"],
-                "gva_decode_ms_per_call": o["decode_ms"],
+                "gva_decode_ms_per_call": o["decode_ms"], "gva_decode_ms_per_call_min": o["decode_ms_min"],
                 "ms_per_step_graph_replay": o["graph_step_ms"],
-                "gva_decode_GBps": per_layer / (o["decode_ms"] * 1e-3) / 1e9,
-                "gva_decode_frac_of_measured_peak": per_layer / (o["decode_ms"] * 1e-3) / 1e9 / peak,
+                "gva_decode_GBps": dec_gbps,
+                "gva_decode_frac_of_measured_peak": dec_gbps / peak,
                 "cache_bytes_per_step": o["cache_bytes"], "kernel": o["kernel"], "partitions": o["partitions"],
                 "total_tokens": int(o["case"].seq_lens.astype(np.int64).sum()) * o["layers"], "steps": o["steps"],
-                "clocks": o["clocks"], "device_status": o["status"]}
+                "repeats": o["step_repeats"], "clocks": o["clocks"], "device_status": o["status"]}
+            # the per-workload fractions also go inside the headline's roofline object (see below)
+            by_workload[other] = {
+                "gva_decode": {"GBps": dec_gbps, "frac_of_measured": dec_gbps / peak, "frac_of_8TBs_nominal": dec_gbps / NOMINAL_HBM_GBPS,
+                               "ms_per_call": o["decode_ms"]},
+                "whole_step": {"GBps": step_gbps, "frac_of_measured": step_gbps / peak, "frac_of_8TBs_nominal": step_gbps / NOMINAL_HBM_GBPS,
+                               "ms_per_step": o["step_ms"], "layers": o["layers"]},
+                "cache_bytes_per_step": o["cache_bytes"]}
 
         gq = measure_gqa(rank, local_rank, dist, short, kernel, torch, gb, harness)
         gq["gva_over_gqa_cache_bytes"] = r["cache_bytes"] / gq["cache_bytes_per_call"]      # 0.53125 = 1/2 + 16/(2*4*64)
@@ -708,25 +779,46 @@ def main() -> None:
         peak, peak_src = load_peaks()
         algo_bytes = case.algorithmic_bytes()
         achieved = algo_bytes / (decode_ms * 1e-3) / 1e9
+        traffic, traffic_src = NCU_TRAFFIC.get(name, (None, None))
+        dec_kernel_gbps = case.cache_bytes() / (decode_ms * 1e-3) / 1e9
+        ceiling = r.get("read_ceiling")
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": traffic,
+                    "traffic_source": (f"{traffic_src}: ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel at full size, "
+                                       "mean of two launches; a profiler figure, not taken in this run") if traffic_src else None,
+                    "peak_source": peak_src,
+                    "kernel": f"gva_decode: {r['kernel']} split-KV decode kernel + LSE combine kernel, timed "
+                              "together over back-to-back calls (the decode kernel alone is ~0.95 of that time)",
+                    "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": decode_ms,
+                    "min_launch_ms": r["decode_ms_min"], "achieved_best_repeat": algo_bytes / (r["decode_ms_min"] * 1e-3) / 1e9,
+                    "repeats": r["decode_repeats"],
+                    "frac_of_8TBs_nominal": achieved / NOMINAL_HBM_GBPS,
+                    "read_only_ceiling": ceiling,
+                    "frac_of_read_only_ceiling": (dec_kernel_gbps / ceiling["GBps"]) if ceiling else None,
+                    "whole_step": {"GBps": value / world, "frac_of_measured": value / world / peak,
+                                   "frac_of_8TBs_nominal": value / world / NOMINAL_HBM_GBPS, "ms_per_step": step_ms}}
+        if by_workload:
+            roofline["by_workload"] = by_workload
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": r["steps"], "warmup": r["warmup"],
             "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": {"bf16": "bf16", "fp8": "e4m3"}.get(case.cache_dtype, "f32"), "data": "synthetic",
             "config": dict(workload_description(name, case, r["layers"]), kernel=r["kernel"],
                            partitions=r["partitions"], replicas=world),
+            "timing": {"protocol": f"repeats of exactly {r['steps']} back-to-back steps between CUDA events on the launching stream, "
+                                   f"at least {MIN_REPEATS} repeats and {MIN_TIMED_WALL_S} s of timed work per loop; ms_per_step is the "
+                                   "median repeat, max over ranks",
+                       "repeats": r["step_repeats"], "ms_per_step_median": step_ms, "ms_per_step_min": r["step_ms_min"]},
             "decode_steps_per_s": world * 1e3 / step_ms,
-            "frac_of_8TBs_nominal": value / world / 8000.0,
+            "frac_of_8TBs_nominal": value / world / NOMINAL_HBM_GBPS,
             "clocks": r["clocks"],
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"],
-                    "ms_per_step": e2e_ms, "matches_device_result": r["e2e_matches"],
+                    "ms_per_step": e2e_ms, "ms_per_step_min": r["e2e_ms_min"], "repeats": r["e2e_repeats"],
+                    "matches_device_result": r["e2e_matches"],
                     "note": "gva_decode_step_host per step, then a stream sync: pinned host q_c/q_r/v_new/k_r/pos/"
                             "seq_lens in, host out; the cache and the maps M are resident state"},
-            "gpu_launches": 3 * r["steps"] * r["layers"],
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES.get(name), "peak_source": peak_src,
-                         "kernel": f"gva_decode: {r['kernel']} split-KV decode kernel + LSE combine kernel, timed "
-                                   "together over back-to-back calls (the decode kernel alone is ~0.91 of that time)",
-                         "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": decode_ms},
+            "gpu_launches": 3 * r["steps"] * r["step_repeats"] * r["layers"],
+            "roofline": roofline,
             "device_status": r["status"],
         }
         if others:

@@ -8,6 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgva.so")
+PROBE_LIB = os.path.join(HERE, "libgva_probe.so")      # the benchmark's read-only streaming probe (not part of the C ABI)
 SOURCES = ["gva_api.cu"]
 HEADERS = ["gva_common.cuh", "gva_small_kernels.cuh", "gva_decode_fma.cuh", "gva_decode_mma.cuh", "gva_decode_fp8.cuh", "gva_prefill.cuh", "gva_project.cuh",
            os.path.join("..", "..", "include", "gva.h")]
@@ -46,5 +47,21 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_probe(force: bool = False) -> str:
+    """Builds the benchmark's read-only streaming probe (csrc/stream_probe.cu) into its own shared object."""
+    src = os.path.join(CSRC, "stream_probe.cu")
+    if not force and os.path.exists(PROBE_LIB) and os.path.getmtime(PROBE_LIB) >= os.path.getmtime(src):
+        return PROBE_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared", "-Xcompiler", "-fPIC",
+           src, "-o", PROBE_LIB]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("nvcc failed building libgva_probe.so")
+    return PROBE_LIB
+
+
 if __name__ == "__main__":
+    build_probe(force=True)
     print(build(force=True, verbose="-v" in sys.argv))
