@@ -238,12 +238,13 @@ def run_reference(args) -> None:
 
 
 # ----------------------------------------------------------------------------------------------
-def timed_repeats(torch, stream, fn, steps: int, sync, min_wall_s: float = MIN_TIMED_WALL_S, min_repeats: int = MIN_REPEATS,
-                  max_repeats: int = 4000):
+def timed_repeats(torch, stream, fn, steps: int, sync, min_wall_s=None, min_repeats=None, max_repeats: int = 4000):
     """Times `fn(i)` in repeats of exactly `steps` back-to-back calls each, CUDA events on the launching stream at every
     repeat boundary; keeps going until at least `min_repeats` repeats and `min_wall_s` seconds of timed device work are
     in.  `sync()` (barrier + device synchronise) brackets each batch of repeats.  Returns the per-call milliseconds of
     every repeat."""
+    min_wall_s = MIN_TIMED_WALL_S if min_wall_s is None else min(min_wall_s, MIN_TIMED_WALL_S)
+    min_repeats = MIN_REPEATS if min_repeats is None else min_repeats
     per_call, i = [], 0
 
     def batch(n_rep: int):
@@ -681,7 +682,12 @@ def main() -> None:
     ap.add_argument("--num-splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--headline-only", action="store_true", help="skip the short runs of the other workloads")
+    ap.add_argument("--min-wall-s", type=float, default=MIN_TIMED_WALL_S,
+                    help="every timed loop runs at least this long (0 for profiler captures, which want few launches)")
+    ap.add_argument("--min-repeats", type=int, default=MIN_REPEATS, help="repeats of --steps calls per timed loop, at least")
     args = ap.parse_args()
+    global MIN_TIMED_WALL_S, MIN_REPEATS
+    MIN_TIMED_WALL_S, MIN_REPEATS = max(0.0, args.min_wall_s), max(1, args.min_repeats)
 
     if args.impl == "reference":
         run_reference(args)

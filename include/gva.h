@@ -73,8 +73,8 @@ typedef struct {
     int32_t d_v;           /* value width: 64 or 128                                                      */
     int32_t d_c;           /* content-key width (only gva_absorb_query uses it): 1..256                   */
     int32_t d_r;           /* RoPE width: 16 or 24 with d_v = 64 (the paper's two tested widths), 32 with d_v = 128;
-                              0 = value-only cache without a positional slice (Section 3.4: "only values, exactly
-                              half"): kr_pool, q_r and kr_new are then unused and may be NULL, scale = 1/sqrt(d_c);
+                              0 = value-only cache without a positional slice (Section 3.4: a cache of values alone is
+                              half of matched GQA's): kr_pool, q_r and kr_new are then unused and may be NULL, scale = 1/sqrt(d_c);
                               gva_decode_step_host, the projections and gva_decode_tokens return GVA_ERR_UNSUPPORTED */
     int32_t page_size;     /* tokens per page, a multiple of 32                                           */
     int32_t cache_dtype;   /* gva_dtype                                                                   */
@@ -104,7 +104,17 @@ typedef struct gva_handle gva_handle; /* opaque host-side state: config, device 
 
 /* Create / destroy a handle for one head configuration on one device.  Validates cfg
  * (GVA_ERR_UNSUPPORTED / GVA_ERR_INVALID_ARG), checks that `device` is compute capability 10.x
- * (GVA_ERR_CUDA otherwise) and raises the kernels' shared-memory limits.  Makes `device` current. */
+ * (GVA_ERR_CUDA otherwise) and raises the kernels' shared-memory limits.  Makes `device` current.
+ *
+ * One handle, one stream at a time.  Besides its host-side state a handle owns a few words of DEVICE-side
+ * scheduling state inside the library image (the counters through which the thread blocks of a decode
+ * kernel share out the tail of the cache stream).  Decode calls on one handle -- gva_decode, gqa_decode,
+ * gva_decode_step(_host), gva_decode_static, gva_decode_tokens, gva_layer_step -- must therefore be
+ * stream-ordered with respect to one another: issue them on one stream, or order the streams with events.
+ * Two such calls that may overlap on the GPU race on those words even if their workspaces differ (wrong
+ * partition of the work, hence wrong results; never a fault).  Use one handle per concurrent stream; handles
+ * are cheap (no device allocation).  The handle is not thread-safe either: one host thread at a time.
+ * gva_destroy only after the last call on the handle has finished on the device. */
 int gva_create(gva_handle **out, const gva_config *cfg, int device);
 int gva_destroy(gva_handle *h);
 
@@ -149,7 +159,7 @@ int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, 
  *                                 per resident thread block (ranges may cross sequence boundaries);
  *                                 n >= 1: every sequence is cut into exactly n ranges.
  * Partial results are merged by log-sum-exp weights in a second kernel.  For fixed arguments the
- * result is bitwise reproducible from run to run. */
+ * result is bitwise reproducible from run to run.  Calls on one handle must be stream-ordered (see gva_create). */
 int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens,
                float *out, float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len,
                int num_splits, int32_t *dev_status, void *stream);
@@ -167,7 +177,12 @@ int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const 
  * allocating library routine.
  *
  *  - Limit: if gva_decode_workspace_bytes(h, B, max_seq_len, num_splits) exceeds
- *    GVA_STATIC_SCRATCH_BYTES the call launches nothing and returns GVA_ERR_STATIC_LIMIT.
+ *    GVA_STATIC_SCRATCH_BYTES the call launches nothing and returns GVA_ERR_STATIC_LIMIT.  At num_splits = 0
+ *    the need grows with the batch (one partial record per sequence on top of a few per thread block), not
+ *    with the context length: on a B200 the five workloads of the benchmark take 2.5 to 5.5 MB (for example
+ *    B = 32 sequences of 32768 tokens, H = 16, d_v = 64: 5.1 MB; B = 64, H = 32, d_v = 128: 3.5 MB), and
+ *    H = 16, d_v = 64 fits up to about B = 2700.  With num_splits = n the need is B * n records of
+ *    H * (d_v + 2) * 4 bytes each.
  *  - Set-up: the first call on each device looks up the array's device address (once per device; the
  *    handle's device must be the current device, otherwise GVA_ERR_INVALID_ARG).  Make that first
  *    call outside any stream capture.
@@ -229,7 +244,7 @@ int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, 
                          void *stream);
 
 /* ---- The projections around the attention (Algorithm 1: q_t = x_t W_Q, v_t = x_t W_V, k^rope_t = (x_t W_r) R_t^T;
- * then "the usual concatenation and output projection"), with the maps folded into the query projection:
+ * then the heads side by side through the output projection), with the maps folded into the query projection:
  * because M_h is fixed at inference, q~_h = (x W_Q^{nope,h}) M_h^T = x (W_Q^{nope,h} M_h^T)  (Eq. absorb), so
  * one product with a packed weight matrix yields the absorbed queries directly and gva_absorb_query drops out.
  *
@@ -259,8 +274,8 @@ int gva_layer_step(gva_handle *h, const gva_cache *cache, const float *x, const 
                    void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
                    int32_t *dev_status, void *stream);
 
-/* ---- Several new tokens per sequence: prefill and chunked prefill (the paper's multi-token form: "standard causal
- * attention with the same content-position split", Section 3.3 and the remark after Algorithm 1), computed in the
+/* ---- Several new tokens per sequence: prefill and chunked prefill (the paper's multi-token form: ordinary causal
+ * attention whose scores keep the content + positional split, Section 3.3 and the remark after Algorithm 1), computed in the
  * absorbed form of Eq. absorb.  Sequence b has ctx_lens[b] tokens cached already and q_len_b = cu_q[b+1] - cu_q[b]
  * new tokens; new token i of sequence b is input row cu_q[b] + i, sits at position t = ctx_lens[b] + i and attends
  * to positions 0..t.  The order of calls is Algorithm 1's, once per chunk instead of once per token:

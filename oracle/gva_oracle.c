@@ -17,7 +17,7 @@
  *   decode    : s_j = q~_h v_{j,g(h)}^T + q^rope_h (k^rope_j)^T ;  o_h = softmax(s/sqrt(d_qk)) V_{g(h)}
  *               with d_qk = d_c + d_r                     (Section 3.3 score equation; Algorithm 1)
  *   gqa       : matched GQA decode over cached K and V    (Section 2, GQA; Section 3.4)
- *   prefill   : standard causal attention with the same content-position split, keys formed explicitly:
+ *   prefill   : ordinary causal attention whose scores are the content term plus the positional term, keys formed explicitly:
  *               K_h = V_g(h) M_h (Eq. kvm), k_j = [K_h,j ; k^rope_j], q_i = [q^nope_i ; q^rope_i R_i^T]
  *               (Section 3.3; the sentence after Algorithm 1 on training / multi-token attention)
  *
@@ -276,7 +276,7 @@ void oracle_gqa_decode(const void *k_pool, const void *v_pool, int dtype, const 
 }
 
 /* ---- the projections around the attention (Algorithm 1: q_t = x_t W_Q, v_t = x_t W_V, x_t W_r; then
- * "the usual concatenation and output projection") ---------------------------------------------------
+ * then the concatenated heads through the output projection) ------------------------------------------
  * Plain matrix product y[b][n] = sum_k x[b][k] W[k][n], fp64. */
 void oracle_matmul(const double *x, const double *W, int B, int K, int N, double *y) {
 #pragma omp parallel for schedule(static)
@@ -302,7 +302,7 @@ void oracle_fold_maps(const double *W_q_nope, const double *M, int d_model, int 
             }
 }
 
-/* ---- prefill / chunked prefill: standard causal attention with the content-position split --------
+/* ---- prefill / chunked prefill: causal attention with content + positional scores ------------------
  * Several query tokens per sequence.  Sequence b has ctx_lens[b] tokens cached before the chunk and
  * q_lens = cu_q[b+1] - cu_q[b] new tokens whose value rows and rotated positional keys are ALREADY in
  * the cache (appended first, as in Algorithm 1); query token i of sequence b sits at position

@@ -1,9 +1,9 @@
 """Second, deliberately naive oracle path: Python lists and the `math` module only.
 
 TEST INFRASTRUCTURE ONLY.  Used to brute-force hand-sized cases and to cross-check the C oracle
-(oracle/gva_oracle.c); written separately from it, following Algorithm 1 of the paper line by
-line in its notation.  Cache values are
-plain Python floats (already widened from whatever storage type).
+(oracle/gva_oracle.c); written separately from it, from the paper's equations (Eq. absorb, Eq. kvm,
+Eq. krope, the score equation of Section 3.3) in its notation.  Cache values are plain Python floats
+(already widened from whatever storage type).
 """
 from __future__ import annotations
 
@@ -42,7 +42,7 @@ def softmax(s: Sequence[float]) -> List[float]:
 
 def decode_head(q_tilde: Sequence[float], q_rope_rot: Sequence[float], V_g: Sequence[Sequence[float]],
                 k_rope: Sequence[Sequence[float]], d_qk: int):
-    """Algorithm 1, the two attention lines for one head:
+    """One head's attention in the absorbed form (Section 3.3 with Eq. absorb):
     s_j = q~ . v_j + q^rope . k^rope_j ;  o = softmax(s / sqrt(d_qk)) V_g.   Returns (o, lse)."""
     T = len(V_g)
     d_v = len(q_tilde)
@@ -101,34 +101,38 @@ def gather_tokens(v_pool, kr_pool, block_table: Optional[Sequence[Sequence[int]]
     return V_tokens, KR_tokens
 
 
+def _vec_mat(x: Sequence[float], W, n_out: int, pick) -> List[float]:
+    """y[c] = sum_m x[m] * pick(W[m], c) for c < n_out: a row vector times a matrix stored row by row."""
+    return [sum(x[m] * pick(W[m], c) for m in range(len(x))) for c in range(n_out)]
+
+
 def layer_decode_step(x, W_Q, W_V, W_r, W_O, M, t: int, V_cache, KR_cache, H: int, G: int, d_c: int, d_r: int,
                       base: float = 10000.0):
-    """Algorithm 1 line by line for ONE sequence, starting from the hidden state x (list of d_model floats).
+    """One sequence's decode step from the hidden state x (list of d_model floats), in the UNABSORBED form: every
+    head's keys are written out as full (d_c + d_r)-wide vectors, the content part reconstructed from the cached
+    values (Eq. kvm: K_h = V_g(h) M_h) and the shared rotated positional key appended to it (Eq. krope and the
+    concatenated-key score of Section 3.3), and attention is plain softmax(q k^T / sqrt(d_qk)) v over those keys.
 
-    W_Q[m][h] = list of d_r + d_c floats (positional slice first, then content slice, as the algorithm's split
-    "q^rope, q^nope" lists them), W_V[m][g] = list of d_v, W_r[m] = list of d_r, W_O[h*d_v + i] = list of d_model.
-    V_cache[g] = list of cached value rows, KR_cache = list of cached rotated positional keys; both are extended
-    in place.  Keys are materialised explicitly (K = V M), nothing is absorbed.  Returns (y, per-head outputs)."""
-    d_model = len(x)
-    d_v = len(M[0])
-    # q_t <- x_t W_Q ; split each head into q^rope, q^nope
-    q = [[sum(x[m] * W_Q[m][h][c] for m in range(d_model)) for c in range(d_r + d_c)] for h in range(H)]
-    q_rope = [q[h][:d_r] for h in range(H)]
-    q_nope = [q[h][d_r:] for h in range(H)]
-    # v_t <- x_t W_V ; append one row per value group
+    W_Q[m][h] = list of d_r + d_c floats (positional slice first, then content slice), W_V[m][g] = list of d_v,
+    W_r[m] = list of d_r, W_O[h*d_v + i] = list of d_model.  V_cache[g] = list of cached value rows, KR_cache = list
+    of cached rotated positional keys; both are extended in place by the new token (position t) before anything
+    attends, so the new token sees itself.  Returns (y, per-head outputs)."""
+    d_model, d_v, d_qk = len(x), len(M[0]), d_c + d_r
+    # 1. the new token's cache entries: one value row per group, one rotated positional key for all heads
     for g in range(G):
-        V_cache[g].append([sum(x[m] * W_V[m][g][i] for m in range(d_model)) for i in range(d_v)])
-    # k^rope_t <- (x_t W_r) R_t^T ; append
-    KR_cache.append(rope([sum(x[m] * W_r[m][k] for m in range(d_model)) for k in range(d_r)], t, base))
+        V_cache[g].append(_vec_mat(x, W_V, d_v, lambda row, i, g=g: row[g][i]))
+    KR_cache.append(rope(_vec_mat(x, W_r, d_r, lambda row, k: row[k]), t, base))
+    n_tok = len(KR_cache)
+    # 2. full queries [q^nope | q^rope R_t^T] and full keys [v_j M_h | k^rope_j], head by head
     outs = []
     for h in range(H):
         g = h // (H // G)
-        qr = rope(q_rope[h], t, base)                                   # q^rope <- q^rope R_t^T
-        keys = [reconstruct_key(v, M[h]) for v in V_cache[g]]           # K^nope = V M_h, materialised
-        s = [(sum(a * b for a, b in zip(q_nope[h], keys[j])) + sum(a * b for a, b in zip(qr, KR_cache[j])))
-             / math.sqrt(d_c + d_r) for j in range(len(keys))]          # scores, with explicit keys instead of q~
-        p = softmax(s)
-        outs.append([sum(p[j] * V_cache[g][j][i] for j in range(len(keys))) for i in range(d_v)])   # o <- softmax(s) V
+        q_full = _vec_mat(x, W_Q, d_qk, lambda row, c, h=h: row[h][c])
+        query = q_full[d_r:] + rope(q_full[:d_r], t, base)
+        keys = [reconstruct_key(V_cache[g][j], M[h]) + list(KR_cache[j]) for j in range(n_tok)]
+        weights = softmax([sum(a * b for a, b in zip(query, keys[j])) / math.sqrt(d_qk) for j in range(n_tok)])
+        outs.append([sum(weights[j] * V_cache[g][j][i] for j in range(n_tok)) for i in range(d_v)])
+    # 3. heads side by side, then the output projection
     concat = [v for o in outs for v in o]
     y = [sum(concat[r] * W_O[r][m] for r in range(len(concat))) for m in range(d_model)]
     return y, outs

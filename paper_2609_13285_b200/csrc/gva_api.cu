@@ -357,7 +357,7 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
     if (cfg->cache_dtype != GVA_F32 && cfg->cache_dtype != GVA_BF16 && cfg->cache_dtype != GVA_E4M3) return GVA_ERR_INVALID_ARG;
     if (cfg->kernel < GVA_KERNEL_AUTO || cfg->kernel > GVA_KERNEL_MMA) return GVA_ERR_INVALID_ARG;
     if (cfg->H % cfg->G != 0 || cfg->H / cfg->G != kHeadsPerGroup) return GVA_ERR_UNSUPPORTED;
-    // d_r = 0 is the value-only cache (no positional slice: Section 3.4, "exactly half")
+    // d_r = 0 is the value-only cache (no positional slice: half the bytes of matched GQA, Section 3.4)
     if (!((cfg->d_v == 64 && (cfg->d_r == 16 || cfg->d_r == 24 || cfg->d_r == 0)) || (cfg->d_v == 128 && (cfg->d_r == 32 || cfg->d_r == 0))))
         return GVA_ERR_UNSUPPORTED;
     if (cfg->G > 8 || cfg->d_c > 256 || cfg->page_size % 32 != 0) return GVA_ERR_UNSUPPORTED;

@@ -1,7 +1,7 @@
 // Causal prefill / chunked-prefill attention over the paged bf16 GVA cache on the 5th-generation tensor
 // cores (tcgen05 + tensor memory), sm_100a.
 //
-// What it computes (the paper's multi-token form: standard causal attention with the content-position split,
+// What it computes (the paper's multi-token form: ordinary causal attention with content + positional scores,
 // Section 3.3 and the remark after Algorithm 1), in the absorbed form of Eq. absorb: for query token i at
 // position t, head h of group g,
 //     s_ij = q~_i,h . v_j,g + q^rope_i,h . k^rope_j   (j <= t),   o_i,h = softmax_j(s_ij / sqrt(d_qk)) V_g.

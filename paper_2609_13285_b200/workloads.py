@@ -114,7 +114,7 @@ class HeadShape:
 SHAPE_A = HeadShape(H=16, G=4, d_v=64, d_c=64, d_r=16)
 SHAPE_B = HeadShape(H=32, G=8, d_v=128, d_c=128, d_r=32)
 SHAPE_C = HeadShape(H=16, G=4, d_v=64, d_c=64, d_r=24)      # the paper's second tested RoPE width (48-byte k_r rows)
-SHAPE_A0 = HeadShape(H=16, G=4, d_v=64, d_c=64, d_r=0)      # value-only cache: no positional slice ("exactly half" of GQA)
+SHAPE_A0 = HeadShape(H=16, G=4, d_v=64, d_c=64, d_r=0)      # value-only cache: no positional slice (half the bytes of matched GQA)
 SHAPE_B0 = HeadShape(H=32, G=8, d_v=128, d_c=128, d_r=0)
 
 

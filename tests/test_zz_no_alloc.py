@@ -44,9 +44,13 @@ def test_static_scratch_decode_matches_workspace_decode_twice():
                 for _rep in range(2):                 # two calls in a row on the same scratch
                     dc.out.fill_(float("nan"))
                     dc.lse.fill_(float("nan"))
+                    torch.cuda.synchronize()
+                    free_before = torch.cuda.mem_get_info()[0]          # cudaMemGetInfo: free device bytes, driver's view
                     gb.gva_decode_static(dc.handle, dc.cache, dc.q_abs, dc.seq_lens, dc.out, dc.lse, case.B,
                                          dc.max_seq_len, num_splits, dc.status)
                     torch.cuda.synchronize()
+                    # the call allocated nothing: not a byte of device memory less than before it
+                    assert torch.cuda.mem_get_info()[0] == free_before
                     assert int(dc.status.item()) == 0
                     a = dc.out.cpu().numpy().astype(np.float64)
                     assert np.isfinite(a).all()
@@ -70,3 +74,18 @@ def test_static_scratch_rejects_requests_beyond_its_size():
         assert "built-in scratch" in gb.status_string(rc)
     finally:
         dc.close()
+
+
+def test_static_scratch_holds_the_five_benchmark_workloads():
+    # at automatic splits every one of the five workloads of the benchmark needs less than the built-in array
+    # (the header says so; this keeps the statement true when the partition or the record layout changes)
+    shapes = {"cfg0": (wl.SHAPE_A, gb.GVA_F32, 1, 128), "cfg1": (wl.SHAPE_A, gb.GVA_BF16, 8, 4096),
+              "cfg2": (wl.SHAPE_A, gb.GVA_BF16, 32, 32768), "cfg3": (wl.SHAPE_B, gb.GVA_BF16, 64, 16384),
+              "cfg4": (wl.SHAPE_A, gb.GVA_BF16, 128, 8193)}
+    for name, (s, dtype, B, T) in shapes.items():
+        h = gb.gva_create(H=s.H, G=s.G, d_v=s.d_v, d_c=s.d_c, d_r=s.d_r, page_size=64, cache_dtype=dtype)
+        try:
+            need = gb.gva_decode_workspace_bytes(h, B, T, 0)
+            assert 0 < need <= gb.GVA_STATIC_SCRATCH_BYTES, (name, need)
+        finally:
+            gb.gva_destroy(h)
