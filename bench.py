@@ -712,7 +712,7 @@ def main() -> None:
     kernel = {"auto": gb.GVA_KERNEL_AUTO, "fma": gb.GVA_KERNEL_FMA, "mma": gb.GVA_KERNEL_MMA}[args.kernel]
 
     name = args.workload
-    if name in ("prefill", "prefill-ncu", "prefill-wide", "layer", "multi", "multi-q1", "multi-q8", "multi-q32", "tokens-q2", "tokens-q4", "tokens-q2-fp8", "tokens-q4-fp8"):      # side workloads on their own (small runs for profiler captures)
+    if name in ("prefill", "prefill-ncu", "prefill-wide", "layer", "multi", "multi-q1", "multi-q8", "multi-q32", "tokens-q2", "tokens-q4", "tokens-q6", "tokens-q8", "tokens-q2-fp8", "tokens-q4-fp8"):      # side workloads on their own (small runs for profiler captures)
         if rank == 0:
             if name == "layer":
                 res = measure_layer(rank, local_rank, None, args, kernel, torch, gb, harness)
@@ -773,6 +773,7 @@ def main() -> None:
         others["decode_multi_cfg2_q4"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=4)
         others["decode_tokens_cfg2_q2"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=2, on_decode_kernel=True)
         others["decode_tokens_cfg2_q4"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=4, on_decode_kernel=True)
+        others["decode_tokens_cfg2_q8"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=8, on_decode_kernel=True)
         others["decode_tokens_cfg2_q4_fp8"] = measure_multi(rank, local_rank, dist, short, torch, gb, harness, q_len=4,
                                                             on_decode_kernel=True, cache_dtype="fp8")
         others["prefill"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness)

@@ -315,7 +315,7 @@ int gva_decode_multi(gva_handle *h, const gva_cache *cache, const float *q_abs, 
                      const int32_t *ctx_lens, float *out, float *lse, void *workspace, size_t workspace_bytes, int B,
                      int n_q, int max_q_len, int max_seq_len, int num_splits, int32_t *dev_status, void *stream);
 
-/* Decode of q_len = 2, 3 or 4 new tokens per sequence at the single-token kernel's cache-stream rate (speculative /
+/* Decode of q_len = 2 .. 8 new tokens per sequence at the single-token kernel's cache-stream rate (speculative /
  * multi-token decode; not in the paper -- Algorithm 1 applied to q_len tokens at once).  The split-KV tensor-core decode
  * kernel of gva_decode carries the 4 * q_len (head, token) pairs of a value group as its MMA columns, so the cache is
  * streamed once for all of them.  Every sequence has exactly q_len new tokens, already appended.
@@ -323,13 +323,25 @@ int gva_decode_multi(gva_handle *h, const gva_cache *cache, const float *q_abs, 
  *   seq_lens [B] i32                      tokens attended by the LAST new token; new token i attends seq_lens[b] - (q_len-1-i)
  *   out      [B * q_len][H][d_v] f32, lse [B * q_len][H] f32 or NULL
  *   workspace                             at least gva_decode_tokens_workspace_bytes(...) bytes, 256-byte aligned
- * bf16 cache, (d_v, d_r) = (64, 16) or (128, 32), tensor-core kernel only; otherwise GVA_ERR_UNSUPPORTED.  The queries
- * and the softmax weights go to the tensor cores as bf16 (their hi/lo halves of the single-token layout carry the second
- * token instead), so results carry bf16-level error like gva_prefill: |out - exact| <= 2e-2 for unit-variance data. */
+ * q_len 2 .. 4: bf16 cache with (d_v, d_r) = (64, 16), (64, 0), (128, 32) or (128, 0), and the e4m3 cache with a positional
+ * slice; q_len 5 .. 8: bf16 cache with d_v = 64, d_r = 16 or 0, G <= 4 and pages of a multiple of 64 tokens; tensor-core
+ * kernel only; otherwise GVA_ERR_UNSUPPORTED.  The queries enter the score product as two bf16 numbers each (hi + lo), the
+ * softmax weights as one (the 8-bit cache: f16 queries and weights), accumulation is f32: |out - exact| <= 2e-2 whatever
+ * the size of the scores. */
 size_t gva_decode_tokens_workspace_bytes(const gva_handle *h, int B, int q_len, int max_seq_len, int num_splits);
 int gva_decode_tokens(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
                       float *lse, void *workspace, size_t workspace_bytes, int B, int q_len, int max_seq_len,
                       int num_splits, int32_t *dev_status, void *stream);
+
+/* The same with a different number of new tokens per sequence (a batch in which some sequences verify eight draft
+ * tokens, some two, some none): sequence b has q_len_b = cu_q[b+1] - cu_q[b] new tokens, 0 <= q_len_b <= max_q_len <= 8,
+ * already appended; its rows of q_abs / out / lse are cu_q[b] .. cu_q[b+1] - 1 (cu_q [B + 1] i32, cu_q[0] = 0,
+ * non-decreasing).  seq_lens[b] = tokens attended by the last new token of b; new token i attends
+ * seq_lens[b] - (q_len_b - 1 - i).  Workspace: gva_decode_tokens_workspace_bytes(h, B, max(max_q_len, 2), ...).
+ * bf16 cache only; shapes as gva_decode_tokens for the given max_q_len.  Same accuracy. */
+int gva_decode_tokens_ragged(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *cu_q,
+                             const int32_t *seq_lens, float *out, float *lse, void *workspace, size_t workspace_bytes, int B,
+                             int max_q_len, int max_seq_len, int num_splits, int32_t *dev_status, void *stream);
 
 /* Geometry of the most recent gva_decode / gqa_decode launch on this handle (reporting only):
  * number of split-KV partitions launched (thread blocks of the decode kernel). */

@@ -24,7 +24,7 @@ GVA_KERNEL_AUTO, GVA_KERNEL_FMA, GVA_KERNEL_MMA = 0, 1, 2
 EXPORTS = ["gva_create", "gva_destroy", "gva_decode_workspace_bytes", "gva_absorb_query", "gva_append_cache",
            "gva_decode", "gva_decode_static", "gqa_decode", "gva_decode_step", "gva_step_scratch_bytes", "gva_decode_step_host", "gva_input_width", "gva_pack_input_weights", "gva_pack_bf16",
            "gva_project_in", "gva_project_out", "gva_layer_step", "gva_last_num_splits", "gva_last_kernel", "gva_last_tile_tokens",
-           "gva_status_string", "gva_append_chunk", "gva_prefill", "gva_decode_multi_workspace_bytes", "gva_decode_multi", "gva_decode_tokens_workspace_bytes", "gva_decode_tokens"]
+           "gva_status_string", "gva_append_chunk", "gva_prefill", "gva_decode_multi_workspace_bytes", "gva_decode_multi", "gva_decode_tokens_workspace_bytes", "gva_decode_tokens", "gva_decode_tokens_ragged"]
 
 
 class GvaConfig(ctypes.Structure):
@@ -81,6 +81,7 @@ def load() -> ctypes.CDLL:
     lib.gva_decode_tokens_workspace_bytes.argtypes = [vp, ip, ip, ip, ip]
     lib.gva_decode_tokens_workspace_bytes.restype = sz
     lib.gva_decode_tokens.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, vp, sz, ip, ip, ip, ip, vp, vp]
+    lib.gva_decode_tokens_ragged.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, vp, vp, sz, ip, ip, ip, ip, vp, vp]
     lib.gva_decode_multi_workspace_bytes.restype = sz
     lib.gva_decode_multi.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, vp, vp, sz, ip, ip, ip, ip, ip, vp, vp]
     lib.gva_decode_static.argtypes = [vp, ctypes.POINTER(GvaCache), vp, vp, vp, vp, ip, ip, ip, vp, vp]
@@ -205,6 +206,17 @@ def gva_decode_tokens(handle: int, cache: GvaCache, q_abs, seq_lens, out, lse, w
                                   int(q_len), int(max_seq_len), int(num_splits), _ptr(dev_status), _stream())
     if check:
         _check(rc, "gva_decode_tokens")
+    return rc
+
+
+def gva_decode_tokens_ragged(handle: int, cache: GvaCache, q_abs, cu_q, seq_lens, out, lse, workspace, B: int, max_q_len: int,
+                             max_seq_len: int, num_splits: int = 0, dev_status=None, check: bool = True) -> int:
+    rc = load().gva_decode_tokens_ragged(handle, ctypes.byref(cache), _ptr(q_abs), _ptr(cu_q), _ptr(seq_lens), _ptr(out), _ptr(lse),
+                                         _ptr(workspace),
+                                         0 if workspace is None else int(workspace.numel() * workspace.element_size()), int(B),
+                                         int(max_q_len), int(max_seq_len), int(num_splits), _ptr(dev_status), _stream())
+    if check:
+        _check(rc, "gva_decode_tokens_ragged")
     return rc
 
 

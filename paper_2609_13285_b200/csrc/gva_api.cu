@@ -636,7 +636,7 @@ int gva_decode_multi(gva_handle *h, const gva_cache *cache, const float *q_abs, 
 static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,
                        float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len, int num_splits,
                        int32_t *dev_status, void *stream, int early_start, const int32_t *append_pos, int q_len = 1,
-                       bool dry = false) {
+                       bool dry = false, const int32_t *cu_q = nullptr) {
     int rc = check_common(h, B, max_seq_len, num_splits);
     if (rc != GVA_OK) return rc;
     if (!cache) return GVA_ERR_INVALID_ARG;
@@ -664,6 +664,8 @@ static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs
     p.early_start = early_start;
     p.append_pos = append_pos;
     p.q_len = q_len;
+    p.cu_q = cu_q;
+    if (cu_q && c.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;      // a count per sequence: 16-bit cache only
     return launch_decode<false>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
                                 static_cast<cudaStream_t>(stream), q_len, dry);
 }
@@ -676,7 +678,7 @@ int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const 
 }
 
 size_t gva_decode_tokens_workspace_bytes(const gva_handle *h, int B, int q_len, int max_seq_len, int num_splits) {
-    if (check_common(h, B, max_seq_len, num_splits) != GVA_OK || q_len < 2 || q_len > 4) return 0;
+    if (check_common(h, B, max_seq_len, num_splits) != GVA_OK || q_len < 2 || q_len > 8) return 0;
     return workspace_layout(h, B, num_splits, q_len).total;
 }
 
@@ -684,9 +686,18 @@ int gva_decode_tokens(gva_handle *h, const gva_cache *cache, const float *q_abs,
                       void *workspace, size_t workspace_bytes, int B, int q_len, int max_seq_len, int num_splits,
                       int32_t *dev_status, void *stream) {
     if (!h) return GVA_ERR_INVALID_ARG;
-    if (q_len < 2 || q_len > 4) return GVA_ERR_UNSUPPORTED;
+    if (q_len < 2 || q_len > 8) return GVA_ERR_UNSUPPORTED;
     return decode_impl(h, cache, q_abs, seq_lens, out, lse, workspace, workspace_bytes, B, max_seq_len, num_splits, dev_status,
                        stream, 0, nullptr, q_len);
+}
+
+int gva_decode_tokens_ragged(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *cu_q, const int32_t *seq_lens,
+                             float *out, float *lse, void *workspace, size_t workspace_bytes, int B, int max_q_len, int max_seq_len,
+                             int num_splits, int32_t *dev_status, void *stream) {
+    if (!h || !cu_q) return GVA_ERR_INVALID_ARG;
+    if (max_q_len < 1 || max_q_len > 8) return GVA_ERR_UNSUPPORTED;
+    return decode_impl(h, cache, q_abs, seq_lens, out, lse, workspace, workspace_bytes, B, max_seq_len, num_splits, dev_status,
+                       stream, 0, nullptr, max_q_len < 2 ? 2 : max_q_len, false, cu_q);
 }
 
 int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const float *q_c, const float *q_r,
@@ -843,8 +854,8 @@ int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, 
     int rc = check_common(h, B, max_seq_len, num_splits);
     if (rc != GVA_OK) return rc;
     if (B == 0) return GVA_OK;
-    if (h->cfg.d_r == 0) return GVA_ERR_UNSUPPORTED;     // the value-only cache goes through the device entry points
-    if (!cache || !M || !q_c_host || !q_r_host || !v_new_host || !kr_new_host || !pos_host || !seq_lens_host || !out_host)
+    const bool rope = h->cfg.d_r > 0;                    // a value-only cache has no positional inputs: q_r_host / kr_new_host may be NULL
+    if (!cache || !M || !q_c_host || (rope && !q_r_host) || !v_new_host || (rope && !kr_new_host) || !pos_host || !seq_lens_host || !out_host)
         return GVA_ERR_INVALID_ARG;
     const StepLayout L = step_layout(h, B, num_splits);
     if (!scratch || scratch_bytes < L.total) return GVA_ERR_WORKSPACE;
@@ -859,9 +870,10 @@ int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, 
     // interconnect: that replaces five small copies, each of which would cost a few microseconds of stream time,
     // by loads and stores inside kernels that run anyway.  Pageable buffers take the staged path.
     const void *hosts[5] = {q_c_host, q_r_host, v_new_host, kr_new_host, out_host};
-    void *mapped[5];
+    void *mapped[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     bool host_mapped = true;
     for (int i = 0; i < 5 && host_mapped; ++i) {
+        if (!rope && (i == 1 || i == 3)) continue;      // unused inputs stay NULL
         cudaPointerAttributes attr;
         if (cudaPointerGetAttributes(&attr, hosts[i]) != cudaSuccess) {
             (void)cudaGetLastError();
@@ -909,12 +921,12 @@ int gva_decode_step_host(gva_handle *h, const gva_cache *cache, const float *M, 
                                q_abs, static_cast<float *>(mapped[4]), nullptr, s + L.ws, L.ws_bytes, B, max_seq_len,
                                num_splits, dev_status, stream);
     }
-    if (!h2d(L.q_c, q_c_host, (size_t)B * c.H * c.d_c * 4) || !h2d(L.q_r, q_r_host, (size_t)B * c.H * c.d_r * 4) ||
-        !h2d(L.v_new, v_new_host, (size_t)B * c.G * c.d_v * 4) || !h2d(L.kr_new, kr_new_host, (size_t)B * c.d_r * 4))
+    if (!h2d(L.q_c, q_c_host, (size_t)B * c.H * c.d_c * 4) || (rope && !h2d(L.q_r, q_r_host, (size_t)B * c.H * c.d_r * 4)) ||
+        !h2d(L.v_new, v_new_host, (size_t)B * c.G * c.d_v * 4) || (rope && !h2d(L.kr_new, kr_new_host, (size_t)B * c.d_r * 4)))
         return GVA_ERR_CUDA;
     float *out = reinterpret_cast<float *>(s + L.out);
-    rc = gva_decode_step(h, cache, M, reinterpret_cast<const float *>(s + L.q_c), reinterpret_cast<const float *>(s + L.q_r),
-                         reinterpret_cast<const float *>(s + L.v_new), reinterpret_cast<const float *>(s + L.kr_new), pos,
+    rc = gva_decode_step(h, cache, M, reinterpret_cast<const float *>(s + L.q_c), rope ? reinterpret_cast<const float *>(s + L.q_r) : nullptr,
+                         reinterpret_cast<const float *>(s + L.v_new), rope ? reinterpret_cast<const float *>(s + L.kr_new) : nullptr, pos,
                          lens, q_abs, out, nullptr, s + L.ws, L.ws_bytes, B, max_seq_len, num_splits, dev_status, stream);
     if (rc != GVA_OK) return rc;
     if (cudaMemcpyAsync(out_host, out, (size_t)B * c.H * c.d_v * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)

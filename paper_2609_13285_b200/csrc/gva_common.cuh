@@ -52,7 +52,8 @@ struct DecodeParams {
     int early_start;             // 1: launched right behind step_front_kernel (see gva_decode_mma.cuh)
     const int32_t *append_pos;   // early_start: position being appended per sequence (its tile must not be read early)
     float scale_log2;            // softmax scale * log2(e)
-    int q_len;                   // multi-token decode: new tokens per sequence (2..4); 0 or 1 otherwise
+    int q_len;                   // multi-token decode: new tokens per sequence (2..8; with cu_q: the most any sequence has); 0 or 1 otherwise
+    const int32_t *cu_q;         // multi-token decode with a different count per sequence: first query row of every sequence ([B + 1]); else NULL
 };
 
 __device__ __forceinline__ void report_error(int32_t *dev_status, int code, int b) {

@@ -370,8 +370,11 @@ __device__ __forceinline__ void decode_producer(const DecodeParams &p, const Blo
 // QL > 1 (multi-token decode, QL = 2 or 4 new tokens per sequence): the 4 heads x QL tokens of a group are the N
 // columns, 8 per N-block, column c = slot * 4 + head with slot the token's index among the new ones; the queries and
 // the weights go in as plain bf16 (the hi/lo halves of the single-token layout have become the second token), slot s
-// attends to seq_len - (QL - 1 - s) tokens, and the partial records and outputs use QL * H pseudo-heads, slot * H + head.
-template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA, int QL = 1>
+// attends to seq_len - (q_len - 1 - s) tokens, and the partial records and outputs use q_len * H pseudo-heads, slot * H + head.
+// CW > 1: the columns of a group are split over CW consumer warps, warp cw taking slots cw * QL .. cw * QL + QL - 1 of
+// the same shared-memory tile (QL = 4, CW = 2: up to eight new tokens per sequence; one such block fills an SM).
+// With DecodeParams::cu_q every sequence has its own number of new tokens (at most q_len, possibly none).
+template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA, int QL = 1, int CW = 1>
 __global__ void __launch_bounds__(32 * 9)
 decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = MmaTraits<DV, DR, TILE, GQA>;
@@ -384,11 +387,12 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     static_assert(QL == 1 || ((QL == 2 || QL == 4) && !GQA && (DR % 16) == 0), "multi-token decode: 2 or 4 new tokens, GVA cache, d_r a multiple of 16");
     constexpr int NBK = QL == 1 ? 1 : QL / 2;     // N-blocks of 8 columns
     const int G = p.G, H = p.H;
-    const int ql = QL == 1 ? 1 : p.q_len;         // new tokens per sequence actually present (<= QL; the other slots stay empty)
+    static_assert(CW == 1 || (QL > 1 && WPG == 1), "column-split warps belong to the multi-token kernel");
+    const int ql = QL == 1 ? 1 : p.q_len;         // new tokens per sequence (<= QL * CW; slots beyond it stay empty)
     const int HQ = H * ql;                        // pseudo-heads of the partial records
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const int n_consumers = G * WPG;
+    const int n_consumers = G * WPG * CW;
     const int stage_bytes = T::stage_bytes(G);
 
     unsigned char *tail = smem + (size_t)NSTAGE * stage_bytes;
@@ -461,8 +465,9 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         }
     } else {
         // ============ consumer: value group g, token chunks [part*CPW, part*CPW + CPW) of every tile ============
-        const int g = warp / WPG;
-        const int part = warp % WPG;
+        const int g = warp / (WPG * CW);
+        const int part = (warp / CW) % WPG;
+        const int slot_base = (warp % CW) * QL;      // multi-token decode: first new-token slot of this warp's columns
         const int jh = lane & 3;          // head within the group this lane's score/output columns belong to
         const int r8 = lane >> 2;         // row within an 8-row block
         // ldmatrix lane addressing inside a 16-token chunk of a 128-byte-swizzled box.  The 16-byte chunk index
@@ -667,18 +672,26 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             float m_run[NBK][2], l_run[NBK][2];   // per column of this lane: columns 2 jh, 2 jh + 1 of every N-block
             const float scale = p.scale_log2;
             // the lane's B-fragment column n = lane / 4 = r8 is (slot 2 nb + n / 4, head n % 4)
+            int cur_ql = ql;                       // new tokens of the current sequence
             auto load_query = [&](int b) {
+                size_t row0 = (size_t)b * ql;
+                cur_ql = ql;
+                if (p.cu_q) {                      // its own count and first query row per sequence
+                    const int r_lo = p.cu_q[b];
+                    row0 = (size_t)r_lo;
+                    cur_ql = min(max(p.cu_q[b + 1] - r_lo, 0), ql);
+                }
 #pragma unroll
                 for (int nb = 0; nb < NBK; ++nb) {
-                    const int slot = 2 * nb + (r8 >> 2), head = r8 & 3;
-                    const bool present = slot < ql;       // an absent slot gets a zero query; its columns are masked everywhere
-                    const float *q = p.q + (((size_t)b * ql + (present ? slot : 0)) * H + g * kHeadsPerGroup + head) * T::DQ;
+                    const int slot = slot_base + 2 * nb + (r8 >> 2), head = r8 & 3;
+                    const bool present = slot < cur_ql;   // an absent slot gets a zero query; its columns are masked everywhere
+                    const float *q = p.q + ((row0 + (present ? slot : 0)) * H + g * kHeadsPerGroup + head) * T::DQ;
 #pragma unroll
                     for (int kk = 0; kk < T::KSTEPS; ++kk)
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
-                            float2 v = *reinterpret_cast<const float2 *>(q + kk * 16 + half * 8 + 2 * jh);
-                            if (!present) v = make_float2(0.f, 0.f);
+                            float2 v = make_float2(0.f, 0.f);
+                            if (present) v = *reinterpret_cast<const float2 *>(q + kk * 16 + half * 8 + 2 * jh);
                             uint32_t w, wl;
                             asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(w) : "f"(v.y), "f"(v.x));
                             asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(wl) : "f"(v.y - __uint_as_float(w & 0xffff0000u)), "f"(v.x - __uint_as_float(w << 16)));
@@ -725,7 +738,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 unsigned char *vt = stage + (size_t)g * T::VTILE_BYTES;
                 const int row0 = part * CPW * 16;
                 // tokens of this tile that slot s may see: n_valid + (tokens of the sequence beyond the tile, capped) - (QL - 1 - s)
-                const int reach = n_valid + ((meta.flags >> 8) & 0xff) - (ql - 1);
+                const int reach = n_valid + min((meta.flags >> 8) & 0xff, max(cur_ql - 1, 0)) - (cur_ql - 1);
                 const bool ragged = n_valid < row0 + CPW * 16;
                 if (ragged) {
                     const int z0 = max(n_valid, row0);
@@ -738,7 +751,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                     __syncwarp();
                 }
-                const bool masked = reach < row0 + CPW * 16 || ql < QL;      // some slot does not see the whole share of this warp
+                const bool masked = reach < row0 + CPW * 16 || cur_ql < slot_base + QL;      // some slot does not see the whole share of this warp
                 const uint32_t vt_u32 = smem_u32(vt) + row0 * 128;
                 const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES) + row0 * T::KR_ROW;
 
@@ -776,8 +789,8 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 float corr[NBK][2], m_use[NBK][2];
 #pragma unroll
                 for (int nb = 0; nb < NBK; ++nb) {
-                    const int slot_l = 2 * nb + (jh >> 1);
-                    const int lim = slot_l < ql ? reach + slot_l : 0;     // tokens of the tile this slot sees (an absent slot: none)
+                    const int slot_l = slot_base + 2 * nb + (jh >> 1);
+                    const int lim = slot_l < cur_ql ? reach + slot_l : 0;     // tokens of the tile this slot sees (an absent slot: none)
                     float tmax[2] = {-INFINITY, -INFINITY};
 #pragma unroll
                     for (int c = 0; c < CPW; ++c) {
@@ -849,9 +862,10 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                             l += __shfl_xor_sync(0xffffffffu, l, 4);
                             l += __shfl_xor_sync(0xffffffffu, l, 8);
                             l += __shfl_xor_sync(0xffffffffu, l, 16);
-                            const int col = 2 * jh + e;                       // column of N-block nb: slot 2 nb + col / 4, head col % 4
-                            if (2 * nb + (col >> 2) >= ql) continue;           // (uniform over the lanes that reduce together)
-                            const size_t rh = (size_t)rec * HQ + (size_t)(2 * nb + (col >> 2)) * H + g * kHeadsPerGroup + (col & 3);
+                            const int col = 2 * jh + e;                       // column of N-block nb: slot slot_base + 2 nb + col / 4, head col % 4
+                            const int slot_w = slot_base + 2 * nb + (col >> 2);
+                            if (slot_w >= cur_ql) continue;                    // (uniform over the lanes that reduce together)
+                            const size_t rh = (size_t)rec * HQ + (size_t)slot_w * H + g * kHeadsPerGroup + (col & 3);
                             float *o_dst = p.rec_o + rh * DV;
 #pragma unroll
                             for (int mt = 0; mt < T::MT; ++mt) {
@@ -914,18 +928,19 @@ inline int mma_blocks_per_sm_cap(const gva_config &cfg, bool gqa, int smem_per_s
     return n < 1 ? 1 : (n > 4 ? 4 : n);
 }
 
-template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA, int QL = 1>
+template <int DV, int DR, int TILE, int NSTAGE, int WPG, bool GQA, int QL = 1, int CW = 1>
 int launch_mma_t(const gva_config &cfg, MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
                  int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream, int *n_blocks_out) {
     using T = MmaTraits<DV, DR, TILE, GQA>;
     const int G = cfg.G;
     const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
-    auto fn = decode_mma_kernel<DV, DR, TILE, NSTAGE, WPG, GQA, QL>;
+    auto fn = decode_mma_kernel<DV, DR, TILE, NSTAGE, WPG, GQA, QL, CW>;
     // the attribute and the occupancy figure are asked for once per (kernel, device, shared-memory size), not per call
     static int s_smem_set[kMaxDevicesCached] = {}, s_occupancy[kMaxDevicesCached] = {};
     const int dev = st.device >= 0 && st.device < kMaxDevicesCached ? st.device : 0;
-    const int threads = 32 * (G * WPG + 1);
+    const int threads = 32 * (G * WPG * CW + 1);
+    if (threads > 32 * 9) return GVA_ERR_UNSUPPORTED;
     if (s_smem_set[dev] != (int)smem || st.device >= kMaxDevicesCached) {
         if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
         int per_sm = 0;
@@ -1017,14 +1032,37 @@ int launch_decode_mma(const gva_config &cfg, MmaHostState &st, int sm_count, int
 inline int launch_decode_mma_multi(const gva_config &cfg, MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p,
                                    int B, int q_len, int max_seq_len, int num_splits, int max_blocks, cudaStream_t stream,
                                    int *n_blocks_out, int *tile_out, int *rec_mult_out) {
-    if (!mma_supported(cfg, false) || q_len < 2 || q_len > 4) return GVA_ERR_UNSUPPORTED;
-    if (!((cfg.d_v == 64 && cfg.d_r == 16) || (cfg.d_v == 128 && cfg.d_r == 32))) return GVA_ERR_UNSUPPORTED;
+    if (!mma_supported(cfg, false) || q_len < 2 || q_len > 8) return GVA_ERR_UNSUPPORTED;
+    if (q_len > 4) {       // five to eight new tokens: two consumer warps per group share each tile's columns; one block per SM with a deeper ring
+        if (!(cfg.d_v == 64 && cfg.G <= 4 && cfg.page_size % 64 == 0)) return GVA_ERR_UNSUPPORTED;
+        if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
+        *tile_out = 64;
+        *rec_mult_out = 1;
+        if (cfg.d_r == 16)
+            return launch_mma_t<64, 16, 64, 5, 1, false, 4, 2>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, stream, n_blocks_out);
+        if (cfg.d_r == 0)
+            return launch_mma_t<64, 0, 64, 5, 1, false, 4, 2>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, stream, n_blocks_out);
+        return GVA_ERR_UNSUPPORTED;
+    }
+    if (!((cfg.d_v == 64 && (cfg.d_r == 16 || cfg.d_r == 0)) || (cfg.d_v == 128 && (cfg.d_r == 32 || cfg.d_r == 0)))) return GVA_ERR_UNSUPPORTED;
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
     *tile_out = mma_tile_for(cfg, false);
     *rec_mult_out = 1;
 #define GVA_MULTI(DV_, DR_, TILE_, QL_)                                                                                       \
     return launch_mma_t<DV_, DR_, TILE_, 3, 1, false, QL_>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, \
                                                             stream, n_blocks_out)
+    if (cfg.d_r == 0) {                 // value-only cache
+        if (cfg.d_v == 64 && *tile_out == 64) {
+            if (q_len == 2) GVA_MULTI(64, 0, 64, 2);
+            GVA_MULTI(64, 0, 64, 4);
+        }
+        if (cfg.d_v == 64) {
+            if (q_len == 2) GVA_MULTI(64, 0, 32, 2);
+            GVA_MULTI(64, 0, 32, 4);
+        }
+        if (q_len == 2) GVA_MULTI(128, 0, 32, 2);
+        GVA_MULTI(128, 0, 32, 4);
+    }
     if (cfg.d_v == 64 && *tile_out == 64) {
         if (q_len == 2) GVA_MULTI(64, 16, 64, 2);
         GVA_MULTI(64, 16, 64, 4);       // three tokens run in the four-token kernel with one slot empty

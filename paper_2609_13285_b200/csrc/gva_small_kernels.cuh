@@ -603,8 +603,12 @@ combine_kernel(DecodeParams p, int wph, int hpb) {
     const int b = blockIdx.x;
     const int h = blockIdx.y * hpb + warp / wph;
     const int part = warp % wph;
-    const bool active = h < p.H;
-    const int hh = active ? h : 0;
+    // multi-token decode with its own count per sequence (cu_q): p.H = q_len * H pseudo-heads, of which sequence b uses the
+    // first (its count) * H, and its output rows start at cu_q[b]
+    const int h_real = p.H / (p.q_len > 1 ? p.q_len : 1);
+    size_t out_row0 = (size_t)b * p.H;
+    bool active = h < p.H;
+    int hh = active ? h : 0;
     if (threadIdx.x == 0) trace(kTrCombineEnterMin, p.epoch);
 
 #pragma unroll 1
@@ -613,6 +617,12 @@ combine_kernel(DecodeParams p, int wph, int hpb) {
         int first = 0, n = 1;                    // dry: record 0 only (always inside the workspace)
         if (!dry) {
             grid_dependency_wait();
+            if (p.cu_q) {      // (an input of the call, but read like everything else only once the stream's earlier work is complete)
+                const int r_lo = p.cu_q[b];
+                active = h < min(max(p.cu_q[b + 1] - r_lo, 0), p.q_len) * h_real;
+                hh = active ? h : 0;
+                out_row0 = (size_t)r_lo * h_real;
+            }
             if (p.num_splits > 0) {
                 first = b * p.num_splits * p.rec_mult;
                 n = p.num_splits * p.rec_mult;
@@ -697,10 +707,10 @@ combine_kernel(DecodeParams p, int wph, int hpb) {
         const float inv = live ? 1.f / L : 0.f;
         const float lse = live ? (mstar + log2f(L)) * kLn2 : -INFINITY;
         if (!dry && active && part == 0) {
-            float *o_dst = p.out + ((size_t)b * p.H + h) * DV + lane * DPL;
+            float *o_dst = p.out + (out_row0 + h) * DV + lane * DPL;
 #pragma unroll
             for (int d = 0; d < DPL; ++d) o_dst[d] = live ? o[d] * inv : 0.f;
-            if (p.lse && lane == 0) p.lse[(size_t)b * p.H + h] = lse;
+            if (p.lse && lane == 0) p.lse[out_row0 + h] = lse;
             if (lane == 0) {
                 trace(kTrCombineOutMin, p.epoch);
                 trace(kTrCombineOutMax, p.epoch);

@@ -229,6 +229,18 @@ class PrefillDeviceCase:
         self._ws = ws
         return self.out, self.lse
 
+    def decode_tokens_ragged(self, num_splits: int = 0):
+        """The same with every sequence's own number of new tokens (at most 8): gva_decode_tokens_ragged."""
+        c = self.pc.cache
+        max_len = int(c.seq_lens.max()) if c.B else 0
+        mq = max(self.max_q_len, 1)
+        need = gb.gva_decode_tokens_workspace_bytes(self.handle, c.B, max(mq, 2), max_len, num_splits)
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=self.q_abs.device)
+        gb.gva_decode_tokens_ragged(self.handle, self.dc.cache, self.q_abs, self.cu_q, self.dc.seq_lens, self.out, self.lse, ws,
+                                    c.B, mq, max_len, num_splits, self.status)
+        self._ws = ws
+        return self.out, self.lse
+
     def close(self) -> None:
         self.dc.close()
 

@@ -310,6 +310,10 @@ def test_decode_tokens_unsupported_and_page_size_32():
         assert int(pd.status.item()) == 0
         assert np.max(np.abs(out[:pc.n_q].cpu().numpy().astype(np.float64) - ref_out)) <= TOL_MAXABS
         ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+        # more than eight new tokens, and five to eight with pages that are not a multiple of 64 tokens, are not built
+        rc = gb.gva_decode_tokens(pd.handle, pd.dc.cache, pd.q_abs, pd.dc.seq_lens, pd.out, pd.lse, ws, 2, 9, 302, 0, check=False)
+        assert rc == gb.GVA_ERR_UNSUPPORTED
+        ws = torch.empty(gb.gva_decode_tokens_workspace_bytes(pd.handle, 2, 5, 302, 0), dtype=torch.uint8, device="cuda")
         rc = gb.gva_decode_tokens(pd.handle, pd.dc.cache, pd.q_abs, pd.dc.seq_lens, pd.out, pd.lse, ws, 2, 5, 302, 0, check=False)
         assert rc == gb.GVA_ERR_UNSUPPORTED
     finally:
@@ -434,3 +438,88 @@ def test_random_cases_through_every_multi_token_entry_point(it):
         assert np.max(np.abs(o - ref)) <= TOL_MAXABS and np.max(np.abs(l - ref_l)) <= TOL_LSE
     finally:
         pd.close()
+
+
+@pytest.mark.parametrize("q_len", [5, 6, 7, 8])
+@pytest.mark.parametrize("shape_name", ["A", "A0"])
+def test_decode_tokens_five_to_eight_new_tokens(q_len, shape_name):
+    # five to eight new tokens per sequence on the split-KV decode kernel (two consumer warps per value group share each
+    # tile's columns), over ragged contexts with poisoned slots, given and automatic split counts, flat and peaked scores
+    shape = wl.SHAPE_A if shape_name == "A" else wl.SHAPE_A0
+    for gain, splits in ((1.0, 0), (6.0, 3)):
+        pc = wl.make_prefill_case("tok8", shape, [4095 - q_len, 0, 63, 700, 64 - q_len], [q_len] * 5, page_size=64, seed=560 + q_len,
+                                  q_gain=gain, poison_unused=True)
+        ref_out, ref_lse = orc.prefill_case(pc)
+        pd = harness.upload_prefill(pc)
+        try:
+            pd.absorb()
+            out, lse = pd.decode_tokens(q_len, num_splits=splits)
+            torch.cuda.synchronize()
+            assert int(pd.status.item()) == 0
+            o = out[:pc.n_q].cpu().numpy().astype(np.float64); l = lse[:pc.n_q].cpu().numpy().astype(np.float64)
+            assert np.isfinite(o).all() and np.isfinite(l).all()
+            assert np.max(np.abs(o - ref_out)) <= TOL_MAXABS and rel_l2(o, ref_out) <= TOL_REL_L2
+            assert np.max(np.abs(l - ref_lse)) <= TOL_LSE
+        finally:
+            pd.close()
+
+
+@pytest.mark.parametrize("case_no", range(6))
+def test_decode_tokens_with_a_count_per_sequence(case_no):
+    # gva_decode_tokens_ragged: every sequence its own number of new tokens (none .. eight), against the chunked-prefill
+    # oracle; rows of sequences without new tokens do not exist, rows past the last one must stay untouched
+    rng = np.random.default_rng(8100 + case_no)
+    B = int(rng.integers(1, 9))
+    max_q = [8, 4, 2, 8, 3, 1][case_no]
+    q = rng.integers(0, max_q + 1, size=B)
+    q[int(rng.integers(0, B))] = max_q
+    ctx = rng.integers(0, 3000, size=B)
+    shape = wl.SHAPE_A if case_no != 4 else wl.SHAPE_B          # (the wide-head shape goes up to four new tokens)
+    pc = wl.make_prefill_case("rag", shape, ctx, q, page_size=64, seed=8200 + case_no, poison_unused=True, paged=bool(case_no % 2))
+    ref_out, ref_lse = orc.prefill_case(pc)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        pd.out.fill_(float("nan")); pd.lse.fill_(float("nan"))
+        out, lse = pd.decode_tokens_ragged(num_splits=0 if case_no % 3 else 2)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out[:pc.n_q].cpu().numpy().astype(np.float64); l = lse[:pc.n_q].cpu().numpy().astype(np.float64)
+        assert np.isfinite(o).all() and np.isfinite(l).all()
+        assert np.max(np.abs(o - ref_out)) <= TOL_MAXABS and np.max(np.abs(l - ref_lse)) <= TOL_LSE
+        assert torch.isnan(out[pc.n_q:]).all()
+    finally:
+        pd.close()
+
+
+def test_value_only_cache_multi_token_and_host_step():
+    # the cache without a positional slice through gva_decode_tokens (2 and 4 new tokens) and through the host-buffer step
+    for q_len in (2, 4):
+        pc = wl.make_prefill_case("vo-tok", wl.SHAPE_A0, [900, 0, 63], [q_len] * 3, page_size=64, seed=570 + q_len)
+        ref_out, _ = orc.prefill_case(pc)
+        pd = harness.upload_prefill(pc)
+        try:
+            pd.absorb()
+            out, _ = pd.decode_tokens(q_len)
+            torch.cuda.synchronize()
+            assert int(pd.status.item()) == 0
+            assert np.max(np.abs(out[:pc.n_q].cpu().numpy().astype(np.float64) - ref_out)) <= TOL_MAXABS
+        finally:
+            pd.close()
+    lens = np.array([300, 64, 1], dtype=np.int32)
+    case = wl.make_case("vo-host", wl.SHAPE_A0, lens, page_size=64, cache_dtype="bf16", seed=575, q_pos=lens - 1, append_pos=lens - 1)
+    dc = harness.upload(case)
+    try:
+        want, _ = dc.step()
+        torch.cuda.synchronize()
+        want = want.clone()
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        h_out = torch.empty(want.shape, dtype=torch.float32).pin_memory()
+        scratch = torch.empty(gb.gva_step_scratch_bytes(dc.handle, case.B, int(lens.max()), 0), dtype=torch.uint8, device="cuda")
+        gb.gva_decode_step_host(dc.handle, dc.cache, dc.M, pin(case.q_c), None, pin(case.v_new), None, pin(case.append_pos),
+                                pin(lens), h_out, scratch, case.B, int(lens.max()), 0, dc.status)
+        torch.cuda.synchronize()
+        assert int(dc.status.item()) == 0
+        assert torch.equal(h_out, want.cpu())
+    finally:
+        dc.close()
