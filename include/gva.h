@@ -75,7 +75,7 @@ typedef struct {
     int32_t d_r;           /* RoPE width: 16 or 24 with d_v = 64 (the paper's two tested widths), 32 with d_v = 128;
                               0 = value-only cache without a positional slice (Section 3.4: a cache of values alone is
                               half of matched GQA's): kr_pool, q_r and kr_new are then unused and may be NULL, scale = 1/sqrt(d_c);
-                              gva_decode_step_host, the projections and gva_decode_tokens return GVA_ERR_UNSUPPORTED */
+                              the projections (gva_project_in / _out, gva_layer_step) return GVA_ERR_UNSUPPORTED */
     int32_t page_size;     /* tokens per page, a multiple of 32                                           */
     int32_t cache_dtype;   /* gva_dtype                                                                   */
     int32_t kernel;        /* gva_kernel                                                                  */
@@ -290,8 +290,8 @@ int gva_append_chunk(gva_handle *h, const gva_cache *cache, const float *v_new, 
 /* Causal attention of the chunk over the cache, which must already hold the chunk's own tokens.
  *   q_abs [n_q][H][d_v+d_r] f32  from gva_absorb_query;  out [n_q][H][d_v] f32;  lse [n_q][H] f32 or NULL
  *   max_q_len                    upper bound on the q_len_b (sizes the launch; longer chunks are cut off)
- * bf16 cache only, page_size a multiple of 64, (d_v, d_r) = (64, 16), (128, 32), (64, 0) or (128, 0); otherwise
- * GVA_ERR_UNSUPPORTED.
+ * bf16 cache only, page_size a multiple of 64, (d_v, d_r) = (64, 16), (64, 24), (128, 32), (64, 0) or (128, 0);
+ * otherwise GVA_ERR_UNSUPPORTED.
  * Runs on the tensor cores with bf16 operands (the absorbed query and the softmax weights are rounded to bf16,
  * accumulation is f32), so results carry bf16-level error: |out - exact| <= 2e-2 for unit-variance data.
  * Device-side errors as in gva_decode; a thread block that meets one stops and leaves its rows of out unwritten. */

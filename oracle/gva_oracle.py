@@ -94,6 +94,8 @@ def rope(x, pos: float, base: float = 10000.0) -> np.ndarray:
     x = _f64(x)
     y = np.empty_like(x)
     d_r = x.shape[-1]
+    if d_r == 0:                     # value-only cache (Section 3.4): there is no positional slice to rotate
+        return y
     xf, yf = x.reshape(-1, d_r), y.reshape(-1, d_r)
     for r in range(xf.shape[0]):
         lib().oracle_rope(_p(xf[r]), ctypes.c_int(d_r), ctypes.c_double(float(pos)), ctypes.c_double(base), _p(yf[r]))

@@ -208,7 +208,7 @@ int max_units_balanced(const gva_handle *h) {
 int max_rec_mult(const gva_handle *h) {
 #ifdef GVA_WITH_MMA
     if (h->cfg.cache_dtype == GVA_E4M3) return GVA_FP8_WPG;
-    return h->cfg.d_v == 64 ? GVA_MMA_WPG64 : 1;
+    return h->cfg.d_v == 64 ? (GVA_MMA_WPG64 > GVA_MULTI_WPG ? GVA_MMA_WPG64 : GVA_MULTI_WPG) : 1;
 #else
     return 1;
 #endif
@@ -1003,8 +1003,8 @@ int gva_input_width(const gva_handle *h) { return h ? input_width(h->cfg) : 0; }
 
 int gva_pack_input_weights(const gva_handle *h, const float *W_q_nope, const float *W_q_rope, const float *W_v,
                            const float *W_r, const float *M, int d_model, uint16_t *W_in) {
-    if (!h || !W_q_nope || !W_q_rope || !W_v || !W_r || !M || !W_in || d_model <= 0) return GVA_ERR_INVALID_ARG;
-    if (h->cfg.d_r == 0) return GVA_ERR_UNSUPPORTED;     // the projections are built for the caches with a positional slice
+    if (!h || !W_q_nope || !W_v || !M || !W_in || d_model <= 0) return GVA_ERR_INVALID_ARG;
+    if (h->cfg.d_r > 0 && (!W_q_rope || !W_r)) return GVA_ERR_INVALID_ARG;     // (a value-only cache has no positional columns)
     if (h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;
     const gva_config &c = h->cfg;
     const int dq = c.d_v + c.d_r, nq = c.H * dq, nv = c.G * c.d_v, N = input_width(c);
@@ -1037,7 +1037,6 @@ int gva_project_in(gva_handle *h, const gva_cache *cache, const float *x, const 
                    const int32_t *pos, float *q_abs, int B, int32_t *dev_status, void *stream) {
     if (!h || !cache || B < 0 || d_model <= 0) return GVA_ERR_INVALID_ARG;
     if (h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;   // the fused projection writes 16- or 32-bit caches
-    if (h->cfg.d_r == 0) return GVA_ERR_UNSUPPORTED;
     if (B == 0) return GVA_OK;
     if (!x || !W_in || !pos || !q_abs || !cache->v_pool || (h->cfg.d_r > 0 && !cache->kr_pool)) return GVA_ERR_INVALID_ARG;
     if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;

@@ -65,7 +65,10 @@ struct PrefillTraits {
     static constexpr int BOXES = DV / 64;                        // 64-dim (128-byte) boxes per value row
     static constexpr int QBOX_BYTES = ROWS * 128;
     static constexpr int QV_BYTES = BOXES * QBOX_BYTES;
-    static constexpr int KR_ROW = DR * 2;                        // 32 or 64 bytes
+    static constexpr int DRP = (DR + 15) / 16 * 16;              // RoPE dims as the MMA sees them: d_r = 24 occupies 32, the
+                                                                 // last 8 zero (the TMA box is wider than the row and reads
+                                                                 // the fill value there; the query's columns are stored as 0)
+    static constexpr int KR_ROW = DRP * 2;                       // 32 or 64 bytes
     static constexpr int QR_BYTES = (ROWS * KR_ROW + 1023) & ~1023;
     static constexpr int VBOX_BYTES = TILE * 128;
     static constexpr int V_BYTES = BOXES * VBOX_BYTES;
@@ -79,9 +82,9 @@ struct PrefillTraits {
     // allow one block per SM, which then takes all 512 columns and holds hi and lo.
     static constexpr int TMEM_COLS = DV == 64 ? 256 : 512;
     static constexpr int NSBUF = 2;
-    static constexpr int COL_S = 0, COL_O = NSBUF * TILE, COL_Q = COL_O + DV, COL_QLO = COL_Q + (DV + DR) / 2;
-    static constexpr bool Q_IN_TMEM = COL_Q + (DV + DR) / 2 <= TMEM_COLS;
-    static constexpr bool LO_IN_TMEM = Q_IN_TMEM && COL_QLO + (DV + DR) / 2 <= TMEM_COLS;
+    static constexpr int COL_S = 0, COL_O = NSBUF * TILE, COL_Q = COL_O + DV, COL_QLO = COL_Q + (DV + DRP) / 2;
+    static constexpr bool Q_IN_TMEM = COL_Q + (DV + DRP) / 2 <= TMEM_COLS;
+    static constexpr bool LO_IN_TMEM = Q_IN_TMEM && COL_QLO + (DV + DRP) / 2 <= TMEM_COLS;
     // Shared memory: whichever of hi (OFF_QV / OFF_QR) and lo (OFF_LOV / OFF_LOR) is not in tensor memory.
     static constexpr int OFF_QV = 0;
     static constexpr int OFF_QR = OFF_QV + (Q_IN_TMEM ? 0 : QV_BYTES);
@@ -93,7 +96,7 @@ struct PrefillTraits {
     static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
     static_assert(NSBUF * TILE + DV <= TMEM_COLS, "the score buffers and O must fit the allocation");
     static constexpr int BLOCKS_PER_SM = 512 / TMEM_COLS;
-    static constexpr int KSTEPS_V = DV / 16, KSTEPS_R = DR / 16;
+    static constexpr int KSTEPS_V = DV / 16, KSTEPS_R = DRP / 16;
     static constexpr int THREADS = 192;
 };
 
@@ -420,9 +423,9 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                 else tmem_st4_nowait(lane_base + T::COL_Q + c * 4, hw);
             }
 #pragma unroll
-            for (int c = 0; c < DR / 8; ++c) {
+            for (int c = 0; c < T::DRP / 8; ++c) {
                 float4 a = make_float4(0.f, 0.f, 0.f, 0.f), bq = a;
-                if (live) {
+                if (live && c * 8 < DR) {
                     a = __ldg(src + DV / 4 + 2 * c);
                     bq = __ldg(src + DV / 4 + 2 * c + 1);
                 }
@@ -756,7 +759,7 @@ merge_splits_kernel(const float *__restrict__ part_o, const float *__restrict__ 
 // ---- host: support check, tensor maps, launch ---------------------------------------------------------
 inline bool prefill_supported(const gva_config &cfg) {
     return cfg.cache_dtype == GVA_BF16 && cfg.page_size % 64 == 0 && cfg.H / cfg.G == kHeadsPerGroup &&
-           ((cfg.d_v == 64 && (cfg.d_r == 16 || cfg.d_r == 0)) || (cfg.d_v == 128 && (cfg.d_r == 32 || cfg.d_r == 0)));
+           ((cfg.d_v == 64 && (cfg.d_r == 16 || cfg.d_r == 24 || cfg.d_r == 0)) || (cfg.d_v == 128 && (cfg.d_r == 32 || cfg.d_r == 0)));
 }
 
 template <int DV, int DR>
@@ -774,8 +777,8 @@ int launch_prefill_t(const gva_config &cfg, const MmaHostState &st, int smem_opt
         return GVA_ERR_CUDA;
     if (DR == 0) {
         tm_k = tm_v;      // value-only cache: there is no positional-key tile to describe (the kernel never uses this map)
-    } else if (!encode_map(st, &tm_k, kr_pool, DR, (uint64_t)p.num_pages * p.P, DR > 0 ? DR : 16, T::TILE,
-                           DR == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B)) {
+    } else if (!encode_map(st, &tm_k, kr_pool, DR, (uint64_t)p.num_pages * p.P, DR > 0 ? T::DRP : 16, T::TILE,
+                           T::DRP == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B)) {
         return GVA_ERR_CUDA;
     }
     const dim3 grid(((max_q_len + T::QTOK - 1) / T::QTOK) * p.num_splits, cfg.G, B);
@@ -802,6 +805,7 @@ inline int launch_prefill(const gva_config &cfg, const MmaHostState &st, int sme
         if (cfg.d_v == 64) return launch_prefill_t<64, 0>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
         return launch_prefill_t<128, 0>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
     }
+    if (cfg.d_v == 64 && cfg.d_r == 24) return launch_prefill_t<64, 24>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
     if (cfg.d_v == 64) return launch_prefill_t<64, 16>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
     return launch_prefill_t<128, 32>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
 }

@@ -33,7 +33,7 @@ def _dev16(a):
     return torch.from_numpy(a.view(np.int16)).cuda()
 
 
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C, wl.SHAPE_A0])
 def test_packed_weights_are_the_fp64_fold_rounded_once(shape):
     case, lw, dc, W_in, W_o = _setup(shape, [5, 70], d_model=64)
     try:
@@ -45,7 +45,8 @@ def test_packed_weights_are_the_fp64_fold_rounded_once(shape):
         dc.close()
 
 
-@pytest.mark.parametrize("shape,B", [(wl.SHAPE_A, 3), (wl.SHAPE_A, 37), (wl.SHAPE_B, 20), (wl.SHAPE_C, 130)])
+@pytest.mark.parametrize("shape,B", [(wl.SHAPE_A, 3), (wl.SHAPE_A, 37), (wl.SHAPE_B, 20), (wl.SHAPE_C, 130), (wl.SHAPE_A0, 37),
+                                     (wl.SHAPE_B0, 5)])
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_project_in_queries_and_append(shape, B, dtype):
     rng = np.random.default_rng(B)
@@ -98,7 +99,7 @@ def test_project_out(B):
         dc.close()
 
 
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_A0, wl.SHAPE_B0])
 def test_whole_layer_step_from_the_hidden_state(shape):
     lens = np.array([1, 64, 65, 700, 2049, 130], dtype=np.int32)
     d_model = 1024

@@ -165,7 +165,7 @@ def test_append_then_prefill_follows_algorithm_order():
 
 
 def test_prefill_rejects_what_it_does_not_support():
-    for kw in (dict(cache_dtype=gb.GVA_F32), dict(d_r=24), dict(page_size=32)):
+    for kw in (dict(cache_dtype=gb.GVA_F32), dict(page_size=32)):
         args = dict(H=16, G=4, d_v=64, d_c=64, d_r=16, page_size=64)
         args.update(kw)
         h = gb.gva_create(**args)
@@ -336,6 +336,28 @@ def test_prefill_and_decode_multi_value_only_cache(shape):
         assert np.max(np.abs(o - ref_out)) <= TOL_MAXABS and rel_l2(o, ref_out) <= TOL_REL_L2
     finally:
         pd.close()
+
+
+def test_prefill_and_decode_multi_rope_width_24():
+    # d_r = 24: 48-byte positional-key rows, which enter the score product as 32 dims of which the last 8 are zero on both sides
+    pc = wl.make_prefill_case("pf24", wl.SHAPE_C, [0, 70, 1000, 63], [130, 33, 5, 64], page_size=64, seed=541, poison_unused=True)
+    check(pc)
+    ref_out, ref_lse = orc.prefill_case(pc)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        for splits in (1, 3):
+            out, lse = pd.decode_multi(num_splits=splits)
+            torch.cuda.synchronize()
+            assert int(pd.status.item()) == 0
+            o = out[:pc.n_q].cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(o - ref_out)) <= TOL_MAXABS and rel_l2(o, ref_out) <= TOL_REL_L2
+            assert np.max(np.abs(lse[:pc.n_q].cpu().numpy() - ref_lse)) <= TOL_LSE
+    finally:
+        pd.close()
+    # peaked scores keep the contract there too (the query enters as hi + lo in all 32 positional columns)
+    pk = wl.make_prefill_case("pf24p", wl.SHAPE_C, [300], [100], page_size=64, seed=542, q_gain=6.0)
+    check(pk)
 
 
 def test_append_then_decode_tokens_follows_algorithm_order():
