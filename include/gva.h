@@ -255,7 +255,8 @@ int gva_input_width(const gva_handle *h);
 
 /* [host] Offline packing of one layer's input projection: folds the maps in fp64 and rounds every entry once to
  * bf16.  W_q_nope [d_model][H][d_c], W_q_rope [d_model][H][d_r], W_v [d_model][G][d_v], W_r [d_model][d_r],
- * M [H][d_v][d_c] f32 (host); W_in [d_model][N_in] bf16 bit patterns (host, caller uploads it). */
+ * M [H][d_v][d_c] f32 (host); W_in [d_model][N_in] bf16 bit patterns (host, caller uploads it).  With a value-only
+ * cache (d_r = 0) there are no positional columns: W_q_rope and W_r are unused and may be NULL. */
 int gva_pack_input_weights(const gva_handle *h, const float *W_q_nope, const float *W_q_rope, const float *W_v,
                            const float *W_r, const float *M, int d_model, uint16_t *W_in);
 /* [host] f32 -> bf16 bit patterns, nearest even (for the output projection W_o). */

@@ -208,7 +208,7 @@ int max_units_balanced(const gva_handle *h) {
 int max_rec_mult(const gva_handle *h) {
 #ifdef GVA_WITH_MMA
     if (h->cfg.cache_dtype == GVA_E4M3) return GVA_FP8_WPG;
-    return h->cfg.d_v == 64 ? (GVA_MMA_WPG64 > GVA_MULTI_WPG ? GVA_MMA_WPG64 : GVA_MULTI_WPG) : 1;
+    return h->cfg.d_v == 64 ? GVA_MMA_WPG64 : 1;
 #else
     return 1;
 #endif

@@ -899,9 +899,6 @@ inline int mma_tile_for(const gva_config &cfg, bool gqa) {
 #ifndef GVA_MMA_WPG64
 #define GVA_MMA_WPG64 1   // build-time tuning knob for the d_v = 64 kernels: 1 or 2 (measured equal; 1 halves the partial records)
 #endif
-#ifndef GVA_MULTI_WPG
-#define GVA_MULTI_WPG 1   // the same for the multi-token kernel over 64-token tiles of a d_v = 64 cache
-#endif
 inline int mma_warps_per_group(const gva_config &cfg, bool /*gqa*/) { return cfg.d_v == 64 ? GVA_MMA_WPG64 : 1; }
 
 inline bool mma_supported(const gva_config &cfg, bool gqa) {
@@ -1054,12 +1051,6 @@ inline int launch_decode_mma_multi(const gva_config &cfg, MmaHostState &st, int 
 #define GVA_MULTI(DV_, DR_, TILE_, QL_)                                                                                       \
     return launch_mma_t<DV_, DR_, TILE_, 3, 1, false, QL_>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, \
                                                             stream, n_blocks_out)
-#define GVA_MULTI_W(DV_, DR_, TILE_, QL_)                                                                                     \
-    do {                                                                                                                      \
-        *rec_mult_out = GVA_MULTI_WPG;                                                                                        \
-        return launch_mma_t<DV_, DR_, TILE_, 3, GVA_MULTI_WPG, false, QL_>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, \
-                                                                         max_blocks, stream, n_blocks_out);                   \
-    } while (0)
     if (cfg.d_r == 0) {                 // value-only cache
         if (cfg.d_v == 64 && *tile_out == 64) {
             if (q_len == 2) GVA_MULTI(64, 0, 64, 2);
@@ -1073,8 +1064,8 @@ inline int launch_decode_mma_multi(const gva_config &cfg, MmaHostState &st, int 
         GVA_MULTI(128, 0, 32, 4);
     }
     if (cfg.d_v == 64 && *tile_out == 64) {
-        if (q_len == 2) GVA_MULTI_W(64, 16, 64, 2);
-        GVA_MULTI_W(64, 16, 64, 4);     // three tokens run in the four-token kernel with one slot empty
+        if (q_len == 2) GVA_MULTI(64, 16, 64, 2);
+        GVA_MULTI(64, 16, 64, 4);       // three tokens run in the four-token kernel with one slot empty
     }
     if (cfg.d_v == 64) {
         if (q_len == 2) GVA_MULTI(64, 16, 32, 2);
@@ -1083,7 +1074,6 @@ inline int launch_decode_mma_multi(const gva_config &cfg, MmaHostState &st, int 
     if (q_len == 2) GVA_MULTI(128, 32, 32, 2);
     GVA_MULTI(128, 32, 32, 4);
 #undef GVA_MULTI
-#undef GVA_MULTI_W
 }
 
 }  // namespace gva
