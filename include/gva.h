@@ -74,8 +74,7 @@ typedef struct {
     int32_t d_c;           /* content-key width (only gva_absorb_query uses it): 1..256                   */
     int32_t d_r;           /* RoPE width: 16 or 24 with d_v = 64 (the paper's two tested widths), 32 with d_v = 128;
                               0 = value-only cache without a positional slice (Section 3.4: a cache of values alone is
-                              half of matched GQA's): kr_pool, q_r and kr_new are then unused and may be NULL, scale = 1/sqrt(d_c);
-                              the projections (gva_project_in / _out, gva_layer_step) return GVA_ERR_UNSUPPORTED */
+                              half of matched GQA's): kr_pool, q_r and kr_new are then unused and may be NULL, scale = 1/sqrt(d_c) */
     int32_t page_size;     /* tokens per page, a multiple of 32                                           */
     int32_t cache_dtype;   /* gva_dtype                                                                   */
     int32_t kernel;        /* gva_kernel                                                                  */
@@ -263,8 +262,10 @@ int gva_pack_input_weights(const gva_handle *h, const float *W_q_nope, const flo
 int gva_pack_bf16(const float *src, uint16_t *dst, size_t n);
 
 /* x [B][d_model] f32 -> q_abs [B][H][d_v+d_r] f32 (positional slice rotated at pos[b]) and the cache append of the
- * new token at pos[b] (value rows rounded to the cache dtype from the f32 product, k^rope rotated in fp64), in one
- * kernel.  Same device-side error rules as gva_append_cache. */
+ * new token at pos[b], in one kernel.  The appended rows are bit for bit what gva_append_cache writes when it is given
+ * the kernel's own f32 products as v_new / kr_new (value rows rounded once to the cache dtype, k^rope rotated in fp64
+ * and rounded once); against products accumulated in higher precision they can differ by one unit in the last place
+ * of the cache dtype.  Same device-side error rules as gva_append_cache. */
 int gva_project_in(gva_handle *h, const gva_cache *cache, const float *x, const void *W_in, int d_model,
                    const int32_t *pos, float *q_abs, int B, int32_t *dev_status, void *stream);
 /* attn [B][H*d_v] f32 (heads concatenated, as gva_decode writes them) x W_o bf16 [H*d_v][d_model] -> y [B][d_model] f32. */

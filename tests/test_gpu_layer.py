@@ -84,6 +84,41 @@ def test_project_in_queries_and_append(shape, B, dtype):
         dc.close()
 
 
+@pytest.mark.parametrize("shape,B", [(wl.SHAPE_A, 37), (wl.SHAPE_B, 9), (wl.SHAPE_C, 130)])
+def test_project_in_appends_the_rows_gva_append_cache_would_write(shape, B):
+    # The fused append rounds its f32 products exactly as gva_append_cache rounds f32 inputs.  The products themselves are read
+    # back from an f32 cache written at position 0 (a rotation by the identity, stored without rounding); appending them with
+    # gva_append_cache at the real positions must then give the same bf16 pools, bit for bit, as the fused kernel wrote.
+    lens = np.random.default_rng(B).integers(1, 600, size=B)
+    d_model = 256
+    case32, lw, dc32, W_in, _ = _setup(shape, lens, d_model, "f32")
+    try:
+        x = torch.from_numpy(lw["x"]).cuda()
+        zero = torch.zeros(B, dtype=torch.int32, device="cuda")
+        gb.gva_project_in(dc32.handle, dc32.cache, x, _dev16(W_in), d_model, zero, dc32.q_abs, B, dc32.status)
+        torch.cuda.synchronize()
+        assert int(dc32.status.item()) == 0
+        v32, k32 = dc32.pools_to_host()
+        pages = [case32.page_of(b, 0) for b in range(B)]
+        c_v = np.stack([v32[pg, :, 0] for pg in pages]).astype(np.float32)           # [B][G][d_v]
+        c_k = np.stack([k32[pg, 0] for pg in pages]).astype(np.float32)              # [B][d_r]
+    finally:
+        dc32.close()
+    case, lw2, dc, W_in2, _ = _setup(shape, lens, d_model, "bf16")
+    try:
+        assert np.array_equal(W_in, W_in2) and np.array_equal(lw["x"], lw2["x"])
+        v_b, k_b = dc.v_pool.clone(), dc.kr_pool.clone()
+        gb.gva_project_in(dc.handle, dc.cache, x, _dev16(W_in), d_model, dc.append_pos, dc.q_abs, B, dc.status)
+        other = gb.make_cache(v_b, k_b, dc.block_table, case.num_pages, case.max_pages_per_seq)
+        gb.gva_append_cache(dc.handle, other, torch.from_numpy(c_v).cuda(), torch.from_numpy(c_k).cuda(), dc.append_pos, B, dc.status)
+        torch.cuda.synchronize()
+        assert int(dc.status.item()) == 0
+        assert torch.equal(dc.v_pool.view(torch.int16), v_b.view(torch.int16))
+        assert torch.equal(dc.kr_pool.view(torch.int16), k_b.view(torch.int16))
+    finally:
+        dc.close()
+
+
 @pytest.mark.parametrize("B", [1, 33, 200])
 def test_project_out(B):
     case, lw, dc, W_in, W_o = _setup(wl.SHAPE_A, [4] * B, d_model=512)
