@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 #include <new>
 
@@ -31,6 +32,7 @@ struct gva_handle {
     int last_kernel;
     int last_tile;
     int epoch;               // number of the last decode call on this handle (see kSync* in gva_common.cuh)
+    int serial;              // number of this handle among all created in this process (see kHdrEpoch)
     int32_t *sync_base;      // device address of the sync arena on this handle's device
     int sync_off, sync_cap;  // the region of the arena in use (words)
     int n_regions;           // regions reserved so far (the earlier, smaller ones are kept until gva_destroy)
@@ -269,6 +271,7 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     if (rc_sync != GVA_OK) return rc_sync;
     p.sync = h->sync_base + h->sync_off;
     p.epoch = dry ? h->epoch : ++h->epoch;      // a dry run prepares, it does not consume an epoch
+    p.hdr_stamp = (int)((((unsigned)h->serial & 2047u) << 20) | ((unsigned)p.epoch & 0xfffffu)) + 1;
     if (h->epoch >= (1 << 30)) h->epoch = 2 + (h->epoch & 1);      // wrap, keeping the parity sequence
     if (kernel == GVA_KERNEL_MMA) {
 #ifdef GVA_WITH_MMA
@@ -407,6 +410,8 @@ int gva_create(gva_handle **out, const gva_config *cfg, int device) {
         h->sync_base = static_cast<int32_t *>(base);
         h->sync_off = h->sync_cap = h->n_regions = 0;
         h->epoch = 0;
+        static std::atomic<int> n_handles{0};
+        h->serial = n_handles.fetch_add(1);
     }
 #ifdef GVA_WITH_MMA
     int rc = mma_host_init(&h->mma, device);

@@ -20,6 +20,10 @@ constexpr int kHdrTotal = 0;        // total tiles
 constexpr int kHdrRanges = 1;       // equal contiguous ranges the tile list is cut into
 constexpr int kHdrU = 2;            // tail units per range
 constexpr int kHdrK = 3;            // tiles per tail unit
+constexpr int kHdrEpoch = 4;        // stamp of the call whose header this is (handle serial and call number), written last
+                                    // (release): a merge block that finds its own call's stamp here may use the header
+                                    // before the decode grid is done.  What stands here before is the stamp of the last
+                                    // call that used this workspace: another number of the same handle or another handle.
 // Device-side scheduling state of one handle ("sync region": int32 words inside the library image).  Every call has an
 // epoch number (1, 2, 3, ...); the call with epoch e uses the words of parity e & 1, and block 0 of its decode kernel
 // clears the words of the other parity for the call after it, so nothing has to be reset at the end of a call and a
@@ -45,6 +49,7 @@ struct DecodeParams {
     int32_t *dev_status;         // nullable
     int32_t *sync;               // this handle's sync region (see kSync*)
     int epoch;                   // this call's number on its handle (>= 1)
+    int hdr_stamp;               // (handle serial % 2048) << 20 | call number % 2^20, + 1: see kHdrEpoch
     int n_rec;                   // records the workspace holds
     int B, H, G, P, num_pages, max_pages;
     int num_splits;              // 0 = balanced flat partition
@@ -258,6 +263,9 @@ __device__ __forceinline__ void block0_duties(const DecodeParams &p, const int *
         }
         reinterpret_cast<int2 *>(p.hdr + kHdrInts)[b] = seg;
     }
+    // every one of the nt threads has stored its part (nt is a multiple of the warp size): publish the call's stamp
+    asm volatile("bar.sync 1, %0;\n" ::"r"(nt) : "memory");
+    if (tid == 0) asm volatile("st.release.gpu.global.b32 [%0], %1;\n" ::"l"(p.hdr + kHdrEpoch), "r"(p.hdr_stamp) : "memory");
 }
 
 // ---- optional in-kernel timeline (build with -DGVA_TRACE) ---------------------------------------------------

@@ -128,6 +128,10 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     }
     // Early start: as in the 16-bit kernel (see decode_mma_kernel).
     const bool early = p.early_start != 0;
+    if (tid == 0) {
+        trace(kTrDecodeEnterMin, p.epoch);
+        trace(kTrDecodeEnterMax, p.epoch);
+    }
     if (!early) grid_dependency_wait();
     compute_tile_offsets<TILE>(p, s_off);   // ends with __syncthreads(): barriers are initialised for everyone
     const BlockWork w = decode_block_work<DV>(p, s_off);
@@ -222,6 +226,10 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             const StageMeta meta = s_meta[st];
             const int n_valid = meta.n_valid;
             if (n_valid < 0) break;       // producer is done
+            if (i == 0 && tid == 0) {
+                trace(kTrFirstTileMin, p.epoch);
+                trace(kTrFirstTileMax, p.epoch);
+            }
             const int b = meta.b;
             if (meta.flags & 1) {         // a new segment: its own softmax state (and query, if the sequence changed)
                 if (b != cur_b) {
@@ -600,6 +608,10 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     }
     // keep shared memory alive until every warp (and every copy in flight) is done
     __syncthreads();
+    if (tid == 0) {
+        trace(kTrDecodeExitMin, p.epoch);
+        trace(kTrDecodeExitMax, p.epoch);
+    }
 }
 
 

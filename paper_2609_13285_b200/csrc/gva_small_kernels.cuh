@@ -611,6 +611,29 @@ combine_kernel(DecodeParams p, int wph, int hpb) {
     int hh = active ? h : 0;
     if (threadIdx.x == 0) trace(kTrCombineEnterMin, p.epoch);
 
+    // The run of records of this sequence is in the workspace header, which block 0 of the decode kernel publishes as one
+    // of the first things it does, followed by the call's stamp.  A merge block that is resident while the decode kernel
+    // streams looks for that stamp now and then (one thread, a few polls microseconds apart) and, once it is there,
+    // fetches its entry ahead of time: the real pass then starts with the records, not with one more round trip.
+    int2 seg_early = make_int2(0, -1);           // y < 0: not fetched
+    if (p.num_splits == 0) {
+        __shared__ int2 s_seg;
+        if (threadIdx.x == 0) {
+            int2 sg = make_int2(0, -1);
+            for (int it = 0; it < 48; ++it) {
+                int v;
+                asm volatile("ld.acquire.gpu.global.b32 %0, [%1];\n" : "=r"(v) : "l"(p.hdr + kHdrEpoch) : "memory");
+                if (v == p.hdr_stamp) {
+                    sg = __ldcg(reinterpret_cast<const int2 *>(p.hdr + kHdrInts) + b);
+                    break;
+                }
+                __nanosleep(it < 10 ? 400 : 4000);      // the header comes early in the decode kernel: look closely at first
+            }
+            s_seg = sg;
+        }
+        __syncthreads();
+        seg_early = s_seg;
+    }
 #pragma unroll 1
     for (int pass = 0; pass < 2; ++pass) {
         const bool dry = pass == 0;
@@ -627,7 +650,7 @@ combine_kernel(DecodeParams p, int wph, int hpb) {
                 first = b * p.num_splits * p.rec_mult;
                 n = p.num_splits * p.rec_mult;
             } else {   // this sequence's run of records, worked out by block 0 of the decode kernel
-                const int2 seg = __ldcg(reinterpret_cast<const int2 *>(p.hdr + kHdrInts) + b);
+                const int2 seg = seg_early.y >= 0 ? seg_early : __ldcg(reinterpret_cast<const int2 *>(p.hdr + kHdrInts) + b);
                 first = seg.x;
                 n = seg.y;
             }
