@@ -384,7 +384,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     // dynamic shared memory is only guaranteed 16-byte aligned: round up to the swizzle atom
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    static_assert(QL == 1 || ((QL == 2 || QL == 4) && !GQA && (DR % 16) == 0), "multi-token decode: 2 or 4 new tokens, GVA cache, d_r a multiple of 16");
+    static_assert(QL == 1 || ((QL == 2 || QL == 4) && !GQA && (DR % 8) == 0), "multi-token decode: 2 or 4 new tokens per warp, GVA cache, d_r a multiple of 8");
     constexpr int NBK = QL == 1 ? 1 : QL / 2;     // N-blocks of 8 columns
     const int G = p.G, H = p.H;
     static_assert(CW == 1 || (QL > 1 && WPG == 1), "column-split warps belong to the multi-token kernel");
@@ -668,6 +668,7 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             // the score product is taken with both (twice the score MMAs): with hi alone a score s is off by about |s| 2^-9,
             // which on sharply peaked rows is what limits the accuracy of the output.
             uint32_t qf[T::KSTEPS][NBK][2], qlo[T::KSTEPS][NBK][2];
+            uint32_t qf8[NBK], qlo8[NBK];          // d_r = 24: B fragments of the last 8 RoPE dims
             float oacc[T::MT][NBK][4];
             float m_run[NBK][2], l_run[NBK][2];   // per column of this lane: columns 2 jh, 2 jh + 1 of every N-block
             const float scale = p.scale_log2;
@@ -698,6 +699,16 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                             qf[kk][nb][half] = w;
                             qlo[kk][nb][half] = wl;
                         }
+                    qf8[nb] = qlo8[nb] = 0;
+                    if constexpr (T::KREM8) {
+                        float2 v = make_float2(0.f, 0.f);
+                        if (present) v = *reinterpret_cast<const float2 *>(q + T::KSTEPS * 16 + 2 * jh);
+                        uint32_t w, wl;
+                        asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(w) : "f"(v.y), "f"(v.x));
+                        asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(wl) : "f"(v.y - __uint_as_float(w & 0xffff0000u)), "f"(v.x - __uint_as_float(w << 16)));
+                        qf8[nb] = w;
+                        qlo8[nb] = wl;
+                    }
                 }
             };
             if (early) grid_dependency_wait();
@@ -781,6 +792,15 @@ decode_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                         for (int nb = 0; nb < NBK; ++nb) {
                             mma_bf16(sacc[c][nb], a, qlo[T::KSTEPS_V + kk][nb][0], qlo[T::KSTEPS_V + kk][nb][1]);
                             mma_bf16(sacc[c][nb], a, qf[T::KSTEPS_V + kk][nb][0], qf[T::KSTEPS_V + kk][nb][1]);
+                        }
+                    }
+                    if constexpr (T::KREM8) {     // dims 16..23: rows 0-7 and 8-15, third 16-byte chunk of each row
+                        uint32_t a2[2];
+                        ldsm_x2(kr_u32 + c * 16 * T::KR_ROW + row_qk * T::KR_ROW + 32, a2);
+#pragma unroll
+                        for (int nb = 0; nb < NBK; ++nb) {
+                            mma_bf16_k8(sacc[c][nb], a2, qlo8[nb]);
+                            mma_bf16_k8(sacc[c][nb], a2, qf8[nb]);
                         }
                     }
                 }
@@ -1038,15 +1058,24 @@ inline int launch_decode_mma_multi(const gva_config &cfg, MmaHostState &st, int 
         if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
         *tile_out = 64;
         *rec_mult_out = 1;
+        if (cfg.d_r == 24)
+            return launch_mma_t<64, 24, 64, 5, 1, false, 4, 2>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, stream, n_blocks_out);
         if (cfg.d_r == 16)
             return launch_mma_t<64, 16, 64, 5, 1, false, 4, 2>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, stream, n_blocks_out);
         if (cfg.d_r == 0)
             return launch_mma_t<64, 0, 64, 5, 1, false, 4, 2>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, stream, n_blocks_out);
         return GVA_ERR_UNSUPPORTED;
     }
-    if (!((cfg.d_v == 64 && (cfg.d_r == 16 || cfg.d_r == 0)) || (cfg.d_v == 128 && (cfg.d_r == 32 || cfg.d_r == 0)))) return GVA_ERR_UNSUPPORTED;
+    if (!((cfg.d_v == 64 && (cfg.d_r == 16 || cfg.d_r == 24 || cfg.d_r == 0)) || (cfg.d_v == 128 && (cfg.d_r == 32 || cfg.d_r == 0)))) return GVA_ERR_UNSUPPORTED;
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
     *tile_out = mma_tile_for(cfg, false);
+    if (cfg.d_r == 24) {                // 48-byte positional rows: the 64-token tile only
+        if (*tile_out != 64) return GVA_ERR_UNSUPPORTED;
+        *rec_mult_out = 1;
+        if (q_len == 2)
+            return launch_mma_t<64, 24, 64, 3, 1, false, 2>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, stream, n_blocks_out);
+        return launch_mma_t<64, 24, 64, 3, 1, false, 4>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, stream, n_blocks_out);
+    }
     *rec_mult_out = 1;
 #define GVA_MULTI(DV_, DR_, TILE_, QL_)                                                                                       \
     return launch_mma_t<DV_, DR_, TILE_, 3, 1, false, QL_>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, max_blocks, \

@@ -423,3 +423,34 @@ def test_value_only_cache_long_context():
     for kernel in KERNELS_BF16:
         _mma_or_skip(kernel)
         U().check_decode(case, kernel)
+
+
+def test_two_handles_take_turns_on_one_workspace():
+    # The merge kernel may pick up the workspace header before the decode kernel has finished, recognising it by a stamp
+    # of (handle, call number).  Two handles whose call numbers run in lockstep share one workspace here, with batches
+    # whose sequences split into different runs of records: a header left by the other handle must never be taken.
+    _mma_or_skip(gb.GVA_KERNEL_MMA)
+    a = wl.make_case("turn-a", wl.SHAPE_A, [9000, 300, 5000, 64, 12000, 1], page_size=64, cache_dtype="bf16", seed=241)
+    b = wl.make_case("turn-b", wl.SHAPE_A, [128, 15000, 2, 7000, 900, 4000], page_size=64, cache_dtype="bf16", seed=242)
+    da, db = harness.upload(a, kernel=gb.GVA_KERNEL_MMA), harness.upload(b, kernel=gb.GVA_KERNEL_MMA)
+    try:
+        ws = da.ensure_workspace(0)
+        if db.ensure_workspace(0).numel() > ws.numel():
+            ws = db.workspace
+        da.workspace = db.workspace = ws
+        da.absorb()
+        db.absorb()
+        torch.cuda.synchronize()
+        ref = {id(da): U().oracle_for_gpu_q(a, da.q_abs)[0], id(db): U().oracle_for_gpu_q(b, db.q_abs)[0]}
+        outs = []
+        for turn in range(8):                       # back to back, no synchronisation in between
+            for d in (da, db):
+                d.decode()
+                outs.append((d, d.out.clone()))
+        torch.cuda.synchronize()
+        assert int(da.status.item()) == 0 and int(db.status.item()) == 0
+        for d, o in outs:
+            assert np.max(np.abs(o.cpu().numpy().astype(np.float64) - ref[id(d)])) <= U().TOL_TIGHT_MAXABS
+    finally:
+        da.close()
+        db.close()

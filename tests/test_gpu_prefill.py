@@ -276,7 +276,7 @@ def test_decode_multi_wide_shape_and_workspace_check():
 
 # ------------------------------------------------------------------ q_len new tokens on the split-KV decode kernel
 @pytest.mark.parametrize("q_len", [2, 3, 4])
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B])
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C])
 @pytest.mark.parametrize("num_splits", [0, 1, 5])
 def test_decode_tokens_matches_oracle(q_len, shape, num_splits):
     # exactly q_len new tokens per sequence over contexts around tile and page boundaries (a context of 0 too: the first
@@ -463,11 +463,11 @@ def test_random_cases_through_every_multi_token_entry_point(it):
 
 
 @pytest.mark.parametrize("q_len", [5, 6, 7, 8])
-@pytest.mark.parametrize("shape_name", ["A", "A0"])
+@pytest.mark.parametrize("shape_name", ["A", "A0", "C"])
 def test_decode_tokens_five_to_eight_new_tokens(q_len, shape_name):
     # five to eight new tokens per sequence on the split-KV decode kernel (two consumer warps per value group share each
     # tile's columns), over ragged contexts with poisoned slots, given and automatic split counts, flat and peaked scores
-    shape = wl.SHAPE_A if shape_name == "A" else wl.SHAPE_A0
+    shape = {"A": wl.SHAPE_A, "A0": wl.SHAPE_A0, "C": wl.SHAPE_C}[shape_name]
     for gain, splits in ((1.0, 0), (6.0, 3)):
         pc = wl.make_prefill_case("tok8", shape, [4095 - q_len, 0, 63, 700, 64 - q_len], [q_len] * 5, page_size=64, seed=560 + q_len,
                                   q_gain=gain, poison_unused=True)
