@@ -971,14 +971,17 @@ int launch_project(const gva_handle *h, ProjParams p, cudaStream_t stream) {
     while (mt < m_tiles) mt *= 2;
     const size_t smem = (size_t)kProjChunk * kProjRowBytes + (size_t)16 * mt * kProjALd * sizeof(float);
     if (smem > (size_t)h->smem_optin) return GVA_ERR_UNSUPPORTED;
-    const bool f32 = MODE == 1 && h->cfg.cache_dtype != GVA_BF16;
+    const bool f32 = MODE == 1 && h->cfg.cache_dtype == GVA_F32;
+    const bool e4m3 = MODE == 1 && h->cfg.cache_dtype == GVA_E4M3;
     void (*fn)(ProjParams, RopeTable) = nullptr;
+#define GVA_PROJ(MT_) (f32 ? project_kernel<MODE, float, MT_> : e4m3 ? project_kernel<MODE, uint8_t, MT_> : project_kernel<MODE, __nv_bfloat16, MT_>)
     switch (mt) {
-        case 1: fn = f32 ? project_kernel<MODE, float, 1> : project_kernel<MODE, __nv_bfloat16, 1>; break;
-        case 2: fn = f32 ? project_kernel<MODE, float, 2> : project_kernel<MODE, __nv_bfloat16, 2>; break;
-        case 4: fn = f32 ? project_kernel<MODE, float, 4> : project_kernel<MODE, __nv_bfloat16, 4>; break;
-        default: fn = f32 ? project_kernel<MODE, float, 8> : project_kernel<MODE, __nv_bfloat16, 8>; break;
+        case 1: fn = GVA_PROJ(1); break;
+        case 2: fn = GVA_PROJ(2); break;
+        case 4: fn = GVA_PROJ(4); break;
+        default: fn = GVA_PROJ(8); break;
     }
+#undef GVA_PROJ
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((p.N + kProjStrip - 1) / kProjStrip, kProjSlices, (p.M + kProjRows - 1) / kProjRows);
@@ -1010,7 +1013,6 @@ int gva_pack_input_weights(const gva_handle *h, const float *W_q_nope, const flo
                            const float *W_r, const float *M, int d_model, uint16_t *W_in) {
     if (!h || !W_q_nope || !W_v || !M || !W_in || d_model <= 0) return GVA_ERR_INVALID_ARG;
     if (h->cfg.d_r > 0 && (!W_q_rope || !W_r)) return GVA_ERR_INVALID_ARG;     // (a value-only cache has no positional columns)
-    if (h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;
     const gva_config &c = h->cfg;
     const int dq = c.d_v + c.d_r, nq = c.H * dq, nv = c.G * c.d_v, N = input_width(c);
     for (int m = 0; m < d_model; ++m) {
@@ -1041,7 +1043,6 @@ int gva_pack_bf16(const float *src, uint16_t *dst, size_t n) {
 int gva_project_in(gva_handle *h, const gva_cache *cache, const float *x, const void *W_in, int d_model,
                    const int32_t *pos, float *q_abs, int B, int32_t *dev_status, void *stream) {
     if (!h || !cache || B < 0 || d_model <= 0) return GVA_ERR_INVALID_ARG;
-    if (h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;   // the fused projection writes 16- or 32-bit caches
     if (B == 0) return GVA_OK;
     if (!x || !W_in || !pos || !q_abs || !cache->v_pool || (h->cfg.d_r > 0 && !cache->kr_pool)) return GVA_ERR_INVALID_ARG;
     if (cache->num_pages <= 0 || cache->max_pages_per_seq <= 0) return GVA_ERR_INVALID_ARG;

@@ -102,7 +102,10 @@ __device__ __forceinline__ void project_epilogue(const ProjParams &p, const Rope
         if (n < nq + nv) {
             const int idx = n - nq, g = idx / p.d_v, d = idx % p.d_v;
             const size_t off = (((size_t)page * p.G + g) * p.P + slot) * p.d_v + d;
-            if constexpr (sizeof(CT) == 2) {
+            if constexpr (sizeof(CT) == 1) {
+                reinterpret_cast<uint16_t *>(reinterpret_cast<uint8_t *>(p.v_pool) + off)[0] =
+                    (uint16_t)((uint32_t)float_to_e4m3_bits(c0) | ((uint32_t)float_to_e4m3_bits(c1) << 8));
+            } else if constexpr (sizeof(CT) == 2) {
                 reinterpret_cast<uint32_t *>(reinterpret_cast<uint16_t *>(p.v_pool) + off)[0] =
                     (uint32_t)float_to_bf16_bits(c0) | ((uint32_t)float_to_bf16_bits(c1) << 16);
             } else {
@@ -113,7 +116,10 @@ __device__ __forceinline__ void project_epilogue(const ProjParams &p, const Rope
             double y0, y1;
             rope_pair((double)c0, (double)c1, t_pos, rope.inv_freq[i], y0, y1);
             const size_t off = ((size_t)page * p.P + slot) * p.d_r + 2 * i;
-            if constexpr (sizeof(CT) == 2) {
+            if constexpr (sizeof(CT) == 1) {
+                reinterpret_cast<uint16_t *>(reinterpret_cast<uint8_t *>(p.kr_pool) + off)[0] =
+                    (uint16_t)((uint32_t)double_to_e4m3_bits(y0) | ((uint32_t)double_to_e4m3_bits(y1) << 8));
+            } else if constexpr (sizeof(CT) == 2) {
                 reinterpret_cast<uint32_t *>(reinterpret_cast<uint16_t *>(p.kr_pool) + off)[0] =
                     (uint32_t)double_to_bf16_bits(y0) | ((uint32_t)double_to_bf16_bits(y1) << 16);
             } else {

@@ -47,8 +47,10 @@ def test_packed_weights_are_the_fp64_fold_rounded_once(shape):
 
 @pytest.mark.parametrize("shape,B", [(wl.SHAPE_A, 3), (wl.SHAPE_A, 37), (wl.SHAPE_B, 20), (wl.SHAPE_C, 130), (wl.SHAPE_A0, 37),
                                      (wl.SHAPE_B0, 5)])
-@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("dtype", ["bf16", "f32", "fp8"])
 def test_project_in_queries_and_append(shape, B, dtype):
+    if dtype == "fp8" and shape.d_r not in (16, 32):
+        pytest.skip("the 8-bit cache is built for the caches with a 16- or 32-wide positional slice")
     rng = np.random.default_rng(B)
     lens = rng.integers(1, 600, size=B)
     d_model = 256
@@ -70,22 +72,24 @@ def test_project_in_queries_and_append(shape, B, dtype):
         P = case.page_size
         touched_v = np.zeros(v1.shape[:3], dtype=bool); touched_k = np.zeros(k1.shape[:2], dtype=bool)
         to64 = wl.pool_to_f64
-        ulp = 2.0 ** -8 if dtype == "bf16" else 2.0 ** -23
+        ulp = {"bf16": 2.0 ** -8, "f32": 2.0 ** -23, "fp8": 2.0 ** -4}[dtype]      # half a unit in the last place, relative
+        tiny = 2.0 ** -10 if dtype == "fp8" else 0.0                                # ... and below the smallest normal, absolute
         for b in range(B):
             t = int(case.append_pos[b]); page, slot = case.page_of(b, t // P), t % P
             touched_v[page, :, slot] = True; touched_k[page, slot] = True
             got_v = to64(v1[page, :, slot]); ref_v = v_new[b]
             # one rounding to the cache type of an f32-accumulated product (error ~1e-6 for unit-scale values)
-            assert np.all(np.abs(got_v - ref_v) <= np.abs(ref_v) * ulp + 1e-5)
+            assert np.all(np.abs(got_v - ref_v) <= np.abs(ref_v) * ulp + tiny + 1e-5)
             got_k = to64(k1[page, slot]); ref_k = orc.rope(kr_new[b], t)
-            assert np.all(np.abs(got_k - ref_k) <= np.abs(ref_k) * ulp + 1e-5)
+            assert np.all(np.abs(got_k - ref_k) <= np.abs(ref_k) * ulp + tiny + 1e-5)
         assert np.array_equal(v1[~touched_v], v0[~touched_v]) and np.array_equal(k1[~touched_k], k0[~touched_k])
     finally:
         dc.close()
 
 
-@pytest.mark.parametrize("shape,B", [(wl.SHAPE_A, 37), (wl.SHAPE_B, 9), (wl.SHAPE_C, 130)])
-def test_project_in_appends_the_rows_gva_append_cache_would_write(shape, B):
+@pytest.mark.parametrize("shape,B,dtype", [(wl.SHAPE_A, 37, "bf16"), (wl.SHAPE_B, 9, "bf16"), (wl.SHAPE_C, 130, "bf16"),
+                                           (wl.SHAPE_A, 37, "fp8"), (wl.SHAPE_B, 9, "fp8")])
+def test_project_in_appends_the_rows_gva_append_cache_would_write(shape, B, dtype):
     # The fused append rounds its f32 products exactly as gva_append_cache rounds f32 inputs.  The products themselves are read
     # back from an f32 cache written at position 0 (a rotation by the identity, stored without rounding); appending them with
     # gva_append_cache at the real positions must then give the same bf16 pools, bit for bit, as the fused kernel wrote.
@@ -104,7 +108,7 @@ def test_project_in_appends_the_rows_gva_append_cache_would_write(shape, B):
         c_k = np.stack([k32[pg, 0] for pg in pages]).astype(np.float32)              # [B][d_r]
     finally:
         dc32.close()
-    case, lw2, dc, W_in2, _ = _setup(shape, lens, d_model, "bf16")
+    case, lw2, dc, W_in2, _ = _setup(shape, lens, d_model, dtype)
     try:
         assert np.array_equal(W_in, W_in2) and np.array_equal(lw["x"], lw2["x"])
         v_b, k_b = dc.v_pool.clone(), dc.kr_pool.clone()
@@ -113,8 +117,8 @@ def test_project_in_appends_the_rows_gva_append_cache_would_write(shape, B):
         gb.gva_append_cache(dc.handle, other, torch.from_numpy(c_v).cuda(), torch.from_numpy(c_k).cuda(), dc.append_pos, B, dc.status)
         torch.cuda.synchronize()
         assert int(dc.status.item()) == 0
-        assert torch.equal(dc.v_pool.view(torch.int16), v_b.view(torch.int16))
-        assert torch.equal(dc.kr_pool.view(torch.int16), k_b.view(torch.int16))
+        assert torch.equal(dc.v_pool.view(torch.uint8), v_b.view(torch.uint8))
+        assert torch.equal(dc.kr_pool.view(torch.uint8), k_b.view(torch.uint8))
     finally:
         dc.close()
 
@@ -134,11 +138,12 @@ def test_project_out(B):
         dc.close()
 
 
-@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_A0, wl.SHAPE_B0])
-def test_whole_layer_step_from_the_hidden_state(shape):
+@pytest.mark.parametrize("shape,dtype", [(wl.SHAPE_A, "bf16"), (wl.SHAPE_B, "bf16"), (wl.SHAPE_A0, "bf16"), (wl.SHAPE_B0, "bf16"),
+                                         (wl.SHAPE_A, "fp8"), (wl.SHAPE_B, "fp8")])
+def test_whole_layer_step_from_the_hidden_state(shape, dtype):
     lens = np.array([1, 64, 65, 700, 2049, 130], dtype=np.int32)
     d_model = 1024
-    case, lw, dc, W_in, W_o = _setup(shape, lens, d_model)
+    case, lw, dc, W_in, W_o = _setup(shape, lens, d_model, dtype)
     try:
         B = case.B
         x = torch.from_numpy(lw["x"]).cuda()
