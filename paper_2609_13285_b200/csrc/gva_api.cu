@@ -1083,8 +1083,9 @@ int gva_layer_step(gva_handle *h, const gva_cache *cache, const float *x, const 
     if (rc != GVA_OK) return rc;
     rc = gva_project_in(h, cache, x, W_in, d_model, pos, q_abs, B, dev_status, stream);
     if (rc != GVA_OK) return rc;
-    rc = gva_decode(h, cache, q_abs, seq_lens, attn, nullptr, workspace, workspace_bytes, B, max_seq_len, num_splits,
-                    dev_status, stream);
+    // (the decode kernel starts early behind the input projection, as it does behind the front kernel of gva_decode_step)
+    rc = decode_impl(h, cache, q_abs, seq_lens, attn, nullptr, workspace, workspace_bytes, B, max_seq_len, num_splits,
+                     dev_status, stream, 1, pos);
     if (rc != GVA_OK) return rc;
     return gva_project_out(h, attn, W_o, d_model, y, B, stream);
 }

@@ -142,7 +142,10 @@ constexpr int kProjALd = kProjChunk + 8;              // f32 row stride of the s
 template <int MODE, typename CT, int MT>
 __global__ void __launch_bounds__(32 * kProjWarps)
 project_kernel(ProjParams p, RopeTable rope) {
-    grid_dependency_launch();
+    // The input projection lets its dependent (the decode kernel of a layer step) start only once it has itself waited
+    // for everything earlier in the stream, as step_front_kernel does: what that kernel does ahead of its own wait then
+    // overlaps with this kernel only.  The output projection has no such follower and releases its dependent at once.
+    if constexpr (MODE != 1) grid_dependency_launch();
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ __align__(16) unsigned char psm[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -158,6 +161,7 @@ project_kernel(ProjParams p, RopeTable rope) {
     const int mt = warp % MT, ng = warp / MT;
     const int m0 = mt * 16;
     grid_dependency_wait();
+    if constexpr (MODE == 1) grid_dependency_launch();
     // the epilogue's position lookups travel with the first chunk
     int ep_pos[2] = {0, 0};
     if constexpr (MODE == 1) {
