@@ -59,8 +59,9 @@ typedef enum {
  * It is built for (d_v, d_r) = (64, 16), (64, 0), (128, 32), (128, 0), G <= 8, pages of a multiple of 64 tokens, with the
  * tensor-core kernel only:
  * gva_absorb_query, gva_append_cache, gva_append_chunk, gva_decode, gva_decode_step, gva_decode_step_host,
- * gva_decode_static, the projections, gva_layer_step and (with a positional slice, d_r > 0) gva_decode_tokens serve it;
- * gqa_decode, gva_prefill, gva_decode_multi and gva_decode_tokens_ragged return GVA_ERR_UNSUPPORTED. */
+ * gva_decode_static, gqa_decode (keys and values as e4m3 codes), the projections, gva_layer_step and (with a positional
+ * slice, d_r > 0) gva_decode_tokens serve it; gva_prefill, gva_decode_multi and gva_decode_tokens_ragged return
+ * GVA_ERR_UNSUPPORTED. */
 typedef enum { GVA_F32 = 0, GVA_BF16 = 1, GVA_E4M3 = 2 } gva_dtype;
 
 /* Which decode kernel gva_decode launches.  AUTO = tensor-core kernel when the cache is bf16 or e4m3,

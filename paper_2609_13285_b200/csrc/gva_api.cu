@@ -266,7 +266,6 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     }
     if (h->cfg.cache_dtype == GVA_E4M3) kernel = GVA_KERNEL_MMA;
     if (q_len > 1 && (GQA || kernel != GVA_KERNEL_MMA)) return GVA_ERR_UNSUPPORTED;   // multi-token decode: tensor-core kernel only
-    if (GQA && h->cfg.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;
     const int rc_sync = ensure_sync(h, w.sync_ints, stream);
     if (rc_sync != GVA_OK) return rc_sync;
     p.sync = h->sync_base + h->sync_off;
@@ -278,7 +277,7 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
         h->mma.dry = dry;
         int rc = h->cfg.cache_dtype == GVA_E4M3
                      ? launch_decode_fp8(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, q_len, max_seq_len, num_splits, stream,
-                                         &h->last_num_splits, &h->last_tile, &p.rec_mult)
+                                         &h->last_num_splits, &h->last_tile, &p.rec_mult, GQA)
                  : q_len > 1 ? launch_decode_mma_multi(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, q_len, max_seq_len, num_splits,
                                                      mma_grid_cap(h, false), stream, &h->last_num_splits, &h->last_tile, &p.rec_mult)
                            : launch_decode_mma<GQA>(h->cfg, h->mma, h->sm_count, h->smem_optin, p, B, max_seq_len, num_splits,

@@ -88,7 +88,9 @@ __device__ __forceinline__ uint32_t split_hi_lo_f16(float x) {
 // QL > 1 (multi-token decode, QL = 2 or 4 new tokens per sequence): as in the 16-bit kernel, the 4 heads x QL tokens of a
 // group are the MMA columns (plain f16 queries and weights, no hi/lo halves), slot s attends to seq_len - (QL - 1 - s)
 // tokens, and the partial records and outputs use QL * H pseudo-heads, slot * H + head.
-template <int DV, int DR, int TILE, int NSTAGE, int WPG, int GMAX, int QL = 1>
+// GQA = true (the matched GQA cache in 8 bits, single token only): a stage holds G key tiles behind the G value tiles and
+// no positional tile; the score product reads group g's key tile, the value product its value tile.
+template <int DV, int DR, int TILE, int NSTAGE, int WPG, int GMAX, int QL = 1, bool GQA = false>
 __global__ void __launch_bounds__(32 * (GMAX * WPG + 1), GMAX <= 4 ? (QL == 1 ? GVA_FP8_BLOCKS_PER_SM : GVA_FP8_QL_BLOCKS(QL)) : (QL == 1 ? 2 : 1))      // register caps: 4 five-warp blocks (d_v = 64) or 2 nine-warp blocks (d_v = 128) per SM
 decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
     using T = Fp8Traits<DV, DR, TILE>;
@@ -100,13 +102,14 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int G = p.G, H = p.H;
     static_assert(QL == 1 || QL == 2 || QL == 4, "multi-token decode: 2 or 4 new tokens");
+    static_assert(!GQA || (QL == 1 && DR == 0), "the GQA cache: single-token decode, no positional slice");
     constexpr int NBK = QL == 1 ? 1 : QL / 2;     // N-blocks of 8 columns
     const int ql = QL == 1 ? 1 : p.q_len;         // new tokens per sequence actually present (<= QL; the other slots stay empty)
     const int HQ = H * ql;                        // pseudo-heads of the partial records
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int n_consumers = G * WPG;
-    const int stage_bytes = T::stage_bytes(G);
+    const int stage_bytes = GQA ? 2 * G * T::VTILE_BYTES : T::stage_bytes(G);
 
     unsigned char *tail = smem + (size_t)NSTAGE * stage_bytes;
     uint64_t *full_bar = reinterpret_cast<uint64_t *>(tail);
@@ -156,10 +159,12 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             decode_producer<TILE, NSTAGE, (QL > 1)>(p, w, s_off, full_bar, empty_bar, s_meta, s_abort, ql,
                 [&](int st, long long page, int slot0, uint32_t bar) {
                     const uint32_t base = smem_u32(smem + (size_t)st * stage_bytes);
-                    mbar_expect_tx(bar, G * T::VTILE_BYTES + T::KR_BYTES);
-                    if constexpr (DR > 0) tma_load_2d_stream(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar, pol);
-                    for (int g = 0; g < G; ++g)
+                    mbar_expect_tx(bar, GQA ? 2 * G * T::VTILE_BYTES : G * T::VTILE_BYTES + T::KR_BYTES);
+                    if constexpr (!GQA && DR > 0) tma_load_2d_stream(base + G * T::VTILE_BYTES, &tm_k, 0, (int)(page * p.P + slot0), bar, pol);
+                    for (int g = 0; g < G; ++g) {
+                        if constexpr (GQA) tma_load_2d_stream(base + (G + g) * T::VTILE_BYTES, &tm_k, 0, (int)((page * G + g) * p.P + slot0), bar, pol);
                         tma_load_2d_stream(base + g * T::VTILE_BYTES, &tm_v, 0, (int)((page * G + g) * p.P + slot0), bar, pol);
+                    }
                 });
         }
     } else {
@@ -259,10 +264,11 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 __syncwarp();
             }
             const uint32_t vt_u32 = smem_u32(vt) + row0 * DV;
+            const uint32_t ks_u32 = GQA ? smem_u32(stage + (size_t)(G + g) * T::VTILE_BYTES) + row0 * DV : vt_u32;   // score source
             uint32_t a_qk[DV / 32], a_pv[DV / 32];            // per pair of pieces: this lane's row address within a chunk
 #pragma unroll
             for (int pr = 0; pr < DV / 32; ++pr) {
-                a_qk[pr] = vt_u32 + off_qk + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_qk) << 4);
+                a_qk[pr] = ks_u32 + off_qk + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_qk) << 4);
                 a_pv[pr] = vt_u32 + off_pv + ((((uint32_t)(2 * pr + ch_ld)) ^ swz_pv) << 4);
             }
             const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES) + row0 * T::KR_ROW;
@@ -635,7 +641,7 @@ inline bool encode_map_u8(const MmaHostState &st, CUtensorMap *map, const void *
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int DV, int DR, int TILE, int QL = 1>
+template <int DV, int DR, int TILE, int QL = 1, bool GQA = false>
 int launch_fp8_t(const gva_config &cfg, MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
                  int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out) {
     using T = Fp8Traits<DV, DR, TILE>;
@@ -643,21 +649,25 @@ int launch_fp8_t(const gva_config &cfg, MmaHostState &st, int sm_count, int smem
     constexpr int wpg = GVA_FP8_WPG;      // warps per group (each takes 1 / wpg of a tile's tokens); one measured fastest
     const int G = cfg.G;
     if (G * wpg + 1 > 9) return GVA_ERR_UNSUPPORTED;
-    const size_t smem = 1024 + (size_t)NSTAGE * T::stage_bytes(G) + T::tail_bytes(B, NSTAGE) + 16;
+    const size_t stage = GQA ? (size_t)2 * G * T::VTILE_BYTES : (size_t)T::stage_bytes(G);
+    const size_t smem = 1024 + (size_t)NSTAGE * stage + T::tail_bytes(B, NSTAGE) + 16;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
-    auto fn = G <= 4 ? decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 4, QL> : decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 8, QL>;
+    auto fn = G <= 4 ? decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 4, QL, GQA> : decode_fp8_kernel<DV, DR, TILE, NSTAGE, wpg, 8, QL, GQA>;
     static int s_smem_set[2][kMaxDevicesCached] = {};      // per (G <= 4 or not, device): the attribute is set once, not per call
     const int dev = st.device >= 0 && st.device < kMaxDevicesCached ? st.device : 0;
     if (s_smem_set[G <= 4][dev] != (int)smem || st.device >= kMaxDevicesCached) {
         if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
         s_smem_set[G <= 4][dev] = (int)smem;
     }
-    const MapPair *mp = st.find(p.v_pool, p.kr_pool, p.num_pages, 2);
+    const void *second = GQA ? p.k_pool : p.kr_pool;
+    const MapPair *mp = st.find(p.v_pool, second, p.num_pages, GQA ? 3 : 2);
     if (!mp) {
-        MapPair *m = st.slot_for(p.v_pool, p.kr_pool, p.num_pages, 2);
+        MapPair *m = st.slot_for(p.v_pool, second, p.num_pages, GQA ? 3 : 2);
         bool ok = encode_map_u8(st, &m->tm_v, p.v_pool, DV, (uint64_t)p.num_pages * G * p.P, DV, TILE,
                                 DV == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
-        if (ok && DR == 0) m->tm_k = m->tm_v;      // value-only cache: no positional tile (the kernel never uses this map)
+        if (ok && GQA) ok = encode_map_u8(st, &m->tm_k, p.k_pool, DV, (uint64_t)p.num_pages * G * p.P, DV, TILE,
+                                          DV == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
+        else if (ok && DR == 0) m->tm_k = m->tm_v;      // value-only cache: no positional tile (the kernel never uses this map)
         else if (ok) ok = encode_map_u8(st, &m->tm_k, p.kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, TILE,
                                         DR == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE);
         if (!ok) {
@@ -674,7 +684,8 @@ int launch_fp8_t(const gva_config &cfg, MmaHostState &st, int sm_count, int smem
         const long long tiles_ub = (long long)B * ((max_seq_len + TILE - 1) / TILE);
         // what the workspace is sized for; the multi-token variants: four (2 tokens) or two (4 tokens) five-warp blocks,
         // or one nine-warp block per SM
-        const int per_sm = QL == 1 ? fp8_blocks_per_sm(cfg) : (G > 4 ? 1 : GVA_FP8_QL_BLOCKS(QL));
+        const int per_sm = GQA ? (DV == 64 && G <= 4 ? 2 : 1)      // twice the tiles per stage: what the shared memory of an SM holds
+                               : QL == 1 ? fp8_blocks_per_sm(cfg) : (G > 4 ? 1 : GVA_FP8_QL_BLOCKS(QL));
         const long long want = (long long)per_sm * sm_count;
         grid = (int)(tiles_ub < want ? (tiles_ub < 1 ? 1 : tiles_ub) : want);
     }
@@ -691,11 +702,16 @@ int launch_fp8_t(const gva_config &cfg, MmaHostState &st, int sm_count, int smem
 
 inline int launch_decode_fp8(const gva_config &cfg, MmaHostState &st, int sm_count, int smem_optin, const DecodeParams &p, int B,
                              int q_len, int max_seq_len, int num_splits, cudaStream_t stream, int *n_blocks_out, int *tile_out,
-                             int *rec_mult_out) {
+                             int *rec_mult_out, bool gqa = false) {
     if (!fp8_supported(cfg)) return GVA_ERR_UNSUPPORTED;
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
     *tile_out = fp8_tile(cfg);
     *rec_mult_out = GVA_FP8_WPG;
+    if (gqa) {             // the matched GQA cache: keys and values of width d_h = d_v per group, single token
+        if (q_len > 1) return GVA_ERR_UNSUPPORTED;
+        if (cfg.d_v == 64) return launch_fp8_t<64, 0, 64, 1, true>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, stream, n_blocks_out);
+        return launch_fp8_t<128, 0, 32, 1, true>(cfg, st, sm_count, smem_optin, p, B, max_seq_len, num_splits, stream, n_blocks_out);
+    }
     if (q_len > 1) {       // multi-token decode: 2..4 new tokens per sequence, caches with a positional slice
         if (q_len > 4 || cfg.d_r == 0) return GVA_ERR_UNSUPPORTED;
 #define GVA_FP8_MULTI(DV_, DR_, TILE_, QL_) \

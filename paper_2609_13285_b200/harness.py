@@ -155,7 +155,7 @@ def upload_gqa(g: dict, device="cuda:0", kernel: int = gb.GVA_KERNEL_AUTO) -> Gq
     dev = torch.device(device)
     d_h = g["d_h"]
     handle = gb.gva_create(H=g["H"], G=g["G"], d_v=d_h, d_c=d_h, d_r=16 if d_h == 64 else 32, page_size=g["page_size"],
-                           cache_dtype=gb.GVA_BF16 if g["cache_dtype"] == "bf16" else gb.GVA_F32, kernel=kernel,
+                           cache_dtype={"bf16": gb.GVA_BF16, "fp8": gb.GVA_E4M3}.get(g["cache_dtype"], gb.GVA_F32), kernel=kernel,
                            device=dev.index or 0)
     B = g["B"]
     return GqaDeviceCase(g=g, handle=handle, k_pool=_dev(g["k_pool"], dev), v_pool=_dev(g["v_pool"], dev),
