@@ -60,7 +60,7 @@ typedef enum {
  * tensor-core kernel only:
  * gva_absorb_query, gva_append_cache, gva_append_chunk, gva_decode, gva_decode_step, gva_decode_step_host,
  * gva_decode_static, gqa_decode (keys and values as e4m3 codes), the projections, gva_layer_step and (with a positional
- * slice, d_r > 0) gva_decode_tokens serve it; gva_prefill, gva_decode_multi and gva_decode_tokens_ragged return
+ * slice, d_r > 0) gva_decode_tokens / gva_decode_tokens_ragged serve it; gva_prefill and gva_decode_multi return
  * GVA_ERR_UNSUPPORTED. */
 typedef enum { GVA_F32 = 0, GVA_BF16 = 1, GVA_E4M3 = 2 } gva_dtype;
 
@@ -341,7 +341,7 @@ int gva_decode_tokens(gva_handle *h, const gva_cache *cache, const float *q_abs,
  * already appended; its rows of q_abs / out / lse are cu_q[b] .. cu_q[b+1] - 1 (cu_q [B + 1] i32, cu_q[0] = 0,
  * non-decreasing).  seq_lens[b] = tokens attended by the last new token of b; new token i attends
  * seq_lens[b] - (q_len_b - 1 - i).  Workspace: gva_decode_tokens_workspace_bytes(h, B, max(max_q_len, 2), ...).
- * bf16 cache only; shapes as gva_decode_tokens for the given max_q_len.  Same accuracy. */
+ * Caches and shapes as gva_decode_tokens for the given max_q_len.  Same accuracy. */
 int gva_decode_tokens_ragged(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *cu_q,
                              const int32_t *seq_lens, float *out, float *lse, void *workspace, size_t workspace_bytes, int B,
                              int max_q_len, int max_seq_len, int num_splits, int32_t *dev_status, void *stream);

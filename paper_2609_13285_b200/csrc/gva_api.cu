@@ -669,7 +669,6 @@ static int decode_impl(gva_handle *h, const gva_cache *cache, const float *q_abs
     p.append_pos = append_pos;
     p.q_len = q_len;
     p.cu_q = cu_q;
-    if (cu_q && c.cache_dtype == GVA_E4M3) return GVA_ERR_UNSUPPORTED;      // a count per sequence: 16-bit cache only
     return launch_decode<false>(h, p, workspace, workspace_bytes, B, max_seq_len, num_splits,
                                 static_cast<cudaStream_t>(stream), q_len, dry);
 }

@@ -396,12 +396,20 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
             float m_run[NBK][2], l_run[NBK][2];   // per column of this lane: columns 2 jh, 2 jh + 1 of every N-block
             const float scale = p.scale_log2;
             // the lane's B-fragment column n = lane / 4 = r8 is (slot 2 nb + n / 4, head n % 4)
+            int cur_ql = ql;                       // new tokens of the current sequence
             auto load_query = [&](int b) {
+                size_t row0q = (size_t)b * ql;
+                cur_ql = ql;
+                if (p.cu_q) {                      // its own count and first query row per sequence
+                    const int r_lo = p.cu_q[b];
+                    row0q = (size_t)r_lo;
+                    cur_ql = min(max(p.cu_q[b + 1] - r_lo, 0), ql);
+                }
 #pragma unroll
                 for (int nb = 0; nb < NBK; ++nb) {
                     const int slot = 2 * nb + (r8 >> 2), head = r8 & 3;
-                    const bool present = slot < ql;       // an absent slot gets a zero query; its columns are masked everywhere
-                    const float *q = p.q + (((size_t)b * ql + (present ? slot : 0)) * H + g * kHeadsPerGroup + head) * T::DQ;
+                    const bool present = slot < cur_ql;   // an absent slot gets a zero query; its columns are masked everywhere
+                    const float *q = p.q + ((row0q + (present ? slot : 0)) * H + g * kHeadsPerGroup + head) * T::DQ;
 #pragma unroll
                     for (int kk = 0; kk < T::KSTEPS; ++kk) {
                         float4 v = *reinterpret_cast<const float4 *>(q + kk * 16 + 4 * jh);
@@ -450,7 +458,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                 unsigned char *vt = stage + (size_t)g * T::VTILE_BYTES;
                 const int row0 = part * CPW * 16;
                 // tokens of this tile that slot s may see: n_valid + (tokens of the sequence beyond the tile, capped) - (QL - 1 - s)
-                const int reach = n_valid + ((meta.flags >> 8) & 0xff) - (ql - 1);
+                const int reach = n_valid + min((meta.flags >> 8) & 0xff, max(cur_ql - 1, 0)) - (cur_ql - 1);
                 const bool ragged = n_valid < row0 + CPW * 16;
                 if (ragged) {
                     const int z0 = max(n_valid, row0);
@@ -460,7 +468,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                     __syncwarp();
                 }
-                const bool masked = reach < row0 + CPW * 16 || ql < QL;      // some slot does not see the whole share of this warp
+                const bool masked = reach < row0 + CPW * 16 || cur_ql < QL;  // some slot does not see the whole share of this warp
                 const uint32_t vt_u32 = smem_u32(vt) + row0 * DV;
                 const uint32_t kr_u32 = smem_u32(stage + (size_t)G * T::VTILE_BYTES) + row0 * T::KR_ROW;
                 uint32_t a_qk[DV / 32], a_pv[DV / 32];
@@ -519,7 +527,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
 #pragma unroll
                 for (int nb = 0; nb < NBK; ++nb) {
                     const int slot_l = 2 * nb + (jh >> 1);
-                    const int lim = slot_l < ql ? reach + slot_l : 0;     // tokens of the tile this slot sees (an absent slot: none)
+                    const int lim = slot_l < cur_ql ? reach + slot_l : 0;     // tokens of the tile this slot sees (an absent slot: none)
                     float tmax[2] = {-INFINITY, -INFINITY};
 #pragma unroll
                     for (int c = 0; c < CPW; ++c) {
@@ -595,7 +603,7 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                             l += __shfl_xor_sync(0xffffffffu, l, 8);
                             l += __shfl_xor_sync(0xffffffffu, l, 16);
                             const int col = 2 * jh + e;                       // column of N-block nb: slot 2 nb + col / 4, head col % 4
-                            if (2 * nb + (col >> 2) >= ql) continue;           // (uniform over the lanes that reduce together)
+                            if (2 * nb + (col >> 2) >= cur_ql) continue;       // (uniform over the lanes that reduce together)
                             const size_t rh = (size_t)rec * HQ + (size_t)(2 * nb + (col >> 2)) * H + g * kHeadsPerGroup + (col & 3);
                             float *o_dst = p.rec_o + rh * DV;
 #pragma unroll

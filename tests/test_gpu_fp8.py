@@ -313,6 +313,34 @@ def test_decode_tokens_matches_oracle(q_len, shape, num_splits):
         pd.close()
 
 
+@pytest.mark.parametrize("case_no", range(4))
+def test_decode_tokens_with_a_count_per_sequence(case_no):
+    # gva_decode_tokens_ragged over the 8-bit cache: every sequence its own number of new tokens (none .. four)
+    rng = np.random.default_rng(8300 + case_no)
+    B = int(rng.integers(1, 9))
+    max_q = [4, 2, 3, 4][case_no]
+    q = rng.integers(0, max_q + 1, size=B)
+    q[int(rng.integers(0, B))] = max_q
+    ctx = rng.integers(0, 3000, size=B)
+    shape = wl.SHAPE_A if case_no != 3 else wl.SHAPE_B
+    pc = wl.make_prefill_case("rag8", shape, ctx, q, page_size=64, cache_dtype="fp8", seed=8400 + case_no, poison_unused=True,
+                              paged=bool(case_no % 2))
+    ref_out, ref_lse = orc.prefill_case(pc)
+    pd = harness.upload_prefill(pc)
+    try:
+        pd.absorb()
+        pd.out.fill_(float("nan")); pd.lse.fill_(float("nan"))
+        out, lse = pd.decode_tokens_ragged(num_splits=0 if case_no % 2 else 2)
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out[:pc.n_q].cpu().numpy().astype(np.float64); l = lse[:pc.n_q].cpu().numpy().astype(np.float64)
+        assert np.isfinite(o).all() and np.isfinite(l).all()
+        assert np.max(np.abs(o - ref_out)) <= 5e-3 and np.max(np.abs(l - ref_lse)) <= 5e-3
+        assert torch.isnan(out[pc.n_q:]).all()
+    finally:
+        pd.close()
+
+
 def test_append_then_decode_tokens_follows_algorithm_order():
     # Algorithm 1 for three new tokens at once over the 8-bit cache: absorb, append all three (bit-exact codes), attend
     q_len = 3
