@@ -60,8 +60,8 @@ typedef enum {
  * tensor-core kernel only:
  * gva_absorb_query, gva_append_cache, gva_append_chunk, gva_decode, gva_decode_step, gva_decode_step_host,
  * gva_decode_static, gqa_decode (keys and values as e4m3 codes), the projections, gva_layer_step and (with a positional
- * slice, d_r > 0) gva_decode_tokens / gva_decode_tokens_ragged serve it; gva_prefill and gva_decode_multi return
- * GVA_ERR_UNSUPPORTED. */
+ * slice, d_r > 0) gva_decode_tokens / gva_decode_tokens_ragged serve it, and so do gva_prefill and gva_decode_multi (the
+ * byte tiles are widened to f16 in shared memory; queries and weights are then f16 instead of bf16). */
 typedef enum { GVA_F32 = 0, GVA_BF16 = 1, GVA_E4M3 = 2 } gva_dtype;
 
 /* Which decode kernel gva_decode launches.  AUTO = tensor-core kernel when the cache is bf16 or e4m3,
@@ -293,8 +293,8 @@ int gva_append_chunk(gva_handle *h, const gva_cache *cache, const float *v_new, 
 /* Causal attention of the chunk over the cache, which must already hold the chunk's own tokens.
  *   q_abs [n_q][H][d_v+d_r] f32  from gva_absorb_query;  out [n_q][H][d_v] f32;  lse [n_q][H] f32 or NULL
  *   max_q_len                    upper bound on the q_len_b (sizes the launch; longer chunks are cut off)
- * bf16 cache only, page_size a multiple of 64, (d_v, d_r) = (64, 16), (64, 24), (128, 32), (64, 0) or (128, 0);
- * otherwise GVA_ERR_UNSUPPORTED.
+ * bf16 or e4m3 cache, page_size a multiple of 64, (d_v, d_r) = (64, 16), (64, 24) (bf16 only), (128, 32), (64, 0) or
+ * (128, 0); otherwise GVA_ERR_UNSUPPORTED.
  * Runs on the tensor cores with bf16 operands (the absorbed query and the softmax weights are rounded to bf16,
  * accumulation is f32), so results carry bf16-level error: |out - exact| <= 2e-2 for unit-variance data.
  * Device-side errors as in gva_decode; a thread block that meets one stops and leaves its rows of out unwritten. */

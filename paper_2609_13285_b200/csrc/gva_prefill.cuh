@@ -36,6 +36,7 @@
 #pragma once
 
 #include "gva_decode_mma.cuh"
+#include "gva_decode_fp8.cuh"
 
 namespace gva {
 
@@ -56,7 +57,10 @@ struct PrefillParams {
     float *part_ml;              // [n_q][H][num_splits][2]     reference (log2 domain) and sum; (-inf, 0) for an empty range
 };
 
-template <int DV, int DR>
+// C8 = true: the 8-bit (e4m3) cache.  TMA lands the byte tiles in a raw region of the stage, the producer warp widens them
+// to f16 (exact: every e4m3 value is an f16 value) into the same swizzled operand tiles the 16-bit cache is loaded into, and
+// every MMA operand of the kernel is f16 instead of bf16 (queries as hi + lo f16, weights as f16).
+template <int DV, int DR, bool C8 = false>
 struct PrefillTraits {
     static constexpr int QTOK = 32;                              // query tokens per block
     static constexpr int ROWS = QTOK * kHeadsPerGroup;           // 128 = MMA M
@@ -73,7 +77,11 @@ struct PrefillTraits {
     static constexpr int VBOX_BYTES = TILE * 128;
     static constexpr int V_BYTES = BOXES * VBOX_BYTES;
     static constexpr int KR_BYTES = TILE * KR_ROW;
-    static constexpr int STAGE_BYTES = V_BYTES + ((KR_BYTES + 1023) & ~1023);
+    static constexpr int KR_PAD = (KR_BYTES + 1023) & ~1023;
+    static constexpr int RAW_V_BYTES = C8 ? TILE * DV : 0;        // the byte tiles as TMA delivers them (rows of d_v / d_r bytes, unswizzled)
+    static constexpr int RAW_K_BYTES = C8 ? TILE * DR : 0;
+    static constexpr int OFF_RAW = V_BYTES + KR_PAD;              // within a stage
+    static constexpr int STAGE_BYTES = OFF_RAW + ((RAW_V_BYTES + RAW_K_BYTES + 1023) & ~1023);
     // Tensor-memory columns: two score buffers (64 each; P overwrites the first 32 of its S), O (DV), and the query as bf16
     // pairs -- q = hi + lo, (DV + DR) / 2 columns each: an MMA whose A operand comes from tensor memory reads only B
     // from shared memory (measured: 128 x 64 x 16 MMAs with both operands in shared memory run at 62 cycles each -- the
@@ -92,7 +100,7 @@ struct PrefillTraits {
     static constexpr int OFF_LOR = OFF_LOV + (LO_IN_TMEM ? 0 : QV_BYTES);
     static constexpr int OFF_STAGE = OFF_LOR + (LO_IN_TMEM ? 0 : QR_BYTES);
     static constexpr int OFF_BAR = OFF_STAGE + NSTAGE * STAGE_BYTES;
-    static constexpr int N_BARS = 2 * NSTAGE + 9;
+    static constexpr int N_BARS = 2 * NSTAGE + 9 + (C8 ? NSTAGE : 0);
     static constexpr int SMEM_BYTES = 1024 + OFF_BAR + N_BARS * 8 + 16;
     static_assert(NSBUF * TILE + DV <= TMEM_COLS, "the score buffers and O must fit the allocation");
     static constexpr int BLOCKS_PER_SM = 512 / TMEM_COLS;
@@ -216,9 +224,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 }
 // Instruction descriptor of kind::f16: f32 accumulator (bits 4-5 = 1), bf16 A and B (bits 7-9, 10-12 = 1),
 // B major in bit 16 (0 = K-major, 1 = MN-major), N / 8 in bits 17-22, M / 16 in bits 24-28.
-__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
-           ((uint32_t)(M >> 4) << 24);
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, bool b_mn_major, bool f16 = false) {
+    return (1u << 4) | ((f16 ? 0u : 1u) << 7) | ((f16 ? 0u : 1u) << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);       // (A / B format fields: 0 = f16, 1 = bf16)
 }
 // Packed pairs of f32 (two lanes of one 64-bit register): one instruction for two multiply-adds / adds.
 __device__ __forceinline__ uint64_t f2_pack(float x, float y) {
@@ -303,11 +311,31 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
 }
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;\n" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+// the pair (x, y) as 16-bit floats of the kernel's operand type: bf16, or f16 over the 8-bit cache
+template <bool F16>
+__device__ __forceinline__ uint32_t pack_op(float x, float y) { return F16 ? pack_f16(x, y) : pack_bf16(x, y); }
+// ... and back to f32 (low, high element)
+template <bool F16>
+__device__ __forceinline__ void unpack_op(uint32_t w, float &x, float &y) {
+    if constexpr (F16) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w));
+        x = f.x;
+        y = f.y;
+    } else {
+        x = __uint_as_float(w << 16);
+        y = __uint_as_float(w & 0xffff0000u);
+    }
+}
 
-template <int DV, int DR>
-__global__ void __launch_bounds__(192, PrefillTraits<DV, DR>::BLOCKS_PER_SM)
+template <int DV, int DR, bool C8 = false>
+__global__ void __launch_bounds__(192, PrefillTraits<DV, DR, C8>::BLOCKS_PER_SM)
 prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k) {
-    using T = PrefillTraits<DV, DR>;
+    using T = PrefillTraits<DV, DR, C8>;
     constexpr int NS = T::NSTAGE;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int b = blockIdx.z, g = blockIdx.y;
@@ -352,6 +380,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
     auto p_full = [&](int i) { return bar0 + 8u * (2 * NS + ((i & 1) ? 8 : 3)); };
     const uint32_t q_ready = bar0 + 8u * (2 * NS + 4), drain = bar0 + 8u * (2 * NS + 5),
                    o_full = bar0 + 8u * (2 * NS + 6), drain2 = bar0 + 8u * (2 * NS + 7);
+    auto raw_full = [&](int s) { return bar0 + 8u * (2 * NS + 9 + s); };     // 8-bit cache: the byte tiles of a stage have landed
     constexpr int NB = T::NSBUF;
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + T::N_BARS);
     volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
@@ -370,6 +399,8 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         mbar_init(drain, 1);
         mbar_init(drain2, 1);
         mbar_init(o_full, 1);
+        if constexpr (C8)
+            for (int s = 0; s < NS; ++s) mbar_init(raw_full(s), 1);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
@@ -400,10 +431,13 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             // allow (with hi alone a score s is off by about |s| 2^-9, which is what limits accuracy on peaked rows).
             const float4 *src = reinterpret_cast<const float4 *>(p.q_abs + ((size_t)(q_begin + q0 + tok) * p.H + h) * (DV + DR));
             auto split4 = [](const float4 &a, uint32_t &h01, uint32_t &h23, uint32_t &l01, uint32_t &l23) {
-                h01 = pack_bf16(a.x, a.y);
-                h23 = pack_bf16(a.z, a.w);
-                l01 = pack_bf16(a.x - __uint_as_float(h01 << 16), a.y - __uint_as_float(h01 & 0xffff0000u));
-                l23 = pack_bf16(a.z - __uint_as_float(h23 << 16), a.w - __uint_as_float(h23 & 0xffff0000u));
+                float b0, b1, b2, b3;
+                h01 = pack_op<C8>(a.x, a.y);
+                h23 = pack_op<C8>(a.z, a.w);
+                unpack_op<C8>(h01, b0, b1);
+                unpack_op<C8>(h23, b2, b3);
+                l01 = pack_op<C8>(a.x - b0, a.y - b1);
+                l23 = pack_op<C8>(a.z - b2, a.w - b3);
             };
             // value dims: 16-byte piece c (8 values) of the row, as swizzled K-major rows in 128-byte boxes; then the RoPE dims
 #pragma unroll
@@ -457,7 +491,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             if (!__all_sync(0xffffffffu, mbar_wait_spin(s_full(j % NB), (j / NB) & 1, s_abort))) { ok = false; break; }   // warp-uniform
             // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
             // (the score product of this tile has completed, the value product starts only after the arrivals below)
-            if ((long long)(t_lo + j + 1) * T::TILE > kv_total) {
+            if (!C8 && (long long)(t_lo + j + 1) * T::TILE > kv_total) {      // (the 8-bit path zeroes them while it widens the tile)
                 if (tid < T::TILE && (long long)(t_lo + j) * T::TILE + tid >= kv_total) {
                     unsigned char *vrow = smem + T::OFF_STAGE + (j % NS) * T::STAGE_BYTES;
 #pragma unroll
@@ -505,7 +539,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                         e1 = fast_exp2(t1);
                     }
                     sum2[(c >> 1) & 1] = f2_add(sum2[(c >> 1) & 1], f2_pack(e0, e1));
-                    pk[c >> 1] = pack_bf16(e0, e1);
+                    pk[c >> 1] = pack_op<C8>(e0, e1);
                 }
                 float sa, sb;
                 f2_unpack(f2_add(sum2[0], sum2[1]), sa, sb);
@@ -599,9 +633,9 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         // ========== MMA issuers: warp 5 the score products, warp 4 the value products (and the TMA loads) ==========
         // One thread sustains about one tcgen05.mma per 110 cycles (measured), and a 128 x 64 x 16 MMA occupies the tensor
         // pipe for 32: two issuing threads per block (and two blocks per SM) are needed to keep the pipe fed.
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = umma_idesc(T::ROWS, T::TILE, false);
-            constexpr uint32_t idesc_o = umma_idesc(T::ROWS, DV, true);
+        if (lane == 0 && (!C8 || warp == 5)) {
+            constexpr uint32_t idesc_s = umma_idesc(T::ROWS, T::TILE, false, C8);
+            constexpr uint32_t idesc_o = umma_idesc(T::ROWS, DV, true, C8);
             constexpr uint64_t kr_swz = T::KR_ROW == 32 ? kSwz32 : kSwz64;
             constexpr uint32_t kr_sbo = 8 * T::KR_ROW;
             // Descriptors differ only in their 14-bit start-address field (low word): the high words and the other low
@@ -717,6 +751,134 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
             tc_fence_before();
         }
     }
+    if constexpr (C8) {
+        if (warp == 4) {
+            // ===== 8-bit cache: the whole warp widens the byte tiles; lane 0 also loads them and issues the value products =====
+            constexpr uint32_t idesc_o = umma_idesc(T::ROWS, DV, true, true);
+            constexpr uint32_t hi128 = (1024u >> 4) | (1u << 14) | ((uint32_t)kSwz128 << 29);
+            constexpr uint32_t lo_mn = ((uint32_t)T::VBOX_BYTES >> 4) << 16;
+            const uint32_t a_st = ((s_base + T::OFF_STAGE) & 0x3FFFFu) >> 4;
+            auto mk = [](uint32_t lo, uint32_t hi) { return (uint64_t)lo | ((uint64_t)hi << 32); };
+            constexpr int KS_O = T::TILE / 16;
+            const uint32_t tmem_c = *s_tmem;
+            bool ok = true;
+            int issued_mma = 0, loaded = 0;
+            auto load_tile = [&](int t) -> bool {        // lane 0
+                const int st = t % NS;
+                const int t0 = (t_lo + t) * T::TILE;
+                const int pj = t0 / p.P, slot0 = t0 % p.P;
+                const long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
+                                                     : (long long)b * p.max_pages + pj;
+                if (page < 0 || page >= p.num_pages) {
+                    report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
+                    *s_abort = 1;
+                    return false;
+                }
+                const uint32_t dst = s_base + T::OFF_STAGE + st * T::STAGE_BYTES + T::OFF_RAW;
+                mbar_expect_tx(raw_full(st), T::RAW_V_BYTES + T::RAW_K_BYTES);
+                tma_load_2d(dst, &tm_v, 0, (int)((page * p.G + g) * p.P + slot0), raw_full(st));
+                if constexpr (DR > 0) tma_load_2d(dst + T::RAW_V_BYTES, &tm_k, 0, (int)(page * p.P + slot0), raw_full(st));
+                ++loaded;
+                return true;
+            };
+            // Widens tile t (which must have been requested) into its stage's operand tiles: 16 codes per step and lane, two
+            // swizzled 16-byte pieces out.  Rows at or beyond the end of the cache become zeros (they may hold anything).
+            auto convert_tile = [&](int t) -> bool {     // whole warp
+                const int st = t % NS;
+                if (!__all_sync(0xffffffffu, mbar_wait_spin(raw_full(st), (t / NS) & 1, s_abort))) return false;
+                unsigned char *stage = smem + T::OFF_STAGE + st * T::STAGE_BYTES;
+                const unsigned char *raw = stage + T::OFF_RAW;
+                const long long tok0 = (long long)(t_lo + t) * T::TILE;
+                constexpr int NPV = T::TILE * (DV / 16) / 32;      // 16-byte pieces per lane
+                uint4 xv[NPV];
+#pragma unroll
+                for (int u = 0; u < NPV; ++u) {                    // all loads first: one shared-memory round trip
+                    const int pc = lane + 32 * u;
+                    xv[u] = *reinterpret_cast<const uint4 *>(raw + (pc / (DV / 16)) * DV + (pc % (DV / 16)) * 16);
+                }
+#pragma unroll
+                for (int u = 0; u < NPV; ++u) {
+                    const int pc = lane + 32 * u;
+                    const int r = pc / (DV / 16), c16 = pc % (DV / 16);
+                    uint4 x = xv[u];
+                    if (tok0 + r >= kv_total) x = make_uint4(0, 0, 0, 0);
+                    uint4 lo4, hi4;
+                    e4m3x4_to_f16x2(x.x, lo4.x, lo4.y);
+                    e4m3x4_to_f16x2(x.y, lo4.z, lo4.w);
+                    e4m3x4_to_f16x2(x.z, hi4.x, hi4.y);
+                    e4m3x4_to_f16x2(x.w, hi4.z, hi4.w);
+                    unsigned char *box = stage + (c16 / 4) * T::VBOX_BYTES;
+                    const int c = (c16 % 4) * 2;
+                    *reinterpret_cast<uint4 *>(box + swz128(r, c)) = lo4;
+                    *reinterpret_cast<uint4 *>(box + swz128(r, c + 1)) = hi4;
+                }
+                if constexpr (DR > 0) {
+                    const unsigned char *rawk = raw + T::RAW_V_BYTES;
+#pragma unroll
+                    for (int pc = lane; pc < T::TILE * (DR / 16); pc += 32) {
+                        const int r = pc / (DR / 16), c16 = pc % (DR / 16);
+                        const uint4 x = *reinterpret_cast<const uint4 *>(rawk + r * DR + c16 * 16);
+                        uint4 lo4, hi4;
+                        e4m3x4_to_f16x2(x.x, lo4.x, lo4.y);
+                        e4m3x4_to_f16x2(x.y, lo4.z, lo4.w);
+                        e4m3x4_to_f16x2(x.z, hi4.x, hi4.y);
+                        e4m3x4_to_f16x2(x.w, hi4.z, hi4.w);
+                        *reinterpret_cast<uint4 *>(stage + T::V_BYTES + swz_kr<T::KR_ROW>(r, 2 * c16)) = lo4;
+                        *reinterpret_cast<uint4 *>(stage + T::V_BYTES + swz_kr<T::KR_ROW>(r, 2 * c16 + 1)) = hi4;
+                    }
+                }
+                fence_async_smem();      // generic-proxy writes before the tensor core's reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(kv_full(st));
+                return true;
+            };
+            if (lane == 0)
+                for (int t = 0; t < NS && t < n_tiles && ok; ++t) ok = load_tile(t);
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+            for (int t = 0; t < NS && t < n_tiles && ok; ++t) ok = convert_tile(t);
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                if (lane == 0) {
+                    // every row has stored P of tile j and finished any rescaling of O
+                    if (!mbar_wait_spin(p_full(j), (j >> 1) & 1, s_abort)) ok = false;
+                    if (ok) {
+                        tc_fence_after();
+                        const uint32_t vb = a_st + (uint32_t)(j % NS) * (T::STAGE_BYTES >> 4);
+#pragma unroll
+                        for (int ks = 0; ks < KS_O; ++ks)
+                            umma_bf16_ts(tmem_c + T::COL_O, tmem_c + T::COL_S + (j % NB) * T::TILE + ks * 8,
+                                         mk((vb + ks * (16 * 128 >> 4)) | lo_mn, hi128), idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
+                        umma_commit(kv_empty(j % NS));
+                        ++issued_mma;
+                        if (j >= 1 && j - 1 + NS < n_tiles) {      // tile j-1 was consumed a tile ago: its stage takes tile j-1+NS
+                            if (!mbar_wait_spin(kv_empty((j - 1) % NS), ((j - 1) / NS) & 1, s_abort)) ok = false;
+                            else ok = load_tile(j - 1 + NS);
+                        }
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                // the tile requested one iteration ago has had that iteration to arrive; it is needed two tiles from now
+                // (widening it ahead of the value product instead, while the softmax warps work, measured slower: 2.87 ms
+                // against 2.60 ms on the prefill benchmark's shape -- the value product is what the chain waits for)
+                if (ok && j >= 2 && j - 2 + NS < n_tiles) ok = convert_tile(j - 2 + NS);
+            }
+            if (lane == 0) {
+                if (ok) umma_commit(o_full);
+                if (*s_abort) {   // copies still in flight must land before the block's shared memory is released
+                    for (int t = max(0, loaded - NS); t < loaded; ++t)
+                        for (int it = 0; it < kDrainPolls && !mbar_try_wait(raw_full(t % NS), (t / NS) & 1); ++it) {}
+                }
+                if (!ok && !*s_abort) {
+                    report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
+                    *s_abort = 1;
+                }
+                if (issued_mma > 0) {
+                    umma_commit(drain2);
+                    for (int it = 0; it < kDrainPolls * 16 && !mbar_try_wait(drain2, 0); ++it) {}
+                }
+                tc_fence_before();
+            }
+        }
+    }
     grid_dependency_launch();
     __syncthreads();
     if (warp == 5) {
@@ -758,24 +920,31 @@ merge_splits_kernel(const float *__restrict__ part_o, const float *__restrict__ 
 
 // ---- host: support check, tensor maps, launch ---------------------------------------------------------
 inline bool prefill_supported(const gva_config &cfg) {
-    return cfg.cache_dtype == GVA_BF16 && cfg.page_size % 64 == 0 && cfg.H / cfg.G == kHeadsPerGroup &&
+    if (cfg.cache_dtype == GVA_E4M3 && cfg.d_r == 24) return false;
+    return (cfg.cache_dtype == GVA_BF16 || cfg.cache_dtype == GVA_E4M3) && cfg.page_size % 64 == 0 && cfg.H / cfg.G == kHeadsPerGroup &&
            ((cfg.d_v == 64 && (cfg.d_r == 16 || cfg.d_r == 24 || cfg.d_r == 0)) || (cfg.d_v == 128 && (cfg.d_r == 32 || cfg.d_r == 0)));
 }
 
-template <int DV, int DR>
+template <int DV, int DR, bool C8 = false>
 int launch_prefill_t(const gva_config &cfg, const MmaHostState &st, int smem_optin, const PrefillParams &p, const void *v_pool,
                      const void *kr_pool, int B, int max_q_len, int n_q, cudaStream_t stream) {
-    using T = PrefillTraits<DV, DR>;
+    using T = PrefillTraits<DV, DR, C8>;
     // never more blocks on an SM than its 512 tensor-memory columns can serve: pad the request if need be
     const size_t floor_bytes = (size_t)227 * 1024 / (T::BLOCKS_PER_SM + 1) + 1024;
     const size_t smem = (size_t)T::SMEM_BYTES < floor_bytes ? floor_bytes : (size_t)T::SMEM_BYTES;
     if (smem > (size_t)smem_optin) return GVA_ERR_UNSUPPORTED;
-    auto fn = prefill_kernel<DV, DR>;
+    auto fn = prefill_kernel<DV, DR, C8>;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GVA_ERR_CUDA;
     CUtensorMap tm_v, tm_k;
-    if (!encode_map(st, &tm_v, v_pool, DV, (uint64_t)p.num_pages * cfg.G * p.P, 64, T::TILE, CU_TENSOR_MAP_SWIZZLE_128B))
+    if constexpr (C8) {       // byte tiles, unswizzled: rows of d_v and of d_r codes
+        if (!encode_map_u8(st, &tm_v, v_pool, DV, (uint64_t)p.num_pages * cfg.G * p.P, DV, T::TILE, CU_TENSOR_MAP_SWIZZLE_NONE))
+            return GVA_ERR_CUDA;
+        if (DR == 0) tm_k = tm_v;
+        else if (!encode_map_u8(st, &tm_k, kr_pool, DR, (uint64_t)p.num_pages * p.P, DR, T::TILE, CU_TENSOR_MAP_SWIZZLE_NONE))
+            return GVA_ERR_CUDA;
+    } else if (!encode_map(st, &tm_v, v_pool, DV, (uint64_t)p.num_pages * cfg.G * p.P, 64, T::TILE, CU_TENSOR_MAP_SWIZZLE_128B)) {
         return GVA_ERR_CUDA;
-    if (DR == 0) {
+    } else if (DR == 0) {
         tm_k = tm_v;      // value-only cache: there is no positional-key tile to describe (the kernel never uses this map)
     } else if (!encode_map(st, &tm_k, kr_pool, DR, (uint64_t)p.num_pages * p.P, DR > 0 ? T::DRP : 16, T::TILE,
                            T::DRP == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B)) {
@@ -801,6 +970,13 @@ inline int launch_prefill(const gva_config &cfg, const MmaHostState &st, int sme
                           const void *v_pool, const void *kr_pool, int B, int max_q_len, int n_q, cudaStream_t stream) {
     if (!prefill_supported(cfg)) return GVA_ERR_UNSUPPORTED;
     if ((uint64_t)p.num_pages * cfg.G * cfg.page_size >= (1ull << 31)) return GVA_ERR_UNSUPPORTED;
+    if (cfg.cache_dtype == GVA_E4M3) {
+        if (cfg.d_v == 64)
+            return cfg.d_r == 16 ? launch_prefill_t<64, 16, true>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream)
+                                 : launch_prefill_t<64, 0, true>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
+        return cfg.d_r == 32 ? launch_prefill_t<128, 32, true>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream)
+                             : launch_prefill_t<128, 0, true>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
+    }
     if (cfg.d_r == 0) {       // value-only cache
         if (cfg.d_v == 64) return launch_prefill_t<64, 0>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);
         return launch_prefill_t<128, 0>(cfg, st, smem_optin, p, v_pool, kr_pool, B, max_q_len, n_q, stream);

@@ -224,16 +224,60 @@ def test_what_the_8_bit_cache_does_not_cover():
         with pytest.raises(gb.GvaError) as e:
             gb.gva_create(cache_dtype=gb.GVA_E4M3, **kw)
         assert e.value.status == gb.GVA_ERR_UNSUPPORTED
-    pc = wl.make_prefill_case("pf8", wl.SHAPE_A, [64, 0], [4, 4], page_size=64, cache_dtype="fp8", seed=811)
+
+
+@pytest.mark.parametrize("shape", [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_A0])
+def test_prefill_and_decode_multi_over_the_8_bit_cache(shape):
+    # the tcgen05 kernel over e4m3 tiles: the producer warp widens them to f16 in shared memory, queries (hi + lo) and
+    # weights are f16; ragged chunks over contexts around tile boundaries, poisoned unused slots, flat and peaked scores
+    for gain in (1.0, 6.0):
+        pc = wl.make_prefill_case("pf8", shape, [0, 70, 1000, 63, 5], [130, 33, 5, 64, 300], page_size=64, cache_dtype="fp8",
+                                  seed=811, poison_unused=True, q_gain=gain)
+        ref_out, ref_lse = orc.prefill_case(pc)
+        pd = harness.upload_prefill(pc)
+        try:
+            pd.absorb()
+            for call in (pd.prefill, lambda: pd.decode_multi(num_splits=0), lambda: pd.decode_multi(num_splits=3)):
+                pd.out.fill_(float("nan"))
+                out, lse = call()
+                torch.cuda.synchronize()
+                assert int(pd.status.item()) == 0
+                o = out[:pc.n_q].cpu().numpy().astype(np.float64); l = lse[:pc.n_q].cpu().numpy().astype(np.float64)
+                assert np.isfinite(o).all() and np.isfinite(l).all()
+                assert np.max(np.abs(o - ref_out)) <= 2e-2, np.max(np.abs(o - ref_out))
+                assert U().rel_l2(o, ref_out) <= 1e-2
+                assert np.max(np.abs(l - ref_lse)) <= 2e-2
+        finally:
+            pd.close()
+
+
+def test_prefill_bench_size_over_the_8_bit_cache_sampled_rows():
+    # the prefill benchmark's shape (8 prompts of 8192 tokens) over e4m3 codes, same launch: sampled query rows one by one
+    # against the decode oracle over the row's prefix, finiteness for the rest
+    pc = wl.make_prefill_case("prefill8", wl.SHAPE_A, [0] * 8, [8192] * 8, page_size=64, cache_dtype="fp8", seed=wl.MASTER_SEED + 7100)
+    c, s = pc.cache, pc.cache.shape
     pd = harness.upload_prefill(pc)
     try:
         pd.absorb()
-        for call in (pd.prefill, lambda: pd.decode_multi(num_splits=0)):
-            with pytest.raises(gb.GvaError) as e:
-                call()
-            assert e.value.status == gb.GVA_ERR_UNSUPPORTED
+        out, lse = pd.prefill()
+        torch.cuda.synchronize()
+        assert int(pd.status.item()) == 0
+        o = out.cpu().numpy().astype(np.float64)
+        l = lse.cpu().numpy().astype(np.float64)
+        q_abs = pd.q_abs.cpu().numpy().astype(np.float64)
     finally:
         pd.close()
+    assert np.isfinite(o).all() and np.isfinite(l).all()
+    T = int(pc.q_lens[0])
+    rng = np.random.default_rng(9)
+    for b in (0, c.B - 1):
+        for t in sorted(set([0, 1, 63, 64, 65, 127, 128, 4095, 4096, T - 33, T - 1] + rng.integers(0, T, size=5).tolist())):
+            n = int(pc.cu_q[b]) + t
+            lens = np.zeros(c.B, dtype=np.int32); lens[b] = t + 1
+            qa = np.zeros((c.B, s.H, s.d_v + s.d_r)); qa[b] = q_abs[n]
+            ref_o, ref_l = orc.decode(c.v_pool, c.kr_pool, c.block_table, lens, qa, s.H, d_c=s.d_c)
+            assert np.max(np.abs(o[n] - ref_o[b])) <= 2e-2, (b, t)
+            assert np.max(np.abs(l[n] - ref_l[b])) <= 2e-2, (b, t)
 
 
 def test_full_size_long_context_sampled():
