@@ -732,15 +732,19 @@ int gva_decode_step(gva_handle *h, const gva_cache *cache, const float *M, const
     a.v_pool = cache->v_pool; a.kr_pool = cache->kr_pool; a.dev_status = dev_status;
     a.B = B; a.H = c.H; a.G = c.G; a.d_v = c.d_v; a.d_c = c.d_c; a.d_r = c.d_r; a.P = c.page_size;
     a.num_pages = cache->num_pages; a.max_pages = cache->max_pages_per_seq;
-    a.n_absorb = c.H * ((B + kAbsorbBatch - 1) / kAbsorbBatch);
+    // sequences per absorb item: 16 where that keeps the grid at one block per SM and the thread mapping allows it
+    a.fold = c.H * ((B + kAbsorbBatch - 1) / kAbsorbBatch) + B > h->sm_count ? 1 : 0;
+    a.batch = (a.fold && kAbsorbBatchMax * c.d_v <= 4 * kAbsorbThreads) ? kAbsorbBatchMax : kAbsorbBatch;
+    a.n_absorb = c.H * ((B + a.batch - 1) / a.batch);
+    const int front_grid = a.fold ? (a.n_absorb > B ? a.n_absorb : B) : a.n_absorb + B;
     a.trace_call = h->epoch + 1;
     const size_t smem = absorb_smem_bytes(c.d_v, c.d_c);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const cudaError_t ce = (c.cache_dtype == GVA_E4M3)
-        ? launch_pdl(step_front_kernel<uint8_t>, dim3(a.n_absorb + B), dim3(kAbsorbThreads), smem, st, a, h->rope)
+        ? launch_pdl(step_front_kernel<uint8_t>, dim3(front_grid), dim3(kAbsorbThreads), smem, st, a, h->rope)
         : (c.cache_dtype == GVA_BF16)
-        ? launch_pdl(step_front_kernel<__nv_bfloat16>, dim3(a.n_absorb + B), dim3(kAbsorbThreads), smem, st, a, h->rope)
-        : launch_pdl(step_front_kernel<float>, dim3(a.n_absorb + B), dim3(kAbsorbThreads), smem, st, a, h->rope);
+        ? launch_pdl(step_front_kernel<__nv_bfloat16>, dim3(front_grid), dim3(kAbsorbThreads), smem, st, a, h->rope)
+        : launch_pdl(step_front_kernel<float>, dim3(front_grid), dim3(kAbsorbThreads), smem, st, a, h->rope);
     if (ce != cudaSuccess) {
         (void)cudaGetLastError();
         return GVA_ERR_CUDA;

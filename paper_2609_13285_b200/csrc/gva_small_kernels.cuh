@@ -46,25 +46,33 @@ __device__ __forceinline__ void rope_pair(double x0, double x1, int pos, double 
 // (row stride d_c + 4 floats: 16-byte aligned for cp.async and conflict-free for 16-byte row-per-thread
 // reads), and reused for kAbsorbBatch sequences.
 constexpr int kAbsorbBatch = 8;
+constexpr int kAbsorbBatchMax = 16;      // the fused front of a decode step takes 16 sequences per block for large batches of
+                                         // the 64-wide shape, so that its grid stays at one block per SM (see step_front_kernel)
 constexpr int kAbsorbThreads = 256;
 
 // Shared-memory row stride of the staged map, in floats: d_c + 4 keeps rows 16-byte aligned for cp.async.
 __host__ __device__ __forceinline__ int absorb_row_stride(int d_c) { return d_c + 4; }
 __host__ __device__ __forceinline__ size_t absorb_smem_bytes(int d_v, int d_c) {
-    return ((size_t)d_v * absorb_row_stride(d_c) + (size_t)kAbsorbBatch * d_c) * sizeof(float);
+    return ((size_t)d_v * absorb_row_stride(d_c) + (size_t)kAbsorbBatchMax * d_c) * sizeof(float);
 }
 
-// One block's share: head h, sequences [b0, b0 + kAbsorbBatch).  All kAbsorbThreads threads must call it.
+// One block's share: head h, sequences [b0, b0 + batch), batch <= kAbsorbBatchMax.  All kAbsorbThreads threads must call it.
 // Every global read is requested up front -- M_h and the query rows as 16-byte cp.async copies straight into
 // shared memory, the RoPE inputs into registers -- so the block pays one memory round trip.
+// `overlap` is called once by every thread while the copies are in flight (a caller's own latency-bound work).
+struct NoOverlap {
+    __device__ __forceinline__ void operator()() const {}
+};
+template <typename Overlap = NoOverlap>
 __device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, const float *__restrict__ q_r,
                                              const float *__restrict__ M, const int32_t *__restrict__ q_pos,
                                              float *__restrict__ q_abs, int B, int H, int d_v, int d_c, int d_r,
-                                             const RopeTable &rope, int h, int b0, float *smem_f) {
+                                             const RopeTable &rope, int h, int b0, float *smem_f, int batch = kAbsorbBatch,
+                                             Overlap overlap = Overlap()) {
     const int ld = absorb_row_stride(d_c);
     float *sM = smem_f;                            // [d_v][ld]
-    float *sq = smem_f + d_v * ld;                 // [kAbsorbBatch][d_c]
-    const int nb = min(kAbsorbBatch, B - b0);
+    float *sq = smem_f + d_v * ld;                 // [batch][d_c]
+    const int nb = min(batch, B - b0);
     const int tid = threadIdx.x;
     const float *Mh = M + (size_t)h * d_v * d_c;
     const int dq = d_v + d_r;
@@ -89,7 +97,7 @@ __device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, cons
     }
     float r0 = 0.f, r1 = 0.f;
     int rpos = 0;
-    const bool has_rope = tid < nb * half;      // nb * half <= 8 * 16 < kAbsorbThreads
+    const bool has_rope = tid < nb * half;      // nb * half <= 16 * 16 = kAbsorbThreads
     if (has_rope) {
         const int bb = tid / half, i = tid % half;
         const size_t src = ((size_t)(b0 + bb) * H + h) * d_r + 2 * i;
@@ -105,11 +113,12 @@ __device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, cons
         dst[0] = __double2float_rn(y0);
         dst[1] = __double2float_rn(y1);
     }
+    overlap();
     if (vec) cp_async_wait<0>();
     __syncthreads();
     // Thread t owns map row i = t % d_v for sequences bb0, bb0 + step, ... (kAbsorbThreads % d_v == 0), so one
     // read of M_h[i][j] feeds up to four independent accumulators.
-    if (kAbsorbThreads % d_v == 0 && kAbsorbBatch * d_v <= 4 * kAbsorbThreads) {
+    if (kAbsorbThreads % d_v == 0 && batch * d_v <= 4 * kAbsorbThreads) {
         const int i = tid % d_v, bb0 = tid / d_v, step = kAbsorbThreads / d_v;
         const float *mrow = sM + i * ld;
         const float *q0 = sq + min(bb0, nb - 1) * d_c, *q1 = sq + min(bb0 + step, nb - 1) * d_c;
@@ -319,53 +328,81 @@ absorb_rows_mma_kernel(const float *__restrict__ q_c, const float *__restrict__ 
 // block-table entry) overlap with them.
 constexpr int kAppendMaxPerThread = 8;    // G * d_v <= 8 * 128 elements (blocks have at least 128 threads)
 
-// One sequence's append.  Every thread of the block must call it (blockDim.x >= 128).
-// Writes input row `row` (v_new[row], kr_new[row]) as token `t` of sequence `seq`.
-template <typename CT>
-__device__ __forceinline__ void append_row(CT *__restrict__ v_pool, CT *__restrict__ kr_pool,
-                                           const int32_t *__restrict__ block_table, const float *__restrict__ v_new,
-                                           const float *__restrict__ kr_new, int G, int d_v, int d_r, int P, int num_pages,
-                                           int max_pages, int32_t *dev_status, const RopeTable &rope, int row, int seq, int t) {
+// One sequence's append in steps, so that a caller can put other work between the loads and what depends on them:
+// append_load requests the new row (nothing it returns is looked at yet), append_locate looks up the page of position t
+// (a dependent load: the position itself usually comes from memory), append_rotate rotates the positional pair,
+// append_store checks the page, rounds and writes.  Every thread of the block must call all four (blockDim.x >= 128).
+// Input row `row` (v_new[row], kr_new[row]) becomes token `t` of sequence `seq`.
+struct AppendRegs {
+    float x[kAppendMaxPerThread];
+    float k0, k1;
+    double y0, y1;       // the rotated pair, once append_rotate has run
+    long long page;      // as looked up; checked by append_store
+    int t;               // -1: position outside the block table (reported by append_locate), nothing is written
+    int rope_tid0;       // threads [rope_tid0, rope_tid0 + d_r / 2) hold the positional pairs
+};
+__device__ __forceinline__ AppendRegs append_load(const float *__restrict__ v_new, const float *__restrict__ kr_new, int G,
+                                                  int d_v, int d_r, int row, int rope_tid0 = 0) {
+    AppendRegs r;
+    r.rope_tid0 = rope_tid0;
     const int n_v = G * d_v;
     const int nt = blockDim.x;
-    const int b = seq;
-    float x[kAppendMaxPerThread];
 #pragma unroll
     for (int u = 0; u < kAppendMaxPerThread; ++u) {
         const int i = u * nt + threadIdx.x;
-        x[u] = (i < n_v) ? v_new[(size_t)row * n_v + i] : 0.f;
+        r.x[u] = (i < n_v) ? v_new[(size_t)row * n_v + i] : 0.f;
     }
-    float k0 = 0.f, k1 = 0.f;
-    if (threadIdx.x < d_r / 2) {
-        k0 = kr_new[(size_t)row * d_r + 2 * threadIdx.x];
-        k1 = kr_new[(size_t)row * d_r + 2 * threadIdx.x + 1];
+    r.k0 = r.k1 = 0.f;
+    const int rk = (int)threadIdx.x - rope_tid0;
+    if (rk >= 0 && rk < d_r / 2) {
+        r.k0 = kr_new[(size_t)row * d_r + 2 * rk];
+        r.k1 = kr_new[(size_t)row * d_r + 2 * rk + 1];
     }
+    r.t = -1;
+    r.page = -1;
+    r.y0 = r.y1 = 0.0;
+    return r;
+}
+__device__ __forceinline__ void append_locate(AppendRegs &r, const int32_t *__restrict__ block_table, int P, int max_pages,
+                                              int32_t *dev_status, int seq, int t) {
     if (t < 0 || t / P >= max_pages) {
-        if (threadIdx.x == 0) report_error(dev_status, GVA_ERR_SEQ_LEN, b);
+        if (threadIdx.x == 0) report_error(dev_status, GVA_ERR_SEQ_LEN, seq);
         return;
     }
-    const long long page = block_table ? (long long)block_table[(size_t)b * max_pages + t / P]
-                                       : (long long)b * max_pages + t / P;
-    if (page < 0 || page >= num_pages) {
-        if (threadIdx.x == 0) report_error(dev_status, GVA_ERR_BAD_PAGE, b);
+    r.t = t;
+    r.page = block_table ? (long long)block_table[(size_t)seq * max_pages + t / P] : (long long)seq * max_pages + t / P;
+}
+// The rotation of the positional pair (fp64).
+__device__ __forceinline__ void append_rotate(AppendRegs &r, int d_r, const RopeTable &rope) {
+    const int i = (int)threadIdx.x - r.rope_tid0;
+    if (r.t >= 0 && i >= 0 && i < d_r / 2) rope_pair((double)r.k0, (double)r.k1, r.t, rope.inv_freq[i], r.y0, r.y1);
+}
+template <typename CT>
+__device__ __forceinline__ void append_store(const AppendRegs &r, CT *__restrict__ v_pool, CT *__restrict__ kr_pool, int G,
+                                             int d_v, int d_r, int P, int num_pages, int32_t *dev_status, int seq) {
+    if (r.t < 0) return;
+    if (r.page < 0 || r.page >= num_pages) {
+        if (threadIdx.x == 0) report_error(dev_status, GVA_ERR_BAD_PAGE, seq);
         return;
     }
-    const int slot = t % P;
+    const int n_v = G * d_v;
+    const int nt = blockDim.x;
+    const long long page = r.page;
+    const int slot = r.t % P;
 #pragma unroll
     for (int u = 0; u < kAppendMaxPerThread; ++u) {
         const int i = u * nt + threadIdx.x;
         if (i < n_v) {
             const int g = i / d_v, d = i % d_v;
             const size_t dst = (((size_t)page * G + g) * P + slot) * d_v + d;
-            if constexpr (sizeof(CT) == 1) reinterpret_cast<uint8_t *>(v_pool)[dst] = float_to_e4m3_bits(x[u]);
-            else if constexpr (sizeof(CT) == 2) reinterpret_cast<uint16_t *>(v_pool)[dst] = float_to_bf16_bits(x[u]);
-            else reinterpret_cast<float *>(v_pool)[dst] = x[u];
+            if constexpr (sizeof(CT) == 1) reinterpret_cast<uint8_t *>(v_pool)[dst] = float_to_e4m3_bits(r.x[u]);
+            else if constexpr (sizeof(CT) == 2) reinterpret_cast<uint16_t *>(v_pool)[dst] = float_to_bf16_bits(r.x[u]);
+            else reinterpret_cast<float *>(v_pool)[dst] = r.x[u];
         }
     }
-    if (threadIdx.x < d_r / 2) {
-        const int i = threadIdx.x;
-        double y0, y1;
-        rope_pair((double)k0, (double)k1, t, rope.inv_freq[i], y0, y1);
+    const int i = (int)threadIdx.x - r.rope_tid0;
+    if (i >= 0 && i < d_r / 2) {
+        const double y0 = r.y0, y1 = r.y1;
         const size_t dst = ((size_t)page * P + slot) * d_r + 2 * i;
         if constexpr (sizeof(CT) == 1) {
             reinterpret_cast<uint8_t *>(kr_pool)[dst] = double_to_e4m3_bits(y0);
@@ -378,6 +415,16 @@ __device__ __forceinline__ void append_row(CT *__restrict__ v_pool, CT *__restri
             reinterpret_cast<float *>(kr_pool)[dst + 1] = __double2float_rn(y1);
         }
     }
+}
+template <typename CT>
+__device__ __forceinline__ void append_row(CT *__restrict__ v_pool, CT *__restrict__ kr_pool,
+                                           const int32_t *__restrict__ block_table, const float *__restrict__ v_new,
+                                           const float *__restrict__ kr_new, int G, int d_v, int d_r, int P, int num_pages,
+                                           int max_pages, int32_t *dev_status, const RopeTable &rope, int row, int seq, int t) {
+    AppendRegs r = append_load(v_new, kr_new, G, d_v, d_r, row);
+    append_locate(r, block_table, P, max_pages, dev_status, seq, t);
+    append_rotate(r, d_r, rope);
+    append_store<CT>(r, v_pool, kr_pool, G, d_v, d_r, P, num_pages, dev_status, seq);
 }
 
 template <typename CT>
@@ -543,8 +590,8 @@ stage_ints_kernel(const int32_t *__restrict__ a_src, const int32_t *__restrict__
 }
 
 // ---- fused front of a decode step: absorb and append in one launch ------------------------------------
-// Blocks [0, n_absorb) run absorb_block (head = block % H, batch tile = block / H); blocks
-// [n_absorb, n_absorb + B) run append_block.  The two are independent of each other.  This kernel
+// Absorb items (head = item % H, batch tile = item / H) and one append per sequence, independent of each other; which
+// block runs what is described in the kernel.  This kernel
 // waits for everything earlier in the stream BEFORE it lets its dependent (the decode kernel) start, so
 // whatever the decode kernel does ahead of its own wait overlaps with this kernel only.
 struct StepFrontParams {
@@ -555,6 +602,8 @@ struct StepFrontParams {
     int32_t *dev_status;
     int B, H, G, d_v, d_c, d_r, P, num_pages, max_pages, n_absorb;
     int trace_call;      // number of the decode call this launch belongs to (timeline builds only)
+    int batch;           // sequences per absorb item: kAbsorbBatch or kAbsorbBatchMax
+    int fold;            // 1: the first B blocks append as well (grid = max(n_absorb, B)); 0: appends have blocks of their own
 };
 
 template <typename CT>
@@ -564,14 +613,35 @@ step_front_kernel(StepFrontParams a, RopeTable rope) {
     grid_dependency_wait();
     grid_dependency_launch();
     if (threadIdx.x == 0) trace(kTrFrontEnterMin, a.trace_call);
+    // Small batches: blocks [0, n_absorb) run one absorb item each, blocks [n_absorb, n_absorb + B) one append each.
+    // Batches whose grid would exceed one block per SM (fold): block x runs absorb item x (x < n_absorb) AND appends sequence
+    // x's new token (x < B), and the 64-wide shape takes 16 sequences per absorb item -- the blocks of this kernel share
+    // their SMs with the decode blocks that were started early, which leave room for one of them at a time, so every block
+    // beyond one per SM is another round.  A folded append requests its loads first, so that they share the absorb item's
+    // memory round trip; its dependent page lookup and its rotation run while the item's copies fly.
+    const int seq_app = a.fold ? (int)blockIdx.x : (int)blockIdx.x - a.n_absorb;
+    const bool appends = seq_app >= 0 && seq_app < a.B;
+    AppendRegs ar;
+    int t_app = 0;
+    if (appends) {     // (its positional pairs sit in the last warp: the first ones rotate the query's)
+        t_app = a.pos[seq_app];
+        ar = append_load(a.v_new, a.kr_new, a.G, a.d_v, a.d_r, seq_app, kAbsorbThreads - 32);
+    }
+    auto locate_and_rotate = [&]() {
+        if (appends) {
+            append_locate(ar, a.block_table, a.P, a.max_pages, a.dev_status, seq_app, t_app);
+            append_rotate(ar, a.d_r, rope);
+        }
+    };
     if ((int)blockIdx.x < a.n_absorb) {
         absorb_block(a.q_c, a.q_r, a.M, a.pos, a.q_abs, a.B, a.H, a.d_v, a.d_c, a.d_r, rope, blockIdx.x % a.H,
-                     (blockIdx.x / a.H) * kAbsorbBatch, smem_f);
+                     (blockIdx.x / a.H) * a.batch, smem_f, a.batch, locate_and_rotate);
     } else {
-        append_block<CT>(static_cast<CT *>(a.v_pool), static_cast<CT *>(a.kr_pool), a.block_table, a.v_new, a.kr_new,
-                         a.pos, a.G, a.d_v, a.d_r, a.P, a.num_pages, a.max_pages, a.dev_status, rope,
-                         blockIdx.x - a.n_absorb);
+        locate_and_rotate();
     }
+    if (appends)
+        append_store<CT>(ar, static_cast<CT *>(a.v_pool), static_cast<CT *>(a.kr_pool), a.G, a.d_v, a.d_r, a.P, a.num_pages,
+                         a.dev_status, seq_app);
     if (threadIdx.x == 0) trace(kTrFrontExitMax, a.trace_call);
 }
 
