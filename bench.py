@@ -35,8 +35,8 @@ UNIT = "GB/s"
 # DRAM traffic of one decode-kernel launch at full size, from ncu (dram__bytes_read.sum + dram__bytes_write.sum, mean of
 # two launches).  A profiler figure cannot be taken inside a timed run: the numbers are those of the named profile,
 # which was captured with the kernels as they are in this tree; the line says where they come from.
-NCU_TRAFFIC = {"cfg2": (0.5 * ((570_726_400 + 3_314_432) + (570_726_144 + 397_824)), "profiles/decode_mma_kernel_cfg2.md"),
-               "cfg2-fp8": (0.5 * ((285_778_688 + 3_652_864) + (285_774_592 + 776_192)), "profiles/decode_fp8_kernel_cfg2.md")}
+NCU_TRAFFIC = {"cfg2": (0.5 * ((570_726_400 + 3_362_560) + (570_728_192 + 1_059_328)), "profiles/decode_mma_kernel_cfg2.md"),
+               "cfg2-fp8": (0.5 * ((285_520_640 + 3_187_200) + (285_505_792 + 892_672)), "profiles/decode_fp8_kernel_cfg2.md")}
 NOMINAL_HBM_GBPS = 8000.0          # the ~8 TB/s the target quotes (context; the roofline denominator is the measured copy rate)
 MIN_TIMED_WALL_S = 0.5             # every timed loop runs at least this long ...
 MIN_REPEATS = 5                    # ... and at least this many repeats of exactly --steps calls each
