@@ -159,7 +159,10 @@ int gva_append_cache(gva_handle *h, const gva_cache *cache, const float *v_new, 
  *                                 per resident thread block (ranges may cross sequence boundaries);
  *                                 n >= 1: every sequence is cut into exactly n ranges.
  * Partial results are merged by log-sum-exp weights in a second kernel.  For fixed arguments the
- * result is bitwise reproducible from run to run.  Calls on one handle must be stream-ordered (see gva_create). */
+ * result is bitwise reproducible from run to run.  Calls on one handle must be stream-ordered (see gva_create).
+ * The call may be captured into a CUDA graph (after one call outside the capture, which sizes the handle's scheduling
+ * state) and replayed with different contents of its device buffers: every call leaves the scheduling words as it
+ * found them, and nothing on the device depends on the call's number changing between replays. */
 int gva_decode(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens,
                float *out, float *lse, void *workspace, size_t workspace_bytes, int B, int max_seq_len,
                int num_splits, int32_t *dev_status, void *stream);

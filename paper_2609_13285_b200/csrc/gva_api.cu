@@ -271,6 +271,14 @@ int launch_decode(gva_handle *h, DecodeParams p, void *workspace, size_t workspa
     p.sync = h->sync_base + h->sync_off;
     p.epoch = dry ? h->epoch : ++h->epoch;      // a dry run prepares, it does not consume an epoch
     p.hdr_stamp = (int)((((unsigned)h->serial & 2047u) << 20) | ((unsigned)p.epoch & 0xfffffu)) + 1;
+    {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) {
+            (void)cudaGetLastError();
+            cap = cudaStreamCaptureStatusActive;      // cannot tell: take the safe side
+        }
+        if (cap != cudaStreamCaptureStatusNone) p.hdr_stamp = 0;
+    }
     if (h->epoch >= (1 << 30)) h->epoch = 2 + (h->epoch & 1);      // wrap, keeping the parity sequence
     if (kernel == GVA_KERNEL_MMA) {
 #ifdef GVA_WITH_MMA

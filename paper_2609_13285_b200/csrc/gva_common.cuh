@@ -49,7 +49,9 @@ struct DecodeParams {
     int32_t *dev_status;         // nullable
     int32_t *sync;               // this handle's sync region (see kSync*)
     int epoch;                   // this call's number on its handle (>= 1)
-    int hdr_stamp;               // (handle serial % 2048) << 20 | call number % 2^20, + 1: see kHdrEpoch
+    int hdr_stamp;               // (handle serial % 2048) << 20 | call number % 2^20, + 1: see kHdrEpoch.  0 = none: a call that
+                                 // is captured into a CUDA graph is replayed with the same number every time, so a header
+                                 // left by the previous replay could not be told from this one's; nothing is fetched early then
     int n_rec;                   // records the workspace holds
     int B, H, G, P, num_pages, max_pages;
     int num_splits;              // 0 = balanced flat partition

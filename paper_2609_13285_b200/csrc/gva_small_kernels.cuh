@@ -686,7 +686,7 @@ combine_kernel(DecodeParams p, int wph, int hpb) {
     // streams looks for that stamp now and then (one thread, a few polls microseconds apart) and, once it is there,
     // fetches its entry ahead of time: the real pass then starts with the records, not with one more round trip.
     int2 seg_early = make_int2(0, -1);           // y < 0: not fetched
-    if (p.num_splits == 0) {
+    if (p.num_splits == 0 && p.hdr_stamp != 0) {      // (no stamp: the call is being captured into a graph, see DecodeParams)
         __shared__ int2 s_seg;
         if (threadIdx.x == 0) {
             int2 sg = make_int2(0, -1);
@@ -710,6 +710,9 @@ combine_kernel(DecodeParams p, int wph, int hpb) {
         int first = 0, n = 1;                    // dry: record 0 only (always inside the workspace)
         if (!dry) {
             grid_dependency_wait();
+            // the decode grid is complete: its tail tickets go back to zero for whoever uses these words next (a later call
+            // of the other parity clears them as well; a replay of this very call from a graph relies on this line)
+            if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.sync[kSyncTicket + (p.epoch & 1)] = 0;
             if (p.cu_q) {      // (an input of the call, but read like everything else only once the stream's earlier work is complete)
                 const int r_lo = p.cu_q[b];
                 active = h < min(max(p.cu_q[b + 1] - r_lo, 0), p.q_len) * h_real;

@@ -454,3 +454,42 @@ def test_two_handles_take_turns_on_one_workspace():
     finally:
         da.close()
         db.close()
+
+
+def test_one_captured_decode_call_replayed_with_changing_lengths():
+    # A single gva_decode call captured in a CUDA graph and replayed: every replay carries the same call number, so
+    # nothing in the device-side scheduling state (tail tickets, the workspace header's stamp) may depend on the number
+    # changing from call to call.  The lengths change between replays (in place, on the device), so that the runs of
+    # records per sequence differ from one replay to the next.
+    _mma_or_skip(gb.GVA_KERNEL_MMA)
+    # (long enough for the balanced partition to hand out tail units dynamically: at least eight tiles per thread block)
+    lens0 = np.array([32768, 30000, 31000, 29000, 32000, 28000, 32768, 30001], dtype=np.int32)
+    case = wl.make_case("graph", wl.SHAPE_A, lens0, page_size=64, cache_dtype="bf16", seed=251)
+    dc = harness.upload(case, kernel=gb.GVA_KERNEL_MMA)
+    try:
+        dc.absorb()
+        ws = dc.ensure_workspace(0)
+        L = int(lens0.max())
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):              # (the binding launches on torch's current stream)
+            dc.decode()                            # warm-up outside the capture: attributes, tensor maps, sync region
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            gb.gva_decode(dc.handle, dc.cache, dc.q_abs, dc.seq_lens, dc.out, dc.lse, ws, case.B, L, 0, dc.status)
+        torch.cuda.synchronize()
+        for lens in (lens0, lens0 - np.array([977, 0, 5000, 8999, 1, 699, 64, 12345], dtype=np.int32), lens0 - 7000, lens0):
+            dc.seq_lens.copy_(torch.from_numpy(lens.astype(np.int32)))
+            dc.out.fill_(float("nan"))
+            torch.cuda.synchronize()
+            g.replay()
+            g.replay()                              # twice back to back: the second finds what the first left behind
+            torch.cuda.synchronize()
+            assert int(dc.status.item()) == 0
+            ref, _ = U().oracle_for_gpu_q(case, dc.q_abs, seq_lens=lens.astype(np.int32))
+            o = dc.out.cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(o - ref)) <= U().TOL_TIGHT_MAXABS, lens
+    finally:
+        dc.close()
