@@ -79,6 +79,9 @@ def make_workload(name: str, rank: int):
     if name == "cfg2-fp8-ncu":   # profiler-sized: 143 MB of 8-bit cache (> L2)
         return wl.make_case("cfg2-fp8-ncu", wl.SHAPE_A, [32768] * 16, page_size=64, cache_dtype="fp8", paged=True,
                             seed=wl.MASTER_SEED + 2000 + shift)
+    if name in ("cfg2-t16k", "cfg2-t64k", "cfg2-t128k"):     # cfg2 at other context lengths: time against length (slope and fixed cost)
+        T = {"cfg2-t16k": 16384, "cfg2-t64k": 65536, "cfg2-t128k": 131072}[name]
+        return wl.config2(seed=wl.MASTER_SEED + 2000 + shift, B=32, T=T)
     if name == "cfg2-ncu":   # profiler-sized: 143 MB of cache (> L2), same shapes and paging as cfg2
         return wl.config2(seed=wl.MASTER_SEED + 2000 + shift, B=16, T=16384)
     raise SystemExit(f"unknown workload {name}")
