@@ -563,12 +563,15 @@ def load_tensor_peak():
     return 1590.0, "fallback (1.59 PFLOP/s, earlier measurement on this pool)"
 
 
-def measure_prefill(rank, local_rank, dist, args, torch, gb, harness, B=8, T=8192, wide=False):
+def measure_prefill(rank, local_rank, dist, args, torch, gb, harness, B=8, T=8192, wide=False, cache_dtype="bf16"):
     """Whole-prompt prefill on the headline head shape: gva_absorb_query + gva_append_chunk + gva_prefill, and the
     attention kernel alone against the tensor roofline (flops of the absorbed form under the causal mask)."""
     from paper_2609_13285_b200 import multirank, workloads as wl
     dev = torch.device("cuda", local_rank)
-    if wide:
+    if cache_dtype != "bf16":
+        pc = wl.make_prefill_case("prefill8", wl.SHAPE_B if wide else wl.SHAPE_A, [0] * B, [T] * B, page_size=64,
+                                  cache_dtype=cache_dtype, seed=wl.MASTER_SEED + 7100 + 7919 * rank)
+    elif wide:
         pc = wl.prefill_bench_case_b(seed=wl.MASTER_SEED + 7200 + 7919 * rank, B=B, T=T)
     else:
         pc = wl.prefill_bench_case(seed=wl.MASTER_SEED + 7100 + 7919 * rank, B=B, T=T)
@@ -609,14 +612,14 @@ def measure_prefill(rank, local_rank, dist, args, torch, gb, harness, B=8, T=819
     peak, src = load_tensor_peak()
     flops = pc.flops()
     tf = flops / (attn_ms * 1e-3) / 1e12
-    res = {"workload": f"whole-prompt prefill, H={sh.H} G={sh.G} d_v={sh.d_v} d_c={sh.d_c} d_r={sh.d_r}, B={B} prompts of T={T} tokens, bf16 cache in "
+    res = {"workload": f"whole-prompt prefill, H={sh.H} G={sh.G} d_v={sh.d_v} d_c={sh.d_c} d_r={sh.d_r}, B={B} prompts of T={T} tokens, {'e4m3' if cache_dtype == 'fp8' else cache_dtype} cache in "
                        "64-token pages (permuted block table), L2 flushed between timed calls",
            "prefill_tokens_per_s": B * T / (whole_ms * 1e-3), "ms_per_step": whole_ms,
            "gva_prefill_ms_per_call": attn_ms, "steps": steps, "device_status": status,
            "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
-                        "traffic": None, "peak_source": src, "kernel": f"prefill_kernel<{sh.d_v},{sh.d_r}> (tcgen05 score and value products)",
+                        "traffic": None, "peak_source": src, "kernel": f"prefill_kernel<{sh.d_v},{sh.d_r}{', 8-bit cache' if cache_dtype == 'fp8' else ''}> (tcgen05 score and value products)",
                         "algorithmic_flops_per_launch": flops, "avg_launch_ms": attn_ms,
-                        "note": "flops = 2 * causal pairs * H * (2 d_v + d_r); bf16 operands, f32 accumulate"}}
+                        "note": "flops = 2 * causal pairs * H * (2 d_v + d_r); " + ("e4m3 tiles widened to f16 in shared memory, f16 operands" if cache_dtype == "fp8" else "bf16 operands") + ", f32 accumulate"}}
     pd.close()
     del flush
     torch.cuda.empty_cache()
@@ -715,7 +718,7 @@ def main() -> None:
     kernel = {"auto": gb.GVA_KERNEL_AUTO, "fma": gb.GVA_KERNEL_FMA, "mma": gb.GVA_KERNEL_MMA}[args.kernel]
 
     name = args.workload
-    if name in ("prefill", "prefill-ncu", "prefill-wide", "layer", "multi", "multi-q1", "multi-q8", "multi-q32", "tokens-q2", "tokens-q4", "tokens-q6", "tokens-q8", "tokens-q2-fp8", "tokens-q4-fp8"):      # side workloads on their own (small runs for profiler captures)
+    if name in ("prefill", "prefill-ncu", "prefill-wide", "prefill-fp8", "layer", "multi", "multi-q1", "multi-q8", "multi-q32", "tokens-q2", "tokens-q4", "tokens-q6", "tokens-q8", "tokens-q2-fp8", "tokens-q4-fp8"):      # side workloads on their own (small runs for profiler captures)
         if rank == 0:
             if name == "layer":
                 res = measure_layer(rank, local_rank, None, args, kernel, torch, gb, harness)
@@ -728,7 +731,8 @@ def main() -> None:
             else:
                 res = measure_prefill(rank, local_rank, None, args, torch, gb, harness,
                                       **({"B": 4, "T": 4096} if name == "prefill-ncu" else
-                                         {"B": 4, "T": 8192, "wide": True} if name == "prefill-wide" else {}))
+                                         {"B": 4, "T": 8192, "wide": True} if name == "prefill-wide" else
+                                         {"cache_dtype": "fp8"} if name == "prefill-fp8" else {}))
             print(json.dumps({"workload": name, **res}))
         if dist is not None:
             dist.barrier()
@@ -781,6 +785,7 @@ def main() -> None:
                                                             on_decode_kernel=True, cache_dtype="fp8")
         others["prefill"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness)
         others["prefill_wide"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness, B=4, T=8192, wide=True)
+        others["prefill_fp8"] = measure_prefill(rank, local_rank, dist, short, torch, gb, harness, cache_dtype="fp8")
 
     if rank == 0:
         case = r["case"]
