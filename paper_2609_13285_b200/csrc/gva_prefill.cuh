@@ -65,7 +65,8 @@ struct PrefillTraits {
     static constexpr int QTOK = 32;                              // query tokens per block
     static constexpr int ROWS = QTOK * kHeadsPerGroup;           // 128 = MMA M
     static constexpr int TILE = 64;                              // cached tokens per tile = MMA N of the score product
-    static constexpr int NSTAGE = 4;
+    static constexpr int NSTAGE = C8 ? 5 : 4;                    // (8-bit cache: one more, so that the tile widened at the top of
+                                                                 //  iteration t was requested two iterations earlier)
     static constexpr int BOXES = DV / 64;                        // 64-dim (128-byte) boxes per value row
     static constexpr int QBOX_BYTES = ROWS * 128;
     static constexpr int QV_BYTES = BOXES * QBOX_BYTES;
@@ -387,7 +388,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
-            mbar_init(kv_full(s), 1);
+            mbar_init(kv_full(s), C8 ? T::ROWS : 1);      // (8-bit cache: one arrival per softmax thread that widened its share)
             mbar_init(kv_empty(s), 1);
         }
         mbar_init(s_full(0), 1);
@@ -483,11 +484,68 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         float m_run = -INFINITY, l_run = 0.f;          // softmax reference (log2 domain) and sum relative to it
         const uint32_t o_addr = lane_base + T::COL_O;
         bool ok = true;
+        // 8-bit cache: the 128 softmax threads widen a tile's e4m3 codes to f16 (exact) from the stage's raw region into its
+        // swizzled operand tiles, 16 codes in and two 16-byte pieces out per step, two or three steps per thread and tile; rows
+        // at or beyond the end of the cache become zeros.  Tile t + 2 is widened at the top of iteration t -- its score
+        // product cannot start before the value product of tile t has released the score buffer -- so the widening is
+        // never on the chain of dependent steps.  (Its stage was refilled only after the value product of tile t + 2 - NS.)
+        auto convert_tile = [&](int t) -> bool {
+            const int st = t % NS;
+            if (!__all_sync(0xffffffffu, mbar_wait_spin(raw_full(st), (t / NS) & 1, s_abort))) return false;
+            unsigned char *stage = smem + T::OFF_STAGE + st * T::STAGE_BYTES;
+            const unsigned char *raw = stage + T::OFF_RAW;
+            const long long tok0 = (long long)(t_lo + t) * T::TILE;
+            constexpr int NPV = T::TILE * (DV / 16) / T::ROWS;      // 16-byte pieces of the value tile per thread
+            uint4 xv[NPV], xk = make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int u = 0; u < NPV; ++u) {                         // all loads first: one shared-memory round trip
+                const int pc = tid + T::ROWS * u;
+                xv[u] = *reinterpret_cast<const uint4 *>(raw + (pc / (DV / 16)) * DV + (pc % (DV / 16)) * 16);
+            }
+            constexpr int NPK = T::TILE * (DR / 16);                // pieces of the positional tile (at most one per thread)
+            static_assert(NPK <= T::ROWS, "one positional piece per thread at most");
+            if (DR > 0 && tid < NPK) xk = *reinterpret_cast<const uint4 *>(raw + T::RAW_V_BYTES + tid * 16);
+#pragma unroll
+            for (int u = 0; u < NPV; ++u) {
+                const int pc = tid + T::ROWS * u;
+                const int r = pc / (DV / 16), c16 = pc % (DV / 16);
+                uint4 x = xv[u];
+                if (tok0 + r >= kv_total) x = make_uint4(0, 0, 0, 0);
+                uint4 lo4, hi4;
+                e4m3x4_to_f16x2(x.x, lo4.x, lo4.y);
+                e4m3x4_to_f16x2(x.y, lo4.z, lo4.w);
+                e4m3x4_to_f16x2(x.z, hi4.x, hi4.y);
+                e4m3x4_to_f16x2(x.w, hi4.z, hi4.w);
+                unsigned char *box = stage + (c16 / 4) * T::VBOX_BYTES;
+                const int c = (c16 % 4) * 2;
+                *reinterpret_cast<uint4 *>(box + swz128(r, c)) = lo4;
+                *reinterpret_cast<uint4 *>(box + swz128(r, c + 1)) = hi4;
+            }
+            if (DR > 0 && tid < NPK) {
+                const int r = tid / (DR > 0 ? DR / 16 : 1), c16 = tid % (DR > 0 ? DR / 16 : 1);
+                uint4 lo4, hi4;
+                e4m3x4_to_f16x2(xk.x, lo4.x, lo4.y);
+                e4m3x4_to_f16x2(xk.y, lo4.z, lo4.w);
+                e4m3x4_to_f16x2(xk.z, hi4.x, hi4.y);
+                e4m3x4_to_f16x2(xk.w, hi4.z, hi4.w);
+                *reinterpret_cast<uint4 *>(stage + T::V_BYTES + swz_kr<T::KR_ROW>(r, 2 * c16)) = lo4;
+                *reinterpret_cast<uint4 *>(stage + T::V_BYTES + swz_kr<T::KR_ROW>(r, 2 * c16 + 1)) = hi4;
+            }
+            fence_async_smem();      // generic-proxy writes before the tensor core's reads
+            mbar_arrive(kv_full(st));
+            return true;
+        };
+        if constexpr (C8) {
+            for (int t = 0; t < 2 && t < n_tiles && ok; ++t) ok = convert_tile(t);
+        }
         // A warp none of whose 8 query tokens is live (short chunks, multi-token decode) only keeps the barrier protocol
         // going: its rows of S, P and O are never used.  (S of tile j complete implies the P barrier of tile j-2 has
         // completed, so an arrival for tile j cannot fall into an earlier phase.)
         const bool warp_dead = warp * 8 >= nv;
-        for (int j = 0; j < n_tiles; ++j) {
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            if constexpr (C8) {
+                if (j + 2 < n_tiles && !convert_tile(j + 2)) { ok = false; break; }
+            }
             if (!__all_sync(0xffffffffu, mbar_wait_spin(s_full(j % NB), (j / NB) & 1, s_abort))) { ok = false; break; }   // warp-uniform
             // rows of the last tile at or beyond the end of the cache may hold anything (NaN): zero them, P = 0 there
             // (the score product of this tile has completed, the value product starts only after the arrivals below)
@@ -633,7 +691,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
         // ========== MMA issuers: warp 5 the score products, warp 4 the value products (and the TMA loads) ==========
         // One thread sustains about one tcgen05.mma per 110 cycles (measured), and a 128 x 64 x 16 MMA occupies the tensor
         // pipe for 32: two issuing threads per block (and two blocks per SM) are needed to keep the pipe fed.
-        if (lane == 0 && (!C8 || warp == 5)) {
+        if (lane == 0) {
             constexpr uint32_t idesc_s = umma_idesc(T::ROWS, T::TILE, false, C8);
             constexpr uint32_t idesc_o = umma_idesc(T::ROWS, DV, true, C8);
             constexpr uint64_t kr_swz = T::KR_ROW == 32 ? kSwz32 : kSwz64;
@@ -707,11 +765,17 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                         return false;
                     }
                     const uint32_t dst = s_base + T::OFF_STAGE + st * T::STAGE_BYTES;
-                    mbar_expect_tx(kv_full(st), T::V_BYTES + T::KR_BYTES);
                     const int row = (int)((page * p.G + g) * p.P + slot0);
+                    if constexpr (C8) {      // byte tiles into the stage's raw region; the softmax warps widen them
+                        mbar_expect_tx(raw_full(st), T::RAW_V_BYTES + T::RAW_K_BYTES);
+                        tma_load_2d(dst + T::OFF_RAW, &tm_v, 0, row, raw_full(st));
+                        if constexpr (DR > 0) tma_load_2d(dst + T::OFF_RAW + T::RAW_V_BYTES, &tm_k, 0, (int)(page * p.P + slot0), raw_full(st));
+                    } else {
+                        mbar_expect_tx(kv_full(st), T::V_BYTES + T::KR_BYTES);
 #pragma unroll
-                    for (int bx = 0; bx < T::BOXES; ++bx) tma_load_2d(dst + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, kv_full(st));
-                    if constexpr (DR > 0) tma_load_2d(dst + T::V_BYTES, &tm_k, 0, (int)(page * p.P + slot0), kv_full(st));   // (no positional tile in a value-only cache)
+                        for (int bx = 0; bx < T::BOXES; ++bx) tma_load_2d(dst + bx * T::VBOX_BYTES, &tm_v, bx * 64, row, kv_full(st));
+                        if constexpr (DR > 0) tma_load_2d(dst + T::V_BYTES, &tm_k, 0, (int)(page * p.P + slot0), kv_full(st));   // (no positional tile in a value-only cache)
+                    }
                     ++loaded;
                     return true;
                 };
@@ -735,7 +799,7 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                 if (ok) umma_commit(o_full);
                 if (*s_abort) {   // copies still in flight must land before the block's shared memory is released
                     for (int t = max(0, loaded - NS); t < loaded; ++t)
-                        for (int it = 0; it < kDrainPolls && !mbar_try_wait(kv_full(t % NS), (t / NS) & 1); ++it) {}
+                        for (int it = 0; it < kDrainPolls && !mbar_try_wait(C8 ? raw_full(t % NS) : kv_full(t % NS), (t / NS) & 1); ++it) {}
                 }
             }
             if (!ok && !*s_abort) {
@@ -749,134 +813,6 @@ prefill_kernel(PrefillParams p, const __grid_constant__ CUtensorMap tm_v, const 
                 for (int it = 0; it < kDrainPolls * 16 && !mbar_try_wait(dr, 0); ++it) {}
             }
             tc_fence_before();
-        }
-    }
-    if constexpr (C8) {
-        if (warp == 4) {
-            // ===== 8-bit cache: the whole warp widens the byte tiles; lane 0 also loads them and issues the value products =====
-            constexpr uint32_t idesc_o = umma_idesc(T::ROWS, DV, true, true);
-            constexpr uint32_t hi128 = (1024u >> 4) | (1u << 14) | ((uint32_t)kSwz128 << 29);
-            constexpr uint32_t lo_mn = ((uint32_t)T::VBOX_BYTES >> 4) << 16;
-            const uint32_t a_st = ((s_base + T::OFF_STAGE) & 0x3FFFFu) >> 4;
-            auto mk = [](uint32_t lo, uint32_t hi) { return (uint64_t)lo | ((uint64_t)hi << 32); };
-            constexpr int KS_O = T::TILE / 16;
-            const uint32_t tmem_c = *s_tmem;
-            bool ok = true;
-            int issued_mma = 0, loaded = 0;
-            auto load_tile = [&](int t) -> bool {        // lane 0
-                const int st = t % NS;
-                const int t0 = (t_lo + t) * T::TILE;
-                const int pj = t0 / p.P, slot0 = t0 % p.P;
-                const long long page = p.block_table ? (long long)p.block_table[(size_t)b * p.max_pages + pj]
-                                                     : (long long)b * p.max_pages + pj;
-                if (page < 0 || page >= p.num_pages) {
-                    report_error(p.dev_status, GVA_ERR_BAD_PAGE, b);
-                    *s_abort = 1;
-                    return false;
-                }
-                const uint32_t dst = s_base + T::OFF_STAGE + st * T::STAGE_BYTES + T::OFF_RAW;
-                mbar_expect_tx(raw_full(st), T::RAW_V_BYTES + T::RAW_K_BYTES);
-                tma_load_2d(dst, &tm_v, 0, (int)((page * p.G + g) * p.P + slot0), raw_full(st));
-                if constexpr (DR > 0) tma_load_2d(dst + T::RAW_V_BYTES, &tm_k, 0, (int)(page * p.P + slot0), raw_full(st));
-                ++loaded;
-                return true;
-            };
-            // Widens tile t (which must have been requested) into its stage's operand tiles: 16 codes per step and lane, two
-            // swizzled 16-byte pieces out.  Rows at or beyond the end of the cache become zeros (they may hold anything).
-            auto convert_tile = [&](int t) -> bool {     // whole warp
-                const int st = t % NS;
-                if (!__all_sync(0xffffffffu, mbar_wait_spin(raw_full(st), (t / NS) & 1, s_abort))) return false;
-                unsigned char *stage = smem + T::OFF_STAGE + st * T::STAGE_BYTES;
-                const unsigned char *raw = stage + T::OFF_RAW;
-                const long long tok0 = (long long)(t_lo + t) * T::TILE;
-                constexpr int NPV = T::TILE * (DV / 16) / 32;      // 16-byte pieces per lane
-                uint4 xv[NPV];
-#pragma unroll
-                for (int u = 0; u < NPV; ++u) {                    // all loads first: one shared-memory round trip
-                    const int pc = lane + 32 * u;
-                    xv[u] = *reinterpret_cast<const uint4 *>(raw + (pc / (DV / 16)) * DV + (pc % (DV / 16)) * 16);
-                }
-#pragma unroll
-                for (int u = 0; u < NPV; ++u) {
-                    const int pc = lane + 32 * u;
-                    const int r = pc / (DV / 16), c16 = pc % (DV / 16);
-                    uint4 x = xv[u];
-                    if (tok0 + r >= kv_total) x = make_uint4(0, 0, 0, 0);
-                    uint4 lo4, hi4;
-                    e4m3x4_to_f16x2(x.x, lo4.x, lo4.y);
-                    e4m3x4_to_f16x2(x.y, lo4.z, lo4.w);
-                    e4m3x4_to_f16x2(x.z, hi4.x, hi4.y);
-                    e4m3x4_to_f16x2(x.w, hi4.z, hi4.w);
-                    unsigned char *box = stage + (c16 / 4) * T::VBOX_BYTES;
-                    const int c = (c16 % 4) * 2;
-                    *reinterpret_cast<uint4 *>(box + swz128(r, c)) = lo4;
-                    *reinterpret_cast<uint4 *>(box + swz128(r, c + 1)) = hi4;
-                }
-                if constexpr (DR > 0) {
-                    const unsigned char *rawk = raw + T::RAW_V_BYTES;
-#pragma unroll
-                    for (int pc = lane; pc < T::TILE * (DR / 16); pc += 32) {
-                        const int r = pc / (DR / 16), c16 = pc % (DR / 16);
-                        const uint4 x = *reinterpret_cast<const uint4 *>(rawk + r * DR + c16 * 16);
-                        uint4 lo4, hi4;
-                        e4m3x4_to_f16x2(x.x, lo4.x, lo4.y);
-                        e4m3x4_to_f16x2(x.y, lo4.z, lo4.w);
-                        e4m3x4_to_f16x2(x.z, hi4.x, hi4.y);
-                        e4m3x4_to_f16x2(x.w, hi4.z, hi4.w);
-                        *reinterpret_cast<uint4 *>(stage + T::V_BYTES + swz_kr<T::KR_ROW>(r, 2 * c16)) = lo4;
-                        *reinterpret_cast<uint4 *>(stage + T::V_BYTES + swz_kr<T::KR_ROW>(r, 2 * c16 + 1)) = hi4;
-                    }
-                }
-                fence_async_smem();      // generic-proxy writes before the tensor core's reads
-                __syncwarp();
-                if (lane == 0) mbar_arrive(kv_full(st));
-                return true;
-            };
-            if (lane == 0)
-                for (int t = 0; t < NS && t < n_tiles && ok; ++t) ok = load_tile(t);
-            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-            for (int t = 0; t < NS && t < n_tiles && ok; ++t) ok = convert_tile(t);
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                if (lane == 0) {
-                    // every row has stored P of tile j and finished any rescaling of O
-                    if (!mbar_wait_spin(p_full(j), (j >> 1) & 1, s_abort)) ok = false;
-                    if (ok) {
-                        tc_fence_after();
-                        const uint32_t vb = a_st + (uint32_t)(j % NS) * (T::STAGE_BYTES >> 4);
-#pragma unroll
-                        for (int ks = 0; ks < KS_O; ++ks)
-                            umma_bf16_ts(tmem_c + T::COL_O, tmem_c + T::COL_S + (j % NB) * T::TILE + ks * 8,
-                                         mk((vb + ks * (16 * 128 >> 4)) | lo_mn, hi128), idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
-                        umma_commit(kv_empty(j % NS));
-                        ++issued_mma;
-                        if (j >= 1 && j - 1 + NS < n_tiles) {      // tile j-1 was consumed a tile ago: its stage takes tile j-1+NS
-                            if (!mbar_wait_spin(kv_empty((j - 1) % NS), ((j - 1) / NS) & 1, s_abort)) ok = false;
-                            else ok = load_tile(j - 1 + NS);
-                        }
-                    }
-                }
-                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                // the tile requested one iteration ago has had that iteration to arrive; it is needed two tiles from now
-                // (widening it ahead of the value product instead, while the softmax warps work, measured slower: 2.87 ms
-                // against 2.60 ms on the prefill benchmark's shape -- the value product is what the chain waits for)
-                if (ok && j >= 2 && j - 2 + NS < n_tiles) ok = convert_tile(j - 2 + NS);
-            }
-            if (lane == 0) {
-                if (ok) umma_commit(o_full);
-                if (*s_abort) {   // copies still in flight must land before the block's shared memory is released
-                    for (int t = max(0, loaded - NS); t < loaded; ++t)
-                        for (int it = 0; it < kDrainPolls && !mbar_try_wait(raw_full(t % NS), (t / NS) & 1); ++it) {}
-                }
-                if (!ok && !*s_abort) {
-                    report_error(p.dev_status, GVA_ERR_TIMEOUT, b);
-                    *s_abort = 1;
-                }
-                if (issued_mma > 0) {
-                    umma_commit(drain2);
-                    for (int it = 0; it < kDrainPolls * 16 && !mbar_try_wait(drain2, 0); ++it) {}
-                }
-                tc_fence_before();
-            }
         }
     }
     grid_dependency_launch();
