@@ -295,6 +295,27 @@ def test_fused_step_is_bitwise_the_three_calls(kernel, shape):
         a.close(); b.close()
 
 
+@pytest.mark.parametrize("shape,dtype", [(wl.SHAPE_A, "bf16"), (wl.SHAPE_B, "bf16"), (wl.SHAPE_C, "bf16"), (wl.SHAPE_A, "fp8")])
+def test_fused_step_of_a_large_batch_is_bitwise_the_three_calls(shape, dtype):
+    # Batches whose front grid would exceed one block per SM take the folded front kernel (appends inside the absorb
+    # blocks, 16 sequences per absorb item for the 64-wide shape): same bits as the three separate calls.
+    rng = np.random.default_rng(77)
+    lens = rng.integers(1, 400, size=300).astype(np.int32)
+    mk = lambda: wl.make_case("fstep-big", shape, lens, page_size=64, cache_dtype=dtype, seed=212,
+                              q_pos=lens - 1, append_pos=lens - 1)
+    a, b = harness.upload(mk()), harness.upload(mk())
+    try:
+        a.absorb(); a.append(); a.decode()
+        b.step()
+        torch.cuda.synchronize()
+        assert int(a.status.item()) == 0 and int(b.status.item()) == 0
+        assert torch.equal(a.q_abs, b.q_abs)
+        assert torch.equal(a.v_pool, b.v_pool) and torch.equal(a.kr_pool, b.kr_pool)
+        assert torch.equal(a.out, b.out) and torch.equal(a.lse, b.lse)
+    finally:
+        a.close(); b.close()
+
+
 @pytest.mark.parametrize("kernel", KERNELS_BF16)
 def test_fused_steps_back_to_back_generate_tokens(kernel):
     # 24 decode steps in a row with no host synchronisation in between: every step appends one token that the
