@@ -514,3 +514,33 @@ def test_one_captured_decode_call_replayed_with_changing_lengths():
             assert np.max(np.abs(o - ref)) <= U().TOL_TIGHT_MAXABS, lens
     finally:
         dc.close()
+
+
+def test_one_captured_fused_step_replayed():
+    # the same for gva_decode_step: a step is idempotent when it is replayed with the same inputs (the appended row is written
+    # again with the same values), so three replays must leave exactly what one direct call leaves
+    _mma_or_skip(gb.GVA_KERNEL_MMA)
+    lens = np.array([32768, 30000, 31000, 29000, 32000, 28000, 32768, 30001], dtype=np.int32)
+    mk = lambda: wl.make_case("graph-step", wl.SHAPE_A, lens, page_size=64, cache_dtype="bf16", seed=252,
+                              q_pos=lens - 1, append_pos=lens - 1)
+    a, b = harness.upload(mk(), kernel=gb.GVA_KERNEL_MMA), harness.upload(mk(), kernel=gb.GVA_KERNEL_MMA)
+    try:
+        a.step()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            b.step()                                # warm-up outside the capture
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            b.step()
+        b.out.fill_(float("nan"))
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        assert int(a.status.item()) == 0 and int(b.status.item()) == 0
+        assert torch.equal(a.out, b.out) and torch.equal(a.lse, b.lse)
+        assert torch.equal(a.v_pool, b.v_pool) and torch.equal(a.kr_pool, b.kr_pool)
+    finally:
+        a.close(); b.close()
