@@ -332,7 +332,7 @@ int gva_decode_multi(gva_handle *h, const gva_cache *cache, const float *q_abs, 
  * q_len 2 .. 4: bf16 cache with (d_v, d_r) = (64, 16), (64, 24) (pages of a multiple of 64 tokens), (64, 0), (128, 32) or
  * (128, 0), and the e4m3 cache with a positional slice; q_len 5 .. 8: bf16 cache with d_v = 64, d_r = 16, 24 or 0, G <= 4
  * and pages of a multiple of 64 tokens; tensor-core kernel only; otherwise GVA_ERR_UNSUPPORTED.  The queries enter the score product as two bf16 numbers each (hi + lo), the
- * softmax weights as one (the 8-bit cache: f16 queries and weights), accumulation is f32: |out - exact| <= 2e-2 whatever
+ * softmax weights as one (the 8-bit cache: f16 instead of bf16), accumulation is f32: |out - exact| <= 2e-2 whatever
  * the size of the scores. */
 size_t gva_decode_tokens_workspace_bytes(const gva_handle *h, int B, int q_len, int max_seq_len, int num_splits);
 int gva_decode_tokens(gva_handle *h, const gva_cache *cache, const float *q_abs, const int32_t *seq_lens, float *out,

@@ -390,8 +390,11 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
         }
         } else {
             // ================= multi-token decode: QL new tokens per sequence, columns = slot * 4 + head =================
-            uint32_t qf[T::KSTEPS][NBK][2];   // B fragments of Q^T (plain f16): column n = lane / 4 of N-block nb, dims in the
+            uint32_t qf[T::KSTEPS][NBK][2];   // B fragments of Q^T (f16): column n = lane / 4 of N-block nb, dims in the
                                               // order the converted A registers present them
+            uint32_t qlo[T::KSTEPS][NBK][2];  // ... and of q - f16(q): the score product is taken with both, so that a score of
+                                              // any size is as exact as the cache's codes allow (with the first half alone a
+                                              // score s is off by about |s| 2^-12, which breaks the contract on peaked rows)
             float oacc[T::MT][NBK][4];
             float m_run[NBK][2], l_run[NBK][2];   // per column of this lane: columns 2 jh, 2 jh + 1 of every N-block
             const float scale = p.scale_log2;
@@ -415,8 +418,12 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                         float4 v = *reinterpret_cast<const float4 *>(q + kk * 16 + 4 * jh);
                         if (!present) v = make_float4(0.f, 0.f, 0.f, 0.f);
                         const __half2 w0 = __floats2half2_rn(v.x, v.y), w1 = __floats2half2_rn(v.z, v.w);
+                        const float2 f0 = __half22float2(w0), f1 = __half22float2(w1);
+                        const __half2 l0 = __floats2half2_rn(v.x - f0.x, v.y - f0.y), l1 = __floats2half2_rn(v.z - f1.x, v.w - f1.y);
                         qf[kk][nb][0] = *reinterpret_cast<const uint32_t *>(&w0);
                         qf[kk][nb][1] = *reinterpret_cast<const uint32_t *>(&w1);
+                        qlo[kk][nb][0] = *reinterpret_cast<const uint32_t *>(&l0);
+                        qlo[kk][nb][1] = *reinterpret_cast<const uint32_t *>(&l1);
                     }
                 }
             };
@@ -496,7 +503,10 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                             e4m3x4_to_f16x2(r[2 * hx], a[0], a[2]);
                             e4m3x4_to_f16x2(r[2 * hx + 1], a[1], a[3]);
 #pragma unroll
-                            for (int nb = 0; nb < NBK; ++nb) mma_f16(sacc[c][nb], a, qf[2 * pr + hx][nb][0], qf[2 * pr + hx][nb][1]);
+                            for (int nb = 0; nb < NBK; ++nb) {
+                                mma_f16(sacc[c][nb], a, qlo[2 * pr + hx][nb][0], qlo[2 * pr + hx][nb][1]);
+                                mma_f16(sacc[c][nb], a, qf[2 * pr + hx][nb][0], qf[2 * pr + hx][nb][1]);
+                            }
                         }
                     }
                     if constexpr (DR == 16) {
@@ -506,7 +516,10 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                         e4m3x4_to_f16x2(r[0], a[0], a[2]);
                         e4m3x4_to_f16x2(r[1], a[1], a[3]);
 #pragma unroll
-                        for (int nb = 0; nb < NBK; ++nb) mma_f16(sacc[c][nb], a, qf[T::KSTEPS_V][nb][0], qf[T::KSTEPS_V][nb][1]);
+                        for (int nb = 0; nb < NBK; ++nb) {
+                            mma_f16(sacc[c][nb], a, qlo[T::KSTEPS_V][nb][0], qlo[T::KSTEPS_V][nb][1]);
+                            mma_f16(sacc[c][nb], a, qf[T::KSTEPS_V][nb][0], qf[T::KSTEPS_V][nb][1]);
+                        }
                     } else if constexpr (DR == 32) {
                         uint32_t r[4];
                         ldsm_x4(kr_u32 + c * 16 * T::KR_ROW + off_kr + ((((uint32_t)ch_ld) ^ swz_kr) << 4), r);
@@ -516,8 +529,10 @@ decode_fp8_kernel(DecodeParams p, const __grid_constant__ CUtensorMap tm_v, cons
                             e4m3x4_to_f16x2(r[2 * hx], a[0], a[2]);
                             e4m3x4_to_f16x2(r[2 * hx + 1], a[1], a[3]);
 #pragma unroll
-                            for (int nb = 0; nb < NBK; ++nb)
+                            for (int nb = 0; nb < NBK; ++nb) {
+                                mma_f16(sacc[c][nb], a, qlo[T::KSTEPS_V + hx][nb][0], qlo[T::KSTEPS_V + hx][nb][1]);
                                 mma_f16(sacc[c][nb], a, qf[T::KSTEPS_V + hx][nb][0], qf[T::KSTEPS_V + hx][nb][1]);
+                            }
                         }
                     }
                 }

@@ -357,6 +357,26 @@ def test_decode_tokens_matches_oracle(q_len, shape, num_splits):
         pd.close()
 
 
+def test_decode_tokens_sharply_peaked_scores():
+    # queries 30 times the unit scale: scaled scores reach +-100 and single rows dominate; the 8-bit multi-token kernel takes the
+    # queries as two f16 numbers each (hi + lo), so outputs and lse stay far inside the contract
+    for q_len in (2, 4):
+        pc = wl.make_prefill_case("tok8p", wl.SHAPE_A, [700, 63, 2047, 0], [q_len] * 4, page_size=64, cache_dtype="fp8", seed=870 + q_len,
+                                  poison_unused=True, q_gain=30.0)
+        ref_out, ref_lse = orc.prefill_case(pc)
+        pd = harness.upload_prefill(pc)
+        try:
+            pd.absorb()
+            out, lse = pd.decode_tokens(q_len)
+            torch.cuda.synchronize()
+            assert int(pd.status.item()) == 0
+            o = out[:pc.n_q].cpu().numpy().astype(np.float64); l = lse[:pc.n_q].cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(o - ref_out)) <= 5e-3, np.max(np.abs(o - ref_out))
+            assert np.max(np.abs(l - ref_lse)) <= 5e-3
+        finally:
+            pd.close()
+
+
 @pytest.mark.parametrize("case_no", range(4))
 def test_decode_tokens_with_a_count_per_sequence(case_no):
     # gva_decode_tokens_ragged over the 8-bit cache: every sequence its own number of new tokens (none .. four)
