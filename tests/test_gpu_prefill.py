@@ -462,6 +462,59 @@ def test_random_cases_through_every_multi_token_entry_point(it):
         pd.close()
 
 
+@pytest.mark.parametrize("block", range(6))
+def test_random_sweep_over_shapes_cache_types_and_score_scales(block):
+    # ten seeded random cases per block: the five head shapes, bf16 and 8-bit caches, queries at 1, 6 and 30 times the unit
+    # scale (scaled scores up to +-100, single rows dominating), through gva_prefill, gva_decode_multi, gva_decode_tokens
+    # and gva_decode_tokens_ragged; one contract for all: |out - oracle| <= 2e-2, |lse - oracle| <= 2e-2
+    rng = np.random.default_rng(4321 + block)
+    shapes = [wl.SHAPE_A, wl.SHAPE_B, wl.SHAPE_C, wl.SHAPE_A0, wl.SHAPE_B0]
+    for it in range(10):
+        shape = shapes[int(rng.integers(0, len(shapes)))]
+        dt = "fp8" if (rng.random() < 0.4 and shape.d_r != 24) else "bf16"
+        B = int(rng.integers(1, 9))
+        ctx = rng.integers(0, 2500, size=B)
+        mode = int(rng.integers(0, 5))
+        gain = float(rng.choice([1.0, 1.0, 6.0, 30.0]))
+        maxq = 8 if (dt == "bf16" and shape.d_v == 64) else 4
+        if dt == "fp8" and shape.d_r == 0 and mode >= 3:
+            mode = 1                                   # the 8-bit multi-token kernel needs a positional slice
+        if mode == 3:
+            q = np.full(B, int(rng.integers(2, maxq + 1)))
+        elif mode == 4:
+            q = rng.integers(0, maxq + 1, size=B)
+            q[int(rng.integers(0, B))] = maxq
+        else:
+            q = rng.integers(0, 260, size=B)
+            if q.sum() == 0:
+                q[0] = 5
+        pc = wl.make_prefill_case("sweep", shape, ctx, q, page_size=64 if rng.random() < 0.8 else 128, cache_dtype=dt,
+                                  seed=19000 + 100 * block + it, poison_unused=True, paged=bool(rng.integers(0, 2)), q_gain=gain)
+        ref, ref_l = orc.prefill_case(pc)
+        pd = harness.upload_prefill(pc)
+        try:
+            pd.absorb()
+            pd.out.fill_(float("nan"))
+            if mode == 0:
+                out, lse = pd.prefill()
+            elif mode == 1:
+                out, lse = pd.decode_multi(num_splits=int(rng.integers(0, 9)))
+            elif mode == 2:
+                out, lse = pd.decode_multi(num_splits=0)
+            elif mode == 3:
+                out, lse = pd.decode_tokens(int(q[0]), num_splits=int(rng.integers(0, 4)))
+            else:
+                out, lse = pd.decode_tokens_ragged(num_splits=int(rng.integers(0, 3)))
+            torch.cuda.synchronize()
+            what = (block, it, mode, shape, dt, gain, q.tolist())
+            assert int(pd.status.item()) == 0, what
+            o = out[:pc.n_q].cpu().numpy().astype(np.float64); l = lse[:pc.n_q].cpu().numpy().astype(np.float64)
+            assert np.isfinite(o).all() and np.isfinite(l).all(), what
+            assert np.max(np.abs(o - ref)) <= TOL_MAXABS and np.max(np.abs(l - ref_l)) <= TOL_LSE, what
+        finally:
+            pd.close()
+
+
 @pytest.mark.parametrize("q_len", [5, 6, 7, 8])
 @pytest.mark.parametrize("shape_name", ["A", "A0", "C"])
 def test_decode_tokens_five_to_eight_new_tokens(q_len, shape_name):
