@@ -18,6 +18,12 @@
  *   - All pointers are DEVICE pointers unless a parameter is marked [host].  The library allocates
  *     no device memory, keeps no caller pointer after a call returns, and never synchronises: every
  *     call enqueues work on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *   - Weights (the maps M, the packed projections W_in and W_o) are constants to the kernels: gva_absorb_query,
+ *     gva_decode_step and the projections request them while the work that precedes the call in the stream may still be
+ *     ending, when that work is a kernel that releases its dependents early (programmatic dependent launch: this
+ *     library's own kernels, which never write weights, or a caller's kernel that executes
+ *     griddepcontrol.launch_dependents).  Such a kernel of the caller's must not be what writes the weights; after
+ *     ordinary kernels and copies nothing is read before they have completed.
  *   - Return value: a gva_status detected on the host before/at launch.  Conditions only the device
  *     can see (a page id outside [0, num_pages), a sequence longer than its block table) are
  *     recorded once in *dev_status (caller-zeroed int32 on the device; may be NULL) as

@@ -160,6 +160,19 @@ project_kernel(ProjParams p, RopeTable rope) {
     const int rows = min(kProjRows, p.M - row0);
     const int mt = warp % MT, ng = warp / MT;
     const int m0 = mt * 16;
+    const uint32_t w_u32 = smem_u32(w_s), a_u32 = smem_u32(a_s);
+    auto request_w = [&](int kc, int kn) {                              // W chunk: kn rows of 8 x 16 bytes
+        const unsigned char *src = reinterpret_cast<const unsigned char *>(p.W);
+        for (int c = tid; c < kn * 8; c += 32 * kProjWarps) {
+            const int k = c >> 3, ch = c & 7;
+            const bool in = n0 + ch * 8 < p.N;                         // columns past N read as zero
+            cp_async16(w_u32 + k * kProjRowBytes + ch * 16,
+                       src + (in ? ((size_t)(k_begin + kc + k) * p.N + n0 + ch * 8) * 2 : 0), in ? 16 : 0);
+        }
+    };
+    // The weights do not come from the work that precedes this kernel in the stream: their first chunk is requested
+    // ahead of the wait for that work, so that its round trip overlaps with the end of the preceding kernel.
+    request_w(0, min(kProjChunk, k_len));
     grid_dependency_wait();
     if constexpr (MODE == 1) grid_dependency_launch();
     // the epilogue's position lookups travel with the first chunk
@@ -176,7 +189,6 @@ project_kernel(ProjParams p, RopeTable rope) {
     for (int t = 0; t < MT; ++t)
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[t][e] = 0.f;
-    const uint32_t w_u32 = smem_u32(w_s), a_u32 = smem_u32(a_s);
     // ldmatrix.x2.trans lane addressing: matrices (k0-7, n-tile) and (k8-15, n-tile); lanes 16-31 repeat 0-15
     const uint32_t b_base = w_u32 + (lane & 15) * kProjRowBytes + ng * MT * 16;
     const float *a_lo = a_s + (m0 + (lane >> 2)) * kProjALd + 2 * (lane & 3);
@@ -186,13 +198,7 @@ project_kernel(ProjParams p, RopeTable rope) {
         const int kn = min(kProjChunk, k_len - kc);
         if (kc > 0) __syncthreads();              // everyone is done with the previous chunk
         {
-            const unsigned char *src = reinterpret_cast<const unsigned char *>(p.W);
-            for (int c = tid; c < kn * 8; c += 32 * kProjWarps) {       // W chunk: kn rows of 8 x 16 bytes
-                const int k = c >> 3, ch = c & 7;
-                const bool in = n0 + ch * 8 < p.N;                     // columns past N read as zero
-                cp_async16(w_u32 + k * kProjRowBytes + ch * 16,
-                           src + (in ? ((size_t)(k_begin + kc + k) * p.N + n0 + ch * 8) * 2 : 0), in ? 16 : 0);
-            }
+            if (kc > 0) request_w(kc, kn);
             const int cpr = kn >> 2;                                    // 16-byte chunks per activation row
             for (int c = tid; c < 16 * MT * cpr; c += 32 * kProjWarps) {
                 const int r = c / cpr, ch = c % cpr;

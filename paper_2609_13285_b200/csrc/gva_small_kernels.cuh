@@ -63,12 +63,28 @@ __host__ __device__ __forceinline__ size_t absorb_smem_bytes(int d_v, int d_c) {
 struct NoOverlap {
     __device__ __forceinline__ void operator()() const {}
 };
+// Requests M_h into the block's shared memory ahead of absorb_block (which is then told that the map is in flight).
+// Returns false when the pointers do not allow 16-byte copies: absorb_block then loads the map itself.
+__device__ __forceinline__ bool absorb_prefetch_map(const float *__restrict__ q_c, const float *__restrict__ M, int d_v, int d_c,
+                                                    int h, float *smem_f) {
+    const bool vec = (d_c & 3) == 0 && (reinterpret_cast<uintptr_t>(q_c) & 15) == 0 && (reinterpret_cast<uintptr_t>(M) & 15) == 0;
+    if (!vec) return false;
+    const int ld = absorb_row_stride(d_c), cpr = d_c >> 2;
+    const float *Mh = M + (size_t)h * d_v * d_c;
+    const uint32_t sM_u32 = smem_u32(smem_f);
+    for (int c = threadIdx.x; c < d_v * cpr; c += kAbsorbThreads) {
+        const int row = c / cpr, col = c % cpr;
+        cp_async16(sM_u32 + (row * ld + col * 4) * 4, Mh + (size_t)row * d_c + col * 4, 16);
+    }
+    cp_async_commit();
+    return true;
+}
 template <typename Overlap = NoOverlap>
 __device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, const float *__restrict__ q_r,
                                              const float *__restrict__ M, const int32_t *__restrict__ q_pos,
                                              float *__restrict__ q_abs, int B, int H, int d_v, int d_c, int d_r,
                                              const RopeTable &rope, int h, int b0, float *smem_f, int batch = kAbsorbBatch,
-                                             Overlap overlap = Overlap()) {
+                                             Overlap overlap = Overlap(), bool map_in_flight = false) {
     const int ld = absorb_row_stride(d_c);
     float *sM = smem_f;                            // [d_v][ld]
     float *sq = smem_f + d_v * ld;                 // [batch][d_c]
@@ -81,9 +97,11 @@ __device__ __forceinline__ void absorb_block(const float *__restrict__ q_c, cons
     if (vec) {
         const int cpr = d_c >> 2;                  // 16-byte chunks per row
         const uint32_t sM_u32 = smem_u32(sM), sq_u32 = smem_u32(sq);
-        for (int c = tid; c < d_v * cpr; c += kAbsorbThreads) {
-            const int row = c / cpr, col = c % cpr;
-            cp_async16(sM_u32 + (row * ld + col * 4) * 4, Mh + (size_t)row * d_c + col * 4, 16);
+        if (!map_in_flight) {
+            for (int c = tid; c < d_v * cpr; c += kAbsorbThreads) {
+                const int row = c / cpr, col = c % cpr;
+                cp_async16(sM_u32 + (row * ld + col * 4) * 4, Mh + (size_t)row * d_c + col * 4, 16);
+            }
         }
         for (int c = tid; c < nb * cpr; c += kAbsorbThreads) {
             const int bb = c / cpr, col = c % cpr;
@@ -170,8 +188,10 @@ absorb_kernel(const float *__restrict__ q_c, const float *__restrict__ q_r, cons
               int d_r, RopeTable rope) {
     grid_dependency_launch();
     extern __shared__ float smem_f[];
+    const bool map_in_flight = absorb_prefetch_map(q_c, M, d_v, d_c, blockIdx.x, smem_f);      // (a weight: see step_front_kernel)
     grid_dependency_wait();
-    absorb_block(q_c, q_r, M, q_pos, q_abs, B, H, d_v, d_c, d_r, rope, blockIdx.x, blockIdx.y * kAbsorbBatch, smem_f);
+    absorb_block(q_c, q_r, M, q_pos, q_abs, B, H, d_v, d_c, d_r, rope, blockIdx.x, blockIdx.y * kAbsorbBatch, smem_f, kAbsorbBatch,
+                 NoOverlap(), map_in_flight);
 }
 
 // ---- absorb for many rows on the tensor cores --------------------------------------------------------
@@ -610,6 +630,10 @@ template <typename CT>
 __global__ void __launch_bounds__(kAbsorbThreads)
 step_front_kernel(StepFrontParams a, RopeTable rope) {
     extern __shared__ float smem_f[];
+    // The map M_h is a weight: it is requested before the wait for the preceding work in the stream (in a decode loop the
+    // merge kernel of the previous step), so that its round trip is over when the step's own inputs may be read.
+    bool map_in_flight = false;
+    if ((int)blockIdx.x < a.n_absorb) map_in_flight = absorb_prefetch_map(a.q_c, a.M, a.d_v, a.d_c, blockIdx.x % a.H, smem_f);
     grid_dependency_wait();
     grid_dependency_launch();
     if (threadIdx.x == 0) trace(kTrFrontEnterMin, a.trace_call);
@@ -635,7 +659,7 @@ step_front_kernel(StepFrontParams a, RopeTable rope) {
     };
     if ((int)blockIdx.x < a.n_absorb) {
         absorb_block(a.q_c, a.q_r, a.M, a.pos, a.q_abs, a.B, a.H, a.d_v, a.d_c, a.d_r, rope, blockIdx.x % a.H,
-                     (blockIdx.x / a.H) * a.batch, smem_f, a.batch, locate_and_rotate);
+                     (blockIdx.x / a.H) * a.batch, smem_f, a.batch, locate_and_rotate, map_in_flight);
     } else {
         locate_and_rotate();
     }
