@@ -138,8 +138,8 @@ def test_project_out(B):
         dc.close()
 
 
-@pytest.mark.parametrize("shape,dtype", [(wl.SHAPE_A, "bf16"), (wl.SHAPE_B, "bf16"), (wl.SHAPE_A0, "bf16"), (wl.SHAPE_B0, "bf16"),
-                                         (wl.SHAPE_A, "fp8"), (wl.SHAPE_B, "fp8")])
+@pytest.mark.parametrize("shape,dtype", [(wl.SHAPE_A, "bf16"), (wl.SHAPE_B, "bf16"), (wl.SHAPE_C, "bf16"), (wl.SHAPE_A0, "bf16"),
+                                         (wl.SHAPE_B0, "bf16"), (wl.SHAPE_A, "fp8"), (wl.SHAPE_B, "fp8"), (wl.SHAPE_A, "f32")])
 def test_whole_layer_step_from_the_hidden_state(shape, dtype):
     lens = np.array([1, 64, 65, 700, 2049, 130], dtype=np.int32)
     d_model = 1024
