@@ -19,11 +19,10 @@
  *     no device memory, keeps no caller pointer after a call returns, and never synchronises: every
  *     call enqueues work on `stream` (a cudaStream_t passed as void*; NULL = default stream).
  *   - Weights (the maps M, the packed projections W_in and W_o) are constants to the kernels: gva_absorb_query,
- *     gva_decode_step and the projections request them while the work that precedes the call in the stream may still be
- *     ending, when that work is a kernel that releases its dependents early (programmatic dependent launch: this
- *     library's own kernels, which never write weights, or a caller's kernel that executes
- *     griddepcontrol.launch_dependents).  Such a kernel of the caller's must not be what writes the weights; after
- *     ordinary kernels and copies nothing is read before they have completed.
+ *     gva_decode_step and the projections are launched as programmatic dependents of the kernel that precedes them in
+ *     the stream and request their weights before they wait for that kernel's completion (all other inputs are read
+ *     after the wait).  The kernel enqueued immediately before such a call must therefore not be the one that writes
+ *     the weights it uses: write them by a copy, or by any earlier kernel.  (The library's own kernels never write weights.)
  *   - Return value: a gva_status detected on the host before/at launch.  Conditions only the device
  *     can see (a page id outside [0, num_pages), a sequence longer than its block table) are
  *     recorded once in *dev_status (caller-zeroed int32 on the device; may be NULL) as

@@ -156,7 +156,7 @@ __host__ __device__ __forceinline__ UnitPlan make_unit_plan(int total, int n_blo
 #ifndef GVA_TAIL_DEN
 #define GVA_TAIL_DEN 8      // build-time knobs: the first tail is 1/GVA_TAIL_DEN of a range, each next one half of that
                             // (measured on the long-context workload, gva_decode / step in us: 16 -> 91.2 / 93.5, 8 -> 90.85 / 92.9,
-                            //  6 -> 91.2 / 93.1, 4 -> 91.5 / 93.3; two tails instead of three: the same)
+                            //  6 -> 91.2 / 93.1, 4 -> 91.5 / 93.3; two tails instead of three: the same; a fourth, single-tile tail: +0.7 / +0.4)
 #define GVA_TAIL_UNITS 3
 #endif
     if (allow_dynamic && per_block >= 8) {
