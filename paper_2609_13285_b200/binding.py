@@ -282,6 +282,30 @@ def gva_decode_step_host(handle: int, cache: GvaCache, M, q_c_host, q_r_host, v_
     return rc
 
 
+def prepare_decode_step_host(handle: int, cache: GvaCache, M, q_c_host, q_r_host, v_new_host, kr_new_host, pos_host,
+                             seq_lens_host, out_host, scratch, B: int, max_seq_len: int, num_splits: int = 0,
+                             dev_status=None):
+    """gva_decode_step_host with its arguments marshalled once: returns a callable that enqueues one step on the stream
+    that was current here and returns the status.  For a serving loop that reuses its buffers: per call the interpreter
+    then makes one foreign call instead of a dozen pointer look-ups.  The tensors are kept alive by the callable."""
+    fn = load().gva_decode_step_host
+    keep = (cache, M, q_c_host, q_r_host, v_new_host, kr_new_host, pos_host, seq_lens_host, out_host, scratch, dev_status)
+    args = (ctypes.c_void_p(handle), ctypes.byref(cache), ctypes.c_void_p(_ptr(M)), ctypes.c_void_p(_ptr(q_c_host)),
+            ctypes.c_void_p(_ptr(q_r_host)), ctypes.c_void_p(_ptr(v_new_host)), ctypes.c_void_p(_ptr(kr_new_host)),
+            ctypes.c_void_p(_ptr(pos_host)), ctypes.c_void_p(_ptr(seq_lens_host)), ctypes.c_void_p(_ptr(out_host)),
+            ctypes.c_void_p(_ptr(scratch)), ctypes.c_size_t(scratch.numel() * scratch.element_size()), ctypes.c_int(int(B)),
+            ctypes.c_int(int(max_seq_len)), ctypes.c_int(int(num_splits)), ctypes.c_void_p(_ptr(dev_status)),
+            ctypes.c_void_p(_stream()))
+
+    def call(_keep=keep) -> int:
+        rc = fn(*args)
+        if rc != GVA_OK:
+            raise GvaError(rc, "gva_decode_step_host")
+        return rc
+
+    return call
+
+
 def gva_input_width(handle: int) -> int:
     return int(load().gva_input_width(handle))
 

@@ -382,6 +382,15 @@ def test_host_buffer_step_matches_device_step(pinned):
         assert int(b.status.item()) == 0
         assert torch.equal(out_h, a.out.cpu())
         assert torch.equal(a.v_pool, b.v_pool) and torch.equal(a.kr_pool, b.kr_pool)
+        # the same call with its arguments marshalled once
+        call = gb.prepare_decode_step_host(b.handle, b.cache, b.M, h[0], h[1], h[2], h[3], h[4], h[5], out_h, scratch, case.B,
+                                           int(lens.max()), 0, b.status)
+        out_h.fill_(float("nan"))
+        for _ in range(2):
+            assert call() == 0
+            torch.cuda.synchronize()
+        assert int(b.status.item()) == 0
+        assert torch.equal(out_h, a.out.cpu())
     finally:
         a.close(); b.close()
 
