@@ -374,20 +374,30 @@ def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with
     if n_layers > 1:
         warmup, steps = max(3, warmup // 5), max(3, steps // 10)
 
+    # The loops reuse their buffers, so every call's arguments are marshalled once (binding.prepare_call) and a step is one
+    # foreign call per kernel-launching entry point: on the two small workloads the interpreter otherwise sets the rate.
+    ws_bytes = ws.numel() * ws.element_size()
+    for lay in layers:
+        src = dc if n_layers == 1 else lay
+        lay.step_calls = [gb.prepare_call("gva_decode_step", dc.handle, c, src.M, src.q_c, src.q_r, src.v_new, src.kr_new,
+                                          dc.append_pos, dc.seq_lens, dc.q_abs, dc.out, dc.lse, ws, ws_bytes, B, max_len, ns,
+                                          dc.status) for c in lay.caches]
+        lay.decode_calls = [gb.prepare_call("gva_decode", dc.handle, c, dc.q_abs, dc.seq_lens, dc.out, dc.lse, ws, ws_bytes,
+                                            B, max_len, ns, dc.status) for c in lay.caches]
+
     def step(i: int):
         for lay in layers:
-            c = lay.caches[i % len(lay.caches)]
-            if n_layers == 1:
-                gb.gva_decode_step(dc.handle, c, dc.M, dc.q_c, dc.q_r, dc.v_new, dc.kr_new, dc.append_pos,
-                                   dc.seq_lens, dc.q_abs, dc.out, dc.lse, ws, B, max_len, ns, dc.status)
-            else:
-                gb.gva_decode_step(dc.handle, c, lay.M, lay.q_c, lay.q_r, lay.v_new, lay.kr_new, dc.append_pos,
-                                   dc.seq_lens, dc.q_abs, dc.out, dc.lse, ws, B, max_len, ns, dc.status)
+            lay.step_calls[i % len(lay.step_calls)]()
+
+    def step_on_current_stream(i: int):      # (a prepared call keeps the stream it was made on: a graph capture has its own)
+        for lay in layers:
+            src = dc if n_layers == 1 else lay
+            gb.gva_decode_step(dc.handle, lay.caches[i % len(lay.caches)], src.M, src.q_c, src.q_r, src.v_new, src.kr_new,
+                               dc.append_pos, dc.seq_lens, dc.q_abs, dc.out, dc.lse, ws, B, max_len, ns, dc.status)
 
     def decode_only(i: int):
         for lay in layers:
-            gb.gva_decode(dc.handle, lay.caches[i % len(lay.caches)], dc.q_abs, dc.seq_lens, dc.out, dc.lse, ws, B,
-                          max_len, ns, dc.status)
+            lay.decode_calls[i % len(lay.decode_calls)]()
 
     def sync_all():
         multirank.barrier(dist)
@@ -413,7 +423,7 @@ def measure(name, rank, local_rank, dist, args, kernel, torch, gb, harness, with
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             for i in range(n_rep):
-                step(i)
+                step_on_current_stream(i)
         g.replay()
         torch.cuda.synchronize()
         reps = max(3, steps // n_rep)

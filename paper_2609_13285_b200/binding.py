@@ -282,6 +282,37 @@ def gva_decode_step_host(handle: int, cache: GvaCache, M, q_c_host, q_r_host, v_
     return rc
 
 
+def prepare_call(name: str, *args):
+    """Any entry point with its arguments marshalled once: `args` as the C signature lists them after the handle's
+    position included (tensors, None, a GvaCache / GqaCache, integers), the trailing stream taken from torch's current
+    stream when left out.  Returns a callable that enqueues the call and returns its status (GvaError on a non-zero one).
+    The arguments are kept alive by the callable; it is for loops that reuse their buffers."""
+    fn = getattr(load(), name)
+    types = fn.argtypes
+    args = list(args)
+    if len(args) == len(types) - 1:
+        args.append(_stream())
+    if len(args) != len(types):
+        raise TypeError(f"{name} takes {len(types)} arguments, {len(args)} given")
+    conv = []
+    for a, t in zip(args, types):
+        if isinstance(a, ctypes.Structure):
+            conv.append(ctypes.byref(a))
+        elif t is ctypes.c_void_p:
+            conv.append(ctypes.c_void_p(a if isinstance(a, int) else _ptr(a)))
+        else:
+            conv.append(t(int(a)))
+    conv = tuple(conv)
+
+    def call(_keep=tuple(args)) -> int:
+        rc = fn(*conv)
+        if rc != GVA_OK:
+            raise GvaError(rc, name)
+        return rc
+
+    return call
+
+
 def prepare_decode_step_host(handle: int, cache: GvaCache, M, q_c_host, q_r_host, v_new_host, kr_new_host, pos_host,
                              seq_lens_host, out_host, scratch, B: int, max_seq_len: int, num_splits: int = 0,
                              dev_status=None):
