@@ -395,6 +395,33 @@ def test_host_buffer_step_matches_device_step(pinned):
         a.close(); b.close()
 
 
+def test_prepared_calls_equal_direct_calls():
+    # binding.prepare_call marshals the arguments once; the enqueued work is the same call
+    lens = np.array([700, 64, 1, 2049, 0], dtype=np.int32)
+    pos = np.maximum(lens - 1, 0)
+    mk = lambda: wl.make_case("prep", wl.SHAPE_A, lens, page_size=64, cache_dtype="bf16", seed=219, q_pos=pos, append_pos=pos)
+    a, b = harness.upload(mk()), harness.upload(mk())
+    try:
+        B, L = a.case.B, int(lens.max())
+        a.absorb(); a.decode()
+        ws = b.ensure_workspace(0)
+        nbytes = ws.numel() * ws.element_size()
+        absorb = gb.prepare_call("gva_absorb_query", b.handle, b.q_c, b.q_r, b.M, b.q_pos, b.q_abs, B)
+        decode = gb.prepare_call("gva_decode", b.handle, b.cache, b.q_abs, b.seq_lens, b.out, b.lse, ws, nbytes, B, L, 0, b.status)
+        for _ in range(2):
+            assert absorb() == 0 and decode() == 0
+        torch.cuda.synchronize()
+        assert int(b.status.item()) == 0
+        assert torch.equal(a.out, b.out) and torch.equal(a.lse, b.lse) and torch.equal(a.q_abs, b.q_abs)
+        with pytest.raises(TypeError):
+            gb.prepare_call("gva_decode", b.handle, b.cache)
+        bad = gb.prepare_call("gva_decode", b.handle, b.cache, b.q_abs, b.seq_lens, b.out, b.lse, ws, 16, B, L, 0, b.status)
+        with pytest.raises(gb.GvaError):
+            bad()                                  # a workspace of 16 bytes: the status comes back as it does from a direct call
+    finally:
+        a.close(); b.close()
+
+
 @pytest.mark.parametrize("kernel", KERNELS_BF16)
 def test_odd_page_size_many_short_sequences_and_one_long(kernel):
     _mma_or_skip(kernel)
