@@ -220,11 +220,12 @@ def run_reference(args) -> None:
     name = args.workload
     case = make_workload(name, 0)
     dt1, _, threads = oracle_sample(case, 1)
-    n = int(max(1, min(case.B, 8.0 / max(dt1, 1e-3))))      # each step: at most ~8 s of CPU work
-    warm = min(args.warmup, 1)
+    # exactly K timed steps after W untimed ones; each step is the oracle on the first n sequences of the workload, n sized so
+    # that the whole run stays near two minutes of CPU work
+    steps, warm = max(1, args.steps), max(0, args.warmup)
+    n = int(max(1, min(case.B, 120.0 / (steps + warm) / max(dt1, 1e-4))))
     for _ in range(warm):
         oracle_sample(case, n)
-    steps = max(1, min(args.steps, 5))
     times, nbytes = [], 0
     for _ in range(steps):
         dt, nbytes, threads = oracle_sample(case, n)
